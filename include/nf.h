@@ -1,0 +1,186 @@
+/*
+ * nf.h -- C ABI of the local-layer training step of adaptive local learning
+ * (NeuroFlux, arXiv 2402.14139) for NVIDIA B200 (sm_100a).
+ *
+ * The paper states the problem as: a CNN segmented into blocks by memory use, an
+ * auxiliary network per layer, block-specific batch sizes, and cached block outputs
+ * (Sections "Overview" and "Design").  The calls below are that statement:
+ * a layer with its auxiliary head (Eq. 1, Eq. 2), one pass of the inner body of
+ * Algorithm 2 over one batch (nf_layer_step), and the forward-only pass that fills
+ * the activation cache of a finished block (nf_block_cache) from which the next
+ * block draws batches of its own size (nf_cache_gather).
+ *
+ * Conventions
+ *  - Every pointer named "device" is a CUDA device pointer, 16-byte aligned; "host"
+ *    is ordinary host memory.  The library allocates no device memory: all state of
+ *    a layer lives in the workspace the caller binds (nf_layer_bind_workspace).
+ *  - Activations are channels-last: x[n][h][w][c], element type float (NF_F32) or
+ *    bfloat16 (NF_BF16).  Parameters cross the ABI as float in the paper's logical
+ *    order: W[Cout][Cin][3][3], Wa[F][Cout][3][3], Wf[classes][4F] where column
+ *    f*4 + u*2 + v of Wf multiplies pooled bin (u,v) of aux filter f.
+ *  - Calls enqueue work on the stream given to nf_set_stream (default stream 0) and
+ *    return without synchronising unless stated.  Buffers must stay valid until the
+ *    stream has passed the call.
+ *  - Return value: NF_OK (0) or a negative nf_status.  Nothing throws, aborts or
+ *    traps.  Conditions found on the device (bad label, non-finite loss, a bounded
+ *    wait that ran out) are OR-ed into a per-layer status word read by nf_layer_status.
+ */
+#ifndef NF_H_
+#define NF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct nf_layer nf_layer;
+typedef struct nf_block nf_block;
+
+enum nf_status {
+  NF_OK = 0,
+  NF_EINVAL = -1,       /* bad argument (NULL, non-positive size, unknown enum) */
+  NF_EALIGN = -2,       /* a device pointer is not 16-byte aligned */
+  NF_ENOWS = -3,        /* no workspace bound, or the bound one is too small */
+  NF_EUNSUPPORTED = -4, /* a shape this build has no kernel for */
+  NF_ECUDA = -5         /* a CUDA runtime call failed; see nf_last_cuda_error() */
+};
+
+/* bits of the device status word */
+enum nf_device_flag {
+  NF_ELABEL = 1,     /* a label was outside [0, classes); it was clamped */
+  NF_ENONFINITE = 2, /* the loss was NaN or infinite */
+  NF_ETIMEOUT = 4    /* a bounded wait inside a kernel ran out; results of that step are invalid */
+};
+
+enum nf_dtype { NF_F32 = 0, NF_BF16 = 1 };
+
+/* Which tensor nf_layer_set_param / nf_layer_get_param address: a parameter id ... */
+enum nf_param {
+  NF_P_W = 0,     /* theta_n: main conv weights  [Cout][Cin][3][3] */
+  NF_P_GAMMA = 1, /* BatchNorm scale             [Cout] */
+  NF_P_BETA = 2,  /* BatchNorm shift             [Cout] */
+  NF_P_WA = 3,    /* beta_n: aux conv weights    [F][Cout][3][3] */
+  NF_P_BA = 4,    /* aux conv bias               [F] */
+  NF_P_WF = 5,    /* gamma_n: linear weights     [classes][4F] */
+  NF_P_BF = 6,    /* linear bias                 [classes] */
+  NF_P_RMEAN = 7, /* running mean                [Cout]  (value only) */
+  NF_P_RVAR = 8   /* running variance            [Cout]  (value only) */
+};
+/* ... plus one of these kinds */
+enum nf_param_kind {
+  NF_K_VALUE = 0,
+  NF_K_MOMENTUM = 0x100, /* the momentum buffer v of the parameter */
+  NF_K_GRAD = 0x200      /* the gradient computed by the last nf_layer_step (get only) */
+};
+
+/* Options fixed before the workspace is sized.  Zero-initialise, then set fields. */
+typedef struct nf_layer_opts {
+  int N;             /* batch size the block trains with (block-specific, Section "Adaptive batching") */
+  int stride;        /* 1 or 2: stride of the main 3x3 convolution (the down-sampling P_n of ResNet shapes) */
+  int maxpool;       /* 1: a 2x2/2 max-pool follows the ReLU and belongs to this layer (P_n of VGG shapes) */
+  int dtype;         /* nf_dtype of x, act_out and of the stored activations */
+  float momentum;    /* SGD momentum; 0 gives the plain update of the paper's Appendix B */
+  float bn_eps;      /* BatchNorm epsilon */
+  float bn_momentum; /* running-statistics momentum */
+  int host_io;       /* 1: reserve staging so nf_layer_step_host can be used */
+} nf_layer_opts;
+
+/* Create the description of layer n with its auxiliary network A_n (Eq. 1, Eq. 2):
+ * conv3x3 Cin->Cout on an H x W input, BatchNorm, ReLU; aux conv3x3 Cout->F, ReLU,
+ * average pooling to 2x2, linear 4F->classes.  Host object only; no device work.
+ * Defaults: N=1, stride 1, no pool, NF_BF16, momentum 0.9, eps 1e-5, bn_momentum 0.1.
+ * Returns NULL if any size is < 1. */
+nf_layer* nf_layer_create(int Cin, int Cout, int H, int W, int F, int classes);
+void nf_layer_destroy(nf_layer* layer);
+
+/* Set the options; invalidates a bound workspace.  NF_EINVAL on bad values (N < 1, stride
+ * not 1 or 2, pool with odd output size, unknown dtype). */
+int nf_layer_configure(nf_layer* layer, const nf_layer_opts* opts);
+
+/* Bytes of device memory the layer needs for parameters, momentum, gradients, stored
+ * activations and reduction scratch at the configured options. */
+size_t nf_layer_workspace_bytes(const nf_layer* layer);
+
+/* Hand the layer its device memory (caller keeps ownership; must outlive the layer's use).
+ * Enqueues a clear of the state region and the default initialisation (gamma = 1, running
+ * variance = 1, everything else 0).  NF_EALIGN if dev is not 256-byte aligned, NF_ENOWS if
+ * bytes < nf_layer_workspace_bytes(). */
+int nf_layer_bind_workspace(nf_layer* layer, void* dev, size_t bytes);
+
+/* Copy a parameter tensor (or its momentum) from/to HOST float memory, n = element count of
+ * that tensor (NF_EINVAL if it differs).  Both synchronise the stream.  Setting a value also
+ * refreshes the reduced-precision copy the kernels read. */
+int nf_layer_set_param(nf_layer* layer, int which, const float* host, size_t n);
+int nf_layer_get_param(nf_layer* layer, int which, float* host, size_t n);
+
+/* One pass of the inner body of Algorithm 2 for this layer on one batch:
+ *   x_{n+1} = ReLU(pool(BN(theta_n * x_n)))            (Eq. 1)      -> act_out
+ *   z_{n+1} = gamma_n F_n beta_n x_{n+1}                (Eq. 2)
+ *   L = mean cross-entropy(z_{n+1}, labels)             (Eq. 3)      -> loss_out
+ *   gradients of (theta_n, beta_n, gamma_n) from L only, no gradient to x_n,
+ *   momentum-SGD update with learning rate lr.
+ * x:       device, [N][H][W][Cin] of the configured dtype; read only.
+ * labels:  device, int32[N], each in [0, classes) (else NF_ELABEL and clamped).
+ * loss_out: device, one float.
+ * act_out: device, [N][Ha][Wa][Cout] of the configured dtype, Ha = Ho/2 with pool else Ho;
+ *          computed with the weights as they were before this call's update; may be a
+ *          slice of a cache buffer.  Required (the aux network reads it).
+ * Asynchronous.  NF_ENOWS without workspace, NF_EINVAL on NULL, NF_EALIGN on alignment. */
+int nf_layer_step(nf_layer* layer, const void* x, const int32_t* labels, float lr, float* loss_out,
+                  void* act_out);
+
+/* Same step with HOST buffers (x, labels in; loss and, if non-NULL, act_out back):
+ * copies in, runs nf_layer_step, copies out, synchronises.  Needs opts.host_io = 1. */
+int nf_layer_step_host(nf_layer* layer, const void* x_host, const int32_t* labels_host, float lr,
+                       float* loss_host, void* act_out_host);
+
+/* OR of nf_device_flag bits raised since the last call; synchronises the stream and clears the word. */
+int nf_layer_status(nf_layer* layer);
+
+/* A block: consecutive layers trained together at one batch size (Algorithm 1's output).
+ * The layers must chain (Cout/Ha/Wa of one = Cin/H/W of the next), share dtype and have
+ * workspaces bound.  The block borrows the layers; destroy it before them. */
+nf_block* nf_block_create(nf_layer* const* layers, int n_layers);
+void nf_block_destroy(nf_block* block);
+
+/* Forward-only pass of a finished block over `count` samples, written to the activation
+ * cache (Section "Efficient forward propagation via prefetching and adaptive batching"):
+ * every layer runs conv, BatchNorm with its RUNNING statistics, ReLU and pool, so a sample's
+ * cached row does not depend on its batch-mates.  No parameter changes.
+ * x: device [count][H][W][Cin] of the first layer; out: device [count][Ha][Wa][Cout] of the
+ * last layer.  count must be in [1, N] of the block's layers (call repeatedly to cover a
+ * dataset); nf_block_cache uses count = N. */
+int nf_block_cache(nf_block* block, const void* x, void* out);
+int nf_block_cache_n(nf_block* block, const void* x, void* out, int count);
+
+/* Re-batching from the cache: out[i] = cache[idx[i]] for i < count, rows of row_bytes bytes
+ * (a multiple of 16); labels likewise if both label pointers are non-NULL.  All device pointers.
+ * Bit-exact copy. */
+int nf_cache_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count,
+                    size_t row_bytes, void* out, int32_t* out_labels);
+
+/* Algorithm 1 (host only, no device work): given each layer's largest feasible batch size,
+ * cap at B and group consecutive layers while |b[i+1]-b[i]| <= rho*b[i]; a block's batch size
+ * is the minimum over its members.  Writes up to n_layers entries of first layer index and
+ * batch size; returns the number of blocks, or NF_EINVAL. */
+int nf_partition(const int* max_batch, int n_layers, int B, double rho, int* block_first, int* block_batch);
+
+/* Stream for all later calls (a cudaStream_t); NULL selects the default stream. */
+int nf_set_stream(void* cuda_stream);
+
+/* Kernel launches enqueued by this library since the process started. */
+long long nf_launch_count(void);
+
+/* Name of the kernel family a configured layer uses for op 0 = main forward,
+ * 1 = main weight gradient, 2 = aux forward, 3 = aux backward: "tcgen05" or "cuda-core". */
+const char* nf_layer_kernel_family(const nf_layer* layer, int op);
+
+const char* nf_strerror(int status);
+const char* nf_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NF_H_ */
