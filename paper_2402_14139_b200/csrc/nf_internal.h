@@ -1,0 +1,111 @@
+// Internal definitions shared by the translation units of libnf (not part of the ABI).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/nf.h"
+
+typedef __nv_bfloat16 bf16;
+
+// Parameter arena: all trainable tensors of a layer, contiguous, in the layout the kernels read.
+//   W  : [tap = kh*3+kw][Cout][Cin]      gamma, beta : [Cout]
+//   Wa : [tap][F][Cout]                  ba : [F]
+//   Wf : [classes][4F]                   bf : [classes]
+// Every tensor starts at a multiple of 64 elements.  Four parallel arenas share the offsets:
+// fp32 value, fp32 momentum, fp32 gradient, bf16 copy of the value.
+enum { NF_NPARAM = 7 };
+
+struct nf_layer {
+  // description
+  int Cin, Cout, H, W, F, classes;
+  nf_layer_opts o;
+  int Ho, Wo, Ha, Wa;  // conv output size; size after the optional pool
+  // arena
+  size_t off[NF_NPARAM], cnt[NF_NPARAM], arena;  // element offsets / counts / total (padded)
+  // workspace
+  char* ws;
+  size_t ws_bytes;
+  int32_t* status;                     // device status word
+  float *val, *mom, *grad;             // arenas
+  bf16* shadow;                        // bf16 arena
+  float *rmean, *rvar;                 // [Cout]
+  float *scale, *shift, *mu, *invstd;  // [Cout] per-step BatchNorm coefficients
+  float *sdz, *sdzx;                   // [Cout] reduced sums for BatchNorm backward
+  void* y;                             // [N][Ho][Wo][Cout] conv output (dtype)
+  void* dy;                            // [N][Ho][Wo][Cout] gradient at conv output (dtype)
+  void* h;                             // [N][Ha][Wa][F] aux conv output after ReLU (dtype)
+  void* dh;                            // [N][Ha][Wa][F]
+  void* da;                            // [N][Ha][Wa][Cout]
+  float *p, *dp;                       // [N][4F]
+  float *logits, *dlogits;             // [N][classes]
+  float* lossn;                        // [N]
+  float* red;                          // reduction scratch (channel partials)
+  size_t red_floats;
+  float* wpart;                        // split-K partials of the weight gradients
+  size_t wpart_floats;
+  void* stage_x;                       // host_io staging
+  int32_t* stage_labels;
+  void* stage_act;
+  float* stage_loss;
+  // kernel families chosen at configure time: 0 = cuda-core, 1 = tcgen05
+  int fam[4];
+};
+
+struct nf_block {
+  int n;
+  nf_layer** layers;
+};
+
+// launch bookkeeping (nf_api.cu)
+extern cudaStream_t g_nf_stream;
+extern long long g_nf_launches;
+int nf_cuda_check(cudaError_t e, const char* what);
+#define NF_CUDA(x)                                        \
+  do {                                                    \
+    if (nf_cuda_check((x), #x) != NF_OK) return NF_ECUDA; \
+  } while (0)
+#define NF_LAUNCHED()                                                          \
+  do {                                                                         \
+    ++g_nf_launches;                                                           \
+    if (nf_cuda_check(cudaGetLastError(), "launch") != NF_OK) return NF_ECUDA; \
+  } while (0)
+
+static inline size_t nf_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline size_t nf_esize(int dtype) { return dtype == NF_F32 ? 4 : 2; }
+
+// ---- generic CUDA-core kernels (nf_ref_kernels.cu): any shape, fp32 or bf16 storage, fp32 accumulate
+int nf_ref_conv(int dtype, const void* x, int N, int H, int W, int Ci, const void* w, long ws_tap, long ws_co,
+                long ws_ci, int flip, const float* bias, int relu, int stride, int Co, void* y);
+int nf_ref_wgrad_splits(int N, int Ho, int Ci, int Co);
+int nf_ref_wgrad(int dtype, const void* x, int N, int H, int W, int Ci, const void* g, int Co, int stride,
+                 float* part, size_t part_floats, float* dw);
+int nf_ref_channel_blocks(size_t P, int C);
+int nf_ref_channel_sums(int dtype, const void* src, size_t P, int C, float* red, size_t red_floats, int* nblocks);
+int nf_ref_bn_finalize(const float* red, int nblocks, int C, double M, const float* gamma, const float* beta,
+                       float eps, float bn_momentum, float* scale, float* shift, float* mu, float* invstd,
+                       float* rmean, float* rvar);
+int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float eps, const float* rmean,
+                          const float* rvar, float* scale, float* shift);
+int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
+                    const float* shift, void* out);
+int nf_ref_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p);
+int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
+                 float* logits, float* dlogits, float* dp, float* lossn, int32_t* status);
+int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
+                    float* gbf, float* loss_out, int32_t* status);
+int nf_ref_dh(int dtype, const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh);
+int nf_ref_sum_partials(const float* red, int nblocks, int C, int which, float* out);
+int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
+                         const float* scale, const float* shift, const float* mu, const float* invstd, float* red,
+                         size_t red_floats, int* nblocks);
+int nf_ref_bn_bwd_finalize(const float* red, int nblocks, int C, float* sdz, float* sdzx, float* ggamma,
+                           float* gbeta);
+int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
+                        const float* scale, const float* shift, const float* mu, const float* invstd,
+                        const float* sdz, const float* sdzx, double M, void* dy);
+int nf_ref_sgd(float* val, float* mom, const float* grad, bf16* shadow, size_t n, float lr, float momentum);
+int nf_ref_shadow(const float* val, bf16* shadow, size_t n);
+int nf_ref_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count, size_t row_bytes,
+                  void* out, int32_t* out_labels);

@@ -1,0 +1,183 @@
+// Generic CUDA-core kernels of the local-layer step: any shape, fp32 or bf16 storage, fp32
+// accumulation, deterministic reductions (fixed-order partials, no floating-point atomics).
+// They carry the fp32 configuration and every shape the tensor-core kernels do not cover.
+#include "nf_internal.h"
+
+namespace {
+
+template <typename T> __device__ __forceinline__ float ldf(const T* p, size_t i);
+template <> __device__ __forceinline__ float ldf<float>(const float* p, size_t i) { return p[i]; }
+template <> __device__ __forceinline__ float ldf<bf16>(const bf16* p, size_t i) { return __bfloat162float(p[i]); }
+template <typename T> __device__ __forceinline__ void stf(T* p, size_t i, float v);
+template <> __device__ __forceinline__ void stf<float>(float* p, size_t i, float v) { p[i] = v; }
+template <> __device__ __forceinline__ void stf<bf16>(bf16* p, size_t i, float v) { p[i] = __float2bfloat16_rn(v); }
+// value as it will read back after being stored in T
+template <typename T> __device__ __forceinline__ float rnd(float v);
+template <> __device__ __forceinline__ float rnd<float>(float v) { return v; }
+template <> __device__ __forceinline__ float rnd<bf16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+
+// ------------------------------------------------------------------ direct 3x3 convolution, pad 1
+// y[n,i,j,co] = act(bias[co] + sum_{kh,kw,ci} w(tap,co,ci) * x[n, i*s+kh-1, j*s+kw-1, ci]).
+// Weight element (tap,co,ci) sits at w[t*ws_tap + co*ws_co + ci*ws_ci] with t = tap, or 8-tap when
+// flip is set (flip + swapped strides turn the same kernel into the input-gradient convolution).
+constexpr int CT_P = 16, CT_CO = 16, CT_CI = 32;
+
+template <typename T>
+__global__ void __launch_bounds__(256) conv_direct_kernel(const T* __restrict__ x, int N, int H, int W, int Ci,
+                                                          const T* __restrict__ w, long ws_tap, long ws_co,
+                                                          long ws_ci, int flip, const float* __restrict__ bias,
+                                                          int relu, int s, int Co, int Ho, int Wo, T* __restrict__ y) {
+  __shared__ float xs[3][CT_P * 2 + 2][CT_CI];
+  __shared__ float wsm[9][CT_CO][CT_CI + 1];
+  const int wt = (Wo + CT_P - 1) / CT_P, ct = (Co + CT_CO - 1) / CT_CO;
+  long b = blockIdx.x;
+  const int jt = b % wt; b /= wt;
+  const int cot = b % ct; b /= ct;
+  const int i = b % Ho;
+  const int n = b / Ho;
+  const int tid = threadIdx.x, co_l = tid % CT_CO, p_l = tid / CT_CO;
+  const int j0 = jt * CT_P, co0 = cot * CT_CO;
+  const int cols = (CT_P - 1) * s + 3;
+  float acc = 0.f;
+  for (int c0 = 0; c0 < Ci; c0 += CT_CI) {
+    const int cn = min(CT_CI, Ci - c0);
+    for (int e = tid; e < 3 * cols * CT_CI; e += 256) {
+      const int c = e % CT_CI, col = (e / CT_CI) % cols, r = e / (CT_CI * cols);
+      const int ii = i * s + r - 1, jj = j0 * s + col - 1;
+      float v = 0.f;
+      if (c < cn && ii >= 0 && ii < H && jj >= 0 && jj < W) v = ldf(x, (((size_t)n * H + ii) * W + jj) * Ci + c0 + c);
+      xs[r][col][c] = v;
+    }
+    for (int e = tid; e < 9 * CT_CO * CT_CI; e += 256) {
+      const int c = e % CT_CI, co = (e / CT_CI) % CT_CO, t = e / (CT_CI * CT_CO);
+      float v = 0.f;
+      if (c < cn && co0 + co < Co)
+        v = ldf(w, (size_t)((flip ? 8 - t : t) * ws_tap + (co0 + co) * ws_co + (c0 + c) * ws_ci));
+      wsm[t][co][c] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+      for (int kw = 0; kw < 3; ++kw) {
+        const float* xr = xs[kh][p_l * s + kw];
+        const float* wr = wsm[kh * 3 + kw][co_l];
+#pragma unroll 8
+        for (int c = 0; c < CT_CI; ++c) acc = fmaf(xr[c], wr[c], acc);
+      }
+    __syncthreads();
+  }
+  const int j = j0 + p_l, co = co0 + co_l;
+  if (j < Wo && co < Co) {
+    if (bias) acc += bias[co];
+    if (relu) acc = fmaxf(acc, 0.f);
+    stf(y, (((size_t)n * Ho + i) * Wo + j) * Co + co, acc);
+  }
+}
+
+// ------------------------------------------------------------------ direct weight gradient
+// part[split][tap][co][ci] = sum over the split's (n,i) rows and all j of g[n,i,j,co] * x[n,i*s+kh-1,j*s+kw-1,ci]
+constexpr int WG_J = 64;
+
+template <typename T>
+__global__ void __launch_bounds__(256) wgrad_direct_kernel(const T* __restrict__ x, int N, int H, int W, int Ci,
+                                                           const T* __restrict__ g, int Co, int s, int Ho, int Wo,
+                                                           int splits, float* __restrict__ part) {
+  __shared__ float gs[WG_J][16];
+  __shared__ float xs[3][WG_J * 2 + 2][16];
+  const int cit = (Ci + 15) / 16, cot = (Co + 15) / 16;
+  int b = blockIdx.x;
+  const int ti = b % cit; b /= cit;
+  const int to = b % cot; b /= cot;
+  const int sp = b;
+  const int tid = threadIdx.x, ci_l = tid % 16, co_l = tid / 16;
+  const int ci0 = ti * 16, co0 = to * 16;
+  const long rows = (long)N * Ho;
+  const long r0 = rows * sp / splits, r1 = rows * (sp + 1) / splits;
+  float acc[9];
+#pragma unroll
+  for (int t = 0; t < 9; ++t) acc[t] = 0.f;
+  for (long r = r0; r < r1; ++r) {
+    const int n = (int)(r / Ho), i = (int)(r % Ho);
+    for (int j0 = 0; j0 < Wo; j0 += WG_J) {
+      const int jn = min(WG_J, Wo - j0);
+      const int cols = (jn - 1) * s + 3;
+      for (int e = tid; e < jn * 16; e += 256) {
+        const int c = e % 16, j = e / 16;
+        gs[j][c] = (co0 + c < Co) ? ldf(g, (((size_t)n * Ho + i) * Wo + j0 + j) * Co + co0 + c) : 0.f;
+      }
+      for (int e = tid; e < 3 * cols * 16; e += 256) {
+        const int c = e % 16, col = (e / 16) % cols, rr = e / (16 * cols);
+        const int ii = i * s + rr - 1, jj = j0 * s + col - 1;
+        float v = 0.f;
+        if (ci0 + c < Ci && ii >= 0 && ii < H && jj >= 0 && jj < W)
+          v = ldf(x, (((size_t)n * H + ii) * W + jj) * Ci + ci0 + c);
+        xs[rr][col][c] = v;
+      }
+      __syncthreads();
+      for (int j = 0; j < jn; ++j) {
+        const float gv = gs[j][co_l];
+#pragma unroll
+        for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+          for (int kw = 0; kw < 3; ++kw) acc[kh * 3 + kw] = fmaf(gv, xs[kh][j * s + kw][ci_l], acc[kh * 3 + kw]);
+      }
+      __syncthreads();
+    }
+  }
+  if (co0 + co_l < Co && ci0 + ci_l < Ci)
+#pragma unroll
+    for (int t = 0; t < 9; ++t) part[(((size_t)sp * 9 + t) * Co + co0 + co_l) * Ci + ci0 + ci_l] = acc[t];
+}
+
+__global__ void sum_splits_kernel(const float* __restrict__ part, int splits, size_t n, float* __restrict__ out) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float s = 0.f;
+  for (int k = 0; k < splits; ++k) s += part[(size_t)k * n + i];
+  out[i] = s;
+}
+
+}  // namespace
+
+int nf_ref_conv(int dtype, const void* x, int N, int H, int W, int Ci, const void* w, long ws_tap, long ws_co,
+                long ws_ci, int flip, const float* bias, int relu, int stride, int Co, void* y) {
+  const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+  const long blocks = (long)N * Ho * ((Wo + CT_P - 1) / CT_P) * ((Co + CT_CO - 1) / CT_CO);
+  if (blocks <= 0 || blocks > 0x7fffffffL) return NF_EUNSUPPORTED;
+  if (dtype == NF_F32)
+    conv_direct_kernel<float><<<(unsigned)blocks, 256, 0, g_nf_stream>>>(
+        (const float*)x, N, H, W, Ci, (const float*)w, ws_tap, ws_co, ws_ci, flip, bias, relu, stride, Co, Ho, Wo, (float*)y);
+  else
+    conv_direct_kernel<bf16><<<(unsigned)blocks, 256, 0, g_nf_stream>>>(
+        (const bf16*)x, N, H, W, Ci, (const bf16*)w, ws_tap, ws_co, ws_ci, flip, bias, relu, stride, Co, Ho, Wo, (bf16*)y);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_wgrad_splits(int N, int Ho, int Ci, int Co) {
+  const long tiles = (long)((Ci + 15) / 16) * ((Co + 15) / 16);
+  long s = 2368 / tiles;
+  if (s < 1) s = 1;
+  if (s > (long)N * Ho) s = (long)N * Ho;
+  return (int)s;
+}
+
+int nf_ref_wgrad(int dtype, const void* x, int N, int H, int W, int Ci, const void* g, int Co, int stride,
+                 float* part, size_t part_floats, float* dw) {
+  const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+  const int splits = nf_ref_wgrad_splits(N, Ho, Ci, Co);
+  const size_t n = (size_t)9 * Co * Ci;
+  if ((size_t)splits * n > part_floats) return NF_ENOWS;
+  const unsigned blocks = (unsigned)(((Ci + 15) / 16) * ((Co + 15) / 16) * splits);
+  if (dtype == NF_F32)
+    wgrad_direct_kernel<float><<<blocks, 256, 0, g_nf_stream>>>((const float*)x, N, H, W, Ci, (const float*)g, Co,
+                                                                stride, Ho, Wo, splits, part);
+  else
+    wgrad_direct_kernel<bf16><<<blocks, 256, 0, g_nf_stream>>>((const bf16*)x, N, H, W, Ci, (const bf16*)g, Co,
+                                                               stride, Ho, Wo, splits, part);
+  NF_LAUNCHED();
+  sum_splits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, g_nf_stream>>>(part, splits, n, dw);
+  NF_LAUNCHED();
+  return NF_OK;
+}
