@@ -1,0 +1,511 @@
+// Memory-bound kernels of the local-layer step: BatchNorm statistics / apply / backward, pooling,
+// the linear + softmax cross-entropy head, momentum SGD and the cache gather.  Storage fp32 or
+// bf16, arithmetic fp32, cross-block sums finished in fp64 in a fixed order (deterministic).
+#include "nf_internal.h"
+#include "nf_ldst.cuh"
+
+namespace {
+
+__host__ __device__ inline int pow2ceil_cap256(int c) {
+  int l = 1;
+  while (l < c && l < 256) l <<= 1;
+  return l;
+}
+
+// dz at full-resolution pixel p = ((n*Ho)+i)*Wo+j, channel c: gradient that reaches the BatchNorm
+// output through ReLU and the optional 2x2 max-pool (first maximum in scan order wins).
+template <typename T>
+__device__ __forceinline__ float dz_at(const T* __restrict__ y, const T* __restrict__ da, size_t p, int c, int C,
+                                       int Ho, int Wo, int pool, float sc, float sh) {
+  const float z = fmaf(ldf(y, p * C + c), sc, sh);
+  if (!(z > 0.f)) return 0.f;
+  if (!pool) return ldf(da, p * C + c);
+  const int j = (int)(p % Wo), i = (int)((p / Wo) % Ho);
+  const size_t n = p / ((size_t)Wo * Ho);
+  const int i0 = i & ~1, j0 = j & ~1;
+  float best = -1.f;
+  int arg = 0;
+#pragma unroll
+  for (int d = 0; d < 4; ++d) {
+    const size_t q = ((n * Ho + i0 + (d >> 1)) * Wo + j0 + (d & 1)) * C + c;
+    const float r = rnd<T>(fmaxf(fmaf(ldf(y, q), sc, sh), 0.f));
+    if (r > best) { best = r; arg = d; }
+  }
+  if (arg != (i - i0) * 2 + (j - j0)) return 0.f;
+  return ldf(da, ((n * (Ho / 2) + i / 2) * (Wo / 2) + j / 2) * C + c);
+}
+
+struct StatsFn {  // (v, v^2) of a stored tensor
+  template <typename T>
+  __device__ __forceinline__ void operator()(const T* src, const T*, size_t p, int c, int C, float& a, float& b) const {
+    const float v = ldf(src, p * C + c);
+    a = v;
+    b = v * v;
+  }
+};
+
+struct BnBwdFn {  // (dz, dz*xhat)
+  int Ho, Wo, pool;
+  const float *scale, *shift, *mu, *invstd;
+  template <typename T>
+  __device__ __forceinline__ void operator()(const T* y, const T* da, size_t p, int c, int C, float& a, float& b) const {
+    const float dz = dz_at(y, da, p, c, C, Ho, Wo, pool, scale[c], shift[c]);
+    a = dz;
+    b = dz * (ldf(y, p * C + c) - mu[c]) * invstd[c];
+  }
+};
+
+// red[(block*2 + k)*C + c] = sum over the block's pixel range of value k at channel c
+template <typename T, typename Fn>
+__global__ void __launch_bounds__(256) channel_reduce_kernel(const T* __restrict__ s0, const T* __restrict__ s1, size_t P,
+                                                             int C, Fn fn, float* __restrict__ red) {
+  __shared__ float sm[2][256];
+  const int lanes = pow2ceil_cap256(C), planes = 256 / lanes;
+  const int lc = threadIdx.x % lanes, pl = threadIdx.x / lanes;
+  const size_t p0 = P * blockIdx.x / gridDim.x, p1 = P * (blockIdx.x + 1) / gridDim.x;
+  for (int c0 = 0; c0 < C; c0 += lanes) {
+    const int c = c0 + lc;
+    float a = 0.f, b = 0.f;
+    if (c < C)
+      for (size_t p = p0 + pl; p < p1; p += planes) {
+        float u, v;
+        fn(s0, s1, p, c, C, u, v);
+        a += u;
+        b += v;
+      }
+    sm[0][threadIdx.x] = a;
+    sm[1][threadIdx.x] = b;
+    __syncthreads();
+    if (pl == 0 && c < C) {
+      float ta = 0.f, tb = 0.f;
+      for (int q = 0; q < planes; ++q) {
+        ta += sm[0][q * lanes + lc];
+        tb += sm[1][q * lanes + lc];
+      }
+      red[((size_t)blockIdx.x * 2 + 0) * C + c] = ta;
+      red[((size_t)blockIdx.x * 2 + 1) * C + c] = tb;
+    }
+    __syncthreads();
+  }
+}
+
+__global__ void bn_finalize_kernel(const float* __restrict__ red, int nb, int C, double M, const float* __restrict__ gamma,
+                                   const float* __restrict__ beta, float eps, float bnm, float* scale, float* shift,
+                                   float* mu, float* invstd, float* rmean, float* rvar) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  double S = 0.0, Q = 0.0;
+  for (int b = 0; b < nb; ++b) {
+    S += (double)red[((size_t)b * 2 + 0) * C + c];
+    Q += (double)red[((size_t)b * 2 + 1) * C + c];
+  }
+  const double m = S / M;
+  double v = Q / M - m * m;
+  if (v < 0.0) v = 0.0;
+  const double is = 1.0 / sqrt(v + (double)eps);
+  const float sc = (float)((double)gamma[c] * is);
+  scale[c] = sc;
+  shift[c] = (float)((double)beta[c] - m * (double)gamma[c] * is);
+  mu[c] = (float)m;
+  invstd[c] = (float)is;
+  if (rmean) {
+    rmean[c] = (float)((1.0 - bnm) * (double)rmean[c] + (double)bnm * m);
+    const double unb = M > 1.0 ? v * M / (M - 1.0) : v;
+    rvar[c] = (float)((1.0 - bnm) * (double)rvar[c] + (double)bnm * unb);
+  }
+}
+
+__global__ void bn_eval_coeffs_kernel(int C, const float* gamma, const float* beta, float eps, const float* rmean,
+                                      const float* rvar, float* scale, float* shift) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  const double is = 1.0 / sqrt((double)rvar[c] + (double)eps);
+  scale[c] = (float)((double)gamma[c] * is);
+  shift[c] = (float)((double)beta[c] - (double)rmean[c] * (double)gamma[c] * is);
+}
+
+// out[n,ia,ja,c] = max over the pool window (or the single pixel) of ReLU(y*scale+shift)
+template <typename T>
+__global__ void bn_apply_kernel(const T* __restrict__ y, int Ho, int Wo, int C, int pool, const float* __restrict__ scale,
+                                const float* __restrict__ shift, size_t total, T* __restrict__ out) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const int c = (int)(e % C);
+  const size_t q = e / C;
+  const float sc = scale[c], sh = shift[c];
+  if (!pool) {
+    stf(out, e, fmaxf(fmaf(ldf(y, e), sc, sh), 0.f));
+    return;
+  }
+  const int Wa = Wo / 2, Ha = Ho / 2;
+  const int ja = (int)(q % Wa), ia = (int)((q / Wa) % Ha);
+  const size_t n = q / ((size_t)Wa * Ha);
+  float best = 0.f;
+#pragma unroll
+  for (int d = 0; d < 4; ++d) {
+    const size_t src = ((n * Ho + 2 * ia + (d >> 1)) * Wo + 2 * ja + (d & 1)) * C + c;
+    best = fmaxf(best, fmaf(ldf(y, src), sc, sh));
+  }
+  stf(out, e, best);
+}
+
+__device__ __forceinline__ void bin_range(int u, int H, int& lo, int& hi) {
+  lo = (u * H) / 2;
+  hi = ((u + 1) * H + 1) / 2;
+}
+
+// p[n][f*4 + u*2 + v] = mean of h over bin (u,v);  one block per (n, bin)
+template <typename T>
+__global__ void __launch_bounds__(256) avgpool_kernel(const T* __restrict__ h, int Ha, int Wa, int F, float* __restrict__ p) {
+  __shared__ float sm[256];
+  const int n = blockIdx.x / 4, bin = blockIdx.x % 4, u = bin / 2, v = bin % 2;
+  int i0, i1, j0, j1;
+  bin_range(u, Ha, i0, i1);
+  bin_range(v, Wa, j0, j1);
+  const int bw = j1 - j0, cnt = (i1 - i0) * bw;
+  const int lanes = pow2ceil_cap256(F), planes = 256 / lanes;
+  const int lf = threadIdx.x % lanes, pl = threadIdx.x / lanes;
+  for (int f0 = 0; f0 < F; f0 += lanes) {
+    const int f = f0 + lf;
+    float a = 0.f;
+    if (f < F)
+      for (int k = pl; k < cnt; k += planes) {
+        const int i = i0 + k / bw, j = j0 + k % bw;
+        a += ldf(h, (((size_t)n * Ha + i) * Wa + j) * F + f);
+      }
+    sm[threadIdx.x] = a;
+    __syncthreads();
+    if (pl == 0 && f < F) {
+      float t = 0.f;
+      for (int q = 0; q < planes; ++q) t += sm[q * lanes + lf];
+      p[(size_t)n * 4 * F + f * 4 + bin] = t / (float)cnt;
+    }
+    __syncthreads();
+  }
+}
+
+__device__ __forceinline__ float block_reduce(float v, float* sm, bool is_max) {
+  const int t = threadIdx.x;
+  sm[t] = v;
+  __syncthreads();
+  for (int s = blockDim.x / 2; s > 0; s >>= 1) {
+    if (t < s) sm[t] = is_max ? fmaxf(sm[t], sm[t + s]) : sm[t] + sm[t + s];
+    __syncthreads();
+  }
+  const float r = sm[0];
+  __syncthreads();
+  return r;
+}
+
+// one block per sample: logits, softmax cross-entropy, dlogits = (softmax-onehot)/N, dp = dlogits * Wf
+__global__ void __launch_bounds__(256) fc_ce_kernel(const float* __restrict__ p, const int32_t* __restrict__ labels, int N,
+                                                    int D, int K, const float* __restrict__ Wf, const float* __restrict__ bf,
+                                                    float* __restrict__ logits, float* __restrict__ dlogits,
+                                                    float* __restrict__ dp, float* __restrict__ lossn, int32_t* status) {
+  extern __shared__ float dyn[];
+  float* ps = dyn;          // [D]
+  float* ls = dyn + D;      // [K]
+  __shared__ float red[256];
+  const int n = blockIdx.x, t = threadIdx.x;
+  for (int d = t; d < D; d += 256) ps[d] = p[(size_t)n * D + d];
+  __syncthreads();
+  float mx = -INFINITY;
+  for (int k = t; k < K; k += 256) {
+    float s = bf[k];
+    const float* w = Wf + (size_t)k * D;
+    for (int d = 0; d < D; ++d) s = fmaf(w[d], ps[d], s);
+    ls[k] = s;
+    logits[(size_t)n * K + k] = s;
+    mx = fmaxf(mx, s);
+  }
+  mx = block_reduce(mx, red, true);
+  float se = 0.f;
+  for (int k = t; k < K; k += 256) se += __expf(ls[k] - mx);
+  se = block_reduce(se, red, false);
+  const float lse = mx + logf(se);
+  int lab = labels[n];
+  if (lab < 0 || lab >= K) {
+    if (t == 0) atomicOr(status, NF_ELABEL);
+    lab = lab < 0 ? 0 : K - 1;
+  }
+  if (t == 0) lossn[n] = lse - ls[lab];
+  const float invN = 1.f / (float)N;
+  for (int k = t; k < K; k += 256) {
+    const float g = (expf(ls[k] - lse) - (k == lab ? 1.f : 0.f)) * invN;
+    ls[k] = g;
+    dlogits[(size_t)n * K + k] = g;
+  }
+  __syncthreads();
+  for (int d = t; d < D; d += 256) {
+    float s = 0.f;
+    for (int k = 0; k < K; ++k) s = fmaf(ls[k], Wf[(size_t)k * D + d], s);
+    dp[(size_t)n * D + d] = s;
+  }
+}
+
+// one block per class k: gWf[k][:] = sum_n dlogits[n][k] p[n][:], gbf[k]; block 0 also reduces the loss
+__global__ void __launch_bounds__(256) fc_wgrad_kernel(const float* __restrict__ p, const float* __restrict__ dl,
+                                                       const float* __restrict__ lossn, int N, int D, int K,
+                                                       float* __restrict__ gWf, float* __restrict__ gbf,
+                                                       float* __restrict__ loss_out, int32_t* status) {
+  const int k = blockIdx.x, t = threadIdx.x;
+  for (int d = t; d < D; d += 256) {
+    float s = 0.f;
+    for (int n = 0; n < N; ++n) s = fmaf(dl[(size_t)n * K + k], p[(size_t)n * D + d], s);
+    gWf[(size_t)k * D + d] = s;
+  }
+  if (t == 0) {
+    float s = 0.f;
+    for (int n = 0; n < N; ++n) s += dl[(size_t)n * K + k];
+    gbf[k] = s;
+  }
+  if (k == 0 && t == 32) {
+    double s = 0.0;
+    for (int n = 0; n < N; ++n) s += (double)lossn[n];
+    const float L = (float)(s / (double)N);
+    *loss_out = L;
+    if (!isfinite(L)) atomicOr(status, NF_ENONFINITE);
+  }
+}
+
+// dh[n,i,j,f] = 1[h>0] * sum over bins containing (i,j) of dp[n][f*4+bin] / |bin|
+template <typename T>
+__global__ void dh_kernel(const T* __restrict__ h, const float* __restrict__ dp, int Ha, int Wa, int F, size_t total,
+                          T* __restrict__ dh) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const int f = (int)(e % F);
+  const size_t q = e / F;
+  const int j = (int)(q % Wa), i = (int)((q / Wa) % Ha);
+  const size_t n = q / ((size_t)Wa * Ha);
+  float g = 0.f;
+  if (ldf(h, e) > 0.f) {
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      int i0, i1;
+      bin_range(u, Ha, i0, i1);
+      if (i < i0 || i >= i1) continue;
+#pragma unroll
+      for (int v = 0; v < 2; ++v) {
+        int j0, j1;
+        bin_range(v, Wa, j0, j1);
+        if (j < j0 || j >= j1) continue;
+        g += dp[n * 4 * F + f * 4 + u * 2 + v] / (float)((i1 - i0) * (j1 - j0));
+      }
+    }
+  }
+  stf(dh, e, g);
+}
+
+__global__ void sum_partials_kernel(const float* __restrict__ red, int nb, int C, int which, float* __restrict__ out) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  double s = 0.0;
+  for (int b = 0; b < nb; ++b) s += (double)red[((size_t)b * 2 + which) * C + c];
+  out[c] = (float)s;
+}
+
+__global__ void bn_bwd_finalize_kernel(const float* __restrict__ red, int nb, int C, float* sdz, float* sdzx, float* gg,
+                                       float* gb) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  double a = 0.0, b = 0.0;
+  for (int k = 0; k < nb; ++k) {
+    a += (double)red[((size_t)k * 2 + 0) * C + c];
+    b += (double)red[((size_t)k * 2 + 1) * C + c];
+  }
+  sdz[c] = (float)a;
+  sdzx[c] = (float)b;
+  gb[c] = (float)a;
+  gg[c] = (float)b;
+}
+
+// dy = gamma*invstd * (dz - sum(dz)/M - xhat * sum(dz*xhat)/M)
+template <typename T>
+__global__ void bn_bwd_apply_kernel(const T* __restrict__ y, const T* __restrict__ da, int Ho, int Wo, int C, int pool,
+                                    const float* __restrict__ scale, const float* __restrict__ shift,
+                                    const float* __restrict__ mu, const float* __restrict__ invstd,
+                                    const float* __restrict__ sdz, const float* __restrict__ sdzx, float invM,
+                                    size_t total, T* __restrict__ dy) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const int c = (int)(e % C);
+  const size_t p = e / C;
+  const float dz = dz_at(y, da, p, c, C, Ho, Wo, pool, scale[c], shift[c]);
+  const float xh = (ldf(y, e) - mu[c]) * invstd[c];
+  stf(dy, e, scale[c] * (dz - sdz[c] * invM - xh * sdzx[c] * invM));
+}
+
+__global__ void sgd_kernel(float* __restrict__ val, float* __restrict__ mom, const float* __restrict__ grad,
+                           bf16* __restrict__ shadow, size_t n, float lr, float mu) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const float v = fmaf(mu, mom[i], grad[i]);
+  const float t = fmaf(-lr, v, val[i]);
+  mom[i] = v;
+  val[i] = t;
+  shadow[i] = __float2bfloat16_rn(t);
+}
+
+__global__ void shadow_kernel(const float* __restrict__ val, bf16* __restrict__ shadow, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) shadow[i] = __float2bfloat16_rn(val[i]);
+}
+
+// out row r = cache row idx[r], 16 bytes per thread
+__global__ void gather_kernel(const uint4* __restrict__ cache, const int32_t* __restrict__ cache_labels,
+                              const int32_t* __restrict__ idx, int count, size_t row16, uint4* __restrict__ out,
+                              int32_t* __restrict__ out_labels) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (size_t)count * row16) return;
+  const size_t r = e / row16, k = e % row16;
+  const size_t src = (size_t)idx[r];
+  out[e] = cache[src * row16 + k];
+  if (k == 0 && out_labels) out_labels[r] = cache_labels[src];
+}
+
+inline unsigned nblk(size_t n, int per) { return (unsigned)((n + per - 1) / per); }
+
+}  // namespace
+
+#define DISPATCH(dtype, CALL_F32, CALL_BF16) \
+  do {                                       \
+    if ((dtype) == NF_F32) { CALL_F32; } else { CALL_BF16; } \
+  } while (0)
+
+int nf_ref_channel_blocks(size_t P, int C) {
+  const int planes = 256 / pow2ceil_cap256(C);
+  size_t nb = (P + (size_t)planes * 16 - 1) / ((size_t)planes * 16);
+  if (nb < 1) nb = 1;
+  if (nb > 1184) nb = 1184;
+  return (int)nb;
+}
+
+int nf_ref_channel_sums(int dtype, const void* src, size_t P, int C, float* red, size_t red_floats, int* nblocks) {
+  const int nb = nf_ref_channel_blocks(P, C);
+  if ((size_t)nb * 2 * C > red_floats) return NF_ENOWS;
+  DISPATCH(dtype,
+           (channel_reduce_kernel<float, StatsFn><<<nb, 256, 0, g_nf_stream>>>((const float*)src, nullptr, P, C, StatsFn(), red)),
+           (channel_reduce_kernel<bf16, StatsFn><<<nb, 256, 0, g_nf_stream>>>((const bf16*)src, nullptr, P, C, StatsFn(), red)));
+  NF_LAUNCHED();
+  *nblocks = nb;
+  return NF_OK;
+}
+
+int nf_ref_bn_finalize(const float* red, int nblocks, int C, double M, const float* gamma, const float* beta,
+                       float eps, float bn_momentum, float* scale, float* shift, float* mu, float* invstd,
+                       float* rmean, float* rvar) {
+  bn_finalize_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(red, nblocks, C, M, gamma, beta, eps, bn_momentum, scale,
+                                                            shift, mu, invstd, rmean, rvar);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float eps, const float* rmean,
+                          const float* rvar, float* scale, float* shift) {
+  bn_eval_coeffs_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(C, gamma, beta, eps, rmean, rvar, scale, shift);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
+                    const float* shift, void* out) {
+  const size_t total = (size_t)N * (pool ? Ho / 2 : Ho) * (pool ? Wo / 2 : Wo) * C;
+  DISPATCH(dtype,
+           (bn_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, Ho, Wo, C, pool, scale, shift, total, (float*)out)),
+           (bn_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, Ho, Wo, C, pool, scale, shift, total, (bf16*)out)));
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p) {
+  DISPATCH(dtype, (avgpool_kernel<float><<<N * 4, 256, 0, g_nf_stream>>>((const float*)h, Ha, Wa, F, p)),
+           (avgpool_kernel<bf16><<<N * 4, 256, 0, g_nf_stream>>>((const bf16*)h, Ha, Wa, F, p)));
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
+                 float* logits, float* dlogits, float* dp, float* lossn, int32_t* status) {
+  const size_t smem = (size_t)(D + K) * sizeof(float);
+  if (smem > 40000) return NF_EUNSUPPORTED;
+  fc_ce_kernel<<<N, 256, smem, g_nf_stream>>>(p, labels, N, D, K, Wf, bf, logits, dlogits, dp, lossn, status);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
+                    float* gbf, float* loss_out, int32_t* status) {
+  fc_wgrad_kernel<<<K, 256, 0, g_nf_stream>>>(p, dlogits, lossn, N, D, K, gWf, gbf, loss_out, status);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_dh(int dtype, const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh) {
+  const size_t total = (size_t)N * Ha * Wa * F;
+  DISPATCH(dtype, (dh_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)h, dp, Ha, Wa, F, total, (float*)dh)),
+           (dh_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)h, dp, Ha, Wa, F, total, (bf16*)dh)));
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_sum_partials(const float* red, int nblocks, int C, int which, float* out) {
+  sum_partials_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(red, nblocks, C, which, out);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
+                         const float* scale, const float* shift, const float* mu, const float* invstd, float* red,
+                         size_t red_floats, int* nblocks) {
+  const size_t P = (size_t)N * Ho * Wo;
+  const int nb = nf_ref_channel_blocks(P, C);
+  if ((size_t)nb * 2 * C > red_floats) return NF_ENOWS;
+  BnBwdFn fn{Ho, Wo, pool, scale, shift, mu, invstd};
+  DISPATCH(dtype,
+           (channel_reduce_kernel<float, BnBwdFn><<<nb, 256, 0, g_nf_stream>>>((const float*)y, (const float*)da, P, C, fn, red)),
+           (channel_reduce_kernel<bf16, BnBwdFn><<<nb, 256, 0, g_nf_stream>>>((const bf16*)y, (const bf16*)da, P, C, fn, red)));
+  NF_LAUNCHED();
+  *nblocks = nb;
+  return NF_OK;
+}
+
+int nf_ref_bn_bwd_finalize(const float* red, int nblocks, int C, float* sdz, float* sdzx, float* ggamma,
+                           float* gbeta) {
+  bn_bwd_finalize_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(red, nblocks, C, sdz, sdzx, ggamma, gbeta);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
+                        const float* scale, const float* shift, const float* mu, const float* invstd,
+                        const float* sdz, const float* sdzx, double M, void* dy) {
+  const size_t total = (size_t)N * Ho * Wo * C;
+  const float invM = (float)(1.0 / M);
+  DISPATCH(dtype,
+           (bn_bwd_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, (const float*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (float*)dy)),
+           (bn_bwd_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, (const bf16*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (bf16*)dy)));
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_sgd(float* val, float* mom, const float* grad, bf16* shadow, size_t n, float lr, float momentum) {
+  sgd_kernel<<<nblk(n, 256), 256, 0, g_nf_stream>>>(val, mom, grad, shadow, n, lr, momentum);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_shadow(const float* val, bf16* shadow, size_t n) {
+  shadow_kernel<<<nblk(n, 256), 256, 0, g_nf_stream>>>(val, shadow, n);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count, size_t row_bytes,
+                  void* out, int32_t* out_labels) {
+  const size_t row16 = row_bytes / 16;
+  gather_kernel<<<nblk((size_t)count * row16, 256), 256, 0, g_nf_stream>>>((const uint4*)cache, cache_labels, idx, count,
+                                                                         row16, (uint4*)out, out_labels);
+  NF_LAUNCHED();
+  return NF_OK;
+}

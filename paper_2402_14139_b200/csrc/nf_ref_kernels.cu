@@ -2,19 +2,9 @@
 // accumulation, deterministic reductions (fixed-order partials, no floating-point atomics).
 // They carry the fp32 configuration and every shape the tensor-core kernels do not cover.
 #include "nf_internal.h"
+#include "nf_ldst.cuh"
 
 namespace {
-
-template <typename T> __device__ __forceinline__ float ldf(const T* p, size_t i);
-template <> __device__ __forceinline__ float ldf<float>(const float* p, size_t i) { return p[i]; }
-template <> __device__ __forceinline__ float ldf<bf16>(const bf16* p, size_t i) { return __bfloat162float(p[i]); }
-template <typename T> __device__ __forceinline__ void stf(T* p, size_t i, float v);
-template <> __device__ __forceinline__ void stf<float>(float* p, size_t i, float v) { p[i] = v; }
-template <> __device__ __forceinline__ void stf<bf16>(bf16* p, size_t i, float v) { p[i] = __float2bfloat16_rn(v); }
-// value as it will read back after being stored in T
-template <typename T> __device__ __forceinline__ float rnd(float v);
-template <> __device__ __forceinline__ float rnd<float>(float v) { return v; }
-template <> __device__ __forceinline__ float rnd<bf16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
 // ------------------------------------------------------------------ direct 3x3 convolution, pad 1
 // y[n,i,j,co] = act(bias[co] + sum_{kh,kw,ci} w(tap,co,ci) * x[n, i*s+kh-1, j*s+kw-1, ci]).
