@@ -1,0 +1,430 @@
+// C ABI of libnf: handles, workspace planning, parameter exchange and the launch sequence of
+// one local-layer step (Algorithm 2 body) and of the cache-filling forward pass.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <vector>
+
+#include "nf_internal.h"
+#include "nf_tc.h"
+
+cudaStream_t g_nf_stream = 0;
+long long g_nf_launches = 0;
+static char g_nf_err[256] = "";
+
+int nf_cuda_check(cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return NF_OK;
+  snprintf(g_nf_err, sizeof g_nf_err, "%s: %s", what, cudaGetErrorString(e));
+  return NF_ECUDA;
+}
+
+namespace {
+
+// Carves the workspace; with base == nullptr only sizes it.
+struct Carver {
+  char* base;
+  size_t off;
+  void* take(size_t bytes) {
+    off = nf_align_up(off, 256);
+    void* p = base ? base + off : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+size_t plan(nf_layer* L, char* base, bool assign) {
+  nf_layer tmp;
+  nf_layer* D = assign ? L : &tmp;
+  if (!assign) tmp = *L;
+  Carver c{base, 0};
+  const size_t es = nf_esize(L->o.dtype);
+  const size_t N = L->o.N, Co = L->Cout, F = L->F, K = L->classes;
+  const size_t ny = N * L->Ho * L->Wo * Co, na = N * L->Ha * L->Wa * Co, nh = N * L->Ha * L->Wa * F;
+  D->status = (int32_t*)c.take(256);
+  D->val = (float*)c.take(L->arena * 4);
+  D->mom = (float*)c.take(L->arena * 4);
+  D->grad = (float*)c.take(L->arena * 4);
+  D->shadow = (bf16*)c.take(L->arena * 2);
+  D->rmean = (float*)c.take(Co * 4);
+  D->rvar = (float*)c.take(Co * 4);
+  D->scale = (float*)c.take(Co * 4);
+  D->shift = (float*)c.take(Co * 4);
+  D->mu = (float*)c.take(Co * 4);
+  D->invstd = (float*)c.take(Co * 4);
+  D->sdz = (float*)c.take(Co * 4);
+  D->sdzx = (float*)c.take(Co * 4);
+  const size_t state_end = c.off;
+  D->y = c.take(ny * es);
+  D->dy = c.take(ny * es);
+  D->h = c.take(nh * es);
+  D->dh = c.take(nh * es);
+  D->da = c.take(na * es);
+  D->p = (float*)c.take(N * 4 * F * 4);
+  D->dp = (float*)c.take(N * 4 * F * 4);
+  D->logits = (float*)c.take(N * K * 4);
+  D->dlogits = (float*)c.take(N * K * 4);
+  D->lossn = (float*)c.take(N * 4);
+  size_t r1 = (size_t)nf_ref_channel_blocks(N * L->Ho * L->Wo, (int)Co) * 2 * Co;
+  size_t r2 = (size_t)nf_ref_channel_blocks(N * L->Ha * L->Wa, (int)F) * 2 * F;
+  D->red_floats = r1 > r2 ? r1 : r2;
+  D->red = (float*)c.take(D->red_floats * 4);
+  size_t w1 = (size_t)nf_ref_wgrad_splits((int)N, L->Ho, L->Cin, (int)Co) * 9 * Co * L->Cin;
+  size_t w2 = (size_t)nf_ref_wgrad_splits((int)N, L->Ha, (int)Co, (int)F) * 9 * F * Co;
+  D->wpart_floats = w1 > w2 ? w1 : w2;
+  const size_t tc = nf_tc_scratch_floats(L);
+  if (tc > D->wpart_floats) D->wpart_floats = tc;
+  D->wpart = (float*)c.take(D->wpart_floats * 4);
+  if (L->o.host_io) {
+    D->stage_x = c.take(N * L->H * L->W * L->Cin * es);
+    D->stage_labels = (int32_t*)c.take(N * 4);
+    D->stage_act = c.take(na * es);
+    D->stage_loss = (float*)c.take(256);
+  } else {
+    D->stage_x = D->stage_act = nullptr;
+    D->stage_labels = nullptr;
+    D->stage_loss = nullptr;
+  }
+  if (assign) L->ws_bytes = state_end;  // bytes cleared at bind time
+  return nf_align_up(c.off, 256);
+}
+
+void derive(nf_layer* L) {
+  const int s = L->o.stride;
+  L->Ho = (L->H - 1) / s + 1;
+  L->Wo = (L->W - 1) / s + 1;
+  L->Ha = L->o.maxpool ? L->Ho / 2 : L->Ho;
+  L->Wa = L->o.maxpool ? L->Wo / 2 : L->Wo;
+  const size_t cnt[NF_NPARAM] = {(size_t)9 * L->Cout * L->Cin, (size_t)L->Cout, (size_t)L->Cout,
+                                 (size_t)9 * L->F * L->Cout,   (size_t)L->F,    (size_t)L->classes * 4 * L->F,
+                                 (size_t)L->classes};
+  size_t o = 0;
+  for (int i = 0; i < NF_NPARAM; ++i) {
+    L->off[i] = o;
+    L->cnt[i] = cnt[i];
+    o = nf_align_up(o + cnt[i], 64);
+  }
+  L->arena = o;
+  nf_tc_select(L);
+}
+
+bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
+
+// logical [A][B][3][3]  <->  kernel [tap][A][B]
+void to_kernel_layout(const float* src, float* dst, size_t A, size_t B) {
+  for (size_t a = 0; a < A; ++a)
+    for (size_t b = 0; b < B; ++b)
+      for (int t = 0; t < 9; ++t) dst[(t * A + a) * B + b] = src[(a * B + b) * 9 + t];
+}
+void from_kernel_layout(const float* src, float* dst, size_t A, size_t B) {
+  for (size_t a = 0; a < A; ++a)
+    for (size_t b = 0; b < B; ++b)
+      for (int t = 0; t < 9; ++t) dst[(a * B + b) * 9 + t] = src[(t * A + a) * B + b];
+}
+
+}  // namespace
+
+extern "C" {
+
+nf_layer* nf_layer_create(int Cin, int Cout, int H, int W, int F, int classes) {
+  if (Cin < 1 || Cout < 1 || H < 1 || W < 1 || F < 1 || classes < 1) return nullptr;
+  nf_layer* L = (nf_layer*)calloc(1, sizeof(nf_layer));
+  if (!L) return nullptr;
+  L->Cin = Cin; L->Cout = Cout; L->H = H; L->W = W; L->F = F; L->classes = classes;
+  L->o.N = 1; L->o.stride = 1; L->o.maxpool = 0; L->o.dtype = NF_BF16;
+  L->o.momentum = 0.9f; L->o.bn_eps = 1e-5f; L->o.bn_momentum = 0.1f; L->o.host_io = 0;
+  derive(L);
+  return L;
+}
+
+void nf_layer_destroy(nf_layer* L) { free(L); }
+
+int nf_layer_configure(nf_layer* L, const nf_layer_opts* o) {
+  if (!L || !o) return NF_EINVAL;
+  if (o->N < 1 || (o->stride != 1 && o->stride != 2) || (o->dtype != NF_F32 && o->dtype != NF_BF16)) return NF_EINVAL;
+  if (!(o->momentum >= 0.f && o->momentum < 1.f) || !(o->bn_eps > 0.f) || !(o->bn_momentum >= 0.f && o->bn_momentum <= 1.f))
+    return NF_EINVAL;
+  const int Ho = (L->H - 1) / o->stride + 1, Wo = (L->W - 1) / o->stride + 1;
+  if (o->maxpool && ((Ho & 1) || (Wo & 1))) return NF_EINVAL;
+  L->o = *o;
+  L->o.maxpool = o->maxpool ? 1 : 0;
+  L->o.host_io = o->host_io ? 1 : 0;
+  L->ws = nullptr;
+  derive(L);
+  return NF_OK;
+}
+
+size_t nf_layer_workspace_bytes(const nf_layer* L) {
+  if (!L) return 0;
+  return plan(const_cast<nf_layer*>(L), nullptr, false);
+}
+
+int nf_layer_bind_workspace(nf_layer* L, void* dev, size_t bytes) {
+  if (!L || !dev) return NF_EINVAL;
+  if ((uintptr_t)dev & 255) return NF_EALIGN;
+  if (bytes < nf_layer_workspace_bytes(L)) return NF_ENOWS;
+  plan(L, (char*)dev, true);
+  L->ws = (char*)dev;
+  NF_CUDA(cudaMemsetAsync(dev, 0, L->ws_bytes, g_nf_stream));
+  std::vector<float> ones(L->Cout, 1.0f);
+  NF_CUDA(cudaMemcpyAsync(L->val + L->off[NF_P_GAMMA], ones.data(), L->Cout * 4, cudaMemcpyHostToDevice, g_nf_stream));
+  NF_CUDA(cudaMemcpyAsync(L->rvar, ones.data(), L->Cout * 4, cudaMemcpyHostToDevice, g_nf_stream));
+  NF_CUDA(cudaStreamSynchronize(g_nf_stream));
+  int rc = nf_ref_shadow(L->val, L->shadow, L->arena);
+  if (rc != NF_OK) return rc;
+  return nf_tc_prepare(L);
+}
+
+static int param_ptr(nf_layer* L, int which, float** dev, size_t* n, int* conv_a, int* conv_b) {
+  const int id = which & 0xff, kind = which & 0xf00;
+  *conv_a = *conv_b = 0;
+  if (id == NF_P_RMEAN || id == NF_P_RVAR) {
+    if (kind != NF_K_VALUE) return NF_EINVAL;
+    *dev = id == NF_P_RMEAN ? L->rmean : L->rvar;
+    *n = L->Cout;
+    return NF_OK;
+  }
+  if (id < 0 || id >= NF_NPARAM) return NF_EINVAL;
+  float* base = kind == NF_K_VALUE ? L->val : kind == NF_K_MOMENTUM ? L->mom : kind == NF_K_GRAD ? L->grad : nullptr;
+  if (!base) return NF_EINVAL;
+  *dev = base + L->off[id];
+  *n = L->cnt[id];
+  if (id == NF_P_W) { *conv_a = L->Cout; *conv_b = L->Cin; }
+  if (id == NF_P_WA) { *conv_a = L->F; *conv_b = L->Cout; }
+  return NF_OK;
+}
+
+int nf_layer_set_param(nf_layer* L, int which, const float* host, size_t n) {
+  if (!L || !host) return NF_EINVAL;
+  if (!L->ws) return NF_ENOWS;
+  if ((which & 0xf00) == NF_K_GRAD) return NF_EINVAL;
+  float* dev; size_t cnt; int A, B;
+  int rc = param_ptr(L, which, &dev, &cnt, &A, &B);
+  if (rc != NF_OK) return rc;
+  if (n != cnt) return NF_EINVAL;
+  std::vector<float> tmp;
+  const float* src = host;
+  if (A) {
+    tmp.resize(cnt);
+    to_kernel_layout(host, tmp.data(), A, B);
+    src = tmp.data();
+  }
+  NF_CUDA(cudaMemcpyAsync(dev, src, cnt * 4, cudaMemcpyHostToDevice, g_nf_stream));
+  NF_CUDA(cudaStreamSynchronize(g_nf_stream));
+  if ((which & 0xf00) == NF_K_VALUE && (which & 0xff) < NF_NPARAM) {
+    rc = nf_ref_shadow(L->val, L->shadow, L->arena);
+    if (rc != NF_OK) return rc;
+    NF_CUDA(cudaStreamSynchronize(g_nf_stream));
+  }
+  return NF_OK;
+}
+
+int nf_layer_get_param(nf_layer* L, int which, float* host, size_t n) {
+  if (!L || !host) return NF_EINVAL;
+  if (!L->ws) return NF_ENOWS;
+  float* dev; size_t cnt; int A, B;
+  int rc = param_ptr(L, which, &dev, &cnt, &A, &B);
+  if (rc != NF_OK) return rc;
+  if (n != cnt) return NF_EINVAL;
+  NF_CUDA(cudaStreamSynchronize(g_nf_stream));
+  if (A) {
+    std::vector<float> tmp(cnt);
+    NF_CUDA(cudaMemcpy(tmp.data(), dev, cnt * 4, cudaMemcpyDeviceToHost));
+    from_kernel_layout(tmp.data(), host, A, B);
+  } else {
+    NF_CUDA(cudaMemcpy(host, dev, cnt * 4, cudaMemcpyDeviceToHost));
+  }
+  return NF_OK;
+}
+
+#define NF_TRY(x)                 \
+  do {                            \
+    int rc_ = (x);                \
+    if (rc_ != NF_OK) return rc_; \
+  } while (0)
+
+int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, float* loss_out, void* act_out) {
+  if (!L || !x || !labels || !loss_out || !act_out) return NF_EINVAL;
+  if (!L->ws) return NF_ENOWS;
+  if (misaligned(x) || misaligned(act_out) || ((uintptr_t)labels & 3) || ((uintptr_t)loss_out & 3)) return NF_EALIGN;
+  const int dt = L->o.dtype, N = L->o.N, Ci = L->Cin, Co = L->Cout, F = L->F, K = L->classes, s = L->o.stride;
+  const int pool = L->o.maxpool, Ho = L->Ho, Wo = L->Wo, Ha = L->Ha, Wa = L->Wa, D = 4 * F;
+  const double M = (double)N * Ho * Wo;
+  const void* Wm = dt == NF_F32 ? (const void*)(L->val + L->off[NF_P_W]) : (const void*)(L->shadow + L->off[NF_P_W]);
+  const void* Wx = dt == NF_F32 ? (const void*)(L->val + L->off[NF_P_WA]) : (const void*)(L->shadow + L->off[NF_P_WA]);
+  float* g = L->grad;
+  int nb = 0;
+
+  // Eq. 1: conv, BatchNorm (batch statistics), ReLU, optional max-pool -> act_out
+  if (L->fam[0]) {
+    NF_TRY(nf_tc_conv_fwd(L, x, nb));
+  } else {
+    NF_TRY(nf_ref_conv(dt, x, N, L->H, L->W, Ci, Wm, (long)Co * Ci, Ci, 1, 0, nullptr, 0, s, Co, L->y));
+    NF_TRY(nf_ref_channel_sums(dt, L->y, (size_t)N * Ho * Wo, Co, L->red, L->red_floats, &nb));
+  }
+  NF_TRY(nf_ref_bn_finalize(L->red, nb, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
+                            L->o.bn_momentum, L->scale, L->shift, L->mu, L->invstd, L->rmean, L->rvar));
+  NF_TRY(nf_ref_bn_apply(dt, L->y, N, Ho, Wo, Co, pool, L->scale, L->shift, act_out));
+  // Eq. 2: aux conv + ReLU, average pool to 2x2, linear; Eq. 3: softmax cross-entropy
+  NF_TRY(nf_ref_conv(dt, act_out, N, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
+  NF_TRY(nf_ref_avgpool(dt, L->h, N, Ha, Wa, F, L->p));
+  NF_TRY(nf_ref_fc_ce(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits,
+                      L->dp, L->lossn, L->status));
+  // gradients of gamma_n, beta_n
+  NF_TRY(nf_ref_fc_wgrad(L->p, L->dlogits, L->lossn, N, D, K, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->status));
+  NF_TRY(nf_ref_dh(dt, L->h, L->dp, N, Ha, Wa, F, L->dh));
+  NF_TRY(nf_ref_wgrad(dt, act_out, N, Ha, Wa, Co, L->dh, F, 1, L->wpart, L->wpart_floats, g + L->off[NF_P_WA]));
+  NF_TRY(nf_ref_channel_sums(dt, L->dh, (size_t)N * Ha * Wa, F, L->red, L->red_floats, &nb));
+  NF_TRY(nf_ref_sum_partials(L->red, nb, F, 0, g + L->off[NF_P_BA]));
+  // gradient at the aux input, back through pool / ReLU / BatchNorm
+  NF_TRY(nf_ref_conv(dt, L->dh, N, Ha, Wa, F, Wx, (long)F * Co, 1, Co, 1, nullptr, 0, 1, Co, L->da));
+  NF_TRY(nf_ref_bn_bwd_reduce(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->red,
+                              L->red_floats, &nb));
+  NF_TRY(nf_ref_bn_bwd_finalize(L->red, nb, Co, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
+  NF_TRY(nf_ref_bn_bwd_apply(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->sdz, L->sdzx,
+                             M, L->dy));
+  // gradient of theta_n (the layer input receives none), then the update
+  if (L->fam[1]) {
+    NF_TRY(nf_tc_wgrad(L, x));
+  } else {
+    NF_TRY(nf_ref_wgrad(dt, x, N, L->H, L->W, Ci, L->dy, Co, s, L->wpart, L->wpart_floats, g + L->off[NF_P_W]));
+  }
+  NF_TRY(nf_ref_sgd(L->val, L->mom, L->grad, L->shadow, L->arena, lr, L->o.momentum));
+  return NF_OK;
+}
+
+int nf_layer_step_host(nf_layer* L, const void* xh, const int32_t* lh, float lr, float* loss_h, void* act_h) {
+  if (!L || !xh || !lh || !loss_h) return NF_EINVAL;
+  if (!L->ws) return NF_ENOWS;
+  if (!L->o.host_io) return NF_EINVAL;
+  const size_t es = nf_esize(L->o.dtype), N = L->o.N;
+  const size_t xb = N * L->H * L->W * L->Cin * es, ab = N * L->Ha * L->Wa * L->Cout * es;
+  NF_CUDA(cudaMemcpyAsync(L->stage_x, xh, xb, cudaMemcpyHostToDevice, g_nf_stream));
+  NF_CUDA(cudaMemcpyAsync(L->stage_labels, lh, N * 4, cudaMemcpyHostToDevice, g_nf_stream));
+  NF_TRY(nf_layer_step(L, L->stage_x, L->stage_labels, lr, L->stage_loss, L->stage_act));
+  NF_CUDA(cudaMemcpyAsync(loss_h, L->stage_loss, 4, cudaMemcpyDeviceToHost, g_nf_stream));
+  if (act_h) NF_CUDA(cudaMemcpyAsync(act_h, L->stage_act, ab, cudaMemcpyDeviceToHost, g_nf_stream));
+  NF_CUDA(cudaStreamSynchronize(g_nf_stream));
+  return NF_OK;
+}
+
+int nf_layer_status(nf_layer* L) {
+  if (!L) return NF_EINVAL;
+  if (!L->ws) return NF_ENOWS;
+  int32_t v = 0;
+  NF_CUDA(cudaStreamSynchronize(g_nf_stream));
+  NF_CUDA(cudaMemcpy(&v, L->status, 4, cudaMemcpyDeviceToHost));
+  NF_CUDA(cudaMemset(L->status, 0, 4));
+  return v;
+}
+
+nf_block* nf_block_create(nf_layer* const* layers, int n) {
+  if (!layers || n < 1) return nullptr;
+  for (int i = 0; i < n; ++i) {
+    if (!layers[i] || !layers[i]->ws) return nullptr;
+    if (i > 0) {
+      const nf_layer *a = layers[i - 1], *b = layers[i];
+      if (a->Cout != b->Cin || a->Ha != b->H || a->Wa != b->W || a->o.dtype != b->o.dtype || a->o.N != b->o.N) return nullptr;
+    }
+  }
+  nf_block* B = (nf_block*)calloc(1, sizeof(nf_block));
+  if (!B) return nullptr;
+  B->layers = (nf_layer**)calloc(n, sizeof(nf_layer*));
+  if (!B->layers) { free(B); return nullptr; }
+  B->n = n;
+  memcpy(B->layers, layers, n * sizeof(nf_layer*));
+  return B;
+}
+
+void nf_block_destroy(nf_block* B) {
+  if (!B) return;
+  free(B->layers);
+  free(B);
+}
+
+int nf_block_cache_n(nf_block* B, const void* x, void* out, int count) {
+  if (!B || !x || !out) return NF_EINVAL;
+  if (count < 1 || count > B->layers[0]->o.N) return NF_EINVAL;
+  if (misaligned(x) || misaligned(out)) return NF_EALIGN;
+  const void* in = x;
+  for (int l = 0; l < B->n; ++l) {
+    nf_layer* L = B->layers[l];
+    const int dt = L->o.dtype;
+    const void* Wm = dt == NF_F32 ? (const void*)(L->val + L->off[NF_P_W]) : (const void*)(L->shadow + L->off[NF_P_W]);
+    void* dst = l == B->n - 1 ? out : L->dy;
+    if (L->fam[0]) {
+      NF_TRY(nf_tc_conv_fwd_eval(L, in, count));
+    } else {
+      NF_TRY(nf_ref_conv(dt, in, count, L->H, L->W, L->Cin, Wm, (long)L->Cout * L->Cin, L->Cin, 1, 0, nullptr, 0,
+                         L->o.stride, L->Cout, L->y));
+    }
+    NF_TRY(nf_ref_bn_eval_coeffs(L->Cout, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps, L->rmean,
+                                 L->rvar, L->scale, L->shift));
+    NF_TRY(nf_ref_bn_apply(dt, L->y, count, L->Ho, L->Wo, L->Cout, L->o.maxpool, L->scale, L->shift, dst));
+    in = dst;
+  }
+  return NF_OK;
+}
+
+int nf_block_cache(nf_block* B, const void* x, void* out) {
+  if (!B) return NF_EINVAL;
+  return nf_block_cache_n(B, x, out, B->layers[0]->o.N);
+}
+
+int nf_cache_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count, size_t row_bytes,
+                    void* out, int32_t* out_labels) {
+  if (!cache || !idx || !out || count < 1 || row_bytes == 0 || (row_bytes & 15)) return NF_EINVAL;
+  if ((cache_labels == nullptr) != (out_labels == nullptr)) return NF_EINVAL;
+  if (misaligned(cache) || misaligned(out)) return NF_EALIGN;
+  return nf_ref_gather(cache, cache_labels, idx, count, row_bytes, out, out_labels);
+}
+
+int nf_partition(const int* max_batch, int n_layers, int Bcap, double rho, int* block_first, int* block_batch) {
+  if (!max_batch || !block_first || !block_batch || n_layers < 1 || Bcap < 1 || !(rho >= 0.0)) return NF_EINVAL;
+  std::vector<int> b(n_layers);
+  for (int i = 0; i < n_layers; ++i) {
+    if (max_batch[i] < 1) return NF_EINVAL;
+    b[i] = max_batch[i] < Bcap ? max_batch[i] : Bcap;
+  }
+  int nblocks = 0, i = 0;
+  while (i < n_layers) {
+    int bs = b[i];
+    block_first[nblocks] = i;
+    while (i + 1 < n_layers && fabs((double)b[i + 1] - (double)b[i]) <= rho * (double)b[i]) {
+      if (b[i + 1] < bs) bs = b[i + 1];
+      ++i;
+    }
+    block_batch[nblocks++] = bs;
+    ++i;
+  }
+  return nblocks;
+}
+
+int nf_set_stream(void* s) {
+  g_nf_stream = (cudaStream_t)s;
+  return NF_OK;
+}
+
+long long nf_launch_count(void) { return g_nf_launches; }
+
+const char* nf_layer_kernel_family(const nf_layer* L, int op) {
+  if (!L || op < 0 || op > 3) return "";
+  return L->fam[op] ? "tcgen05" : "cuda-core";
+}
+
+const char* nf_strerror(int st) {
+  switch (st) {
+    case NF_OK: return "ok";
+    case NF_EINVAL: return "invalid argument";
+    case NF_EALIGN: return "misaligned device pointer";
+    case NF_ENOWS: return "workspace missing or too small";
+    case NF_EUNSUPPORTED: return "unsupported shape";
+    case NF_ECUDA: return "CUDA runtime error";
+    default: return "unknown status";
+  }
+}
+
+const char* nf_last_cuda_error(void) { return g_nf_err; }
+
+}  // extern "C"

@@ -220,7 +220,7 @@ __global__ void __launch_bounds__(256) fc_ce_kernel(const float* __restrict__ p,
   }
   mx = block_reduce(mx, red, true);
   float se = 0.f;
-  for (int k = t; k < K; k += 256) se += __expf(ls[k] - mx);
+  for (int k = t; k < K; k += 256) se += expf(ls[k] - mx);
   se = block_reduce(se, red, false);
   const float lse = mx + logf(se);
   int lab = labels[n];

@@ -1,0 +1,16 @@
+// Tensor-core (tcgen05 / TMEM / TMA) convolution kernels: interface used by the step sequencer.
+#pragma once
+#include "nf_internal.h"
+
+// Chooses, per operation, whether the configured shape runs on the tcgen05 kernels (L->fam[]).
+void nf_tc_select(nf_layer* L);
+// Floats of split-K scratch the tensor-core weight gradient needs (0 if unused).
+size_t nf_tc_scratch_floats(const nf_layer* L);
+// Called once the workspace is bound: encodes the TMA descriptors that point into it.
+int nf_tc_prepare(nf_layer* L);
+// y = conv(x) in bf16 plus per-CTA channel partials (sum, sum of squares) in L->red; nb = partial count.
+int nf_tc_conv_fwd(nf_layer* L, const void* x, int& nb);
+// Same convolution for `count` samples without statistics (cache-filling forward).
+int nf_tc_conv_fwd_eval(nf_layer* L, const void* x, int count);
+// grad(W) = wgrad(x, L->dy) into the gradient arena.
+int nf_tc_wgrad(nf_layer* L, const void* x);

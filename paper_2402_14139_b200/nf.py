@@ -1,0 +1,229 @@
+"""Thin ctypes binding of libnf.so: argument marshalling only, same names as include/nf.h.
+
+Every step of the path runs inside the library's CUDA kernels.  There is no CPU fallback: if
+libnf.so is missing or a call fails, an exception is raised.  torch is used for device memory
+and streams only.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libnf.so")
+
+NF_OK, NF_EINVAL, NF_EALIGN, NF_ENOWS, NF_EUNSUPPORTED, NF_ECUDA = 0, -1, -2, -3, -4, -5
+NF_ELABEL, NF_ENONFINITE, NF_ETIMEOUT = 1, 2, 4
+NF_F32, NF_BF16 = 0, 1
+NF_P_W, NF_P_GAMMA, NF_P_BETA, NF_P_WA, NF_P_BA, NF_P_WF, NF_P_BF, NF_P_RMEAN, NF_P_RVAR = range(9)
+NF_K_VALUE, NF_K_MOMENTUM, NF_K_GRAD = 0, 0x100, 0x200
+PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P_BA, Wf=NF_P_WF, bf=NF_P_BF,
+                 rmean=NF_P_RMEAN, rvar=NF_P_RVAR)
+
+EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_layer_workspace_bytes",
+           "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
+           "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
+           "nf_block_cache_n", "nf_cache_gather", "nf_partition", "nf_set_stream", "nf_launch_count",
+           "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
+
+
+class NfError(RuntimeError):
+    pass
+
+
+class nf_layer_opts(C.Structure):
+    _fields_ = [("N", C.c_int), ("stride", C.c_int), ("maxpool", C.c_int), ("dtype", C.c_int),
+                ("momentum", C.c_float), ("bn_eps", C.c_float), ("bn_momentum", C.c_float), ("host_io", C.c_int)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C-ABI library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_SO):
+            raise NfError(f"{_SO} not found: build it with `python -m paper_2402_14139_b200.build`")
+        L = C.CDLL(_SO)
+        vp, ip, fp = C.c_void_p, C.c_void_p, C.c_void_p
+        L.nf_layer_create.restype = vp
+        L.nf_layer_create.argtypes = [C.c_int] * 6
+        L.nf_layer_destroy.restype = None
+        L.nf_layer_destroy.argtypes = [vp]
+        L.nf_layer_configure.argtypes = [vp, C.POINTER(nf_layer_opts)]
+        L.nf_layer_workspace_bytes.restype = C.c_size_t
+        L.nf_layer_workspace_bytes.argtypes = [vp]
+        L.nf_layer_bind_workspace.argtypes = [vp, vp, C.c_size_t]
+        L.nf_layer_set_param.argtypes = [vp, C.c_int, fp, C.c_size_t]
+        L.nf_layer_get_param.argtypes = [vp, C.c_int, fp, C.c_size_t]
+        L.nf_layer_step.argtypes = [vp, vp, ip, C.c_float, fp, vp]
+        L.nf_layer_step_host.argtypes = [vp, vp, ip, C.c_float, fp, vp]
+        L.nf_layer_status.argtypes = [vp]
+        L.nf_block_create.restype = vp
+        L.nf_block_create.argtypes = [C.POINTER(vp), C.c_int]
+        L.nf_block_destroy.restype = None
+        L.nf_block_destroy.argtypes = [vp]
+        L.nf_block_cache.argtypes = [vp, vp, vp]
+        L.nf_block_cache_n.argtypes = [vp, vp, vp, C.c_int]
+        L.nf_cache_gather.argtypes = [vp, ip, ip, C.c_int, C.c_size_t, vp, ip]
+        L.nf_partition.argtypes = [C.POINTER(C.c_int), C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int),
+                                   C.POINTER(C.c_int)]
+        L.nf_set_stream.argtypes = [vp]
+        L.nf_launch_count.restype = C.c_longlong
+        L.nf_layer_kernel_family.restype = C.c_char_p
+        L.nf_layer_kernel_family.argtypes = [vp, C.c_int]
+        L.nf_strerror.restype = C.c_char_p
+        L.nf_strerror.argtypes = [C.c_int]
+        L.nf_last_cuda_error.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def _check(rc: int, what: str):
+    if rc != NF_OK:
+        msg = lib().nf_strerror(rc).decode()
+        if rc == NF_ECUDA:
+            msg += ": " + lib().nf_last_cuda_error().decode()
+        raise NfError(f"{what}: {msg} ({rc})")
+
+
+def nf_strerror(rc: int) -> str:
+    return lib().nf_strerror(rc).decode()
+
+
+def nf_launch_count() -> int:
+    return int(lib().nf_launch_count())
+
+
+def nf_set_stream(stream=None):
+    """stream: a torch.cuda.Stream, a raw cudaStream_t integer, or None for the default stream."""
+    h = 0 if stream is None else int(getattr(stream, "cuda_stream", stream))
+    _check(lib().nf_set_stream(C.c_void_p(h)), "nf_set_stream")
+
+
+def nf_partition(max_batch, B: int, rho: float):
+    """Algorithm 1: returns [(first_layer, last_layer, batch_size)] (0-based, inclusive)."""
+    n = len(max_batch)
+    mb = (C.c_int * n)(*[int(v) for v in max_batch])
+    first, bs = (C.c_int * n)(), (C.c_int * n)()
+    nb = lib().nf_partition(mb, n, int(B), float(rho), first, bs)
+    if nb < 0:
+        _check(nb, "nf_partition")
+    out = []
+    for i in range(nb):
+        last = (first[i + 1] - 1) if i + 1 < nb else n - 1
+        out.append((first[i], last, bs[i]))
+    return out
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+class Layer:
+    """One layer with its auxiliary head on the current CUDA device (wraps nf_layer_* calls)."""
+
+    def __init__(self, Cin, Cout, H, W, F, classes, N, stride=1, maxpool=False, dtype=NF_BF16, momentum=0.9,
+                 bn_eps=1e-5, bn_momentum=0.1, host_io=False, device="cuda"):
+        import torch
+        self._torch = torch
+        self.Cin, self.Cout, self.H, self.W, self.F, self.classes, self.N = Cin, Cout, H, W, F, classes, N
+        self.stride, self.maxpool, self.dtype = stride, bool(maxpool), dtype
+        self.Ho, self.Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+        self.Ha, self.Wa = (self.Ho // 2, self.Wo // 2) if maxpool else (self.Ho, self.Wo)
+        self.h = lib().nf_layer_create(Cin, Cout, H, W, F, classes)
+        if not self.h:
+            raise NfError("nf_layer_create failed")
+        o = nf_layer_opts(N, stride, int(maxpool), dtype, momentum, bn_eps, bn_momentum, int(host_io))
+        _check(lib().nf_layer_configure(self.h, C.byref(o)), "nf_layer_configure")
+        self.ws_bytes = int(lib().nf_layer_workspace_bytes(self.h))
+        self.ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device=device)
+        base = (self.ws.data_ptr() + 255) // 256 * 256
+        _check(lib().nf_layer_bind_workspace(self.h, C.c_void_p(base), self.ws_bytes), "nf_layer_bind_workspace")
+        self.shapes = dict(W=(Cout, Cin, 3, 3), gamma=(Cout,), beta=(Cout,), Wa=(F, Cout, 3, 3), ba=(F,),
+                           Wf=(classes, 4 * F), bf=(classes,), rmean=(Cout,), rvar=(Cout,))
+        self.tdtype = torch.float32 if dtype == NF_F32 else torch.bfloat16
+        self.device = device
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().nf_layer_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_param(self, name, array, kind=NF_K_VALUE):
+        a = np.ascontiguousarray(array, dtype=np.float32).reshape(self.shapes[name])
+        _check(lib().nf_layer_set_param(self.h, PARAM_IDS[name] | kind, a.ctypes.data_as(C.c_void_p), a.size),
+               f"nf_layer_set_param({name})")
+
+    def get_param(self, name, kind=NF_K_VALUE):
+        a = np.empty(self.shapes[name], dtype=np.float32)
+        _check(lib().nf_layer_get_param(self.h, PARAM_IDS[name] | kind, a.ctypes.data_as(C.c_void_p), a.size),
+               f"nf_layer_get_param({name})")
+        return a
+
+    def new_act(self):
+        return self._torch.empty((self.N, self.Ha, self.Wa, self.Cout), dtype=self.tdtype, device=self.device)
+
+    def step(self, x, labels, lr, loss_out, act_out):
+        """nf_layer_step on device tensors: x [N,H,W,Cin], labels int32 [N], loss_out float32 [1],
+        act_out [N,Ha,Wa,Cout]; asynchronous."""
+        _check(lib().nf_layer_step(self.h, _ptr(x), _ptr(labels), float(lr), _ptr(loss_out), _ptr(act_out)),
+               "nf_layer_step")
+
+    def step_host(self, x_host, labels_host, lr, loss_host, act_host=None):
+        """nf_layer_step_host on host tensors (pinned for speed); synchronous."""
+        _check(lib().nf_layer_step_host(self.h, _ptr(x_host), _ptr(labels_host), float(lr), _ptr(loss_host),
+                                        _ptr(act_host)), "nf_layer_step_host")
+
+    def status(self) -> int:
+        rc = lib().nf_layer_status(self.h)
+        if rc < 0:
+            _check(rc, "nf_layer_status")
+        return rc
+
+    def kernel_family(self, op: int) -> str:
+        return lib().nf_layer_kernel_family(self.h, op).decode()
+
+
+class Block:
+    """Consecutive layers trained at one batch size (wraps nf_block_*)."""
+
+    def __init__(self, layers):
+        self.layers = list(layers)
+        arr = (C.c_void_p * len(layers))(*[l.h for l in layers])
+        self.h = lib().nf_block_create(arr, len(layers))
+        if not self.h:
+            raise NfError("nf_block_create failed: layers do not chain or have no workspace")
+
+    def cache(self, x, out, count=None):
+        if count is None:
+            _check(lib().nf_block_cache(self.h, _ptr(x), _ptr(out)), "nf_block_cache")
+        else:
+            _check(lib().nf_block_cache_n(self.h, _ptr(x), _ptr(out), int(count)), "nf_block_cache_n")
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().nf_block_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def nf_cache_gather(cache, cache_labels, idx, out, out_labels):
+    """out[i] = cache[idx[i]] (rows) and labels likewise; device tensors, idx int32."""
+    row_bytes = cache[0].numel() * cache.element_size()
+    _check(lib().nf_cache_gather(_ptr(cache), _ptr(cache_labels), _ptr(idx), int(idx.numel()), row_bytes, _ptr(out),
+                                 _ptr(out_labels)), "nf_cache_gather")
