@@ -1,0 +1,74 @@
+"""CPU-side checks of the C-ABI library: it loads without a GPU, exports every symbol the header
+declares, and its host-only entry points behave (no kernel is launched here)."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import nfo
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def nf():
+    from paper_2402_14139_b200 import build
+    build.build()
+    from paper_2402_14139_b200 import nf as mod
+    return mod
+
+
+def test_every_declared_symbol_is_exported(nf):
+    hdr = open(os.path.join(ROOT, "include", "nf.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    declared = sorted(set(re.findall(r"\b(nf_[a-z_0-9]+)\s*\(", hdr)))
+    assert len(declared) >= 20
+    L = nf.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+    assert sorted(nf.EXPORTS) == declared
+
+
+def test_create_configure_and_workspace_size_are_host_only(nf):
+    L = nf.lib()
+    assert not L.nf_layer_create(0, 16, 32, 32, 4, 10)
+    h = L.nf_layer_create(3, 16, 32, 32, 4, 10)
+    assert h
+    o = nf.nf_layer_opts(8, 1, 0, nf.NF_F32, 0.9, 1e-5, 0.1, 0)
+    assert L.nf_layer_configure(h, C.byref(o)) == nf.NF_OK
+    small = L.nf_layer_workspace_bytes(h)
+    o.N = 64
+    assert L.nf_layer_configure(h, C.byref(o)) == nf.NF_OK
+    assert L.nf_layer_workspace_bytes(h) > small > 0
+    for bad in (dict(N=0), dict(stride=3), dict(dtype=7), dict(momentum=1.5)):
+        ob = nf.nf_layer_opts(8, 1, 0, nf.NF_F32, 0.9, 1e-5, 0.1, 0)
+        for k, v in bad.items():
+            setattr(ob, k, v)
+        assert L.nf_layer_configure(h, C.byref(ob)) == nf.NF_EINVAL
+    h2 = L.nf_layer_create(3, 16, 31, 31, 4, 10)   # 31x31 output cannot be max-pooled 2x2
+    op = nf.nf_layer_opts(8, 1, 1, nf.NF_F32, 0.9, 1e-5, 0.1, 0)
+    assert L.nf_layer_configure(h2, C.byref(op)) == nf.NF_EINVAL
+    # calls that need a workspace refuse without one
+    assert L.nf_layer_step(h, None, None, 0.1, None, None) == nf.NF_EINVAL
+    buf = np.zeros(16, dtype=np.float32)
+    assert L.nf_layer_get_param(h, nf.NF_P_GAMMA, buf.ctypes.data_as(C.c_void_p), 16) == nf.NF_ENOWS
+    L.nf_layer_destroy(h)
+    L.nf_layer_destroy(h2)
+    assert nf.nf_strerror(nf.NF_ENOWS) and nf.nf_strerror(nf.NF_OK) == "ok"
+
+
+def test_partition_matches_checker_and_paper_example(nf):
+    gold = os.path.join(ROOT, "tests", "golden", "vgg19_max_batch_630mb.txt")
+    mb = [int(v) for v in [ln for ln in open(gold) if not ln.startswith("#")][0].split()]
+    assert nf.nf_partition(mb, 512, 0.4) == [(0, 2, 30), (3, 3, 60), (4, 7, 90), (8, 11, 195), (12, 15, 512)]
+    rng = np.random.default_rng(1)
+    for _ in range(200):
+        n = int(rng.integers(1, 20))
+        v = rng.integers(1, 2000, n).tolist()
+        B = int(rng.integers(1, 1500))
+        rho = float(rng.choice([0.0, 0.1, 0.4, 0.7]))
+        assert nf.nf_partition(v, B, rho) == nfo.partition(v, B, rho)
+    with pytest.raises(nf.NfError):
+        nf.nf_partition([10, 0], 100, 0.4)

@@ -1,0 +1,118 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU checker, element by element,
+on the same seeded inputs.  Tolerances are those of parity_util.TOL."""
+import numpy as np
+import pytest
+
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2402_14139_b200 import nf
+    nf.lib()
+    return nf, torch
+
+
+# config 1 of the benchmark suite: single fp32 layer, 8x3x32x32, 3->16, F=4, 10 classes
+CFG1 = dict(N=8, Cin=3, Cout=16, H=32, W=32, F=4, classes=10, stride=1, pool=False)
+
+SMALL = [
+    dict(N=4, Cin=3, Cout=5, H=6, W=6, F=3, classes=7, stride=1, pool=False),      # ragged channel counts
+    dict(N=3, Cin=2, Cout=4, H=8, W=8, F=2, classes=5, stride=2, pool=False),      # stride 2
+    dict(N=3, Cin=3, Cout=4, H=8, W=8, F=3, classes=4, stride=1, pool=True),       # max-pool layer
+    dict(N=2, Cin=2, Cout=3, H=5, W=7, F=2, classes=3, stride=1, pool=False),      # odd sizes, overlapping bins
+    dict(N=2, Cin=35, Cout=18, H=19, W=21, F=5, classes=11, stride=2, pool=False), # several tiles + ragged tails
+    dict(N=1, Cin=1, Cout=1, H=1, W=1, F=1, classes=2, stride=1, pool=False),      # degenerate 1x1
+    dict(N=2, Cin=4, Cout=8, H=2, W=2, F=2, classes=3, stride=1, pool=True),       # pool down to 1x1
+]
+
+
+def test_config1_fp32_single_step(env):
+    nf, torch = env
+    w = pu.check_step(nf, torch, CFG1, seed=0x4E460001, dtype=nf.NF_F32, lr=0.01, steps=1)
+    print("config1 fp32 worst relative errors:", w)
+
+
+def test_config1_fp32_three_steps(env):
+    nf, torch = env
+    pu.check_step(nf, torch, CFG1, seed=0x4E460001, dtype=nf.NF_F32, lr=0.01, steps=3)
+
+
+@pytest.mark.parametrize("ci", range(len(SMALL)))
+def test_small_shapes_fp32(env, ci):
+    nf, torch = env
+    pu.check_step(nf, torch, SMALL[ci], seed=100 + ci, dtype=nf.NF_F32, lr=0.05, steps=2)
+
+
+@pytest.mark.parametrize("ci", range(len(SMALL) - 2))
+def test_small_shapes_bf16(env, ci):
+    nf, torch = env
+    pu.check_step(nf, torch, SMALL[ci], seed=200 + ci, dtype=nf.NF_BF16, lr=0.05, steps=1)
+
+
+def test_uniform_head_loss_is_log_classes(env):
+    nf, torch = env
+    c = CFG1
+    P, x, y = pu.seeded_case(c, 5, bf16=False)
+    P["Wf"][:] = 0
+    P["bf"][:] = 0
+    G = pu.gpu_layer(nf, c, P, nf.NF_F32)
+    loss = torch.zeros(1, device="cuda")
+    act = G.new_act()
+    G.step(pu.to_device_nhwc(torch, x, 0), torch.from_numpy(y).cuda(), 0.0, loss, act)
+    assert abs(float(loss.item()) - np.log(10)) <= 1e-5 * np.log(10)
+    g = G.get_param("bf", nf.NF_K_GRAD)
+    assert abs(g.sum()) < 1e-6          # softmax-CE gradients sum to zero across classes
+
+
+def test_bad_label_is_flagged_and_clamped(env):
+    nf, torch = env
+    c = CFG1
+    P, x, y = pu.seeded_case(c, 6, bf16=False)
+    G = pu.gpu_layer(nf, c, P, nf.NF_F32)
+    y = y.copy()
+    y[3] = 10
+    loss = torch.zeros(1, device="cuda")
+    G.step(pu.to_device_nhwc(torch, x, 0), torch.from_numpy(y).cuda(), 0.0, loss, G.new_act())
+    assert G.status() & nf.NF_ELABEL
+    assert G.status() == 0
+    assert np.isfinite(float(loss.item()))
+
+
+def test_argument_errors(env):
+    nf, torch = env
+    c = CFG1
+    P, x, y = pu.seeded_case(c, 7, bf16=False)
+    G = pu.gpu_layer(nf, c, P, nf.NF_F32)
+    xd = pu.to_device_nhwc(torch, x, 0)
+    yd = torch.from_numpy(y).cuda()
+    loss = torch.zeros(1, device="cuda")
+    act = G.new_act()
+    with pytest.raises(nf.NfError):
+        G.step(xd, yd, 0.1, loss, None)                      # act_out is required
+    with pytest.raises(nf.NfError):
+        G.step(xd.view(-1)[1:], yd, 0.1, loss, act)          # 4-byte offset: not 16-byte aligned
+    with pytest.raises(nf.NfError):
+        G.set_param("W", np.zeros((16, 3, 3, 3), np.float32), kind=nf.NF_K_GRAD)
+
+
+def test_step_host_matches_device_step(env):
+    nf, torch = env
+    c = CFG1
+    P, x, y = pu.seeded_case(c, 8, bf16=False)
+    A = pu.gpu_layer(nf, c, P, nf.NF_F32)
+    B = pu.gpu_layer(nf, c, P, nf.NF_F32, host_io=True)
+    xh = torch.from_numpy(np.ascontiguousarray(np.transpose(x, (0, 2, 3, 1)))).pin_memory()
+    yh = torch.from_numpy(y).pin_memory()
+    loss_a = torch.zeros(1, device="cuda")
+    act_a = A.new_act()
+    A.step(xh.cuda(), yh.cuda(), 0.01, loss_a, act_a)
+    loss_h = torch.zeros(1).pin_memory()
+    act_h = torch.empty(act_a.shape, dtype=act_a.dtype).pin_memory()
+    B.step_host(xh, yh, 0.01, loss_h, act_h)
+    assert float(loss_h.item()) == float(loss_a.item())
+    assert torch.equal(act_h, act_a.cpu())
+    assert np.array_equal(A.get_param("W"), B.get_param("W"))
