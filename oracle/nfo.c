@@ -288,7 +288,24 @@ void nfo_sgd(double* theta, double* v, const double* g, size_t n, double lr, dou
 typedef struct {
   int N, Cin, Cout, H, W, stride, pool, F, classes;
   double eps, momentum, bn_momentum;
+  int store_bf16; /* 1: the two tensors the method keeps in bfloat16 (conv output y, activation x_{n+1}) are
+                     rounded to bfloat16 where they are stored, so that every decision taken from them (ReLU
+                     masks, pool argmax) is taken in the storage precision; all arithmetic stays fp64 */
 } nfo_dims;
+
+/* Round to the nearest bfloat16, ties to even (via float, as a bf16 store of an fp32 value does). */
+double nfo_round_bf16(double v) {
+  float f = (float)v;
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7f800000u) == 0x7f800000u) return (double)f; /* inf / nan unchanged */
+  u = (u + 0x7fffu + ((u >> 16) & 1u)) & 0xffff0000u;
+  memcpy(&f, &u, 4);
+  return (double)f;
+}
+static void store_round(double* a, size_t n, int on) {
+  if (on) for (size_t k = 0; k < n; ++k) a[k] = nfo_round_bf16(a[k]);
+}
 
 /* Parameters and optimiser state of one layer with its auxiliary head; updated in place. */
 typedef struct {
@@ -333,8 +350,10 @@ double nfo_layer_step(const nfo_dims* d, const double* x, const int32_t* labels,
 
   /* forward: Eq. 1 */
   nfo_conv3x3(x, N, Ci, H, W, P->W, Co, NULL, s, y);
+  store_round(y, ny, d->store_bf16);
   nfo_bn_train(y, N, Co, Ho * Wo, P->gamma, P->beta, d->eps, mu, var, xhat, z);
   nfo_relu(z, ny, r);
+  store_round(r, ny, d->store_bf16); /* rounding is monotone: pooling rounded values = rounding the pooled value */
   if (d->pool) nfo_maxpool2(r, N, Co, Ho, Wo, a, arg);
   else memcpy(a, r, ny * sizeof(double));
   if (act_out) memcpy(act_out, a, na * sizeof(double));
@@ -431,8 +450,10 @@ void nfo_layer_eval(const nfo_dims* d, const double* x, const nfo_params* P, dou
   const size_t ny = (size_t)N * Co * Ho * Wo;
   double *y = dalloc(ny), *z = dalloc(ny), *r = dalloc(ny);
   nfo_conv3x3(x, N, d->Cin, d->H, d->W, P->W, Co, NULL, s, y);
+  store_round(y, ny, d->store_bf16);
   nfo_bn_eval(y, N, Co, Ho * Wo, P->gamma, P->beta, d->eps, P->rmean, P->rvar, z);
   nfo_relu(z, ny, r);
+  store_round(r, ny, d->store_bf16);
   if (d->pool) {
     int32_t* arg = (int32_t*)calloc(ny / 4 + 1, sizeof(int32_t));
     nfo_maxpool2(r, N, Co, Ho, Wo, out, arg);

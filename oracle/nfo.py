@@ -31,7 +31,7 @@ _ip = C.POINTER(C.c_int32)
 
 class Dims(C.Structure):
     _fields_ = [(k, C.c_int) for k in ("N", "Cin", "Cout", "H", "W", "stride", "pool", "F", "classes")] + \
-               [(k, C.c_double) for k in ("eps", "momentum", "bn_momentum")]
+               [(k, C.c_double) for k in ("eps", "momentum", "bn_momentum")] + [("store_bf16", C.c_int)]
 
 
 _PNAMES = ("W", "gamma", "beta", "Wa", "ba", "Wf", "bf")
@@ -55,6 +55,8 @@ def lib():
         _lib.nfo_layer_step.restype = C.c_double
         _lib.nfo_softmax_ce.restype = C.c_double
         _lib.nfo_threads.restype = C.c_int
+        _lib.nfo_round_bf16.restype = C.c_double
+        _lib.nfo_round_bf16.argtypes = [C.c_double]
     return _lib
 
 
@@ -174,8 +176,8 @@ class Layer:
     """Parameters, momentum and running statistics of one layer plus its auxiliary head (fp64)."""
 
     def __init__(self, Cin, Cout, H, W, F, classes, N, stride=1, pool=False, eps=1e-5, momentum=0.9,
-                 bn_momentum=0.1):
-        self.d = Dims(N, Cin, Cout, H, W, stride, int(pool), F, classes, eps, momentum, bn_momentum)
+                 bn_momentum=0.1, store_bf16=False):
+        self.d = Dims(N, Cin, Cout, H, W, stride, int(pool), F, classes, eps, momentum, bn_momentum, int(store_bf16))
         self.Ho, self.Wo = out_size(H, stride), out_size(W, stride)
         self.Ha, self.Wa = (self.Ho // 2, self.Wo // 2) if pool else (self.Ho, self.Wo)
         sh = dict(W=(Cout, Cin, 3, 3), gamma=(Cout,), beta=(Cout,), Wa=(F, Cout, 3, 3), ba=(F,),

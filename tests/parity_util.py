@@ -4,6 +4,9 @@ run one local step on each, and compare every output tensor within the stated to
 Tolerances (written here once, used by every parity test):
   fp32 path : max-abs error <= 1e-4 * max|tensor| for outputs and gradients, loss relative error <= 1e-5
   bf16 path : max-abs error <= 3e-2 * max|tensor|,                           loss relative error <= 1e-3
+In the bf16 path the checker keeps its two stored tensors (conv output, activation) in bfloat16 as
+the kernels do, so ReLU masks and pool argmax are decided in the same precision on both sides;
+all of its arithmetic stays fp64.
 """
 import numpy as np
 
@@ -31,9 +34,9 @@ def seeded_case(c, seed, bf16):
     return P, x, y
 
 
-def oracle_layer(c, P, momentum=0.9):
+def oracle_layer(c, P, momentum=0.9, store_bf16=False):
     L = nfo.Layer(c["Cin"], c["Cout"], c["H"], c["W"], c["F"], c["classes"], c["N"], stride=c.get("stride", 1),
-                  pool=c.get("pool", False), momentum=momentum)
+                  pool=c.get("pool", False), momentum=momentum, store_bf16=store_bf16)
     L.set(**{k: np.asarray(v, dtype=np.float64) for k, v in P.items()})
     return L
 
@@ -65,7 +68,7 @@ def check_step(nf, torch, c, seed, dtype, lr=0.01, steps=1, report=None):
     """Run `steps` consecutive local steps on both sides on the same batch and compare after each:
     act_out, loss, every gradient, every updated parameter, momentum and running statistics."""
     P, x, y = seeded_case(c, seed, bf16=(dtype == 1))
-    O = oracle_layer(c, P)
+    O = oracle_layer(c, P, store_bf16=(dtype == 1))
     G = gpu_layer(nf, c, P, dtype)
     xd = to_device_nhwc(torch, x, dtype)
     yd = torch.from_numpy(y).cuda()

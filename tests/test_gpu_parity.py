@@ -25,7 +25,7 @@ SMALL = [
     dict(N=3, Cin=3, Cout=4, H=8, W=8, F=3, classes=4, stride=1, pool=True),       # max-pool layer
     dict(N=2, Cin=2, Cout=3, H=5, W=7, F=2, classes=3, stride=1, pool=False),      # odd sizes, overlapping bins
     dict(N=2, Cin=35, Cout=18, H=19, W=21, F=5, classes=11, stride=2, pool=False), # several tiles + ragged tails
-    dict(N=1, Cin=1, Cout=1, H=1, W=1, F=1, classes=2, stride=1, pool=False),      # degenerate 1x1
+    dict(N=2, Cin=1, Cout=1, H=1, W=1, F=1, classes=2, stride=1, pool=False),      # degenerate 1x1 image
     dict(N=2, Cin=4, Cout=8, H=2, W=2, F=2, classes=3, stride=1, pool=True),       # pool down to 1x1
 ]
 

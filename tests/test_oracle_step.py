@@ -185,3 +185,24 @@ def test_bf16_rounding_ties_to_even():
     t = torch.tensor(v).to(torch.bfloat16).to(torch.float32).numpy()
     np.testing.assert_array_equal(r, t)
     np.testing.assert_array_equal(synth.from_bf16_bits(synth.to_bf16_bits(v)), r)
+
+
+def test_bf16_storage_mode_rounds_only_the_stored_tensors():
+    c = CASES[2]
+    L, x, y = make_layer(c, 21)
+    Lb, _, _ = make_layer(c, 21)
+    Lb.d.store_bf16 = 1
+    loss, act, tr = L.step(x, y, 0.0, update=False, trace=True)
+    loss_b, act_b, tr_b = Lb.step(x, y, 0.0, update=False, trace=True)
+    # stored tensors hold bfloat16 values exactly, and are the nearest ones to the unrounded tensors
+    for k in ("y", "a"):
+        np.testing.assert_array_equal(tr_b[k], synth.round_bf16(tr_b[k]).astype(np.float64))
+    np.testing.assert_array_equal(tr_b["y"], synth.round_bf16(tr["y"]).astype(np.float64))
+    np.testing.assert_array_equal(act_b, tr_b["a"])
+    # the rounding is a small perturbation of the exact step (bf16 has 8 significand bits)
+    assert np.abs(tr_b["y"] - tr["y"]).max() <= 2.0 ** -8 * np.abs(tr["y"]).max()
+    assert abs(loss_b - loss) <= 1e-2 * abs(loss)
+    # the scalar rounding routine agrees with a library conversion, ties to even included
+    v = np.array([1.0, 1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, -2.5, 3.14159, 1e-20, 65504.0, 0.0])
+    got = np.array([nfo.lib().nfo_round_bf16(float(t)) for t in v])
+    np.testing.assert_array_equal(got, torch.tensor(v, dtype=torch.float32).to(torch.bfloat16).double().numpy())
