@@ -1,0 +1,304 @@
+#!/usr/bin/env python
+"""Benchmark of the local-layer training step (one JSON line on stdout).
+
+  python bench.py --gpus N --steps K --warmup W [--workload c4|c2] [--impl reference]
+
+A step = one pass of the whole hot path over one batch: every layer of the block runs its local
+step in turn (conv+BN+ReLU forward, aux head forward/backward, weight gradients, SGD update).
+Multi-GPU: independent replicas, one process per GPU (the step has no exchange to shard over),
+timed as the max over ranks; value = images of all ranks / that time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "local-layer train-step images/s (bf16)"
+FALLBACK_PEAKS = dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0)
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"]))), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML every 100 ms."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.sm, self.reasons, self.max_mhz = index, False, [], set(), None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+        while not self.stop_flag:
+            try:
+                self.sm.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.1)
+
+    def summary(self):
+        return dict(sm_mhz=float(np.median(self.sm)) if self.sm else None, sm_max_mhz=self.max_mhz,
+                    reasons=sorted(self.reasons))
+
+
+def build_block(nf, torch, wl, bi, seed, host_io):
+    """Layers of block bi with Kaiming-normal conv/linear weights (seeded), as an nf.Block."""
+    from paper_2402_14139_b200 import synth
+    N, ls = wl["blocks"][bi]
+    dt = nf.NF_F32 if wl["dtype"] == "f32" else nf.NF_BF16
+    layers = []
+    for li, l in enumerate(ls):
+        L = nf.Layer(l["Cin"], l["Cout"], l["H"], l["W"], l["F"], wl["classes"], N, stride=l["stride"],
+                     maxpool=l["pool"], dtype=dt, host_io=(host_io and li == 0))
+        t = 100 * (bi * 32 + li)
+        L.set_param("W", synth.normal(seed, t + 1, L.shapes["W"], np.sqrt(2.0 / (9 * l["Cin"]))))
+        L.set_param("Wa", synth.normal(seed, t + 2, L.shapes["Wa"], np.sqrt(2.0 / (9 * l["Cout"]))))
+        L.set_param("Wf", synth.normal(seed, t + 3, L.shapes["Wf"], np.sqrt(2.0 / (4 * l["F"]))))
+        layers.append(L)
+    return nf.Block(layers), layers
+
+
+def op_model(l, N, classes, es, fam):
+    """Algorithmic work of each traced op of one layer step: ('tensor'|'alu', flops) or ('hbm', bytes)."""
+    from paper_2402_14139_b200 import workloads as W
+    fl = W.step_flops(l, N)
+    Ho, Wo = (l["H"] - 1) // l["stride"] + 1, (l["W"] - 1) // l["stride"] + 1
+    Ha, Wa = W.out_hw(l)
+    ny, na, nh = N * Ho * Wo * l["Cout"], N * Ha * Wa * l["Cout"], N * Ha * Wa * l["F"]
+    nparam = 9 * l["Cin"] * l["Cout"] + 2 * l["Cout"] + 9 * l["Cout"] * l["F"] + l["F"] + classes * (4 * l["F"] + 1)
+    tc = lambda k: "tensor" if fam[k] == "tcgen05" else "alu"
+    return dict(conv_fwd=(tc(0), fl["conv_fwd"]), wgrad=(tc(1), fl["wgrad"]), aux_fwd=(tc(2), fl["aux_fwd"]),
+                aux_bwd=(tc(3), fl["aux_bwd"]),
+                bn_fwd=("hbm", es * (ny + na)),            # read y, write a
+                bn_bwd=("hbm", es * (2 * ny + na)),        # read y and da, write dy
+                head=("hbm", es * nh + 4 * N * (8 * l["F"] + 2 * classes)),
+                sgd=("hbm", 18 * nparam))                  # theta, v read+write (fp32), g read, bf16 copy write
+
+
+def run_ours(args, rank, world):
+    import torch
+    from paper_2402_14139_b200 import nf, workloads
+    nf.lib()
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    wl = workloads.ALL[args.workload]()
+    bi = 0
+    N, ls = wl["blocks"][bi]
+    seed = 0x4E460000 + int(args.workload[1]) + 1000 * rank
+    es = 4 if wl["dtype"] == "f32" else 2
+    tdt = torch.float32 if es == 4 else torch.bfloat16
+    stream = torch.cuda.current_stream()
+    nf.nf_set_stream(stream)
+    block, layers = build_block(nf, torch, wl, bi, seed, host_io=True)
+    C, H, Wd = ls[0]["Cin"], ls[0]["H"], ls[0]["W"]
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    x_bytes = N * H * Wd * C * es
+    # inputs smaller than L2 (126 MB) are rotated through a pool larger than L2
+    n_pool = 1 if x_bytes > 256e6 else min(64, int(300e6 // max(x_bytes, 1)) + 2)
+    xs = [torch.randn((N, H, Wd, C), generator=g, device="cuda", dtype=torch.float32).to(tdt) for _ in range(n_pool)]
+    labels = torch.randint(0, wl["classes"], (N,), generator=g, device="cuda", dtype=torch.int32)
+    loss = torch.zeros(len(ls), dtype=torch.float32, device="cuda")
+    flush = torch.empty(int(256e6), dtype=torch.uint8, device="cuda") if n_pool == 1 and x_bytes <= 256e6 else None
+    lr = 0.01
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        block.step(xs[i % n_pool], labels, lr, loss)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = nf.nf_launch_count()
+    nf.nf_trace_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        block.step(xs[i % n_pool], labels, lr, loss)
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    trace = nf.nf_trace_read(len(ls))
+    nf.nf_trace_enable(False)
+    launches = nf.nf_launch_count() - launches0
+    sampler.stop_flag = True
+    sampler.join(timeout=2)
+    status = [L.status() for L in layers]
+    losses = loss.cpu().tolist()
+    if any(status) or not all(np.isfinite(losses)):
+        raise RuntimeError(f"device status {status}, losses {losses}")
+
+    # end to end: host buffers through the C ABI, copies inside the timed region
+    xh = xs[0].cpu().pin_memory()
+    lh = labels.cpu().pin_memory()
+    loss_h = torch.zeros(len(ls), dtype=torch.float32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+    block.step_host(xh, lh, lr, loss_h)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        block.step_host(xh, lh, lr, loss_h)
+    barrier()
+    e2e_s = time.perf_counter() - t0
+
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms, e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_s = float(t[0]), float(t[1])
+
+    peaks, peak_src = load_peaks()
+    fam = [[L.kernel_family(k) for k in range(4)] for L in layers]
+    kernels, best = [], None
+    tot_ms = sum(v[0] for v in trace.values())
+    for (op, slot), (tms, cnt) in sorted(trace.items(), key=lambda kv: -kv[1][0]):
+        kind, work = op_model(ls[slot], N, wl["classes"], es, fam[slot])[op]
+        per = tms / cnt
+        if kind == "hbm":
+            ach, peak, unit = work / per / 1e6, peaks["hbm_gbs"], "GB/s"
+        else:
+            ach, peak, unit = work / per / 1e9, peaks["bf16_tflops_sustained"], "TFLOP/s"
+        rec = dict(op=op, layer=slot, bound=kind, ms_per_launch=round(per, 4), share=round(tms / tot_ms, 4),
+                   achieved=round(ach, 2), peak=peak, unit=unit, frac=round(ach / peak, 4))
+        kernels.append(rec)
+        if best is None:
+            best = rec
+    roof = dict(bound=best["bound"], achieved=best["achieved"], peak=best["peak"], unit=best["unit"],
+                frac=best["frac"], traffic=None, kernel=f'{best["op"]}[layer {best["layer"]}]',
+                peak_source=f"{peak_src} (sustained bf16 figure: kernel timed inside a long step)"
+                if best["bound"] != "hbm" else peak_src)
+
+    out = None
+    if rank == 0:
+        images = N * args.steps * world
+        out = dict(metric=METRIC, value=round(images / (ms / 1e3), 2), unit="images/s", n_gpus=world, steps=args.steps,
+                   warmup=args.warmup, ms_per_step=round(ms / args.steps, 4), higher_is_better=True, scaling="weak",
+                   vs_baseline=None, dtype="bf16" if es == 2 else "f32", data="synthetic",
+                   config=dict(workload=f"{wl['name']}: " + workloads.ALL[args.workload].__doc__.split(".")[0].strip(),
+                               batch=N, layers=len(ls), l2="inputs larger than L2" if n_pool == 1 else
+                               f"{n_pool} input batches rotated (pool larger than L2)", replicas=world,
+                               kernel_families=fam),
+                   clocks=sampler.summary(), gpu_launches=int(launches),
+                   e2e=dict(value=round(N * e2e_steps * world / e2e_s, 2), unit="images/s",
+                            h2d_bytes_per_step=int(x_bytes + 4 * N), d2h_bytes_per_step=int(4 * len(ls))),
+                   roofline=roof, kernels=kernels, final_losses=[round(v, 4) for v in losses])
+    return out, wl, bi
+
+
+def oracle_sample(wl, bi, n_sample, seed, steps=1):
+    """Times the CPU checker, as it stands, on n_sample images through every layer of the block."""
+    from oracle import nfo
+    from paper_2402_14139_b200 import synth
+    N, ls = wl["blocks"][bi]
+    layers = []
+    for li, l in enumerate(ls):
+        L = nfo.Layer(l["Cin"], l["Cout"], l["H"], l["W"], l["F"], wl["classes"], n_sample, stride=l["stride"],
+                      pool=l["pool"], store_bf16=(wl["dtype"] == "bf16"))
+        L.set(W=synth.normal(seed, 100 * li + 1, L.shapes["W"], np.sqrt(2.0 / (9 * l["Cin"]))),
+              Wa=synth.normal(seed, 100 * li + 2, L.shapes["Wa"], np.sqrt(2.0 / (9 * l["Cout"]))),
+              Wf=synth.normal(seed, 100 * li + 3, L.shapes["Wf"], np.sqrt(2.0 / (4 * l["F"]))))
+        layers.append(L)
+    x0 = synth.normal(seed, 7, (n_sample, ls[0]["Cin"], ls[0]["H"], ls[0]["W"]))
+    y = synth.labels(seed, 8, n_sample, wl["classes"])
+    times = []
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        x = x0
+        for L in layers:
+            _, x, _ = L.step(x, y, 0.01)
+        times.append(time.perf_counter() - t0)
+    return times, nfo.threads()
+
+
+def run_reference(args):
+    """The reference arm: the CPU checker on the host cores, same metric and workload."""
+    from paper_2402_14139_b200 import workloads
+    wl = workloads.ALL[args.workload]()
+    n_sample = 1 if args.workload == "c4" else min(8, wl["blocks"][0][0])
+    oracle_sample(wl, 0, n_sample, 1, steps=max(0, min(args.warmup, 1)))
+    times, cores = oracle_sample(wl, 0, n_sample, 2, steps=args.steps)
+    total = sum(times)
+    v = round(n_sample * args.steps / total, 4)
+    sample = f"{n_sample} image(s) per step through all {len(wl['blocks'][0][1])} layers of the block"
+    return dict(impl="reference", metric=METRIC, value=v, unit="images/s", n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=round(1e3 * total / args.steps, 2), higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=f"{wl['name']}: " + workloads.ALL[args.workload].__doc__.split(".")[0].strip(),
+                            sample=sample),
+                cpu_baseline=dict(value=v, unit="images/s", cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=v, unit="images/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c4", choices=["c2", "c4"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank, world = int(os.environ.get("RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args)), flush=True)
+        return
+    out, wl, bi = run_ours(args, rank, world)
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            n_sample = 4 if args.workload == "c4" else wl["blocks"][bi][0]
+            times, cores = oracle_sample(wl, bi, n_sample, 3)
+            out["cpu_baseline"] = dict(value=round(n_sample / times[0], 4), unit="images/s", cores=cores, kind="oracle",
+                                       sample=f"one step of {n_sample} images through all layers of the block "
+                                              f"({times[0]:.1f} s)")
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -155,6 +155,20 @@ void nf_block_destroy(nf_block* block);
 int nf_block_cache(nf_block* block, const void* x, void* out);
 int nf_block_cache_n(nf_block* block, const void* x, void* out, int count);
 
+/* One pass of Algorithm 2's inner loop over ALL layers of the block on one batch: layer 1 steps
+ * on x, every later layer steps on the activation its predecessor just produced (computed before
+ * that predecessor's update), each with its own local loss.
+ * x: device [N][H][W][Cin] of the first layer; labels: device int32[N];
+ * loss_out: device float[n_layers] (one local loss per layer);
+ * act_out: device [N][Ha][Wa][Cout] of the last layer, or NULL to keep it in the layer's workspace. */
+int nf_block_step(nf_block* block, const void* x, const int32_t* labels, float lr, float* loss_out, void* act_out);
+
+/* The same pass with HOST buffers: copies x and labels in, runs nf_block_step, copies the n_layers
+ * losses (and, if act_out_host is non-NULL, the last activation) back, synchronises.
+ * The first layer must have been configured with host_io = 1. */
+int nf_block_step_host(nf_block* block, const void* x_host, const int32_t* labels_host, float lr,
+                       float* loss_host, void* act_out_host);
+
 /* Re-batching from the cache: out[i] = cache[idx[i]] for i < count, rows of row_bytes bytes
  * (a multiple of 16); labels likewise if both label pointers are non-NULL.  All device pointers.
  * Bit-exact copy. */
@@ -169,6 +183,18 @@ int nf_partition(const int* max_batch, int n_layers, int B, double rho, int* blo
 
 /* Stream for all later calls (a cudaStream_t); NULL selects the default stream. */
 int nf_set_stream(void* cuda_stream);
+
+/* Per-operation device timing (CUDA events on the library's stream around each group of kernels).
+ * nf_trace_enable(1) starts recording and clears the totals; nf_trace_read synchronises the stream
+ * and returns, for op in [0, NF_TRACE_OPS) and layer position slot in [0, NF_TRACE_SLOTS) (the index
+ * of the layer inside the block for nf_block_step, 0 for a bare nf_layer_step), the summed
+ * milliseconds and the number of timed groups.
+ * Ops: 0 main conv forward (+statistics partials), 1 BatchNorm finalize+apply, 2 aux conv forward,
+ * 3 pooling + linear + cross-entropy forward/backward, 4 aux conv backward (dh, weight and input
+ * gradients), 5 BatchNorm backward, 6 main conv weight gradient, 7 SGD update. */
+enum { NF_TRACE_OPS = 8, NF_TRACE_SLOTS = 32 };
+int nf_trace_enable(int on);
+int nf_trace_read(int op, int slot, double* ms_total, long long* groups);
 
 /* Kernel launches enqueued by this library since the process started. */
 long long nf_launch_count(void);

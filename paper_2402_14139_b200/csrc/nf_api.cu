@@ -22,6 +22,45 @@ int nf_cuda_check(cudaError_t e, const char* what) {
 
 namespace {
 
+// ---- per-operation event timing
+struct TraceRec { cudaEvent_t a, b; int op, slot; };
+std::vector<TraceRec> g_recs;
+size_t g_rec_used = 0;
+bool g_trace_on = false;
+double g_trace_ms[NF_TRACE_OPS][NF_TRACE_SLOTS];
+long long g_trace_cnt[NF_TRACE_OPS][NF_TRACE_SLOTS];
+int g_trace_slot = 0;
+
+void trace_begin(int op) {
+  if (!g_trace_on) return;
+  if (g_rec_used == g_recs.size()) {
+    if (g_recs.size() >= 65536) return;
+    TraceRec r;
+    if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) return;
+    g_recs.push_back(r);
+  }
+  g_recs[g_rec_used].op = op;
+  g_recs[g_rec_used].slot = g_trace_slot;
+  cudaEventRecord(g_recs[g_rec_used].a, g_nf_stream);
+}
+void trace_end() {
+  if (!g_trace_on || g_rec_used >= g_recs.size()) return;
+  cudaEventRecord(g_recs[g_rec_used].b, g_nf_stream);
+  ++g_rec_used;
+}
+int trace_flush() {
+  NF_CUDA(cudaStreamSynchronize(g_nf_stream));
+  for (size_t i = 0; i < g_rec_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, g_recs[i].a, g_recs[i].b) == cudaSuccess) {
+      g_trace_ms[g_recs[i].op][g_recs[i].slot] += ms;
+      g_trace_cnt[g_recs[i].op][g_recs[i].slot] += 1;
+    }
+  }
+  g_rec_used = 0;
+  return NF_OK;
+}
+
 // Carves the workspace; with base == nullptr only sizes it.
 struct Carver {
   char* base;
@@ -61,6 +100,7 @@ size_t plan(nf_layer* L, char* base, bool assign) {
   D->h = c.take(nh * es);
   D->dh = c.take(nh * es);
   D->da = c.take(na * es);
+  D->act = c.take(na * es);
   D->p = (float*)c.take(N * 4 * F * 4);
   D->dp = (float*)c.take(N * 4 * F * 4);
   D->logits = (float*)c.take(N * K * 4);
@@ -257,40 +297,57 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
   int nb = 0;
 
   // Eq. 1: conv, BatchNorm (batch statistics), ReLU, optional max-pool -> act_out
+  trace_begin(0);
   if (L->fam[0]) {
     NF_TRY(nf_tc_conv_fwd(L, x, nb));
   } else {
     NF_TRY(nf_ref_conv(dt, x, N, L->H, L->W, Ci, Wm, (long)Co * Ci, Ci, 1, 0, nullptr, 0, s, Co, L->y));
     NF_TRY(nf_ref_channel_sums(dt, L->y, (size_t)N * Ho * Wo, Co, L->red, L->red_floats, &nb));
   }
+  trace_end();
+  trace_begin(1);
   NF_TRY(nf_ref_bn_finalize(L->red, nb, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
                             L->o.bn_momentum, L->scale, L->shift, L->mu, L->invstd, L->rmean, L->rvar));
   NF_TRY(nf_ref_bn_apply(dt, L->y, N, Ho, Wo, Co, pool, L->scale, L->shift, act_out));
+  trace_end();
   // Eq. 2: aux conv + ReLU, average pool to 2x2, linear; Eq. 3: softmax cross-entropy
+  trace_begin(2);
   NF_TRY(nf_ref_conv(dt, act_out, N, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
+  trace_end();
+  trace_begin(3);
   NF_TRY(nf_ref_avgpool(dt, L->h, N, Ha, Wa, F, L->p));
   NF_TRY(nf_ref_fc_ce(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits,
                       L->dp, L->lossn, L->status));
   // gradients of gamma_n, beta_n
   NF_TRY(nf_ref_fc_wgrad(L->p, L->dlogits, L->lossn, N, D, K, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->status));
+  trace_end();
+  trace_begin(4);
   NF_TRY(nf_ref_dh(dt, L->h, L->dp, N, Ha, Wa, F, L->dh));
   NF_TRY(nf_ref_wgrad(dt, act_out, N, Ha, Wa, Co, L->dh, F, 1, L->wpart, L->wpart_floats, g + L->off[NF_P_WA]));
   NF_TRY(nf_ref_channel_sums(dt, L->dh, (size_t)N * Ha * Wa, F, L->red, L->red_floats, &nb));
   NF_TRY(nf_ref_sum_partials(L->red, nb, F, 0, g + L->off[NF_P_BA]));
-  // gradient at the aux input, back through pool / ReLU / BatchNorm
+  // gradient at the aux input
   NF_TRY(nf_ref_conv(dt, L->dh, N, Ha, Wa, F, Wx, (long)F * Co, 1, Co, 1, nullptr, 0, 1, Co, L->da));
+  trace_end();
+  // back through pool / ReLU / BatchNorm
+  trace_begin(5);
   NF_TRY(nf_ref_bn_bwd_reduce(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->red,
                               L->red_floats, &nb));
   NF_TRY(nf_ref_bn_bwd_finalize(L->red, nb, Co, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
   NF_TRY(nf_ref_bn_bwd_apply(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->sdz, L->sdzx,
                              M, L->dy));
+  trace_end();
   // gradient of theta_n (the layer input receives none), then the update
+  trace_begin(6);
   if (L->fam[1]) {
     NF_TRY(nf_tc_wgrad(L, x));
   } else {
     NF_TRY(nf_ref_wgrad(dt, x, N, L->H, L->W, Ci, L->dy, Co, s, L->wpart, L->wpart_floats, g + L->off[NF_P_W]));
   }
+  trace_end();
+  trace_begin(7);
   NF_TRY(nf_ref_sgd(L->val, L->mom, L->grad, L->shadow, L->arena, lr, L->o.momentum));
+  trace_end();
   return NF_OK;
 }
 
@@ -370,6 +427,53 @@ int nf_block_cache_n(nf_block* B, const void* x, void* out, int count) {
 int nf_block_cache(nf_block* B, const void* x, void* out) {
   if (!B) return NF_EINVAL;
   return nf_block_cache_n(B, x, out, B->layers[0]->o.N);
+}
+
+int nf_block_step(nf_block* B, const void* x, const int32_t* labels, float lr, float* loss_out, void* act_out) {
+  if (!B || !x || !labels || !loss_out) return NF_EINVAL;
+  const void* in = x;
+  for (int l = 0; l < B->n; ++l) {
+    nf_layer* L = B->layers[l];
+    void* dst = (l == B->n - 1 && act_out) ? act_out : L->act;
+    g_trace_slot = l < NF_TRACE_SLOTS ? l : NF_TRACE_SLOTS - 1;
+    const int rc = nf_layer_step(L, in, labels, lr, loss_out + l, dst);
+    g_trace_slot = 0;
+    if (rc != NF_OK) return rc;
+    in = dst;
+  }
+  return NF_OK;
+}
+
+int nf_block_step_host(nf_block* B, const void* xh, const int32_t* lh, float lr, float* loss_h, void* act_h) {
+  if (!B || !xh || !lh || !loss_h) return NF_EINVAL;
+  nf_layer* L0 = B->layers[0];
+  nf_layer* Ll = B->layers[B->n - 1];
+  if (!L0->o.host_io || B->n > 64) return NF_EINVAL;
+  const size_t es = nf_esize(L0->o.dtype), N = L0->o.N;
+  NF_CUDA(cudaMemcpyAsync(L0->stage_x, xh, N * L0->H * L0->W * L0->Cin * es, cudaMemcpyHostToDevice, g_nf_stream));
+  NF_CUDA(cudaMemcpyAsync(L0->stage_labels, lh, N * 4, cudaMemcpyHostToDevice, g_nf_stream));
+  NF_TRY(nf_block_step(B, L0->stage_x, L0->stage_labels, lr, L0->stage_loss, nullptr));
+  NF_CUDA(cudaMemcpyAsync(loss_h, L0->stage_loss, 4 * (size_t)B->n, cudaMemcpyDeviceToHost, g_nf_stream));
+  if (act_h)
+    NF_CUDA(cudaMemcpyAsync(act_h, Ll->act, N * Ll->Ha * Ll->Wa * Ll->Cout * es, cudaMemcpyDeviceToHost, g_nf_stream));
+  NF_CUDA(cudaStreamSynchronize(g_nf_stream));
+  return NF_OK;
+}
+
+int nf_trace_enable(int on) {
+  if (trace_flush() != NF_OK) return NF_ECUDA;
+  g_trace_on = on != 0;
+  memset(g_trace_ms, 0, sizeof g_trace_ms);
+  memset(g_trace_cnt, 0, sizeof g_trace_cnt);
+  return NF_OK;
+}
+
+int nf_trace_read(int op, int slot, double* ms_total, long long* groups) {
+  if (op < 0 || op >= NF_TRACE_OPS || slot < 0 || slot >= NF_TRACE_SLOTS || !ms_total || !groups) return NF_EINVAL;
+  if (trace_flush() != NF_OK) return NF_ECUDA;
+  *ms_total = g_trace_ms[op][slot];
+  *groups = g_trace_cnt[op][slot];
+  return NF_OK;
 }
 
 int nf_cache_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count, size_t row_bytes,

@@ -38,6 +38,7 @@ struct nf_layer {
   void* h;                             // [N][Ha][Wa][F] aux conv output after ReLU (dtype)
   void* dh;                            // [N][Ha][Wa][F]
   void* da;                            // [N][Ha][Wa][Cout]
+  void* act;                           // [N][Ha][Wa][Cout] activation kept here when the caller gives no buffer
   float *p, *dp;                       // [N][4F]
   float *logits, *dlogits;             // [N][classes]
   float* lossn;                        // [N]

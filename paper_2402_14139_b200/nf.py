@@ -25,7 +25,8 @@ PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P
 EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_layer_workspace_bytes",
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
-           "nf_block_cache_n", "nf_cache_gather", "nf_partition", "nf_set_stream", "nf_launch_count",
+           "nf_block_cache_n", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
+           "nf_cache_gather", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
 
@@ -68,6 +69,10 @@ def lib():
         L.nf_block_destroy.argtypes = [vp]
         L.nf_block_cache.argtypes = [vp, vp, vp]
         L.nf_block_cache_n.argtypes = [vp, vp, vp, C.c_int]
+        L.nf_block_step.argtypes = [vp, vp, ip, C.c_float, fp, vp]
+        L.nf_block_step_host.argtypes = [vp, vp, ip, C.c_float, fp, vp]
+        L.nf_trace_enable.argtypes = [C.c_int]
+        L.nf_trace_read.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
         L.nf_cache_gather.argtypes = [vp, ip, ip, C.c_int, C.c_size_t, vp, ip]
         L.nf_partition.argtypes = [C.POINTER(C.c_int), C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int),
                                    C.POINTER(C.c_int)]
@@ -116,6 +121,25 @@ def nf_partition(max_batch, B: int, rho: float):
     for i in range(nb):
         last = (first[i + 1] - 1) if i + 1 < nb else n - 1
         out.append((first[i], last, bs[i]))
+    return out
+
+
+TRACE_OPS = ("conv_fwd", "bn_fwd", "aux_fwd", "head", "aux_bwd", "bn_bwd", "wgrad", "sgd")
+
+
+def nf_trace_enable(on: bool):
+    _check(lib().nf_trace_enable(int(on)), "nf_trace_enable")
+
+
+def nf_trace_read(slots: int = 1):
+    """{(op name, layer slot): (total ms, timed groups)} since nf_trace_enable(True); synchronises."""
+    out = {}
+    for i, name in enumerate(TRACE_OPS):
+        for s in range(slots):
+            ms, n = C.c_double(), C.c_longlong()
+            _check(lib().nf_trace_read(i, s, C.byref(ms), C.byref(n)), "nf_trace_read")
+            if n.value:
+                out[(name, s)] = (ms.value, n.value)
     return out
 
 
@@ -209,6 +233,15 @@ class Block:
             _check(lib().nf_block_cache(self.h, _ptr(x), _ptr(out)), "nf_block_cache")
         else:
             _check(lib().nf_block_cache_n(self.h, _ptr(x), _ptr(out), int(count)), "nf_block_cache_n")
+
+    def step(self, x, labels, lr, loss_out, act_out=None):
+        """nf_block_step: loss_out is a float32 device tensor with one entry per layer."""
+        _check(lib().nf_block_step(self.h, _ptr(x), _ptr(labels), float(lr), _ptr(loss_out), _ptr(act_out)),
+               "nf_block_step")
+
+    def step_host(self, x_host, labels_host, lr, loss_host, act_host=None):
+        _check(lib().nf_block_step_host(self.h, _ptr(x_host), _ptr(labels_host), float(lr), _ptr(loss_host),
+                                        _ptr(act_host)), "nf_block_step_host")
 
     def close(self):
         if getattr(self, "h", None):
