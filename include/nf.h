@@ -175,6 +175,21 @@ int nf_block_step_host(nf_block* block, const void* x_host, const int32_t* label
 int nf_cache_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count,
                     size_t row_bytes, void* out, int32_t* out_labels);
 
+/* Stand-alone forms of the two dense contractions of the step (Eq. 1's theta_n x_n and the
+ * gradient of Algorithm 2's line "compute the gradient" with respect to theta_n), for callers that compose
+ * their own step and for kernel-level checks.  All pointers device; activations channels-last of
+ * `dtype`; weights w and the result dw are laid out [kh*3+kw][Cout][Cin] (w of `dtype`, dw float).
+ *   nf_conv3x3_forward: y[n][i][j][co] = sum w[tap][co][ci] * x[n][i*stride+kh-1][j*stride+kw-1][ci], zero padding.
+ *   nf_conv3x3_wgrad:   dw[tap][co][ci] = sum over n,i,j of g[n][i][j][co] * x[n][i*stride+kh-1][j*stride+kw-1][ci];
+ *     needs nf_conv3x3_wgrad_scratch_bytes() of device scratch for its split partial sums (fully
+ *     overwritten, nothing has to be cleared); NF_ENOWS if scratch_bytes is smaller.
+ * Asynchronous on the library's stream. */
+int nf_conv3x3_forward(int dtype, const void* x, const void* w, int N, int H, int W, int Cin, int Cout, int stride,
+                       void* y);
+size_t nf_conv3x3_wgrad_scratch_bytes(int N, int H, int W, int Cin, int Cout, int stride);
+int nf_conv3x3_wgrad(int dtype, const void* x, const void* g, int N, int H, int W, int Cin, int Cout, int stride,
+                     void* scratch, size_t scratch_bytes, float* dw);
+
 /* Algorithm 1 (host only, no device work): given each layer's largest feasible batch size,
  * cap at B and group consecutive layers while |b[i+1]-b[i]| <= rho*b[i]; a block's batch size
  * is the minimum over its members.  Writes up to n_layers entries of first layer index and

@@ -484,6 +484,31 @@ int nf_cache_gather(const void* cache, const int32_t* cache_labels, const int32_
   return nf_ref_gather(cache, cache_labels, idx, count, row_bytes, out, out_labels);
 }
 
+static bool conv_args_ok(int dtype, int N, int H, int W, int Cin, int Cout, int stride) {
+  return (dtype == NF_F32 || dtype == NF_BF16) && N >= 1 && H >= 1 && W >= 1 && Cin >= 1 && Cout >= 1 &&
+         (stride == 1 || stride == 2);
+}
+
+int nf_conv3x3_forward(int dtype, const void* x, const void* w, int N, int H, int W, int Cin, int Cout, int stride,
+                       void* y) {
+  if (!x || !w || !y || !conv_args_ok(dtype, N, H, W, Cin, Cout, stride)) return NF_EINVAL;
+  if (misaligned(x) || misaligned(w) || misaligned(y)) return NF_EALIGN;
+  return nf_ref_conv(dtype, x, N, H, W, Cin, w, (long)Cout * Cin, Cin, 1, 0, nullptr, 0, stride, Cout, y);
+}
+
+size_t nf_conv3x3_wgrad_scratch_bytes(int N, int H, int W, int Cin, int Cout, int stride) {
+  if (!conv_args_ok(NF_F32, N, H, W, Cin, Cout, stride)) return 0;
+  const int Ho = (H - 1) / stride + 1;
+  return (size_t)nf_ref_wgrad_splits(N, Ho, Cin, Cout) * 9 * Cout * Cin * sizeof(float);
+}
+
+int nf_conv3x3_wgrad(int dtype, const void* x, const void* g, int N, int H, int W, int Cin, int Cout, int stride,
+                     void* scratch, size_t scratch_bytes, float* dw) {
+  if (!x || !g || !scratch || !dw || !conv_args_ok(dtype, N, H, W, Cin, Cout, stride)) return NF_EINVAL;
+  if (misaligned(x) || misaligned(g) || misaligned(scratch) || misaligned(dw)) return NF_EALIGN;
+  return nf_ref_wgrad(dtype, x, N, H, W, Cin, g, Cout, stride, (float*)scratch, scratch_bytes / sizeof(float), dw);
+}
+
 int nf_partition(const int* max_batch, int n_layers, int Bcap, double rho, int* block_first, int* block_batch) {
   if (!max_batch || !block_first || !block_batch || n_layers < 1 || Bcap < 1 || !(rho >= 0.0)) return NF_EINVAL;
   std::vector<int> b(n_layers);

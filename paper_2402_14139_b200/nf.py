@@ -26,7 +26,7 @@ EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_laye
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
            "nf_block_cache_n", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
-           "nf_cache_gather", "nf_partition", "nf_set_stream", "nf_launch_count",
+           "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
 
@@ -74,6 +74,10 @@ def lib():
         L.nf_trace_enable.argtypes = [C.c_int]
         L.nf_trace_read.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
         L.nf_cache_gather.argtypes = [vp, ip, ip, C.c_int, C.c_size_t, vp, ip]
+        L.nf_conv3x3_forward.argtypes = [C.c_int, vp, vp] + [C.c_int] * 6 + [vp]
+        L.nf_conv3x3_wgrad_scratch_bytes.restype = C.c_size_t
+        L.nf_conv3x3_wgrad_scratch_bytes.argtypes = [C.c_int] * 6
+        L.nf_conv3x3_wgrad.argtypes = [C.c_int, vp, vp] + [C.c_int] * 6 + [vp, C.c_size_t, vp]
         L.nf_partition.argtypes = [C.POINTER(C.c_int), C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int),
                                    C.POINTER(C.c_int)]
         L.nf_set_stream.argtypes = [vp]
@@ -260,3 +264,22 @@ def nf_cache_gather(cache, cache_labels, idx, out, out_labels):
     row_bytes = cache[0].numel() * cache.element_size()
     _check(lib().nf_cache_gather(_ptr(cache), _ptr(cache_labels), _ptr(idx), int(idx.numel()), row_bytes, _ptr(out),
                                  _ptr(out_labels)), "nf_cache_gather")
+
+
+def nf_conv3x3_forward(dtype, x, w, stride, y):
+    """y = conv3x3(x, w): x [N,H,W,Cin], w [9,Cout,Cin] (both of dtype), y [N,Ho,Wo,Cout]; device tensors."""
+    N, H, W, Cin = x.shape
+    _check(lib().nf_conv3x3_forward(dtype, _ptr(x), _ptr(w), N, H, W, Cin, w.shape[1], stride, _ptr(y)),
+           "nf_conv3x3_forward")
+
+
+def nf_conv3x3_wgrad_scratch_bytes(N, H, W, Cin, Cout, stride) -> int:
+    return int(lib().nf_conv3x3_wgrad_scratch_bytes(N, H, W, Cin, Cout, stride))
+
+
+def nf_conv3x3_wgrad(dtype, x, g, stride, scratch, dw):
+    """dw [9,Cout,Cin] float32 = weight gradient of conv3x3 for input x and output gradient g; scratch is a
+    uint8 device tensor of at least nf_conv3x3_wgrad_scratch_bytes()."""
+    N, H, W, Cin = x.shape
+    _check(lib().nf_conv3x3_wgrad(dtype, _ptr(x), _ptr(g), N, H, W, Cin, g.shape[3], stride, _ptr(scratch),
+                                  scratch.numel(), _ptr(dw)), "nf_conv3x3_wgrad")

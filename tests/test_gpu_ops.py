@@ -1,0 +1,60 @@
+"""GPU parity of the stand-alone contractions (conv forward, weight gradient) against the CPU checker."""
+import numpy as np
+import pytest
+
+from oracle import nfo
+from paper_2402_14139_b200 import synth
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [  # N, Cin, Cout, H, W, stride
+    (2, 3, 5, 9, 7, 1),
+    (3, 20, 33, 12, 10, 2),
+    (2, 64, 64, 32, 32, 1),
+    (2, 64, 128, 16, 16, 2),
+    (1, 128, 64, 8, 24, 1),
+]
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2402_14139_b200 import nf
+    nf.lib()
+    return nf, torch
+
+
+def _case(shape, seed, bf16):
+    N, Ci, Co, H, W, s = shape
+    r = (lambda a: synth.round_bf16(a).astype(np.float64)) if bf16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    x = r(synth.normal(seed, 1, (N, Ci, H, W)))
+    w = r(synth.normal(seed, 2, (Co, Ci, 3, 3), np.sqrt(2.0 / (9 * Ci))))
+    Ho, Wo = nfo.out_size(H, s), nfo.out_size(W, s)
+    g = r(synth.normal(seed, 3, (N, Co, Ho, Wo)))
+    return x, w, g
+
+
+@pytest.mark.parametrize("si", range(len(SHAPES)))
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_conv_forward_and_wgrad(env, si, dtype):
+    nf, torch = env
+    shape = SHAPES[si]
+    N, Ci, Co, H, W, s = shape
+    x, w, g = _case(shape, 300 + si, dtype == 1)
+    tol = pu.TOL[dtype]["t"]
+    td = torch.float32 if dtype == 0 else torch.bfloat16
+    xd = pu.to_device_nhwc(torch, x, dtype)
+    gd = pu.to_device_nhwc(torch, g, dtype)
+    wk = np.ascontiguousarray(np.transpose(w.reshape(Co, Ci, 9), (2, 0, 1)))          # [tap][Cout][Cin]
+    wd = torch.from_numpy(wk.astype(np.float32)).to(device="cuda", dtype=td)
+    yd = torch.empty((N, gd.shape[1], gd.shape[2], Co), device="cuda", dtype=td)
+    nf.nf_conv3x3_forward(dtype, xd, wd, s, yd)
+    assert pu.max_err(pu.from_device_nhwc(yd), nfo.conv3x3(x, w, None, s)) <= tol
+    scratch = torch.empty(nf.nf_conv3x3_wgrad_scratch_bytes(N, H, W, Ci, Co, s), dtype=torch.uint8, device="cuda")
+    dw = torch.empty((9, Co, Ci), device="cuda", dtype=torch.float32)
+    nf.nf_conv3x3_wgrad(dtype, xd, gd, s, scratch, dw)
+    ref = np.transpose(nfo.conv3x3_wgrad(x, g, s).reshape(Co, Ci, 9), (2, 0, 1))
+    assert pu.max_err(dw.cpu().numpy(), ref) <= tol
+    with pytest.raises(nf.NfError):
+        nf.nf_conv3x3_wgrad(dtype, xd, gd, s, scratch[:16], dw)     # scratch too small
