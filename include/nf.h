@@ -190,6 +190,28 @@ size_t nf_conv3x3_wgrad_scratch_bytes(int N, int H, int W, int Cin, int Cout, in
 int nf_conv3x3_wgrad(int dtype, const void* x, const void* g, int N, int H, int W, int Cin, int Cout, int stride,
                      void* scratch, size_t scratch_bytes, float* dw);
 
+/* The same weight gradient for callers that cannot hand over scratch memory.  (The paper has no
+ * counterpart; this is a convenience of this library.)  Some callers are unable to allocate on the
+ * device at the moment they need the gradient: a trainer that has already given its whole memory
+ * budget to activations and caches, as the budgeted setting this method is built for does by
+ * design, or code running where a device allocation's implicit synchronisation is unwelcome.  This
+ * variant keeps the split partial sums in a fixed array inside the library image instead:
+ *  - the array is NF_STATIC_SCRATCH_BYTES (16 MiB) and is held by every GPU that loads the library
+ *    until the process exits;
+ *  - a problem whose nf_conv3x3_wgrad_scratch_bytes() exceeds that is refused with NF_ENOWS and
+ *    nothing is launched;
+ *  - the first call on each device looks up the array's device address (with that device current);
+ *    make that first call before starting any stream capture;
+ *  - all calls share the one array and it keeps whatever the previous call left.  Nothing in it
+ *    has to start at zero (every partial that is read is written first by the same call), but two
+ *    calls that overlap on the GPU (different streams, different host threads) race on it: run
+ *    them one after the other.
+ * It makes no cudaMalloc/cudaFree and calls no allocating routine.  Arguments and result are
+ * those of nf_conv3x3_wgrad without the scratch pair. */
+#define NF_STATIC_SCRATCH_BYTES (16u << 20)
+int nf_conv3x3_wgrad_static(int dtype, const void* x, const void* g, int N, int H, int W, int Cin, int Cout,
+                            int stride, float* dw);
+
 /* Algorithm 1 (host only, no device work): given each layer's largest feasible batch size,
  * cap at B and group consecutive layers while |b[i+1]-b[i]| <= rho*b[i]; a block's batch size
  * is the minimum over its members.  Writes up to n_layers entries of first layer index and

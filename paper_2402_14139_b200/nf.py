@@ -26,7 +26,7 @@ EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_laye
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
            "nf_block_cache_n", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
-           "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_partition", "nf_set_stream", "nf_launch_count",
+           "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
 
@@ -78,6 +78,7 @@ def lib():
         L.nf_conv3x3_wgrad_scratch_bytes.restype = C.c_size_t
         L.nf_conv3x3_wgrad_scratch_bytes.argtypes = [C.c_int] * 6
         L.nf_conv3x3_wgrad.argtypes = [C.c_int, vp, vp] + [C.c_int] * 6 + [vp, C.c_size_t, vp]
+        L.nf_conv3x3_wgrad_static.argtypes = [C.c_int, vp, vp] + [C.c_int] * 6 + [vp]
         L.nf_partition.argtypes = [C.POINTER(C.c_int), C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int),
                                    C.POINTER(C.c_int)]
         L.nf_set_stream.argtypes = [vp]
@@ -283,3 +284,15 @@ def nf_conv3x3_wgrad(dtype, x, g, stride, scratch, dw):
     N, H, W, Cin = x.shape
     _check(lib().nf_conv3x3_wgrad(dtype, _ptr(x), _ptr(g), N, H, W, Cin, g.shape[3], stride, _ptr(scratch),
                                   scratch.numel(), _ptr(dw)), "nf_conv3x3_wgrad")
+
+
+NF_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def nf_conv3x3_wgrad_static(dtype, x, g, stride, dw):
+    """nf_conv3x3_wgrad for callers with no scratch to give: the partial sums go to a 16 MiB array built
+    into the library, so nothing is allocated.  Problems that need more are refused (NfError).  Calls
+    share that array, so do not let two of them overlap on the GPU."""
+    N, H, W, Cin = x.shape
+    _check(lib().nf_conv3x3_wgrad_static(dtype, _ptr(x), _ptr(g), N, H, W, Cin, g.shape[3], stride, _ptr(dw)),
+           "nf_conv3x3_wgrad_static")
