@@ -186,6 +186,8 @@ int nf_cache_gather(const void* cache, const int32_t* cache_labels, const int32_
  * Asynchronous on the library's stream. */
 int nf_conv3x3_forward(int dtype, const void* x, const void* w, int N, int H, int W, int Cin, int Cout, int stride,
                        void* y);
+/* OR of nf_device_flag bits raised by the stand-alone operations since the last call; synchronises. */
+int nf_op_status(void);
 size_t nf_conv3x3_wgrad_scratch_bytes(int N, int H, int W, int Cin, int Cout, int stride);
 int nf_conv3x3_wgrad(int dtype, const void* x, const void* g, int N, int H, int W, int Cin, int Cout, int stride,
                      void* scratch, size_t scratch_bytes, float* dw);

@@ -109,6 +109,8 @@ size_t plan(nf_layer* L, char* base, bool assign) {
   size_t r1 = (size_t)nf_ref_channel_blocks(N * L->Ho * L->Wo, (int)Co) * 2 * Co;
   size_t r2 = (size_t)nf_ref_channel_blocks(N * L->Ha * L->Wa, (int)F) * 2 * F;
   D->red_floats = r1 > r2 ? r1 : r2;
+  const size_t r3 = nf_tc_red_floats(L);
+  if (r3 > D->red_floats) D->red_floats = r3;
   D->red = (float*)c.take(D->red_floats * 4);
   size_t w1 = (size_t)nf_ref_wgrad_splits((int)N, L->Ho, L->Cin, (int)Co) * 9 * Co * L->Cin;
   size_t w2 = (size_t)nf_ref_wgrad_splits((int)N, L->Ha, (int)Co, (int)F) * 9 * F * Co;
@@ -493,6 +495,10 @@ int nf_conv3x3_forward(int dtype, const void* x, const void* w, int N, int H, in
                        void* y) {
   if (!x || !w || !y || !conv_args_ok(dtype, N, H, W, Cin, Cout, stride)) return NF_EINVAL;
   if (misaligned(x) || misaligned(w) || misaligned(y)) return NF_EALIGN;
+  if (dtype == NF_BF16 && stride == 1) {
+    const int rc = nf_tc_conv3x3_forward(x, w, N, H, W, Cin, Cout, y);
+    if (rc != NF_EUNSUPPORTED) return rc;
+  }
   return nf_ref_conv(dtype, x, N, H, W, Cin, w, (long)Cout * Cin, Cin, 1, 0, nullptr, 0, stride, Cout, y);
 }
 
@@ -507,6 +513,12 @@ int nf_conv3x3_wgrad(int dtype, const void* x, const void* g, int N, int H, int 
   if (!x || !g || !scratch || !dw || !conv_args_ok(dtype, N, H, W, Cin, Cout, stride)) return NF_EINVAL;
   if (misaligned(x) || misaligned(g) || misaligned(scratch) || misaligned(dw)) return NF_EALIGN;
   return nf_ref_wgrad(dtype, x, N, H, W, Cin, g, Cout, stride, (float*)scratch, scratch_bytes / sizeof(float), dw);
+}
+
+int nf_op_status(void) {
+  int32_t v = 0;
+  const int rc = nf_tc_op_status(&v);
+  return rc == NF_OK ? (int)v : rc;
 }
 
 int nf_partition(const int* max_batch, int n_layers, int Bcap, double rho, int* block_first, int* block_batch) {

@@ -1,9 +1,380 @@
-// Tensor-core convolution kernels (placeholder selection: everything on the CUDA-core family).
+// Tensor-core convolution kernels for sm_100a: implicit GEMM on tcgen05.mma with accumulators in
+// tensor memory, operands staged in shared memory by TMA, warp-specialised persistent CTAs.
+//
+// Forward (Eq. 1's theta_n x_n, stride 1, Cin and Cout multiples of 64):
+//   GEMM view  D[pixel, co] = sum_{tap, ci} X[pixel shifted by tap, ci] * W[tap][co][ci]
+//   M tile = 128 output pixels = a BW x BH patch of one image, N tile = BN output channels,
+//   K loop  = (Cin/64 channel chunks) x (3 column taps kw); for each such step ONE TMA box of
+//   (BH+2) rows x BW pixels x 64 channels lands in shared memory (zero fill outside the image is
+//   the padding) and serves the three row taps kh = 0,1,2 by advancing the operand descriptor by
+//   kh rows, so the input is fetched 3(BH+2)/BH times from L2 instead of 9 times.
+//   Epilogue: TMEM -> registers -> bf16 -> swizzled shared tile -> TMA store of y; the per-channel
+//   sum and sum of squares of the stored (rounded) values are accumulated per CTA for BatchNorm.
+#include <cuda.h>
+
+#include "nf_ptx.cuh"
 #include "nf_tc.h"
 
-void nf_tc_select(nf_layer* L) { L->fam[0] = L->fam[1] = L->fam[2] = L->fam[3] = 0; }
+namespace {
+
+constexpr int kThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
+constexpr int kMaxStages = 8;
+
+struct FwdParams {
+  int N, H, W, Cin, Cout;
+  int BW, BH, tiles_w, tiles_h, n_tiles, total_tiles, kchunks, stages;
+  int stats;
+  float* red;       // [grid * parts][2][Cout] channel partials (pre-zeroed)
+  int32_t* status;  // device status word
+};
+
+struct TcPlan {
+  int ok, BW, BH, BN, stages, grid, parts;
+  size_t smem;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+                   const __grid_constant__ CUtensorMap tm_y, const FwdParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int a_bytes = (p.BH + 2) * p.BW * 128;
+  constexpr int b_bytes = 3 * BN * 128;
+  const int stage_bytes = a_bytes + b_bytes;
+  constexpr int kSub = BN / 64;  // 64-channel sub-tiles of the output staging
+  uint8_t* stg = smem + (size_t)p.stages * stage_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + kSub * 16384);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + kMaxStages;
+  uint64_t* tfull = bars + 2 * kMaxStages;
+  uint64_t* tempty = tfull + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ksteps = 3 * p.kchunks;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(&tfull[a], 1);
+      ptx::mbar_init(&tempty[a], 128);
+    }
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tmap(&tm_x);
+    ptx::prefetch_tmap(&tm_w);
+    ptx::prefetch_tmap(&tm_y);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, 2 * BN);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- producer: one TMA box of activations + three weight tiles per k-step
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x) {
+      const int nt = t % p.n_tiles, m = t / p.n_tiles;
+      const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = m / (p.tiles_w * p.tiles_h);
+      for (int ks = 0; ks < ksteps; ++ks, ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) { ok = false; break; }
+        if (lane == 0) {
+          const int kw = ks % 3, ck = ks / 3;
+          uint8_t* a_s = smem + (size_t)s * stage_bytes;
+          ptx::mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
+          ptx::tma_load_4d(a_s, &tm_x, &full[s], ck * 64, w0 + kw - 1, h0 - 1, n);
+          ptx::tma_load_4d(a_s + a_bytes, &tm_w, &full[s], ck * 64, nt * BN, kw, 0);
+        }
+        __syncwarp();
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    constexpr uint32_t idesc = ptx::idesc_bf16(128, BN, 0, 0);
+    uint32_t it = 0, tl = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++tl) {
+      const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&tempty[acc], aph ^ 1, abort_flag))) break;
+      ptx::tc_fence_after();
+      const uint32_t d = tmem_base + acc * BN;
+      for (int ks = 0; ks < ksteps; ++ks, ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[s], ph, abort_flag))) { ok = false; break; }
+        ptx::tc_fence_after();
+        if (lane == 0) {
+          const uint32_t a_base = ptx::smem_u32(smem + (size_t)s * stage_bytes);
+          const uint32_t b_base = a_base + a_bytes;
+#pragma unroll
+          for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const uint64_t ad = ptx::sdesc_sw128(a_base + kh * p.BW * 128 + k * 32, 16, 1024);
+              const uint64_t bd = ptx::sdesc_sw128(b_base + kh * BN * 128 + k * 32, 16, 1024);
+              ptx::mma_f16(d, ad, bd, idesc, (ks | kh | k) != 0);
+            }
+          ptx::mma_commit(&empty[s]);
+        }
+        __syncwarp();
+      }
+      if (ok && lane == 0) ptx::mma_commit(&tfull[acc]);
+      __syncwarp();
+    }
+  } else {
+    // ---------------- epilogue: 128 threads, thread <-> output pixel (TMEM lane)
+    const int et = threadIdx.x - 64;
+    const int lg = warp & 3;          // TMEM lane group this warp may read
+    const int r = lg * 32 + lane;     // row of the tile = pixel (r % BW, r / BW)
+    constexpr int kRowsPer = BN >= 128 ? 128 : 64;  // rows each thread sums for its channel
+    const int sc = et % BN, shalf = et / BN;        // stats: channel and row half of this thread
+    float ssum = 0.f, ssq = 0.f;
+    uint32_t tl = 0;
+    int my_nt = blockIdx.x % p.n_tiles;
+    for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++tl) {
+      const int nt = t % p.n_tiles, m = t / p.n_tiles;
+      const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = m / (p.tiles_w * p.tiles_h);
+      const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+      ptx::mbar_wait(&tfull[acc], aph, abort_flag);  // sets the abort flag itself when it gives up
+      ptx::tc_fence_after();
+      if (et == 0) {
+        ptx::tma_store_wait_read();  // the previous tile's store has finished reading the staging tile
+        *epi_go = *abort_flag ? 0 : 1;  // one thread decides for all 128, so nobody is left alone at a barrier
+      }
+      ptx::named_barrier(1, 128);
+      if (!*epi_go) break;
+#pragma unroll
+      for (int j = 0; j < BN / 32; ++j) {
+        uint32_t v[32];
+        ptx::tmem_ld32(tmem_base + ((uint32_t)(lg * 32) << 16) + acc * BN + j * 32, v);
+        ptx::tmem_ld_wait();
+        uint8_t* sub = stg + ((j * 32) / 64) * 16384 + r * 128;
+        const int u0 = ((j * 32) % 64) / 8;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[q * 8 + 2 * e]), __uint_as_float(v[q * 8 + 2 * e + 1]));
+            w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+          }
+          *reinterpret_cast<uint4*>(sub + (((u0 + q) ^ (r & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&tempty[acc]);
+      ptx::fence_async_smem();
+      ptx::named_barrier(1, 128);
+      if (et == 0) {
+#pragma unroll
+        for (int sb = 0; sb < kSub; ++sb) ptx::tma_store_4d(&tm_y, stg + sb * 16384, nt * BN + sb * 64, w0, h0, n);
+        ptx::tma_store_commit();
+      }
+      if (p.stats) {
+        const uint8_t* col = stg + (sc / 64) * 16384 + (sc % 8) * 2;
+        const int u = (sc % 64) / 8;
+        const int rb = shalf * kRowsPer;
+#pragma unroll 8
+        for (int rr = 0; rr < kRowsPer; ++rr) {
+          const int row = rb + rr;
+          const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(col + row * 128 + ((u ^ (row & 7)) * 16)));
+          ssum += v;
+          ssq = fmaf(v, v, ssq);
+        }
+      }
+    }
+    if (et == 0) ptx::tma_store_wait_all();
+    if (p.stats) {
+      constexpr int parts = 128 / BN > 0 ? 128 / BN : 1;
+      const size_t b = (size_t)blockIdx.x * parts + shalf;
+      p.red[(b * 2 + 0) * p.Cout + my_nt * BN + sc] = ssum;
+      p.red[(b * 2 + 1) * p.Cout + my_nt * BN + sc] = ssq;
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(p.status, NF_ETIMEOUT);
+    // give copies still in flight time to land before the shared memory is released
+    const unsigned long long t0 = ptx::globaltimer();
+    while (ptx::globaltimer() - t0 < 2000000ull) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, 2 * BN);
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor, 4 dims (innermost first), 128-byte swizzle, zero fill outside
+int make_map4(CUtensorMap* m, const void* base, const uint64_t dims[4], const uint32_t box[4]) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return NF_ECUDA;
+  cuuint64_t gdim[4] = {dims[0], dims[1], dims[2], dims[3]};
+  cuuint64_t gstr[3] = {dims[0] * 2, dims[0] * dims[1] * 2, dims[0] * dims[1] * dims[2] * 2};
+  cuuint32_t bx[4] = {box[0], box[1], box[2], box[3]};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gdim, gstr, bx, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? NF_OK : nf_cuda_check(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+}
+
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      n = 148;
+  }
+  return n;
+}
+
+TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N) {
+  TcPlan pl{};
+  if (Cin % 64 || Cout % 64) return pl;
+  const int cand[3][2] = {{16, 8}, {32, 4}, {8, 16}};
+  for (auto& c : cand)
+    if (W % c[0] == 0 && H % c[1] == 0) {
+      pl.BW = c[0];
+      pl.BH = c[1];
+      break;
+    }
+  if (!pl.BW) return pl;
+  pl.BN = Cout % 128 == 0 ? 128 : 64;
+  const size_t stage = (size_t)(pl.BH + 2) * pl.BW * 128 + 3 * pl.BN * 128;
+  const size_t fixed = (size_t)(pl.BN / 64) * 16384 + 1024 + 1024;  // staging + barriers + alignment slack
+  int st = (int)((232448 - fixed) / stage);
+  if (st > kMaxStages) st = kMaxStages;
+  if (st < 2) return pl;
+  pl.stages = st;
+  pl.smem = (size_t)st * stage + fixed;
+  pl.parts = pl.BN >= 128 ? 1 : 128 / pl.BN;
+  const int n_tiles = Cout / pl.BN;
+  const long total = (long)N * (H / pl.BH) * (W / pl.BW) * n_tiles;
+  long g = sm_count();
+  g -= g % n_tiles;  // every CTA keeps one channel tile for its whole life
+  if (g < n_tiles) g = n_tiles;
+  if (g > total) g = total;
+  pl.grid = (int)g;
+  pl.ok = 1;
+  return pl;
+}
+
+template <int BN>
+int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const FwdParams& p) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    NF_CUDA(cudaFuncSetAttribute(conv_fwd_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    attr_done = true;
+  }
+  conv_fwd_tc_kernel<BN><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mw, my, p);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int run_fwd(int N, int H, int W, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
+            size_t red_floats, int32_t* status, int* nb) {
+  const TcPlan pl = plan_fwd(H, W, Cin, Cout, N);
+  if (!pl.ok) return NF_EUNSUPPORTED;
+  CUtensorMap mx, mw, my;
+  const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
+  const uint32_t bx[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH + 2, 1};
+  const uint64_t dw[4] = {(uint64_t)Cin, (uint64_t)Cout, 3, 3};
+  const uint32_t bw[4] = {64, (uint32_t)pl.BN, 1, 3};
+  const uint64_t dy[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
+  const uint32_t by[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH, 1};
+  int rc;
+  if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
+  if ((rc = make_map4(&mw, w, dw, bw)) != NF_OK) return rc;
+  if ((rc = make_map4(&my, y, dy, by)) != NF_OK) return rc;
+  FwdParams p{};
+  p.N = N; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout;
+  p.BW = pl.BW; p.BH = pl.BH; p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.n_tiles = Cout / pl.BN;
+  p.total_tiles = N * p.tiles_h * p.tiles_w * p.n_tiles;
+  p.kchunks = Cin / 64; p.stages = pl.stages; p.stats = stats; p.red = red; p.status = status;
+  if (stats) {
+    const size_t need = (size_t)pl.grid * pl.parts * 2 * Cout;
+    if (need > red_floats) return NF_ENOWS;
+    NF_CUDA(cudaMemsetAsync(red, 0, need * sizeof(float), g_nf_stream));
+    *nb = pl.grid * pl.parts;
+  }
+  return pl.BN == 128 ? launch_fwd<128>(pl, mx, mw, my, p) : launch_fwd<64>(pl, mx, mw, my, p);
+}
+
+}  // namespace
+
+void nf_tc_select(nf_layer* L) {
+  L->fam[0] = L->fam[1] = L->fam[2] = L->fam[3] = 0;
+  if (L->o.dtype != NF_BF16) return;
+  if (L->o.stride == 1 && plan_fwd(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[0] = 1;
+}
+
 size_t nf_tc_scratch_floats(const nf_layer*) { return 0; }
+
+size_t nf_tc_red_floats(const nf_layer* L) {
+  if (!L->fam[0]) return 0;
+  const TcPlan pl = plan_fwd(L->H, L->W, L->Cin, L->Cout, L->o.N);
+  return (size_t)sm_count() * pl.parts * 2 * L->Cout;
+}
+
 int nf_tc_prepare(nf_layer*) { return NF_OK; }
-int nf_tc_conv_fwd(nf_layer*, const void*, int&) { return NF_EUNSUPPORTED; }
-int nf_tc_conv_fwd_eval(nf_layer*, const void*, int) { return NF_EUNSUPPORTED; }
+
+int nf_tc_conv_fwd(nf_layer* L, const void* x, int& nb) {
+  return run_fwd(L->o.N, L->H, L->W, L->Cin, L->Cout, x, L->shadow + L->off[NF_P_W], L->y, 1, L->red, L->red_floats,
+                 L->status, &nb);
+}
+
+int nf_tc_conv_fwd_eval(nf_layer* L, const void* x, int count) {
+  int nb = 0;
+  return run_fwd(count, L->H, L->W, L->Cin, L->Cout, x, L->shadow + L->off[NF_P_W], L->y, 0, nullptr, 0, L->status, &nb);
+}
+
 int nf_tc_wgrad(nf_layer*, const void*) { return NF_EUNSUPPORTED; }
+
+static __device__ int32_t g_op_status;  // status word of the stand-alone operations
+
+int nf_tc_conv3x3_forward(const void* x, const void* w, int N, int H, int W, int Cin, int Cout, void* y) {
+  static int32_t* st = nullptr;
+  if (!st) NF_CUDA(cudaGetSymbolAddress((void**)&st, g_op_status));
+  int nb = 0;
+  return run_fwd(N, H, W, Cin, Cout, x, w, y, 0, nullptr, 0, st, &nb);
+}
+
+int nf_tc_op_status(int32_t* out) {
+  NF_CUDA(cudaStreamSynchronize(g_nf_stream));
+  NF_CUDA(cudaMemcpyFromSymbol(out, g_op_status, sizeof(int32_t)));
+  const int32_t zero = 0;
+  NF_CUDA(cudaMemcpyToSymbol(g_op_status, &zero, sizeof(int32_t)));
+  return NF_OK;
+}

@@ -14,3 +14,9 @@ int nf_tc_conv_fwd(nf_layer* L, const void* x, int& nb);
 int nf_tc_conv_fwd_eval(nf_layer* L, const void* x, int count);
 // grad(W) = wgrad(x, L->dy) into the gradient arena.
 int nf_tc_wgrad(nf_layer* L, const void* x);
+// Floats of channel-partial scratch (L->red) the tensor-core forward needs.
+size_t nf_tc_red_floats(const nf_layer* L);
+// Stand-alone forward on the tensor-core path (NF_EUNSUPPORTED if the shape is not covered) and the
+// status word (nf_device_flag bits) of the stand-alone operations.
+int nf_tc_conv3x3_forward(const void* x, const void* w, int N, int H, int W, int Cin, int Cout, void* y);
+int nf_tc_op_status(int32_t* out);

@@ -26,7 +26,7 @@ EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_laye
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
            "nf_block_cache_n", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
-           "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_partition", "nf_set_stream", "nf_launch_count",
+           "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_op_status", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
 
@@ -296,3 +296,10 @@ def nf_conv3x3_wgrad_static(dtype, x, g, stride, dw):
     N, H, W, Cin = x.shape
     _check(lib().nf_conv3x3_wgrad_static(dtype, _ptr(x), _ptr(g), N, H, W, Cin, g.shape[3], stride, _ptr(dw)),
            "nf_conv3x3_wgrad_static")
+
+
+def nf_op_status() -> int:
+    rc = lib().nf_op_status()
+    if rc < 0:
+        _check(rc, "nf_op_status")
+    return rc

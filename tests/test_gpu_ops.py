@@ -14,6 +14,10 @@ SHAPES = [  # N, Cin, Cout, H, W, stride
     (2, 64, 64, 32, 32, 1),
     (2, 64, 128, 16, 16, 2),
     (1, 128, 64, 8, 24, 1),
+    (2, 128, 128, 32, 32, 1),   # tensor-core forward: two channel chunks, 128-wide channel tile
+    (1, 64, 64, 64, 48, 1),     # tensor-core forward: 16x8 pixel tiles, several tiles per CTA row
+    (3, 64, 192, 8, 32, 1),     # tensor-core forward: 32x4 pixel tiles, three 64-wide channel tiles
+    (1, 64, 64, 16, 8, 1),      # tensor-core forward: 8x16 pixel tiles, a single tile
 ]
 
 
@@ -51,6 +55,7 @@ def test_conv_forward_and_wgrad(env, si, dtype):
     yd = torch.empty((N, gd.shape[1], gd.shape[2], Co), device="cuda", dtype=td)
     nf.nf_conv3x3_forward(dtype, xd, wd, s, yd)
     assert pu.max_err(pu.from_device_nhwc(yd), nfo.conv3x3(x, w, None, s)) <= tol
+    assert nf.nf_op_status() == 0
     scratch = torch.empty(nf.nf_conv3x3_wgrad_scratch_bytes(N, H, W, Ci, Co, s), dtype=torch.uint8, device="cuda")
     dw = torch.empty((9, Co, Ci), device="cuda", dtype=torch.float32)
     nf.nf_conv3x3_wgrad(dtype, xd, gd, s, scratch, dw)

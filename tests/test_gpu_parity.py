@@ -116,3 +116,23 @@ def test_step_host_matches_device_step(env):
     assert float(loss_h.item()) == float(loss_a.item())
     assert torch.equal(act_h, act_a.cpu())
     assert np.array_equal(A.get_param("W"), B.get_param("W"))
+
+
+# shapes the tcgen05 kernels cover (bf16, channel counts multiples of 64, tileable image sizes)
+TC = [
+    dict(N=4, Cin=64, Cout=64, H=32, W=32, F=16, classes=10, stride=1, pool=False),
+    dict(N=2, Cin=128, Cout=128, H=16, W=16, F=16, classes=10, stride=1, pool=True),
+    dict(N=3, Cin=64, Cout=128, H=16, W=32, F=8, classes=20, stride=1, pool=False),
+]
+
+
+@pytest.mark.parametrize("ci", range(len(TC)))
+def test_tensor_core_shapes_bf16(env, ci):
+    nf, torch = env
+    c = TC[ci]
+    P, x, y = pu.seeded_case(c, 1, bf16=True)
+    G = pu.gpu_layer(nf, c, P, nf.NF_BF16)
+    assert G.kernel_family(0) == "tcgen05"
+    G.close()
+    w = pu.check_step(nf, torch, c, seed=400 + ci, dtype=nf.NF_BF16, lr=0.02, steps=2)
+    print(w)
