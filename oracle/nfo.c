@@ -288,9 +288,12 @@ void nfo_sgd(double* theta, double* v, const double* g, size_t n, double lr, dou
 typedef struct {
   int N, Cin, Cout, H, W, stride, pool, F, classes;
   double eps, momentum, bn_momentum;
-  int store_bf16; /* 1: the two tensors the method keeps in bfloat16 (conv output y, activation x_{n+1}) are
-                     rounded to bfloat16 where they are stored, so that every decision taken from them (ReLU
-                     masks, pool argmax) is taken in the storage precision; all arithmetic stays fp64 */
+  int store_bf16; /* 1: bf16 configuration ("bf16 operands, wider accumulate").  The two tensors the method keeps
+                     in bfloat16 (conv output y, activation x_{n+1}) are rounded to bfloat16 where they are
+                     stored, so that every decision taken from them (ReLU masks, pool argmax) is taken in the
+                     storage precision, and the two convolutions read bfloat16 copies of their weights W and
+                     Wa (the master weights, their momentum and their update stay unrounded; the gradient of
+                     the copy is applied to the master).  All arithmetic stays fp64. */
 } nfo_dims;
 
 /* Round to the nearest bfloat16, ties to even (via float, as a bf16 store of an fp32 value does). */
@@ -348,8 +351,15 @@ double nfo_layer_step(const nfo_dims* d, const double* x, const int32_t* labels,
   double *gW = dalloc((size_t)Co * Ci * 9), *gg = dalloc(Co), *gb = dalloc(Co);
   double *gWa = dalloc((size_t)F * Co * 9), *gba = dalloc(F), *gWf = dalloc((size_t)K * D), *gbf = dalloc(K);
 
+  /* operand copies of the conv weights (bfloat16 in the bf16 configuration) */
+  double *Wq = dalloc((size_t)Co * Ci * 9), *Waq = dalloc((size_t)F * Co * 9);
+  memcpy(Wq, P->W, sizeof(double) * (size_t)Co * Ci * 9);
+  memcpy(Waq, P->Wa, sizeof(double) * (size_t)F * Co * 9);
+  store_round(Wq, (size_t)Co * Ci * 9, d->store_bf16);
+  store_round(Waq, (size_t)F * Co * 9, d->store_bf16);
+
   /* forward: Eq. 1 */
-  nfo_conv3x3(x, N, Ci, H, W, P->W, Co, NULL, s, y);
+  nfo_conv3x3(x, N, Ci, H, W, Wq, Co, NULL, s, y);
   store_round(y, ny, d->store_bf16);
   nfo_bn_train(y, N, Co, Ho * Wo, P->gamma, P->beta, d->eps, mu, var, xhat, z);
   nfo_relu(z, ny, r);
@@ -358,7 +368,7 @@ double nfo_layer_step(const nfo_dims* d, const double* x, const int32_t* labels,
   else memcpy(a, r, ny * sizeof(double));
   if (act_out) memcpy(act_out, a, na * sizeof(double));
   /* auxiliary network: Eq. 2 */
-  nfo_conv3x3(a, N, Co, Ha, Wa, P->Wa, F, P->ba, 1, hpre);
+  nfo_conv3x3(a, N, Co, Ha, Wa, Waq, F, P->ba, 1, hpre);
   nfo_relu(hpre, nh, h);
   nfo_avgpool_2x2(h, N, F, Ha, Wa, p);
   nfo_fc(p, N, D, P->Wf, P->bf, K, logits);
@@ -392,7 +402,7 @@ double nfo_layer_step(const nfo_dims* d, const double* x, const int32_t* labels,
       for (int k = 0; k < Ha * Wa; ++k) sb += dh[((size_t)n * F + f) * Ha * Wa + k];
     gba[f] = sb;
   }
-  nfo_conv3x3_dgrad(P->Wa, Co, F, dh, N, Ha, Wa, 1, da);
+  nfo_conv3x3_dgrad(Waq, Co, F, dh, N, Ha, Wa, 1, da);
   /* back through down-sampling and ReLU to the BatchNorm output */
   if (d->pool) {
     for (int n = 0; n < N; ++n)
@@ -436,6 +446,7 @@ double nfo_layer_step(const nfo_dims* d, const double* x, const int32_t* labels,
     }
   }
 
+  free(Wq); free(Waq);
   free(y); free(xhat); free(z); free(r); free(a); free(mu); free(var); free(arg);
   free(hpre); free(h); free(p); free(logits); free(dlogits); free(dp); free(dh); free(da);
   free(dr); free(dz); free(dy); free(gW); free(gg); free(gb); free(gWa); free(gba); free(gWf); free(gbf);
@@ -449,7 +460,11 @@ void nfo_layer_eval(const nfo_dims* d, const double* x, const nfo_params* P, dou
   const int Ho = nfo_out_size(d->H, s), Wo = nfo_out_size(d->W, s);
   const size_t ny = (size_t)N * Co * Ho * Wo;
   double *y = dalloc(ny), *z = dalloc(ny), *r = dalloc(ny);
-  nfo_conv3x3(x, N, d->Cin, d->H, d->W, P->W, Co, NULL, s, y);
+  double* Wq = dalloc((size_t)Co * d->Cin * 9);
+  memcpy(Wq, P->W, sizeof(double) * (size_t)Co * d->Cin * 9);
+  store_round(Wq, (size_t)Co * d->Cin * 9, d->store_bf16);
+  nfo_conv3x3(x, N, d->Cin, d->H, d->W, Wq, Co, NULL, s, y);
+  free(Wq);
   store_round(y, ny, d->store_bf16);
   nfo_bn_eval(y, N, Co, Ho * Wo, P->gamma, P->beta, d->eps, P->rmean, P->rvar, z);
   nfo_relu(z, ny, r);

@@ -190,7 +190,9 @@ def test_bf16_rounding_ties_to_even():
 def test_bf16_storage_mode_rounds_only_the_stored_tensors():
     c = CASES[2]
     L, x, y = make_layer(c, 21)
+    L.set(W=synth.round_bf16(L.p["W"]), Wa=synth.round_bf16(L.p["Wa"]))   # bf16-valued conv weights on both
     Lb, _, _ = make_layer(c, 21)
+    Lb.set(W=L.p["W"], Wa=L.p["Wa"])
     Lb.d.store_bf16 = 1
     loss, act, tr = L.step(x, y, 0.0, update=False, trace=True)
     loss_b, act_b, tr_b = Lb.step(x, y, 0.0, update=False, trace=True)
@@ -202,6 +204,19 @@ def test_bf16_storage_mode_rounds_only_the_stored_tensors():
     # the rounding is a small perturbation of the exact step (bf16 has 8 significand bits)
     assert np.abs(tr_b["y"] - tr["y"]).max() <= 2.0 ** -8 * np.abs(tr["y"]).max()
     assert abs(loss_b - loss) <= 1e-2 * abs(loss)
+    # conv weights are read through bfloat16 copies: masters with bf16 values give the same step as the
+    # default mode does once y and a are rounded; masters themselves are never rounded by the update
+    Lm, _, _ = make_layer(c, 21)
+    Lm.set(W=synth.round_bf16(Lm.p["W"]), Wa=synth.round_bf16(Lm.p["Wa"]))
+    Lq, _, _ = make_layer(c, 21)
+    Lq.set(W=synth.round_bf16(Lq.p["W"]), Wa=synth.round_bf16(Lq.p["Wa"]))
+    Lq.d.store_bf16 = 1
+    Lb2, _, _ = make_layer(c, 21)
+    Lb2.d.store_bf16 = 1
+    l_q, a_q, _ = Lq.step(x, y, 0.1, update=True)
+    l_b2, a_b2, _ = Lb2.step(x, y, 0.1, update=True)
+    assert l_q == l_b2 and np.array_equal(a_q, a_b2)          # rounding the operand copy == rounded masters
+    assert not np.array_equal(Lb2.p["W"], synth.round_bf16(Lb2.p["W"]).astype(np.float64))  # masters stay unrounded
     # the scalar rounding routine agrees with a library conversion, ties to even included
     v = np.array([1.0, 1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, -2.5, 3.14159, 1e-20, 65504.0, 0.0])
     got = np.array([nfo.lib().nfo_round_bf16(float(t)) for t in v])
