@@ -121,7 +121,7 @@ def test_step_host_matches_device_step(env):
 # shapes the tcgen05 kernels cover (bf16, channel counts multiples of 64, tileable image sizes)
 TC = [
     dict(N=4, Cin=64, Cout=64, H=32, W=32, F=16, classes=10, stride=1, pool=False),
-    dict(N=2, Cin=128, Cout=128, H=16, W=16, F=16, classes=10, stride=1, pool=True),
+    dict(N=6, Cin=128, Cout=128, H=16, W=16, F=16, classes=10, stride=1, pool=True),
     dict(N=3, Cin=64, Cout=128, H=16, W=32, F=8, classes=20, stride=1, pool=False),
 ]
 
