@@ -219,6 +219,165 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   }
 }
 
+
+// ---------------------------------------------------------------- weight gradient
+// dW[tap][co][ci] = sum over pixels of dy[pixel, co] * x[pixel shifted by tap, ci]  (stride 1).
+// GEMM view per 64-channel block pair (ci chunk, co chunk): the K dimension is the pixel index, so
+// both operands are MN-major in shared memory exactly as TMA delivers the channels-last tiles:
+//   A (M = 128 rows) = two stacked (tap, 64 input channels) chunks taken from the three
+//       column-shifted activation boxes; the second chunk sits one leading-dimension offset away
+//       (BW rows for the next row tap, or one box for the next column tap),
+//   B (N = 64)       = the dy tile of the 64 output channels,
+//   K                = 16 pixels per instruction, 128 pixels per pipeline stage.
+// Five instructions per 16 pixels cover the nine taps (the last one half empty); their five
+// 128 x 64 accumulators stay in tensor memory over the CTA's whole pixel range (split-K); at the
+// end they are written to a per-CTA partial that a second kernel sums in a fixed order.
+struct WgParams {
+  int N, H, W, Cin, Cout;
+  int BW, BH, tiles_w, tiles_h, pix_tiles, ci_chunks, co_chunks, splits;
+  float* part;      // [splits][9][Cout][Cin]
+  int32_t* status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_dy, const WgParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr int kStages = 2;
+  const int copy_bytes = (p.BH + 2) * p.BW * 128;
+  const int stage_bytes = 3 * copy_bytes + 16384;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * stage_bytes);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + kStages;
+  uint64_t* done = bars + 2 * kStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  constexpr uint32_t kCols = 512;  // 5 accumulators x 64 columns, rounded up to a power of two
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int blocks = p.ci_chunks * p.co_chunks;
+  const int blk = blockIdx.x % blocks, sp = blockIdx.x / blocks;
+  const int cic = blk % p.ci_chunks, coc = blk / p.ci_chunks;
+  const int t0 = (int)((long)p.pix_tiles * sp / p.splits), t1 = (int)((long)p.pix_tiles * (sp + 1) / p.splits);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    ptx::mbar_init(done, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tmap(&tm_x);
+    ptx::prefetch_tmap(&tm_dy);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    uint32_t it = 0;
+    for (int t = t0; t < t1; ++t, ++it) {
+      const int s = it % kStages;
+      const uint32_t ph = (it / kStages) & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) break;
+      if (lane == 0) {
+        const int w0 = (t % p.tiles_w) * p.BW, h0 = ((t / p.tiles_w) % p.tiles_h) * p.BH, n = t / (p.tiles_w * p.tiles_h);
+        uint8_t* st = smem + (size_t)s * stage_bytes;
+        ptx::mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
+#pragma unroll
+        for (int kw = 0; kw < 3; ++kw) ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, w0 + kw - 1, h0 - 1, n);
+        ptx::tma_load_4d(st + 3 * copy_bytes, &tm_dy, &full[s], coc * 64, w0, h0, n);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    constexpr uint32_t idesc = ptx::idesc_bf16(128, 64, 1, 1);
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = t0; t < t1; ++t, ++it) {
+      const int s = it % kStages;
+      const uint32_t ph = (it / kStages) & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[s], ph, abort_flag))) { ok = false; break; }
+      ptx::tc_fence_after();
+      if (lane == 0) {
+        const uint32_t xb = ptx::smem_u32(smem + (size_t)s * stage_bytes);
+        const uint32_t gb = xb + 3 * copy_bytes;
+        const uint32_t row = p.BW * 128;  // bytes of one image row of the box
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint32_t koff = k * 16 * 128;  // 16 pixels per instruction
+          const uint64_t bd = ptx::sdesc_sw128(gb + koff, 16, 1024);
+          const uint32_t acc = (it | k) != 0;
+#pragma unroll
+          for (int kw = 0; kw < 3; ++kw)  // taps (kh=0,kw) and (kh=1,kw): second chunk one image row further
+            ptx::mma_f16(tmem_base + kw * 64, ptx::sdesc_sw128(xb + kw * copy_bytes + koff, row, 1024), bd, idesc, acc);
+          // taps (kh=2,kw=0) and (kh=2,kw=1): second chunk one box further
+          ptx::mma_f16(tmem_base + 192, ptx::sdesc_sw128(xb + 2 * row + koff, copy_bytes, 1024), bd, idesc, acc);
+          // tap (kh=2,kw=2); rows 64..127 of this accumulator are not used (their operand rows fall on the
+          // rows after the box, which are still inside this stage's buffer)
+          ptx::mma_f16(tmem_base + 256, ptx::sdesc_sw128(xb + 2 * copy_bytes + 2 * row + koff, row, 1024), bd, idesc, acc);
+        }
+        ptx::mma_commit(&empty[s]);
+      }
+      __syncwarp();
+    }
+    if (ok && lane == 0) ptx::mma_commit(done);
+    __syncwarp();
+  } else {
+    // epilogue: after the last MMA, lane m of tensor memory = row m of the stacked (tap, ci) chunks
+    const int lg = warp & 3, m = lg * 32 + lane;
+    if (ptx::mbar_wait(done, 0, abort_flag) && t1 > t0) {
+      ptx::tc_fence_after();
+      const size_t plane = (size_t)p.Cout * p.Cin;
+      float* base = p.part + (size_t)sp * 9 * plane + (size_t)(coc * 64) * p.Cin + cic * 64 + (m & 63);
+#pragma unroll 1
+      for (int j = 0; j < 5; ++j) {
+        // taps of accumulator j: rows 0..63 -> tapA, rows 64..127 -> tapB (kh*3+kw)
+        const int tapA = j < 3 ? j : (j == 3 ? 6 : 8);
+        const int tapB = j < 3 ? 3 + j : (j == 3 ? 7 : -1);
+        const int tap = m < 64 ? tapA : tapB;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          uint32_t v[32];
+          ptx::tmem_ld32(tmem_base + ((uint32_t)(lg * 32) << 16) + j * 64 + q * 32, v);
+          ptx::tmem_ld_wait();
+          if (tap >= 0) {
+            float* dst = base + (size_t)tap * plane + (size_t)(q * 32) * p.Cin;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) dst[(size_t)e * p.Cin] = __uint_as_float(v[e]);
+          }
+        }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(p.status, NF_ETIMEOUT);
+    const unsigned long long tt = ptx::globaltimer();
+    while (ptx::globaltimer() - tt < 2000000ull) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kCols);
+  }
+}
+
+__global__ void sum_parts_kernel(const float* __restrict__ part, int splits, size_t n, float* __restrict__ out) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float s = 0.f;
+  for (int k = 0; k < splits; ++k) s += part[(size_t)k * n + i];
+  out[i] = s;
+}
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -332,15 +491,79 @@ int run_fwd(int N, int H, int W, int Cin, int Cout, const void* x, const void* w
   return pl.BN == 128 ? launch_fwd<128>(pl, mx, mw, my, p) : launch_fwd<64>(pl, mx, mw, my, p);
 }
 
+struct WgPlan {
+  int ok, BW, BH, splits, grid;
+  size_t smem, part_floats;
+};
+
+WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N) {
+  WgPlan pl{};
+  if (Cin % 64 || Cout % 64) return pl;
+  const int cand[3][2] = {{16, 8}, {32, 4}, {8, 16}};
+  for (auto& c : cand)
+    if (W % c[0] == 0 && H % c[1] == 0) {
+      pl.BW = c[0];
+      pl.BH = c[1];
+      break;
+    }
+  if (!pl.BW) return pl;
+  const size_t stage = (size_t)3 * (pl.BH + 2) * pl.BW * 128 + 16384;
+  pl.smem = 2 * stage + 1024 + 1024;
+  if (pl.smem > 232448) return pl;
+  const int blocks = (Cin / 64) * (Cout / 64);
+  const long pix_tiles = (long)N * (H / pl.BH) * (W / pl.BW);
+  long sp = sm_count() / blocks;
+  if (sp < 1) sp = 1;
+  if (sp > pix_tiles) sp = pix_tiles;
+  pl.splits = (int)sp;
+  pl.grid = (int)(sp * blocks);
+  pl.part_floats = (size_t)sp * 9 * Cout * Cin;
+  pl.ok = 1;
+  return pl;
+}
+
+int run_wgrad(int N, int H, int W, int Cin, int Cout, const void* x, const void* dy, float* part, size_t part_floats,
+              float* dw, int32_t* status) {
+  const WgPlan pl = plan_wgrad(H, W, Cin, Cout, N);
+  if (!pl.ok) return NF_EUNSUPPORTED;
+  if (pl.part_floats > part_floats) return NF_ENOWS;
+  CUtensorMap mx, mg;
+  const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
+  const uint32_t bx[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH + 2, 1};
+  const uint64_t dg[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
+  const uint32_t bg[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH, 1};
+  int rc;
+  if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
+  if ((rc = make_map4(&mg, dy, dg, bg)) != NF_OK) return rc;
+  WgParams p{};
+  p.N = N; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout; p.BW = pl.BW; p.BH = pl.BH;
+  p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.pix_tiles = N * p.tiles_h * p.tiles_w;
+  p.ci_chunks = Cin / 64; p.co_chunks = Cout / 64; p.splits = pl.splits; p.part = part; p.status = status;
+  static bool attr_done = false;
+  if (!attr_done) {
+    NF_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    attr_done = true;
+  }
+  conv_wgrad_tc_kernel<<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mg, p);
+  NF_LAUNCHED();
+  const size_t n = (size_t)9 * Cout * Cin;
+  sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, g_nf_stream>>>(part, pl.splits, n, dw);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
 }  // namespace
 
 void nf_tc_select(nf_layer* L) {
   L->fam[0] = L->fam[1] = L->fam[2] = L->fam[3] = 0;
   if (L->o.dtype != NF_BF16) return;
   if (L->o.stride == 1 && plan_fwd(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[0] = 1;
+  if (L->o.stride == 1 && plan_wgrad(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[1] = 1;
 }
 
-size_t nf_tc_scratch_floats(const nf_layer*) { return 0; }
+size_t nf_tc_scratch_floats(const nf_layer* L) {
+  return L->fam[1] ? plan_wgrad(L->H, L->W, L->Cin, L->Cout, L->o.N).part_floats : 0;
+}
 
 size_t nf_tc_red_floats(const nf_layer* L) {
   if (!L->fam[0]) return 0;
@@ -360,7 +583,15 @@ int nf_tc_conv_fwd_eval(nf_layer* L, const void* x, int count) {
   return run_fwd(count, L->H, L->W, L->Cin, L->Cout, x, L->shadow + L->off[NF_P_W], L->y, 0, nullptr, 0, L->status, &nb);
 }
 
-int nf_tc_wgrad(nf_layer*, const void*) { return NF_EUNSUPPORTED; }
+int nf_tc_wgrad(nf_layer* L, const void* x) {
+  return run_wgrad(L->o.N, L->H, L->W, L->Cin, L->Cout, x, L->dy, L->wpart, L->wpart_floats, L->grad + L->off[NF_P_W],
+                   L->status);
+}
+
+size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout) {
+  const WgPlan pl = plan_wgrad(H, W, Cin, Cout, N);
+  return pl.ok ? pl.part_floats : 0;
+}
 
 static __device__ int32_t g_op_status;  // status word of the stand-alone operations
 
@@ -369,6 +600,13 @@ int nf_tc_conv3x3_forward(const void* x, const void* w, int N, int H, int W, int
   if (!st) NF_CUDA(cudaGetSymbolAddress((void**)&st, g_op_status));
   int nb = 0;
   return run_fwd(N, H, W, Cin, Cout, x, w, y, 0, nullptr, 0, st, &nb);
+}
+
+int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int Cin, int Cout, float* part,
+                        size_t part_floats, float* dw) {
+  static int32_t* st = nullptr;
+  if (!st) NF_CUDA(cudaGetSymbolAddress((void**)&st, g_op_status));
+  return run_wgrad(N, H, W, Cin, Cout, x, g, part, part_floats, dw, st);
 }
 
 int nf_tc_op_status(int32_t* out) {
