@@ -314,7 +314,11 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
   trace_end();
   // Eq. 2: aux conv + ReLU, average pool to 2x2, linear; Eq. 3: softmax cross-entropy
   trace_begin(2);
-  NF_TRY(nf_ref_conv(dt, act_out, N, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
+  if (L->fam[2]) {
+    NF_TRY(nf_tc_aux_fwd(L, act_out));
+  } else {
+    NF_TRY(nf_ref_conv(dt, act_out, N, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
+  }
   trace_end();
   trace_begin(3);
   NF_TRY(nf_ref_avgpool(dt, L->h, N, Ha, Wa, F, L->p));

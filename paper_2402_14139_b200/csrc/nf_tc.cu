@@ -24,8 +24,10 @@ struct FwdParams {
   int N, H, W, Cin, Cout;
   int BW, BH, tiles_w, tiles_h, n_tiles, total_tiles, kchunks, stages;
   int stats;
-  float* red;       // [grid * parts][2][Cout] channel partials (pre-zeroed)
-  int32_t* status;  // device status word
+  float* red;         // [grid * parts][2][Cout] channel partials (pre-zeroed)
+  int32_t* status;    // device status word
+  const float* bias;  // EPI 1: per-channel bias added before the ReLU
+  bf16* out;          // EPI 1: destination [N][H][W][Cout], written straight from registers
 };
 
 struct TcPlan {
@@ -33,7 +35,10 @@ struct TcPlan {
   size_t smem;
 };
 
-template <int BN>
+// EPI 0: y in bf16 through a TMA store plus BatchNorm partial sums (BN = 64 or 128).
+// EPI 1: bias + ReLU, channels [0, Cout) of a BN-wide tile written directly (aux conv; Cout <= BN <= 64,
+//        weight rows beyond Cout are zero-filled by TMA).
+template <int BN, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_y, const FwdParams p) {
@@ -42,7 +47,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   const int a_bytes = (p.BH + 2) * p.BW * 128;
   constexpr int b_bytes = 3 * BN * 128;
   const int stage_bytes = a_bytes + b_bytes;
-  constexpr int kSub = BN / 64;  // 64-channel sub-tiles of the output staging
+  constexpr int kSub = EPI == 0 ? BN / 64 : 0;  // 64-channel sub-tiles of the output staging
   uint8_t* stg = smem + (size_t)p.stages * stage_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(stg + kSub * 16384);
   uint64_t* full = bars;
@@ -71,8 +76,9 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     ptx::prefetch_tmap(&tm_w);
     ptx::prefetch_tmap(&tm_y);
   }
+  constexpr uint32_t kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;
   if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, 2 * BN);
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
     ptx::tmem_relinquish();
   }
   ptx::tc_fence_before();
@@ -136,6 +142,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     }
   } else {
     // ---------------- epilogue: 128 threads, thread <-> output pixel (TMEM lane)
+    if constexpr (EPI == 0) {
     const int et = threadIdx.x - 64;
     const int lg = warp & 3;          // TMEM lane group this warp may read
     const int r = lg * 32 + lane;     // row of the tile = pixel (r % BW, r / BW)
@@ -202,6 +209,54 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       const size_t b = (size_t)blockIdx.x * parts + shalf;
       p.red[(b * 2 + 0) * p.Cout + my_nt * BN + sc] = ssum;
       p.red[(b * 2 + 1) * p.Cout + my_nt * BN + sc] = ssq;
+    }
+    } else {
+      const int et = threadIdx.x - 64;
+      const int lg = warp & 3;
+      const int r = lg * 32 + lane;
+      uint32_t tl = 0;
+      for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++tl) {
+        const int m = t / p.n_tiles;
+        const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = m / (p.tiles_w * p.tiles_h);
+        const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+        ptx::mbar_wait(&tfull[acc], aph, abort_flag);
+        ptx::tc_fence_after();
+        if (et == 0) *epi_go = *abort_flag ? 0 : 1;
+        ptx::named_barrier(1, 128);
+        if (!*epi_go) break;
+        bf16* dst = p.out + (((size_t)n * p.H + h0 + r / p.BW) * p.W + w0 + r % p.BW) * p.Cout;
+#pragma unroll
+        for (int j = 0; j < BN / 16; ++j) {
+          uint32_t v[16];
+          ptx::tmem_ld16(tmem_base + ((uint32_t)(lg * 32) << 16) + acc * BN + j * 16, v);
+          ptx::tmem_ld_wait();
+          if (j * 16 < p.Cout) {
+            uint32_t w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const int c = j * 16 + 2 * e;
+              const float a0 = c < p.Cout ? fmaxf(__uint_as_float(v[2 * e]) + p.bias[c], 0.f) : 0.f;
+              const float a1 = c + 1 < p.Cout ? fmaxf(__uint_as_float(v[2 * e + 1]) + p.bias[c + 1], 0.f) : 0.f;
+              const __nv_bfloat162 b2 = __floats2bfloat162_rn(a0, a1);
+              w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+            }
+            const int c0 = j * 16;
+            if ((p.Cout & 7) == 0) {
+              *reinterpret_cast<uint4*>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+              if (c0 + 8 < p.Cout) *reinterpret_cast<uint4*>(dst + c0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+            } else if ((p.Cout & 3) == 0) {
+#pragma unroll
+              for (int g4 = 0; g4 < 4; ++g4)
+                if (c0 + 4 * g4 < p.Cout) *reinterpret_cast<uint2*>(dst + c0 + 4 * g4) = make_uint2(w[2 * g4], w[2 * g4 + 1]);
+            } else {
+              for (int e = 0; e < 16 && c0 + e < p.Cout; ++e)
+                dst[c0 + e] = __ushort_as_bfloat16((unsigned short)((w[e >> 1] >> ((e & 1) * 16)) & 0xffffu));
+            }
+          }
+        }
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(&tempty[acc]);
+      }
     }
   }
 
@@ -419,9 +474,10 @@ int sm_count() {
   return n;
 }
 
-TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N) {
+TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0) {
   TcPlan pl{};
-  if (Cin % 64 || Cout % 64) return pl;
+  if (Cin % 64) return pl;
+  if (epi == 0 ? (Cout % 64 != 0) : (Cout > 64)) return pl;
   const int cand[3][2] = {{16, 8}, {32, 4}, {8, 16}};
   for (auto& c : cand)
     if (W % c[0] == 0 && H % c[1] == 0) {
@@ -430,16 +486,16 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N) {
       break;
     }
   if (!pl.BW) return pl;
-  pl.BN = Cout % 128 == 0 ? 128 : 64;
+  pl.BN = epi == 0 ? (Cout % 128 == 0 ? 128 : 64) : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64);
   const size_t stage = (size_t)(pl.BH + 2) * pl.BW * 128 + 3 * pl.BN * 128;
-  const size_t fixed = (size_t)(pl.BN / 64) * 16384 + 1024 + 1024;  // staging + barriers + alignment slack
+  const size_t fixed = (size_t)(epi == 0 ? pl.BN / 64 : 0) * 16384 + 1024 + 1024;  // staging + barriers + alignment slack
   int st = (int)((232448 - fixed) / stage);
   if (st > kMaxStages) st = kMaxStages;
   if (st < 2) return pl;
   pl.stages = st;
   pl.smem = (size_t)st * stage + fixed;
   pl.parts = pl.BN >= 128 ? 1 : 128 / pl.BN;
-  const int n_tiles = Cout / pl.BN;
+  const int n_tiles = epi == 0 ? Cout / pl.BN : 1;
   const long total = (long)N * (H / pl.BH) * (W / pl.BW) * n_tiles;
   long g = sm_count();
   g -= g % n_tiles;  // every CTA keeps one channel tile for its whole life
@@ -450,21 +506,22 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N) {
   return pl;
 }
 
-template <int BN>
+template <int BN, int EPI>
 int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const FwdParams& p) {
   static bool attr_done = false;
   if (!attr_done) {
-    NF_CUDA(cudaFuncSetAttribute(conv_fwd_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    NF_CUDA(cudaFuncSetAttribute(conv_fwd_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
   }
-  conv_fwd_tc_kernel<BN><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mw, my, p);
+  conv_fwd_tc_kernel<BN, EPI><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mw, my, p);
   NF_LAUNCHED();
   return NF_OK;
 }
 
+// epi 0: y through TMA + optional statistics.  epi 1: out = ReLU(conv + bias) written directly (y unused).
 int run_fwd(int N, int H, int W, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
-            size_t red_floats, int32_t* status, int* nb) {
-  const TcPlan pl = plan_fwd(H, W, Cin, Cout, N);
+            size_t red_floats, int32_t* status, int* nb, int epi = 0, const float* bias = nullptr) {
+  const TcPlan pl = plan_fwd(H, W, Cin, Cout, N, epi);
   if (!pl.ok) return NF_EUNSUPPORTED;
   CUtensorMap mx, mw, my;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
@@ -476,10 +533,15 @@ int run_fwd(int N, int H, int W, int Cin, int Cout, const void* x, const void* w
   int rc;
   if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
   if ((rc = make_map4(&mw, w, dw, bw)) != NF_OK) return rc;
-  if ((rc = make_map4(&my, y, dy, by)) != NF_OK) return rc;
+  if (epi == 0) {
+    if ((rc = make_map4(&my, y, dy, by)) != NF_OK) return rc;
+  } else {
+    my = mx;  // not used by this epilogue
+  }
   FwdParams p{};
   p.N = N; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout;
-  p.BW = pl.BW; p.BH = pl.BH; p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.n_tiles = Cout / pl.BN;
+  p.BW = pl.BW; p.BH = pl.BH; p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.n_tiles = epi == 0 ? Cout / pl.BN : 1;
+  p.bias = bias; p.out = (bf16*)y;
   p.total_tiles = N * p.tiles_h * p.tiles_w * p.n_tiles;
   p.kchunks = Cin / 64; p.stages = pl.stages; p.stats = stats; p.red = red; p.status = status;
   if (stats) {
@@ -488,7 +550,9 @@ int run_fwd(int N, int H, int W, int Cin, int Cout, const void* x, const void* w
     NF_CUDA(cudaMemsetAsync(red, 0, need * sizeof(float), g_nf_stream));
     *nb = pl.grid * pl.parts;
   }
-  return pl.BN == 128 ? launch_fwd<128>(pl, mx, mw, my, p) : launch_fwd<64>(pl, mx, mw, my, p);
+  if (epi == 0) return pl.BN == 128 ? launch_fwd<128, 0>(pl, mx, mw, my, p) : launch_fwd<64, 0>(pl, mx, mw, my, p);
+  return pl.BN == 16 ? launch_fwd<16, 1>(pl, mx, mw, my, p)
+                     : pl.BN == 32 ? launch_fwd<32, 1>(pl, mx, mw, my, p) : launch_fwd<64, 1>(pl, mx, mw, my, p);
 }
 
 struct WgPlan {
@@ -559,6 +623,7 @@ void nf_tc_select(nf_layer* L) {
   if (L->o.dtype != NF_BF16) return;
   if (L->o.stride == 1 && plan_fwd(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[0] = 1;
   if (L->o.stride == 1 && plan_wgrad(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[1] = 1;
+  if (plan_fwd(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).ok) L->fam[2] = 1;
 }
 
 size_t nf_tc_scratch_floats(const nf_layer* L) {
@@ -581,6 +646,12 @@ int nf_tc_conv_fwd(nf_layer* L, const void* x, int& nb) {
 int nf_tc_conv_fwd_eval(nf_layer* L, const void* x, int count) {
   int nb = 0;
   return run_fwd(count, L->H, L->W, L->Cin, L->Cout, x, L->shadow + L->off[NF_P_W], L->y, 0, nullptr, 0, L->status, &nb);
+}
+
+int nf_tc_aux_fwd(nf_layer* L, const void* a) {
+  int nb = 0;
+  return run_fwd(L->o.N, L->Ha, L->Wa, L->Cout, L->F, a, L->shadow + L->off[NF_P_WA], L->h, 0, nullptr, 0, L->status, &nb, 1,
+                 L->val + L->off[NF_P_BA]);
 }
 
 int nf_tc_wgrad(nf_layer* L, const void* x) {

@@ -24,3 +24,5 @@ int nf_tc_op_status(int32_t* out);
 size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout);
 int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int Cin, int Cout, float* part,
                         size_t part_floats, float* dw);
+// Aux conv forward on tensor cores: L->h = ReLU(conv(a, Wa) + ba) in bf16.
+int nf_tc_aux_fwd(nf_layer* L, const void* a);

@@ -123,6 +123,10 @@ TC = [
     dict(N=4, Cin=64, Cout=64, H=32, W=32, F=16, classes=10, stride=1, pool=False),
     dict(N=6, Cin=128, Cout=128, H=16, W=16, F=16, classes=10, stride=1, pool=True),
     dict(N=3, Cin=64, Cout=128, H=16, W=32, F=8, classes=20, stride=1, pool=False),
+    dict(N=4, Cin=64, Cout=64, H=16, W=16, F=4, classes=10, stride=1, pool=False),    # aux tile padded 4 -> 16
+    dict(N=4, Cin=64, Cout=64, H=16, W=16, F=32, classes=10, stride=1, pool=False),
+    dict(N=4, Cin=64, Cout=64, H=16, W=16, F=64, classes=10, stride=1, pool=True),
+    dict(N=4, Cin=64, Cout=64, H=16, W=16, F=12, classes=10, stride=1, pool=False),   # F not a multiple of 8
 ]
 
 
@@ -132,7 +136,7 @@ def test_tensor_core_shapes_bf16(env, ci):
     c = TC[ci]
     P, x, y = pu.seeded_case(c, 1, bf16=True)
     G = pu.gpu_layer(nf, c, P, nf.NF_BF16)
-    assert G.kernel_family(0) == "tcgen05"
+    assert G.kernel_family(0) == "tcgen05" and G.kernel_family(1) == "tcgen05"
     G.close()
     w = pu.check_step(nf, torch, c, seed=400 + ci, dtype=nf.NF_BF16, lr=0.02, steps=2)
     print(w)
