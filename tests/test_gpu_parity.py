@@ -125,7 +125,7 @@ TC = [
     dict(N=3, Cin=64, Cout=128, H=16, W=32, F=8, classes=20, stride=1, pool=False),
     dict(N=4, Cin=64, Cout=64, H=16, W=16, F=4, classes=10, stride=1, pool=False),    # aux tile padded 4 -> 16
     dict(N=4, Cin=64, Cout=64, H=16, W=16, F=32, classes=10, stride=1, pool=False),
-    dict(N=4, Cin=64, Cout=64, H=16, W=16, F=64, classes=10, stride=1, pool=True),
+    dict(N=12, Cin=64, Cout=64, H=16, W=16, F=64, classes=10, stride=1, pool=True),
     dict(N=4, Cin=64, Cout=64, H=16, W=16, F=12, classes=10, stride=1, pool=False),   # F not a multiple of 8
 ]
 
