@@ -329,7 +329,11 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
   trace_end();
   trace_begin(4);
   NF_TRY(nf_ref_dh(dt, L->h, L->dp, N, Ha, Wa, F, L->dh));
-  NF_TRY(nf_ref_wgrad(dt, act_out, N, Ha, Wa, Co, L->dh, F, 1, L->wpart, L->wpart_floats, g + L->off[NF_P_WA]));
+  if (L->fam[3]) {
+    NF_TRY(nf_tc_aux_wgrad(L, act_out));
+  } else {
+    NF_TRY(nf_ref_wgrad(dt, act_out, N, Ha, Wa, Co, L->dh, F, 1, L->wpart, L->wpart_floats, g + L->off[NF_P_WA]));
+  }
   NF_TRY(nf_ref_channel_sums(dt, L->dh, (size_t)N * Ha * Wa, F, L->red, L->red_floats, &nb));
   NF_TRY(nf_ref_sum_partials(L->red, nb, F, 0, g + L->off[NF_P_BA]));
   // gradient at the aux input

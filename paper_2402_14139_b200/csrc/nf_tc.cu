@@ -294,20 +294,27 @@ struct WgParams {
   int32_t* status;
 };
 
+// NB = width of the output-gradient tile in channels (64: main conv, one 64-channel chunk per CTA;
+// 16/32/64: aux conv with F <= NB filters, rows of 2*NB bytes with the matching TMA swizzle).
+template <int NB>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_dy, const WgParams p) {
+  constexpr int kBRow = NB * 2;                                // bytes of one pixel row of the dy tile
+  constexpr uint32_t kBLayout = NB == 64 ? 2 : NB == 32 ? 4 : 6;  // swizzle of that tile
+  constexpr int kBTile = 128 * kBRow;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int kStages = 2;
   const int copy_bytes = (p.BH + 2) * p.BW * 128;
-  const int stage_bytes = 3 * copy_bytes + 16384;
+  const int stage_bytes = 3 * copy_bytes + 16384;  // the dy tile always gets 16 KB so the unused rows read by the
+                                                   // half-empty fifth instruction stay inside the stage
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * stage_bytes);
   uint64_t* full = bars;
   uint64_t* empty = bars + kStages;
   uint64_t* done = bars + 2 * kStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  constexpr uint32_t kCols = 512;  // 5 accumulators x 64 columns, rounded up to a power of two
+  constexpr uint32_t kCols = NB == 64 ? 512 : NB == 32 ? 256 : 128;  // 5 accumulators x NB columns, power of two
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int blocks = p.ci_chunks * p.co_chunks;
@@ -344,15 +351,15 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       if (lane == 0) {
         const int w0 = (t % p.tiles_w) * p.BW, h0 = ((t / p.tiles_w) % p.tiles_h) * p.BH, n = t / (p.tiles_w * p.tiles_h);
         uint8_t* st = smem + (size_t)s * stage_bytes;
-        ptx::mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
+        ptx::mbar_expect_tx(&full[s], (uint32_t)(3 * copy_bytes + kBTile));
 #pragma unroll
         for (int kw = 0; kw < 3; ++kw) ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, w0 + kw - 1, h0 - 1, n);
-        ptx::tma_load_4d(st + 3 * copy_bytes, &tm_dy, &full[s], coc * 64, w0, h0, n);
+        ptx::tma_load_4d(st + 3 * copy_bytes, &tm_dy, &full[s], coc * NB, w0, h0, n);
       }
       __syncwarp();
     }
   } else if (warp == 1) {
-    constexpr uint32_t idesc = ptx::idesc_bf16(128, 64, 1, 1);
+    constexpr uint32_t idesc = ptx::idesc_bf16(128, NB, 1, 1);
     uint32_t it = 0;
     bool ok = true;
     for (int t = t0; t < t1; ++t, ++it) {
@@ -367,16 +374,16 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint32_t koff = k * 16 * 128;  // 16 pixels per instruction
-          const uint64_t bd = ptx::sdesc_sw128(gb + koff, 16, 1024);
+          const uint64_t bd = ptx::sdesc(gb + k * 16 * kBRow, 16, 8 * kBRow, kBLayout);
           const uint32_t acc = (it | k) != 0;
 #pragma unroll
           for (int kw = 0; kw < 3; ++kw)  // taps (kh=0,kw) and (kh=1,kw): second chunk one image row further
-            ptx::mma_f16(tmem_base + kw * 64, ptx::sdesc_sw128(xb + kw * copy_bytes + koff, row, 1024), bd, idesc, acc);
+            ptx::mma_f16(tmem_base + kw * NB, ptx::sdesc_sw128(xb + kw * copy_bytes + koff, row, 1024), bd, idesc, acc);
           // taps (kh=2,kw=0) and (kh=2,kw=1): second chunk one box further
-          ptx::mma_f16(tmem_base + 192, ptx::sdesc_sw128(xb + 2 * row + koff, copy_bytes, 1024), bd, idesc, acc);
+          ptx::mma_f16(tmem_base + 3 * NB, ptx::sdesc_sw128(xb + 2 * row + koff, copy_bytes, 1024), bd, idesc, acc);
           // tap (kh=2,kw=2); rows 64..127 of this accumulator are not used (their operand rows fall on the
           // rows after the box, which are still inside this stage's buffer)
-          ptx::mma_f16(tmem_base + 256, ptx::sdesc_sw128(xb + 2 * copy_bytes + 2 * row + koff, row, 1024), bd, idesc, acc);
+          ptx::mma_f16(tmem_base + 4 * NB, ptx::sdesc_sw128(xb + 2 * copy_bytes + 2 * row + koff, row, 1024), bd, idesc, acc);
         }
         ptx::mma_commit(&empty[s]);
       }
@@ -390,7 +397,8 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     if (ptx::mbar_wait(done, 0, abort_flag) && t1 > t0) {
       ptx::tc_fence_after();
       const size_t plane = (size_t)p.Cout * p.Cin;
-      float* base = p.part + (size_t)sp * 9 * plane + (size_t)(coc * 64) * p.Cin + cic * 64 + (m & 63);
+      float* base = p.part + (size_t)sp * 9 * plane + (size_t)(coc * NB) * p.Cin + cic * 64 + (m & 63);
+      const int co_left = p.Cout - coc * NB;  // output channels of this chunk that exist (aux: F may be < NB)
 #pragma unroll 1
       for (int j = 0; j < 5; ++j) {
         // taps of accumulator j: rows 0..63 -> tapA, rows 64..127 -> tapB (kh*3+kw)
@@ -398,14 +406,15 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         const int tapB = j < 3 ? 3 + j : (j == 3 ? 7 : -1);
         const int tap = m < 64 ? tapA : tapB;
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          uint32_t v[32];
-          ptx::tmem_ld32(tmem_base + ((uint32_t)(lg * 32) << 16) + j * 64 + q * 32, v);
+        for (int q = 0; q < NB / 16; ++q) {
+          uint32_t v[16];
+          ptx::tmem_ld16(tmem_base + ((uint32_t)(lg * 32) << 16) + j * NB + q * 16, v);
           ptx::tmem_ld_wait();
           if (tap >= 0) {
-            float* dst = base + (size_t)tap * plane + (size_t)(q * 32) * p.Cin;
+            float* dst = base + (size_t)tap * plane + (size_t)(q * 16) * p.Cin;
 #pragma unroll
-            for (int e = 0; e < 32; ++e) dst[(size_t)e * p.Cin] = __uint_as_float(v[e]);
+            for (int e = 0; e < 16; ++e)
+              if (q * 16 + e < co_left) dst[(size_t)e * p.Cin] = __uint_as_float(v[e]);
           }
         }
       }
@@ -450,8 +459,10 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 tensor, 4 dims (innermost first), 128-byte swizzle, zero fill outside
+// bf16 tensor, 4 dims (innermost first), zero fill outside; the swizzle span equals the inner box (32/64/128 bytes)
 int make_map4(CUtensorMap* m, const void* base, const uint64_t dims[4], const uint32_t box[4]) {
+  const CUtensorMapSwizzle sw = box[0] * 2 >= 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                : box[0] * 2 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
   EncodeTiledFn fn = encode_fn();
   if (!fn) return NF_ECUDA;
   cuuint64_t gdim[4] = {dims[0], dims[1], dims[2], dims[3]};
@@ -459,7 +470,7 @@ int make_map4(CUtensorMap* m, const void* base, const uint64_t dims[4], const ui
   cuuint32_t bx[4] = {box[0], box[1], box[2], box[3]};
   cuuint32_t es[4] = {1, 1, 1, 1};
   const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gdim, gstr, bx, es,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? NF_OK : nf_cuda_check(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
 }
@@ -556,13 +567,15 @@ int run_fwd(int N, int H, int W, int Cin, int Cout, const void* x, const void* w
 }
 
 struct WgPlan {
-  int ok, BW, BH, splits, grid;
+  int ok, BW, BH, NB, splits, grid;
   size_t smem, part_floats;
 };
 
-WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N) {
+// aux = 0: main conv (Cout a multiple of 64).  aux = 1: aux conv (Cout = F <= 64, a multiple of 8).
+WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0) {
   WgPlan pl{};
-  if (Cin % 64 || Cout % 64) return pl;
+  if (Cin % 64) return pl;
+  if (aux ? (Cout > 64 || Cout % 8) : (Cout % 64 != 0)) return pl;
   const int cand[3][2] = {{16, 8}, {32, 4}, {8, 16}};
   for (auto& c : cand)
     if (W % c[0] == 0 && H % c[1] == 0) {
@@ -574,7 +587,8 @@ WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N) {
   const size_t stage = (size_t)3 * (pl.BH + 2) * pl.BW * 128 + 16384;
   pl.smem = 2 * stage + 1024 + 1024;
   if (pl.smem > 232448) return pl;
-  const int blocks = (Cin / 64) * (Cout / 64);
+  pl.NB = aux ? (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64) : 64;
+  const int blocks = (Cin / 64) * (aux ? 1 : Cout / 64);
   const long pix_tiles = (long)N * (H / pl.BH) * (W / pl.BW);
   long sp = sm_count() / blocks;
   if (sp < 1) sp = 1;
@@ -586,30 +600,38 @@ WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N) {
   return pl;
 }
 
+template <int NB>
+int launch_wgrad(const WgPlan& pl, const CUtensorMap& mx, const CUtensorMap& mg, const WgParams& p) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    NF_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    attr_done = true;
+  }
+  conv_wgrad_tc_kernel<NB><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mg, p);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
 int run_wgrad(int N, int H, int W, int Cin, int Cout, const void* x, const void* dy, float* part, size_t part_floats,
-              float* dw, int32_t* status) {
-  const WgPlan pl = plan_wgrad(H, W, Cin, Cout, N);
+              float* dw, int32_t* status, int aux = 0) {
+  const WgPlan pl = plan_wgrad(H, W, Cin, Cout, N, aux);
   if (!pl.ok) return NF_EUNSUPPORTED;
   if (pl.part_floats > part_floats) return NF_ENOWS;
   CUtensorMap mx, mg;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
   const uint32_t bx[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH + 2, 1};
   const uint64_t dg[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t bg[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH, 1};
+  const uint32_t bg[4] = {(uint32_t)pl.NB, (uint32_t)pl.BW, (uint32_t)pl.BH, 1};
   int rc;
   if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
   if ((rc = make_map4(&mg, dy, dg, bg)) != NF_OK) return rc;
   WgParams p{};
   p.N = N; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout; p.BW = pl.BW; p.BH = pl.BH;
   p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.pix_tiles = N * p.tiles_h * p.tiles_w;
-  p.ci_chunks = Cin / 64; p.co_chunks = Cout / 64; p.splits = pl.splits; p.part = part; p.status = status;
-  static bool attr_done = false;
-  if (!attr_done) {
-    NF_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
-    attr_done = true;
-  }
-  conv_wgrad_tc_kernel<<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mg, p);
-  NF_LAUNCHED();
+  p.ci_chunks = Cin / 64; p.co_chunks = aux ? 1 : Cout / 64; p.splits = pl.splits; p.part = part; p.status = status;
+  if ((rc = pl.NB == 64 ? launch_wgrad<64>(pl, mx, mg, p) : pl.NB == 32 ? launch_wgrad<32>(pl, mx, mg, p)
+                                                                         : launch_wgrad<16>(pl, mx, mg, p)) != NF_OK)
+    return rc;
   const size_t n = (size_t)9 * Cout * Cin;
   sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, g_nf_stream>>>(part, pl.splits, n, dw);
   NF_LAUNCHED();
@@ -624,10 +646,13 @@ void nf_tc_select(nf_layer* L) {
   if (L->o.stride == 1 && plan_fwd(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[0] = 1;
   if (L->o.stride == 1 && plan_wgrad(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[1] = 1;
   if (plan_fwd(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).ok) L->fam[2] = 1;
+  if (plan_wgrad(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).ok) L->fam[3] = 1;
 }
 
 size_t nf_tc_scratch_floats(const nf_layer* L) {
-  return L->fam[1] ? plan_wgrad(L->H, L->W, L->Cin, L->Cout, L->o.N).part_floats : 0;
+  const size_t a = L->fam[1] ? plan_wgrad(L->H, L->W, L->Cin, L->Cout, L->o.N).part_floats : 0;
+  const size_t b = L->fam[3] ? plan_wgrad(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).part_floats : 0;
+  return a > b ? a : b;
 }
 
 size_t nf_tc_red_floats(const nf_layer* L) {
@@ -657,6 +682,11 @@ int nf_tc_aux_fwd(nf_layer* L, const void* a) {
 int nf_tc_wgrad(nf_layer* L, const void* x) {
   return run_wgrad(L->o.N, L->H, L->W, L->Cin, L->Cout, x, L->dy, L->wpart, L->wpart_floats, L->grad + L->off[NF_P_W],
                    L->status);
+}
+
+int nf_tc_aux_wgrad(nf_layer* L, const void* a) {
+  return run_wgrad(L->o.N, L->Ha, L->Wa, L->Cout, L->F, a, L->dh, L->wpart, L->wpart_floats, L->grad + L->off[NF_P_WA],
+                   L->status, 1);
 }
 
 size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout) {

@@ -26,3 +26,5 @@ int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int C
                         size_t part_floats, float* dw);
 // Aux conv forward on tensor cores: L->h = ReLU(conv(a, Wa) + ba) in bf16.
 int nf_tc_aux_fwd(nf_layer* L, const void* a);
+// Aux conv weight gradient on tensor cores: grad(Wa) = wgrad(a, L->dh).
+int nf_tc_aux_wgrad(nf_layer* L, const void* a);
