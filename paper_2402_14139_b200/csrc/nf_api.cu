@@ -337,7 +337,11 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
   NF_TRY(nf_ref_channel_sums(dt, L->dh, (size_t)N * Ha * Wa, F, L->red, L->red_floats, &nb));
   NF_TRY(nf_ref_sum_partials(L->red, nb, F, 0, g + L->off[NF_P_BA]));
   // gradient at the aux input
-  NF_TRY(nf_ref_conv(dt, L->dh, N, Ha, Wa, F, Wx, (long)F * Co, 1, Co, 1, nullptr, 0, 1, Co, L->da));
+  if (L->fam[3]) {
+    NF_TRY(nf_tc_aux_dgrad(L));
+  } else {
+    NF_TRY(nf_ref_conv(dt, L->dh, N, Ha, Wa, F, Wx, (long)F * Co, 1, Co, 1, nullptr, 0, 1, Co, L->da));
+  }
   trace_end();
   // back through pool / ReLU / BatchNorm
   trace_begin(5);

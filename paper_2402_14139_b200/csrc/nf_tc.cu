@@ -31,22 +31,29 @@ struct FwdParams {
 };
 
 struct TcPlan {
-  int ok, BW, BH, BN, stages, grid, parts;
+  int ok, BW, BH, BN, KC, stages, grid, parts;
   size_t smem;
 };
 
 // EPI 0: y in bf16 through a TMA store plus BatchNorm partial sums (BN = 64 or 128).
 // EPI 1: bias + ReLU, channels [0, Cout) of a BN-wide tile written directly (aux conv; Cout <= BN <= 64,
 //        weight rows beyond Cout are zero-filled by TMA).
-template <int BN, int EPI>
+// KC  : channels per K chunk of the activation box (64, or 16/32 for the narrow dh tensor of the aux
+//       input gradient; rows of 2*KC bytes with the matching TMA swizzle).
+// BMN : 0 = weights [tap][co][ci] read K-major (forward); 1 = weights [tap][f][c] read MN-major with the
+//       taps mirrored, which makes the same kernel the input-gradient convolution da = dh (*) Wa^T.
+template <int BN, int EPI, int KC = 64, int BMN = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_y, const FwdParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int a_bytes = (p.BH + 2) * p.BW * 128;
-  constexpr int b_bytes = 3 * BN * 128;
-  const int stage_bytes = a_bytes + b_bytes;
+  constexpr int kARow = KC * 2;  // bytes of one pixel row of the activation box
+  constexpr uint32_t kALayout = KC == 64 ? 2 : KC == 32 ? 4 : 6;
+  const int a_bytes = (p.BH + 2) * p.BW * kARow;
+  const int a_stride = (a_bytes + 1023) & ~1023;  // keeps the weight tiles 1024-byte aligned
+  constexpr int b_bytes = BMN ? (BN / 64) * 3 * KC * 128 : 3 * BN * 128;
+  const int stage_bytes = a_stride + b_bytes;
   constexpr int kSub = EPI == 0 ? BN / 64 : 0;  // 64-channel sub-tiles of the output staging
   uint8_t* stg = smem + (size_t)p.stages * stage_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(stg + kSub * 16384);
@@ -100,16 +107,22 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         if (lane == 0) {
           const int kw = ks % 3, ck = ks / 3;
           uint8_t* a_s = smem + (size_t)s * stage_bytes;
-          ptx::mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
-          ptx::tma_load_4d(a_s, &tm_x, &full[s], ck * 64, w0 + kw - 1, h0 - 1, n);
-          ptx::tma_load_4d(a_s + a_bytes, &tm_w, &full[s], ck * 64, nt * BN, kw, 0);
+          ptx::mbar_expect_tx(&full[s], (uint32_t)(a_bytes + b_bytes));
+          ptx::tma_load_4d(a_s, &tm_x, &full[s], ck * KC, w0 + kw - 1, h0 - 1, n);
+          if constexpr (BMN) {
+#pragma unroll
+            for (int hf = 0; hf < BN / 64; ++hf)  // [half][kh][KC rows of f][64 channels], mirrored column tap
+              ptx::tma_load_4d(a_s + a_stride + hf * 3 * KC * 128, &tm_w, &full[s], nt * BN + hf * 64, 0, 2 - kw, 0);
+          } else {
+            ptx::tma_load_4d(a_s + a_stride, &tm_w, &full[s], ck * 64, nt * BN, kw, 0);
+          }
         }
         __syncwarp();
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer
-    constexpr uint32_t idesc = ptx::idesc_bf16(128, BN, 0, 0);
+    constexpr uint32_t idesc = ptx::idesc_bf16(128, BN, 0, BMN);
     uint32_t it = 0, tl = 0;
     bool ok = true;
     for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++tl) {
@@ -124,13 +137,14 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         ptx::tc_fence_after();
         if (lane == 0) {
           const uint32_t a_base = ptx::smem_u32(smem + (size_t)s * stage_bytes);
-          const uint32_t b_base = a_base + a_bytes;
+          const uint32_t b_base = a_base + a_stride;
 #pragma unroll
           for (int kh = 0; kh < 3; ++kh)
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const uint64_t ad = ptx::sdesc_sw128(a_base + kh * p.BW * 128 + k * 32, 16, 1024);
-              const uint64_t bd = ptx::sdesc_sw128(b_base + kh * BN * 128 + k * 32, 16, 1024);
+            for (int k = 0; k < KC / 16; ++k) {
+              const uint64_t ad = ptx::sdesc(a_base + kh * p.BW * kARow + k * 32, 16, 8 * kARow, kALayout);
+              const uint64_t bd = BMN ? ptx::sdesc_sw128(b_base + (2 - kh) * KC * 128 + k * 16 * 128, 3 * KC * 128, 1024)
+                                      : ptx::sdesc_sw128(b_base + kh * BN * 128 + k * 32, 16, 1024);
               ptx::mma_f16(d, ad, bd, idesc, (ks | kh | k) != 0);
             }
           ptx::mma_commit(&empty[s]);
@@ -485,10 +499,12 @@ int sm_count() {
   return n;
 }
 
+// mode 0: main forward (y + statistics), 1: aux forward (bias + ReLU, Cout = F), 2: aux input gradient
+// (Cin = F <= 64 and a multiple of 8, Cout a multiple of 64, mirrored MN-major weights).
 TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0) {
   TcPlan pl{};
-  if (Cin % 64) return pl;
-  if (epi == 0 ? (Cout % 64 != 0) : (Cout > 64)) return pl;
+  if (epi == 2 ? (Cin > 64 || Cin % 8 || Cout % 64) : (Cin % 64 != 0)) return pl;
+  if (epi == 0 ? (Cout % 64 != 0) : epi == 1 ? (Cout > 64) : false) return pl;
   const int cand[3][2] = {{16, 8}, {32, 4}, {8, 16}};
   for (auto& c : cand)
     if (W % c[0] == 0 && H % c[1] == 0) {
@@ -497,16 +513,18 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0) {
       break;
     }
   if (!pl.BW) return pl;
-  pl.BN = epi == 0 ? (Cout % 128 == 0 ? 128 : 64) : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64);
-  const size_t stage = (size_t)(pl.BH + 2) * pl.BW * 128 + 3 * pl.BN * 128;
-  const size_t fixed = (size_t)(epi == 0 ? pl.BN / 64 : 0) * 16384 + 1024 + 1024;  // staging + barriers + alignment slack
+  pl.BN = epi != 1 ? (Cout % 128 == 0 ? 128 : 64) : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64);
+  pl.KC = epi == 2 ? (Cin <= 16 ? 16 : Cin <= 32 ? 32 : 64) : 64;
+  const size_t a_stride = ((size_t)(pl.BH + 2) * pl.BW * pl.KC * 2 + 1023) & ~(size_t)1023;
+  const size_t stage = a_stride + (epi == 2 ? (size_t)(pl.BN / 64) * 3 * pl.KC * 128 : (size_t)3 * pl.BN * 128);
+  const size_t fixed = (size_t)(epi != 1 ? pl.BN / 64 : 0) * 16384 + 1024 + 1024;  // staging + barriers + alignment slack
   int st = (int)((232448 - fixed) / stage);
   if (st > kMaxStages) st = kMaxStages;
   if (st < 2) return pl;
   pl.stages = st;
   pl.smem = (size_t)st * stage + fixed;
   pl.parts = pl.BN >= 128 ? 1 : 128 / pl.BN;
-  const int n_tiles = epi == 0 ? Cout / pl.BN : 1;
+  const int n_tiles = epi != 1 ? Cout / pl.BN : 1;
   const long total = (long)N * (H / pl.BH) * (W / pl.BW) * n_tiles;
   long g = sm_count();
   g -= g % n_tiles;  // every CTA keeps one channel tile for its whole life
@@ -517,14 +535,14 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0) {
   return pl;
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, int KC = 64, int BMN = 0>
 int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const FwdParams& p) {
   static bool attr_done = false;
   if (!attr_done) {
-    NF_CUDA(cudaFuncSetAttribute(conv_fwd_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    NF_CUDA(cudaFuncSetAttribute(conv_fwd_tc_kernel<BN, EPI, KC, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
   }
-  conv_fwd_tc_kernel<BN, EPI><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mw, my, p);
+  conv_fwd_tc_kernel<BN, EPI, KC, BMN><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mw, my, p);
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -536,25 +554,27 @@ int run_fwd(int N, int H, int W, int Cin, int Cout, const void* x, const void* w
   if (!pl.ok) return NF_EUNSUPPORTED;
   CUtensorMap mx, mw, my;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t bx[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH + 2, 1};
-  const uint64_t dw[4] = {(uint64_t)Cin, (uint64_t)Cout, 3, 3};
-  const uint32_t bw[4] = {64, (uint32_t)pl.BN, 1, 3};
+  const uint32_t bx[4] = {(uint32_t)pl.KC, (uint32_t)pl.BW, (uint32_t)pl.BH + 2, 1};
+  // forward: weights [kh][kw][Cout][Cin] -> box of BN rows x 64 ci for three kh; input gradient: weights
+  // [kh][kw][F][Cout] -> box of KC rows of f x 64 c for three kh
+  const uint64_t dw[4] = {(uint64_t)(epi == 2 ? Cout : Cin), (uint64_t)(epi == 2 ? Cin : Cout), 3, 3};
+  const uint32_t bw[4] = {64, (uint32_t)(epi == 2 ? pl.KC : pl.BN), 1, 3};
   const uint64_t dy[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
   const uint32_t by[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH, 1};
   int rc;
   if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
   if ((rc = make_map4(&mw, w, dw, bw)) != NF_OK) return rc;
-  if (epi == 0) {
+  if (epi != 1) {
     if ((rc = make_map4(&my, y, dy, by)) != NF_OK) return rc;
   } else {
     my = mx;  // not used by this epilogue
   }
   FwdParams p{};
   p.N = N; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout;
-  p.BW = pl.BW; p.BH = pl.BH; p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.n_tiles = epi == 0 ? Cout / pl.BN : 1;
+  p.BW = pl.BW; p.BH = pl.BH; p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.n_tiles = epi != 1 ? Cout / pl.BN : 1;
   p.bias = bias; p.out = (bf16*)y;
   p.total_tiles = N * p.tiles_h * p.tiles_w * p.n_tiles;
-  p.kchunks = Cin / 64; p.stages = pl.stages; p.stats = stats; p.red = red; p.status = status;
+  p.kchunks = epi == 2 ? 1 : Cin / 64; p.stages = pl.stages; p.stats = stats; p.red = red; p.status = status;
   if (stats) {
     const size_t need = (size_t)pl.grid * pl.parts * 2 * Cout;
     if (need > red_floats) return NF_ENOWS;
@@ -562,6 +582,13 @@ int run_fwd(int N, int H, int W, int Cin, int Cout, const void* x, const void* w
     *nb = pl.grid * pl.parts;
   }
   if (epi == 0) return pl.BN == 128 ? launch_fwd<128, 0>(pl, mx, mw, my, p) : launch_fwd<64, 0>(pl, mx, mw, my, p);
+  if (epi == 2) {
+    if (pl.BN == 128)
+      return pl.KC == 16 ? launch_fwd<128, 0, 16, 1>(pl, mx, mw, my, p)
+                         : pl.KC == 32 ? launch_fwd<128, 0, 32, 1>(pl, mx, mw, my, p) : launch_fwd<128, 0, 64, 1>(pl, mx, mw, my, p);
+    return pl.KC == 16 ? launch_fwd<64, 0, 16, 1>(pl, mx, mw, my, p)
+                       : pl.KC == 32 ? launch_fwd<64, 0, 32, 1>(pl, mx, mw, my, p) : launch_fwd<64, 0, 64, 1>(pl, mx, mw, my, p);
+  }
   return pl.BN == 16 ? launch_fwd<16, 1>(pl, mx, mw, my, p)
                      : pl.BN == 32 ? launch_fwd<32, 1>(pl, mx, mw, my, p) : launch_fwd<64, 1>(pl, mx, mw, my, p);
 }
@@ -646,7 +673,7 @@ void nf_tc_select(nf_layer* L) {
   if (L->o.stride == 1 && plan_fwd(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[0] = 1;
   if (L->o.stride == 1 && plan_wgrad(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[1] = 1;
   if (plan_fwd(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).ok) L->fam[2] = 1;
-  if (plan_wgrad(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).ok) L->fam[3] = 1;
+  if (plan_wgrad(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).ok && plan_fwd(L->Ha, L->Wa, L->F, L->Cout, L->o.N, 2).ok) L->fam[3] = 1;
 }
 
 size_t nf_tc_scratch_floats(const nf_layer* L) {
@@ -682,6 +709,12 @@ int nf_tc_aux_fwd(nf_layer* L, const void* a) {
 int nf_tc_wgrad(nf_layer* L, const void* x) {
   return run_wgrad(L->o.N, L->H, L->W, L->Cin, L->Cout, x, L->dy, L->wpart, L->wpart_floats, L->grad + L->off[NF_P_W],
                    L->status);
+}
+
+int nf_tc_aux_dgrad(nf_layer* L) {
+  int nb = 0;
+  return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->shadow + L->off[NF_P_WA], L->da, 0, nullptr, 0, L->status,
+                 &nb, 2);
 }
 
 int nf_tc_aux_wgrad(nf_layer* L, const void* a) {

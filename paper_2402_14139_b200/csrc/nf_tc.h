@@ -28,3 +28,5 @@ int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int C
 int nf_tc_aux_fwd(nf_layer* L, const void* a);
 // Aux conv weight gradient on tensor cores: grad(Wa) = wgrad(a, L->dh).
 int nf_tc_aux_wgrad(nf_layer* L, const void* a);
+// Aux conv input gradient on tensor cores: L->da = dgrad(L->dh, Wa) in bf16.
+int nf_tc_aux_dgrad(nf_layer* L);
