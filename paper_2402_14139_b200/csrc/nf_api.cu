@@ -507,8 +507,8 @@ int nf_conv3x3_forward(int dtype, const void* x, const void* w, int N, int H, in
                        void* y) {
   if (!x || !w || !y || !conv_args_ok(dtype, N, H, W, Cin, Cout, stride)) return NF_EINVAL;
   if (misaligned(x) || misaligned(w) || misaligned(y)) return NF_EALIGN;
-  if (dtype == NF_BF16 && stride == 1) {
-    const int rc = nf_tc_conv3x3_forward(x, w, N, H, W, Cin, Cout, y);
+  if (dtype == NF_BF16) {
+    const int rc = nf_tc_conv3x3_forward(x, w, N, H, W, Cin, Cout, stride, y);
     if (rc != NF_EUNSUPPORTED) return rc;
   }
   return nf_ref_conv(dtype, x, N, H, W, Cin, w, (long)Cout * Cin, Cin, 1, 0, nullptr, 0, stride, Cout, y);
@@ -518,10 +518,8 @@ size_t nf_conv3x3_wgrad_scratch_bytes(int N, int H, int W, int Cin, int Cout, in
   if (!conv_args_ok(NF_F32, N, H, W, Cin, Cout, stride)) return 0;
   const int Ho = (H - 1) / stride + 1;
   size_t fl = (size_t)nf_ref_wgrad_splits(N, Ho, Cin, Cout) * 9 * Cout * Cin;
-  if (stride == 1) {
-    const size_t tc = nf_tc_conv3x3_wgrad_scratch_floats(N, H, W, Cin, Cout);
-    if (tc > fl) fl = tc;
-  }
+  const size_t tc = nf_tc_conv3x3_wgrad_scratch_floats(N, H, W, Cin, Cout, stride);
+  if (tc > fl) fl = tc;
   return fl * sizeof(float);
 }
 
@@ -529,8 +527,8 @@ int nf_conv3x3_wgrad(int dtype, const void* x, const void* g, int N, int H, int 
                      void* scratch, size_t scratch_bytes, float* dw) {
   if (!x || !g || !scratch || !dw || !conv_args_ok(dtype, N, H, W, Cin, Cout, stride)) return NF_EINVAL;
   if (misaligned(x) || misaligned(g) || misaligned(scratch) || misaligned(dw)) return NF_EALIGN;
-  if (dtype == NF_BF16 && stride == 1) {
-    const int rc = nf_tc_conv3x3_wgrad(x, g, N, H, W, Cin, Cout, (float*)scratch, scratch_bytes / sizeof(float), dw);
+  if (dtype == NF_BF16) {
+    const int rc = nf_tc_conv3x3_wgrad(x, g, N, H, W, Cin, Cout, stride, (float*)scratch, scratch_bytes / sizeof(float), dw);
     if (rc != NF_EUNSUPPORTED) return rc;
   }
   return nf_ref_wgrad(dtype, x, N, H, W, Cin, g, Cout, stride, (float*)scratch, scratch_bytes / sizeof(float), dw);

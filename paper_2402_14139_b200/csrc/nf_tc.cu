@@ -42,7 +42,9 @@ struct TcPlan {
 //       input gradient; rows of 2*KC bytes with the matching TMA swizzle).
 // BMN : 0 = weights [tap][co][ci] read K-major (forward); 1 = weights [tap][f][c] read MN-major with the
 //       taps mirrored, which makes the same kernel the input-gradient convolution da = dh (*) Wa^T.
-template <int BN, int EPI, int KC = 64, int BMN = 0>
+// PT  : 1 = one TMA box per tap (stride-2 convolution: the box is gathered with element stride 2, so the
+//       three row taps cannot share a box); p.H, p.W are then the OUTPUT sizes.
+template <int BN, int EPI, int KC = 64, int BMN = 0, int PT = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_y, const FwdParams p) {
@@ -50,9 +52,9 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int kARow = KC * 2;  // bytes of one pixel row of the activation box
   constexpr uint32_t kALayout = KC == 64 ? 2 : KC == 32 ? 4 : 6;
-  const int a_bytes = (p.BH + 2) * p.BW * kARow;
+  const int a_bytes = (PT ? p.BH : p.BH + 2) * p.BW * kARow;
   const int a_stride = (a_bytes + 1023) & ~1023;  // keeps the weight tiles 1024-byte aligned
-  constexpr int b_bytes = BMN ? (BN / 64) * 3 * KC * 128 : 3 * BN * 128;
+  constexpr int b_bytes = PT ? BN * 128 : BMN ? (BN / 64) * 3 * KC * 128 : 3 * BN * 128;
   const int stage_bytes = a_stride + b_bytes;
   constexpr int kSub = EPI == 0 ? BN / 64 : 0;  // 64-channel sub-tiles of the output staging
   uint8_t* stg = smem + (size_t)p.stages * stage_bytes;
@@ -66,7 +68,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ksteps = 3 * p.kchunks;
+  const int ksteps = (PT ? 9 : 3) * p.kchunks;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -105,16 +107,22 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         const uint32_t ph = (it / p.stages) & 1;
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) { ok = false; break; }
         if (lane == 0) {
-          const int kw = ks % 3, ck = ks / 3;
           uint8_t* a_s = smem + (size_t)s * stage_bytes;
           ptx::mbar_expect_tx(&full[s], (uint32_t)(a_bytes + b_bytes));
-          ptx::tma_load_4d(a_s, &tm_x, &full[s], ck * KC, w0 + kw - 1, h0 - 1, n);
-          if constexpr (BMN) {
-#pragma unroll
-            for (int hf = 0; hf < BN / 64; ++hf)  // [half][kh][KC rows of f][64 channels], mirrored column tap
-              ptx::tma_load_4d(a_s + a_stride + hf * 3 * KC * 128, &tm_w, &full[s], nt * BN + hf * 64, 0, 2 - kw, 0);
+          if constexpr (PT) {
+            const int tap = ks % 9, ck = ks / 9, kh = tap / 3, kw = tap % 3;
+            ptx::tma_load_4d(a_s, &tm_x, &full[s], ck * KC, 2 * w0 + kw - 1, 2 * h0 + kh - 1, n);
+            ptx::tma_load_4d(a_s + a_stride, &tm_w, &full[s], ck * 64, nt * BN, kw, kh);
           } else {
-            ptx::tma_load_4d(a_s + a_stride, &tm_w, &full[s], ck * 64, nt * BN, kw, 0);
+            const int kw = ks % 3, ck = ks / 3;
+            ptx::tma_load_4d(a_s, &tm_x, &full[s], ck * KC, w0 + kw - 1, h0 - 1, n);
+            if constexpr (BMN) {
+#pragma unroll
+              for (int hf = 0; hf < BN / 64; ++hf)  // [half][kh][KC rows of f][64 channels], mirrored column tap
+                ptx::tma_load_4d(a_s + a_stride + hf * 3 * KC * 128, &tm_w, &full[s], nt * BN + hf * 64, 0, 2 - kw, 0);
+            } else {
+              ptx::tma_load_4d(a_s + a_stride, &tm_w, &full[s], ck * 64, nt * BN, kw, 0);
+            }
           }
         }
         __syncwarp();
@@ -139,7 +147,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           const uint32_t a_base = ptx::smem_u32(smem + (size_t)s * stage_bytes);
           const uint32_t b_base = a_base + a_stride;
 #pragma unroll
-          for (int kh = 0; kh < 3; ++kh)
+          for (int kh = 0; kh < (PT ? 1 : 3); ++kh)
 #pragma unroll
             for (int k = 0; k < KC / 16; ++k) {
               const uint64_t ad = ptx::sdesc(a_base + kh * p.BW * kARow + k * 32, 16, 8 * kARow, kALayout);
@@ -310,7 +318,10 @@ struct WgParams {
 
 // NB = width of the output-gradient tile in channels (64: main conv, one 64-channel chunk per CTA;
 // 16/32/64: aux conv with F <= NB filters, rows of 2*NB bytes with the matching TMA swizzle).
-template <int NB>
+// S2 = 1: stride-2 convolution.  The shifted activation tiles are gathered by TMA with element stride 2,
+// one 128-pixel tile per tap; a CTA then owns one kernel row kh (grid dimension) with its three column
+// taps: taps (kh,0) and (kh,1) stacked in one instruction, tap (kh,2) in a second, half-empty one.
+template <int NB, int S2>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_dy, const WgParams p) {
   constexpr int kBRow = NB * 2;                                // bytes of one pixel row of the dy tile
@@ -318,21 +329,26 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   constexpr int kBTile = 128 * kBRow;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr int kStages = 2;
-  const int copy_bytes = (p.BH + 2) * p.BW * 128;
+  constexpr int kStages = S2 ? 3 : 2;
+  constexpr int kJobs = S2 ? 2 : 5;  // instructions (accumulators) per 16 pixels
+  const int copy_bytes = S2 ? 16384 : (p.BH + 2) * p.BW * 128;
   const int stage_bytes = 3 * copy_bytes + 16384;  // the dy tile always gets 16 KB so the unused rows read by the
-                                                   // half-empty fifth instruction stay inside the stage
+                                                   // half-empty last instruction stay inside the stage
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * stage_bytes);
   uint64_t* full = bars;
   uint64_t* empty = bars + kStages;
   uint64_t* done = bars + 2 * kStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  constexpr uint32_t kCols = NB == 64 ? 512 : NB == 32 ? 256 : 128;  // 5 accumulators x NB columns, power of two
+  constexpr uint32_t kNeed = kJobs * NB;
+  constexpr uint32_t kCols = kNeed <= 32 ? 32 : kNeed <= 64 ? 64 : kNeed <= 128 ? 128 : kNeed <= 256 ? 256 : 512;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int blocks = p.ci_chunks * p.co_chunks;
-  const int blk = blockIdx.x % blocks, sp = blockIdx.x / blocks;
+  const int blk = blockIdx.x % blocks;
+  const int rest = blockIdx.x / blocks;
+  const int khg = S2 ? rest % 3 : 0;            // kernel row owned by this CTA (stride 2 only)
+  const int sp = S2 ? rest / 3 : rest;
   const int cic = blk % p.ci_chunks, coc = blk / p.ci_chunks;
   const int t0 = (int)((long)p.pix_tiles * sp / p.splits), t1 = (int)((long)p.pix_tiles * (sp + 1) / p.splits);
 
@@ -367,7 +383,12 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         uint8_t* st = smem + (size_t)s * stage_bytes;
         ptx::mbar_expect_tx(&full[s], (uint32_t)(3 * copy_bytes + kBTile));
 #pragma unroll
-        for (int kw = 0; kw < 3; ++kw) ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, w0 + kw - 1, h0 - 1, n);
+        for (int kw = 0; kw < 3; ++kw) {
+          if constexpr (S2)
+            ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, 2 * w0 + kw - 1, 2 * h0 + khg - 1, n);
+          else
+            ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, w0 + kw - 1, h0 - 1, n);
+        }
         ptx::tma_load_4d(st + 3 * copy_bytes, &tm_dy, &full[s], coc * NB, w0, h0, n);
       }
       __syncwarp();
@@ -390,14 +411,20 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           const uint32_t koff = k * 16 * 128;  // 16 pixels per instruction
           const uint64_t bd = ptx::sdesc(gb + k * 16 * kBRow, 16, 8 * kBRow, kBLayout);
           const uint32_t acc = (it | k) != 0;
+          if constexpr (S2) {
+            // taps (kh,0) and (kh,1): second chunk one tile further; tap (kh,2): rows 64..127 unused
+            ptx::mma_f16(tmem_base, ptx::sdesc_sw128(xb + koff, copy_bytes, 1024), bd, idesc, acc);
+            ptx::mma_f16(tmem_base + NB, ptx::sdesc_sw128(xb + 2 * copy_bytes + koff, copy_bytes, 1024), bd, idesc, acc);
+          } else {
 #pragma unroll
-          for (int kw = 0; kw < 3; ++kw)  // taps (kh=0,kw) and (kh=1,kw): second chunk one image row further
-            ptx::mma_f16(tmem_base + kw * NB, ptx::sdesc_sw128(xb + kw * copy_bytes + koff, row, 1024), bd, idesc, acc);
-          // taps (kh=2,kw=0) and (kh=2,kw=1): second chunk one box further
-          ptx::mma_f16(tmem_base + 3 * NB, ptx::sdesc_sw128(xb + 2 * row + koff, copy_bytes, 1024), bd, idesc, acc);
-          // tap (kh=2,kw=2); rows 64..127 of this accumulator are not used (their operand rows fall on the
-          // rows after the box, which are still inside this stage's buffer)
-          ptx::mma_f16(tmem_base + 4 * NB, ptx::sdesc_sw128(xb + 2 * copy_bytes + 2 * row + koff, row, 1024), bd, idesc, acc);
+            for (int kw = 0; kw < 3; ++kw)  // taps (kh=0,kw) and (kh=1,kw): second chunk one image row further
+              ptx::mma_f16(tmem_base + kw * NB, ptx::sdesc_sw128(xb + kw * copy_bytes + koff, row, 1024), bd, idesc, acc);
+            // taps (kh=2,kw=0) and (kh=2,kw=1): second chunk one box further
+            ptx::mma_f16(tmem_base + 3 * NB, ptx::sdesc_sw128(xb + 2 * row + koff, copy_bytes, 1024), bd, idesc, acc);
+            // tap (kh=2,kw=2); rows 64..127 of this accumulator are not used (their operand rows fall on the
+            // rows after the box, which are still inside this stage's buffer)
+            ptx::mma_f16(tmem_base + 4 * NB, ptx::sdesc_sw128(xb + 2 * copy_bytes + 2 * row + koff, row, 1024), bd, idesc, acc);
+          }
         }
         ptx::mma_commit(&empty[s]);
       }
@@ -414,10 +441,16 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       float* base = p.part + (size_t)sp * 9 * plane + (size_t)(coc * NB) * p.Cin + cic * 64 + (m & 63);
       const int co_left = p.Cout - coc * NB;  // output channels of this chunk that exist (aux: F may be < NB)
 #pragma unroll 1
-      for (int j = 0; j < 5; ++j) {
+      for (int j = 0; j < kJobs; ++j) {
         // taps of accumulator j: rows 0..63 -> tapA, rows 64..127 -> tapB (kh*3+kw)
-        const int tapA = j < 3 ? j : (j == 3 ? 6 : 8);
-        const int tapB = j < 3 ? 3 + j : (j == 3 ? 7 : -1);
+        int tapA, tapB;
+        if constexpr (S2) {
+          tapA = khg * 3 + (j == 0 ? 0 : 2);
+          tapB = j == 0 ? khg * 3 + 1 : -1;
+        } else {
+          tapA = j < 3 ? j : (j == 3 ? 6 : 8);
+          tapB = j < 3 ? 3 + j : (j == 3 ? 7 : -1);
+        }
         const int tap = m < 64 ? tapA : tapB;
 #pragma unroll
         for (int q = 0; q < NB / 16; ++q) {
@@ -474,15 +507,17 @@ EncodeTiledFn encode_fn() {
 }
 
 // bf16 tensor, 4 dims (innermost first), zero fill outside; the swizzle span equals the inner box (32/64/128 bytes)
-int make_map4(CUtensorMap* m, const void* base, const uint64_t dims[4], const uint32_t box[4]) {
+int make_map4(CUtensorMap* m, const void* base, const uint64_t dims[4], const uint32_t box[4], int spatial_stride = 1) {
   const CUtensorMapSwizzle sw = box[0] * 2 >= 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                 : box[0] * 2 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
   EncodeTiledFn fn = encode_fn();
   if (!fn) return NF_ECUDA;
   cuuint64_t gdim[4] = {dims[0], dims[1], dims[2], dims[3]};
   cuuint64_t gstr[3] = {dims[0] * 2, dims[0] * dims[1] * 2, dims[0] * dims[1] * dims[2] * 2};
-  cuuint32_t bx[4] = {box[0], box[1], box[2], box[3]};
-  cuuint32_t es[4] = {1, 1, 1, 1};
+  // with an element stride s along w and h the box spans s*box elements and keeps every s-th one
+  const cuuint32_t ss = (cuuint32_t)spatial_stride;
+  cuuint32_t bx[4] = {box[0], box[1] * ss, box[2] * ss, box[3]};
+  cuuint32_t es[4] = {1, ss, ss, 1};
   const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gdim, gstr, bx, es,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -501,8 +536,10 @@ int sm_count() {
 
 // mode 0: main forward (y + statistics), 1: aux forward (bias + ReLU, Cout = F), 2: aux input gradient
 // (Cin = F <= 64 and a multiple of 8, Cout a multiple of 64, mirrored MN-major weights).
-TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0) {
+// H, W: OUTPUT size (equal to the input size for stride 1).
+TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride = 1) {
   TcPlan pl{};
+  if (stride == 2 && (epi != 0 || Cin % 64)) return pl;
   if (epi == 2 ? (Cin > 64 || Cin % 8 || Cout % 64) : (Cin % 64 != 0)) return pl;
   if (epi == 0 ? (Cout % 64 != 0) : epi == 1 ? (Cout > 64) : false) return pl;
   const int cand[3][2] = {{16, 8}, {32, 4}, {8, 16}};
@@ -515,8 +552,9 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0) {
   if (!pl.BW) return pl;
   pl.BN = epi != 1 ? (Cout % 128 == 0 ? 128 : 64) : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64);
   pl.KC = epi == 2 ? (Cin <= 16 ? 16 : Cin <= 32 ? 32 : 64) : 64;
-  const size_t a_stride = ((size_t)(pl.BH + 2) * pl.BW * pl.KC * 2 + 1023) & ~(size_t)1023;
-  const size_t stage = a_stride + (epi == 2 ? (size_t)(pl.BN / 64) * 3 * pl.KC * 128 : (size_t)3 * pl.BN * 128);
+  const size_t a_stride = ((size_t)(stride == 2 ? pl.BH : pl.BH + 2) * pl.BW * pl.KC * 2 + 1023) & ~(size_t)1023;
+  const size_t stage = a_stride + (stride == 2 ? (size_t)pl.BN * 128
+                                               : epi == 2 ? (size_t)(pl.BN / 64) * 3 * pl.KC * 128 : (size_t)3 * pl.BN * 128);
   const size_t fixed = (size_t)(epi != 1 ? pl.BN / 64 : 0) * 16384 + 1024 + 1024;  // staging + barriers + alignment slack
   int st = (int)((232448 - fixed) / stage);
   if (st > kMaxStages) st = kMaxStages;
@@ -535,34 +573,36 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0) {
   return pl;
 }
 
-template <int BN, int EPI, int KC = 64, int BMN = 0>
+template <int BN, int EPI, int KC = 64, int BMN = 0, int PT = 0>
 int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const FwdParams& p) {
   static bool attr_done = false;
   if (!attr_done) {
-    NF_CUDA(cudaFuncSetAttribute(conv_fwd_tc_kernel<BN, EPI, KC, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    NF_CUDA(cudaFuncSetAttribute(conv_fwd_tc_kernel<BN, EPI, KC, BMN, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
   }
-  conv_fwd_tc_kernel<BN, EPI, KC, BMN><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mw, my, p);
+  conv_fwd_tc_kernel<BN, EPI, KC, BMN, PT><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mw, my, p);
   NF_LAUNCHED();
   return NF_OK;
 }
 
 // epi 0: y through TMA + optional statistics.  epi 1: out = ReLU(conv + bias) written directly (y unused).
-int run_fwd(int N, int H, int W, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
-            size_t red_floats, int32_t* status, int* nb, int epi = 0, const float* bias = nullptr) {
-  const TcPlan pl = plan_fwd(H, W, Cin, Cout, N, epi);
+// H, W are the INPUT size; stride 2 halves them (rounding up) for the output.
+int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
+            size_t red_floats, int32_t* status, int* nb, int epi = 0, const float* bias = nullptr, int stride = 1) {
+  const int H = (Hin - 1) / stride + 1, W = (Win - 1) / stride + 1;
+  const TcPlan pl = plan_fwd(H, W, Cin, Cout, N, epi, stride);
   if (!pl.ok) return NF_EUNSUPPORTED;
   CUtensorMap mx, mw, my;
-  const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t bx[4] = {(uint32_t)pl.KC, (uint32_t)pl.BW, (uint32_t)pl.BH + 2, 1};
+  const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)Win, (uint64_t)Hin, (uint64_t)N};
+  const uint32_t bx[4] = {(uint32_t)pl.KC, (uint32_t)pl.BW, (uint32_t)(stride == 2 ? pl.BH : pl.BH + 2), 1};
   // forward: weights [kh][kw][Cout][Cin] -> box of BN rows x 64 ci for three kh; input gradient: weights
   // [kh][kw][F][Cout] -> box of KC rows of f x 64 c for three kh
   const uint64_t dw[4] = {(uint64_t)(epi == 2 ? Cout : Cin), (uint64_t)(epi == 2 ? Cin : Cout), 3, 3};
-  const uint32_t bw[4] = {64, (uint32_t)(epi == 2 ? pl.KC : pl.BN), 1, 3};
+  const uint32_t bw[4] = {64, (uint32_t)(epi == 2 ? pl.KC : pl.BN), 1, (uint32_t)(stride == 2 ? 1 : 3)};
   const uint64_t dy[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
   const uint32_t by[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH, 1};
   int rc;
-  if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
+  if ((rc = make_map4(&mx, x, dx, bx, stride)) != NF_OK) return rc;
   if ((rc = make_map4(&mw, w, dw, bw)) != NF_OK) return rc;
   if (epi != 1) {
     if ((rc = make_map4(&my, y, dy, by)) != NF_OK) return rc;
@@ -581,6 +621,8 @@ int run_fwd(int N, int H, int W, int Cin, int Cout, const void* x, const void* w
     NF_CUDA(cudaMemsetAsync(red, 0, need * sizeof(float), g_nf_stream));
     *nb = pl.grid * pl.parts;
   }
+  if (epi == 0 && stride == 2)
+    return pl.BN == 128 ? launch_fwd<128, 0, 64, 0, 1>(pl, mx, mw, my, p) : launch_fwd<64, 0, 64, 0, 1>(pl, mx, mw, my, p);
   if (epi == 0) return pl.BN == 128 ? launch_fwd<128, 0>(pl, mx, mw, my, p) : launch_fwd<64, 0>(pl, mx, mw, my, p);
   if (epi == 2) {
     if (pl.BN == 128)
@@ -599,9 +641,10 @@ struct WgPlan {
 };
 
 // aux = 0: main conv (Cout a multiple of 64).  aux = 1: aux conv (Cout = F <= 64, a multiple of 8).
-WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0) {
+// H, W: size of the gradient tensor (the conv OUTPUT; equals the input size for stride 1).
+WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0, int stride = 1) {
   WgPlan pl{};
-  if (Cin % 64) return pl;
+  if (Cin % 64 || (stride == 2 && aux)) return pl;
   if (aux ? (Cout > 64 || Cout % 8) : (Cout % 64 != 0)) return pl;
   const int cand[3][2] = {{16, 8}, {32, 4}, {8, 16}};
   for (auto& c : cand)
@@ -611,54 +654,59 @@ WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0) {
       break;
     }
   if (!pl.BW) return pl;
-  const size_t stage = (size_t)3 * (pl.BH + 2) * pl.BW * 128 + 16384;
-  pl.smem = 2 * stage + 1024 + 1024;
+  const size_t stage = stride == 2 ? 65536 : (size_t)3 * (pl.BH + 2) * pl.BW * 128 + 16384;
+  pl.smem = (stride == 2 ? 3 : 2) * stage + 1024 + 1024;
   if (pl.smem > 232448) return pl;
   pl.NB = aux ? (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64) : 64;
   const int blocks = (Cin / 64) * (aux ? 1 : Cout / 64);
   const long pix_tiles = (long)N * (H / pl.BH) * (W / pl.BW);
-  long sp = sm_count() / blocks;
+  const int groups = stride == 2 ? 3 : 1;  // kernel rows handled by separate CTAs
+  long sp = sm_count() / (blocks * groups);
   if (sp < 1) sp = 1;
   if (sp > pix_tiles) sp = pix_tiles;
   pl.splits = (int)sp;
-  pl.grid = (int)(sp * blocks);
+  pl.grid = (int)(sp * blocks * groups);
   pl.part_floats = (size_t)sp * 9 * Cout * Cin;
   pl.ok = 1;
   return pl;
 }
 
-template <int NB>
+template <int NB, int S2 = 0>
 int launch_wgrad(const WgPlan& pl, const CUtensorMap& mx, const CUtensorMap& mg, const WgParams& p) {
   static bool attr_done = false;
   if (!attr_done) {
-    NF_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    NF_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel<NB, S2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
   }
-  conv_wgrad_tc_kernel<NB><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mg, p);
+  conv_wgrad_tc_kernel<NB, S2><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mg, p);
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int run_wgrad(int N, int H, int W, int Cin, int Cout, const void* x, const void* dy, float* part, size_t part_floats,
-              float* dw, int32_t* status, int aux = 0) {
-  const WgPlan pl = plan_wgrad(H, W, Cin, Cout, N, aux);
+// Hin, Win: INPUT size; the gradient tensor has the strided output size.
+int run_wgrad(int N, int Hin, int Win, int Cin, int Cout, const void* x, const void* dy, float* part, size_t part_floats,
+              float* dw, int32_t* status, int aux = 0, int stride = 1) {
+  const int H = (Hin - 1) / stride + 1, W = (Win - 1) / stride + 1;
+  const WgPlan pl = plan_wgrad(H, W, Cin, Cout, N, aux, stride);
   if (!pl.ok) return NF_EUNSUPPORTED;
   if (pl.part_floats > part_floats) return NF_ENOWS;
   CUtensorMap mx, mg;
-  const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t bx[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH + 2, 1};
+  const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)Win, (uint64_t)Hin, (uint64_t)N};
+  const uint32_t bx[4] = {64, (uint32_t)pl.BW, (uint32_t)(stride == 2 ? pl.BH : pl.BH + 2), 1};
   const uint64_t dg[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
   const uint32_t bg[4] = {(uint32_t)pl.NB, (uint32_t)pl.BW, (uint32_t)pl.BH, 1};
   int rc;
-  if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
+  if ((rc = make_map4(&mx, x, dx, bx, stride)) != NF_OK) return rc;
   if ((rc = make_map4(&mg, dy, dg, bg)) != NF_OK) return rc;
   WgParams p{};
   p.N = N; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout; p.BW = pl.BW; p.BH = pl.BH;
   p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.pix_tiles = N * p.tiles_h * p.tiles_w;
   p.ci_chunks = Cin / 64; p.co_chunks = aux ? 1 : Cout / 64; p.splits = pl.splits; p.part = part; p.status = status;
-  if ((rc = pl.NB == 64 ? launch_wgrad<64>(pl, mx, mg, p) : pl.NB == 32 ? launch_wgrad<32>(pl, mx, mg, p)
-                                                                         : launch_wgrad<16>(pl, mx, mg, p)) != NF_OK)
-    return rc;
+  if (stride == 2)
+    rc = launch_wgrad<64, 1>(pl, mx, mg, p);
+  else
+    rc = pl.NB == 64 ? launch_wgrad<64>(pl, mx, mg, p) : pl.NB == 32 ? launch_wgrad<32>(pl, mx, mg, p) : launch_wgrad<16>(pl, mx, mg, p);
+  if (rc != NF_OK) return rc;
   const size_t n = (size_t)9 * Cout * Cin;
   sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, g_nf_stream>>>(part, pl.splits, n, dw);
   NF_LAUNCHED();
@@ -670,21 +718,21 @@ int run_wgrad(int N, int H, int W, int Cin, int Cout, const void* x, const void*
 void nf_tc_select(nf_layer* L) {
   L->fam[0] = L->fam[1] = L->fam[2] = L->fam[3] = 0;
   if (L->o.dtype != NF_BF16) return;
-  if (L->o.stride == 1 && plan_fwd(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[0] = 1;
-  if (L->o.stride == 1 && plan_wgrad(L->H, L->W, L->Cin, L->Cout, L->o.N).ok) L->fam[1] = 1;
+  if (plan_fwd(L->Ho, L->Wo, L->Cin, L->Cout, L->o.N, 0, L->o.stride).ok) L->fam[0] = 1;
+  if (plan_wgrad(L->Ho, L->Wo, L->Cin, L->Cout, L->o.N, 0, L->o.stride).ok) L->fam[1] = 1;
   if (plan_fwd(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).ok) L->fam[2] = 1;
   if (plan_wgrad(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).ok && plan_fwd(L->Ha, L->Wa, L->F, L->Cout, L->o.N, 2).ok) L->fam[3] = 1;
 }
 
 size_t nf_tc_scratch_floats(const nf_layer* L) {
-  const size_t a = L->fam[1] ? plan_wgrad(L->H, L->W, L->Cin, L->Cout, L->o.N).part_floats : 0;
+  const size_t a = L->fam[1] ? plan_wgrad(L->Ho, L->Wo, L->Cin, L->Cout, L->o.N, 0, L->o.stride).part_floats : 0;
   const size_t b = L->fam[3] ? plan_wgrad(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).part_floats : 0;
   return a > b ? a : b;
 }
 
 size_t nf_tc_red_floats(const nf_layer* L) {
   if (!L->fam[0]) return 0;
-  const TcPlan pl = plan_fwd(L->H, L->W, L->Cin, L->Cout, L->o.N);
+  const TcPlan pl = plan_fwd(L->Ho, L->Wo, L->Cin, L->Cout, L->o.N, 0, L->o.stride);
   return (size_t)sm_count() * pl.parts * 2 * L->Cout;
 }
 
@@ -692,12 +740,13 @@ int nf_tc_prepare(nf_layer*) { return NF_OK; }
 
 int nf_tc_conv_fwd(nf_layer* L, const void* x, int& nb) {
   return run_fwd(L->o.N, L->H, L->W, L->Cin, L->Cout, x, L->shadow + L->off[NF_P_W], L->y, 1, L->red, L->red_floats,
-                 L->status, &nb);
+                 L->status, &nb, 0, nullptr, L->o.stride);
 }
 
 int nf_tc_conv_fwd_eval(nf_layer* L, const void* x, int count) {
   int nb = 0;
-  return run_fwd(count, L->H, L->W, L->Cin, L->Cout, x, L->shadow + L->off[NF_P_W], L->y, 0, nullptr, 0, L->status, &nb);
+  return run_fwd(count, L->H, L->W, L->Cin, L->Cout, x, L->shadow + L->off[NF_P_W], L->y, 0, nullptr, 0, L->status, &nb, 0,
+                 nullptr, L->o.stride);
 }
 
 int nf_tc_aux_fwd(nf_layer* L, const void* a) {
@@ -708,7 +757,7 @@ int nf_tc_aux_fwd(nf_layer* L, const void* a) {
 
 int nf_tc_wgrad(nf_layer* L, const void* x) {
   return run_wgrad(L->o.N, L->H, L->W, L->Cin, L->Cout, x, L->dy, L->wpart, L->wpart_floats, L->grad + L->off[NF_P_W],
-                   L->status);
+                   L->status, 0, L->o.stride);
 }
 
 int nf_tc_aux_dgrad(nf_layer* L) {
@@ -722,25 +771,25 @@ int nf_tc_aux_wgrad(nf_layer* L, const void* a) {
                    L->status, 1);
 }
 
-size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout) {
-  const WgPlan pl = plan_wgrad(H, W, Cin, Cout, N);
+size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout, int stride) {
+  const WgPlan pl = plan_wgrad((H - 1) / stride + 1, (W - 1) / stride + 1, Cin, Cout, N, 0, stride);
   return pl.ok ? pl.part_floats : 0;
 }
 
 static __device__ int32_t g_op_status;  // status word of the stand-alone operations
 
-int nf_tc_conv3x3_forward(const void* x, const void* w, int N, int H, int W, int Cin, int Cout, void* y) {
+int nf_tc_conv3x3_forward(const void* x, const void* w, int N, int H, int W, int Cin, int Cout, int stride, void* y) {
   static int32_t* st = nullptr;
   if (!st) NF_CUDA(cudaGetSymbolAddress((void**)&st, g_op_status));
   int nb = 0;
-  return run_fwd(N, H, W, Cin, Cout, x, w, y, 0, nullptr, 0, st, &nb);
+  return run_fwd(N, H, W, Cin, Cout, x, w, y, 0, nullptr, 0, st, &nb, 0, nullptr, stride);
 }
 
-int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int Cin, int Cout, float* part,
+int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int Cin, int Cout, int stride, float* part,
                         size_t part_floats, float* dw) {
   static int32_t* st = nullptr;
   if (!st) NF_CUDA(cudaGetSymbolAddress((void**)&st, g_op_status));
-  return run_wgrad(N, H, W, Cin, Cout, x, g, part, part_floats, dw, st);
+  return run_wgrad(N, H, W, Cin, Cout, x, g, part, part_floats, dw, st, 0, stride);
 }
 
 int nf_tc_op_status(int32_t* out) {

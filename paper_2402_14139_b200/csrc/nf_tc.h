@@ -18,11 +18,11 @@ int nf_tc_wgrad(nf_layer* L, const void* x);
 size_t nf_tc_red_floats(const nf_layer* L);
 // Stand-alone forward on the tensor-core path (NF_EUNSUPPORTED if the shape is not covered) and the
 // status word (nf_device_flag bits) of the stand-alone operations.
-int nf_tc_conv3x3_forward(const void* x, const void* w, int N, int H, int W, int Cin, int Cout, void* y);
+int nf_tc_conv3x3_forward(const void* x, const void* w, int N, int H, int W, int Cin, int Cout, int stride, void* y);
 int nf_tc_op_status(int32_t* out);
 // Stand-alone weight gradient on the tensor-core path and the split-K scratch (floats) it needs (0: shape not covered).
-size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout);
-int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int Cin, int Cout, float* part,
+size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout, int stride);
+int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int Cin, int Cout, int stride, float* part,
                         size_t part_floats, float* dw);
 // Aux conv forward on tensor cores: L->h = ReLU(conv(a, Wa) + ba) in bf16.
 int nf_tc_aux_fwd(nf_layer* L, const void* a);
