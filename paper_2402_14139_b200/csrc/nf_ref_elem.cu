@@ -364,6 +364,166 @@ __global__ void gather_kernel(const uint4* __restrict__ cache, const int32_t* __
   if (k == 0 && out_labels) out_labels[r] = cache_labels[src];
 }
 
+
+// ------------------------------------------------------------------ vectorised bf16 paths (C % 8 == 0, no pool)
+// One thread owns 8 consecutive channels of a pixel: 16-byte loads and stores, coalesced along channels.
+struct bf16x8 { uint4 u; };
+__device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 t = __bfloat1622float2(h[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+__device__ __forceinline__ uint4 pack8(const float (&f)[8]) {
+  uint4 u;
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+  return u;
+}
+
+// out = ReLU(y*scale+shift); grid-stride over (pixel, channel group)
+__global__ void __launch_bounds__(256) bn_apply_vec_kernel(const uint4* __restrict__ y, int C8, const float* __restrict__ scale,
+                                                           const float* __restrict__ shift, size_t total8,
+                                                           uint4* __restrict__ out) {
+  extern __shared__ float cs[];  // scale[C], shift[C]
+  const int C = C8 * 8;
+  for (int i = threadIdx.x; i < C; i += 256) {
+    cs[i] = scale[i];
+    cs[C + i] = shift[i];
+  }
+  __syncthreads();
+  for (size_t e = (size_t)blockIdx.x * 256 + threadIdx.x; e < total8; e += (size_t)gridDim.x * 256) {
+    const int c0 = (int)(e % C8) * 8;
+    float v[8];
+    unpack8(__ldg(y + e), v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = fmaxf(fmaf(v[i], cs[c0 + i], cs[C + c0 + i]), 0.f);
+    out[e] = pack8(v);
+  }
+}
+
+// partial sums of (dz, dz*xhat) with dz = da * 1[y*scale+shift > 0]; red[(block*2+k)*C + c]
+__global__ void __launch_bounds__(256) bn_bwd_reduce_vec_kernel(const uint4* __restrict__ y, const uint4* __restrict__ da,
+                                                                size_t P, int C8, const float* __restrict__ scale,
+                                                                const float* __restrict__ shift, const float* __restrict__ mu,
+                                                                const float* __restrict__ invstd, float* __restrict__ red) {
+  __shared__ float sm[16][256];
+  const int C = C8 * 8;
+  const int planes = 256 / C8, g = threadIdx.x % C8, pl = threadIdx.x / C8;
+  const int c0 = g * 8;
+  float sc[8], sh[8], m[8], is[8], a[8], b[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    sc[i] = scale[c0 + i]; sh[i] = shift[c0 + i]; m[i] = mu[c0 + i]; is[i] = invstd[c0 + i];
+    a[i] = 0.f; b[i] = 0.f;
+  }
+  const size_t p0 = P * blockIdx.x / gridDim.x, p1 = P * (blockIdx.x + 1) / gridDim.x;
+  if (pl < planes)
+    for (size_t p = p0 + pl; p < p1; p += planes) {
+      float yv[8], dv[8];
+      unpack8(__ldg(y + p * C8 + g), yv);
+      unpack8(__ldg(da + p * C8 + g), dv);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float dz = fmaf(yv[i], sc[i], sh[i]) > 0.f ? dv[i] : 0.f;
+        a[i] += dz;
+        b[i] = fmaf(dz, (yv[i] - m[i]) * is[i], b[i]);
+      }
+    }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    sm[i][threadIdx.x] = a[i];
+    sm[8 + i][threadIdx.x] = b[i];
+  }
+  __syncthreads();
+  // thread t < 2*C finishes value k = t / C of channel c = t % C
+  for (int t = threadIdx.x; t < 2 * C; t += 256) {
+    const int k = t / C, c = t % C, gg = c / 8, i = c % 8;
+    float s = 0.f;
+    for (int q = 0; q < planes; ++q) s += sm[k * 8 + i][q * C8 + gg];
+    red[((size_t)blockIdx.x * 2 + k) * C + c] = s;
+  }
+}
+
+// dy = scale * (dz - sum(dz)/M - xhat * sum(dz*xhat)/M)
+__global__ void __launch_bounds__(256) bn_bwd_apply_vec_kernel(const uint4* __restrict__ y, const uint4* __restrict__ da, int C8,
+                                                               const float* __restrict__ scale, const float* __restrict__ shift,
+                                                               const float* __restrict__ mu, const float* __restrict__ invstd,
+                                                               const float* __restrict__ sdz, const float* __restrict__ sdzx,
+                                                               float invM, size_t total8, uint4* __restrict__ dy) {
+  extern __shared__ float cs[];  // per channel: scale, shift, mu, invstd, sdz/M, sdzx/M
+  const int C = C8 * 8;
+  for (int i = threadIdx.x; i < C; i += 256) {
+    cs[i] = scale[i];
+    cs[C + i] = shift[i];
+    cs[2 * C + i] = mu[i];
+    cs[3 * C + i] = invstd[i];
+    cs[4 * C + i] = sdz[i] * invM;
+    cs[5 * C + i] = sdzx[i] * invM;
+  }
+  __syncthreads();
+  for (size_t e = (size_t)blockIdx.x * 256 + threadIdx.x; e < total8; e += (size_t)gridDim.x * 256) {
+    const int c0 = (int)(e % C8) * 8;
+    float yv[8], dv[8], o[8];
+    unpack8(__ldg(y + e), yv);
+    unpack8(__ldg(da + e), dv);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int c = c0 + i;
+      const float dz = fmaf(yv[i], cs[c], cs[C + c]) > 0.f ? dv[i] : 0.f;
+      const float xh = (yv[i] - cs[2 * C + c]) * cs[3 * C + c];
+      o[i] = cs[c] * (dz - cs[4 * C + c] - xh * cs[5 * C + c]);
+    }
+    dy[e] = pack8(o);
+  }
+}
+
+// partial sums of (v, v^2) of a bf16 tensor; same layout of partials as channel_reduce_kernel
+__global__ void __launch_bounds__(256) channel_sums_vec_kernel(const uint4* __restrict__ src, size_t P, int C8,
+                                                               float* __restrict__ red) {
+  __shared__ float sm[16][256];
+  const int C = C8 * 8;
+  const int planes = 256 / C8, g = threadIdx.x % C8, pl = threadIdx.x / C8;
+  float a[8], b[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a[i] = b[i] = 0.f;
+  const size_t p0 = P * blockIdx.x / gridDim.x, p1 = P * (blockIdx.x + 1) / gridDim.x;
+  if (pl < planes)
+    for (size_t p = p0 + pl; p < p1; p += planes) {
+      float v[8];
+      unpack8(__ldg(src + p * C8 + g), v);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        a[i] += v[i];
+        b[i] = fmaf(v[i], v[i], b[i]);
+      }
+    }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    sm[i][threadIdx.x] = a[i];
+    sm[8 + i][threadIdx.x] = b[i];
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < 2 * C; t += 256) {
+    const int k = t / C, c = t % C, gg = c / 8, i = c % 8;
+    float s = 0.f;
+    for (int q = 0; q < planes; ++q) s += sm[k * 8 + i][q * C8 + gg];
+    red[((size_t)blockIdx.x * 2 + k) * C + c] = s;
+  }
+}
+
+inline bool vec_ok(int dtype, int C, int pool) { return dtype == NF_BF16 && C % 8 == 0 && C <= 1024 && !pool; }
+inline int vec_blocks(size_t work_items) {
+  size_t b = (work_items + 256 * 8 - 1) / (256 * 8);
+  if (b < 1) b = 1;
+  if (b > 148 * 8) b = 148 * 8;
+  return (int)b;
+}
+
 inline unsigned nblk(size_t n, int per) { return (unsigned)((n + per - 1) / per); }
 
 }  // namespace
@@ -384,6 +544,12 @@ int nf_ref_channel_blocks(size_t P, int C) {
 int nf_ref_channel_sums(int dtype, const void* src, size_t P, int C, float* red, size_t red_floats, int* nblocks) {
   const int nb = nf_ref_channel_blocks(P, C);
   if ((size_t)nb * 2 * C > red_floats) return NF_ENOWS;
+  if (vec_ok(dtype, C, 0) && 256 % (C / 8) == 0) {
+    channel_sums_vec_kernel<<<nb, 256, 0, g_nf_stream>>>((const uint4*)src, P, C / 8, red);
+    NF_LAUNCHED();
+    *nblocks = nb;
+    return NF_OK;
+  }
   DISPATCH(dtype,
            (channel_reduce_kernel<float, StatsFn><<<nb, 256, 0, g_nf_stream>>>((const float*)src, nullptr, P, C, StatsFn(), red)),
            (channel_reduce_kernel<bf16, StatsFn><<<nb, 256, 0, g_nf_stream>>>((const bf16*)src, nullptr, P, C, StatsFn(), red)));
@@ -411,6 +577,12 @@ int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float ep
 int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
                     const float* shift, void* out) {
   const size_t total = (size_t)N * (pool ? Ho / 2 : Ho) * (pool ? Wo / 2 : Wo) * C;
+  if (vec_ok(dtype, C, pool)) {
+    bn_apply_vec_kernel<<<vec_blocks(total / 8), 256, 2 * C * sizeof(float), g_nf_stream>>>((const uint4*)y, C / 8, scale, shift,
+                                                                                         total / 8, (uint4*)out);
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   DISPATCH(dtype,
            (bn_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, Ho, Wo, C, pool, scale, shift, total, (float*)out)),
            (bn_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, Ho, Wo, C, pool, scale, shift, total, (bf16*)out)));
@@ -461,6 +633,12 @@ int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho
   const size_t P = (size_t)N * Ho * Wo;
   const int nb = nf_ref_channel_blocks(P, C);
   if ((size_t)nb * 2 * C > red_floats) return NF_ENOWS;
+  if (vec_ok(dtype, C, pool) && 256 % (C / 8) == 0) {
+    bn_bwd_reduce_vec_kernel<<<nb, 256, 0, g_nf_stream>>>((const uint4*)y, (const uint4*)da, P, C / 8, scale, shift, mu, invstd, red);
+    NF_LAUNCHED();
+    *nblocks = nb;
+    return NF_OK;
+  }
   BnBwdFn fn{Ho, Wo, pool, scale, shift, mu, invstd};
   DISPATCH(dtype,
            (channel_reduce_kernel<float, BnBwdFn><<<nb, 256, 0, g_nf_stream>>>((const float*)y, (const float*)da, P, C, fn, red)),
@@ -482,6 +660,12 @@ int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho,
                         const float* sdz, const float* sdzx, double M, void* dy) {
   const size_t total = (size_t)N * Ho * Wo * C;
   const float invM = (float)(1.0 / M);
+  if (vec_ok(dtype, C, pool)) {
+    bn_bwd_apply_vec_kernel<<<vec_blocks(total / 8), 256, 6 * C * sizeof(float), g_nf_stream>>>(
+        (const uint4*)y, (const uint4*)da, C / 8, scale, shift, mu, invstd, sdz, sdzx, invM, total / 8, (uint4*)dy);
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   DISPATCH(dtype,
            (bn_bwd_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, (const float*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (float*)dy)),
            (bn_bwd_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, (const bf16*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (bf16*)dy)));
