@@ -121,7 +121,7 @@ def run_ours(args, rank, world):
     wl = workloads.ALL[args.workload]()
     bi = 0
     N, ls = wl["blocks"][bi]
-    seed = 0x4E460000 + int(args.workload[1]) + 1000 * rank
+    seed = 0x4E460000 + int(args.workload[1]) + 1000 * rank + (50 if args.workload.endswith("s") else 0)
     es = 4 if wl["dtype"] == "f32" else 2
     tdt = torch.float32 if es == 4 else torch.bfloat16
     stream = torch.cuda.current_stream()
@@ -256,7 +256,7 @@ def run_reference(args):
     """The reference arm: the CPU checker on the host cores, same metric and workload."""
     from paper_2402_14139_b200 import workloads
     wl = workloads.ALL[args.workload]()
-    n_sample = 1 if args.workload == "c4" else min(8, wl["blocks"][0][0])
+    n_sample = 1 if args.workload.startswith("c4") else min(8, wl["blocks"][0][0])
     oracle_sample(wl, 0, n_sample, 1, steps=max(0, min(args.warmup, 1)))
     times, cores = oracle_sample(wl, 0, n_sample, 2, steps=args.steps)
     total = sum(times)
@@ -276,7 +276,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c4", choices=["c2", "c4"])
+    ap.add_argument("--workload", default="c4", choices=["c2", "c4", "c4s"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -289,7 +289,7 @@ def main():
     out, wl, bi = run_ours(args, rank, world)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            n_sample = 4 if args.workload == "c4" else wl["blocks"][bi][0]
+            n_sample = 4 if args.workload.startswith("c4") else wl["blocks"][bi][0]
             times, cores = oracle_sample(wl, bi, n_sample, 3)
             out["cpu_baseline"] = dict(value=round(n_sample / times[0], 4), unit="images/s", cores=cores, kind="oracle",
                                        sample=f"one step of {n_sample} images through all layers of the block "

@@ -54,6 +54,14 @@ def c4():
     return dict(name="c4", dtype="bf16", classes=1000, in_shape=(64, 224, 224), blocks=[(64, ls)])
 
 
+def c4s():
+    """c4 with batch 24 (input 154 MB, still larger than L2): the case profiler captures run on."""
+    d = c4()
+    d["name"] = "c4s"
+    d["blocks"] = [(24, d["blocks"][0][1])]
+    return d
+
+
 VGG16 = [64, 64, "P", 128, 128, "P", 256, 256, 256, "P", 512, 512, 512, "P", 512, 512, 512, "P"]
 
 
@@ -101,4 +109,4 @@ def step_flops(l, N):
     return dict(conv_fwd=main, wgrad=main, aux_fwd=aux, aux_bwd=2 * aux)
 
 
-ALL = dict(c1=c1, c2=c2, c3=c3, c4=c4, c5=c5)
+ALL = dict(c1=c1, c2=c2, c3=c3, c4=c4, c5=c5, c4s=c4s)
