@@ -31,7 +31,7 @@ struct FwdParams {
 };
 
 struct TcPlan {
-  int ok, BW, BH, BN, KC, stages, grid, parts;
+  int ok, BW, BH, BN, KC, RW, stages, grid, parts;
   size_t smem;
 };
 
@@ -44,7 +44,9 @@ struct TcPlan {
 //       taps mirrored, which makes the same kernel the input-gradient convolution da = dh (*) Wa^T.
 // PT  : 1 = one TMA box per tap (stride-2 convolution: the box is gathered with element stride 2, so the
 //       three row taps cannot share a box); p.H, p.W are then the OUTPUT sizes.
-template <int BN, int EPI, int KC = 64, int BMN = 0, int PT = 0>
+// RW  : 1 = all nine weight tiles of the CTA's channel tile stay resident in shared memory for the whole
+//       kernel (single 64-channel K chunk, 9*BN*128 bytes); the pipeline then carries activations only.
+template <int BN, int EPI, int KC = 64, int BMN = 0, int PT = 0, int RW = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_y, const FwdParams p) {
@@ -54,16 +56,19 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   constexpr uint32_t kALayout = KC == 64 ? 2 : KC == 32 ? 4 : 6;
   const int a_bytes = (PT ? p.BH : p.BH + 2) * p.BW * kARow;
   const int a_stride = (a_bytes + 1023) & ~1023;  // keeps the weight tiles 1024-byte aligned
-  constexpr int b_bytes = PT ? BN * 128 : BMN ? (BN / 64) * 3 * KC * 128 : 3 * BN * 128;
+  constexpr int b_bytes = RW ? 0 : PT ? BN * 128 : BMN ? (BN / 64) * 3 * KC * 128 : 3 * BN * 128;
+  constexpr int w_bytes = RW ? 9 * BN * 128 : 0;  // resident weights [kw][kh][BN][64]
   const int stage_bytes = a_stride + b_bytes;
   constexpr int kSub = EPI == 0 ? BN / 64 : 0;  // 64-channel sub-tiles of the output staging
-  uint8_t* stg = smem + (size_t)p.stages * stage_bytes;
+  uint8_t* wres = smem + (size_t)p.stages * stage_bytes;
+  uint8_t* stg = wres + w_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(stg + kSub * 16384);
   uint64_t* full = bars;
   uint64_t* empty = bars + kMaxStages;
   uint64_t* tfull = bars + 2 * kMaxStages;
   uint64_t* tempty = tfull + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+  uint64_t* wfull = tempty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wfull + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
@@ -79,6 +84,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       ptx::mbar_init(&tfull[a], 1);
       ptx::mbar_init(&tempty[a], 128);
     }
+    ptx::mbar_init(wfull, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tmap(&tm_x);
@@ -99,6 +105,14 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     // ---------------- producer: one TMA box of activations + three weight tiles per k-step
     uint32_t it = 0;
     bool ok = true;
+    if constexpr (RW) {
+      if (lane == 0 && blockIdx.x < p.total_tiles) {
+        ptx::mbar_expect_tx(wfull, (uint32_t)w_bytes);
+#pragma unroll
+        for (int kw = 0; kw < 3; ++kw) ptx::tma_load_4d(wres + kw * 3 * BN * 128, &tm_w, wfull, 0, (blockIdx.x % p.n_tiles) * BN, kw, 0);
+      }
+      __syncwarp();
+    }
     for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x) {
       const int nt = t % p.n_tiles, m = t / p.n_tiles;
       const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = m / (p.tiles_w * p.tiles_h);
@@ -120,7 +134,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 #pragma unroll
               for (int hf = 0; hf < BN / 64; ++hf)  // [half][kh][KC rows of f][64 channels], mirrored column tap
                 ptx::tma_load_4d(a_s + a_stride + hf * 3 * KC * 128, &tm_w, &full[s], nt * BN + hf * 64, 0, 2 - kw, 0);
-            } else {
+            } else if constexpr (!RW) {
               ptx::tma_load_4d(a_s + a_stride, &tm_w, &full[s], ck * 64, nt * BN, kw, 0);
             }
           }
@@ -133,6 +147,13 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     constexpr uint32_t idesc = ptx::idesc_bf16(128, BN, 0, BMN);
     uint32_t it = 0, tl = 0;
     bool ok = true;
+    // descriptors differ only in their 14-bit address field: constant upper parts, address added per use
+    const uint64_t a_hi = ptx::sdesc(0, 16, 8 * kARow, kALayout);
+    const uint64_t b_hi = BMN ? ptx::sdesc(0, 3 * KC * 128, 1024, 2) : ptx::sdesc(0, 16, 1024, 2);
+    const uint32_t a_row16 = (uint32_t)(p.BW * kARow) >> 4;  // one image row of the box, in 16-byte units
+    if constexpr (RW) {
+      if (blockIdx.x < p.total_tiles) ok = __all_sync(0xffffffffu, ptx::mbar_wait(wfull, 0, abort_flag));
+    }
     for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++tl) {
       const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(&tempty[acc], aph ^ 1, abort_flag))) break;
@@ -145,14 +166,15 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         ptx::tc_fence_after();
         if (lane == 0) {
           const uint32_t a_base = ptx::smem_u32(smem + (size_t)s * stage_bytes);
-          const uint32_t b_base = a_base + a_stride;
+          const uint32_t a16 = a_base >> 4;
+          const uint32_t b16 = RW ? (ptx::smem_u32(wres) + (ks % 3) * 3 * BN * 128) >> 4 : (a_base + a_stride) >> 4;
 #pragma unroll
           for (int kh = 0; kh < (PT ? 1 : 3); ++kh)
 #pragma unroll
             for (int k = 0; k < KC / 16; ++k) {
-              const uint64_t ad = ptx::sdesc(a_base + kh * p.BW * kARow + k * 32, 16, 8 * kARow, kALayout);
-              const uint64_t bd = BMN ? ptx::sdesc_sw128(b_base + (2 - kh) * KC * 128 + k * 16 * 128, 3 * KC * 128, 1024)
-                                      : ptx::sdesc_sw128(b_base + kh * BN * 128 + k * 32, 16, 1024);
+              const uint64_t ad = a_hi | (uint64_t)(a16 + kh * a_row16 + k * 2);
+              const uint64_t bd = b_hi | (uint64_t)(BMN ? b16 + (((2 - kh) * KC * 128 + k * 16 * 128) >> 4)
+                                                        : b16 + ((kh * BN * 128 + k * 32) >> 4));
               ptx::mma_f16(d, ad, bd, idesc, (ks | kh | k) != 0);
             }
           ptx::mma_commit(&empty[s]);
@@ -404,26 +426,30 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       ptx::tc_fence_after();
       if (lane == 0) {
         const uint32_t xb = ptx::smem_u32(smem + (size_t)s * stage_bytes);
-        const uint32_t gb = xb + 3 * copy_bytes;
-        const uint32_t row = p.BW * 128;  // bytes of one image row of the box
+        const uint32_t x16 = xb >> 4, g16 = (xb + 3 * copy_bytes) >> 4;
+        const uint32_t row16 = (uint32_t)(p.BW * 128) >> 4, copy16 = (uint32_t)copy_bytes >> 4;
+        // descriptors differ only in the address field; the leading-dimension offset selects what is stacked
+        const uint64_t a_row_hi = ptx::sdesc(0, p.BW * 128, 1024, 2);   // second chunk one image row further
+        const uint64_t a_copy_hi = ptx::sdesc(0, copy_bytes, 1024, 2);  // second chunk one box / tile further
+        const uint64_t b_hi = ptx::sdesc(0, 16, 8 * kBRow, kBLayout);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          const uint32_t koff = k * 16 * 128;  // 16 pixels per instruction
-          const uint64_t bd = ptx::sdesc(gb + k * 16 * kBRow, 16, 8 * kBRow, kBLayout);
+          const uint32_t k16 = k * 128;  // 16 pixels x 128 bytes, in 16-byte units
+          const uint64_t bd = b_hi | (uint64_t)(g16 + k * kBRow);
           const uint32_t acc = (it | k) != 0;
           if constexpr (S2) {
             // taps (kh,0) and (kh,1): second chunk one tile further; tap (kh,2): rows 64..127 unused
-            ptx::mma_f16(tmem_base, ptx::sdesc_sw128(xb + koff, copy_bytes, 1024), bd, idesc, acc);
-            ptx::mma_f16(tmem_base + NB, ptx::sdesc_sw128(xb + 2 * copy_bytes + koff, copy_bytes, 1024), bd, idesc, acc);
+            ptx::mma_f16(tmem_base, a_copy_hi | (uint64_t)(x16 + k16), bd, idesc, acc);
+            ptx::mma_f16(tmem_base + NB, a_copy_hi | (uint64_t)(x16 + 2 * copy16 + k16), bd, idesc, acc);
           } else {
 #pragma unroll
             for (int kw = 0; kw < 3; ++kw)  // taps (kh=0,kw) and (kh=1,kw): second chunk one image row further
-              ptx::mma_f16(tmem_base + kw * NB, ptx::sdesc_sw128(xb + kw * copy_bytes + koff, row, 1024), bd, idesc, acc);
+              ptx::mma_f16(tmem_base + kw * NB, a_row_hi | (uint64_t)(x16 + kw * copy16 + k16), bd, idesc, acc);
             // taps (kh=2,kw=0) and (kh=2,kw=1): second chunk one box further
-            ptx::mma_f16(tmem_base + 3 * NB, ptx::sdesc_sw128(xb + 2 * row + koff, copy_bytes, 1024), bd, idesc, acc);
+            ptx::mma_f16(tmem_base + 3 * NB, a_copy_hi | (uint64_t)(x16 + 2 * row16 + k16), bd, idesc, acc);
             // tap (kh=2,kw=2); rows 64..127 of this accumulator are not used (their operand rows fall on the
             // rows after the box, which are still inside this stage's buffer)
-            ptx::mma_f16(tmem_base + 4 * NB, ptx::sdesc_sw128(xb + 2 * copy_bytes + 2 * row + koff, row, 1024), bd, idesc, acc);
+            ptx::mma_f16(tmem_base + 4 * NB, a_row_hi | (uint64_t)(x16 + 2 * copy16 + 2 * row16 + k16), bd, idesc, acc);
           }
         }
         ptx::mma_commit(&empty[s]);
@@ -553,9 +579,10 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride 
   pl.BN = epi != 1 ? (Cout % 128 == 0 ? 128 : 64) : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64);
   pl.KC = epi == 2 ? (Cin <= 16 ? 16 : Cin <= 32 ? 32 : 64) : 64;
   const size_t a_stride = ((size_t)(stride == 2 ? pl.BH : pl.BH + 2) * pl.BW * pl.KC * 2 + 1023) & ~(size_t)1023;
-  const size_t stage = a_stride + (stride == 2 ? (size_t)pl.BN * 128
+  pl.RW = (stride == 1 && epi != 2 && Cin == 64 && pl.BN <= 64) ? 1 : 0;  // weights resident in shared memory
+  const size_t stage = a_stride + (pl.RW ? 0 : stride == 2 ? (size_t)pl.BN * 128
                                                : epi == 2 ? (size_t)(pl.BN / 64) * 3 * pl.KC * 128 : (size_t)3 * pl.BN * 128);
-  const size_t fixed = (size_t)(epi != 1 ? pl.BN / 64 : 0) * 16384 + 1024 + 1024;  // staging + barriers + alignment slack
+  const size_t fixed = (size_t)(epi != 1 ? pl.BN / 64 : 0) * 16384 + (pl.RW ? (size_t)9 * pl.BN * 128 : 0) + 1024 + 1024;
   int st = (int)((232448 - fixed) / stage);
   if (st > kMaxStages) st = kMaxStages;
   if (st < 2) return pl;
@@ -573,14 +600,14 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride 
   return pl;
 }
 
-template <int BN, int EPI, int KC = 64, int BMN = 0, int PT = 0>
+template <int BN, int EPI, int KC = 64, int BMN = 0, int PT = 0, int RW = 0>
 int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const FwdParams& p) {
   static bool attr_done = false;
   if (!attr_done) {
-    NF_CUDA(cudaFuncSetAttribute(conv_fwd_tc_kernel<BN, EPI, KC, BMN, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    NF_CUDA(cudaFuncSetAttribute(conv_fwd_tc_kernel<BN, EPI, KC, BMN, PT, RW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
   }
-  conv_fwd_tc_kernel<BN, EPI, KC, BMN, PT><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mw, my, p);
+  conv_fwd_tc_kernel<BN, EPI, KC, BMN, PT, RW><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mw, my, p);
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -623,7 +650,11 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
   }
   if (epi == 0 && stride == 2)
     return pl.BN == 128 ? launch_fwd<128, 0, 64, 0, 1>(pl, mx, mw, my, p) : launch_fwd<64, 0, 64, 0, 1>(pl, mx, mw, my, p);
+  if (epi == 0 && pl.RW) return launch_fwd<64, 0, 64, 0, 0, 1>(pl, mx, mw, my, p);
   if (epi == 0) return pl.BN == 128 ? launch_fwd<128, 0>(pl, mx, mw, my, p) : launch_fwd<64, 0>(pl, mx, mw, my, p);
+  if (epi == 1 && pl.RW)
+    return pl.BN == 16 ? launch_fwd<16, 1, 64, 0, 0, 1>(pl, mx, mw, my, p)
+                       : pl.BN == 32 ? launch_fwd<32, 1, 64, 0, 0, 1>(pl, mx, mw, my, p) : launch_fwd<64, 1, 64, 0, 0, 1>(pl, mx, mw, my, p);
   if (epi == 2) {
     if (pl.BN == 128)
       return pl.KC == 16 ? launch_fwd<128, 0, 16, 1>(pl, mx, mw, my, p)
