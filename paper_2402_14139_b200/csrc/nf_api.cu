@@ -321,21 +321,36 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
   }
   trace_end();
   trace_begin(3);
-  NF_TRY(nf_ref_avgpool(dt, L->h, N, Ha, Wa, F, L->p));
+  {
+    int rc = dt == NF_BF16 ? nf_ref_avgpool_fast(L->h, N, Ha, Wa, F, L->wpart, L->wpart_floats, L->p) : NF_EUNSUPPORTED;
+    if (rc == NF_EUNSUPPORTED) rc = nf_ref_avgpool(dt, L->h, N, Ha, Wa, F, L->p);
+    if (rc != NF_OK) return rc;
+  }
   NF_TRY(nf_ref_fc_ce(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits,
                       L->dp, L->lossn, L->status));
   // gradients of gamma_n, beta_n
   NF_TRY(nf_ref_fc_wgrad(L->p, L->dlogits, L->lossn, N, D, K, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->status));
   trace_end();
   trace_begin(4);
-  NF_TRY(nf_ref_dh(dt, L->h, L->dp, N, Ha, Wa, F, L->dh));
+  int dh_nb = 0;
+  {
+    int rc = dt == NF_BF16 ? nf_ref_dh_fast(L->h, L->dp, N, Ha, Wa, F, L->dh, L->red, L->red_floats, &dh_nb) : NF_EUNSUPPORTED;
+    if (rc == NF_EUNSUPPORTED) {
+      dh_nb = 0;
+      rc = nf_ref_dh(dt, L->h, L->dp, N, Ha, Wa, F, L->dh);
+    }
+    if (rc != NF_OK) return rc;
+  }
+  if (dh_nb) NF_TRY(nf_ref_sum_partials(L->red, dh_nb, F, 0, g + L->off[NF_P_BA]));
   if (L->fam[3]) {
     NF_TRY(nf_tc_aux_wgrad(L, act_out));
   } else {
     NF_TRY(nf_ref_wgrad(dt, act_out, N, Ha, Wa, Co, L->dh, F, 1, L->wpart, L->wpart_floats, g + L->off[NF_P_WA]));
   }
-  NF_TRY(nf_ref_channel_sums(dt, L->dh, (size_t)N * Ha * Wa, F, L->red, L->red_floats, &nb));
-  NF_TRY(nf_ref_sum_partials(L->red, nb, F, 0, g + L->off[NF_P_BA]));
+  if (!dh_nb) {
+    NF_TRY(nf_ref_channel_sums(dt, L->dh, (size_t)N * Ha * Wa, F, L->red, L->red_floats, &nb));
+    NF_TRY(nf_ref_sum_partials(L->red, nb, F, 0, g + L->off[NF_P_BA]));
+  }
   // gradient at the aux input
   if (L->fam[3]) {
     NF_TRY(nf_tc_aux_dgrad(L));

@@ -92,6 +92,10 @@ int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float ep
 int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
                     const float* shift, void* out);
 int nf_ref_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p);
+// bf16 fast paths (F % 8 == 0, even Ha and Wa); NF_EUNSUPPORTED means "use the generic kernel"
+int nf_ref_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part, size_t part_floats, float* p);
+int nf_ref_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh, float* red, size_t red_floats,
+                   int* nblocks);
 int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
                  float* logits, float* dlogits, float* dp, float* lossn, int32_t* status);
 int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,

@@ -516,6 +516,88 @@ __global__ void __launch_bounds__(256) channel_sums_vec_kernel(const uint4* __re
   }
 }
 
+
+// dh = 1[h>0] * dp[n][f*4+bin]/|bin| for even sizes (every pixel lies in exactly one bin), 8 filters per
+// thread, fused with the per-filter sum of dh (the aux bias gradient): red[(block*2+0)*F + f].
+__global__ void __launch_bounds__(256) dh_vec_kernel(const uint4* __restrict__ h, const float* __restrict__ dp, int Ha, int Wa,
+                                                     int F8, size_t P, uint4* __restrict__ dh, float* __restrict__ red) {
+  __shared__ float sm[8][256];
+  const int F = F8 * 8;
+  const int planes = 256 / F8, g = threadIdx.x % F8, pl = threadIdx.x / F8;
+  const float inv_bin = 1.f / (float)((Ha / 2) * (Wa / 2));
+  float a[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a[i] = 0.f;
+  const size_t p0 = P * blockIdx.x / gridDim.x, p1 = P * (blockIdx.x + 1) / gridDim.x;
+  for (size_t p = p0 + pl; p < p1; p += planes) {
+    const int j = (int)(p % Wa), i = (int)((p / Wa) % Ha);
+    const size_t n = p / ((size_t)Wa * Ha);
+    const int bin = (i >= Ha / 2 ? 2 : 0) + (j >= Wa / 2 ? 1 : 0);
+    float hv[8], o[8];
+    unpack8(__ldg(h + p * F8 + g), hv);
+    const float* d = dp + n * 4 * F + (size_t)(g * 8) * 4 + bin;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      o[e] = hv[e] > 0.f ? d[e * 4] * inv_bin : 0.f;
+    }
+    const uint4 packed = pack8(o);
+    dh[p * F8 + g] = packed;
+    float r[8];
+    unpack8(packed, r);  // the bias gradient sums the values as stored
+#pragma unroll
+    for (int e = 0; e < 8; ++e) a[e] += r[e];
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) sm[e][threadIdx.x] = a[e];
+  __syncthreads();
+  for (int t = threadIdx.x; t < F; t += 256) {
+    const int gg = t / 8, e = t % 8;
+    float s = 0.f;
+    for (int q = 0; q < planes; ++q) s += sm[e][q * F8 + gg];
+    red[((size_t)blockIdx.x * 2 + 0) * F + t] = s;
+    red[((size_t)blockIdx.x * 2 + 1) * F + t] = 0.f;
+  }
+}
+
+// average pool, stage 1: partial bin sums over a slice of rows; part[(n*4+bin)*S + s][F]
+__global__ void __launch_bounds__(256) avgpool_part_vec_kernel(const uint4* __restrict__ h, int Ha, int Wa, int F8, int S,
+                                                               float* __restrict__ part) {
+  __shared__ float sm[8][256];
+  const int F = F8 * 8;
+  const int planes = 256 / F8, g = threadIdx.x % F8, pl = threadIdx.x / F8;
+  const int sidx = blockIdx.x % S, bin = (blockIdx.x / S) % 4, n = blockIdx.x / (4 * S);
+  const int bh = Ha / 2, bw = Wa / 2, i0 = (bin >> 1) * bh, j0 = (bin & 1) * bw;
+  const int cnt = bh * bw, k0 = (int)((long)cnt * sidx / S), k1 = (int)((long)cnt * (sidx + 1) / S);
+  float a[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a[i] = 0.f;
+  for (int k = k0 + pl; k < k1; k += planes) {
+    const int i = i0 + k / bw, j = j0 + k % bw;
+    float v[8];
+    unpack8(__ldg(h + (((size_t)n * Ha + i) * Wa + j) * F8 + g), v);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) a[e] += v[e];
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) sm[e][threadIdx.x] = a[e];
+  __syncthreads();
+  for (int t = threadIdx.x; t < F; t += 256) {
+    const int gg = t / 8, e = t % 8;
+    float s = 0.f;
+    for (int q = 0; q < planes; ++q) s += sm[e][q * F8 + gg];
+    part[(size_t)blockIdx.x * F + t] = s;
+  }
+}
+// stage 2: p[n][f*4+bin] = sum over slices / |bin|
+__global__ void avgpool_finish_kernel(const float* __restrict__ part, int N, int F, int S, float inv_cnt, float* __restrict__ p) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= N * 4 * F) return;
+  const int f = e % F, bin = (e / F) % 4, n = e / (4 * F);
+  float s = 0.f;
+  for (int k = 0; k < S; ++k) s += part[((size_t)(n * 4 + bin) * S + k) * F + f];
+  p[(size_t)n * 4 * F + f * 4 + bin] = s * inv_cnt;
+}
+
 inline bool vec_ok(int dtype, int C, int pool) { return dtype == NF_BF16 && C % 8 == 0 && C <= 1024 && !pool; }
 inline int vec_blocks(size_t work_items) {
   size_t b = (work_items + 256 * 8 - 1) / (256 * 8);
@@ -587,6 +669,38 @@ int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int 
            (bn_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, Ho, Wo, C, pool, scale, shift, total, (float*)out)),
            (bn_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, Ho, Wo, C, pool, scale, shift, total, (bf16*)out)));
   NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_avgpool_slices(int N, int Ha, int Wa) {
+  const long cnt = (long)(Ha / 2) * (Wa / 2);
+  long S = 1184 / ((long)N * 4);
+  if (S > cnt / 64) S = cnt / 64;
+  if (S < 1) S = 1;
+  return (int)S;
+}
+
+int nf_ref_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part, size_t part_floats, float* p) {
+  if (F % 8 || 256 % (F / 8) || (Ha & 1) || (Wa & 1)) return NF_EUNSUPPORTED;
+  const int S = nf_ref_avgpool_slices(N, Ha, Wa);
+  if ((size_t)N * 4 * S * F > part_floats) return NF_EUNSUPPORTED;
+  avgpool_part_vec_kernel<<<N * 4 * S, 256, 0, g_nf_stream>>>((const uint4*)h, Ha, Wa, F / 8, S, part);
+  NF_LAUNCHED();
+  avgpool_finish_kernel<<<nblk((size_t)N * 4 * F, 256), 256, 0, g_nf_stream>>>(part, N, F, S, 1.f / (float)((Ha / 2) * (Wa / 2)), p);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+// dh with the fused aux-bias gradient partials (bf16, F % 8 == 0, even sizes); nblocks partials in red
+int nf_ref_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh, float* red, size_t red_floats,
+                   int* nblocks) {
+  if (F % 8 || 256 % (F / 8) || (Ha & 1) || (Wa & 1)) return NF_EUNSUPPORTED;
+  const size_t P = (size_t)N * Ha * Wa;
+  const int nb = nf_ref_channel_blocks(P, F);
+  if ((size_t)nb * 2 * F > red_floats) return NF_EUNSUPPORTED;
+  dh_vec_kernel<<<nb, 256, 0, g_nf_stream>>>((const uint4*)h, dp, Ha, Wa, F / 8, P, (uint4*)dh, red);
+  NF_LAUNCHED();
+  *nblocks = nb;
   return NF_OK;
 }
 
