@@ -89,16 +89,37 @@ __global__ void __launch_bounds__(256) channel_reduce_kernel(const T* __restrict
   }
 }
 
+
+// Sums the per-block partials of 32 consecutive channels: block (32 channels x 32 lanes over the partials),
+// fp64, fixed order.  Returns the two totals to the threads with threadIdx.y == 0.
+__device__ __forceinline__ void reduce_partials32(const float* __restrict__ red, int nb, int C, double& S, double& Q) {
+  __shared__ double sm[2][32][33];
+  const int c = blockIdx.x * 32 + threadIdx.x;
+  double a = 0.0, b = 0.0;
+  if (c < C)
+    for (int k = threadIdx.y; k < nb; k += 32) {
+      a += (double)red[((size_t)k * 2 + 0) * C + c];
+      b += (double)red[((size_t)k * 2 + 1) * C + c];
+    }
+  sm[0][threadIdx.y][threadIdx.x] = a;
+  sm[1][threadIdx.y][threadIdx.x] = b;
+  __syncthreads();
+  S = 0.0;
+  Q = 0.0;
+  if (threadIdx.y == 0)
+    for (int k = 0; k < 32; ++k) {
+      S += sm[0][k][threadIdx.x];
+      Q += sm[1][k][threadIdx.x];
+    }
+}
+
 __global__ void bn_finalize_kernel(const float* __restrict__ red, int nb, int C, double M, const float* __restrict__ gamma,
                                    const float* __restrict__ beta, float eps, float bnm, float* scale, float* shift,
                                    float* mu, float* invstd, float* rmean, float* rvar) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= C) return;
-  double S = 0.0, Q = 0.0;
-  for (int b = 0; b < nb; ++b) {
-    S += (double)red[((size_t)b * 2 + 0) * C + c];
-    Q += (double)red[((size_t)b * 2 + 1) * C + c];
-  }
+  double S, Q;
+  reduce_partials32(red, nb, C, S, Q);
+  const int c = blockIdx.x * 32 + threadIdx.x;
+  if (c >= C || threadIdx.y != 0) return;
   const double m = S / M;
   double v = Q / M - m * m;
   if (v < 0.0) v = 0.0;
@@ -298,22 +319,19 @@ __global__ void dh_kernel(const T* __restrict__ h, const float* __restrict__ dp,
 }
 
 __global__ void sum_partials_kernel(const float* __restrict__ red, int nb, int C, int which, float* __restrict__ out) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= C) return;
-  double s = 0.0;
-  for (int b = 0; b < nb; ++b) s += (double)red[((size_t)b * 2 + which) * C + c];
-  out[c] = (float)s;
+  double S, Q;
+  reduce_partials32(red, nb, C, S, Q);
+  const int c = blockIdx.x * 32 + threadIdx.x;
+  if (c >= C || threadIdx.y != 0) return;
+  out[c] = (float)(which ? Q : S);
 }
 
 __global__ void bn_bwd_finalize_kernel(const float* __restrict__ red, int nb, int C, float* sdz, float* sdzx, float* gg,
                                        float* gb) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= C) return;
-  double a = 0.0, b = 0.0;
-  for (int k = 0; k < nb; ++k) {
-    a += (double)red[((size_t)k * 2 + 0) * C + c];
-    b += (double)red[((size_t)k * 2 + 1) * C + c];
-  }
+  double a, b;
+  reduce_partials32(red, nb, C, a, b);
+  const int c = blockIdx.x * 32 + threadIdx.x;
+  if (c >= C || threadIdx.y != 0) return;
   sdz[c] = (float)a;
   sdzx[c] = (float)b;
   gb[c] = (float)a;
@@ -643,7 +661,7 @@ int nf_ref_channel_sums(int dtype, const void* src, size_t P, int C, float* red,
 int nf_ref_bn_finalize(const float* red, int nblocks, int C, double M, const float* gamma, const float* beta,
                        float eps, float bn_momentum, float* scale, float* shift, float* mu, float* invstd,
                        float* rmean, float* rvar) {
-  bn_finalize_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(red, nblocks, C, M, gamma, beta, eps, bn_momentum, scale,
+  bn_finalize_kernel<<<nblk(C, 32), dim3(32, 32), 0, g_nf_stream>>>(red, nblocks, C, M, gamma, beta, eps, bn_momentum, scale,
                                                             shift, mu, invstd, rmean, rvar);
   NF_LAUNCHED();
   return NF_OK;
@@ -736,7 +754,7 @@ int nf_ref_dh(int dtype, const void* h, const float* dp, int N, int Ha, int Wa, 
 }
 
 int nf_ref_sum_partials(const float* red, int nblocks, int C, int which, float* out) {
-  sum_partials_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(red, nblocks, C, which, out);
+  sum_partials_kernel<<<nblk(C, 32), dim3(32, 32), 0, g_nf_stream>>>(red, nblocks, C, which, out);
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -764,7 +782,7 @@ int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho
 
 int nf_ref_bn_bwd_finalize(const float* red, int nblocks, int C, float* sdz, float* sdzx, float* ggamma,
                            float* gbeta) {
-  bn_bwd_finalize_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(red, nblocks, C, sdz, sdzx, ggamma, gbeta);
+  bn_bwd_finalize_kernel<<<nblk(C, 32), dim3(32, 32), 0, g_nf_stream>>>(red, nblocks, C, sdz, sdzx, ggamma, gbeta);
   NF_LAUNCHED();
   return NF_OK;
 }
