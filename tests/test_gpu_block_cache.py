@@ -1,0 +1,112 @@
+"""GPU tests of the block-level calls: nf_block_step chains layer steps, nf_block_cache is the eval-mode
+forward the checker computes (and is per-sample), nf_cache_gather re-batches bit-exactly."""
+import numpy as np
+import pytest
+
+from paper_2402_14139_b200 import synth
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2402_14139_b200 import nf
+    nf.lib()
+    nf.nf_set_stream(None)
+    return nf, torch
+
+
+def _two_layer(nf, torch, dtype, N, seed, pool_first=True, C=64, F=16):
+    c1 = dict(N=N, Cin=C, Cout=C, H=16, W=16, F=F, classes=10, stride=1, pool=pool_first)
+    hw = 8 if pool_first else 16
+    c2 = dict(N=N, Cin=C, Cout=2 * C, H=hw, W=hw, F=8, classes=10, stride=1, pool=False)
+    cases = []
+    for k, c in enumerate((c1, c2)):
+        P, x, y = pu.seeded_case(c, seed + k, bf16=(dtype == 1))
+        cases.append((c, P, x, y))
+    return cases
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_block_step_equals_chained_layer_steps(env, dtype):
+    nf, torch = env
+    cases = _two_layer(nf, torch, dtype, 6, 700)
+    A = [pu.gpu_layer(nf, c, P, dtype) for c, P, _, _ in cases]
+    B = [pu.gpu_layer(nf, c, P, dtype) for c, P, _, _ in cases]
+    blk = nf.Block(B)
+    x = pu.to_device_nhwc(torch, cases[0][2], dtype)
+    lab = torch.from_numpy(cases[0][3]).cuda()
+    la = torch.zeros(2, device="cuda")
+    a1, a2 = A[0].new_act(), A[1].new_act()
+    A[0].step(x, lab, 0.01, la[0:1], a1)
+    A[1].step(a1, lab, 0.01, la[1:2], a2)
+    lb = torch.zeros(2, device="cuda")
+    b2 = B[1].new_act()
+    blk.step(x, lab, 0.01, lb, b2)
+    torch.cuda.synchronize()
+    assert torch.equal(la, lb) and torch.equal(a2, b2)
+    for k in range(2):
+        for name in pu.PNAMES:
+            assert np.array_equal(A[k].get_param(name), B[k].get_param(name))
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_block_cache_matches_checker_eval_forward_and_is_per_sample(env, dtype):
+    nf, torch = env
+    N = 6
+    cases = _two_layer(nf, torch, dtype, N, 710)
+    G = [pu.gpu_layer(nf, c, P, dtype) for c, P, _, _ in cases]
+    O = [pu.oracle_layer(c, P, store_bf16=(dtype == 1)) for c, P, _, _ in cases]
+    blk = nf.Block(G)
+    x = cases[0][2]
+    lab = cases[0][3]
+    # one training step on both sides so that running statistics are not the initial 0/1
+    xd = pu.to_device_nhwc(torch, x, dtype)
+    loss = torch.zeros(2, device="cuda")
+    blk.step(xd, torch.from_numpy(lab).cuda(), 0.01, loss)
+    _, a_o, _ = O[0].step(x, lab, 0.01)
+    O[1].step(a_o, lab, 0.01)
+    if dtype == 1:   # take the checker's state on both sides (see parity_util.check_step)
+        for g, o in zip(G, O):
+            for k in pu.PNAMES:
+                v32 = o.p[k].astype(np.float32)
+                o.set(**{k: v32})
+                g.set_param(k, v32)
+            for k in ("rmean", "rvar"):
+                v32 = getattr(o, k).astype(np.float32)
+                o.set(**{k: v32})
+                g.set_param(k, v32)
+    out = G[1].new_act()
+    blk.cache(xd, out)
+    torch.cuda.synchronize()
+    ref = O[1].eval_forward(O[0].eval_forward(x))
+    assert pu.max_err(pu.from_device_nhwc(out), ref) <= pu.TOL[dtype]["t"]
+    # a sample's cached row does not depend on its batch-mates: sample 3 alone, and a count of 2 < N
+    one = torch.zeros_like(out)
+    blk.cache(xd[3:4].contiguous(), one, count=1)
+    two = torch.zeros_like(out)
+    blk.cache(xd[4:6].contiguous(), two, count=2)
+    torch.cuda.synchronize()
+    assert torch.equal(one[0], out[3]) and torch.equal(two[:2], out[4:6])
+    with pytest.raises(nf.NfError):
+        blk.cache(xd, out, count=N + 1)
+    assert all(l.status() == 0 for l in G)
+
+
+def test_cache_gather_is_bit_exact(env):
+    nf, torch = env
+    K, row = 300, (4, 4, 24)
+    cache = torch.from_numpy(synth.to_bf16_bits(synth.normal(3, 1, (K,) + row)).view(np.int16)).cuda().view(torch.bfloat16)
+    labels = torch.from_numpy(synth.labels(3, 2, K, 100)).cuda()
+    for it, n in enumerate((1, 77, 300)):
+        idx = torch.from_numpy(synth.permutation(5 + it, 1, K)[:n].copy()).cuda()
+        out = torch.zeros((n,) + row, dtype=torch.bfloat16, device="cuda")
+        out_l = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        nf.nf_cache_gather(cache, labels, idx, out, out_l)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), cache[idx.long()].view(torch.int16))
+        assert torch.equal(out_l, labels[idx.long()])
+    with pytest.raises(nf.NfError):
+        nf.nf_cache_gather(cache, labels, idx, out, None)      # labels in without labels out
