@@ -1,0 +1,153 @@
+"""GPU parity on the shapes of the benchmark workloads c2, c3 and c5 (c1 and c4 have their own files).
+
+Every compared step starts from seeded parameters and from inputs produced by the generators or by the
+CHECKER (never by the GPU): layer l+1 of a chain is fed the checker's activation of layer l, which is
+bf16-valued in the bf16 configurations and therefore identical on both sides."""
+import numpy as np
+import pytest
+
+from paper_2402_14139_b200 import synth, workloads
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2402_14139_b200 import nf
+    nf.lib()
+    nf.nf_set_stream(None)
+    return nf, torch
+
+
+def _cfg(l, N, classes):
+    return dict(N=N, Cin=l["Cin"], Cout=l["Cout"], H=l["H"], W=l["W"], F=l["F"], classes=classes, stride=l["stride"],
+                pool=l["pool"])
+
+
+def _step_both(nf, torch, c, P, x, y, lr=0.01):
+    """One step on both sides from the same state; returns (worst errors, checker's act_out, layers)."""
+    O = pu.oracle_layer(c, P, store_bf16=True)
+    G = pu.gpu_layer(nf, c, P, nf.NF_BF16)
+    xd = pu.to_device_nhwc(torch, x, 1)
+    loss_d = torch.zeros(1, device="cuda")
+    act_d = G.new_act()
+    loss_o, act_o, tr = O.step(x, y, lr, update=True, grads=True)
+    G.step(xd, torch.from_numpy(y).cuda(), lr, loss_d, act_d)
+    torch.cuda.synchronize()
+    assert G.status() == 0
+    tol = pu.TOL[1]
+    errs = dict(loss=abs(float(loss_d.item()) - loss_o) / abs(loss_o), act=pu.max_err(pu.from_device_nhwc(act_d), act_o))
+    for k in pu.PNAMES:
+        errs["g" + k] = pu.max_err(G.get_param(k, nf.NF_K_GRAD), tr["g" + k])
+        errs["p" + k] = pu.max_err(G.get_param(k), O.p[k])
+    assert errs["loss"] <= tol["loss"], errs
+    assert max(v for k, v in errs.items() if k != "loss") <= tol["t"], errs
+    return errs, act_o, O, G
+
+
+def test_c2_vgg_block_full_batch_chain(env):
+    nf, torch = env
+    wl = workloads.c2()
+    N, ls = wl["blocks"][0]
+    x = synth.round_bf16(synth.normal(0x4E460002, 8, (N, 3, 32, 32))).astype(np.float64)
+    y = synth.labels(0x4E460002, 9, N, wl["classes"])
+    for li, l in enumerate(ls):
+        c = _cfg(l, N, wl["classes"])
+        P, _, _ = pu.seeded_case(dict(c, N=1), 0x4E460200 + li, bf16=True)
+        errs, x, O, G = _step_both(nf, torch, c, P, x, y)
+        fam = [G.kernel_family(k) for k in range(4)]
+        assert fam == (["cuda-core", "cuda-core", "tcgen05", "tcgen05"] if li == 0 else ["tcgen05"] * 4), fam
+        G.close()
+
+
+C3_PICKS = [(0, 0), (0, 1), (1, 0), (2, 0), (3, 3)]   # (block, layer in block): stem, 64->64, two stride-2 layers, 512->512
+
+
+@pytest.mark.parametrize("pick", range(len(C3_PICKS)))
+def test_c3_resnet_shaped_layers_at_block_batch_size(env, pick):
+    nf, torch = env
+    wl = workloads.c3()
+    b, li = C3_PICKS[pick]
+    N, ls = wl["blocks"][b]
+    l = ls[li]
+    c = _cfg(l, N, wl["classes"])
+    seed = 0x4E460300 + 16 * b + li
+    P, _, _ = pu.seeded_case(dict(c, N=1), seed, bf16=True)
+    x = synth.normal(seed, 8, (N, l["Cin"], l["H"], l["W"]))
+    if l["Cin"] != 3:
+        x = np.maximum(x, 0.0)                              # deeper layers see post-ReLU activations
+    x = synth.round_bf16(x).astype(np.float64)
+    y = synth.labels(seed, 9, N, wl["classes"])
+    _, _, _, G = _step_both(nf, torch, c, P, x, y)
+    G.close()
+
+
+def test_c5_partition_train_cache_rebatch_next_block(env):
+    """The mechanism of the full pass on VGG-16 shapes, at a scale the checker finishes in seconds:
+    Algorithm 1 on the analytic memory model -> train block 1 -> cache its output for the whole
+    (small) dataset -> re-batch by a seeded permutation -> train block 2 on the cached activations."""
+    nf, torch = env
+    wl = workloads.c5()
+    ls = wl["layers"]
+    per_image = [workloads.layer_bytes_per_image(l, wl["classes"]) for l in ls]
+    max_batch = [int(4e9 // b) for b in per_image]
+    blocks = nf.nf_partition(max_batch, 10000, 0.4)
+    assert [(f, l) for f, l, _ in blocks] == [(0, 1), (2, 3), (4, 6), (7, 9), (10, 12)]       # one block per VGG stage
+    assert all(bs == min(max_batch[f:l + 1]) for f, l, bs in blocks)
+    assert [bs for _, _, bs in blocks] == sorted(bs for _, _, bs in blocks)                    # later blocks: larger batches
+
+    K, N1, N2, classes = 12, 4, 6, wl["classes"]      # dataset of 12 images; block 1 trains at 4, block 2 at 6
+    data = synth.round_bf16(synth.normal(0x4E460005, 8, (K, 3, 64, 64))).astype(np.float64)
+    labels = synth.labels(0x4E460005, 9, K, classes)
+    b1 = ls[0:2]
+    O1, G1 = [], []
+    for li, l in enumerate(b1):
+        c = _cfg(l, N1, classes)
+        P, _, _ = pu.seeded_case(dict(c, N=1), 0x4E460500 + li, bf16=True)
+        O1.append(pu.oracle_layer(c, P, store_bf16=True))
+        G1.append(pu.gpu_layer(nf, c, P, nf.NF_BF16))
+    blk1 = nf.Block(G1)
+    loss = torch.zeros(2, device="cuda")
+    for s in range(K // N1):                                # one epoch over the dataset at block 1's batch size
+        xb, yb = data[s * N1:(s + 1) * N1], labels[s * N1:(s + 1) * N1]
+        blk1.step(pu.to_device_nhwc(torch, xb, 1), torch.from_numpy(yb).cuda(), 0.01, loss)
+        _, a, _ = O1[0].step(xb, yb, 0.01)
+        l2, _, _ = O1[1].step(a, yb, 0.01)
+        for g, o in zip(G1, O1):                            # both sides continue from the checker's state
+            for k in pu.PNAMES:
+                v32, m32 = o.p[k].astype(np.float32), o.v[k].astype(np.float32)
+                o.set(**{k: v32, "v" + k: m32})
+                g.set_param(k, v32)
+                g.set_param(k, m32, kind=nf.NF_K_MOMENTUM)
+            for k in ("rmean", "rvar"):
+                v32 = getattr(o, k).astype(np.float32)
+                o.set(**{k: v32})
+                g.set_param(k, v32)
+    torch.cuda.synchronize()
+    assert abs(float(loss[1].item()) - l2) <= 3e-3 * abs(l2)
+    # cache: block 1's output for all K samples (chunks of N1), against the checker's eval forward
+    cache = torch.zeros((K, 32, 32, 64), dtype=torch.bfloat16, device="cuda")
+    for s in range(K // N1):
+        blk1.cache(pu.to_device_nhwc(torch, data[s * N1:(s + 1) * N1], 1), cache[s * N1:(s + 1) * N1])
+    ref_cache = O1[1].eval_forward(O1[0].eval_forward(data))
+    torch.cuda.synchronize()
+    assert pu.max_err(pu.from_device_nhwc(cache), ref_cache) <= pu.TOL[1]["t"]
+    # re-batch at block 2's size: indices and labels bit-exact, rows bit-exact
+    perm = synth.permutation(0x4E460005, 77, K)
+    idx = torch.from_numpy(perm[:N2].copy()).cuda()
+    lab_d = torch.from_numpy(labels).cuda()
+    xb2 = torch.zeros((N2, 32, 32, 64), dtype=torch.bfloat16, device="cuda")
+    yb2 = torch.zeros(N2, dtype=torch.int32, device="cuda")
+    nf.nf_cache_gather(cache, lab_d, idx, xb2, yb2)
+    torch.cuda.synchronize()
+    assert np.array_equal(yb2.cpu().numpy(), labels[perm[:N2]])
+    assert torch.equal(xb2.view(torch.int16), cache[idx.long()].view(torch.int16))
+    # block 2, first layer, on the re-batched cache; the checker gets ITS OWN cached rows
+    l = ls[2]
+    c = _cfg(l, N2, classes)
+    P, _, _ = pu.seeded_case(dict(c, N=1), 0x4E460510, bf16=True)
+    x2 = synth.round_bf16(ref_cache[perm[:N2]]).astype(np.float64)
+    _, _, _, G2 = _step_both(nf, torch, c, P, x2, labels[perm[:N2]])
+    G2.close()
