@@ -81,11 +81,12 @@ def vgg_layers(cfg, S, aux_per_stage, Cin=3):
 
 
 def c5(block_batches=None):
-    """VGG-16-shaped net on 64x64x3, 200 classes; aux filters 64,32,16,8,4 per stage; one block per stage
-    unless the partitioner says otherwise (block_batches = [(first, last, batch)])."""
+    """VGG-16-shaped net on 64x64x3, 200 classes; aux filters 64,32,16,8,4 per stage.  The default blocks
+    (block_batches = [(first, last, batch)]) are what Algorithm 1 returns for layer_bytes_per_image() under a
+    4 GB budget with rho = 0.4 and the batch size capped at the 10 000-image dataset: five blocks."""
     ls = vgg_layers(VGG16, 64, [64, 32, 16, 8, 4])
     if block_batches is None:
-        block_batches = [(0, 1, 64), (2, 3, 128), (4, 6, 256), (7, 9, 512), (10, 12, 512)]
+        block_batches = [(0, 0, 1260), (1, 1, 1904), (2, 3, 3045), (4, 5, 5935), (6, 12, 8602)]
     blocks = [(bs, ls[f:l + 1]) for f, l, bs in block_batches]
     return dict(name="c5", dtype="bf16", classes=200, in_shape=(3, 64, 64), blocks=blocks, layers=ls)
 

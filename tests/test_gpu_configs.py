@@ -94,14 +94,17 @@ def test_c5_partition_train_cache_rebatch_next_block(env):
     per_image = [workloads.layer_bytes_per_image(l, wl["classes"]) for l in ls]
     max_batch = [int(4e9 // b) for b in per_image]
     blocks = nf.nf_partition(max_batch, 10000, 0.4)
-    assert [(f, l) for f, l, _ in blocks] == [(0, 1), (2, 3), (4, 6), (7, 9), (10, 12)]       # one block per VGG stage
+    from oracle import nfo
+    assert blocks == nfo.partition(max_batch, 10000, 0.4)
+    # five blocks under the 4 GB budget; with this library's buffers the early, memory-hungry layers stand alone
+    assert [(f, l) for f, l, _ in blocks] == [(0, 0), (1, 1), (2, 3), (4, 5), (6, 12)]
     assert all(bs == min(max_batch[f:l + 1]) for f, l, bs in blocks)
     assert [bs for _, _, bs in blocks] == sorted(bs for _, _, bs in blocks)                    # later blocks: larger batches
 
     K, N1, N2, classes = 12, 4, 6, wl["classes"]      # dataset of 12 images; block 1 trains at 4, block 2 at 6
     data = synth.round_bf16(synth.normal(0x4E460005, 8, (K, 3, 64, 64))).astype(np.float64)
     labels = synth.labels(0x4E460005, 9, K, classes)
-    b1 = ls[0:2]
+    b1 = ls[blocks[0][0]:blocks[1][1] + 1]      # the first two (single-layer) blocks trained as one chain here
     O1, G1 = [], []
     for li, l in enumerate(b1):
         c = _cfg(l, N1, classes)
