@@ -75,6 +75,22 @@ class ClockSampler(threading.Thread):
                     reasons=sorted(self.reasons))
 
 
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of a list of floats over all ranks (replicas are timed as the slowest one)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def aggregate_images_per_s(images_per_rank, world, ms_max):
+    """Whole-job throughput of `world` independent replicas: all images / the slowest replica's time."""
+    return images_per_rank * world / (ms_max / 1e3)
+
+
 def build_block(nf, torch, wl, bi, seed, host_io):
     """Layers of block bi with Kaiming-normal conv/linear weights (seeded), as an nf.Block."""
     from paper_2402_14139_b200 import synth
@@ -183,11 +199,7 @@ def run_ours(args, rank, world):
     barrier()
     e2e_s = time.perf_counter() - t0
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms, e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_s = float(t[0]), float(t[1])
+    ms, e2e_s = max_over_ranks([ms, e2e_s], world, "cuda")
 
     peaks, peak_src = load_peaks()
     fam = [[L.kernel_family(k) for k in range(4)] for L in layers]
@@ -212,8 +224,7 @@ def run_ours(args, rank, world):
 
     out = None
     if rank == 0:
-        images = N * args.steps * world
-        out = dict(metric=METRIC, value=round(images / (ms / 1e3), 2), unit="images/s", n_gpus=world, steps=args.steps,
+        out = dict(metric=METRIC, value=round(aggregate_images_per_s(N * args.steps, world, ms), 2), unit="images/s", n_gpus=world, steps=args.steps,
                    warmup=args.warmup, ms_per_step=round(ms / args.steps, 4), higher_is_better=True, scaling="weak",
                    vs_baseline=None, dtype="bf16" if es == 2 else "f32", data="synthetic",
                    config=dict(workload=f"{wl['name']}: " + workloads.ALL[args.workload].__doc__.split(".")[0].strip(),
@@ -221,7 +232,7 @@ def run_ours(args, rank, world):
                                f"{n_pool} input batches rotated (pool larger than L2)", replicas=world,
                                kernel_families=fam),
                    clocks=sampler.summary(), gpu_launches=int(launches),
-                   e2e=dict(value=round(N * e2e_steps * world / e2e_s, 2), unit="images/s",
+                   e2e=dict(value=round(aggregate_images_per_s(N * e2e_steps, world, e2e_s * 1e3), 2), unit="images/s",
                             h2d_bytes_per_step=int(x_bytes + 4 * N), d2h_bytes_per_step=int(4 * len(ls))),
                    roofline=roof, kernels=kernels, final_losses=[round(v, 4) for v in losses])
     return out, wl, bi
