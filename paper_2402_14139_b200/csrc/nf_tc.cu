@@ -319,6 +319,203 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 }
 
 
+// ---------------------------------------------------------------- forward, 64 -> 64 channels, column taps folded into N
+// With a 64-wide N tile an MMA is bound by the bytes of its operands, not by its arithmetic.  This
+// variant widens N to 192: D'[pixel, (kw, co)] = sum_{kh, ci} X[pixel shifted by kh rows, ci] * W[kh][kw][co][ci],
+// i.e. the three column taps become three 64-column groups of one accumulator and only the three row
+// taps remain in the K loop (12 instructions of N = 192 per tile instead of 36 of N = 64, one
+// activation box per tile instead of three).  The output is the shift-add
+//   y[h, w, co] = D'[(h, w-1), kw=0, co] + D'[(h, w), kw=1, co] + D'[(h, w+1), kw=2, co],
+// done in the epilogue with warp shuffles: a tile is 16 columns x 8 rows of pixels of which the outer
+// two columns are halo, so the left/right neighbours of every output pixel are adjacent TMEM lanes of the
+// same warp.  14 x 8 output pixels per tile; needs W % 14 == 0 and H % 8 == 0.
+struct FoldParams {
+  int N, H, W, tiles_w, tiles_h, total_tiles, stages, stats;
+  float* red;       // [grid * 2][2][64]
+  int32_t* status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+                     const __grid_constant__ CUtensorMap tm_y, const FoldParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr int kABytes = 10 * 16 * 128;  // (8+2) rows x 16 pixels x 64 channels
+  constexpr int kWBytes = 9 * 64 * 128;   // [kh][kw*64 + co][64 ci]
+  uint8_t* wres = smem + (size_t)p.stages * kABytes;
+  uint8_t* stg = wres + kWBytes;          // 112 output pixels x 128 bytes
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + 16384);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + kMaxStages;
+  uint64_t* tfull = bars + 2 * kMaxStages;
+  uint64_t* tempty = tfull + 2;
+  uint64_t* wfull = tempty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wfull + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);
+  constexpr uint32_t kTmemCols = 512;  // two accumulators of 192 columns
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(&tfull[a], 1);
+      ptx::mbar_init(&tempty[a], 128);
+    }
+    ptx::mbar_init(wfull, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tmap(&tm_x);
+    ptx::prefetch_tmap(&tm_w);
+    ptx::prefetch_tmap(&tm_y);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0 && blockIdx.x < p.total_tiles) {
+      ptx::mbar_expect_tx(wfull, (uint32_t)kWBytes);
+#pragma unroll
+      for (int kh = 0; kh < 3; ++kh) ptx::tma_load_4d(wres + kh * 3 * 64 * 128, &tm_w, wfull, 0, 0, 0, kh);
+    }
+    __syncwarp();
+    uint32_t it = 0;
+    for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++it) {
+      const int s = it % p.stages;
+      const uint32_t ph = (it / p.stages) & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) break;
+      if (lane == 0) {
+        const int w0 = (t % p.tiles_w) * 14, h0 = ((t / p.tiles_w) % p.tiles_h) * 8, n = t / (p.tiles_w * p.tiles_h);
+        ptx::mbar_expect_tx(&full[s], (uint32_t)kABytes);
+        ptx::tma_load_4d(smem + (size_t)s * kABytes, &tm_x, &full[s], 0, w0 - 1, h0 - 1, n);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    constexpr uint32_t idesc = ptx::idesc_bf16(128, 192, 0, 0);
+    const uint64_t hi = ptx::sdesc(0, 16, 1024, 2);
+    const uint32_t w16 = ptx::smem_u32(wres) >> 4;
+    uint32_t it = 0;
+    bool ok = blockIdx.x >= p.total_tiles || __all_sync(0xffffffffu, ptx::mbar_wait(wfull, 0, abort_flag));
+    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++it) {
+      const uint32_t acc = it & 1, aph = (it >> 1) & 1;
+      const int s = it % p.stages;
+      const uint32_t ph = (it / p.stages) & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&tempty[acc], aph ^ 1, abort_flag))) break;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[s], ph, abort_flag))) break;
+      ptx::tc_fence_after();
+      if (lane == 0) {
+        const uint32_t a16 = ptx::smem_u32(smem + (size_t)s * kABytes) >> 4;
+        const uint32_t d = tmem_base + acc * 256;
+#pragma unroll
+        for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            ptx::mma_f16(d, hi | (uint64_t)(a16 + kh * 128 + k * 2), hi | (uint64_t)(w16 + kh * 1536 + k * 2), idesc, (kh | k) != 0);
+        ptx::mma_commit(&empty[s]);
+        ptx::mma_commit(&tfull[acc]);
+      }
+      __syncwarp();
+    }
+  } else {
+    const int et = threadIdx.x - 64;
+    const int lg = warp & 3;
+    const int r = lg * 32 + lane;            // TMEM lane = extended-tile pixel (we = r % 16, h = r / 16)
+    const int we = r & 15, hh = r >> 4;
+    const bool valid = we >= 1 && we <= 14;
+    const int orow = (we - 1) + 14 * hh;     // row of the output staging tile
+    const int sc = et & 63, shalf = et >> 6; // stats: channel, and which 56 of the 112 rows
+    float ssum = 0.f, ssq = 0.f;
+    uint32_t tl = 0;
+    for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++tl) {
+      const int w0 = (t % p.tiles_w) * 14, h0 = ((t / p.tiles_w) % p.tiles_h) * 8, n = t / (p.tiles_w * p.tiles_h);
+      const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+      ptx::mbar_wait(&tfull[acc], aph, abort_flag);
+      ptx::tc_fence_after();
+      if (et == 0) {
+        ptx::tma_store_wait_read();
+        *epi_go = *abort_flag ? 0 : 1;
+      }
+      ptx::named_barrier(1, 128);
+      if (!*epi_go) break;
+      const uint32_t tbase = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * 256;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {          // 16 output channels at a time
+        uint32_t v0[16], v1[16], v2[16];
+        ptx::tmem_ld16(tbase + q * 16, v0);
+        ptx::tmem_ld16(tbase + 64 + q * 16, v1);
+        ptx::tmem_ld16(tbase + 128 + q * 16, v2);
+        ptx::tmem_ld_wait();
+        uint32_t w[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          float o[2];
+#pragma unroll
+          for (int h2 = 0; h2 < 2; ++h2) {
+            const int c = 2 * e + h2;
+            const float left = __shfl_up_sync(0xffffffffu, __uint_as_float(v0[c]), 1);     // kw = 0 term of pixel w-1
+            const float right = __shfl_down_sync(0xffffffffu, __uint_as_float(v2[c]), 1);  // kw = 2 term of pixel w+1
+            o[h2] = left + __uint_as_float(v1[c]) + right;
+          }
+          const __nv_bfloat162 b2 = __floats2bfloat162_rn(o[0], o[1]);
+          w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+        }
+        if (valid) {
+          uint8_t* dst = stg + orow * 128;
+          *reinterpret_cast<uint4*>(dst + (((2 * q) ^ (orow & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(dst + (((2 * q + 1) ^ (orow & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&tempty[acc]);
+      ptx::fence_async_smem();
+      ptx::named_barrier(1, 128);
+      if (et == 0) {
+        ptx::tma_store_4d(&tm_y, stg, 0, w0, h0, n);
+        ptx::tma_store_commit();
+      }
+      if (p.stats) {
+        const uint8_t* col = stg + (sc & 7) * 2;
+        const int u = sc >> 3;
+#pragma unroll 8
+        for (int rr = 0; rr < 56; ++rr) {
+          const int row = shalf * 56 + rr;
+          const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(col + row * 128 + ((u ^ (row & 7)) * 16)));
+          ssum += v;
+          ssq = fmaf(v, v, ssq);
+        }
+      }
+    }
+    if (et == 0) ptx::tma_store_wait_all();
+    if (p.stats) {
+      const size_t b = (size_t)blockIdx.x * 2 + shalf;
+      p.red[(b * 2 + 0) * 64 + sc] = ssum;
+      p.red[(b * 2 + 1) * 64 + sc] = ssq;
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(p.status, NF_ETIMEOUT);
+    const unsigned long long t0 = ptx::globaltimer();
+    while (ptx::globaltimer() - t0 < 2000000ull) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
 // ---------------------------------------------------------------- weight gradient
 // dW[tap][co][ci] = sum over pixels of dy[pixel, co] * x[pixel shifted by tap, ci]  (stride 1).
 // GEMM view per 64-channel block pair (ci chunk, co chunk): the K dimension is the pixel index, so
@@ -612,11 +809,54 @@ int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, c
   return NF_OK;
 }
 
+bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride) {
+  return epi == 0 && stride == 1 && Cin == 64 && Cout == 64 && W % 14 == 0 && H % 8 == 0;
+}
+
+int run_fold(int N, int H, int W, const void* x, const void* w, void* y, int stats, float* red, size_t red_floats,
+             int32_t* status, int* nb) {
+  CUtensorMap mx, mw, my;
+  const uint64_t dx[4] = {64, (uint64_t)W, (uint64_t)H, (uint64_t)N};
+  const uint32_t bx[4] = {64, 16, 10, 1};
+  const uint64_t dw[4] = {64, 64, 3, 3};
+  const uint32_t bw[4] = {64, 64, 3, 1};
+  const uint32_t by[4] = {64, 14, 8, 1};
+  int rc;
+  if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
+  if ((rc = make_map4(&mw, w, dw, bw)) != NF_OK) return rc;
+  if ((rc = make_map4(&my, y, dx, by)) != NF_OK) return rc;
+  FoldParams p{};
+  p.N = N; p.H = H; p.W = W; p.tiles_w = W / 14; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h;
+  p.stats = stats; p.red = red; p.status = status;
+  const size_t fixed = 9 * 64 * 128 + 16384 + 1024 + 1024;
+  int st = (int)((232448 - fixed) / (10 * 16 * 128));
+  if (st > kMaxStages) st = kMaxStages;
+  p.stages = st;
+  const size_t smem = (size_t)st * 10 * 16 * 128 + fixed;
+  int grid = sm_count();
+  if (grid > p.total_tiles) grid = p.total_tiles;
+  if (stats) {
+    const size_t need = (size_t)grid * 2 * 2 * 64;
+    if (need > red_floats) return NF_ENOWS;
+    NF_CUDA(cudaMemsetAsync(red, 0, need * sizeof(float), g_nf_stream));
+    *nb = grid * 2;
+  }
+  static bool attr_done = false;
+  if (!attr_done) {
+    NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    attr_done = true;
+  }
+  conv_fwd_fold_kernel<<<grid, kThreads, smem, g_nf_stream>>>(mx, mw, my, p);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
 // epi 0: y through TMA + optional statistics.  epi 1: out = ReLU(conv + bias) written directly (y unused).
 // H, W are the INPUT size; stride 2 halves them (rounding up) for the output.
 int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
             size_t red_floats, int32_t* status, int* nb, int epi = 0, const float* bias = nullptr, int stride = 1) {
   const int H = (Hin - 1) / stride + 1, W = (Win - 1) / stride + 1;
+  if (fold_ok(H, W, Cin, Cout, epi, stride)) return run_fold(N, H, W, x, w, y, stats, red, red_floats, status, nb);
   const TcPlan pl = plan_fwd(H, W, Cin, Cout, N, epi, stride);
   if (!pl.ok) return NF_EUNSUPPORTED;
   CUtensorMap mx, mw, my;

@@ -20,6 +20,9 @@ SHAPES = [  # N, Cin, Cout, H, W, stride
     (1, 64, 64, 16, 8, 1),      # tensor-core forward: 8x16 pixel tiles, a single tile
     (2, 64, 128, 32, 32, 2),    # tensor-core stride 2: 16x16 output, strided TMA boxes
     (1, 128, 64, 64, 32, 2),    # tensor-core stride 2: two channel chunks, 32x16 output
+    (2, 64, 64, 16, 28, 1),     # 64->64 forward with the column taps folded into N: 14-pixel-wide tiles
+    (1, 64, 64, 8, 14, 1),      # the same kernel on a single tile
+    (3, 64, 64, 24, 56, 1),     # several tiles per CTA row and per image
     (2, 64, 64, 31, 33, 2),     # stride 2 with odd input sizes: 16x17 output is not tileable -> CUDA-core path
 ]
 

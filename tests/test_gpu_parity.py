@@ -128,6 +128,7 @@ TC = [
     dict(N=12, Cin=64, Cout=64, H=16, W=16, F=64, classes=10, stride=1, pool=True),
     dict(N=4, Cin=64, Cout=64, H=16, W=16, F=12, classes=10, stride=1, pool=False),   # F not a multiple of 8
     dict(N=6, Cin=64, Cout=128, H=32, W=32, F=16, classes=10, stride=2, pool=False),  # stride-2 tensor-core kernels
+    dict(N=3, Cin=64, Cout=64, H=16, W=112, F=16, classes=10, stride=1, pool=False),  # folded-tap forward (W % 14 == 0)
 ]
 
 
