@@ -330,21 +330,30 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 // two columns are halo, so the left/right neighbours of every output pixel are adjacent TMEM lanes of the
 // same warp.  14 x 8 output pixels per tile; needs W % 14 == 0 and H % 8 == 0.
 struct FoldParams {
-  int N, H, W, tiles_w, tiles_h, total_tiles, stages, stats;
-  float* red;       // [grid * 2][2][64]
+  int N, H, W, Cout, kchunks, tiles_w, tiles_h, total_tiles, stages, stats;
+  float* red;         // EPI 0: [grid * 2][2][64]
   int32_t* status;
+  const float* bias;  // EPI 1
+  bf16* out;          // EPI 1: [N][H][W][Cout]
 };
 
+// G   : width of one column-tap group of the accumulator (N = 3*G): 64 for the main conv, 16/32/64 for the
+//       aux conv with F <= G filters (weight rows beyond F are zero-filled by TMA).
+// EPI : 0 = y in bf16 through a TMA store + BatchNorm partial sums (G = 64, Cout = 64);
+//       1 = bias + ReLU, F channels written straight from registers (aux conv forward).
+// Cin = 64 * kchunks; all 9 * kchunks weight tiles stay resident in shared memory.
+template <int G, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                      const __grid_constant__ CUtensorMap tm_y, const FoldParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr int kABytes = 10 * 16 * 128;  // (8+2) rows x 16 pixels x 64 channels
-  constexpr int kWBytes = 9 * 64 * 128;   // [kh][kw*64 + co][64 ci]
+  constexpr int kABytes = 10 * 16 * 128;      // (8+2) rows x 16 pixels x 64 channels
+  constexpr int kWTile = 3 * G * 128;         // one kernel row of one chunk: [kw*G + co][64 ci]
+  const int w_bytes = 3 * p.kchunks * kWTile; // [chunk][kh][kw*G + co][64 ci]
   uint8_t* wres = smem + (size_t)p.stages * kABytes;
-  uint8_t* stg = wres + kWBytes;          // 112 output pixels x 128 bytes
-  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + 16384);
+  uint8_t* stg = wres + w_bytes;              // EPI 0: 112 output pixels x 128 bytes
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (EPI == 0 ? 16384 : 0));
   uint64_t* full = bars;
   uint64_t* empty = bars + kMaxStages;
   uint64_t* tfull = bars + 2 * kMaxStages;
@@ -353,7 +362,8 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wfull + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);
-  constexpr uint32_t kTmemCols = 512;  // two accumulators of 192 columns
+  constexpr uint32_t kAccStride = G == 64 ? 256 : 128;  // columns between the two accumulators
+  constexpr uint32_t kTmemCols = 2 * kAccStride;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -383,47 +393,56 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 
   if (warp == 0) {
     if (lane == 0 && blockIdx.x < p.total_tiles) {
-      ptx::mbar_expect_tx(wfull, (uint32_t)kWBytes);
+      ptx::mbar_expect_tx(wfull, (uint32_t)w_bytes);
+      for (int ck = 0; ck < p.kchunks; ++ck)
 #pragma unroll
-      for (int kh = 0; kh < 3; ++kh) ptx::tma_load_4d(wres + kh * 3 * 64 * 128, &tm_w, wfull, 0, 0, 0, kh);
+        for (int kh = 0; kh < 3; ++kh) ptx::tma_load_4d(wres + (ck * 3 + kh) * kWTile, &tm_w, wfull, ck * 64, 0, 0, kh);
     }
     __syncwarp();
     uint32_t it = 0;
-    for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++it) {
-      const int s = it % p.stages;
-      const uint32_t ph = (it / p.stages) & 1;
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) break;
-      if (lane == 0) {
-        const int w0 = (t % p.tiles_w) * 14, h0 = ((t / p.tiles_w) % p.tiles_h) * 8, n = t / (p.tiles_w * p.tiles_h);
-        ptx::mbar_expect_tx(&full[s], (uint32_t)kABytes);
-        ptx::tma_load_4d(smem + (size_t)s * kABytes, &tm_x, &full[s], 0, w0 - 1, h0 - 1, n);
+    bool ok = true;
+    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x) {
+      const int w0 = (t % p.tiles_w) * 14, h0 = ((t / p.tiles_w) % p.tiles_h) * 8, n = t / (p.tiles_w * p.tiles_h);
+      for (int ck = 0; ck < p.kchunks; ++ck, ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) { ok = false; break; }
+        if (lane == 0) {
+          ptx::mbar_expect_tx(&full[s], (uint32_t)kABytes);
+          ptx::tma_load_4d(smem + (size_t)s * kABytes, &tm_x, &full[s], ck * 64, w0 - 1, h0 - 1, n);
+        }
+        __syncwarp();
       }
-      __syncwarp();
     }
   } else if (warp == 1) {
-    constexpr uint32_t idesc = ptx::idesc_bf16(128, 192, 0, 0);
+    constexpr uint32_t idesc = ptx::idesc_bf16(128, 3 * G, 0, 0);
     const uint64_t hi = ptx::sdesc(0, 16, 1024, 2);
     const uint32_t w16 = ptx::smem_u32(wres) >> 4;
-    uint32_t it = 0;
+    uint32_t it = 0, tl = 0;
     bool ok = blockIdx.x >= p.total_tiles || __all_sync(0xffffffffu, ptx::mbar_wait(wfull, 0, abort_flag));
-    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++it) {
-      const uint32_t acc = it & 1, aph = (it >> 1) & 1;
-      const int s = it % p.stages;
-      const uint32_t ph = (it / p.stages) & 1;
+    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++tl) {
+      const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(&tempty[acc], aph ^ 1, abort_flag))) break;
-      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[s], ph, abort_flag))) break;
       ptx::tc_fence_after();
-      if (lane == 0) {
-        const uint32_t a16 = ptx::smem_u32(smem + (size_t)s * kABytes) >> 4;
-        const uint32_t d = tmem_base + acc * 256;
+      const uint32_t d = tmem_base + acc * kAccStride;
+      for (int ck = 0; ck < p.kchunks; ++ck, ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[s], ph, abort_flag))) { ok = false; break; }
+        ptx::tc_fence_after();
+        if (lane == 0) {
+          const uint32_t a16 = ptx::smem_u32(smem + (size_t)s * kABytes) >> 4;
 #pragma unroll
-        for (int kh = 0; kh < 3; ++kh)
+          for (int kh = 0; kh < 3; ++kh)
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            ptx::mma_f16(d, hi | (uint64_t)(a16 + kh * 128 + k * 2), hi | (uint64_t)(w16 + kh * 1536 + k * 2), idesc, (kh | k) != 0);
-        ptx::mma_commit(&empty[s]);
-        ptx::mma_commit(&tfull[acc]);
+            for (int k = 0; k < 4; ++k)
+              ptx::mma_f16(d, hi | (uint64_t)(a16 + kh * 128 + k * 2),
+                           hi | (uint64_t)(w16 + (ck * 3 + kh) * (kWTile >> 4) + k * 2), idesc, (ck | kh | k) != 0);
+          ptx::mma_commit(&empty[s]);
+        }
+        __syncwarp();
       }
+      if (ok && lane == 0) ptx::mma_commit(&tfull[acc]);
       __syncwarp();
     }
   } else {
@@ -442,18 +461,19 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       ptx::mbar_wait(&tfull[acc], aph, abort_flag);
       ptx::tc_fence_after();
       if (et == 0) {
-        ptx::tma_store_wait_read();
+        if constexpr (EPI == 0) ptx::tma_store_wait_read();
         *epi_go = *abort_flag ? 0 : 1;
       }
       ptx::named_barrier(1, 128);
       if (!*epi_go) break;
-      const uint32_t tbase = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * 256;
+      const uint32_t tbase = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * kAccStride;
+      bf16* gdst = EPI == 1 ? p.out + (((size_t)n * p.H + h0 + hh) * p.W + w0 + we - 1) * p.Cout : nullptr;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {          // 16 output channels at a time
+      for (int q = 0; q < G / 16; ++q) {     // 16 output channels at a time
         uint32_t v0[16], v1[16], v2[16];
         ptx::tmem_ld16(tbase + q * 16, v0);
-        ptx::tmem_ld16(tbase + 64 + q * 16, v1);
-        ptx::tmem_ld16(tbase + 128 + q * 16, v2);
+        ptx::tmem_ld16(tbase + G + q * 16, v1);
+        ptx::tmem_ld16(tbase + 2 * G + q * 16, v2);
         ptx::tmem_ld_wait();
         uint32_t w[8];
 #pragma unroll
@@ -465,41 +485,57 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             const float left = __shfl_up_sync(0xffffffffu, __uint_as_float(v0[c]), 1);     // kw = 0 term of pixel w-1
             const float right = __shfl_down_sync(0xffffffffu, __uint_as_float(v2[c]), 1);  // kw = 2 term of pixel w+1
             o[h2] = left + __uint_as_float(v1[c]) + right;
+            if constexpr (EPI == 1) {
+              const int ch = q * 16 + c;
+              o[h2] = ch < p.Cout ? fmaxf(o[h2] + p.bias[ch], 0.f) : 0.f;
+            }
           }
           const __nv_bfloat162 b2 = __floats2bfloat162_rn(o[0], o[1]);
           w[e] = *reinterpret_cast<const uint32_t*>(&b2);
         }
-        if (valid) {
-          uint8_t* dst = stg + orow * 128;
-          *reinterpret_cast<uint4*>(dst + (((2 * q) ^ (orow & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(dst + (((2 * q + 1) ^ (orow & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+        if constexpr (EPI == 0) {
+          if (valid) {
+            uint8_t* dst = stg + orow * 128;
+            *reinterpret_cast<uint4*>(dst + (((2 * q) ^ (orow & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(dst + (((2 * q + 1) ^ (orow & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+          }
+        } else {
+          const int c0 = q * 16;             // Cout is a multiple of 8 here
+          if (valid && c0 < p.Cout) {
+            *reinterpret_cast<uint4*>(gdst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+            if (c0 + 8 < p.Cout) *reinterpret_cast<uint4*>(gdst + c0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+          }
         }
       }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&tempty[acc]);
-      ptx::fence_async_smem();
-      ptx::named_barrier(1, 128);
-      if (et == 0) {
-        ptx::tma_store_4d(&tm_y, stg, 0, w0, h0, n);
-        ptx::tma_store_commit();
-      }
-      if (p.stats) {
-        const uint8_t* col = stg + (sc & 7) * 2;
-        const int u = sc >> 3;
+      if constexpr (EPI == 0) {
+        ptx::fence_async_smem();
+        ptx::named_barrier(1, 128);
+        if (et == 0) {
+          ptx::tma_store_4d(&tm_y, stg, 0, w0, h0, n);
+          ptx::tma_store_commit();
+        }
+        if (p.stats) {
+          const uint8_t* col = stg + (sc & 7) * 2;
+          const int u = sc >> 3;
 #pragma unroll 8
-        for (int rr = 0; rr < 56; ++rr) {
-          const int row = shalf * 56 + rr;
-          const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(col + row * 128 + ((u ^ (row & 7)) * 16)));
-          ssum += v;
-          ssq = fmaf(v, v, ssq);
+          for (int rr = 0; rr < 56; ++rr) {
+            const int row = shalf * 56 + rr;
+            const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(col + row * 128 + ((u ^ (row & 7)) * 16)));
+            ssum += v;
+            ssq = fmaf(v, v, ssq);
+          }
         }
       }
     }
-    if (et == 0) ptx::tma_store_wait_all();
-    if (p.stats) {
-      const size_t b = (size_t)blockIdx.x * 2 + shalf;
-      p.red[(b * 2 + 0) * 64 + sc] = ssum;
-      p.red[(b * 2 + 1) * 64 + sc] = ssq;
+    if constexpr (EPI == 0) {
+      if (et == 0) ptx::tma_store_wait_all();
+      if (p.stats) {
+        const size_t b = (size_t)blockIdx.x * 2 + shalf;
+        p.red[(b * 2 + 0) * 64 + sc] = ssum;
+        p.red[(b * 2 + 1) * 64 + sc] = ssq;
+      }
     }
   }
 
@@ -809,30 +845,55 @@ int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, c
   return NF_OK;
 }
 
+// The folded-tap kernel covers: main forward 64 -> 64 (epi 0) and the aux forward with F <= 64, F % 8 == 0
+// (epi 1), when W % 14 == 0, H % 8 == 0 and all weight tiles fit in shared memory beside >= 3 activation stages.
+int fold_group(int Cout, int epi) { return epi == 0 ? 64 : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64); }
 bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride) {
-  return epi == 0 && stride == 1 && Cin == 64 && Cout == 64 && W % 14 == 0 && H % 8 == 0;
+  if (stride != 1 || W % 14 || H % 8 || Cin % 64) return false;
+  if (epi == 0 ? (Cin != 64 || Cout != 64) : epi == 1 ? (Cout > 64 || Cout % 8) : true) return false;
+  const size_t wbytes = (size_t)9 * (Cin / 64) * fold_group(Cout, epi) * 128;
+  return wbytes + (epi == 0 ? 16384 : 0) + 2048 + 3 * 20480 <= 232448;
 }
 
-int run_fold(int N, int H, int W, const void* x, const void* w, void* y, int stats, float* red, size_t red_floats,
-             int32_t* status, int* nb) {
+template <int G, int EPI>
+int launch_fold(int grid, size_t smem, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const FoldParams& p) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel<G, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    attr_done = true;
+  }
+  conv_fwd_fold_kernel<G, EPI><<<grid, kThreads, smem, g_nf_stream>>>(mx, mw, my, p);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
+             size_t red_floats, int32_t* status, int* nb, int epi, const float* bias) {
+  const int G = fold_group(Cout, epi);
   CUtensorMap mx, mw, my;
-  const uint64_t dx[4] = {64, (uint64_t)W, (uint64_t)H, (uint64_t)N};
+  const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
   const uint32_t bx[4] = {64, 16, 10, 1};
-  const uint64_t dw[4] = {64, 64, 3, 3};
-  const uint32_t bw[4] = {64, 64, 3, 1};
+  const uint64_t dw[4] = {(uint64_t)Cin, (uint64_t)Cout, 3, 3};
+  const uint32_t bw[4] = {64, (uint32_t)G, 3, 1};
+  const uint64_t dy[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
   const uint32_t by[4] = {64, 14, 8, 1};
   int rc;
   if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
   if ((rc = make_map4(&mw, w, dw, bw)) != NF_OK) return rc;
-  if ((rc = make_map4(&my, y, dx, by)) != NF_OK) return rc;
+  if (epi == 0) {
+    if ((rc = make_map4(&my, y, dy, by)) != NF_OK) return rc;
+  } else {
+    my = mx;
+  }
   FoldParams p{};
-  p.N = N; p.H = H; p.W = W; p.tiles_w = W / 14; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h;
-  p.stats = stats; p.red = red; p.status = status;
-  const size_t fixed = 9 * 64 * 128 + 16384 + 1024 + 1024;
-  int st = (int)((232448 - fixed) / (10 * 16 * 128));
+  p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = Cin / 64;
+  p.tiles_w = W / 14; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h;
+  p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
+  const size_t fixed = (size_t)9 * p.kchunks * G * 128 + (epi == 0 ? 16384 : 0) + 1024 + 1024;
+  int st = (int)((232448 - fixed) / 20480);
   if (st > kMaxStages) st = kMaxStages;
   p.stages = st;
-  const size_t smem = (size_t)st * 10 * 16 * 128 + fixed;
+  const size_t smem = (size_t)st * 20480 + fixed;
   int grid = sm_count();
   if (grid > p.total_tiles) grid = p.total_tiles;
   if (stats) {
@@ -841,14 +902,9 @@ int run_fold(int N, int H, int W, const void* x, const void* w, void* y, int sta
     NF_CUDA(cudaMemsetAsync(red, 0, need * sizeof(float), g_nf_stream));
     *nb = grid * 2;
   }
-  static bool attr_done = false;
-  if (!attr_done) {
-    NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
-    attr_done = true;
-  }
-  conv_fwd_fold_kernel<<<grid, kThreads, smem, g_nf_stream>>>(mx, mw, my, p);
-  NF_LAUNCHED();
-  return NF_OK;
+  if (epi == 0) return launch_fold<64, 0>(grid, smem, mx, mw, my, p);
+  return G == 16 ? launch_fold<16, 1>(grid, smem, mx, mw, my, p)
+                 : G == 32 ? launch_fold<32, 1>(grid, smem, mx, mw, my, p) : launch_fold<64, 1>(grid, smem, mx, mw, my, p);
 }
 
 // epi 0: y through TMA + optional statistics.  epi 1: out = ReLU(conv + bias) written directly (y unused).
@@ -856,7 +912,8 @@ int run_fold(int N, int H, int W, const void* x, const void* w, void* y, int sta
 int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
             size_t red_floats, int32_t* status, int* nb, int epi = 0, const float* bias = nullptr, int stride = 1) {
   const int H = (Hin - 1) / stride + 1, W = (Win - 1) / stride + 1;
-  if (fold_ok(H, W, Cin, Cout, epi, stride)) return run_fold(N, H, W, x, w, y, stats, red, red_floats, status, nb);
+  if (fold_ok(H, W, Cin, Cout, epi, stride))
+    return run_fold(N, H, W, Cin, Cout, x, w, y, stats, red, red_floats, status, nb, epi, bias);
   const TcPlan pl = plan_fwd(H, W, Cin, Cout, N, epi, stride);
   if (!pl.ok) return NF_EUNSUPPORTED;
   CUtensorMap mx, mw, my;

@@ -129,6 +129,8 @@ TC = [
     dict(N=4, Cin=64, Cout=64, H=16, W=16, F=12, classes=10, stride=1, pool=False),   # F not a multiple of 8
     dict(N=6, Cin=64, Cout=128, H=32, W=32, F=16, classes=10, stride=2, pool=False),  # stride-2 tensor-core kernels
     dict(N=3, Cin=64, Cout=64, H=16, W=112, F=16, classes=10, stride=1, pool=False),  # folded-tap forward (W % 14 == 0)
+    dict(N=3, Cin=64, Cout=128, H=16, W=112, F=8, classes=10, stride=1, pool=False),  # folded aux forward, two K chunks, F < 16
+    dict(N=3, Cin=64, Cout=64, H=16, W=112, F=40, classes=10, stride=1, pool=False),  # folded aux forward, group width 64
 ]
 
 
