@@ -128,11 +128,121 @@ __global__ void sum_splits_kernel(const float* __restrict__ part, int splits, si
   out[i] = s;
 }
 
+
+// ------------------------------------------------------------------ first-layer kernels (Cin <= 4)
+// An RGB input gives a K dimension of only 27: too thin for the tensor cores and, with 6-byte pixels,
+// not addressable by TMA.  One thread computes 16 output channels of one pixel from its 3x3xCin patch held
+// in registers; weights sit in shared memory and are read as warp-wide broadcasts.
+template <typename T>
+__global__ void __launch_bounds__(256) conv_smallc_kernel(const T* __restrict__ x, int N, int H, int W, int Ci,
+                                                          const T* __restrict__ w, int s, int Co, int Ho, int Wo,
+                                                          T* __restrict__ y) {
+  extern __shared__ float wsm[];  // [tap][ci][co]
+  for (int e = threadIdx.y * 32 + threadIdx.x; e < 9 * Ci * Co; e += blockDim.x * blockDim.y) {
+    const int co = e % Co, ci = (e / Co) % Ci, t = e / (Co * Ci);
+    wsm[e] = ldf(w, ((size_t)t * Co + co) * Ci + ci);
+  }
+  __syncthreads();
+  const size_t P = (size_t)N * Ho * Wo;
+  const size_t pix = (size_t)blockIdx.x * 32 + threadIdx.x;
+  if (pix >= P) return;
+  const int j = (int)(pix % Wo), i = (int)((pix / Wo) % Ho);
+  const size_t n = pix / ((size_t)Wo * Ho);
+  float patch[36];
+#pragma unroll
+  for (int t = 0; t < 9; ++t) {
+    const int ii = i * s + t / 3 - 1, jj = j * s + t % 3 - 1;
+    const bool in = ii >= 0 && ii < H && jj >= 0 && jj < W;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) patch[t * 4 + c] = (in && c < Ci) ? ldf(x, ((n * H + ii) * W + jj) * Ci + c) : 0.f;
+  }
+  const int co0 = threadIdx.y * 16;
+  float acc[16];
+#pragma unroll
+  for (int k = 0; k < 16; ++k) acc[k] = 0.f;
+#pragma unroll
+  for (int t = 0; t < 9; ++t)
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      if (c < Ci) {
+        const float xv = patch[t * 4 + c];
+        const float* wr = wsm + (t * Ci + c) * Co + co0;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) acc[k] = fmaf(xv, wr[k], acc[k]);
+      }
+#pragma unroll
+  for (int k = 0; k < 16; ++k) stf(y, pix * Co + co0 + k, acc[k]);
+}
+
+// part[split][tap][co][ci]: thread (co, lane) sums its 9*Ci products over the pixels lane, lane+4, ... of the
+// split's rows; the 3 input rows of an output row are staged in shared memory and read as broadcasts.
+template <typename T>
+__global__ void __launch_bounds__(512) wgrad_smallc_kernel(const T* __restrict__ x, int N, int H, int W, int Ci,
+                                                           const T* __restrict__ g, int Co, int s, int Ho, int Wo,
+                                                           int splits, float* __restrict__ part) {
+  extern __shared__ float sm[];           // xrow[3][W + 2][4]  then  red[4][Co][36]
+  float* xrow = sm;
+  float* red = sm + 3 * (W + 2) * 4;
+  const int co = threadIdx.x, ln = threadIdx.y, tid = ln * blockDim.x + co, nthr = blockDim.x * 4;
+  const long rows = (long)N * Ho;
+  const long r0 = rows * blockIdx.x / splits, r1 = rows * (blockIdx.x + 1) / splits;
+  float acc[36];
+#pragma unroll
+  for (int k = 0; k < 36; ++k) acc[k] = 0.f;
+  for (long r = r0; r < r1; ++r) {
+    const int n = (int)(r / Ho), i = (int)(r % Ho);
+    __syncthreads();
+    for (int e = tid; e < 3 * (W + 2) * 4; e += nthr) {
+      const int c = e & 3, col = (e >> 2) % (W + 2), rr = (e >> 2) / (W + 2);
+      const int ii = i * s + rr - 1, jj = col - 1;
+      xrow[e] = (c < Ci && ii >= 0 && ii < H && jj >= 0 && jj < W) ? ldf(x, (((size_t)n * H + ii) * W + jj) * Ci + c) : 0.f;
+    }
+    __syncthreads();
+    for (int j = ln; j < Wo; j += 4) {
+      const float gv = ldf(g, (((size_t)n * Ho + i) * Wo + j) * Co + co);
+#pragma unroll
+      for (int t = 0; t < 9; ++t) {
+        const float4 xv = *reinterpret_cast<const float4*>(xrow + ((t / 3) * (W + 2) + j * s + t % 3) * 4);
+        acc[t * 4 + 0] = fmaf(gv, xv.x, acc[t * 4 + 0]);
+        acc[t * 4 + 1] = fmaf(gv, xv.y, acc[t * 4 + 1]);
+        acc[t * 4 + 2] = fmaf(gv, xv.z, acc[t * 4 + 2]);
+        acc[t * 4 + 3] = fmaf(gv, xv.w, acc[t * 4 + 3]);
+      }
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < 36; ++k) red[(ln * Co + co) * 36 + k] = acc[k];
+  __syncthreads();
+  if (ln == 0)
+    for (int t = 0; t < 9; ++t)
+      for (int c = 0; c < Ci; ++c) {
+        float v = 0.f;
+        for (int q = 0; q < 4; ++q) v += red[(q * Co + co) * 36 + t * 4 + c];
+        part[(((size_t)blockIdx.x * 9 + t) * Co + co) * Ci + c] = v;
+      }
+}
+
+inline bool smallc_ok(int Ci, int Co, int W) { return Ci <= 4 && Co % 16 == 0 && Co <= 128 && W <= 512; }
+
 }  // namespace
 
 int nf_ref_conv(int dtype, const void* x, int N, int H, int W, int Ci, const void* w, long ws_tap, long ws_co,
                 long ws_ci, int flip, const float* bias, int relu, int stride, int Co, void* y) {
   const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+  if (smallc_ok(Ci, Co, W) && !flip && !bias && !relu && ws_ci == 1 && ws_co == Ci && ws_tap == (long)Co * Ci) {
+    const size_t P = (size_t)N * Ho * Wo;
+    const dim3 blk(32, Co / 16);
+    const size_t sm = (size_t)9 * Ci * Co * sizeof(float);
+    if (dtype == NF_F32)
+      conv_smallc_kernel<float><<<(unsigned)((P + 31) / 32), blk, sm, g_nf_stream>>>((const float*)x, N, H, W, Ci, (const float*)w,
+                                                                                   stride, Co, Ho, Wo, (float*)y);
+    else
+      conv_smallc_kernel<bf16><<<(unsigned)((P + 31) / 32), blk, sm, g_nf_stream>>>((const bf16*)x, N, H, W, Ci, (const bf16*)w,
+                                                                                  stride, Co, Ho, Wo, (bf16*)y);
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   const long blocks = (long)N * Ho * ((Wo + CT_P - 1) / CT_P) * ((Co + CT_CO - 1) / CT_CO);
   if (blocks <= 0 || blocks > 0x7fffffffL) return NF_EUNSUPPORTED;
   if (dtype == NF_F32)
@@ -146,6 +256,10 @@ int nf_ref_conv(int dtype, const void* x, int N, int H, int W, int Ci, const voi
 }
 
 int nf_ref_wgrad_splits(int N, int Ho, int Ci, int Co) {
+  if (Ci <= 4 && Co % 16 == 0 && Co <= 128) {  // first-layer kernel: one block per slice of rows
+    long sp = (long)N * Ho;
+    return (int)(sp > 1184 ? 1184 : sp);
+  }
   const long tiles = (long)((Ci + 15) / 16) * ((Co + 15) / 16);
   long s = 2368 / tiles;
   if (s < 1) s = 1;
@@ -159,6 +273,26 @@ int nf_ref_wgrad(int dtype, const void* x, int N, int H, int W, int Ci, const vo
   const int splits = nf_ref_wgrad_splits(N, Ho, Ci, Co);
   const size_t n = (size_t)9 * Co * Ci;
   if ((size_t)splits * n > part_floats) return NF_ENOWS;
+  if (smallc_ok(Ci, Co, W)) {
+    const dim3 blk(Co, 4);
+    const size_t sm = ((size_t)3 * (W + 2) * 4 + (size_t)4 * Co * 36) * sizeof(float);  // <= 24.7 KB + 73.7 KB
+    static bool attr_done = false;
+    if (!attr_done) {
+      NF_CUDA(cudaFuncSetAttribute(wgrad_smallc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+      NF_CUDA(cudaFuncSetAttribute(wgrad_smallc_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+      attr_done = true;
+    }
+    if (dtype == NF_F32)
+      wgrad_smallc_kernel<float><<<splits, blk, sm, g_nf_stream>>>((const float*)x, N, H, W, Ci, (const float*)g, Co, stride, Ho, Wo,
+                                                                 splits, part);
+    else
+      wgrad_smallc_kernel<bf16><<<splits, blk, sm, g_nf_stream>>>((const bf16*)x, N, H, W, Ci, (const bf16*)g, Co, stride, Ho, Wo,
+                                                                splits, part);
+    NF_LAUNCHED();
+    sum_splits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, g_nf_stream>>>(part, splits, n, dw);
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   const unsigned blocks = (unsigned)(((Ci + 15) / 16) * ((Co + 15) / 16) * splits);
   if (dtype == NF_F32)
     wgrad_direct_kernel<float><<<blocks, 256, 0, g_nf_stream>>>((const float*)x, N, H, W, Ci, (const float*)g, Co,
