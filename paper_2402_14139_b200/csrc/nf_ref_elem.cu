@@ -424,6 +424,37 @@ __global__ void __launch_bounds__(256) bn_apply_vec_kernel(const uint4* __restri
   }
 }
 
+
+// per-thread constants variant (256 % C8 == 0)
+__global__ void __launch_bounds__(256) bn_apply_vec2_kernel(const uint4* __restrict__ y, int C8, const float* __restrict__ scale,
+                                                            const float* __restrict__ shift, size_t total8, uint4* __restrict__ out) {
+  const int c0 = (threadIdx.x % C8) * 8;
+  float A[8], B[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    A[i] = scale[c0 + i];
+    B[i] = shift[c0 + i];
+  }
+  const size_t stride = (size_t)gridDim.x * 256;
+  for (size_t e0 = (size_t)blockIdx.x * 256 + threadIdx.x; e0 < total8; e0 += 2 * stride) {
+    const size_t e1 = e0 + stride;
+    const bool two = e1 < total8;
+    const uint4 ya = __ldg(y + e0);
+    const uint4 yb = two ? __ldg(y + e1) : ya;
+    float v[8];
+    unpack8(ya, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = fmaxf(fmaf(v[i], A[i], B[i]), 0.f);
+    out[e0] = pack8(v);
+    if (two) {
+      unpack8(yb, v);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = fmaxf(fmaf(v[i], A[i], B[i]), 0.f);
+      out[e1] = pack8(v);
+    }
+  }
+}
+
 // partial sums of (dz, dz*xhat) with dz = da * 1[y*scale+shift > 0]; red[(block*2+k)*C + c]
 __global__ void __launch_bounds__(256) bn_bwd_reduce_vec_kernel(const uint4* __restrict__ y, const uint4* __restrict__ da,
                                                                 size_t P, int C8, const float* __restrict__ scale,
@@ -440,8 +471,30 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_vec_kernel(const uint4* __r
     a[i] = 0.f; b[i] = 0.f;
   }
   const size_t p0 = P * blockIdx.x / gridDim.x, p1 = P * (blockIdx.x + 1) / gridDim.x;
-  if (pl < planes)
-    for (size_t p = p0 + pl; p < p1; p += planes) {
+  if (pl < planes) {
+    size_t p = p0 + pl;
+    for (; p + planes < p1; p += 2 * (size_t)planes) {  // two pixels per iteration: four 16-byte loads in flight
+      const uint4 y0 = __ldg(y + p * C8 + g), d0 = __ldg(da + p * C8 + g);
+      const uint4 y1 = __ldg(y + (p + planes) * C8 + g), d1 = __ldg(da + (p + planes) * C8 + g);
+      float yv[8], dv[8];
+      unpack8(y0, yv);
+      unpack8(d0, dv);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float dz = fmaf(yv[i], sc[i], sh[i]) > 0.f ? dv[i] : 0.f;
+        a[i] += dz;
+        b[i] = fmaf(dz, (yv[i] - m[i]) * is[i], b[i]);
+      }
+      unpack8(y1, yv);
+      unpack8(d1, dv);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float dz = fmaf(yv[i], sc[i], sh[i]) > 0.f ? dv[i] : 0.f;
+        a[i] += dz;
+        b[i] = fmaf(dz, (yv[i] - m[i]) * is[i], b[i]);
+      }
+    }
+    for (; p < p1; p += planes) {
       float yv[8], dv[8];
       unpack8(__ldg(y + p * C8 + g), yv);
       unpack8(__ldg(da + p * C8 + g), dv);
@@ -452,6 +505,7 @@ __global__ void __launch_bounds__(256) bn_bwd_reduce_vec_kernel(const uint4* __r
         b[i] = fmaf(dz, (yv[i] - m[i]) * is[i], b[i]);
       }
     }
+  }
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     sm[i][threadIdx.x] = a[i];
@@ -484,19 +538,84 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_vec_kernel(const uint4* __re
     cs[5 * C + i] = sdzx[i] * invM;
   }
   __syncthreads();
-  for (size_t e = (size_t)blockIdx.x * 256 + threadIdx.x; e < total8; e += (size_t)gridDim.x * 256) {
-    const int c0 = (int)(e % C8) * 8;
+  const size_t stride = (size_t)gridDim.x * 256;
+  for (size_t e0 = (size_t)blockIdx.x * 256 + threadIdx.x; e0 < total8; e0 += 2 * stride) {  // two vectors per iteration
+    const size_t e1 = e0 + stride;
+    const bool two = e1 < total8;
+    const uint4 ya = __ldg(y + e0), da0 = __ldg(da + e0);
+    uint4 yb = ya, db = da0;
+    if (two) {
+      yb = __ldg(y + e1);
+      db = __ldg(da + e1);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if (h == 1 && !two) break;
+      const size_t e = h ? e1 : e0;
+      const int c0 = (int)(e % C8) * 8;
+      float yv[8], dv[8], o[8];
+      unpack8(h ? yb : ya, yv);
+      unpack8(h ? db : da0, dv);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int c = c0 + i;
+        const float dz = fmaf(yv[i], cs[c], cs[C + c]) > 0.f ? dv[i] : 0.f;
+        const float xh = (yv[i] - cs[2 * C + c]) * cs[3 * C + c];
+        o[i] = cs[c] * (dz - cs[4 * C + c] - xh * cs[5 * C + c]);
+      }
+      dy[e] = pack8(o);
+    }
+  }
+}
+
+
+// Same result with per-thread constants: when 256 % C8 == 0 a thread keeps its 8 channels over the whole
+// grid-stride loop, and dy = s*dz + k1*y + k0 with k1 = -s*m2*invstd, k0 = s*(m2*invstd*mu - m1),
+// m1 = sum(dz)/M, m2 = sum(dz*xhat)/M: five instructions per element.
+__global__ void __launch_bounds__(256) bn_bwd_apply_vec2_kernel(const uint4* __restrict__ y, const uint4* __restrict__ da, int C8,
+                                                                const float* __restrict__ scale, const float* __restrict__ shift,
+                                                                const float* __restrict__ mu, const float* __restrict__ invstd,
+                                                                const float* __restrict__ sdz, const float* __restrict__ sdzx,
+                                                                float invM, size_t total8, uint4* __restrict__ dy) {
+  const int c0 = (threadIdx.x % C8) * 8;
+  float A[8], B[8], K1[8], K0[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float s = scale[c0 + i], m1 = sdz[c0 + i] * invM, m2 = sdzx[c0 + i] * invM, is = invstd[c0 + i];
+    A[i] = s;
+    B[i] = shift[c0 + i];
+    K1[i] = -s * m2 * is;
+    K0[i] = s * (m2 * is * mu[c0 + i] - m1);
+  }
+  const size_t stride = (size_t)gridDim.x * 256;
+  for (size_t e0 = (size_t)blockIdx.x * 256 + threadIdx.x; e0 < total8; e0 += 2 * stride) {
+    const size_t e1 = e0 + stride;
+    const bool two = e1 < total8;
+    const uint4 ya = __ldg(y + e0), da0 = __ldg(da + e0);
+    uint4 yb = ya, db = da0;
+    if (two) {
+      yb = __ldg(y + e1);
+      db = __ldg(da + e1);
+    }
     float yv[8], dv[8], o[8];
-    unpack8(__ldg(y + e), yv);
-    unpack8(__ldg(da + e), dv);
+    unpack8(ya, yv);
+    unpack8(da0, dv);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const int c = c0 + i;
-      const float dz = fmaf(yv[i], cs[c], cs[C + c]) > 0.f ? dv[i] : 0.f;
-      const float xh = (yv[i] - cs[2 * C + c]) * cs[3 * C + c];
-      o[i] = cs[c] * (dz - cs[4 * C + c] - xh * cs[5 * C + c]);
+      const float dz = fmaf(yv[i], A[i], B[i]) > 0.f ? dv[i] : 0.f;
+      o[i] = fmaf(A[i], dz, fmaf(K1[i], yv[i], K0[i]));
     }
-    dy[e] = pack8(o);
+    dy[e0] = pack8(o);
+    if (two) {
+      unpack8(yb, yv);
+      unpack8(db, dv);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float dz = fmaf(yv[i], A[i], B[i]) > 0.f ? dv[i] : 0.f;
+        o[i] = fmaf(A[i], dz, fmaf(K1[i], yv[i], K0[i]));
+      }
+      dy[e1] = pack8(o);
+    }
   }
 }
 
@@ -620,7 +739,7 @@ inline bool vec_ok(int dtype, int C, int pool) { return dtype == NF_BF16 && C % 
 inline int vec_blocks(size_t work_items) {
   size_t b = (work_items + 256 * 8 - 1) / (256 * 8);
   if (b < 1) b = 1;
-  if (b > 148 * 8) b = 148 * 8;
+  if (b > 148 * 16) b = 148 * 16;
   return (int)b;
 }
 
@@ -677,6 +796,11 @@ int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float ep
 int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
                     const float* shift, void* out) {
   const size_t total = (size_t)N * (pool ? Ho / 2 : Ho) * (pool ? Wo / 2 : Wo) * C;
+  if (vec_ok(dtype, C, pool) && 256 % (C / 8) == 0) {
+    bn_apply_vec2_kernel<<<vec_blocks(total / 8), 256, 0, g_nf_stream>>>((const uint4*)y, C / 8, scale, shift, total / 8, (uint4*)out);
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   if (vec_ok(dtype, C, pool)) {
     bn_apply_vec_kernel<<<vec_blocks(total / 8), 256, 2 * C * sizeof(float), g_nf_stream>>>((const uint4*)y, C / 8, scale, shift,
                                                                                          total / 8, (uint4*)out);
@@ -792,6 +916,12 @@ int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho,
                         const float* sdz, const float* sdzx, double M, void* dy) {
   const size_t total = (size_t)N * Ho * Wo * C;
   const float invM = (float)(1.0 / M);
+  if (vec_ok(dtype, C, pool) && 256 % (C / 8) == 0) {
+    bn_bwd_apply_vec2_kernel<<<vec_blocks(total / 8), 256, 0, g_nf_stream>>>((const uint4*)y, (const uint4*)da, C / 8, scale, shift, mu,
+                                                                            invstd, sdz, sdzx, invM, total / 8, (uint4*)dy);
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   if (vec_ok(dtype, C, pool)) {
     bn_bwd_apply_vec_kernel<<<vec_blocks(total / 8), 256, 6 * C * sizeof(float), g_nf_stream>>>(
         (const uint4*)y, (const uint4*)da, C / 8, scale, shift, mu, invstd, sdz, sdzx, invM, total / 8, (uint4*)dy);
