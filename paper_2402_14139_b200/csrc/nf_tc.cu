@@ -566,7 +566,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 // end they are written to a per-CTA partial that a second kernel sums in a fixed order.
 struct WgParams {
   int N, H, W, Cin, Cout;
-  int BW, BH, tiles_w, tiles_h, pix_tiles, ci_chunks, co_chunks, splits;
+  int BW, BH, tiles_w, tiles_h, pix_tiles, ci_chunks, co_chunks, splits, stages;
   float* part;      // [splits][9][Cout][Cin]
   int32_t* status;
 };
@@ -723,6 +723,147 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
               if (q * 16 + e < co_left) dst[(size_t)e * p.Cin] = __uint_as_float(v[e]);
           }
         }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(p.status, NF_ETIMEOUT);
+    const unsigned long long tt = ptx::globaltimer();
+    while (ptx::globaltimer() - tt < 2000000ull) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kCols);
+  }
+}
+
+// ---------------------------------------------------------------- weight gradient, stride 1, column shift on the gradient
+// dW[kh,kw][co][ci] = sum_{i,j} dy[i,j,co] * x[i+kh-1, j+kw-1, ci].  With j' = j+kw-1 this is
+//   sum over the pixels (i,j') of the x grid of  x[i+kh-1, j', ci] * dy[i, j'-kw+1, co]   (dy = 0 outside),
+// so the column tap can sit on the gradient operand: ONE activation box (BH+2 rows, no column copies)
+// and three column-shifted gradient tiles per stage.  Per 16 pixels two instructions:
+//   A (M = 128) = rows kh=0 and kh=1 of the box stacked (second one half empty: kh=2 + unused rows),
+//   B (N = 3*NB) = the three shifted gradient tiles side by side (MN-major atoms one tile apart).
+// Fewer operand bytes per useful FLOP than stacking all nine taps on the activation side.
+template <int NB>
+__global__ void __launch_bounds__(kThreads, 1)
+conv_wgrad_kw_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_dy, const WgParams p) {
+  constexpr int kBRow = NB * 2;
+  constexpr uint32_t kBLayout = NB == 64 ? 2 : NB == 32 ? 4 : 6;
+  constexpr int kBTile = 128 * kBRow;                 // one shifted gradient tile
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int box_bytes = (p.BH + 2) * p.BW * 128;
+  const int g_region = 3 * kBTile < 4096 ? 4096 : 3 * kBTile;  // >= 32 rows after the box for the unused operand rows
+  const int stage_bytes = box_bytes + g_region;
+  const int stages = p.stages;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + kMaxStages;
+  uint64_t* done = bars + 2 * kMaxStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  constexpr uint32_t kAcc = NB == 64 ? 256 : 3 * NB <= 64 ? 64 : 128;  // columns reserved per accumulator
+  constexpr uint32_t kCols = 2 * kAcc;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int blocks = p.ci_chunks * p.co_chunks;
+  const int blk = blockIdx.x % blocks, sp = blockIdx.x / blocks;
+  const int cic = blk % p.ci_chunks, coc = blk / p.ci_chunks;
+  const int t0 = (int)((long)p.pix_tiles * sp / p.splits), t1 = (int)((long)p.pix_tiles * (sp + 1) / p.splits);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    ptx::mbar_init(done, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tmap(&tm_x);
+    ptx::prefetch_tmap(&tm_dy);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    uint32_t it = 0;
+    for (int t = t0; t < t1; ++t, ++it) {
+      const int s = it % stages;
+      const uint32_t ph = (it / stages) & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) break;
+      if (lane == 0) {
+        const int w0 = (t % p.tiles_w) * p.BW, h0 = ((t / p.tiles_w) % p.tiles_h) * p.BH, n = t / (p.tiles_w * p.tiles_h);
+        uint8_t* st = smem + (size_t)s * stage_bytes;
+        ptx::mbar_expect_tx(&full[s], (uint32_t)(box_bytes + 3 * kBTile));
+        ptx::tma_load_4d(st, &tm_x, &full[s], cic * 64, w0, h0 - 1, n);
+#pragma unroll
+        for (int kw = 0; kw < 3; ++kw)  // gradient column j = j' - kw + 1
+          ptx::tma_load_4d(st + box_bytes + kw * kBTile, &tm_dy, &full[s], coc * NB, w0 - kw + 1, h0, n);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    constexpr uint32_t idesc = ptx::idesc_bf16(128, 3 * NB, 1, 1);
+    const uint64_t a_hi = ptx::sdesc(0, p.BW * 128, 1024, 2);      // second 64 rows: one image row further
+    const uint64_t b_hi = ptx::sdesc(0, kBTile, 8 * kBRow, kBLayout);  // next N atom: next shifted tile
+    const uint32_t row16 = (uint32_t)(p.BW * 128) >> 4;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = t0; t < t1; ++t, ++it) {
+      const int s = it % stages;
+      const uint32_t ph = (it / stages) & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[s], ph, abort_flag))) { ok = false; break; }
+      ptx::tc_fence_after();
+      if (lane == 0) {
+        const uint32_t xb = ptx::smem_u32(smem + (size_t)s * stage_bytes);
+        const uint32_t x16 = xb >> 4, g16 = (xb + box_bytes) >> 4;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint64_t bd = b_hi | (uint64_t)(g16 + k * kBRow);   // 16 pixels x kBRow bytes = k * kBRow sixteen-byte units
+          const uint32_t acc = (it | k) != 0;
+          ptx::mma_f16(tmem_base, a_hi | (uint64_t)(x16 + k * 128), bd, idesc, acc);                      // kh = 0 | 1
+          ptx::mma_f16(tmem_base + kAcc, a_hi | (uint64_t)(x16 + 2 * row16 + k * 128), bd, idesc, acc);  // kh = 2 | unused
+        }
+        ptx::mma_commit(&empty[s]);
+      }
+      __syncwarp();
+    }
+    if (ok && lane == 0) ptx::mma_commit(done);
+    __syncwarp();
+  } else {
+    const int lg = warp & 3, m = lg * 32 + lane;
+    if (ptx::mbar_wait(done, 0, abort_flag) && t1 > t0) {
+      ptx::tc_fence_after();
+      const size_t plane = (size_t)p.Cout * p.Cin;
+      float* base = p.part + (size_t)sp * 9 * plane + (size_t)(coc * NB) * p.Cin + cic * 64 + (m & 63);
+      const int co_left = p.Cout - coc * NB;
+#pragma unroll 1
+      for (int j = 0; j < 2; ++j) {
+        const int kh = j == 0 ? (m < 64 ? 0 : 1) : (m < 64 ? 2 : -1);
+#pragma unroll 1
+        for (int kw = 0; kw < 3; ++kw)
+#pragma unroll
+          for (int q = 0; q < NB / 16; ++q) {
+            uint32_t v[16];
+            ptx::tmem_ld16(tmem_base + ((uint32_t)(lg * 32) << 16) + j * kAcc + kw * NB + q * 16, v);
+            ptx::tmem_ld_wait();
+            if (kh >= 0) {
+              float* dst = base + (size_t)(kh * 3 + kw) * plane + (size_t)(q * 16) * p.Cin;
+#pragma unroll
+              for (int e = 0; e < 16; ++e)
+                if (q * 16 + e < co_left) dst[(size_t)e * p.Cin] = __uint_as_float(v[e]);
+            }
+          }
       }
     }
   }
@@ -964,7 +1105,7 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
 }
 
 struct WgPlan {
-  int ok, BW, BH, NB, splits, grid;
+  int ok, BW, BH, NB, splits, grid, stages;
   size_t smem, part_floats;
 };
 
@@ -982,10 +1123,15 @@ WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0, int strid
       break;
     }
   if (!pl.BW) return pl;
-  const size_t stage = stride == 2 ? 65536 : (size_t)3 * (pl.BH + 2) * pl.BW * 128 + 16384;
-  pl.smem = (stride == 2 ? 3 : 2) * stage + 1024 + 1024;
-  if (pl.smem > 232448) return pl;
   pl.NB = aux ? (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64) : 64;
+  size_t g_region = (size_t)3 * 128 * pl.NB * 2;
+  if (g_region < 4096) g_region = 4096;
+  const size_t stage = stride == 2 ? 65536 : (size_t)(pl.BH + 2) * pl.BW * 128 + g_region;
+  pl.stages = stride == 2 ? 3 : (int)((232448 - 2048) / stage);
+  if (pl.stages > kMaxStages) pl.stages = kMaxStages;
+  if (pl.stages < 2) return pl;
+  pl.smem = (size_t)pl.stages * stage + 1024 + 1024;
+  if (pl.smem > 232448) return pl;
   const int blocks = (Cin / 64) * (aux ? 1 : Cout / 64);
   const long pix_tiles = (long)N * (H / pl.BH) * (W / pl.BW);
   const int groups = stride == 2 ? 3 : 1;  // kernel rows handled by separate CTAs
@@ -997,6 +1143,18 @@ WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0, int strid
   pl.part_floats = (size_t)sp * 9 * Cout * Cin;
   pl.ok = 1;
   return pl;
+}
+
+template <int NB>
+int launch_wgrad_kw(const WgPlan& pl, const CUtensorMap& mx, const CUtensorMap& mg, const WgParams& p) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    NF_CUDA(cudaFuncSetAttribute(conv_wgrad_kw_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    attr_done = true;
+  }
+  conv_wgrad_kw_kernel<NB><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mg, p);
+  NF_LAUNCHED();
+  return NF_OK;
 }
 
 template <int NB, int S2 = 0>
@@ -1030,10 +1188,12 @@ int run_wgrad(int N, int Hin, int Win, int Cin, int Cout, const void* x, const v
   p.N = N; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout; p.BW = pl.BW; p.BH = pl.BH;
   p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.pix_tiles = N * p.tiles_h * p.tiles_w;
   p.ci_chunks = Cin / 64; p.co_chunks = aux ? 1 : Cout / 64; p.splits = pl.splits; p.part = part; p.status = status;
+  p.stages = pl.stages;
   if (stride == 2)
     rc = launch_wgrad<64, 1>(pl, mx, mg, p);
   else
-    rc = pl.NB == 64 ? launch_wgrad<64>(pl, mx, mg, p) : pl.NB == 32 ? launch_wgrad<32>(pl, mx, mg, p) : launch_wgrad<16>(pl, mx, mg, p);
+    rc = pl.NB == 64 ? launch_wgrad_kw<64>(pl, mx, mg, p)
+                     : pl.NB == 32 ? launch_wgrad_kw<32>(pl, mx, mg, p) : launch_wgrad_kw<16>(pl, mx, mg, p);
   if (rc != NF_OK) return rc;
   const size_t n = (size_t)9 * Cout * Cin;
   sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, g_nf_stream>>>(part, pl.splits, n, dw);
