@@ -19,6 +19,7 @@ namespace {
 
 constexpr int kThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
 constexpr int kMaxStages = 8;
+constexpr int kFoldThreads = 320;  // folded-tap forward: producer, MMA issuer and two epilogue groups of four warps
 
 struct FwdParams {
   int N, H, W, Cin, Cout;
@@ -331,7 +332,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 // same warp.  14 x 8 output pixels per tile; needs W % 14 == 0 and H % 8 == 0.
 struct FoldParams {
   int N, H, W, Cout, kchunks, tiles_w, tiles_h, total_tiles, stages, stats;
-  float* red;         // EPI 0: [grid * 2][2][64]
+  float* red;         // EPI 0: [grid * 4][2][64]
   int32_t* status;
   const float* bias;  // EPI 1
   bf16* out;          // EPI 1: [N][H][W][Cout]
@@ -343,7 +344,7 @@ struct FoldParams {
 //       1 = bias + ReLU, F channels written straight from registers (aux conv forward).
 // Cin = 64 * kchunks; all 9 * kchunks weight tiles stay resident in shared memory.
 template <int G, int EPI>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kFoldThreads, 1)
 conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                      const __grid_constant__ CUtensorMap tm_y, const FoldParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -353,7 +354,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   const int w_bytes = 3 * p.kchunks * kWTile; // [chunk][kh][kw*G + co][64 ci]
   uint8_t* wres = smem + (size_t)p.stages * kABytes;
   uint8_t* stg = wres + w_bytes;              // EPI 0: 112 output pixels x 128 bytes
-  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (EPI == 0 ? 16384 : 0));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (EPI == 0 ? 2 * 16384 : 0));  // one staging tile per epilogue group
   uint64_t* full = bars;
   uint64_t* empty = bars + kMaxStages;
   uint64_t* tfull = bars + 2 * kMaxStages;
@@ -361,7 +362,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   uint64_t* wfull = tempty + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wfull + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);
+  volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);  // [2], one per epilogue group
   constexpr uint32_t kAccStride = G == 64 ? 256 : 128;  // columns between the two accumulators
   constexpr uint32_t kTmemCols = 2 * kAccStride;
 
@@ -446,7 +447,10 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       __syncwarp();
     }
   } else {
-    const int et = threadIdx.x - 64;
+    // two epilogue groups of 128 threads; group g owns accumulator g and takes every second tile of the CTA
+    const int grp = (threadIdx.x - 64) >> 7;
+    const int et = (threadIdx.x - 64) & 127;
+    uint8_t* const stg_g = stg + grp * 16384;
     const int lg = warp & 3;
     const int r = lg * 32 + lane;            // TMEM lane = extended-tile pixel (we = r % 16, h = r / 16)
     const int we = r & 15, hh = r >> 4;
@@ -454,18 +458,18 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     const int orow = (we - 1) + 14 * hh;     // row of the output staging tile
     const int sc = et & 63, shalf = et >> 6; // stats: channel, and which 56 of the 112 rows
     float ssum = 0.f, ssq = 0.f;
-    uint32_t tl = 0;
-    for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++tl) {
-      const int w0 = (t % p.tiles_w) * 14, h0 = ((t / p.tiles_w) % p.tiles_h) * 8, n = t / (p.tiles_w * p.tiles_h);
-      const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+    uint32_t tl = grp;
+    for (long t = blockIdx.x + (long)grp * gridDim.x; t < p.total_tiles; t += 2L * gridDim.x, tl += 2) {
+      const int w0 = (int)(t % p.tiles_w) * 14, h0 = (int)((t / p.tiles_w) % p.tiles_h) * 8, n = (int)(t / (p.tiles_w * p.tiles_h));
+      const uint32_t acc = grp, aph = (tl >> 1) & 1;
       ptx::mbar_wait(&tfull[acc], aph, abort_flag);
       ptx::tc_fence_after();
       if (et == 0) {
         if constexpr (EPI == 0) ptx::tma_store_wait_read();
-        *epi_go = *abort_flag ? 0 : 1;
+        epi_go[grp] = *abort_flag ? 0 : 1;
       }
-      ptx::named_barrier(1, 128);
-      if (!*epi_go) break;
+      ptx::named_barrier(1 + grp, 128);
+      if (!epi_go[grp]) break;
       const uint32_t tbase = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * kAccStride;
       bf16* gdst = EPI == 1 ? p.out + (((size_t)n * p.H + h0 + hh) * p.W + w0 + we - 1) * p.Cout : nullptr;
 #pragma unroll
@@ -495,7 +499,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         }
         if constexpr (EPI == 0) {
           if (valid) {
-            uint8_t* dst = stg + orow * 128;
+            uint8_t* dst = stg_g + orow * 128;
             *reinterpret_cast<uint4*>(dst + (((2 * q) ^ (orow & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
             *reinterpret_cast<uint4*>(dst + (((2 * q + 1) ^ (orow & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
           }
@@ -511,13 +515,13 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       ptx::mbar_arrive(&tempty[acc]);
       if constexpr (EPI == 0) {
         ptx::fence_async_smem();
-        ptx::named_barrier(1, 128);
+        ptx::named_barrier(1 + grp, 128);
         if (et == 0) {
-          ptx::tma_store_4d(&tm_y, stg, 0, w0, h0, n);
+          ptx::tma_store_4d(&tm_y, stg_g, 0, w0, h0, n);
           ptx::tma_store_commit();
         }
         if (p.stats) {
-          const uint8_t* col = stg + (sc & 7) * 2;
+          const uint8_t* col = stg_g + (sc & 7) * 2;
           const int u = sc >> 3;
 #pragma unroll 8
           for (int rr = 0; rr < 56; ++rr) {
@@ -532,7 +536,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     if constexpr (EPI == 0) {
       if (et == 0) ptx::tma_store_wait_all();
       if (p.stats) {
-        const size_t b = (size_t)blockIdx.x * 2 + shalf;
+        const size_t b = (size_t)blockIdx.x * 4 + grp * 2 + shalf;
         p.red[(b * 2 + 0) * 64 + sc] = ssum;
         p.red[(b * 2 + 1) * 64 + sc] = ssq;
       }
@@ -993,7 +997,7 @@ bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride) {
   if (stride != 1 || W % 14 || H % 8 || Cin % 64) return false;
   if (epi == 0 ? (Cin != 64 || Cout != 64) : epi == 1 ? (Cout > 64 || Cout % 8) : true) return false;
   const size_t wbytes = (size_t)9 * (Cin / 64) * fold_group(Cout, epi) * 128;
-  return wbytes + (epi == 0 ? 16384 : 0) + 2048 + 3 * 20480 <= 232448;
+  return wbytes + (epi == 0 ? 2 * 16384 : 0) + 2048 + 3 * 20480 <= 232448;
 }
 
 template <int G, int EPI>
@@ -1003,7 +1007,7 @@ int launch_fold(int grid, size_t smem, const CUtensorMap& mx, const CUtensorMap&
     NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel<G, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
   }
-  conv_fwd_fold_kernel<G, EPI><<<grid, kThreads, smem, g_nf_stream>>>(mx, mw, my, p);
+  conv_fwd_fold_kernel<G, EPI><<<grid, kFoldThreads, smem, g_nf_stream>>>(mx, mw, my, p);
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -1030,7 +1034,7 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = Cin / 64;
   p.tiles_w = W / 14; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h;
   p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
-  const size_t fixed = (size_t)9 * p.kchunks * G * 128 + (epi == 0 ? 16384 : 0) + 1024 + 1024;
+  const size_t fixed = (size_t)9 * p.kchunks * G * 128 + (epi == 0 ? 2 * 16384 : 0) + 1024 + 1024;
   int st = (int)((232448 - fixed) / 20480);
   if (st > kMaxStages) st = kMaxStages;
   p.stages = st;
@@ -1038,10 +1042,10 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   int grid = sm_count();
   if (grid > p.total_tiles) grid = p.total_tiles;
   if (stats) {
-    const size_t need = (size_t)grid * 2 * 2 * 64;
+    const size_t need = (size_t)grid * 4 * 2 * 64;
     if (need > red_floats) return NF_ENOWS;
     NF_CUDA(cudaMemsetAsync(red, 0, need * sizeof(float), g_nf_stream));
-    *nb = grid * 2;
+    *nb = grid * 4;
   }
   if (epi == 0) return launch_fold<64, 0>(grid, smem, mx, mw, my, p);
   return G == 16 ? launch_fold<16, 1>(grid, smem, mx, mw, my, p)
@@ -1221,7 +1225,7 @@ size_t nf_tc_scratch_floats(const nf_layer* L) {
 size_t nf_tc_red_floats(const nf_layer* L) {
   if (!L->fam[0]) return 0;
   const TcPlan pl = plan_fwd(L->Ho, L->Wo, L->Cin, L->Cout, L->o.N, 0, L->o.stride);
-  return (size_t)sm_count() * pl.parts * 2 * L->Cout;
+  return (size_t)sm_count() * (pl.parts < 4 ? 4 : pl.parts) * 2 * L->Cout;  // the folded kernel writes 4 partials per CTA
 }
 
 int nf_tc_prepare(nf_layer*) { return NF_OK; }
