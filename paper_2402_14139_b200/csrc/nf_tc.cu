@@ -331,7 +331,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 // two columns are halo, so the left/right neighbours of every output pixel are adjacent TMEM lanes of the
 // same warp.  14 x 8 output pixels per tile; needs W % 14 == 0 and H % 8 == 0.
 struct FoldParams {
-  int N, H, W, Cout, kchunks, tiles_w, tiles_h, total_tiles, stages, stats;
+  int N, H, W, Cout, kchunks, n_tiles, tiles_w, tiles_h, total_tiles, stages, stats;
   float* red;         // EPI 0: [grid * 4][2][64]
   int32_t* status;
   const float* bias;  // EPI 1
@@ -343,14 +343,19 @@ struct FoldParams {
 // EPI : 0 = y in bf16 through a TMA store + BatchNorm partial sums (G = 64, Cout = 64);
 //       1 = bias + ReLU, F channels written straight from registers (aux conv forward).
 // Cin = 64 * kchunks; all 9 * kchunks weight tiles stay resident in shared memory.
-template <int G, int EPI>
+// KC / MIR: KC = channels of the activation box (64; 16 or 32 for the aux input gradient whose input dh has F
+// channels), MIR = 1 reads the weights [tap][f][c] MN-major with both taps mirrored (input-gradient convolution;
+// the CTA's 64-channel output tile is blockIdx.x % n_tiles).
+template <int G, int EPI, int KC = 64, int MIR = 0>
 __global__ void __launch_bounds__(kFoldThreads, 1)
 conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                      const __grid_constant__ CUtensorMap tm_y, const FoldParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr int kABytes = 10 * 16 * 128;      // (8+2) rows x 16 pixels x 64 channels
-  constexpr int kWTile = 3 * G * 128;         // one kernel row of one chunk: [kw*G + co][64 ci]
+  constexpr int kARow = KC * 2;               // bytes of one pixel of the activation box
+  constexpr uint32_t kALayout = KC == 64 ? 2 : KC == 32 ? 4 : 6;
+  constexpr int kABytes = 10 * 16 * kARow;    // (8+2) rows x 16 pixels x KC channels
+  constexpr int kWTile = MIR ? 3 * KC * 128 : 3 * G * 128;  // one kernel row: [kw*G + co][64 ci], or mirrored [kw][f][64 c]
   const int w_bytes = 3 * p.kchunks * kWTile; // [chunk][kh][kw*G + co][64 ci]
   uint8_t* wres = smem + (size_t)p.stages * kABytes;
   uint8_t* stg = wres + w_bytes;              // EPI 0: 112 output pixels x 128 bytes
@@ -397,27 +402,30 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       ptx::mbar_expect_tx(wfull, (uint32_t)w_bytes);
       for (int ck = 0; ck < p.kchunks; ++ck)
 #pragma unroll
-        for (int kh = 0; kh < 3; ++kh) ptx::tma_load_4d(wres + (ck * 3 + kh) * kWTile, &tm_w, wfull, ck * 64, 0, 0, kh);
+        for (int kh = 0; kh < 3; ++kh)
+          ptx::tma_load_4d(wres + (ck * 3 + kh) * kWTile, &tm_w, wfull, MIR ? (int)(blockIdx.x % p.n_tiles) * 64 : ck * 64, 0, 0, kh);
     }
     __syncwarp();
     uint32_t it = 0;
     bool ok = true;
     for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x) {
-      const int w0 = (t % p.tiles_w) * 14, h0 = ((t / p.tiles_w) % p.tiles_h) * 8, n = t / (p.tiles_w * p.tiles_h);
+      const int m = t / p.n_tiles;
+      const int w0 = (m % p.tiles_w) * 14, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
       for (int ck = 0; ck < p.kchunks; ++ck, ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) { ok = false; break; }
         if (lane == 0) {
           ptx::mbar_expect_tx(&full[s], (uint32_t)kABytes);
-          ptx::tma_load_4d(smem + (size_t)s * kABytes, &tm_x, &full[s], ck * 64, w0 - 1, h0 - 1, n);
+          ptx::tma_load_4d(smem + (size_t)s * kABytes, &tm_x, &full[s], ck * KC, w0 - 1, h0 - 1, n);
         }
         __syncwarp();
       }
     }
   } else if (warp == 1) {
-    constexpr uint32_t idesc = ptx::idesc_bf16(128, 3 * G, 0, 0);
-    const uint64_t hi = ptx::sdesc(0, 16, 1024, 2);
+    constexpr uint32_t idesc = ptx::idesc_bf16(128, 3 * G, 0, MIR);
+    const uint64_t a_hi = ptx::sdesc(0, 16, 8 * kARow, kALayout);
+    const uint64_t b_hi = MIR ? ptx::sdesc(0, KC * 128, 1024, 2) : ptx::sdesc(0, 16, 1024, 2);
     const uint32_t w16 = ptx::smem_u32(wres) >> 4;
     uint32_t it = 0, tl = 0;
     bool ok = blockIdx.x >= p.total_tiles || __all_sync(0xffffffffu, ptx::mbar_wait(wfull, 0, abort_flag));
@@ -436,9 +444,12 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
           for (int kh = 0; kh < 3; ++kh)
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              ptx::mma_f16(d, hi | (uint64_t)(a16 + kh * 128 + k * 2),
-                           hi | (uint64_t)(w16 + (ck * 3 + kh) * (kWTile >> 4) + k * 2), idesc, (ck | kh | k) != 0);
+            for (int k = 0; k < KC / 16; ++k) {
+              const uint64_t ad = a_hi | (uint64_t)(a16 + kh * (16 * kARow >> 4) + k * 2);
+              const uint64_t bd = MIR ? b_hi | (uint64_t)(w16 + (2 - kh) * (kWTile >> 4) + k * 128)   // mirrored row tap, 16 f rows on
+                                      : b_hi | (uint64_t)(w16 + (ck * 3 + kh) * (kWTile >> 4) + k * 2);
+              ptx::mma_f16(d, ad, bd, idesc, (ck | kh | k) != 0);
+            }
           ptx::mma_commit(&empty[s]);
         }
         __syncwarp();
@@ -460,7 +471,9 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     float ssum = 0.f, ssq = 0.f;
     uint32_t tl = grp;
     for (long t = blockIdx.x + (long)grp * gridDim.x; t < p.total_tiles; t += 2L * gridDim.x, tl += 2) {
-      const int w0 = (int)(t % p.tiles_w) * 14, h0 = (int)((t / p.tiles_w) % p.tiles_h) * 8, n = (int)(t / (p.tiles_w * p.tiles_h));
+      const int nt = (int)(t % p.n_tiles);
+      const long m = t / p.n_tiles;
+      const int w0 = (int)(m % p.tiles_w) * 14, h0 = (int)((m / p.tiles_w) % p.tiles_h) * 8, n = (int)(m / (p.tiles_w * p.tiles_h));
       const uint32_t acc = grp, aph = (tl >> 1) & 1;
       ptx::mbar_wait(&tfull[acc], aph, abort_flag);
       ptx::tc_fence_after();
@@ -475,9 +488,9 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
       for (int q = 0; q < G / 16; ++q) {     // 16 output channels at a time
         uint32_t v0[16], v1[16], v2[16];
-        ptx::tmem_ld16(tbase + q * 16, v0);
+        ptx::tmem_ld16(tbase + (MIR ? 2 * G : 0) + q * 16, v0);  // group feeding the pixel on the left
         ptx::tmem_ld16(tbase + G + q * 16, v1);
-        ptx::tmem_ld16(tbase + 2 * G + q * 16, v2);
+        ptx::tmem_ld16(tbase + (MIR ? 0 : 2 * G) + q * 16, v2);  // group feeding the pixel on the right
         ptx::tmem_ld_wait();
         uint32_t w[8];
 #pragma unroll
@@ -517,7 +530,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         ptx::fence_async_smem();
         ptx::named_barrier(1 + grp, 128);
         if (et == 0) {
-          ptx::tma_store_4d(&tm_y, stg_g, 0, w0, h0, n);
+          ptx::tma_store_4d(&tm_y, stg_g, nt * 64, w0, h0, n);
           ptx::tma_store_commit();
         }
         if (p.stats) {
@@ -990,24 +1003,27 @@ int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, c
   return NF_OK;
 }
 
-// The folded-tap kernel covers: main forward 64 -> 64 (epi 0) and the aux forward with F <= 64, F % 8 == 0
-// (epi 1), when W % 14 == 0, H % 8 == 0 and all weight tiles fit in shared memory beside >= 3 activation stages.
-int fold_group(int Cout, int epi) { return epi == 0 ? 64 : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64); }
+// The folded-tap kernel covers, when W % 14 == 0 and H % 8 == 0: the main forward 64 -> 64 (epi 0), the aux
+// forward with F <= 64, F % 8 == 0 (epi 1) if all weight tiles fit in shared memory beside >= 3 activation
+// stages, and the aux input gradient F -> Cout (epi 2; F <= 32, F % 8 == 0, Cout % 64 == 0).
+int fold_group(int Cout, int epi) { return epi != 1 ? 64 : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64); }
 bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride) {
-  if (stride != 1 || W % 14 || H % 8 || Cin % 64) return false;
-  if (epi == 0 ? (Cin != 64 || Cout != 64) : epi == 1 ? (Cout > 64 || Cout % 8) : true) return false;
+  if (stride != 1 || W % 14 || H % 8) return false;
+  if (epi == 2) return Cin <= 32 && Cin % 8 == 0 && Cout % 64 == 0;
+  if (Cin % 64) return false;
+  if (epi == 0 ? (Cin != 64 || Cout != 64) : (Cout > 64 || Cout % 8)) return false;
   const size_t wbytes = (size_t)9 * (Cin / 64) * fold_group(Cout, epi) * 128;
   return wbytes + (epi == 0 ? 2 * 16384 : 0) + 2048 + 3 * 20480 <= 232448;
 }
 
-template <int G, int EPI>
+template <int G, int EPI, int KC = 64, int MIR = 0>
 int launch_fold(int grid, size_t smem, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const FoldParams& p) {
   static bool attr_done = false;
   if (!attr_done) {
-    NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel<G, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel<G, EPI, KC, MIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
   }
-  conv_fwd_fold_kernel<G, EPI><<<grid, kFoldThreads, smem, g_nf_stream>>>(mx, mw, my, p);
+  conv_fwd_fold_kernel<G, EPI, KC, MIR><<<grid, kFoldThreads, smem, g_nf_stream>>>(mx, mw, my, p);
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -1015,31 +1031,38 @@ int launch_fold(int grid, size_t smem, const CUtensorMap& mx, const CUtensorMap&
 int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
              size_t red_floats, int32_t* status, int* nb, int epi, const float* bias) {
   const int G = fold_group(Cout, epi);
+  const int KC = epi == 2 ? (Cin <= 16 ? 16 : 32) : 64;
   CUtensorMap mx, mw, my;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t bx[4] = {64, 16, 10, 1};
-  const uint64_t dw[4] = {(uint64_t)Cin, (uint64_t)Cout, 3, 3};
-  const uint32_t bw[4] = {64, (uint32_t)G, 3, 1};
+  const uint32_t bx[4] = {(uint32_t)KC, 16, 10, 1};
+  // forward: weights [kh][kw][Cout][Cin], box = G rows of co x 64 ci for the three kw of one kh;
+  // input gradient: weights [kh][kw][F][Cout], box = KC rows of f x 64 c for the three kw of one kh
+  const uint64_t dw[4] = {(uint64_t)(epi == 2 ? Cout : Cin), (uint64_t)(epi == 2 ? Cin : Cout), 3, 3};
+  const uint32_t bw[4] = {64, (uint32_t)(epi == 2 ? KC : G), 3, 1};
   const uint64_t dy[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
   const uint32_t by[4] = {64, 14, 8, 1};
   int rc;
   if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
   if ((rc = make_map4(&mw, w, dw, bw)) != NF_OK) return rc;
-  if (epi == 0) {
+  if (epi != 1) {
     if ((rc = make_map4(&my, y, dy, by)) != NF_OK) return rc;
   } else {
     my = mx;
   }
   FoldParams p{};
-  p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = Cin / 64;
-  p.tiles_w = W / 14; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h;
+  p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = epi == 2 ? 1 : Cin / 64; p.n_tiles = epi == 2 ? Cout / 64 : 1;
+  p.tiles_w = W / 14; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
   p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
-  const size_t fixed = (size_t)9 * p.kchunks * G * 128 + (epi == 0 ? 2 * 16384 : 0) + 1024 + 1024;
-  int st = (int)((232448 - fixed) / 20480);
+  const size_t a_bytes = (size_t)10 * 16 * KC * 2;
+  const size_t wbytes = epi == 2 ? (size_t)9 * KC * 128 : (size_t)9 * p.kchunks * G * 128;
+  const size_t fixed = wbytes + (epi != 1 ? 2 * 16384 : 0) + 1024 + 1024;
+  int st = (int)((232448 - fixed) / a_bytes);
   if (st > kMaxStages) st = kMaxStages;
   p.stages = st;
-  const size_t smem = (size_t)st * 20480 + fixed;
+  const size_t smem = (size_t)st * a_bytes + fixed;
   int grid = sm_count();
+  grid -= grid % p.n_tiles;  // a CTA keeps one output-channel tile (and its resident weights) for its whole life
+  if (grid < p.n_tiles) grid = p.n_tiles;
   if (grid > p.total_tiles) grid = p.total_tiles;
   if (stats) {
     const size_t need = (size_t)grid * 4 * 2 * 64;
@@ -1048,6 +1071,7 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
     *nb = grid * 4;
   }
   if (epi == 0) return launch_fold<64, 0>(grid, smem, mx, mw, my, p);
+  if (epi == 2) return KC == 16 ? launch_fold<64, 0, 16, 1>(grid, smem, mx, mw, my, p) : launch_fold<64, 0, 32, 1>(grid, smem, mx, mw, my, p);
   return G == 16 ? launch_fold<16, 1>(grid, smem, mx, mw, my, p)
                  : G == 32 ? launch_fold<32, 1>(grid, smem, mx, mw, my, p) : launch_fold<64, 1>(grid, smem, mx, mw, my, p);
 }

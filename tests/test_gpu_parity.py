@@ -131,6 +131,7 @@ TC = [
     dict(N=3, Cin=64, Cout=64, H=16, W=112, F=16, classes=10, stride=1, pool=False),  # folded-tap forward (W % 14 == 0)
     dict(N=3, Cin=64, Cout=128, H=16, W=112, F=8, classes=10, stride=1, pool=False),  # folded aux forward, two K chunks, F < 16
     dict(N=3, Cin=64, Cout=64, H=16, W=112, F=40, classes=10, stride=1, pool=False),  # folded aux forward, group width 64
+    dict(N=3, Cin=64, Cout=64, H=16, W=112, F=32, classes=10, stride=1, pool=False),  # folded aux input gradient, 32-channel K
 ]
 
 
