@@ -24,6 +24,7 @@ constexpr int kFoldThreads = 320;  // folded-tap forward: producer, MMA issuer a
 struct FwdParams {
   int N, H, W, Cin, Cout;
   int BW, BH, tiles_w, tiles_h, n_tiles, total_tiles, kchunks, stages;
+  int stride, BI;     // PT mode: conv stride and images per tile (BW*BH*BI = 128)
   int stats;
   float* red;         // [grid * parts][2][Cout] channel partials (pre-zeroed)
   int32_t* status;    // device status word
@@ -32,7 +33,7 @@ struct FwdParams {
 };
 
 struct TcPlan {
-  int ok, BW, BH, BN, KC, RW, stages, grid, parts;
+  int ok, BW, BH, BI, PT, BN, KC, RW, stages, grid, parts;
   size_t smem;
 };
 
@@ -43,8 +44,9 @@ struct TcPlan {
 //       input gradient; rows of 2*KC bytes with the matching TMA swizzle).
 // BMN : 0 = weights [tap][co][ci] read K-major (forward); 1 = weights [tap][f][c] read MN-major with the
 //       taps mirrored, which makes the same kernel the input-gradient convolution da = dh (*) Wa^T.
-// PT  : 1 = one TMA box per tap (stride-2 convolution: the box is gathered with element stride 2, so the
-//       three row taps cannot share a box); p.H, p.W are then the OUTPUT sizes.
+// PT  : 1 = one TMA box per tap: stride-2 convolutions (the box is gathered with element stride 2, so the
+//       three row taps cannot share a box) and feature maps smaller than a tile, where a tile spans BI whole
+//       images (8x8x2, 4x4x8, 2x2x32); p.H, p.W are the OUTPUT sizes.
 // RW  : 1 = all nine weight tiles of the CTA's channel tile stay resident in shared memory for the whole
 //       kernel (single 64-channel K chunk, 9*BN*128 bytes); the pipeline then carries activations only.
 template <int BN, int EPI, int KC = 64, int BMN = 0, int PT = 0, int RW = 0>
@@ -55,9 +57,9 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int kARow = KC * 2;  // bytes of one pixel row of the activation box
   constexpr uint32_t kALayout = KC == 64 ? 2 : KC == 32 ? 4 : 6;
-  const int a_bytes = (PT ? p.BH : p.BH + 2) * p.BW * kARow;
+  const int a_bytes = PT ? 128 * kARow : (p.BH + 2) * p.BW * kARow;
   const int a_stride = (a_bytes + 1023) & ~1023;  // keeps the weight tiles 1024-byte aligned
-  constexpr int b_bytes = RW ? 0 : PT ? BN * 128 : BMN ? (BN / 64) * 3 * KC * 128 : 3 * BN * 128;
+  constexpr int b_bytes = RW ? 0 : PT ? (BMN ? (BN / 64) * KC * 128 : BN * 128) : BMN ? (BN / 64) * 3 * KC * 128 : 3 * BN * 128;
   constexpr int w_bytes = RW ? 9 * BN * 128 : 0;  // resident weights [kw][kh][BN][64]
   const int stage_bytes = a_stride + b_bytes;
   constexpr int kSub = EPI == 0 ? BN / 64 : 0;  // 64-channel sub-tiles of the output staging
@@ -116,7 +118,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     }
     for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x) {
       const int nt = t % p.n_tiles, m = t / p.n_tiles;
-      const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = m / (p.tiles_w * p.tiles_h);
+      const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = (m / (p.tiles_w * p.tiles_h)) * p.BI;
       for (int ks = 0; ks < ksteps; ++ks, ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
@@ -126,8 +128,14 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           ptx::mbar_expect_tx(&full[s], (uint32_t)(a_bytes + b_bytes));
           if constexpr (PT) {
             const int tap = ks % 9, ck = ks / 9, kh = tap / 3, kw = tap % 3;
-            ptx::tma_load_4d(a_s, &tm_x, &full[s], ck * KC, 2 * w0 + kw - 1, 2 * h0 + kh - 1, n);
-            ptx::tma_load_4d(a_s + a_stride, &tm_w, &full[s], ck * 64, nt * BN, kw, kh);
+            ptx::tma_load_4d(a_s, &tm_x, &full[s], ck * KC, p.stride * w0 + kw - 1, p.stride * h0 + kh - 1, n);
+            if constexpr (BMN) {
+#pragma unroll
+              for (int hf = 0; hf < BN / 64; ++hf)  // [half][KC rows of f][64 channels], both taps mirrored
+                ptx::tma_load_4d(a_s + a_stride + hf * KC * 128, &tm_w, &full[s], nt * BN + hf * 64, 0, 2 - kw, 2 - kh);
+            } else {
+              ptx::tma_load_4d(a_s + a_stride, &tm_w, &full[s], ck * 64, nt * BN, kw, kh);
+            }
           } else {
             const int kw = ks % 3, ck = ks / 3;
             ptx::tma_load_4d(a_s, &tm_x, &full[s], ck * KC, w0 + kw - 1, h0 - 1, n);
@@ -150,7 +158,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     bool ok = true;
     // descriptors differ only in their 14-bit address field: constant upper parts, address added per use
     const uint64_t a_hi = ptx::sdesc(0, 16, 8 * kARow, kALayout);
-    const uint64_t b_hi = BMN ? ptx::sdesc(0, 3 * KC * 128, 1024, 2) : ptx::sdesc(0, 16, 1024, 2);
+    const uint64_t b_hi = BMN ? ptx::sdesc(0, (PT ? 1 : 3) * KC * 128, 1024, 2) : ptx::sdesc(0, 16, 1024, 2);
     const uint32_t a_row16 = (uint32_t)(p.BW * kARow) >> 4;  // one image row of the box, in 16-byte units
     if constexpr (RW) {
       if (blockIdx.x < p.total_tiles) ok = __all_sync(0xffffffffu, ptx::mbar_wait(wfull, 0, abort_flag));
@@ -174,7 +182,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 #pragma unroll
             for (int k = 0; k < KC / 16; ++k) {
               const uint64_t ad = a_hi | (uint64_t)(a16 + kh * a_row16 + k * 2);
-              const uint64_t bd = b_hi | (uint64_t)(BMN ? b16 + (((2 - kh) * KC * 128 + k * 16 * 128) >> 4)
+              const uint64_t bd = b_hi | (uint64_t)(BMN ? b16 + (((PT ? 0 : (2 - kh) * KC * 128) + k * 16 * 128) >> 4)
                                                         : b16 + ((kh * BN * 128 + k * 32) >> 4));
               ptx::mma_f16(d, ad, bd, idesc, (ks | kh | k) != 0);
             }
@@ -198,7 +206,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     int my_nt = blockIdx.x % p.n_tiles;
     for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++tl) {
       const int nt = t % p.n_tiles, m = t / p.n_tiles;
-      const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = m / (p.tiles_w * p.tiles_h);
+      const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = (m / (p.tiles_w * p.tiles_h)) * p.BI;
       const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
       ptx::mbar_wait(&tfull[acc], aph, abort_flag);  // sets the abort flag itself when it gives up
       ptx::tc_fence_after();
@@ -262,20 +270,22 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       uint32_t tl = 0;
       for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++tl) {
         const int m = t / p.n_tiles;
-        const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = m / (p.tiles_w * p.tiles_h);
+        const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = (m / (p.tiles_w * p.tiles_h)) * p.BI;
         const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
         ptx::mbar_wait(&tfull[acc], aph, abort_flag);
         ptx::tc_fence_after();
         if (et == 0) *epi_go = *abort_flag ? 0 : 1;
         ptx::named_barrier(1, 128);
         if (!*epi_go) break;
-        bf16* dst = p.out + (((size_t)n * p.H + h0 + r / p.BW) * p.W + w0 + r % p.BW) * p.Cout;
+        const int img = r / (p.BW * p.BH);  // image of this pixel inside a multi-image tile
+        const bool img_ok = n + img < p.N;
+        bf16* dst = p.out + (((size_t)(n + img) * p.H + h0 + (r / p.BW) % p.BH) * p.W + w0 + r % p.BW) * p.Cout;
 #pragma unroll
         for (int j = 0; j < BN / 16; ++j) {
           uint32_t v[16];
           ptx::tmem_ld16(tmem_base + ((uint32_t)(lg * 32) << 16) + acc * BN + j * 16, v);
           ptx::tmem_ld_wait();
-          if (j * 16 < p.Cout) {
+          if (j * 16 < p.Cout && img_ok) {
             uint32_t w[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
@@ -583,14 +593,15 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 // end they are written to a per-CTA partial that a second kernel sums in a fixed order.
 struct WgParams {
   int N, H, W, Cin, Cout;
-  int BW, BH, tiles_w, tiles_h, pix_tiles, ci_chunks, co_chunks, splits, stages;
+  int BW, BH, tiles_w, tiles_h, pix_tiles, ci_chunks, co_chunks, splits, stages, stride, BI;
   float* part;      // [splits][9][Cout][Cin]
   int32_t* status;
 };
 
 // NB = width of the output-gradient tile in channels (64: main conv, one 64-channel chunk per CTA;
 // 16/32/64: aux conv with F <= NB filters, rows of 2*NB bytes with the matching TMA swizzle).
-// S2 = 1: stride-2 convolution.  The shifted activation tiles are gathered by TMA with element stride 2,
+// S2 = 1: per-tap mode (stride-2 convolutions, and feature maps smaller than a tile where a tile spans BI
+// whole images).  The shifted activation tiles are gathered by TMA, with element stride 2 for stride 2,
 // one 128-pixel tile per tap; a CTA then owns one kernel row kh (grid dimension) with its three column
 // taps: taps (kh,0) and (kh,1) stacked in one instruction, tap (kh,2) in a second, half-empty one.
 template <int NB, int S2>
@@ -651,13 +662,13 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       const uint32_t ph = (it / kStages) & 1;
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) break;
       if (lane == 0) {
-        const int w0 = (t % p.tiles_w) * p.BW, h0 = ((t / p.tiles_w) % p.tiles_h) * p.BH, n = t / (p.tiles_w * p.tiles_h);
+        const int w0 = (t % p.tiles_w) * p.BW, h0 = ((t / p.tiles_w) % p.tiles_h) * p.BH, n = (t / (p.tiles_w * p.tiles_h)) * p.BI;
         uint8_t* st = smem + (size_t)s * stage_bytes;
         ptx::mbar_expect_tx(&full[s], (uint32_t)(3 * copy_bytes + kBTile));
 #pragma unroll
         for (int kw = 0; kw < 3; ++kw) {
           if constexpr (S2)
-            ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, 2 * w0 + kw - 1, 2 * h0 + khg - 1, n);
+            ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, p.stride * w0 + kw - 1, p.stride * h0 + khg - 1, n);
           else
             ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, w0 + kw - 1, h0 - 1, n);
         }
@@ -954,25 +965,36 @@ int sm_count() {
 // mode 0: main forward (y + statistics), 1: aux forward (bias + ReLU, Cout = F), 2: aux input gradient
 // (Cin = F <= 64 and a multiple of 8, Cout a multiple of 64, mirrored MN-major weights).
 // H, W: OUTPUT size (equal to the input size for stride 1).
+// Pixel tile of 128 output pixels: a BW x BH patch of one image, or (per-tap mode only) BI whole images
+// of a small feature map.  Returns false when the size does not tile.
+bool pick_tile(int H, int W, bool allow_multi, int* BW, int* BH, int* BI) {
+  const int cand[3][2] = {{16, 8}, {32, 4}, {8, 16}};
+  for (auto& c : cand)
+    if (W % c[0] == 0 && H % c[1] == 0) {
+      *BW = c[0]; *BH = c[1]; *BI = 1;
+      return true;
+    }
+  if (allow_multi && W * H <= 64 && W >= 2 && 128 % (W * H) == 0 && (W & (W - 1)) == 0) {  // 8x8, 4x4, 2x2, 8x4 ...
+    *BW = W; *BH = H; *BI = 128 / (W * H);
+    return true;
+  }
+  return false;
+}
+
 TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride = 1) {
   TcPlan pl{};
   if (stride == 2 && (epi != 0 || Cin % 64)) return pl;
   if (epi == 2 ? (Cin > 64 || Cin % 8 || Cout % 64) : (Cin % 64 != 0)) return pl;
   if (epi == 0 ? (Cout % 64 != 0) : epi == 1 ? (Cout > 64) : false) return pl;
-  const int cand[3][2] = {{16, 8}, {32, 4}, {8, 16}};
-  for (auto& c : cand)
-    if (W % c[0] == 0 && H % c[1] == 0) {
-      pl.BW = c[0];
-      pl.BH = c[1];
-      break;
-    }
-  if (!pl.BW) return pl;
+  if (!pick_tile(H, W, true, &pl.BW, &pl.BH, &pl.BI)) return pl;
+  pl.PT = (stride == 2 || pl.BI > 1) ? 1 : 0;
   pl.BN = epi != 1 ? (Cout % 128 == 0 ? 128 : 64) : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64);
   pl.KC = epi == 2 ? (Cin <= 16 ? 16 : Cin <= 32 ? 32 : 64) : 64;
-  const size_t a_stride = ((size_t)(stride == 2 ? pl.BH : pl.BH + 2) * pl.BW * pl.KC * 2 + 1023) & ~(size_t)1023;
-  pl.RW = (stride == 1 && epi != 2 && Cin == 64 && pl.BN <= 64) ? 1 : 0;  // weights resident in shared memory
-  const size_t stage = a_stride + (pl.RW ? 0 : stride == 2 ? (size_t)pl.BN * 128
-                                               : epi == 2 ? (size_t)(pl.BN / 64) * 3 * pl.KC * 128 : (size_t)3 * pl.BN * 128);
+  const size_t a_stride = pl.PT ? (size_t)128 * pl.KC * 2 : ((size_t)(pl.BH + 2) * pl.BW * pl.KC * 2 + 1023) & ~(size_t)1023;
+  pl.RW = (!pl.PT && epi != 2 && Cin == 64 && pl.BN <= 64) ? 1 : 0;  // weights resident in shared memory
+  const size_t b_stage = pl.RW ? 0 : pl.PT ? (epi == 2 ? (size_t)(pl.BN / 64) * pl.KC * 128 : (size_t)pl.BN * 128)
+                                           : epi == 2 ? (size_t)(pl.BN / 64) * 3 * pl.KC * 128 : (size_t)3 * pl.BN * 128;
+  const size_t stage = ((a_stride + 1023) & ~(size_t)1023) + b_stage;
   const size_t fixed = (size_t)(epi != 1 ? pl.BN / 64 : 0) * 16384 + (pl.RW ? (size_t)9 * pl.BN * 128 : 0) + 1024 + 1024;
   int st = (int)((232448 - fixed) / stage);
   if (st > kMaxStages) st = kMaxStages;
@@ -981,7 +1003,7 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride 
   pl.smem = (size_t)st * stage + fixed;
   pl.parts = pl.BN >= 128 ? 1 : 128 / pl.BN;
   const int n_tiles = epi != 1 ? Cout / pl.BN : 1;
-  const long total = (long)N * (H / pl.BH) * (W / pl.BW) * n_tiles;
+  const long total = (long)((N + pl.BI - 1) / pl.BI) * (H / pl.BH) * (W / pl.BW) * n_tiles;
   long g = sm_count();
   g -= g % n_tiles;  // every CTA keeps one channel tile for its whole life
   if (g < n_tiles) g = n_tiles;
@@ -1087,13 +1109,13 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
   if (!pl.ok) return NF_EUNSUPPORTED;
   CUtensorMap mx, mw, my;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)Win, (uint64_t)Hin, (uint64_t)N};
-  const uint32_t bx[4] = {(uint32_t)pl.KC, (uint32_t)pl.BW, (uint32_t)(stride == 2 ? pl.BH : pl.BH + 2), 1};
+  const uint32_t bx[4] = {(uint32_t)pl.KC, (uint32_t)pl.BW, (uint32_t)(pl.PT ? pl.BH : pl.BH + 2), (uint32_t)pl.BI};
   // forward: weights [kh][kw][Cout][Cin] -> box of BN rows x 64 ci for three kh; input gradient: weights
   // [kh][kw][F][Cout] -> box of KC rows of f x 64 c for three kh
   const uint64_t dw[4] = {(uint64_t)(epi == 2 ? Cout : Cin), (uint64_t)(epi == 2 ? Cin : Cout), 3, 3};
-  const uint32_t bw[4] = {64, (uint32_t)(epi == 2 ? pl.KC : pl.BN), 1, (uint32_t)(stride == 2 ? 1 : 3)};
+  const uint32_t bw[4] = {64, (uint32_t)(epi == 2 ? pl.KC : pl.BN), 1, (uint32_t)(pl.PT ? 1 : 3)};
   const uint64_t dy[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t by[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH, 1};
+  const uint32_t by[4] = {64, (uint32_t)pl.BW, (uint32_t)pl.BH, (uint32_t)pl.BI};
   int rc;
   if ((rc = make_map4(&mx, x, dx, bx, stride)) != NF_OK) return rc;
   if ((rc = make_map4(&mw, w, dw, bw)) != NF_OK) return rc;
@@ -1106,7 +1128,8 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
   p.N = N; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout;
   p.BW = pl.BW; p.BH = pl.BH; p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.n_tiles = epi != 1 ? Cout / pl.BN : 1;
   p.bias = bias; p.out = (bf16*)y;
-  p.total_tiles = N * p.tiles_h * p.tiles_w * p.n_tiles;
+  p.total_tiles = ((N + pl.BI - 1) / pl.BI) * p.tiles_h * p.tiles_w * p.n_tiles;
+  p.stride = stride; p.BI = pl.BI;
   p.kchunks = epi == 2 ? 1 : Cin / 64; p.stages = pl.stages; p.stats = stats; p.red = red; p.status = status;
   if (stats) {
     const size_t need = (size_t)pl.grid * pl.parts * 2 * Cout;
@@ -1114,8 +1137,17 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
     NF_CUDA(cudaMemsetAsync(red, 0, need * sizeof(float), g_nf_stream));
     *nb = pl.grid * pl.parts;
   }
-  if (epi == 0 && stride == 2)
-    return pl.BN == 128 ? launch_fwd<128, 0, 64, 0, 1>(pl, mx, mw, my, p) : launch_fwd<64, 0, 64, 0, 1>(pl, mx, mw, my, p);
+  if (pl.PT) {  // per-tap boxes: stride 2, or several small images per tile
+    if (epi == 0) return pl.BN == 128 ? launch_fwd<128, 0, 64, 0, 1>(pl, mx, mw, my, p) : launch_fwd<64, 0, 64, 0, 1>(pl, mx, mw, my, p);
+    if (epi == 1)
+      return pl.BN == 16 ? launch_fwd<16, 1, 64, 0, 1>(pl, mx, mw, my, p)
+                         : pl.BN == 32 ? launch_fwd<32, 1, 64, 0, 1>(pl, mx, mw, my, p) : launch_fwd<64, 1, 64, 0, 1>(pl, mx, mw, my, p);
+    if (pl.BN == 128)
+      return pl.KC == 16 ? launch_fwd<128, 0, 16, 1, 1>(pl, mx, mw, my, p)
+                         : pl.KC == 32 ? launch_fwd<128, 0, 32, 1, 1>(pl, mx, mw, my, p) : launch_fwd<128, 0, 64, 1, 1>(pl, mx, mw, my, p);
+    return pl.KC == 16 ? launch_fwd<64, 0, 16, 1, 1>(pl, mx, mw, my, p)
+                       : pl.KC == 32 ? launch_fwd<64, 0, 32, 1, 1>(pl, mx, mw, my, p) : launch_fwd<64, 0, 64, 1, 1>(pl, mx, mw, my, p);
+  }
   if (epi == 0 && pl.RW) return launch_fwd<64, 0, 64, 0, 0, 1>(pl, mx, mw, my, p);
   if (epi == 0) return pl.BN == 128 ? launch_fwd<128, 0>(pl, mx, mw, my, p) : launch_fwd<64, 0>(pl, mx, mw, my, p);
   if (epi == 1 && pl.RW)
@@ -1133,7 +1165,7 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
 }
 
 struct WgPlan {
-  int ok, BW, BH, NB, splits, grid, stages;
+  int ok, BW, BH, BI, PT, NB, splits, grid, stages;
   size_t smem, part_floats;
 };
 
@@ -1143,26 +1175,20 @@ WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0, int strid
   WgPlan pl{};
   if (Cin % 64 || (stride == 2 && aux)) return pl;
   if (aux ? (Cout > 64 || Cout % 8) : (Cout % 64 != 0)) return pl;
-  const int cand[3][2] = {{16, 8}, {32, 4}, {8, 16}};
-  for (auto& c : cand)
-    if (W % c[0] == 0 && H % c[1] == 0) {
-      pl.BW = c[0];
-      pl.BH = c[1];
-      break;
-    }
-  if (!pl.BW) return pl;
+  if (!pick_tile(H, W, true, &pl.BW, &pl.BH, &pl.BI)) return pl;
+  pl.PT = (stride == 2 || pl.BI > 1) ? 1 : 0;
   pl.NB = aux ? (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64) : 64;
   size_t g_region = (size_t)3 * 128 * pl.NB * 2;
   if (g_region < 4096) g_region = 4096;
-  const size_t stage = stride == 2 ? 65536 : (size_t)(pl.BH + 2) * pl.BW * 128 + g_region;
-  pl.stages = stride == 2 ? 3 : (int)((232448 - 2048) / stage);
+  const size_t stage = pl.PT ? 65536 : (size_t)(pl.BH + 2) * pl.BW * 128 + g_region;
+  pl.stages = pl.PT ? 3 : (int)((232448 - 2048) / stage);
   if (pl.stages > kMaxStages) pl.stages = kMaxStages;
   if (pl.stages < 2) return pl;
   pl.smem = (size_t)pl.stages * stage + 1024 + 1024;
   if (pl.smem > 232448) return pl;
   const int blocks = (Cin / 64) * (aux ? 1 : Cout / 64);
-  const long pix_tiles = (long)N * (H / pl.BH) * (W / pl.BW);
-  const int groups = stride == 2 ? 3 : 1;  // kernel rows handled by separate CTAs
+  const long pix_tiles = (long)((N + pl.BI - 1) / pl.BI) * (H / pl.BH) * (W / pl.BW);
+  const int groups = pl.PT ? 3 : 1;  // kernel rows handled by separate CTAs
   long sp = sm_count() / (blocks * groups);
   if (sp < 1) sp = 1;
   if (sp > pix_tiles) sp = pix_tiles;
@@ -1206,19 +1232,20 @@ int run_wgrad(int N, int Hin, int Win, int Cin, int Cout, const void* x, const v
   if (pl.part_floats > part_floats) return NF_ENOWS;
   CUtensorMap mx, mg;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)Win, (uint64_t)Hin, (uint64_t)N};
-  const uint32_t bx[4] = {64, (uint32_t)pl.BW, (uint32_t)(stride == 2 ? pl.BH : pl.BH + 2), 1};
+  const uint32_t bx[4] = {64, (uint32_t)pl.BW, (uint32_t)(pl.PT ? pl.BH : pl.BH + 2), (uint32_t)pl.BI};
   const uint64_t dg[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t bg[4] = {(uint32_t)pl.NB, (uint32_t)pl.BW, (uint32_t)pl.BH, 1};
+  const uint32_t bg[4] = {(uint32_t)pl.NB, (uint32_t)pl.BW, (uint32_t)pl.BH, (uint32_t)pl.BI};
   int rc;
   if ((rc = make_map4(&mx, x, dx, bx, stride)) != NF_OK) return rc;
   if ((rc = make_map4(&mg, dy, dg, bg)) != NF_OK) return rc;
   WgParams p{};
   p.N = N; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout; p.BW = pl.BW; p.BH = pl.BH;
-  p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.pix_tiles = N * p.tiles_h * p.tiles_w;
+  p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.pix_tiles = ((N + pl.BI - 1) / pl.BI) * p.tiles_h * p.tiles_w;
+  p.stride = stride; p.BI = pl.BI;
   p.ci_chunks = Cin / 64; p.co_chunks = aux ? 1 : Cout / 64; p.splits = pl.splits; p.part = part; p.status = status;
   p.stages = pl.stages;
-  if (stride == 2)
-    rc = launch_wgrad<64, 1>(pl, mx, mg, p);
+  if (pl.PT)
+    rc = pl.NB == 64 ? launch_wgrad<64, 1>(pl, mx, mg, p) : pl.NB == 32 ? launch_wgrad<32, 1>(pl, mx, mg, p) : launch_wgrad<16, 1>(pl, mx, mg, p);
   else
     rc = pl.NB == 64 ? launch_wgrad_kw<64>(pl, mx, mg, p)
                      : pl.NB == 32 ? launch_wgrad_kw<32>(pl, mx, mg, p) : launch_wgrad_kw<16>(pl, mx, mg, p);

@@ -23,6 +23,11 @@ SHAPES = [  # N, Cin, Cout, H, W, stride
     (2, 64, 64, 16, 28, 1),     # 64->64 forward with the column taps folded into N: 14-pixel-wide tiles
     (1, 64, 64, 8, 14, 1),      # the same kernel on a single tile
     (3, 64, 64, 24, 56, 1),     # several tiles per CTA row and per image
+    (4, 64, 64, 8, 8, 1),       # small feature map: tiles of two whole 8x8 images, one TMA box per tap
+    (5, 64, 128, 8, 8, 1),      # the same with a ragged last tile (5 images, 2 per tile)
+    (16, 128, 128, 4, 4, 1),    # eight 4x4 images per tile, two channel chunks
+    (6, 128, 128, 16, 16, 2),   # stride 2 down to 8x8: strided boxes over two images
+    (3, 256, 64, 4, 4, 1),
     (2, 64, 64, 31, 33, 2),     # stride 2 with odd input sizes: 16x17 output is not tileable -> CUDA-core path
 ]
 

@@ -132,6 +132,9 @@ TC = [
     dict(N=3, Cin=64, Cout=128, H=16, W=112, F=8, classes=10, stride=1, pool=False),  # folded aux forward, two K chunks, F < 16
     dict(N=3, Cin=64, Cout=64, H=16, W=112, F=40, classes=10, stride=1, pool=False),  # folded aux forward, group width 64
     dict(N=3, Cin=64, Cout=64, H=16, W=112, F=32, classes=10, stride=1, pool=False),  # folded aux input gradient, 32-channel K
+    dict(N=9, Cin=128, Cout=128, H=8, W=8, F=16, classes=10, stride=1, pool=True),    # 8x8 maps: 2 images per tile (ragged), aux at 4x4
+    dict(N=16, Cin=64, Cout=64, H=4, W=4, F=8, classes=10, stride=1, pool=False),     # 4x4 maps: 8 images per tile
+    dict(N=12, Cin=64, Cout=128, H=16, W=16, F=32, classes=10, stride=2, pool=False), # stride 2 down to 8x8, multi-image tiles
 ]
 
 
