@@ -735,6 +735,139 @@ __global__ void avgpool_finish_kernel(const float* __restrict__ part, int N, int
   p[(size_t)n * 4 * F + f * 4 + bin] = s * inv_cnt;
 }
 
+
+// ------------------------------------------------------------------ vectorised bf16 paths for pooled layers
+// One thread owns 8 channels of one POOLED pixel: it reads the four conv outputs of the 2x2 window.
+__device__ __forceinline__ size_t win_base(size_t q, int Ho, int Wo, int C8) {  // q = pooled pixel index
+  const int Wa = Wo / 2, Ha = Ho / 2;
+  const int ja = (int)(q % Wa), ia = (int)((q / Wa) % Ha);
+  const size_t n = q / ((size_t)Wa * Ha);
+  return ((n * Ho + 2 * ia) * Wo + 2 * ja) * C8;
+}
+
+__global__ void __launch_bounds__(256) bn_apply_pool_vec_kernel(const uint4* __restrict__ y, int Ho, int Wo, int C8,
+                                                                const float* __restrict__ scale, const float* __restrict__ shift,
+                                                                size_t total8, uint4* __restrict__ out) {
+  const int c0 = (threadIdx.x % C8) * 8;
+  float A[8], B[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { A[i] = scale[c0 + i]; B[i] = shift[c0 + i]; }
+  for (size_t e = (size_t)blockIdx.x * 256 + threadIdx.x; e < total8; e += (size_t)gridDim.x * 256) {
+    const size_t b = win_base(e / C8, Ho, Wo, C8) + e % C8;
+    const uint4 v4[4] = {__ldg(y + b), __ldg(y + b + C8), __ldg(y + b + (size_t)Wo * C8), __ldg(y + b + (size_t)Wo * C8 + C8)};
+    float best[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) best[i] = 0.f;
+#pragma unroll
+    for (int d = 0; d < 4; ++d) {
+      float v[8];
+      unpack8(v4[d], v);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) best[i] = fmaxf(best[i], fmaf(v[i], A[i], B[i]));
+    }
+    out[e] = pack8(best);
+  }
+}
+
+// dz of the four window positions: the first maximum (scan order) of the bf16-rounded ReLU outputs takes da
+// if its pre-activation is positive.  arg[i] = winning position of channel i, or -1.
+__device__ __forceinline__ void pool_winner(const float (&yv)[4][8], const float (&A)[8], const float (&B)[8], int (&arg)[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float best = -1.f;
+    int a = 0;
+    float zbest = 0.f;
+#pragma unroll
+    for (int d = 0; d < 4; ++d) {
+      const float z = fmaf(yv[d][i], A[i], B[i]);
+      const float r = __bfloat162float(__float2bfloat16_rn(fmaxf(z, 0.f)));
+      if (r > best) { best = r; a = d; zbest = z; }
+    }
+    arg[i] = zbest > 0.f ? a : -1;
+  }
+}
+
+__global__ void __launch_bounds__(256) bn_bwd_reduce_pool_vec_kernel(const uint4* __restrict__ y, const uint4* __restrict__ da,
+                                                                     size_t Pq, int Ho, int Wo, int C8,
+                                                                     const float* __restrict__ scale, const float* __restrict__ shift,
+                                                                     const float* __restrict__ mu, const float* __restrict__ invstd,
+                                                                     float* __restrict__ red) {
+  __shared__ float sm[16][256];
+  const int C = C8 * 8;
+  const int planes = 256 / C8, g = threadIdx.x % C8, pl = threadIdx.x / C8;
+  const int c0 = g * 8;
+  float A[8], B[8], m[8], is[8], a[8], b[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    A[i] = scale[c0 + i]; B[i] = shift[c0 + i]; m[i] = mu[c0 + i]; is[i] = invstd[c0 + i];
+    a[i] = 0.f; b[i] = 0.f;
+  }
+  const size_t q0 = Pq * blockIdx.x / gridDim.x, q1 = Pq * (blockIdx.x + 1) / gridDim.x;
+  for (size_t q = q0 + pl; q < q1; q += planes) {
+    const size_t bb = win_base(q, Ho, Wo, C8) + g;
+    const uint4 v4[4] = {__ldg(y + bb), __ldg(y + bb + C8), __ldg(y + bb + (size_t)Wo * C8), __ldg(y + bb + (size_t)Wo * C8 + C8)};
+    float yv[4][8], dv[8];
+#pragma unroll
+    for (int d = 0; d < 4; ++d) unpack8(v4[d], yv[d]);
+    unpack8(__ldg(da + q * C8 + g), dv);
+    int arg[8];
+    pool_winner(yv, A, B, arg);
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (arg[i] >= 0) {
+        const float yy = arg[i] == 0 ? yv[0][i] : arg[i] == 1 ? yv[1][i] : arg[i] == 2 ? yv[2][i] : yv[3][i];
+        a[i] += dv[i];
+        b[i] = fmaf(dv[i], (yy - m[i]) * is[i], b[i]);
+      }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    sm[i][threadIdx.x] = a[i];
+    sm[8 + i][threadIdx.x] = b[i];
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < 2 * C; t += 256) {
+    const int k = t / C, c = t % C, gg = c / 8, i = c % 8;
+    float s = 0.f;
+    for (int qq = 0; qq < planes; ++qq) s += sm[k * 8 + i][qq * C8 + gg];
+    red[((size_t)blockIdx.x * 2 + k) * C + c] = s;
+  }
+}
+
+__global__ void __launch_bounds__(256) bn_bwd_apply_pool_vec_kernel(const uint4* __restrict__ y, const uint4* __restrict__ da, int Ho,
+                                                                    int Wo, int C8, const float* __restrict__ scale,
+                                                                    const float* __restrict__ shift, const float* __restrict__ mu,
+                                                                    const float* __restrict__ invstd, const float* __restrict__ sdz,
+                                                                    const float* __restrict__ sdzx, float invM, size_t total8,
+                                                                    uint4* __restrict__ dy) {
+  const int c0 = (threadIdx.x % C8) * 8;
+  float A[8], B[8], K1[8], K0[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float s = scale[c0 + i], m1 = sdz[c0 + i] * invM, m2 = sdzx[c0 + i] * invM, is = invstd[c0 + i];
+    A[i] = s; B[i] = shift[c0 + i];
+    K1[i] = -s * m2 * is;
+    K0[i] = s * (m2 * is * mu[c0 + i] - m1);
+  }
+  for (size_t e = (size_t)blockIdx.x * 256 + threadIdx.x; e < total8; e += (size_t)gridDim.x * 256) {  // e over pooled vectors
+    const size_t bb = win_base(e / C8, Ho, Wo, C8) + e % C8;
+    const size_t off[4] = {0, (size_t)C8, (size_t)Wo * C8, (size_t)Wo * C8 + C8};
+    float yv[4][8], dv[8];
+#pragma unroll
+    for (int d = 0; d < 4; ++d) unpack8(__ldg(y + bb + off[d]), yv[d]);
+    unpack8(__ldg(da + e), dv);
+    int arg[8];
+    pool_winner(yv, A, B, arg);
+#pragma unroll
+    for (int d = 0; d < 4; ++d) {
+      float o[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) o[i] = fmaf(A[i], arg[i] == d ? dv[i] : 0.f, fmaf(K1[i], yv[d][i], K0[i]));
+      dy[bb + off[d]] = pack8(o);
+    }
+  }
+}
+
 inline bool vec_ok(int dtype, int C, int pool) { return dtype == NF_BF16 && C % 8 == 0 && C <= 1024 && !pool; }
 inline int vec_blocks(size_t work_items) {
   size_t b = (work_items + 256 * 8 - 1) / (256 * 8);
@@ -796,6 +929,12 @@ int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float ep
 int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
                     const float* shift, void* out) {
   const size_t total = (size_t)N * (pool ? Ho / 2 : Ho) * (pool ? Wo / 2 : Wo) * C;
+  if (pool && vec_ok(dtype, C, 0) && 256 % (C / 8) == 0) {
+    bn_apply_pool_vec_kernel<<<vec_blocks(total / 8), 256, 0, g_nf_stream>>>((const uint4*)y, Ho, Wo, C / 8, scale, shift, total / 8,
+                                                                            (uint4*)out);
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   if (vec_ok(dtype, C, pool) && 256 % (C / 8) == 0) {
     bn_apply_vec2_kernel<<<vec_blocks(total / 8), 256, 0, g_nf_stream>>>((const uint4*)y, C / 8, scale, shift, total / 8, (uint4*)out);
     NF_LAUNCHED();
@@ -889,6 +1028,13 @@ int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho
   const size_t P = (size_t)N * Ho * Wo;
   const int nb = nf_ref_channel_blocks(P, C);
   if ((size_t)nb * 2 * C > red_floats) return NF_ENOWS;
+  if (pool && vec_ok(dtype, C, 0) && 256 % (C / 8) == 0) {
+    bn_bwd_reduce_pool_vec_kernel<<<nb, 256, 0, g_nf_stream>>>((const uint4*)y, (const uint4*)da, P / 4, Ho, Wo, C / 8, scale, shift, mu,
+                                                              invstd, red);
+    NF_LAUNCHED();
+    *nblocks = nb;
+    return NF_OK;
+  }
   if (vec_ok(dtype, C, pool) && 256 % (C / 8) == 0) {
     bn_bwd_reduce_vec_kernel<<<nb, 256, 0, g_nf_stream>>>((const uint4*)y, (const uint4*)da, P, C / 8, scale, shift, mu, invstd, red);
     NF_LAUNCHED();
@@ -916,6 +1062,12 @@ int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho,
                         const float* sdz, const float* sdzx, double M, void* dy) {
   const size_t total = (size_t)N * Ho * Wo * C;
   const float invM = (float)(1.0 / M);
+  if (pool && vec_ok(dtype, C, 0) && 256 % (C / 8) == 0) {
+    bn_bwd_apply_pool_vec_kernel<<<vec_blocks(total / 32), 256, 0, g_nf_stream>>>((const uint4*)y, (const uint4*)da, Ho, Wo, C / 8, scale,
+                                                                                 shift, mu, invstd, sdz, sdzx, invM, total / 32, (uint4*)dy);
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   if (vec_ok(dtype, C, pool) && 256 % (C / 8) == 0) {
     bn_bwd_apply_vec2_kernel<<<vec_blocks(total / 8), 256, 0, g_nf_stream>>>((const uint4*)y, (const uint4*)da, C / 8, scale, shift, mu,
                                                                             invstd, sdz, sdzx, invM, total / 8, (uint4*)dy);
