@@ -153,16 +153,53 @@ void derive(nf_layer* L) {
 
 bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
 
-// logical [A][B][3][3]  <->  kernel [tap][A][B]
-void to_kernel_layout(const float* src, float* dst, size_t A, size_t B) {
+// logical [A][B][3][3]  <->  kernel [tap][Ap][B] (rows A..Ap-1 are padding, kept zero)
+void to_kernel_layout(const float* src, float* dst, size_t A, size_t Ap, size_t B) {
   for (size_t a = 0; a < A; ++a)
     for (size_t b = 0; b < B; ++b)
-      for (int t = 0; t < 9; ++t) dst[(t * A + a) * B + b] = src[(a * B + b) * 9 + t];
+      for (int t = 0; t < 9; ++t) dst[(t * Ap + a) * B + b] = src[(a * B + b) * 9 + t];
 }
-void from_kernel_layout(const float* src, float* dst, size_t A, size_t B) {
+void from_kernel_layout(const float* src, float* dst, size_t A, size_t Ap, size_t B) {
   for (size_t a = 0; a < A; ++a)
     for (size_t b = 0; b < B; ++b)
-      for (int t = 0; t < 9; ++t) dst[(a * B + b) * 9 + t] = src[(t * A + a) * B + b];
+      for (int t = 0; t < 9; ++t) dst[(a * B + b) * 9 + t] = src[(t * Ap + a) * B + b];
+}
+
+// Converts one parameter tensor between the caller's logical form (n_log floats) and the padded kernel
+// form (cnt floats, zero in the padding).  dir 0: logical -> kernel, 1: kernel -> logical.
+void convert_param(const nf_layer* L, int id, const float* src, float* dst, int dir) {
+  const size_t F = L->Flog, Fp = L->F, Co = L->Cout, K = L->classes;
+  switch (id) {
+    case NF_P_W:
+      if (dir == 0) to_kernel_layout(src, dst, Co, Co, L->Cin); else from_kernel_layout(src, dst, Co, Co, L->Cin);
+      break;
+    case NF_P_WA:
+      if (dir == 0) to_kernel_layout(src, dst, F, Fp, Co); else from_kernel_layout(src, dst, F, Fp, Co);
+      break;
+    case NF_P_BA:
+      memcpy(dst, src, F * sizeof(float));
+      break;
+    case NF_P_WF:
+      for (size_t k = 0; k < K; ++k)
+        if (dir == 0) memcpy(dst + k * 4 * Fp, src + k * 4 * F, 4 * F * sizeof(float));
+        else memcpy(dst + k * 4 * F, src + k * 4 * Fp, 4 * F * sizeof(float));
+      break;
+    default: {
+      const size_t n = id == NF_P_BF ? K : Co;
+      memcpy(dst, src, n * sizeof(float));
+    }
+  }
+}
+
+size_t logical_count(const nf_layer* L, int id) {
+  switch (id) {
+    case NF_P_W: return (size_t)9 * L->Cout * L->Cin;
+    case NF_P_WA: return (size_t)9 * L->Flog * L->Cout;
+    case NF_P_BA: return L->Flog;
+    case NF_P_WF: return (size_t)L->classes * 4 * L->Flog;
+    case NF_P_BF: return L->classes;
+    default: return L->Cout;
+  }
 }
 
 }  // namespace
@@ -173,7 +210,7 @@ nf_layer* nf_layer_create(int Cin, int Cout, int H, int W, int F, int classes) {
   if (Cin < 1 || Cout < 1 || H < 1 || W < 1 || F < 1 || classes < 1) return nullptr;
   nf_layer* L = (nf_layer*)calloc(1, sizeof(nf_layer));
   if (!L) return nullptr;
-  L->Cin = Cin; L->Cout = Cout; L->H = H; L->W = W; L->F = F; L->classes = classes;
+  L->Cin = Cin; L->Cout = Cout; L->H = H; L->W = W; L->Flog = F; L->F = (F + 7) / 8 * 8; L->classes = classes;
   L->o.N = 1; L->o.stride = 1; L->o.maxpool = 0; L->o.dtype = NF_BF16;
   L->o.momentum = 0.9f; L->o.bn_eps = 1e-5f; L->o.bn_momentum = 0.1f; L->o.host_io = 0;
   derive(L);
@@ -244,17 +281,13 @@ int nf_layer_set_param(nf_layer* L, int which, const float* host, size_t n) {
   float* dev; size_t cnt; int A, B;
   int rc = param_ptr(L, which, &dev, &cnt, &A, &B);
   if (rc != NF_OK) return rc;
-  if (n != cnt) return NF_EINVAL;
-  std::vector<float> tmp;
-  const float* src = host;
-  if (A) {
-    tmp.resize(cnt);
-    to_kernel_layout(host, tmp.data(), A, B);
-    src = tmp.data();
-  }
-  NF_CUDA(cudaMemcpyAsync(dev, src, cnt * 4, cudaMemcpyHostToDevice, g_nf_stream));
+  const int id = which & 0xff;
+  if (n != logical_count(L, id)) return NF_EINVAL;
+  std::vector<float> tmp(cnt, 0.f);
+  convert_param(L, id, host, tmp.data(), 0);
+  NF_CUDA(cudaMemcpyAsync(dev, tmp.data(), cnt * 4, cudaMemcpyHostToDevice, g_nf_stream));
   NF_CUDA(cudaStreamSynchronize(g_nf_stream));
-  if ((which & 0xf00) == NF_K_VALUE && (which & 0xff) < NF_NPARAM) {
+  if ((which & 0xf00) == NF_K_VALUE && id < NF_NPARAM) {
     rc = nf_ref_shadow(L->val, L->shadow, L->arena);
     if (rc != NF_OK) return rc;
     NF_CUDA(cudaStreamSynchronize(g_nf_stream));
@@ -268,15 +301,12 @@ int nf_layer_get_param(nf_layer* L, int which, float* host, size_t n) {
   float* dev; size_t cnt; int A, B;
   int rc = param_ptr(L, which, &dev, &cnt, &A, &B);
   if (rc != NF_OK) return rc;
-  if (n != cnt) return NF_EINVAL;
+  const int id = which & 0xff;
+  if (n != logical_count(L, id)) return NF_EINVAL;
   NF_CUDA(cudaStreamSynchronize(g_nf_stream));
-  if (A) {
-    std::vector<float> tmp(cnt);
-    NF_CUDA(cudaMemcpy(tmp.data(), dev, cnt * 4, cudaMemcpyDeviceToHost));
-    from_kernel_layout(tmp.data(), host, A, B);
-  } else {
-    NF_CUDA(cudaMemcpy(host, dev, cnt * 4, cudaMemcpyDeviceToHost));
-  }
+  std::vector<float> tmp(cnt);
+  NF_CUDA(cudaMemcpy(tmp.data(), dev, cnt * 4, cudaMemcpyDeviceToHost));
+  convert_param(L, id, tmp.data(), host, 1);
   return NF_OK;
 }
 

@@ -19,7 +19,9 @@ enum { NF_NPARAM = 7 };
 
 struct nf_layer {
   // description
-  int Cin, Cout, H, W, F, classes;
+  int Cin, Cout, H, W, F, classes;  // F = aux filters as the kernels see them: the caller's count rounded up to a
+                                    // multiple of 8; the extra filters have zero weights, get zero gradients, stay zero
+  int Flog;                         // the caller's aux filter count
   nf_layer_opts o;
   int Ho, Wo, Ha, Wa;  // conv output size; size after the optional pool
   // arena
