@@ -133,6 +133,22 @@ __global__ void sum_splits_kernel(const float* __restrict__ part, int splits, si
 // An RGB input gives a K dimension of only 27: too thin for the tensor cores and, with 6-byte pixels,
 // not addressable by TMA.  One thread computes 16 output channels of one pixel from its 3x3xCin patch held
 // in registers; weights sit in shared memory and are read as warp-wide broadcasts.
+template <typename T> __device__ __forceinline__ void store16(T* dst, const float (&v)[16]);
+template <> __device__ __forceinline__ void store16<float>(float* dst, const float (&v)[16]) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) reinterpret_cast<float4*>(dst)[k] = make_float4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+}
+template <> __device__ __forceinline__ void store16<bf16>(bf16* dst, const float (&v)[16]) {
+  uint32_t w[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+    w[k] = *reinterpret_cast<const uint32_t*>(&b2);
+  }
+  reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+  reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) conv_smallc_kernel(const T* __restrict__ x, int N, int H, int W, int Ci,
                                                           const T* __restrict__ w, int s, int Co, int Ho, int Wo,
@@ -144,34 +160,39 @@ __global__ void __launch_bounds__(256) conv_smallc_kernel(const T* __restrict__ 
   }
   __syncthreads();
   const size_t P = (size_t)N * Ho * Wo;
-  const size_t pix = (size_t)blockIdx.x * 32 + threadIdx.x;
-  if (pix >= P) return;
-  const int j = (int)(pix % Wo), i = (int)((pix / Wo) % Ho);
-  const size_t n = pix / ((size_t)Wo * Ho);
-  float patch[36];
-#pragma unroll
-  for (int t = 0; t < 9; ++t) {
-    const int ii = i * s + t / 3 - 1, jj = j * s + t % 3 - 1;
-    const bool in = ii >= 0 && ii < H && jj >= 0 && jj < W;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) patch[t * 4 + c] = (in && c < Ci) ? ldf(x, ((n * H + ii) * W + jj) * Ci + c) : 0.f;
-  }
   const int co0 = threadIdx.y * 16;
-  float acc[16];
+  for (size_t pix = (size_t)blockIdx.x * 32 + threadIdx.x; pix < P; pix += (size_t)gridDim.x * 32) {  // weights loaded once per block
+    const int j = (int)(pix % Wo), i = (int)((pix / Wo) % Ho);
+    const size_t n = pix / ((size_t)Wo * Ho);
+    float patch[36];
 #pragma unroll
-  for (int k = 0; k < 16; ++k) acc[k] = 0.f;
+    for (int t = 0; t < 9; ++t) {
+      const int ii = i * s + t / 3 - 1, jj = j * s + t % 3 - 1;
+      const bool in = ii >= 0 && ii < H && jj >= 0 && jj < W;
 #pragma unroll
-  for (int t = 0; t < 9; ++t)
+      for (int c = 0; c < 4; ++c) patch[t * 4 + c] = (in && c < Ci) ? ldf(x, ((n * H + ii) * W + jj) * Ci + c) : 0.f;
+    }
+    float acc[16];
 #pragma unroll
-    for (int c = 0; c < 4; ++c)
-      if (c < Ci) {
-        const float xv = patch[t * 4 + c];
-        const float* wr = wsm + (t * Ci + c) * Co + co0;
+    for (int k = 0; k < 16; ++k) acc[k] = 0.f;
 #pragma unroll
-        for (int k = 0; k < 16; ++k) acc[k] = fmaf(xv, wr[k], acc[k]);
-      }
+    for (int t = 0; t < 9; ++t)
 #pragma unroll
-  for (int k = 0; k < 16; ++k) stf(y, pix * Co + co0 + k, acc[k]);
+      for (int c = 0; c < 4; ++c)
+        if (c < Ci) {
+          const float xv = patch[t * 4 + c];
+          const float4* wr = reinterpret_cast<const float4*>(wsm + (t * Ci + c) * Co + co0);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float4 wv = wr[k];
+            acc[4 * k] = fmaf(xv, wv.x, acc[4 * k]);
+            acc[4 * k + 1] = fmaf(xv, wv.y, acc[4 * k + 1]);
+            acc[4 * k + 2] = fmaf(xv, wv.z, acc[4 * k + 2]);
+            acc[4 * k + 3] = fmaf(xv, wv.w, acc[4 * k + 3]);
+          }
+        }
+    store16(y + pix * Co + co0, acc);
+  }
 }
 
 // part[split][tap][co][ci]: thread (co, lane) sums its 9*Ci products over the pixels lane, lane+4, ... of the
@@ -180,35 +201,43 @@ template <typename T>
 __global__ void __launch_bounds__(512) wgrad_smallc_kernel(const T* __restrict__ x, int N, int H, int W, int Ci,
                                                            const T* __restrict__ g, int Co, int s, int Ho, int Wo,
                                                            int splits, float* __restrict__ part) {
-  extern __shared__ float sm[];           // xrow[3][W + 2][4]  then  red[4][Co][36]
+  extern __shared__ float sm[];           // xrow[(R-1)*s + 3][W + 2][4]  then  red[4][Co][36]
+  constexpr int R = 4;                    // output rows staged per synchronisation
+  const int xr = (R - 1) * s + 3;
   float* xrow = sm;
-  float* red = sm + 3 * (W + 2) * 4;
+  float* red = sm + xr * (W + 2) * 4;
   const int co = threadIdx.x, ln = threadIdx.y, tid = ln * blockDim.x + co, nthr = blockDim.x * 4;
   const long rows = (long)N * Ho;
   const long r0 = rows * blockIdx.x / splits, r1 = rows * (blockIdx.x + 1) / splits;
   float acc[36];
 #pragma unroll
   for (int k = 0; k < 36; ++k) acc[k] = 0.f;
-  for (long r = r0; r < r1; ++r) {
+  for (long r = r0; r < r1;) {
     const int n = (int)(r / Ho), i = (int)(r % Ho);
+    int nr = R;
+    if (nr > r1 - r) nr = (int)(r1 - r);
+    if (nr > Ho - i) nr = Ho - i;          // stay inside one image
+    const int need = (nr - 1) * s + 3;
     __syncthreads();
-    for (int e = tid; e < 3 * (W + 2) * 4; e += nthr) {
+    for (int e = tid; e < need * (W + 2) * 4; e += nthr) {
       const int c = e & 3, col = (e >> 2) % (W + 2), rr = (e >> 2) / (W + 2);
       const int ii = i * s + rr - 1, jj = col - 1;
       xrow[e] = (c < Ci && ii >= 0 && ii < H && jj >= 0 && jj < W) ? ldf(x, (((size_t)n * H + ii) * W + jj) * Ci + c) : 0.f;
     }
     __syncthreads();
-    for (int j = ln; j < Wo; j += 4) {
-      const float gv = ldf(g, (((size_t)n * Ho + i) * Wo + j) * Co + co);
+    for (int q = 0; q < nr; ++q)
+      for (int j = ln; j < Wo; j += 4) {
+        const float gv = ldf(g, (((size_t)n * Ho + i + q) * Wo + j) * Co + co);
 #pragma unroll
-      for (int t = 0; t < 9; ++t) {
-        const float4 xv = *reinterpret_cast<const float4*>(xrow + ((t / 3) * (W + 2) + j * s + t % 3) * 4);
-        acc[t * 4 + 0] = fmaf(gv, xv.x, acc[t * 4 + 0]);
-        acc[t * 4 + 1] = fmaf(gv, xv.y, acc[t * 4 + 1]);
-        acc[t * 4 + 2] = fmaf(gv, xv.z, acc[t * 4 + 2]);
-        acc[t * 4 + 3] = fmaf(gv, xv.w, acc[t * 4 + 3]);
+        for (int t = 0; t < 9; ++t) {
+          const float4 xv = *reinterpret_cast<const float4*>(xrow + ((q * s + t / 3) * (W + 2) + j * s + t % 3) * 4);
+          acc[t * 4 + 0] = fmaf(gv, xv.x, acc[t * 4 + 0]);
+          acc[t * 4 + 1] = fmaf(gv, xv.y, acc[t * 4 + 1]);
+          acc[t * 4 + 2] = fmaf(gv, xv.z, acc[t * 4 + 2]);
+          acc[t * 4 + 3] = fmaf(gv, xv.w, acc[t * 4 + 3]);
+        }
       }
-    }
+    r += nr;
   }
   __syncthreads();
 #pragma unroll
@@ -234,11 +263,14 @@ int nf_ref_conv(int dtype, const void* x, int N, int H, int W, int Ci, const voi
     const size_t P = (size_t)N * Ho * Wo;
     const dim3 blk(32, Co / 16);
     const size_t sm = (size_t)9 * Ci * Co * sizeof(float);
+    size_t nblk_ = (P + 31) / 32;
+    if (nblk_ > 148 * 16) nblk_ = 148 * 16;
+    const unsigned grid = (unsigned)nblk_;
     if (dtype == NF_F32)
-      conv_smallc_kernel<float><<<(unsigned)((P + 31) / 32), blk, sm, g_nf_stream>>>((const float*)x, N, H, W, Ci, (const float*)w,
+      conv_smallc_kernel<float><<<grid, blk, sm, g_nf_stream>>>((const float*)x, N, H, W, Ci, (const float*)w,
                                                                                    stride, Co, Ho, Wo, (float*)y);
     else
-      conv_smallc_kernel<bf16><<<(unsigned)((P + 31) / 32), blk, sm, g_nf_stream>>>((const bf16*)x, N, H, W, Ci, (const bf16*)w,
+      conv_smallc_kernel<bf16><<<grid, blk, sm, g_nf_stream>>>((const bf16*)x, N, H, W, Ci, (const bf16*)w,
                                                                                   stride, Co, Ho, Wo, (bf16*)y);
     NF_LAUNCHED();
     return NF_OK;
@@ -275,11 +307,11 @@ int nf_ref_wgrad(int dtype, const void* x, int N, int H, int W, int Ci, const vo
   if ((size_t)splits * n > part_floats) return NF_ENOWS;
   if (smallc_ok(Ci, Co, W)) {
     const dim3 blk(Co, 4);
-    const size_t sm = ((size_t)3 * (W + 2) * 4 + (size_t)4 * Co * 36) * sizeof(float);  // <= 24.7 KB + 73.7 KB
+    const size_t sm = ((size_t)(3 * stride + 3) * (W + 2) * 4 + (size_t)4 * Co * 36) * sizeof(float);
     static bool attr_done = false;
     if (!attr_done) {
-      NF_CUDA(cudaFuncSetAttribute(wgrad_smallc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
-      NF_CUDA(cudaFuncSetAttribute(wgrad_smallc_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+      NF_CUDA(cudaFuncSetAttribute(wgrad_smallc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+      NF_CUDA(cudaFuncSetAttribute(wgrad_smallc_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
       attr_done = true;
     }
     if (dtype == NF_F32)
