@@ -27,6 +27,14 @@ METRIC = "local-layer train-step images/s (bf16)"
 FALLBACK_PEAKS = dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0)
 
 
+# DRAM bytes per image (read + write) of the kernels behind each traced op on the c4 layers 64->64 at 224x224,
+# from one ncu capture of the batch-24 case (profiles/ncu_full_c4s_conv_bn_kernels.md); every tensor is streamed
+# once, so traffic grows in proportion to the batch.  Valid for the kernels as captured; None elsewhere.
+NCU_TRAFFIC_C4_BYTES_PER_IMAGE = dict(conv_fwd=(154.27 + 106.01) * 1e6 / 24, wgrad=(324.01 + 3.51) * 1e6 / 24,
+                                      bn_bwd=(308.30 + 3.82 + 308.34 + 123.60) * 1e6 / 24,
+                                      bn_fwd=(154.15 + 109.90) * 1e6 / 24)
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -219,8 +227,11 @@ def run_ours(args, rank, world):
         kernels.append(rec)
         if best is None:
             best = rec
+    traffic = None
+    if wl["name"] in ("c4", "c4s") and best["layer"] in (0, 1) and best["op"] in NCU_TRAFFIC_C4_BYTES_PER_IMAGE:
+        traffic = round(NCU_TRAFFIC_C4_BYTES_PER_IMAGE[best["op"]] * N)
     roof = dict(bound=best["bound"], achieved=best["achieved"], peak=best["peak"], unit=best["unit"],
-                frac=best["frac"], traffic=None, kernel=f'{best["op"]}[layer {best["layer"]}]',
+                frac=best["frac"], traffic=traffic, kernel=f'{best["op"]}[layer {best["layer"]}]',
                 peak_source=f"{peak_src} (sustained bf16 figure: kernel timed inside a long step)"
                 if best["bound"] != "hbm" else peak_src)
 

@@ -580,17 +580,12 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 }
 
 // ---------------------------------------------------------------- weight gradient
-// dW[tap][co][ci] = sum over pixels of dy[pixel, co] * x[pixel shifted by tap, ci]  (stride 1).
-// GEMM view per 64-channel block pair (ci chunk, co chunk): the K dimension is the pixel index, so
-// both operands are MN-major in shared memory exactly as TMA delivers the channels-last tiles:
-//   A (M = 128 rows) = two stacked (tap, 64 input channels) chunks taken from the three
-//       column-shifted activation boxes; the second chunk sits one leading-dimension offset away
-//       (BW rows for the next row tap, or one box for the next column tap),
-//   B (N = 64)       = the dy tile of the 64 output channels,
-//   K                = 16 pixels per instruction, 128 pixels per pipeline stage.
-// Five instructions per 16 pixels cover the nine taps (the last one half empty); their five
-// 128 x 64 accumulators stay in tensor memory over the CTA's whole pixel range (split-K); at the
-// end they are written to a per-CTA partial that a second kernel sums in a fixed order.
+// dW[tap][co][ci] = sum over pixels of dy[pixel, co] * x[pixel shifted by tap, ci].  The K dimension of the
+// GEMM is the pixel index, so both operands are MN-major in shared memory exactly as TMA delivers the
+// channels-last tiles.  Work is split over (64-input-channel chunk, output-channel chunk) pairs and over
+// the pixel tiles (split-K): accumulators stay in tensor memory over a CTA's whole pixel range and are
+// written as per-CTA partials that a second kernel sums in a fixed order.  Two kernels: the per-tap form
+// below (stride 2 and small feature maps) and conv_wgrad_kw_kernel (stride 1).
 struct WgParams {
   int N, H, W, Cin, Cout;
   int BW, BH, tiles_w, tiles_h, pix_tiles, ci_chunks, co_chunks, splits, stages, stride, BI;
@@ -600,9 +595,9 @@ struct WgParams {
 
 // NB = width of the output-gradient tile in channels (64: main conv, one 64-channel chunk per CTA;
 // 16/32/64: aux conv with F <= NB filters, rows of 2*NB bytes with the matching TMA swizzle).
-// S2 = 1: per-tap mode (stride-2 convolutions, and feature maps smaller than a tile where a tile spans BI
-// whole images).  The shifted activation tiles are gathered by TMA, with element stride 2 for stride 2,
-// one 128-pixel tile per tap; a CTA then owns one kernel row kh (grid dimension) with its three column
+// Per-tap form (S2 is always 1): stride-2 convolutions, and feature maps smaller than a tile where a tile
+// spans BI whole images.  The shifted activation tiles are gathered by TMA, with element stride 2 for
+// stride 2, one 128-pixel tile per tap; a CTA then owns one kernel row kh (grid dimension) with its three column
 // taps: taps (kh,0) and (kh,1) stacked in one instruction, tap (kh,2) in a second, half-empty one.
 template <int NB, int S2>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -612,9 +607,10 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   constexpr int kBTile = 128 * kBRow;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr int kStages = S2 ? 3 : 2;
-  constexpr int kJobs = S2 ? 2 : 5;  // instructions (accumulators) per 16 pixels
-  const int copy_bytes = S2 ? 16384 : (p.BH + 2) * p.BW * 128;
+  static_assert(S2 == 1, "stride 1 on tileable maps uses conv_wgrad_kw_kernel");
+  constexpr int kStages = 3;
+  constexpr int kJobs = 2;  // instructions (accumulators) per 16 pixels
+  constexpr int copy_bytes = 16384;  // one 128-pixel tap tile
   const int stage_bytes = 3 * copy_bytes + 16384;  // the dy tile always gets 16 KB so the unused rows read by the
                                                    // half-empty last instruction stay inside the stage
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * stage_bytes);
@@ -630,8 +626,8 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   const int blocks = p.ci_chunks * p.co_chunks;
   const int blk = blockIdx.x % blocks;
   const int rest = blockIdx.x / blocks;
-  const int khg = S2 ? rest % 3 : 0;            // kernel row owned by this CTA (stride 2 only)
-  const int sp = S2 ? rest / 3 : rest;
+  const int khg = rest % 3;  // kernel row owned by this CTA
+  const int sp = rest / 3;
   const int cic = blk % p.ci_chunks, coc = blk / p.ci_chunks;
   const int t0 = (int)((long)p.pix_tiles * sp / p.splits), t1 = (int)((long)p.pix_tiles * (sp + 1) / p.splits);
 
@@ -666,12 +662,8 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         uint8_t* st = smem + (size_t)s * stage_bytes;
         ptx::mbar_expect_tx(&full[s], (uint32_t)(3 * copy_bytes + kBTile));
 #pragma unroll
-        for (int kw = 0; kw < 3; ++kw) {
-          if constexpr (S2)
-            ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, p.stride * w0 + kw - 1, p.stride * h0 + khg - 1, n);
-          else
-            ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, w0 + kw - 1, h0 - 1, n);
-        }
+        for (int kw = 0; kw < 3; ++kw)
+          ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, p.stride * w0 + kw - 1, p.stride * h0 + khg - 1, n);
         ptx::tma_load_4d(st + 3 * copy_bytes, &tm_dy, &full[s], coc * NB, w0, h0, n);
       }
       __syncwarp();
@@ -688,30 +680,18 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       if (lane == 0) {
         const uint32_t xb = ptx::smem_u32(smem + (size_t)s * stage_bytes);
         const uint32_t x16 = xb >> 4, g16 = (xb + 3 * copy_bytes) >> 4;
-        const uint32_t row16 = (uint32_t)(p.BW * 128) >> 4, copy16 = (uint32_t)copy_bytes >> 4;
-        // descriptors differ only in the address field; the leading-dimension offset selects what is stacked
-        const uint64_t a_row_hi = ptx::sdesc(0, p.BW * 128, 1024, 2);   // second chunk one image row further
-        const uint64_t a_copy_hi = ptx::sdesc(0, copy_bytes, 1024, 2);  // second chunk one box / tile further
+        const uint32_t copy16 = (uint32_t)copy_bytes >> 4;
+        // descriptors differ only in the address field; the second stacked chunk sits one tap tile further
+        const uint64_t a_copy_hi = ptx::sdesc(0, copy_bytes, 1024, 2);
         const uint64_t b_hi = ptx::sdesc(0, 16, 8 * kBRow, kBLayout);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint32_t k16 = k * 128;  // 16 pixels x 128 bytes, in 16-byte units
           const uint64_t bd = b_hi | (uint64_t)(g16 + k * kBRow);
           const uint32_t acc = (it | k) != 0;
-          if constexpr (S2) {
-            // taps (kh,0) and (kh,1): second chunk one tile further; tap (kh,2): rows 64..127 unused
-            ptx::mma_f16(tmem_base, a_copy_hi | (uint64_t)(x16 + k16), bd, idesc, acc);
-            ptx::mma_f16(tmem_base + NB, a_copy_hi | (uint64_t)(x16 + 2 * copy16 + k16), bd, idesc, acc);
-          } else {
-#pragma unroll
-            for (int kw = 0; kw < 3; ++kw)  // taps (kh=0,kw) and (kh=1,kw): second chunk one image row further
-              ptx::mma_f16(tmem_base + kw * NB, a_row_hi | (uint64_t)(x16 + kw * copy16 + k16), bd, idesc, acc);
-            // taps (kh=2,kw=0) and (kh=2,kw=1): second chunk one box further
-            ptx::mma_f16(tmem_base + 3 * NB, a_copy_hi | (uint64_t)(x16 + 2 * row16 + k16), bd, idesc, acc);
-            // tap (kh=2,kw=2); rows 64..127 of this accumulator are not used (their operand rows fall on the
-            // rows after the box, which are still inside this stage's buffer)
-            ptx::mma_f16(tmem_base + 4 * NB, a_row_hi | (uint64_t)(x16 + 2 * copy16 + 2 * row16 + k16), bd, idesc, acc);
-          }
+          // taps (kh,0) and (kh,1): second chunk one tile further; tap (kh,2): rows 64..127 unused
+          ptx::mma_f16(tmem_base, a_copy_hi | (uint64_t)(x16 + k16), bd, idesc, acc);
+          ptx::mma_f16(tmem_base + NB, a_copy_hi | (uint64_t)(x16 + 2 * copy16 + k16), bd, idesc, acc);
         }
         ptx::mma_commit(&empty[s]);
       }
@@ -730,14 +710,8 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll 1
       for (int j = 0; j < kJobs; ++j) {
         // taps of accumulator j: rows 0..63 -> tapA, rows 64..127 -> tapB (kh*3+kw)
-        int tapA, tapB;
-        if constexpr (S2) {
-          tapA = khg * 3 + (j == 0 ? 0 : 2);
-          tapB = j == 0 ? khg * 3 + 1 : -1;
-        } else {
-          tapA = j < 3 ? j : (j == 3 ? 6 : 8);
-          tapB = j < 3 ? 3 + j : (j == 3 ? 7 : -1);
-        }
+        const int tapA = khg * 3 + (j == 0 ? 0 : 2);
+        const int tapB = j == 0 ? khg * 3 + 1 : -1;
         const int tap = m < 64 ? tapA : tapB;
 #pragma unroll
         for (int q = 0; q < NB / 16; ++q) {
