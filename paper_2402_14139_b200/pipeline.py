@@ -1,0 +1,114 @@
+"""Block-wise local learning over a dataset resident in HBM (Algorithm 2 with its outer loops, the
+activation cache and the re-batching step), driven through the C-ABI binding.
+
+For each block in order: for each epoch, a seeded permutation of the sample indices is cut into
+batches of the block's own batch size (a last partial batch is dropped), every batch is assembled by
+nf_cache_gather from the block's input set (the images for block 1, the cached activations of the
+previous block otherwise) and stepped through all layers of the block with nf_block_step.  When a
+block has finished, its output for every sample is written to the cache by nf_block_cache (forward
+only, running statistics) and becomes the next block's input set.  Earlier blocks are never run again.
+
+    python -m paper_2402_14139_b200.pipeline --workload c5 --images 10000 --epochs 3
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import time
+
+import numpy as np
+
+from . import synth, workloads
+
+
+def build_layers(nf, wl, block_index, seed):
+    """nf.Layer objects of one block with seeded Kaiming-normal weights, and the nf.Block over them."""
+    N, ls = wl["blocks"][block_index]
+    dt = nf.NF_F32 if wl["dtype"] == "f32" else nf.NF_BF16
+    layers = []
+    for li, l in enumerate(ls):
+        L = nf.Layer(l["Cin"], l["Cout"], l["H"], l["W"], l["F"], wl["classes"], N, stride=l["stride"], maxpool=l["pool"], dtype=dt)
+        t = 100 * (block_index * 32 + li)
+        L.set_param("W", synth.normal(seed, t + 1, L.shapes["W"], np.sqrt(2.0 / (9 * l["Cin"]))))
+        L.set_param("Wa", synth.normal(seed, t + 2, L.shapes["Wa"], np.sqrt(2.0 / (9 * l["Cout"]))))
+        L.set_param("Wf", synth.normal(seed, t + 3, L.shapes["Wf"], np.sqrt(2.0 / (4 * l["F"]))))
+        layers.append(L)
+    return layers, nf.Block(layers)
+
+
+def train_blockwise(nf, torch, wl, data, labels, epochs=1, lr=0.01, seed=1, log=None):
+    """data: device tensor [K, H, W, C] of the first layer's dtype; labels: device int32 [K].
+    Returns a list of per-block records (batch size, steps, seconds, images/s, last losses)."""
+    K = data.shape[0]
+    report = []
+    cur = data
+    for bi, (N, ls) in enumerate(wl["blocks"]):
+        N = min(N, K)
+        capped = dict(wl, blocks=[(N, l2) if i == bi else (n2, l2) for i, (n2, l2) in enumerate(wl["blocks"])])
+        layers, block = build_layers(nf, capped, bi, seed)
+        xb = torch.empty((N,) + tuple(cur.shape[1:]), dtype=cur.dtype, device=cur.device)
+        yb = torch.empty(N, dtype=torch.int32, device=cur.device)
+        loss = torch.zeros(len(ls), dtype=torch.float32, device=cur.device)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        steps = 0
+        for ep in range(epochs):
+            perm = torch.from_numpy(synth.permutation(seed + 7919 * bi, ep, K)).to(cur.device)
+            for s in range(K // N):
+                nf.nf_cache_gather(cur, labels, perm[s * N:(s + 1) * N].contiguous(), xb, yb)
+                block.step(xb, yb, lr, loss)
+                steps += 1
+        torch.cuda.synchronize()
+        t_train = time.perf_counter() - t0
+        status = [L.status() for L in layers]
+        if any(status):
+            raise RuntimeError(f"block {bi}: device status {status}")
+        # fill the cache: the block's output for every sample, in chunks of the block's batch size
+        last = layers[-1]
+        out = torch.empty((K, last.Ha, last.Wa, last.Cout), dtype=cur.dtype, device=cur.device)
+        t1 = time.perf_counter()
+        for s in range(0, K, N):
+            cnt = min(N, K - s)
+            block.cache(cur[s:s + cnt], out[s:s + cnt], count=cnt)
+        torch.cuda.synchronize()
+        t_cache = time.perf_counter() - t1
+        rec = dict(block=bi, layers=len(ls), batch=N, steps=steps, train_s=round(t_train, 4), cache_s=round(t_cache, 4),
+                   train_images_per_s=round(steps * N / max(t_train, 1e-9), 1), losses=[round(v, 4) for v in loss.cpu().tolist()])
+        report.append(rec)
+        if log:
+            log(rec)
+        block.close()
+        for L in layers:
+            L.close()
+        cur = out
+    return report, cur
+
+
+def main():
+    import torch
+    from . import nf
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="c5", choices=sorted(workloads.ALL))
+    ap.add_argument("--images", type=int, default=10000)
+    ap.add_argument("--epochs", type=int, default=3)
+    ap.add_argument("--lr", type=float, default=0.01)
+    args = ap.parse_args()
+    nf.lib()
+    nf.nf_set_stream(torch.cuda.current_stream())
+    wl = workloads.ALL[args.workload]()
+    C, H, W = wl["in_shape"]
+    g = torch.Generator(device="cuda")
+    g.manual_seed(0x4E460005)
+    tdt = torch.float32 if wl["dtype"] == "f32" else torch.bfloat16
+    data = torch.randn((args.images, H, W, C), generator=g, device="cuda", dtype=torch.float32).to(tdt)
+    labels = torch.randint(0, wl["classes"], (args.images,), generator=g, device="cuda", dtype=torch.int32)
+    t0 = time.perf_counter()
+    report, _ = train_blockwise(nf, torch, wl, data, labels, epochs=args.epochs, lr=args.lr, log=lambda r: print(json.dumps(r), flush=True))
+    wall = time.perf_counter() - t0
+    n_layers = sum(len(ls) for _, ls in wl["blocks"])
+    print(json.dumps(dict(workload=wl["name"], images=args.images, epochs=args.epochs, layers=n_layers, wall_s=round(wall, 3),
+                          images_per_s_whole_pass=round(args.images * args.epochs / wall, 1))))
+
+
+if __name__ == "__main__":
+    main()
