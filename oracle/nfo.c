@@ -478,3 +478,25 @@ void nfo_layer_eval(const nfo_dims* d, const double* x, const nfo_params* P, dou
   }
   free(y); free(z); free(r);
 }
+
+/* Early-exit prediction of one layer (Section "Trained output CNN": every layer with its auxiliary
+ * network is a prospective exit).  Forward only, normalisation with the running statistics:
+ * act_out = x_{n+1} (Eq. 1), logits = z_{n+1} = gamma_n F_n beta_n x_{n+1} (Eq. 2).  The class is the
+ * arg-max of the logits (taken by the caller: first maximum). */
+void nfo_layer_predict(const nfo_dims* d, const double* x, const nfo_params* P, double* act_out, double* logits) {
+  const int N = d->N, Co = d->Cout, F = d->F, K = d->classes, s = d->stride;
+  const int Ho = nfo_out_size(d->H, s), Wo = nfo_out_size(d->W, s);
+  const int Ha = d->pool ? Ho / 2 : Ho, Wa = d->pool ? Wo / 2 : Wo;
+  const size_t na = (size_t)N * Co * Ha * Wa, nh = (size_t)N * F * Ha * Wa;
+  double *a = dalloc(na), *hpre = dalloc(nh), *h = dalloc(nh), *p = dalloc((size_t)N * 4 * F);
+  nfo_layer_eval(d, x, P, a);
+  double* Waq = dalloc((size_t)F * Co * 9);
+  memcpy(Waq, P->Wa, sizeof(double) * (size_t)F * Co * 9);
+  store_round(Waq, (size_t)F * Co * 9, d->store_bf16);
+  nfo_conv3x3(a, N, Co, Ha, Wa, Waq, F, P->ba, 1, hpre);
+  nfo_relu(hpre, nh, h);
+  nfo_avgpool_2x2(h, N, F, Ha, Wa, p);
+  nfo_fc(p, N, 4 * F, P->Wf, P->bf, K, logits);
+  if (act_out) memcpy(act_out, a, na * sizeof(double));
+  free(a); free(hpre); free(h); free(p); free(Waq);
+}

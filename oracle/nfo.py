@@ -248,6 +248,23 @@ class Layer:
                                     C.byref(P), _d(act), C.byref(T) if T is not None else None, int(update))
         return float(loss), act, arrs
 
+    def predict(self, x):
+        """Early-exit prediction for any batch size: (act_out, logits, classes); class = first arg-max."""
+        x = _c64(x)
+        d = Dims.from_buffer_copy(self.d)
+        d.N = x.shape[0]
+        act = np.empty((d.N, d.Cout, self.Ha, self.Wa))
+        logits = np.empty((d.N, d.classes))
+        P = self._params()
+        lib().nfo_layer_predict(C.byref(d), _d(x), C.byref(P), _d(act), _d(logits))
+        return act, logits, np.argmax(logits, axis=1).astype(np.int32)
+
+    def n_params(self):
+        """(main-path parameters W, gamma, beta; aux-head parameters Wa, ba, Wf, bf)."""
+        main = sum(self.p[k].size for k in ("W", "gamma", "beta"))
+        aux = sum(self.p[k].size for k in ("Wa", "ba", "Wf", "bf"))
+        return main, aux
+
     def eval_forward(self, x):
         """Eval-mode forward (running statistics) for any batch size."""
         x = _c64(x)
@@ -257,6 +274,16 @@ class Layer:
         P = self._params()
         lib().nfo_layer_eval(C.byref(d), _d(x), C.byref(P), _d(out))
         return out
+
+
+def select_exit(val_accuracy, params):
+    """Exit-point rule of the paper's "Trained output CNN" section: the layer whose early-exit model has the
+    highest validation accuracy; among equals, the one with the fewest parameters.  Returns its index."""
+    best = 0
+    for i in range(1, len(val_accuracy)):
+        if val_accuracy[i] > val_accuracy[best] or (val_accuracy[i] == val_accuracy[best] and params[i] < params[best]):
+            best = i
+    return best
 
 
 def partition(max_batch, B, rho):

@@ -221,3 +221,30 @@ def test_bf16_storage_mode_rounds_only_the_stored_tensors():
     v = np.array([1.0, 1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, -2.5, 3.14159, 1e-20, 65504.0, 0.0])
     got = np.array([nfo.lib().nfo_round_bf16(float(t)) for t in v])
     np.testing.assert_array_equal(got, torch.tensor(v, dtype=torch.float32).to(torch.bfloat16).double().numpy())
+
+
+def test_early_exit_prediction_against_library_ops_and_selection_rule():
+    c = CASES[2]
+    L, x, y = make_layer(c, 31)
+    L.step(x, y, 0.05)                       # running statistics away from their initial values
+    act, logits, cls = L.predict(x)
+    F = torch.nn.functional
+    t = lambda a: torch.tensor(np.asarray(a, dtype=np.float64))
+    with torch.no_grad():
+        z = F.batch_norm(F.conv2d(t(x), t(L.p["W"]), None, stride=c["stride"], padding=1), t(L.rmean), t(L.rvar),
+                         t(L.p["gamma"]), t(L.p["beta"]), training=False, eps=1e-5)
+        a = F.max_pool2d(F.relu(z), 2)
+        h = F.relu(F.conv2d(a, t(L.p["Wa"]), t(L.p["ba"]), padding=1))
+        lg = F.linear(F.adaptive_avg_pool2d(h, 2).flatten(1), t(L.p["Wf"]), t(L.p["bf"]))
+    np.testing.assert_allclose(act, a.numpy(), atol=1e-12)
+    np.testing.assert_allclose(logits, lg.numpy(), atol=1e-12)
+    np.testing.assert_array_equal(cls, lg.numpy().argmax(axis=1))
+    np.testing.assert_array_equal(act, L.eval_forward(x))
+    # per-sample: a prediction does not depend on the batch it is evaluated in
+    np.testing.assert_array_equal(L.predict(x[1:2])[1][0], logits[1])
+    # selection: highest accuracy wins; equal accuracy -> fewer parameters (the figure's "layer 5" situation)
+    assert nfo.select_exit([0.31, 0.52, 0.64, 0.64, 0.63], [10, 20, 30, 40, 50]) == 2
+    assert nfo.select_exit([0.7, 0.7, 0.7], [30, 20, 25]) == 1
+    assert nfo.select_exit([0.2], [5]) == 0
+    main, aux = L.n_params()
+    assert main == c["Cout"] * c["Cin"] * 9 + 2 * c["Cout"] and aux == c["F"] * c["Cout"] * 9 + c["F"] + c["classes"] * (4 * c["F"] + 1)
