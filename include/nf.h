@@ -155,6 +155,22 @@ void nf_block_destroy(nf_block* block);
 int nf_block_cache(nf_block* block, const void* x, void* out);
 int nf_block_cache_n(nf_block* block, const void* x, void* out, int count);
 
+/* Early-exit evaluation (Section "Trained output CNN": every layer with its auxiliary network is a
+ * prospective exit point).  Forward only, BatchNorm with running statistics, no parameter changes:
+ *   act_out = x_{n+1} for `count` samples (device, [count][Ha][Wa][Cout]; NULL keeps it in the workspace),
+ *   logits_out = z_{n+1} (device float [count][classes]; may be NULL),
+ *   pred_out = arg-max class per sample, first maximum (device int32 [count]).
+ * count must be in [1, N].  Feed act_out to the next layer's nf_layer_predict to evaluate deeper exits. */
+int nf_layer_predict(nf_layer* layer, const void* x, int count, void* act_out, float* logits_out, int32_t* pred_out);
+
+/* Parameters of a layer: part 0 = main path (W, gamma, beta), 1 = auxiliary network (Wa, ba, Wf, bf), 2 = both.
+ * An early-exit model at layer n holds the main parts of layers 1..n plus the auxiliary part of layer n. */
+long long nf_layer_param_count(const nf_layer* layer, int part);
+
+/* Exit selection (host only): the index with the highest validation accuracy; among equals the one with the
+ * fewest parameters.  NF_EINVAL on bad arguments. */
+int nf_select_exit(const double* val_accuracy, const long long* params, int n_layers);
+
 /* One pass of Algorithm 2's inner loop over ALL layers of the block on one batch: layer 1 steps
  * on x, every later layer steps on the activation its predecessor just produced (computed before
  * that predecessor's update), each with its own local loss.

@@ -345,7 +345,7 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
   // Eq. 2: aux conv + ReLU, average pool to 2x2, linear; Eq. 3: softmax cross-entropy
   trace_begin(2);
   if (L->fam[2]) {
-    NF_TRY(nf_tc_aux_fwd(L, act_out));
+    NF_TRY(nf_tc_aux_fwd(L, act_out, N));
   } else {
     NF_TRY(nf_ref_conv(dt, act_out, N, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
   }
@@ -459,6 +459,8 @@ void nf_block_destroy(nf_block* B) {
   free(B);
 }
 
+static int layer_eval_forward(nf_layer* L, const void* in, int count, void* dst);
+
 int nf_block_cache_n(nf_block* B, const void* x, void* out, int count) {
   if (!B || !x || !out) return NF_EINVAL;
   if (count < 1 || count > B->layers[0]->o.N) return NF_EINVAL;
@@ -466,21 +468,64 @@ int nf_block_cache_n(nf_block* B, const void* x, void* out, int count) {
   const void* in = x;
   for (int l = 0; l < B->n; ++l) {
     nf_layer* L = B->layers[l];
-    const int dt = L->o.dtype;
-    const void* Wm = dt == NF_F32 ? (const void*)(L->val + L->off[NF_P_W]) : (const void*)(L->shadow + L->off[NF_P_W]);
     void* dst = l == B->n - 1 ? out : L->dy;
-    if (L->fam[0]) {
-      NF_TRY(nf_tc_conv_fwd_eval(L, in, count));
-    } else {
-      NF_TRY(nf_ref_conv(dt, in, count, L->H, L->W, L->Cin, Wm, (long)L->Cout * L->Cin, L->Cin, 1, 0, nullptr, 0,
-                         L->o.stride, L->Cout, L->y));
-    }
-    NF_TRY(nf_ref_bn_eval_coeffs(L->Cout, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps, L->rmean,
-                                 L->rvar, L->scale, L->shift));
-    NF_TRY(nf_ref_bn_apply(dt, L->y, count, L->Ho, L->Wo, L->Cout, L->o.maxpool, L->scale, L->shift, dst));
+    NF_TRY(layer_eval_forward(L, in, count, dst));
     in = dst;
   }
   return NF_OK;
+}
+
+// eval-mode forward of one layer for `count` samples into dst (conv, running-statistics BatchNorm, ReLU, pool)
+static int layer_eval_forward(nf_layer* L, const void* in, int count, void* dst) {
+  const int dt = L->o.dtype;
+  const void* Wm = dt == NF_F32 ? (const void*)(L->val + L->off[NF_P_W]) : (const void*)(L->shadow + L->off[NF_P_W]);
+  if (L->fam[0]) {
+    NF_TRY(nf_tc_conv_fwd_eval(L, in, count));
+  } else {
+    NF_TRY(nf_ref_conv(dt, in, count, L->H, L->W, L->Cin, Wm, (long)L->Cout * L->Cin, L->Cin, 1, 0, nullptr, 0, L->o.stride,
+                       L->Cout, L->y));
+  }
+  NF_TRY(nf_ref_bn_eval_coeffs(L->Cout, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps, L->rmean, L->rvar,
+                               L->scale, L->shift));
+  return nf_ref_bn_apply(dt, L->y, count, L->Ho, L->Wo, L->Cout, L->o.maxpool, L->scale, L->shift, dst);
+}
+
+int nf_layer_predict(nf_layer* L, const void* x, int count, void* act_out, float* logits_out, int32_t* pred_out) {
+  if (!L || !x || !pred_out) return NF_EINVAL;
+  if (!L->ws) return NF_ENOWS;
+  if (count < 1 || count > L->o.N) return NF_EINVAL;
+  if (misaligned(x) || (act_out && misaligned(act_out))) return NF_EALIGN;
+  const int dt = L->o.dtype, Co = L->Cout, F = L->F, Ha = L->Ha, Wa = L->Wa;
+  void* a = act_out ? act_out : L->act;
+  NF_TRY(layer_eval_forward(L, x, count, a));
+  const void* Wx = dt == NF_F32 ? (const void*)(L->val + L->off[NF_P_WA]) : (const void*)(L->shadow + L->off[NF_P_WA]);
+  if (L->fam[2]) {
+    NF_TRY(nf_tc_aux_fwd(L, a, count));
+  } else {
+    NF_TRY(nf_ref_conv(dt, a, count, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
+  }
+  {
+    int rc = dt == NF_BF16 ? nf_ref_avgpool_fast(L->h, count, Ha, Wa, F, L->wpart, L->wpart_floats, L->p) : NF_EUNSUPPORTED;
+    if (rc == NF_EUNSUPPORTED) rc = nf_ref_avgpool(dt, L->h, count, Ha, Wa, F, L->p);
+    if (rc != NF_OK) return rc;
+  }
+  // the caller's logits have `classes` columns over the logical 4*Flog inputs; the padded inputs are zero
+  return nf_ref_fc_predict(L->p, count, 4 * F, L->classes, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], logits_out, pred_out);
+}
+
+long long nf_layer_param_count(const nf_layer* L, int part) {
+  if (!L) return NF_EINVAL;
+  const long long main = 9LL * L->Cout * L->Cin + 2LL * L->Cout;
+  const long long aux = 9LL * L->Flog * L->Cout + L->Flog + (long long)L->classes * (4 * L->Flog + 1);
+  return part == 0 ? main : part == 1 ? aux : main + aux;
+}
+
+int nf_select_exit(const double* val_accuracy, const long long* params, int n_layers) {
+  if (!val_accuracy || !params || n_layers < 1) return NF_EINVAL;
+  int best = 0;
+  for (int i = 1; i < n_layers; ++i)
+    if (val_accuracy[i] > val_accuracy[best] || (val_accuracy[i] == val_accuracy[best] && params[i] < params[best])) best = i;
+  return best;
 }
 
 int nf_block_cache(nf_block* B, const void* x, void* out) {

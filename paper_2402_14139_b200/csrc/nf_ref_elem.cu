@@ -264,6 +264,40 @@ __global__ void __launch_bounds__(256) fc_ce_kernel(const float* __restrict__ p,
   }
 }
 
+
+// one block per sample: logits = Wf p + bf (optionally stored) and the class = first arg-max
+__global__ void __launch_bounds__(256) fc_predict_kernel(const float* __restrict__ p, int D, int K, const float* __restrict__ Wf,
+                                                         const float* __restrict__ bf, float* __restrict__ logits,
+                                                         int32_t* __restrict__ pred) {
+  extern __shared__ float dyn[];
+  float* ps = dyn;
+  __shared__ float bv[256];
+  __shared__ int bi[256];
+  const int n = blockIdx.x, t = threadIdx.x;
+  for (int d = t; d < D; d += 256) ps[d] = p[(size_t)n * D + d];
+  __syncthreads();
+  float best = -INFINITY;
+  int arg = 0x7fffffff;
+  for (int k = t; k < K; k += 256) {
+    float s = bf[k];
+    const float* w = Wf + (size_t)k * D;
+    for (int d = 0; d < D; ++d) s = fmaf(w[d], ps[d], s);
+    if (logits) logits[(size_t)n * K + k] = s;
+    if (s > best) { best = s; arg = k; }   // k ascending within a thread: keeps the first maximum
+  }
+  bv[t] = best;
+  bi[t] = arg;
+  __syncthreads();
+  for (int s2 = 128; s2 > 0; s2 >>= 1) {
+    if (t < s2 && (bv[t + s2] > bv[t] || (bv[t + s2] == bv[t] && bi[t + s2] < bi[t]))) {
+      bv[t] = bv[t + s2];
+      bi[t] = bi[t + s2];
+    }
+    __syncthreads();
+  }
+  if (t == 0) pred[n] = bi[0];
+}
+
 // one block per class k: gWf[k][:] = sum_n dlogits[n][k] p[n][:], gbf[k]; block 0 also reduces the loss
 __global__ void __launch_bounds__(256) fc_wgrad_kernel(const float* __restrict__ p, const float* __restrict__ dl,
                                                        const float* __restrict__ lossn, int N, int D, int K,
@@ -997,6 +1031,14 @@ int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, con
   const size_t smem = (size_t)(D + K) * sizeof(float);
   if (smem > 40000) return NF_EUNSUPPORTED;
   fc_ce_kernel<<<N, 256, smem, g_nf_stream>>>(p, labels, N, D, K, Wf, bf, logits, dlogits, dp, lossn, status);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_fc_predict(const float* p, int N, int D, int K, const float* Wf, const float* bf, float* logits, int32_t* pred) {
+  const size_t smem = (size_t)D * sizeof(float);
+  if (smem > 40000) return NF_EUNSUPPORTED;
+  fc_predict_kernel<<<N, 256, smem, g_nf_stream>>>(p, D, K, Wf, bf, logits, pred);
   NF_LAUNCHED();
   return NF_OK;
 }

@@ -1266,9 +1266,9 @@ int nf_tc_conv_fwd_eval(nf_layer* L, const void* x, int count) {
                  nullptr, L->o.stride);
 }
 
-int nf_tc_aux_fwd(nf_layer* L, const void* a) {
+int nf_tc_aux_fwd(nf_layer* L, const void* a, int count) {
   int nb = 0;
-  return run_fwd(L->o.N, L->Ha, L->Wa, L->Cout, L->F, a, L->shadow + L->off[NF_P_WA], L->h, 0, nullptr, 0, L->status, &nb, 1,
+  return run_fwd(count, L->Ha, L->Wa, L->Cout, L->F, a, L->shadow + L->off[NF_P_WA], L->h, 0, nullptr, 0, L->status, &nb, 1,
                  L->val + L->off[NF_P_BA]);
 }
 

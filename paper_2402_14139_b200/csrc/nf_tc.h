@@ -24,8 +24,8 @@ int nf_tc_op_status(int32_t* out);
 size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout, int stride);
 int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int Cin, int Cout, int stride, float* part,
                         size_t part_floats, float* dw);
-// Aux conv forward on tensor cores: L->h = ReLU(conv(a, Wa) + ba) in bf16.
-int nf_tc_aux_fwd(nf_layer* L, const void* a);
+// Aux conv forward on tensor cores for `count` samples: L->h = ReLU(conv(a, Wa) + ba) in bf16.
+int nf_tc_aux_fwd(nf_layer* L, const void* a, int count);
 // Aux conv weight gradient on tensor cores: grad(Wa) = wgrad(a, L->dh).
 int nf_tc_aux_wgrad(nf_layer* L, const void* a);
 // Aux conv input gradient on tensor cores: L->da = dgrad(L->dh, Wa) in bf16.

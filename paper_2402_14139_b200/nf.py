@@ -25,7 +25,7 @@ PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P
 EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_layer_workspace_bytes",
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
-           "nf_block_cache_n", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
+           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
            "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_op_status", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
@@ -69,6 +69,10 @@ def lib():
         L.nf_block_destroy.argtypes = [vp]
         L.nf_block_cache.argtypes = [vp, vp, vp]
         L.nf_block_cache_n.argtypes = [vp, vp, vp, C.c_int]
+        L.nf_layer_predict.argtypes = [vp, vp, C.c_int, vp, fp, ip]
+        L.nf_layer_param_count.restype = C.c_longlong
+        L.nf_layer_param_count.argtypes = [vp, C.c_int]
+        L.nf_select_exit.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.c_int]
         L.nf_block_step.argtypes = [vp, vp, ip, C.c_float, fp, vp]
         L.nf_block_step_host.argtypes = [vp, vp, ip, C.c_float, fp, vp]
         L.nf_trace_enable.argtypes = [C.c_int]
@@ -148,6 +152,17 @@ def nf_trace_read(slots: int = 1):
     return out
 
 
+def nf_select_exit(val_accuracy, params) -> int:
+    """Index of the exit with the highest validation accuracy, fewest parameters among equals."""
+    n = len(val_accuracy)
+    acc = (C.c_double * n)(*[float(v) for v in val_accuracy])
+    par = (C.c_longlong * n)(*[int(v) for v in params])
+    rc = lib().nf_select_exit(acc, par, n)
+    if rc < 0:
+        _check(rc, "nf_select_exit")
+    return rc
+
+
 def _ptr(t):
     return C.c_void_p(t.data_ptr()) if t is not None else None
 
@@ -212,6 +227,14 @@ class Layer:
         """nf_layer_step_host on host tensors (pinned for speed); synchronous."""
         _check(lib().nf_layer_step_host(self.h, _ptr(x_host), _ptr(labels_host), float(lr), _ptr(loss_host),
                                         _ptr(act_host)), "nf_layer_step_host")
+
+    def predict(self, x, pred_out, act_out=None, logits_out=None, count=None):
+        """nf_layer_predict: early-exit forward for `count` (default N) samples; device tensors."""
+        _check(lib().nf_layer_predict(self.h, _ptr(x), int(self.N if count is None else count), _ptr(act_out), _ptr(logits_out),
+                                      _ptr(pred_out)), "nf_layer_predict")
+
+    def param_count(self, part=2) -> int:
+        return int(lib().nf_layer_param_count(self.h, part))
 
     def status(self) -> int:
         rc = lib().nf_layer_status(self.h)

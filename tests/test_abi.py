@@ -72,3 +72,17 @@ def test_partition_matches_checker_and_paper_example(nf):
         assert nf.nf_partition(v, B, rho) == nfo.partition(v, B, rho)
     with pytest.raises(nf.NfError):
         nf.nf_partition([10, 0], 100, 0.4)
+
+
+def test_select_exit_rule_matches_checker_on_the_host():
+    """Highest validation accuracy wins; equal accuracies go to the smaller model; the first of full ties."""
+    from oracle import nfo
+    from paper_2402_14139_b200 import nf, synth
+    assert nf.nf_select_exit([0.5, 0.7, 0.7, 0.6], [10, 30, 20, 40]) == 2
+    assert nf.nf_select_exit([0.7, 0.7], [20, 20]) == 0
+    assert nf.nf_select_exit([0.1], [5]) == 0
+    for t in range(50):
+        n = 1 + t % 9
+        acc = [round(float(v) * 4) / 4 for v in synth.uniform01(0x4E46E200, t, n)]     # many ties
+        par = [int(v * 5) for v in synth.uniform01(0x4E46E201, t, n)]
+        assert nf.nf_select_exit(acc, par) == nfo.select_exit(acc, par)
