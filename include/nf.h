@@ -163,6 +163,10 @@ int nf_block_cache_n(nf_block* block, const void* x, void* out, int count);
  * count must be in [1, N].  Feed act_out to the next layer's nf_layer_predict to evaluate deeper exits. */
 int nf_layer_predict(nf_layer* layer, const void* x, int count, void* act_out, float* logits_out, int32_t* pred_out);
 
+/* Validation accuracy of an exit: *count += #{i < n : a[i] == b[i]} (device int32 arrays, device 64-bit counter that
+ * the caller zeroes; integer accumulation, so the result does not depend on launch order). */
+int nf_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count);
+
 /* Parameters of a layer: part 0 = main path (W, gamma, beta), 1 = auxiliary network (Wa, ba, Wf, bf), 2 = both.
  * An early-exit model at layer n holds the main parts of layers 1..n plus the auxiliary part of layer n. */
 long long nf_layer_param_count(const nf_layer* layer, int part);

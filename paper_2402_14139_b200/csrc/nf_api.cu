@@ -513,6 +513,11 @@ int nf_layer_predict(nf_layer* L, const void* x, int count, void* act_out, float
   return nf_ref_fc_predict(L->p, count, 4 * F, L->classes, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], logits_out, pred_out);
 }
 
+int nf_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count) {
+  if (!a || !b || !count || n < 1) return NF_EINVAL;
+  return nf_ref_count_equal(a, b, n, count);
+}
+
 long long nf_layer_param_count(const nf_layer* L, int part) {
   if (!L) return NF_EINVAL;
   const long long main = 9LL * L->Cout * L->Cin + 2LL * L->Cout;

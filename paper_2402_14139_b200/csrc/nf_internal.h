@@ -100,6 +100,7 @@ int nf_ref_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F,
                    int* nblocks);
 int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
                  float* logits, float* dlogits, float* dp, float* lossn, int32_t* status);
+int nf_ref_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count);
 int nf_ref_fc_predict(const float* p, int N, int D, int K, const float* Wf, const float* bf, float* logits, int32_t* pred);
 int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
                     float* gbf, float* loss_out, int32_t* status);

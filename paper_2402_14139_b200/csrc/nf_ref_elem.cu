@@ -1,6 +1,7 @@
 // Memory-bound kernels of the local-layer step: BatchNorm statistics / apply / backward, pooling,
 // the linear + softmax cross-entropy head, momentum SGD and the cache gather.  Storage fp32 or
 // bf16, arithmetic fp32, cross-block sums finished in fp64 in a fixed order (deterministic).
+#include <algorithm>
 #include "nf_internal.h"
 #include "nf_ldst.cuh"
 
@@ -1031,6 +1032,21 @@ int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, con
   const size_t smem = (size_t)(D + K) * sizeof(float);
   if (smem > 40000) return NF_EUNSUPPORTED;
   fc_ce_kernel<<<N, 256, smem, g_nf_stream>>>(p, labels, N, D, K, Wf, bf, logits, dlogits, dp, lossn, status);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+__global__ void __launch_bounds__(256) count_equal_kernel(const int32_t* __restrict__ a, const int32_t* __restrict__ b, long long n,
+                                                          unsigned long long* __restrict__ count) {
+  unsigned c = 0;
+  for (long long i = blockIdx.x * 256LL + threadIdx.x; i < n; i += 256LL * gridDim.x) c += a[i] == b[i];
+  c = __reduce_add_sync(0xffffffffu, c);
+  if ((threadIdx.x & 31) == 0 && c) atomicAdd(count, (unsigned long long)c);   // integer sum: order-independent
+}
+
+int nf_ref_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count) {
+  const int blocks = (int)std::min<long long>((n + 255) / 256, 1184);
+  count_equal_kernel<<<blocks, 256, 0, g_nf_stream>>>(a, b, n, count);
   NF_LAUNCHED();
   return NF_OK;
 }

@@ -25,7 +25,7 @@ PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P
 EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_layer_workspace_bytes",
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
-           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
+           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
            "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_op_status", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
@@ -72,6 +72,7 @@ def lib():
         L.nf_layer_predict.argtypes = [vp, vp, C.c_int, vp, fp, ip]
         L.nf_layer_param_count.restype = C.c_longlong
         L.nf_layer_param_count.argtypes = [vp, C.c_int]
+        L.nf_count_equal.argtypes = [ip, ip, C.c_longlong, vp]
         L.nf_select_exit.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.c_int]
         L.nf_block_step.argtypes = [vp, vp, ip, C.c_float, fp, vp]
         L.nf_block_step_host.argtypes = [vp, vp, ip, C.c_float, fp, vp]
@@ -150,6 +151,11 @@ def nf_trace_read(slots: int = 1):
             if n.value:
                 out[(name, s)] = (ms.value, n.value)
     return out
+
+
+def nf_count_equal(a, b, count_out):
+    """count_out (device int64[1]) += number of equal entries of the device int32 tensors a and b."""
+    _check(lib().nf_count_equal(_ptr(a), _ptr(b), int(a.numel()), _ptr(count_out)), "nf_count_equal")
 
 
 def nf_select_exit(val_accuracy, params) -> int:

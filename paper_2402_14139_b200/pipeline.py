@@ -8,6 +8,10 @@ previous block otherwise) and stepped through all layers of the block with nf_bl
 block has finished, its output for every sample is written to the cache by nf_block_cache (forward
 only, running statistics) and becomes the next block's input set.  Earlier blocks are never run again.
 
+With a validation set, every trained layer is also evaluated as an exit point (nf_layer_predict on the
+validation activations that the earlier layers produced, nf_count_equal against the labels); the
+resulting (layer, accuracy, parameters) table goes through nf_select_exit.
+
     python -m paper_2402_14139_b200.pipeline --workload c5 --images 10000 --epochs 3
 """
 from __future__ import annotations
@@ -36,12 +40,35 @@ def build_layers(nf, wl, block_index, seed):
     return layers, nf.Block(layers)
 
 
-def train_blockwise(nf, torch, wl, data, labels, epochs=1, lr=0.01, seed=1, log=None):
-    """data: device tensor [K, H, W, C] of the first layer's dtype; labels: device int32 [K].
-    Returns a list of per-block records (batch size, steps, seconds, images/s, last losses)."""
+def evaluate_exits(nf, torch, layers, N, val_cur, val_labels):
+    """Run the validation activations through the layers of one trained block, each layer as an exit.
+    Returns ([correct count per layer], the block's output for the validation set)."""
+    V = val_cur.shape[0]
+    counts = torch.zeros(len(layers), dtype=torch.int64, device=val_cur.device)
+    pred = torch.empty(N, dtype=torch.int32, device=val_cur.device)
+    acts = [L.new_act() for L in layers]
+    last = layers[-1]
+    out = torch.empty((V, last.Ha, last.Wa, last.Cout), dtype=val_cur.dtype, device=val_cur.device)
+    for s in range(0, V, N):
+        cnt = min(N, V - s)
+        x = val_cur[s:s + cnt]
+        for li, L in enumerate(layers):
+            dst = out[s:s + cnt] if li == len(layers) - 1 else acts[li]
+            L.predict(x, pred, act_out=dst, count=cnt)
+            nf.nf_count_equal(pred[:cnt], val_labels[s:s + cnt], counts[li:li + 1])
+            x = dst
+    return counts.cpu().tolist(), out
+
+
+def train_blockwise(nf, torch, wl, data, labels, epochs=1, lr=0.01, seed=1, log=None, val=None):
+    """data: device tensor [K, H, W, C] of the first layer's dtype; labels: device int32 [K];
+    val: optional (device tensor [V, H, W, C], device int32 [V]) validation set.
+    Returns (per-block records, the last block's cached output) and, with val, also the exit report
+    dict(table=[(layer, accuracy, parameters)], selected=layer index)."""
     K = data.shape[0]
     report = []
     cur = data
+    val_cur, exits, main_params = (val[0] if val else None), [], 0
     for bi, (N, ls) in enumerate(wl["blocks"]):
         N = min(N, K)
         capped = dict(wl, blocks=[(N, l2) if i == bi else (n2, l2) for i, (n2, l2) in enumerate(wl["blocks"])])
@@ -75,12 +102,21 @@ def train_blockwise(nf, torch, wl, data, labels, epochs=1, lr=0.01, seed=1, log=
         rec = dict(block=bi, layers=len(ls), batch=N, steps=steps, train_s=round(t_train, 4), cache_s=round(t_cache, 4),
                    train_images_per_s=round(steps * N / max(t_train, 1e-9), 1), losses=[round(v, 4) for v in loss.cpu().tolist()])
         report.append(rec)
+        if val:
+            correct, val_cur = evaluate_exits(nf, torch, layers, N, val_cur, val[1])
+            for L, c in zip(layers, correct):       # exit at layer n: main paths of layers 1..n + the aux head of layer n
+                main_params += L.param_count(0)
+                exits.append((len(exits), c / val[0].shape[0], main_params + L.param_count(1)))
+            rec["exit_val_accuracy"] = [round(e[1], 4) for e in exits[-len(layers):]]
         if log:
             log(rec)
         block.close()
         for L in layers:
             L.close()
         cur = out
+    if val:
+        sel = nf.nf_select_exit([e[1] for e in exits], [e[2] for e in exits])
+        return report, cur, dict(table=exits, selected=sel)
     return report, cur
 
 
@@ -92,6 +128,7 @@ def main():
     ap.add_argument("--images", type=int, default=10000)
     ap.add_argument("--epochs", type=int, default=3)
     ap.add_argument("--lr", type=float, default=0.01)
+    ap.add_argument("--val-images", type=int, default=0, help="evaluate every layer as an exit on this many held-out images")
     args = ap.parse_args()
     nf.lib()
     nf.nf_set_stream(torch.cuda.current_stream())
@@ -102,9 +139,16 @@ def main():
     tdt = torch.float32 if wl["dtype"] == "f32" else torch.bfloat16
     data = torch.randn((args.images, H, W, C), generator=g, device="cuda", dtype=torch.float32).to(tdt)
     labels = torch.randint(0, wl["classes"], (args.images,), generator=g, device="cuda", dtype=torch.int32)
+    val = None
+    if args.val_images:
+        val = (torch.randn((args.val_images, H, W, C), generator=g, device="cuda", dtype=torch.float32).to(tdt),
+               torch.randint(0, wl["classes"], (args.val_images,), generator=g, device="cuda", dtype=torch.int32))
     t0 = time.perf_counter()
-    report, _ = train_blockwise(nf, torch, wl, data, labels, epochs=args.epochs, lr=args.lr, log=lambda r: print(json.dumps(r), flush=True))
+    res = train_blockwise(nf, torch, wl, data, labels, epochs=args.epochs, lr=args.lr, log=lambda r: print(json.dumps(r), flush=True),
+                          val=val)
     wall = time.perf_counter() - t0
+    if val:
+        print(json.dumps(dict(exit_table=[(l, round(a, 4), p) for l, a, p in res[2]["table"]], selected_exit=res[2]["selected"])))
     n_layers = sum(len(ls) for _, ls in wl["blocks"])
     print(json.dumps(dict(workload=wl["name"], images=args.images, epochs=args.epochs, layers=n_layers, wall_s=round(wall, 3),
                           images_per_s_whole_pass=round(args.images * args.epochs / wall, 1))))

@@ -33,3 +33,34 @@ def test_blockwise_pass_runs_and_learns_a_learnable_task():
     assert out.shape == (K, 8, 8, 128) and torch.isfinite(out.float()).all()
     assert all(np.isfinite(r["losses"]).all() for r in report)
     assert report[0]["losses"][-1] < 0.7 * np.log(4)       # the local loss of block 1's last layer fell well below chance
+
+
+def test_exit_evaluation_over_the_blockwise_pass():
+    """Every trained layer is evaluated as an exit on held-out samples of the same learnable task: accuracies are
+    counts over the validation set, parameter totals grow with depth, the selected exit follows the rule, and the
+    deepest exits classify the task they were trained on."""
+    import torch
+    from oracle import nfo
+    from paper_2402_14139_b200 import nf
+    nf.lib()
+    nf.nf_set_stream(None)
+
+    def make(K, tid):
+        x = synth.normal(5, tid, (K, 16, 16, 3))
+        lab = (np.arange(K) % 4).astype(np.int32)
+        for k in range(K):
+            u, v = lab[k] // 2, lab[k] % 2
+            x[k, u * 8:(u + 1) * 8, v * 8:(v + 1) * 8, :] += 2.0
+        return torch.from_numpy(synth.round_bf16(x)).cuda().to(torch.bfloat16), torch.from_numpy(lab).cuda()
+
+    data, labels = make(24, 1)
+    val = make(20, 2)                         # 20 is not a multiple of either block's batch size: ragged last chunk
+    report, out, ex = pipeline.train_blockwise(nf, torch, _wl(), data, labels, epochs=25, lr=0.05, seed=3, val=val)
+    table = ex["table"]
+    assert [t[0] for t in table] == [0, 1, 2]
+    assert all(abs(t[1] * 20 - round(t[1] * 20)) < 1e-9 and 0.0 <= t[1] <= 1.0 for t in table)
+    main = [9 * 3 * 64 + 128, 9 * 64 * 64 + 128, 9 * 64 * 128 + 256]
+    aux = [9 * 64 * 8 + 8 + 4 * (32 + 1), 9 * 64 * 8 + 8 + 4 * (32 + 1), 9 * 128 * 16 + 16 + 4 * (64 + 1)]
+    assert [t[2] for t in table] == [main[0] + aux[0], main[0] + main[1] + aux[1], sum(main) + aux[2]]
+    assert ex["selected"] == nfo.select_exit([t[1] for t in table], [t[2] for t in table])
+    assert max(t[1] for t in table) >= 0.9
