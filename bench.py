@@ -31,7 +31,6 @@ FALLBACK_PEAKS = dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=
 # from one ncu capture of the batch-24 case (profiles/ncu_full_c4s_conv_bn_kernels.md); every tensor is streamed
 # once, so traffic grows in proportion to the batch.  Valid for the kernels as captured; None elsewhere.
 NCU_TRAFFIC_C4_BYTES_PER_IMAGE = dict(conv_fwd=(154.27 + 106.01) * 1e6 / 24, wgrad=(324.01 + 3.51) * 1e6 / 24,
-                                      bn_bwd=(308.30 + 3.82 + 308.34 + 123.60) * 1e6 / 24,
                                       bn_fwd=(154.15 + 109.90) * 1e6 / 24)
 
 
@@ -117,20 +116,24 @@ def build_block(nf, torch, wl, bi, seed, host_io):
 
 
 def op_model(l, N, classes, es, fam):
-    """Algorithmic work of each traced op of one layer step: ('tensor'|'alu', flops) or ('hbm', bytes)."""
+    """Algorithmic work of each traced op of one layer step: kind -> ('tensor'|'alu', flops, bytes) for the
+    contractions (the caller takes whichever of the two rooflines binds) or ('hbm', None, bytes)."""
     from paper_2402_14139_b200 import workloads as W
     fl = W.step_flops(l, N)
     Ho, Wo = (l["H"] - 1) // l["stride"] + 1, (l["W"] - 1) // l["stride"] + 1
     Ha, Wa = W.out_hw(l)
+    nx = N * l["H"] * l["W"] * l["Cin"]
     ny, na, nh = N * Ho * Wo * l["Cout"], N * Ha * Wa * l["Cout"], N * Ha * Wa * l["F"]
     nparam = 9 * l["Cin"] * l["Cout"] + 2 * l["Cout"] + 9 * l["Cout"] * l["F"] + l["F"] + classes * (4 * l["F"] + 1)
     tc = lambda k: "tensor" if fam[k] == "tcgen05" else "alu"
-    return dict(conv_fwd=(tc(0), fl["conv_fwd"]), wgrad=(tc(1), fl["wgrad"]), aux_fwd=(tc(2), fl["aux_fwd"]),
-                aux_bwd=(tc(3), fl["aux_bwd"]),
-                bn_fwd=("hbm", es * (ny + na)),            # read y, write a
-                bn_bwd=("hbm", es * (2 * ny + na)),        # read y and da, write dy
-                head=("hbm", es * nh + 4 * N * (8 * l["F"] + 2 * classes)),
-                sgd=("hbm", 18 * nparam))                  # theta, v read+write (fp32), g read, bf16 copy write
+    return dict(conv_fwd=(tc(0), fl["conv_fwd"], es * (nx + ny)),          # read x, write y
+                wgrad=(tc(1), fl["wgrad"], es * (nx + ny)),                # read x and dy
+                aux_fwd=(tc(2), fl["aux_fwd"], es * (na + nh)),            # read a, write h
+                aux_bwd=(tc(3), fl["aux_bwd"], es * (4 * nh + 2 * na)),    # h -> dh; a, dh -> gWa; dh -> da
+                bn_fwd=("hbm", None, es * (ny + na)),                      # read y, write a
+                bn_bwd=("hbm", None, es * (2 * ny + na)),                  # read y and da, write dy
+                head=("hbm", None, es * nh + 4 * N * (8 * l["F"] + 2 * classes)),
+                sgd=("hbm", None, 18 * nparam))                            # theta, v read+write (fp32), g read, bf16 copy write
 
 
 def run_ours(args, rank, world):
@@ -216,12 +219,15 @@ def run_ours(args, rank, world):
     kernels, best = [], None
     tot_ms = sum(v[0] for v in trace.values())
     for (op, slot), (tms, cnt) in sorted(trace.items(), key=lambda kv: -kv[1][0]):
-        kind, work = op_model(ls[slot], N, wl["classes"], es, fam[slot])[op]
+        kind, flops, nbytes = op_model(ls[slot], N, wl["classes"], es, fam[slot])[op]
         per = tms / cnt
+        # a contraction with few filters moves more bytes per flop than the machine balance: its bound is HBM
+        if kind != "hbm" and nbytes / (peaks["hbm_gbs"] * 1e9) > flops / (peaks["bf16_tflops_sustained"] * 1e12):
+            kind = "hbm"
         if kind == "hbm":
-            ach, peak, unit = work / per / 1e6, peaks["hbm_gbs"], "GB/s"
+            ach, peak, unit = nbytes / per / 1e6, peaks["hbm_gbs"], "GB/s"
         else:
-            ach, peak, unit = work / per / 1e9, peaks["bf16_tflops_sustained"], "TFLOP/s"
+            ach, peak, unit = flops / per / 1e9, peaks["bf16_tflops_sustained"], "TFLOP/s"
         rec = dict(op=op, layer=slot, bound=kind, ms_per_launch=round(per, 4), share=round(tms / tot_ms, 4),
                    achieved=round(ach, 2), peak=peak, unit=unit, frac=round(ach / peak, 4))
         kernels.append(rec)

@@ -382,16 +382,21 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
     NF_TRY(nf_ref_sum_partials(L->red, nb, F, 0, g + L->off[NF_P_BA]));
   }
   // gradient at the aux input
+  int bn_nb = 0;  // > 0: the input-gradient kernel has already left the BatchNorm-backward partial sums in L->red
   if (L->fam[3]) {
-    NF_TRY(nf_tc_aux_dgrad(L));
+    NF_TRY(nf_tc_aux_dgrad(L, &bn_nb));
   } else {
     NF_TRY(nf_ref_conv(dt, L->dh, N, Ha, Wa, F, Wx, (long)F * Co, 1, Co, 1, nullptr, 0, 1, Co, L->da));
   }
   trace_end();
   // back through pool / ReLU / BatchNorm
   trace_begin(5);
-  NF_TRY(nf_ref_bn_bwd_reduce(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->red,
-                              L->red_floats, &nb));
+  if (bn_nb) {
+    nb = bn_nb;
+  } else {
+    NF_TRY(nf_ref_bn_bwd_reduce(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->red,
+                                L->red_floats, &nb));
+  }
   NF_TRY(nf_ref_bn_bwd_finalize(L->red, nb, Co, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
   NF_TRY(nf_ref_bn_bwd_apply(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->sdz, L->sdzx,
                              M, L->dy));

@@ -342,8 +342,9 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 // same warp.  14 x 8 output pixels per tile; needs W % 14 == 0 and H % 8 == 0.
 struct FoldParams {
   int N, H, W, Cout, kchunks, n_tiles, tiles_w, tiles_h, total_tiles, stages, stats;
-  float* red;         // EPI 0: [grid * 4][2][64]
+  float* red;         // EPI 0, stats != 0: [grid / n_tiles * 8][2][Cout]
   int32_t* status;
+  const float *bn_scale, *bn_shift, *bn_mu, *bn_invstd;  // stats == 2
   const float* bias;  // EPI 1
   bf16* out;          // EPI 1: [N][H][W][Cout]
 };
@@ -353,13 +354,17 @@ struct FoldParams {
 // EPI : 0 = y in bf16 through a TMA store + BatchNorm partial sums (G = 64, Cout = 64);
 //       1 = bias + ReLU, F channels written straight from registers (aux conv forward).
 // Cin = 64 * kchunks; all 9 * kchunks weight tiles stay resident in shared memory.
+// stats (EPI 0): 1 = per-channel sums of (y, y^2) of the stored values (BatchNorm forward statistics);
+//       2 = the output is the gradient da at a BatchNorm+ReLU output of the same shape: per-channel sums of
+//       (dz, dz * xhat) with dz = da * 1[y2*scale+shift > 0], xhat = (y2 - mu) * invstd, where the tile of the
+//       pre-normalisation values y2 is fetched through tm_y2 (BatchNorm backward reduction fused into the producer of da).
 // KC / MIR: KC = channels of the activation box (64; 16 or 32 for the aux input gradient whose input dh has F
 // channels), MIR = 1 reads the weights [tap][f][c] MN-major with both taps mirrored (input-gradient convolution;
 // the CTA's 64-channel output tile is blockIdx.x % n_tiles).
 template <int G, int EPI, int KC = 64, int MIR = 0>
 __global__ void __launch_bounds__(kFoldThreads, 1)
 conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-                     const __grid_constant__ CUtensorMap tm_y, const FoldParams p) {
+                     const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_y2, const FoldParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int kARow = KC * 2;               // bytes of one pixel of the activation box
@@ -369,13 +374,16 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   const int w_bytes = 3 * p.kchunks * kWTile; // [chunk][kh][kw*G + co][64 ci]
   uint8_t* wres = smem + (size_t)p.stages * kABytes;
   uint8_t* stg = wres + w_bytes;              // EPI 0: 112 output pixels x 128 bytes
-  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (EPI == 0 ? 2 * 16384 : 0));  // one staging tile per epilogue group
+  uint8_t* ybuf = stg + 2 * 16384;            // EPI 0, stats 2: two tiles of y2 per epilogue group
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (EPI == 0 ? (p.stats == 2 ? 6 : 2) * 16384 : 0));  // one staging tile per epilogue group
   uint64_t* full = bars;
   uint64_t* empty = bars + kMaxStages;
   uint64_t* tfull = bars + 2 * kMaxStages;
   uint64_t* tempty = tfull + 2;
   uint64_t* wfull = tempty + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wfull + 1);
+  uint64_t* yfull = wfull + 1;
+  uint64_t* yempty = yfull + 4;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(yempty + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);  // [2], one per epilogue group
   constexpr uint32_t kAccStride = G == 64 ? 256 : 128;  // columns between the two accumulators
@@ -391,12 +399,17 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       ptx::mbar_init(&tfull[a], 1);
       ptx::mbar_init(&tempty[a], 128);
     }
+    for (int a = 0; a < 4; ++a) {
+      ptx::mbar_init(&yfull[a], 1);
+      ptx::mbar_init(&yempty[a], 128);
+    }
     ptx::mbar_init(wfull, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tmap(&tm_x);
     ptx::prefetch_tmap(&tm_w);
     ptx::prefetch_tmap(&tm_y);
+    ptx::prefetch_tmap(&tm_y2);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, kTmemCols);
@@ -416,9 +429,9 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           ptx::tma_load_4d(wres + (ck * 3 + kh) * kWTile, &tm_w, wfull, MIR ? (int)(blockIdx.x % p.n_tiles) * 64 : ck * 64, 0, 0, kh);
     }
     __syncwarp();
-    uint32_t it = 0;
+    uint32_t it = 0, tl = 0;
     bool ok = true;
-    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x) {
+    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++tl) {
       const int m = t / p.n_tiles;
       const int w0 = (m % p.tiles_w) * 14, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
       for (int ck = 0; ck < p.kchunks; ++ck, ++it) {
@@ -430,6 +443,17 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           ptx::tma_load_4d(smem + (size_t)s * kABytes, &tm_x, &full[s], ck * KC, w0 - 1, h0 - 1, n);
         }
         __syncwarp();
+      }
+      if constexpr (EPI == 0) {
+        if (ok && p.stats == 2) {  // the y2 tile of this output tile, for the epilogue group that owns it
+          const uint32_t k2 = tl >> 1, slot = (tl & 1) * 2 + (k2 & 1);
+          if (!__all_sync(0xffffffffu, ptx::mbar_wait(&yempty[slot], ((k2 >> 1) & 1) ^ 1, abort_flag))) break;
+          if (lane == 0) {
+            ptx::mbar_expect_tx(&yfull[slot], 14 * 8 * 128);
+            ptx::tma_load_4d(ybuf + slot * 16384, &tm_y2, &yfull[slot], (t % p.n_tiles) * 64, w0, h0, n);
+          }
+          __syncwarp();
+        }
       }
     }
   } else if (warp == 1) {
@@ -477,8 +501,18 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     const int we = r & 15, hh = r >> 4;
     const bool valid = we >= 1 && we <= 14;
     const int orow = (we - 1) + 14 * hh;     // row of the output staging tile
-    const int sc = et & 63, shalf = et >> 6; // stats: channel, and which 56 of the 112 rows
-    float ssum = 0.f, ssq = 0.f;
+    // statistics: a thread owns 8 channels (one 16-byte chunk of a pixel row) and the 7 rows rg, rg+16, ...
+    const int schunk = et & 7, srg = et >> 3;
+    float s1[8], s2[8], bsc[8], bsh[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s1[i] = s2[i] = bsc[i] = bsh[i] = 0.f;
+    if constexpr (EPI == 0) {
+      if (p.stats == 2) {
+        const int ch = (int)(blockIdx.x % p.n_tiles) * 64 + schunk * 8;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { bsc[i] = p.bn_scale[ch + i]; bsh[i] = p.bn_shift[ch + i]; }
+      }
+    }
     uint32_t tl = grp;
     for (long t = blockIdx.x + (long)grp * gridDim.x; t < p.total_tiles; t += 2L * gridDim.x, tl += 2) {
       const int nt = (int)(t % p.n_tiles);
@@ -543,25 +577,71 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           ptx::tma_store_4d(&tm_y, stg_g, nt * 64, w0, h0, n);
           ptx::tma_store_commit();
         }
-        if (p.stats) {
-          const uint8_t* col = stg_g + (sc & 7) * 2;
-          const int u = sc >> 3;
-#pragma unroll 8
-          for (int rr = 0; rr < 56; ++rr) {
-            const int row = shalf * 56 + rr;
-            const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(col + row * 128 + ((u ^ (row & 7)) * 16)));
-            ssum += v;
-            ssq = fmaf(v, v, ssq);
+        if (p.stats == 2) {
+          // sums of dz and dz*y2 (the caller of the kernel gets sum dz*xhat = invstd * (sum dz*y2 - mu * sum dz))
+          const uint32_t k2 = tl >> 1, slot = grp * 2 + (k2 & 1);
+          ptx::mbar_wait(&yfull[slot], (k2 >> 1) & 1, abort_flag);
+          const uint8_t* yb = ybuf + slot * 16384;
+#pragma unroll
+          for (int rr = 0; rr < 7; ++rr) {
+            const int row = srg + 16 * rr;
+            const int off = row * 128 + ((schunk ^ (row & 7)) * 16);
+            const uint4 dq = *reinterpret_cast<const uint4*>(stg_g + off);
+            const uint4 yq = *reinterpret_cast<const uint4*>(yb + off);
+            const uint32_t dw[4] = {dq.x, dq.y, dq.z, dq.w}, yw[4] = {yq.x, yq.y, yq.z, yq.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float d0 = __uint_as_float(dw[e] << 16), d1 = __uint_as_float(dw[e] & 0xffff0000u);
+              const float y0 = __uint_as_float(yw[e] << 16), y1 = __uint_as_float(yw[e] & 0xffff0000u);
+              const float z0 = fmaf(y0, bsc[2 * e], bsh[2 * e]) > 0.f ? d0 : 0.f;
+              const float z1 = fmaf(y1, bsc[2 * e + 1], bsh[2 * e + 1]) > 0.f ? d1 : 0.f;
+              s1[2 * e] += z0;
+              s1[2 * e + 1] += z1;
+              s2[2 * e] = fmaf(z0, y0, s2[2 * e]);
+              s2[2 * e + 1] = fmaf(z1, y1, s2[2 * e + 1]);
+            }
+          }
+          ptx::mbar_arrive(&yempty[slot]);
+        } else if (p.stats) {
+#pragma unroll
+          for (int rr = 0; rr < 7; ++rr) {
+            const int row = srg + 16 * rr;
+            const uint4 vq = *reinterpret_cast<const uint4*>(stg_g + row * 128 + ((schunk ^ (row & 7)) * 16));
+            const uint32_t vw[4] = {vq.x, vq.y, vq.z, vq.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float v0 = __uint_as_float(vw[e] << 16), v1 = __uint_as_float(vw[e] & 0xffff0000u);
+              s1[2 * e] += v0;
+              s1[2 * e + 1] += v1;
+              s2[2 * e] = fmaf(v0, v0, s2[2 * e]);
+              s2[2 * e + 1] = fmaf(v1, v1, s2[2 * e + 1]);
+            }
           }
         }
       }
     }
     if constexpr (EPI == 0) {
       if (et == 0) ptx::tma_store_wait_all();
-      if (p.stats) {
-        const size_t b = (size_t)blockIdx.x * 4 + grp * 2 + shalf;
-        p.red[(b * 2 + 0) * 64 + sc] = ssum;
-        p.red[(b * 2 + 1) * 64 + sc] = ssq;
+      if (p.stats) {  // one partial per warp: lanes with the same chunk (lane & 7) are added in a fixed order
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 8);
+          s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], 8);
+          s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 16);
+          s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], 16);
+        }
+        if (lane < 8) {
+          const size_t b = (size_t)(blockIdx.x / p.n_tiles) * 8 + grp * 4 + lg;
+          const int ch = (int)(blockIdx.x % p.n_tiles) * 64 + lane * 8;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            float second = s2[i];
+            if (p.stats == 2)
+              second = (float)((double)p.bn_invstd[ch + i] * ((double)s2[i] - (double)p.bn_mu[ch + i] * (double)s1[i]));
+            p.red[(b * 2 + 0) * p.Cout + ch + i] = s1[i];
+            p.red[(b * 2 + 1) * p.Cout + ch + i] = second;
+          }
+        }
       }
     }
   }
@@ -1013,22 +1093,29 @@ bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride) {
 }
 
 template <int G, int EPI, int KC = 64, int MIR = 0>
-int launch_fold(int grid, size_t smem, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const FoldParams& p) {
+int launch_fold(int grid, size_t smem, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const CUtensorMap& my2,
+                const FoldParams& p) {
   static bool attr_done = false;
   if (!attr_done) {
     NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel<G, EPI, KC, MIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
   }
-  conv_fwd_fold_kernel<G, EPI, KC, MIR><<<grid, kFoldThreads, smem, g_nf_stream>>>(mx, mw, my, p);
+  conv_fwd_fold_kernel<G, EPI, KC, MIR><<<grid, kFoldThreads, smem, g_nf_stream>>>(mx, mw, my, my2, p);
   NF_LAUNCHED();
   return NF_OK;
 }
 
+// BatchNorm-backward inputs of the fused reduction (stats 2): y2 has the shape of the output
+struct BnBwdIn {
+  const void* y2;
+  const float *scale, *shift, *mu, *invstd;
+};
+
 int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
-             size_t red_floats, int32_t* status, int* nb, int epi, const float* bias) {
+             size_t red_floats, int32_t* status, int* nb, int epi, const float* bias, const BnBwdIn* bn = nullptr) {
   const int G = fold_group(Cout, epi);
   const int KC = epi == 2 ? (Cin <= 16 ? 16 : 32) : 64;
-  CUtensorMap mx, mw, my;
+  CUtensorMap mx, mw, my, my2;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
   const uint32_t bx[4] = {(uint32_t)KC, 16, 10, 1};
   // forward: weights [kh][kw][Cout][Cin], box = G rows of co x 64 ci for the three kw of one kh;
@@ -1045,13 +1132,19 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   } else {
     my = mx;
   }
+  my2 = my;
+  if (stats == 2) {
+    if (epi != 2 || !bn) return NF_EINVAL;
+    if ((rc = make_map4(&my2, bn->y2, dy, by)) != NF_OK) return rc;
+  }
   FoldParams p{};
+  if (bn) { p.bn_scale = bn->scale; p.bn_shift = bn->shift; p.bn_mu = bn->mu; p.bn_invstd = bn->invstd; }
   p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = epi == 2 ? 1 : Cin / 64; p.n_tiles = epi == 2 ? Cout / 64 : 1;
   p.tiles_w = W / 14; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
   p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
   const size_t a_bytes = (size_t)10 * 16 * KC * 2;
   const size_t wbytes = epi == 2 ? (size_t)9 * KC * 128 : (size_t)9 * p.kchunks * G * 128;
-  const size_t fixed = wbytes + (epi != 1 ? 2 * 16384 : 0) + 1024 + 1024;
+  const size_t fixed = wbytes + (epi != 1 ? (stats == 2 ? 6 : 2) * 16384 : 0) + 1024 + 1024;
   int st = (int)((232448 - fixed) / a_bytes);
   if (st > kMaxStages) st = kMaxStages;
   p.stages = st;
@@ -1061,15 +1154,15 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   if (grid < p.n_tiles) grid = p.n_tiles;
   if (grid > p.total_tiles) grid = p.total_tiles;
   if (stats) {
-    const size_t need = (size_t)grid * 4 * 2 * 64;
+    const size_t need = (size_t)(grid / p.n_tiles) * 8 * 2 * Cout;  // every CTA writes all of its 8 partials
     if (need > red_floats) return NF_ENOWS;
-    NF_CUDA(cudaMemsetAsync(red, 0, need * sizeof(float), g_nf_stream));
-    *nb = grid * 4;
+    *nb = grid / p.n_tiles * 8;
   }
-  if (epi == 0) return launch_fold<64, 0>(grid, smem, mx, mw, my, p);
-  if (epi == 2) return KC == 16 ? launch_fold<64, 0, 16, 1>(grid, smem, mx, mw, my, p) : launch_fold<64, 0, 32, 1>(grid, smem, mx, mw, my, p);
-  return G == 16 ? launch_fold<16, 1>(grid, smem, mx, mw, my, p)
-                 : G == 32 ? launch_fold<32, 1>(grid, smem, mx, mw, my, p) : launch_fold<64, 1>(grid, smem, mx, mw, my, p);
+  if (epi == 0) return launch_fold<64, 0>(grid, smem, mx, mw, my, my2, p);
+  if (epi == 2)
+    return KC == 16 ? launch_fold<64, 0, 16, 1>(grid, smem, mx, mw, my, my2, p) : launch_fold<64, 0, 32, 1>(grid, smem, mx, mw, my, my2, p);
+  return G == 16 ? launch_fold<16, 1>(grid, smem, mx, mw, my, my2, p)
+                 : G == 32 ? launch_fold<32, 1>(grid, smem, mx, mw, my, my2, p) : launch_fold<64, 1>(grid, smem, mx, mw, my, my2, p);
 }
 
 // epi 0: y through TMA + optional statistics.  epi 1: out = ReLU(conv + bias) written directly (y unused).
@@ -1248,9 +1341,12 @@ size_t nf_tc_scratch_floats(const nf_layer* L) {
 }
 
 size_t nf_tc_red_floats(const nf_layer* L) {
-  if (!L->fam[0]) return 0;
+  size_t need = 0;
+  if (L->fam[3]) need = (size_t)sm_count() * 8 * 2 * L->Cout;  // input-gradient kernel with the fused BatchNorm-backward sums
+  if (!L->fam[0]) return need;
   const TcPlan pl = plan_fwd(L->Ho, L->Wo, L->Cin, L->Cout, L->o.N, 0, L->o.stride);
-  return (size_t)sm_count() * (pl.parts < 4 ? 4 : pl.parts) * 2 * L->Cout;  // the folded kernel writes 4 partials per CTA
+  const size_t fwd = (size_t)sm_count() * (pl.parts < 8 ? 8 : pl.parts) * 2 * L->Cout;  // the folded kernel writes 8 partials per CTA
+  return fwd > need ? fwd : need;
 }
 
 int nf_tc_prepare(nf_layer*) { return NF_OK; }
@@ -1277,8 +1373,16 @@ int nf_tc_wgrad(nf_layer* L, const void* x) {
                    L->status, 0, L->o.stride);
 }
 
-int nf_tc_aux_dgrad(nf_layer* L) {
+int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb) {
   int nb = 0;
+  *bn_nb = 0;
+  // without a pool da has the shape of y: the folded kernel also reduces (dz, dz*xhat) per channel while it holds the tile
+  if (!L->o.maxpool && fold_ok(L->Ha, L->Wa, L->F, L->Cout, 2, 1) &&
+      (size_t)(sm_count() / (L->Cout / 64)) * 8 * 2 * L->Cout <= L->red_floats) {
+    const BnBwdIn bn{L->y, L->scale, L->shift, L->mu, L->invstd};
+    return run_fold(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->shadow + L->off[NF_P_WA], L->da, 2, L->red, L->red_floats,
+                    L->status, bn_nb, 2, nullptr, &bn);
+  }
   return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->shadow + L->off[NF_P_WA], L->da, 0, nullptr, 0, L->status,
                  &nb, 2);
 }

@@ -28,5 +28,7 @@ int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int C
 int nf_tc_aux_fwd(nf_layer* L, const void* a, int count);
 // Aux conv weight gradient on tensor cores: grad(Wa) = wgrad(a, L->dh).
 int nf_tc_aux_wgrad(nf_layer* L, const void* a);
-// Aux conv input gradient on tensor cores: L->da = dgrad(L->dh, Wa) in bf16.
-int nf_tc_aux_dgrad(nf_layer* L);
+// Aux conv input gradient on tensor cores: L->da = dgrad(L->dh, Wa) in bf16.  Where the kernel can also reduce
+// the BatchNorm-backward sums (no pool, folded-tap shape) it leaves *bn_nb > 0 partial blocks in L->red
+// ([block][2][Cout]: sum dz, sum dz*xhat); otherwise *bn_nb = 0.
+int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb);
