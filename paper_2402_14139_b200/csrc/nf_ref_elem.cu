@@ -97,11 +97,26 @@ __device__ __forceinline__ void reduce_partials32(const float* __restrict__ red,
   __shared__ double sm[2][32][33];
   const int c = blockIdx.x * 32 + threadIdx.x;
   double a = 0.0, b = 0.0;
-  if (c < C)
-    for (int k = threadIdx.y; k < nb; k += 32) {
+  if (c < C) {
+    int k = threadIdx.y;
+    for (; k + 7 * 32 < nb; k += 8 * 32) {  // eight independent pairs of loads in flight, added in index order
+      float u[8], v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        u[j] = red[((size_t)(k + 32 * j) * 2 + 0) * C + c];
+        v[j] = red[((size_t)(k + 32 * j) * 2 + 1) * C + c];
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        a += (double)u[j];
+        b += (double)v[j];
+      }
+    }
+    for (; k < nb; k += 32) {
       a += (double)red[((size_t)k * 2 + 0) * C + c];
       b += (double)red[((size_t)k * 2 + 1) * C + c];
     }
+  }
   sm[0][threadIdx.y][threadIdx.x] = a;
   sm[1][threadIdx.y][threadIdx.x] = b;
   __syncthreads();
@@ -258,10 +273,38 @@ __global__ void __launch_bounds__(256) fc_ce_kernel(const float* __restrict__ p,
     dlogits[(size_t)n * K + k] = g;
   }
   __syncthreads();
-  for (int d = t; d < D; d += 256) {
+  // dp[d] = sum_k g[k] Wf[k][d]: the classes are cut into G contiguous ranges (G = 256 / D lanes per d when D <= 128),
+  // every range is summed in index order and the G range sums are added in range order
+  const int G = D <= 128 ? 256 / D : 1;
+  if (G > 1) {
+    const int d = t % D, kg = t / D;
     float s = 0.f;
-    for (int k = 0; k < K; ++k) s = fmaf(ls[k], Wf[(size_t)k * D + d], s);
-    dp[(size_t)n * D + d] = s;
+    if (kg < G) {
+      const int per = (K + G - 1) / G, k0 = kg * per, k1 = min(K, k0 + per);
+      int k = k0;
+      for (; k + 3 < k1; k += 4) {
+        const float w0 = Wf[(size_t)k * D + d], w1 = Wf[(size_t)(k + 1) * D + d], w2 = Wf[(size_t)(k + 2) * D + d],
+                    w3 = Wf[(size_t)(k + 3) * D + d];
+        s = fmaf(ls[k], w0, s);
+        s = fmaf(ls[k + 1], w1, s);
+        s = fmaf(ls[k + 2], w2, s);
+        s = fmaf(ls[k + 3], w3, s);
+      }
+      for (; k < k1; ++k) s = fmaf(ls[k], Wf[(size_t)k * D + d], s);
+    }
+    red[t] = s;
+    __syncthreads();
+    if (t < D) {
+      float tot = 0.f;
+      for (int g = 0; g < G; ++g) tot += red[g * D + t];
+      dp[(size_t)n * D + t] = tot;
+    }
+  } else {
+    for (int d = t; d < D; d += 256) {
+      float s = 0.f;
+      for (int k = 0; k < K; ++k) s = fmaf(ls[k], Wf[(size_t)k * D + d], s);
+      dp[(size_t)n * D + d] = s;
+    }
   }
 }
 
@@ -701,12 +744,12 @@ __global__ void __launch_bounds__(256) dh_vec_kernel(const uint4* __restrict__ h
 #pragma unroll
   for (int i = 0; i < 8; ++i) a[i] = 0.f;
   const size_t p0 = P * blockIdx.x / gridDim.x, p1 = P * (blockIdx.x + 1) / gridDim.x;
-  for (size_t p = p0 + pl; p < p1; p += planes) {
+  auto one = [&](size_t p, const uint4 hq) {
     const int j = (int)(p % Wa), i = (int)((p / Wa) % Ha);
     const size_t n = p / ((size_t)Wa * Ha);
     const int bin = (i >= Ha / 2 ? 2 : 0) + (j >= Wa / 2 ? 1 : 0);
     float hv[8], o[8];
-    unpack8(__ldg(h + p * F8 + g), hv);
+    unpack8(hq, hv);
     const float* d = dp + n * 4 * F + (size_t)(g * 8) * 4 + bin;
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
@@ -718,7 +761,16 @@ __global__ void __launch_bounds__(256) dh_vec_kernel(const uint4* __restrict__ h
     unpack8(packed, r);  // the bias gradient sums the values as stored
 #pragma unroll
     for (int e = 0; e < 8; ++e) a[e] += r[e];
+  };
+  size_t p = p0 + pl;
+  for (; p + 3 * (size_t)planes < p1; p += 4 * (size_t)planes) {  // four loads in flight, handled in index order
+    uint4 q[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) q[u] = __ldg(h + (p + (size_t)u * planes) * F8 + g);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) one(p + (size_t)u * planes, q[u]);
   }
+  for (; p < p1; p += planes) one(p, __ldg(h + p * F8 + g));
 #pragma unroll
   for (int e = 0; e < 8; ++e) sm[e][threadIdx.x] = a[e];
   __syncthreads();
@@ -743,10 +795,26 @@ __global__ void __launch_bounds__(256) avgpool_part_vec_kernel(const uint4* __re
   float a[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) a[i] = 0.f;
-  for (int k = k0 + pl; k < k1; k += planes) {
-    const int i = i0 + k / bw, j = j0 + k % bw;
+  const uint4* hn = h + (size_t)n * Ha * Wa * F8 + g;
+  int k = k0 + pl;
+  for (; k + 3 * planes < k1; k += 4 * planes) {  // four loads in flight, added in index order
+    uint4 q[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int kk = k + u * planes;
+      q[u] = __ldg(hn + ((size_t)(i0 + kk / bw) * Wa + j0 + kk % bw) * F8);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      float v[8];
+      unpack8(q[u], v);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) a[e] += v[e];
+    }
+  }
+  for (; k < k1; k += planes) {
     float v[8];
-    unpack8(__ldg(h + (((size_t)n * Ha + i) * Wa + j) * F8 + g), v);
+    unpack8(__ldg(hn + ((size_t)(i0 + k / bw) * Wa + j0 + k % bw) * F8), v);
 #pragma unroll
     for (int e = 0; e < 8; ++e) a[e] += v[e];
   }

@@ -963,12 +963,31 @@ conv_wgrad_kw_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   }
 }
 
-__global__ void sum_parts_kernel(const float* __restrict__ part, int splits, size_t n, float* __restrict__ out) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
+__global__ void __launch_bounds__(256) sum_parts_kernel(const float* __restrict__ part, int splits, size_t n, float* __restrict__ out) {
+  // 32 consecutive elements x 8 lanes over the splits; each lane adds its splits in index order, lane sums are added in lane order
+  __shared__ float sm[8][33];
+  const size_t i = (size_t)blockIdx.x * 32 + threadIdx.x;
   float s = 0.f;
-  for (int k = 0; k < splits; ++k) s += part[(size_t)k * n + i];
-  out[i] = s;
+  if (i < n) {
+    int k = threadIdx.y;
+    for (; k + 3 * 8 < splits; k += 4 * 8) {
+      const float a = part[(size_t)k * n + i], b = part[(size_t)(k + 8) * n + i], c = part[(size_t)(k + 16) * n + i],
+                  d = part[(size_t)(k + 24) * n + i];
+      s += a;
+      s += b;
+      s += c;
+      s += d;
+    }
+    for (; k < splits; k += 8) s += part[(size_t)k * n + i];
+  }
+  sm[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0 && i < n) {
+    float t = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) t += sm[j][threadIdx.x];
+    out[i] = t;
+  }
 }
 
 // ---------------------------------------------------------------- host side
@@ -1318,7 +1337,7 @@ int run_wgrad(int N, int Hin, int Win, int Cin, int Cout, const void* x, const v
                      : pl.NB == 32 ? launch_wgrad_kw<32>(pl, mx, mg, p) : launch_wgrad_kw<16>(pl, mx, mg, p);
   if (rc != NF_OK) return rc;
   const size_t n = (size_t)9 * Cout * Cin;
-  sum_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, g_nf_stream>>>(part, pl.splits, n, dw);
+  sum_parts_kernel<<<(unsigned)((n + 31) / 32), dim3(32, 8), 0, g_nf_stream>>>(part, pl.splits, n, dw);
   NF_LAUNCHED();
   return NF_OK;
 }
