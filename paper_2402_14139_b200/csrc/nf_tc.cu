@@ -514,10 +514,11 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       }
     }
     uint32_t tl = grp;
-    for (long t = blockIdx.x + (long)grp * gridDim.x; t < p.total_tiles; t += 2L * gridDim.x, tl += 2) {
-      const int nt = (int)(t % p.n_tiles);
-      const long m = t / p.n_tiles;
-      const int w0 = (int)(m % p.tiles_w) * 14, h0 = (int)((m / p.tiles_w) % p.tiles_h) * 8, n = (int)(m / (p.tiles_w * p.tiles_h));
+    // 32-bit tile arithmetic (the host keeps total_tiles below 2^30): 64-bit divisions here cost about a quarter of the tile time
+    for (int t = blockIdx.x + grp * gridDim.x; t < p.total_tiles; t += 2 * gridDim.x, tl += 2) {
+      const int nt = t % p.n_tiles;
+      const int m = t / p.n_tiles;
+      const int w0 = (m % p.tiles_w) * 14, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
       const uint32_t acc = grp, aph = (tl >> 1) & 1;
       ptx::mbar_wait(&tfull[acc], aph, abort_flag);
       ptx::tc_fence_after();
@@ -1160,6 +1161,7 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   if (bn) { p.bn_scale = bn->scale; p.bn_shift = bn->shift; p.bn_mu = bn->mu; p.bn_invstd = bn->invstd; }
   p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = epi == 2 ? 1 : Cin / 64; p.n_tiles = epi == 2 ? Cout / 64 : 1;
   p.tiles_w = W / 14; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
+  if ((long long)N * p.tiles_w * p.tiles_h * p.n_tiles > (1ll << 30)) return NF_EUNSUPPORTED;
   p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
   const size_t a_bytes = (size_t)10 * 16 * KC * 2;
   const size_t wbytes = epi == 2 ? (size_t)9 * KC * 128 : (size_t)9 * p.kchunks * G * 128;
