@@ -222,6 +222,41 @@ void nfo_avgpool_2x2_bwd(const double* dp, int N, int F, int H, int W, double* d
         }
 }
 
+/* F_n of Eq. 2 as adaptive MAX pooling to 2x2 (the paper names max or average pooling): the same bins as the
+ * average pool; arg receives the position i*W+j of the first maximum of each bin in row-major scan order. */
+void nfo_maxpool_2x2_adaptive(const double* h, int N, int F, int H, int W, double* p, int32_t* arg) {
+  for (int n = 0; n < N; ++n)
+    for (int f = 0; f < F; ++f)
+      for (int u = 0; u < 2; ++u)
+        for (int v = 0; v < 2; ++v) {
+          int i0, i1, j0, j1;
+          bin_range(u, H, &i0, &i1);
+          bin_range(v, W, &j0, &j1);
+          double m = h[IDX4(n, f, i0, j0, F, H, W)];
+          int32_t at = i0 * W + j0;
+          for (int i = i0; i < i1; ++i)
+            for (int j = j0; j < j1; ++j) {
+              const double t = h[IDX4(n, f, i, j, F, H, W)];
+              if (t > m) { m = t; at = i * W + j; }
+            }
+          const size_t o = (((size_t)n * F + f) * 2 + u) * 2 + v;
+          p[o] = m;
+          arg[o] = at;
+        }
+}
+
+/* Its backward: the whole of dp goes to the element that was the maximum of the bin; an element that is the
+ * maximum of two overlapping bins (odd sizes) receives both. */
+void nfo_maxpool_2x2_adaptive_bwd(const double* dp, const int32_t* arg, int N, int F, int H, int W, double* dh) {
+  memset(dh, 0, sizeof(double) * (size_t)N * F * H * W);
+  for (int n = 0; n < N; ++n)
+    for (int f = 0; f < F; ++f)
+      for (int b = 0; b < 4; ++b) {
+        const size_t o = ((size_t)n * F + f) * 4 + b;
+        dh[((size_t)n * F + f) * H * W + arg[o]] += dp[o];
+      }
+}
+
 /* gamma_n in Eq. 2: logits[n,k] = bf[k] + sum_d Wf[k,d] * p[n,d]. */
 void nfo_fc(const double* p, int N, int D, const double* Wf, const double* bf, int K, double* logits) {
   for (int n = 0; n < N; ++n)
@@ -249,6 +284,20 @@ double nfo_softmax_ce(const double* logits, const int32_t* labels, int N, int K,
         dlogits[(size_t)n * K + k] = (exp(l[k] - lse) - (k == labels[n] ? 1.0 : 0.0)) / (double)N;
   }
   return loss / (double)N;
+}
+
+/* Eq. 3 with the mean-squared-error loss against one-hot targets t: L = (1/(N K)) sum_{n,k} (logits - t)^2,
+ * dlogits = 2 (logits - t) / (N K).  dlogits may be NULL. */
+double nfo_mse_onehot(const double* logits, const int32_t* labels, int N, int K, double* dlogits) {
+  double loss = 0.0;
+  const double inv = 1.0 / ((double)N * (double)K);
+  for (int n = 0; n < N; ++n)
+    for (int k = 0; k < K; ++k) {
+      const double e = logits[(size_t)n * K + k] - (k == labels[n] ? 1.0 : 0.0);
+      loss += e * e;
+      if (dlogits) dlogits[(size_t)n * K + k] = 2.0 * e * inv;
+    }
+  return loss * inv;
 }
 
 /* Backward of train-mode BatchNorm.  With M = N*HW:
@@ -294,6 +343,10 @@ typedef struct {
                      storage precision, and the two convolutions read bfloat16 copies of their weights W and
                      Wa (the master weights, their momentum and their update stay unrounded; the gradient of
                      the copy is applied to the master).  All arithmetic stays fp64. */
+  int loss;       /* the loss of Eq. 3: 0 = cross entropy, 1 = mean squared error against one-hot targets */
+  int aux_pool;   /* F_n of Eq. 2: 0 = adaptive average pool to 2x2, 1 = adaptive max pool to 2x2.  In the bf16
+                     configuration the auxiliary activation h is then rounded to bfloat16 where it is stored, so that
+                     the arg-max of a bin is decided among the stored values. */
 } nfo_dims;
 
 /* Round to the nearest bfloat16, ties to even (via float, as a bf16 store of an fp32 value does). */
@@ -370,10 +423,16 @@ double nfo_layer_step(const nfo_dims* d, const double* x, const int32_t* labels,
   /* auxiliary network: Eq. 2 */
   nfo_conv3x3(a, N, Co, Ha, Wa, Waq, F, P->ba, 1, hpre);
   nfo_relu(hpre, nh, h);
-  nfo_avgpool_2x2(h, N, F, Ha, Wa, p);
+  int32_t* parg = (int32_t*)calloc((size_t)N * D, sizeof(int32_t));
+  if (d->aux_pool == 1) {
+    store_round(h, nh, d->store_bf16);
+    nfo_maxpool_2x2_adaptive(h, N, F, Ha, Wa, p, parg);
+  } else {
+    nfo_avgpool_2x2(h, N, F, Ha, Wa, p);
+  }
   nfo_fc(p, N, D, P->Wf, P->bf, K, logits);
   /* loss: Eq. 3 */
-  const double loss = nfo_softmax_ce(logits, labels, N, K, dlogits);
+  const double loss = d->loss == 1 ? nfo_mse_onehot(logits, labels, N, K, dlogits) : nfo_softmax_ce(logits, labels, N, K, dlogits);
 
   /* gradients of gamma_n: dWf = dlogits^T p ; dbf = sum_n dlogits ; dp = dlogits Wf */
   for (int k = 0; k < K; ++k) {
@@ -393,7 +452,9 @@ double nfo_layer_step(const nfo_dims* d, const double* x, const int32_t* labels,
       dp[(size_t)n * D + j] = sp;
     }
   /* gradients of beta_n */
-  nfo_avgpool_2x2_bwd(dp, N, F, Ha, Wa, dh);
+  if (d->aux_pool == 1) nfo_maxpool_2x2_adaptive_bwd(dp, parg, N, F, Ha, Wa, dh);
+  else nfo_avgpool_2x2_bwd(dp, N, F, Ha, Wa, dh);
+  free(parg);
   for (size_t k = 0; k < nh; ++k) if (!(hpre[k] > 0.0)) dh[k] = 0.0;
   nfo_conv3x3_wgrad(a, N, Co, Ha, Wa, dh, F, 1, gWa);
   for (int f = 0; f < F; ++f) {
@@ -495,7 +556,14 @@ void nfo_layer_predict(const nfo_dims* d, const double* x, const nfo_params* P, 
   store_round(Waq, (size_t)F * Co * 9, d->store_bf16);
   nfo_conv3x3(a, N, Co, Ha, Wa, Waq, F, P->ba, 1, hpre);
   nfo_relu(hpre, nh, h);
-  nfo_avgpool_2x2(h, N, F, Ha, Wa, p);
+  if (d->aux_pool == 1) {
+    int32_t* parg = (int32_t*)calloc((size_t)N * 4 * F, sizeof(int32_t));
+    store_round(h, nh, d->store_bf16);
+    nfo_maxpool_2x2_adaptive(h, N, F, Ha, Wa, p, parg);
+    free(parg);
+  } else {
+    nfo_avgpool_2x2(h, N, F, Ha, Wa, p);
+  }
   nfo_fc(p, N, 4 * F, P->Wf, P->bf, K, logits);
   if (act_out) memcpy(act_out, a, na * sizeof(double));
   free(a); free(hpre); free(h); free(p); free(Waq);

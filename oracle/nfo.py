@@ -31,7 +31,8 @@ _ip = C.POINTER(C.c_int32)
 
 class Dims(C.Structure):
     _fields_ = [(k, C.c_int) for k in ("N", "Cin", "Cout", "H", "W", "stride", "pool", "F", "classes")] + \
-               [(k, C.c_double) for k in ("eps", "momentum", "bn_momentum")] + [("store_bf16", C.c_int)]
+               [(k, C.c_double) for k in ("eps", "momentum", "bn_momentum")] + \
+               [(k, C.c_int) for k in ("store_bf16", "loss", "aux_pool")]
 
 
 _PNAMES = ("W", "gamma", "beta", "Wa", "ba", "Wf", "bf")
@@ -54,6 +55,7 @@ def lib():
         _lib = C.CDLL(build())
         _lib.nfo_layer_step.restype = C.c_double
         _lib.nfo_softmax_ce.restype = C.c_double
+        _lib.nfo_mse_onehot.restype = C.c_double
         _lib.nfo_threads.restype = C.c_int
         _lib.nfo_round_bf16.restype = C.c_double
         _lib.nfo_round_bf16.argtypes = [C.c_double]
@@ -148,6 +150,34 @@ def avgpool_2x2_bwd(dp, H, W):
     return dh
 
 
+def maxpool_2x2_adaptive(h):
+    """Adaptive max pool to 2x2 and the position i*W+j of the first maximum of every bin."""
+    h = _c64(h)
+    N, F, H, W = h.shape
+    p = np.empty((N, F, 2, 2))
+    arg = np.empty((N, F, 2, 2), dtype=np.int32)
+    lib().nfo_maxpool_2x2_adaptive(_d(h), N, F, H, W, _d(p), arg.ctypes.data_as(_ip))
+    return p, arg
+
+
+def maxpool_2x2_adaptive_bwd(dp, arg, H, W):
+    dp = _c64(dp)
+    arg = np.ascontiguousarray(arg, dtype=np.int32)
+    N, F = dp.shape[:2]
+    dh = np.empty((N, F, H, W))
+    lib().nfo_maxpool_2x2_adaptive_bwd(_d(dp), arg.ctypes.data_as(_ip), N, F, H, W, _d(dh))
+    return dh
+
+
+def mse_onehot(logits, labels):
+    logits = _c64(logits)
+    labels = np.ascontiguousarray(labels, dtype=np.int32)
+    N, K = logits.shape
+    dl = np.empty_like(logits)
+    loss = lib().nfo_mse_onehot(_d(logits), labels.ctypes.data_as(_ip), N, K, _d(dl))
+    return float(loss), dl
+
+
 def fc(p, Wf, bf):
     p, Wf, bf = _c64(p), _c64(Wf), _c64(bf)
     N, D = p.shape
@@ -176,8 +206,9 @@ class Layer:
     """Parameters, momentum and running statistics of one layer plus its auxiliary head (fp64)."""
 
     def __init__(self, Cin, Cout, H, W, F, classes, N, stride=1, pool=False, eps=1e-5, momentum=0.9,
-                 bn_momentum=0.1, store_bf16=False):
-        self.d = Dims(N, Cin, Cout, H, W, stride, int(pool), F, classes, eps, momentum, bn_momentum, int(store_bf16))
+                 bn_momentum=0.1, store_bf16=False, loss="ce", aux_pool="avg"):
+        self.d = Dims(N, Cin, Cout, H, W, stride, int(pool), F, classes, eps, momentum, bn_momentum, int(store_bf16),
+                      {"ce": 0, "mse": 1}[loss], {"avg": 0, "max": 1}[aux_pool])
         self.Ho, self.Wo = out_size(H, stride), out_size(W, stride)
         self.Ha, self.Wa = (self.Ho // 2, self.Wo // 2) if pool else (self.Ho, self.Wo)
         sh = dict(W=(Cout, Cin, 3, 3), gamma=(Cout,), beta=(Cout,), Wa=(F, Cout, 3, 3), ba=(F,),

@@ -199,3 +199,55 @@ def test_linear_memory_model_on_paper_points():
     t = nfo.max_batch_from_line(slope, icpt, 630.0)
     assert icpt + slope * t <= 630.0 < icpt + slope * (t + 1)
     assert t == 36
+
+
+def test_mse_loss_against_library_closed_form_and_finite_differences():
+    """Eq. 3 with the mean-squared-error loss: library mse_loss on one-hot targets (and its autograd
+    gradient), the closed form for constant logits, and a central finite difference of one entry."""
+    import torch
+    N, K = 5, 7
+    logits = synth.normal(61, 1, (N, K))
+    labels = synth.labels(61, 2, N, K)
+    loss, dl = nfo.mse_onehot(logits, labels)
+    zt = torch.tensor(logits, dtype=torch.float64, requires_grad=True)
+    tt = torch.nn.functional.one_hot(torch.tensor(labels.astype(np.int64)), K).to(torch.float64)
+    ref = torch.nn.functional.mse_loss(zt, tt)
+    ref.backward()
+    assert abs(loss - float(ref.detach())) < 1e-14
+    np.testing.assert_allclose(dl, zt.grad.numpy(), atol=1e-15)
+    # constant logits c: L = ((K-1) c^2 + (c-1)^2) / K whatever the labels
+    c = 0.3
+    assert abs(nfo.mse_onehot(np.full((4, K), c), synth.labels(61, 3, 4, K))[0] - ((K - 1) * c * c + (c - 1) ** 2) / K) < 1e-15
+    e = 1e-6
+    lp, lm = logits.copy(), logits.copy()
+    lp[2, 3] += e
+    lm[2, 3] -= e
+    assert abs((nfo.mse_onehot(lp, labels)[0] - nfo.mse_onehot(lm, labels)[0]) / (2 * e) - dl[2, 3]) < 1e-9
+
+
+def test_adaptive_maxpool_even_odd_ties_and_adjoint_routing():
+    """F_n as max pooling: even sizes against a reshape-max, odd sizes against hand-computed overlapping bins,
+    the first maximum on ties, and the backward routes each bin's gradient to exactly that position."""
+    h = synth.normal(62, 1, (2, 3, 4, 6))
+    p, arg = nfo.maxpool_2x2_adaptive(h)
+    np.testing.assert_array_equal(p, h.reshape(2, 3, 2, 2, 2, 3).max(axis=(3, 5)))
+    for n in range(2):
+        for f in range(3):
+            for b in range(4):
+                i, j = divmod(int(arg[n, f, b // 2, b % 2]), 6)
+                assert h[n, f, i, j] == p[n, f, b // 2, b % 2] and i // 2 == b // 2 and j // 3 == b % 2
+    h3 = np.arange(9.0).reshape(1, 1, 3, 3)            # bins overlap in the middle row and column
+    p3, a3 = nfo.maxpool_2x2_adaptive(h3)
+    np.testing.assert_array_equal(p3[0, 0], [[4.0, 5.0], [7.0, 8.0]])
+    np.testing.assert_array_equal(a3[0, 0], [[4, 5], [7, 8]])
+    ties = np.zeros((1, 1, 4, 4))
+    ties[0, 0, 1, 0] = ties[0, 0, 0, 1] = 2.0         # two equal maxima in bin (0,0): row-major scan meets (0,1) first
+    assert nfo.maxpool_2x2_adaptive(ties)[1][0, 0, 0, 0] == 1
+    dp = synth.normal(62, 2, (2, 3, 2, 2))
+    dh = nfo.maxpool_2x2_adaptive_bwd(dp, arg, 4, 6)
+    assert np.count_nonzero(dh) == dp.size and abs(dh.sum() - dp.sum()) < 1e-13
+    assert abs((p * dp).sum() - (h * dh).sum()) < 1e-12          # <pool(h), dp> = <h, pool^T dp> at the chosen positions
+    c = np.zeros((1, 1, 3, 3))
+    c[0, 0, 1, 1] = 5.0                                # the centre of an odd map is the maximum of all four bins
+    pc, ac = nfo.maxpool_2x2_adaptive(c)
+    assert nfo.maxpool_2x2_adaptive_bwd(np.ones((1, 1, 2, 2)), ac, 3, 3)[0, 0, 1, 1] == 4.0

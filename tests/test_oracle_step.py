@@ -248,3 +248,52 @@ def test_early_exit_prediction_against_library_ops_and_selection_rule():
     assert nfo.select_exit([0.2], [5]) == 0
     main, aux = L.n_params()
     assert main == c["Cout"] * c["Cin"] * 9 + 2 * c["Cout"] and aux == c["F"] * c["Cout"] * 9 + c["F"] + c["classes"] * (4 * c["F"] + 1)
+
+
+VARIANTS = [("mse", "avg"), ("ce", "max"), ("mse", "max")]
+
+
+@pytest.mark.parametrize("vi", range(len(VARIANTS)))
+@pytest.mark.parametrize("ci", range(len(CASES)))
+def test_loss_and_downsampling_variants_against_library_autograd(ci, vi):
+    """The alternatives the paper names for the loss (mean squared error) and the down-sampling F_n (max
+    pooling): one step re-derived with the library's mse_loss / adaptive_max_pool2d, autograd and SGD."""
+    c = CASES[ci]
+    loss_kind, pool_kind = VARIANTS[vi]
+    L, x, y = make_layer(c, 31 + ci)
+    L2 = nfo.Layer(c["Cin"], c["Cout"], c["H"], c["W"], c["F"], c["classes"], c["N"], stride=c["stride"], pool=c["pool"],
+                   loss=loss_kind, aux_pool=pool_kind)
+    L2.set(**L.p)
+    tp = {k: torch.tensor(v.copy(), dtype=torch.float64, requires_grad=True) for k, v in L.p.items()}
+    opt = torch.optim.SGD(list(tp.values()), lr=0.05, momentum=0.9)
+    rm, rv = torch.zeros(c["Cout"], dtype=torch.float64), torch.ones(c["Cout"], dtype=torch.float64)
+    xt, yt = torch.tensor(x), torch.tensor(y.astype(np.int64))
+    F = torch.nn.functional
+    a = F.relu(F.batch_norm(F.conv2d(xt, tp["W"], None, stride=c["stride"], padding=1), rm, rv, tp["gamma"], tp["beta"],
+                            training=True, momentum=0.1, eps=1e-5))
+    if c["pool"]:
+        a = F.max_pool2d(a, 2)
+    h = F.relu(F.conv2d(a, tp["Wa"], tp["ba"], padding=1))
+    p = (F.adaptive_max_pool2d(h, 2) if pool_kind == "max" else F.adaptive_avg_pool2d(h, 2)).flatten(1)
+    logits = F.linear(p, tp["Wf"], tp["bf"])
+    loss_t = F.mse_loss(logits, F.one_hot(yt, c["classes"]).to(torch.float64)) if loss_kind == "mse" else F.cross_entropy(logits, yt)
+    loss_t.backward()
+    grads = {k: v.grad.detach().numpy().copy() for k, v in tp.items()}
+    opt.step()
+    loss, act, tr = L2.step(x, y, 0.05, update=True, trace=True)
+    assert abs(loss - float(loss_t.detach())) <= 1e-12 * max(1, abs(loss))
+    for k, g in [("W", "gW"), ("gamma", "ggamma"), ("beta", "gbeta"), ("Wa", "gWa"), ("ba", "gba"), ("Wf", "gWf"), ("bf", "gbf")]:
+        np.testing.assert_allclose(tr[g], grads[k], atol=1e-11 * max(1.0, np.abs(grads[k]).max()), err_msg=k)
+        np.testing.assert_allclose(L2.p[k], tp[k].detach().numpy(), atol=1e-12, err_msg=k)
+    # the variant really differs from the default step
+    assert abs(loss - L.step(x, y, 0.05, update=False)[0]) > 1e-6
+    # early-exit logits use the same down-sampling
+    with torch.no_grad():
+        ae = F.relu(F.batch_norm(F.conv2d(xt, tp["W"], None, stride=c["stride"], padding=1), rm, rv, tp["gamma"], tp["beta"],
+                                 training=False, eps=1e-5))
+        if c["pool"]:
+            ae = F.max_pool2d(ae, 2)
+        he = F.relu(F.conv2d(ae, tp["Wa"], tp["ba"], padding=1))
+        pe = (F.adaptive_max_pool2d(he, 2) if pool_kind == "max" else F.adaptive_avg_pool2d(he, 2)).flatten(1)
+        le = F.linear(pe, tp["Wf"], tp["bf"])
+    np.testing.assert_allclose(L2.predict(x)[1], le.numpy(), atol=1e-11)
