@@ -85,7 +85,12 @@ typedef struct nf_layer_opts {
   float bn_eps;      /* BatchNorm epsilon */
   float bn_momentum; /* running-statistics momentum */
   int host_io;       /* 1: reserve staging so nf_layer_step_host can be used */
+  int loss;          /* nf_loss: the loss of Eq. 3 ("e.g., Mean Squared Error or Cross Entropy Error"); 0 = cross entropy */
+  int aux_pool;      /* nf_aux_pool: the down-sampling F_n of Eq. 2 ("such as max pooling or average pooling"); 0 = average */
 } nf_layer_opts;
+
+enum nf_loss { NF_LOSS_CE = 0, NF_LOSS_MSE = 1 };        /* MSE: mean over batch and classes of (z - onehot)^2 */
+enum nf_aux_pool { NF_POOL_AVG = 0, NF_POOL_MAX = 1 };   /* both adaptive to 2x2; max: first maximum of a bin in row-major order */
 
 /* Create the description of layer n with its auxiliary network A_n (Eq. 1, Eq. 2):
  * conv3x3 Cin->Cout on an H x W input, BatchNorm, ReLU; aux conv3x3 Cout->F, ReLU,

@@ -103,6 +103,7 @@ size_t plan(nf_layer* L, char* base, bool assign) {
   D->act = c.take(na * es);
   D->p = (float*)c.take(N * 4 * F * 4);
   D->dp = (float*)c.take(N * 4 * F * 4);
+  D->parg = (int32_t*)c.take(N * 4 * F * 4);
   D->logits = (float*)c.take(N * K * 4);
   D->dlogits = (float*)c.take(N * K * 4);
   D->lossn = (float*)c.take(N * 4);
@@ -226,6 +227,7 @@ int nf_layer_configure(nf_layer* L, const nf_layer_opts* o) {
     return NF_EINVAL;
   const int Ho = (L->H - 1) / o->stride + 1, Wo = (L->W - 1) / o->stride + 1;
   if (o->maxpool && ((Ho & 1) || (Wo & 1))) return NF_EINVAL;
+  if ((o->loss != NF_LOSS_CE && o->loss != NF_LOSS_MSE) || (o->aux_pool != NF_POOL_AVG && o->aux_pool != NF_POOL_MAX)) return NF_EINVAL;
   L->o = *o;
   L->o.maxpool = o->maxpool ? 1 : 0;
   L->o.host_io = o->host_io ? 1 : 0;
@@ -351,19 +353,23 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
   }
   trace_end();
   trace_begin(3);
-  {
+  if (L->o.aux_pool == NF_POOL_MAX) {
+    NF_TRY(nf_ref_auxmax(dt, L->h, N, Ha, Wa, F, L->p, L->parg));
+  } else {
     int rc = dt == NF_BF16 ? nf_ref_avgpool_fast(L->h, N, Ha, Wa, F, L->wpart, L->wpart_floats, L->p) : NF_EUNSUPPORTED;
     if (rc == NF_EUNSUPPORTED) rc = nf_ref_avgpool(dt, L->h, N, Ha, Wa, F, L->p);
     if (rc != NF_OK) return rc;
   }
   NF_TRY(nf_ref_fc_ce(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits,
-                      L->dp, L->lossn, L->status));
+                      L->dp, L->lossn, L->status, L->o.loss));
   // gradients of gamma_n, beta_n
   NF_TRY(nf_ref_fc_wgrad(L->p, L->dlogits, L->lossn, N, D, K, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->status));
   trace_end();
   trace_begin(4);
   int dh_nb = 0;
-  {
+  if (L->o.aux_pool == NF_POOL_MAX) {
+    NF_TRY(nf_ref_dh_max(dt, L->h, L->dp, L->parg, N, Ha, Wa, F, L->dh));
+  } else {
     int rc = dt == NF_BF16 ? nf_ref_dh_fast(L->h, L->dp, N, Ha, Wa, F, L->dh, L->red, L->red_floats, &dh_nb) : NF_EUNSUPPORTED;
     if (rc == NF_EUNSUPPORTED) {
       dh_nb = 0;
@@ -509,7 +515,9 @@ int nf_layer_predict(nf_layer* L, const void* x, int count, void* act_out, float
   } else {
     NF_TRY(nf_ref_conv(dt, a, count, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
   }
-  {
+  if (L->o.aux_pool == NF_POOL_MAX) {
+    NF_TRY(nf_ref_auxmax(dt, L->h, count, Ha, Wa, F, L->p, L->parg));
+  } else {
     int rc = dt == NF_BF16 ? nf_ref_avgpool_fast(L->h, count, Ha, Wa, F, L->wpart, L->wpart_floats, L->p) : NF_EUNSUPPORTED;
     if (rc == NF_EUNSUPPORTED) rc = nf_ref_avgpool(dt, L->h, count, Ha, Wa, F, L->p);
     if (rc != NF_OK) return rc;

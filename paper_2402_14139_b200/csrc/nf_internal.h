@@ -42,6 +42,7 @@ struct nf_layer {
   void* da;                            // [N][Ha][Wa][Cout]
   void* act;                           // [N][Ha][Wa][Cout] activation kept here when the caller gives no buffer
   float *p, *dp;                       // [N][4F]
+  int32_t* parg;                       // [N][4F] position i*Wa+j of each bin's maximum (max-pool down-sampling only)
   float *logits, *dlogits;             // [N][classes]
   float* lossn;                        // [N]
   float* red;                          // reduction scratch (channel partials)
@@ -99,8 +100,10 @@ int nf_ref_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part
 int nf_ref_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh, float* red, size_t red_floats,
                    int* nblocks);
 int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
-                 float* logits, float* dlogits, float* dp, float* lossn, int32_t* status);
+                 float* logits, float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind);
 int nf_ref_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count);
+int nf_ref_auxmax(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p, int32_t* parg);
+int nf_ref_dh_max(int dtype, const void* h, const float* dp, const int32_t* parg, int N, int Ha, int Wa, int F, void* dh);
 int nf_ref_fc_predict(const float* p, int N, int D, int K, const float* Wf, const float* bf, float* logits, int32_t* pred);
 int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
                     float* gbf, float* loss_out, int32_t* status);

@@ -221,6 +221,69 @@ __global__ void __launch_bounds__(256) avgpool_kernel(const T* __restrict__ h, i
   }
 }
 
+// Max-pool down-sampling: p[n][f*4 + bin] = max of h over bin (u,v), parg = position i*Wa+j of the FIRST maximum in
+// row-major order; one block per (n, bin).  A thread scans its pixels in increasing order and keeps the first
+// maximum; the lanes of a filter are then combined preferring the larger value, the smaller position on ties.
+template <typename T>
+__global__ void __launch_bounds__(256) auxmax_kernel(const T* __restrict__ h, int Ha, int Wa, int F, float* __restrict__ p,
+                                                     int32_t* __restrict__ parg) {
+  __shared__ float sv[256];
+  __shared__ int si[256];
+  const int n = blockIdx.x / 4, bin = blockIdx.x % 4, u = bin / 2, v = bin % 2;
+  int i0, i1, j0, j1;
+  bin_range(u, Ha, i0, i1);
+  bin_range(v, Wa, j0, j1);
+  const int bw = j1 - j0, cnt = (i1 - i0) * bw;
+  const int lanes = pow2ceil_cap256(F), planes = 256 / lanes;
+  const int lf = threadIdx.x % lanes, pl = threadIdx.x / lanes;
+  for (int f0 = 0; f0 < F; f0 += lanes) {
+    const int f = f0 + lf;
+    float best = -INFINITY;
+    int at = 0x7fffffff;
+    if (f < F)
+      for (int k = pl; k < cnt; k += planes) {
+        const int i = i0 + k / bw, j = j0 + k % bw;
+        const float t = ldf(h, (((size_t)n * Ha + i) * Wa + j) * F + f);
+        if (t > best) { best = t; at = i * Wa + j; }
+      }
+    sv[threadIdx.x] = best;
+    si[threadIdx.x] = at;
+    __syncthreads();
+    if (pl == 0 && f < F) {
+      float b = sv[lf];
+      int a = si[lf];
+      for (int q = 1; q < planes; ++q) {
+        const float t = sv[q * lanes + lf];
+        const int ti = si[q * lanes + lf];
+        if (t > b || (t == b && ti < a)) { b = t; a = ti; }
+      }
+      p[(size_t)n * 4 * F + f * 4 + bin] = b;
+      parg[(size_t)n * 4 * F + f * 4 + bin] = a;
+    }
+    __syncthreads();
+  }
+}
+
+// dh[n,i,j,f] = 1[h>0] * sum over the bins whose maximum sits at (i,j) of dp[n][f*4+bin]
+template <typename T>
+__global__ void dh_max_kernel(const T* __restrict__ h, const float* __restrict__ dp, const int32_t* __restrict__ parg, int Ha, int Wa,
+                              int F, size_t total, T* __restrict__ dh) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const int f = (int)(e % F);
+  const size_t q = e / F;
+  const int j = (int)(q % Wa), i = (int)((q / Wa) % Ha);
+  const size_t n = q / ((size_t)Wa * Ha);
+  float g = 0.f;
+  if (ldf(h, e) > 0.f) {
+    const int pos = i * Wa + j;
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+      if (parg[n * 4 * F + f * 4 + b] == pos) g += dp[n * 4 * F + f * 4 + b];
+  }
+  stf(dh, e, g);
+}
+
 __device__ __forceinline__ float block_reduce(float v, float* sm, bool is_max) {
   const int t = threadIdx.x;
   sm[t] = v;
@@ -238,7 +301,8 @@ __device__ __forceinline__ float block_reduce(float v, float* sm, bool is_max) {
 __global__ void __launch_bounds__(256) fc_ce_kernel(const float* __restrict__ p, const int32_t* __restrict__ labels, int N,
                                                     int D, int K, const float* __restrict__ Wf, const float* __restrict__ bf,
                                                     float* __restrict__ logits, float* __restrict__ dlogits,
-                                                    float* __restrict__ dp, float* __restrict__ lossn, int32_t* status) {
+                                                    float* __restrict__ dp, float* __restrict__ lossn, int32_t* status,
+                                                    int loss_kind) {
   extern __shared__ float dyn[];
   float* ps = dyn;          // [D]
   float* ls = dyn + D;      // [K]
@@ -256,21 +320,35 @@ __global__ void __launch_bounds__(256) fc_ce_kernel(const float* __restrict__ p,
     mx = fmaxf(mx, s);
   }
   mx = block_reduce(mx, red, true);
-  float se = 0.f;
-  for (int k = t; k < K; k += 256) se += expf(ls[k] - mx);
-  se = block_reduce(se, red, false);
-  const float lse = mx + logf(se);
   int lab = labels[n];
   if (lab < 0 || lab >= K) {
     if (t == 0) atomicOr(status, NF_ELABEL);
     lab = lab < 0 ? 0 : K - 1;
   }
-  if (t == 0) lossn[n] = lse - ls[lab];
-  const float invN = 1.f / (float)N;
-  for (int k = t; k < K; k += 256) {
-    const float g = (expf(ls[k] - lse) - (k == lab ? 1.f : 0.f)) * invN;
-    ls[k] = g;
-    dlogits[(size_t)n * K + k] = g;
+  if (loss_kind == 1) {
+    // mean squared error against the one-hot target: lossn = sum_k e^2 / K, dlogits = 2 e / (N K)
+    float se = 0.f;
+    const float sc = 2.f / ((float)N * (float)K);
+    for (int k = t; k < K; k += 256) {
+      const float e = ls[k] - (k == lab ? 1.f : 0.f);
+      se = fmaf(e, e, se);
+      ls[k] = e * sc;
+      dlogits[(size_t)n * K + k] = e * sc;
+    }
+    se = block_reduce(se, red, false);
+    if (t == 0) lossn[n] = se / (float)K;
+  } else {
+    float se = 0.f;
+    for (int k = t; k < K; k += 256) se += expf(ls[k] - mx);
+    se = block_reduce(se, red, false);
+    const float lse = mx + logf(se);
+    if (t == 0) lossn[n] = lse - ls[lab];
+    const float invN = 1.f / (float)N;
+    for (int k = t; k < K; k += 256) {
+      const float g = (expf(ls[k] - lse) - (k == lab ? 1.f : 0.f)) * invN;
+      ls[k] = g;
+      dlogits[(size_t)n * K + k] = g;
+    }
   }
   __syncthreads();
   // dp[d] = sum_k g[k] Wf[k][d]: the classes are cut into G contiguous ranges (G = 256 / D lanes per d when D <= 128),
@@ -1096,10 +1174,10 @@ int nf_ref_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float
 }
 
 int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
-                 float* logits, float* dlogits, float* dp, float* lossn, int32_t* status) {
+                 float* logits, float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind) {
   const size_t smem = (size_t)(D + K) * sizeof(float);
   if (smem > 40000) return NF_EUNSUPPORTED;
-  fc_ce_kernel<<<N, 256, smem, g_nf_stream>>>(p, labels, N, D, K, Wf, bf, logits, dlogits, dp, lossn, status);
+  fc_ce_kernel<<<N, 256, smem, g_nf_stream>>>(p, labels, N, D, K, Wf, bf, logits, dlogits, dp, lossn, status, loss_kind);
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -1130,6 +1208,21 @@ int nf_ref_fc_predict(const float* p, int N, int D, int K, const float* Wf, cons
 int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
                     float* gbf, float* loss_out, int32_t* status) {
   fc_wgrad_kernel<<<K, 256, 0, g_nf_stream>>>(p, dlogits, lossn, N, D, K, gWf, gbf, loss_out, status);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_auxmax(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p, int32_t* parg) {
+  DISPATCH(dtype, (auxmax_kernel<float><<<N * 4, 256, 0, g_nf_stream>>>((const float*)h, Ha, Wa, F, p, parg)),
+           (auxmax_kernel<bf16><<<N * 4, 256, 0, g_nf_stream>>>((const bf16*)h, Ha, Wa, F, p, parg)));
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_dh_max(int dtype, const void* h, const float* dp, const int32_t* parg, int N, int Ha, int Wa, int F, void* dh) {
+  const size_t total = (size_t)N * Ha * Wa * F;
+  DISPATCH(dtype, (dh_max_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)h, dp, parg, Ha, Wa, F, total, (float*)dh)),
+           (dh_max_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)h, dp, parg, Ha, Wa, F, total, (bf16*)dh)));
   NF_LAUNCHED();
   return NF_OK;
 }

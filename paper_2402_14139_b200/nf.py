@@ -17,6 +17,8 @@ _SO = os.path.join(_HERE, "libnf.so")
 NF_OK, NF_EINVAL, NF_EALIGN, NF_ENOWS, NF_EUNSUPPORTED, NF_ECUDA = 0, -1, -2, -3, -4, -5
 NF_ELABEL, NF_ENONFINITE, NF_ETIMEOUT = 1, 2, 4
 NF_F32, NF_BF16 = 0, 1
+NF_LOSS_CE, NF_LOSS_MSE = 0, 1
+NF_POOL_AVG, NF_POOL_MAX = 0, 1
 NF_P_W, NF_P_GAMMA, NF_P_BETA, NF_P_WA, NF_P_BA, NF_P_WF, NF_P_BF, NF_P_RMEAN, NF_P_RVAR = range(9)
 NF_K_VALUE, NF_K_MOMENTUM, NF_K_GRAD = 0, 0x100, 0x200
 PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P_BA, Wf=NF_P_WF, bf=NF_P_BF,
@@ -36,7 +38,8 @@ class NfError(RuntimeError):
 
 class nf_layer_opts(C.Structure):
     _fields_ = [("N", C.c_int), ("stride", C.c_int), ("maxpool", C.c_int), ("dtype", C.c_int),
-                ("momentum", C.c_float), ("bn_eps", C.c_float), ("bn_momentum", C.c_float), ("host_io", C.c_int)]
+                ("momentum", C.c_float), ("bn_eps", C.c_float), ("bn_momentum", C.c_float), ("host_io", C.c_int),
+                ("loss", C.c_int), ("aux_pool", C.c_int)]
 
 
 _lib = None
@@ -177,7 +180,7 @@ class Layer:
     """One layer with its auxiliary head on the current CUDA device (wraps nf_layer_* calls)."""
 
     def __init__(self, Cin, Cout, H, W, F, classes, N, stride=1, maxpool=False, dtype=NF_BF16, momentum=0.9,
-                 bn_eps=1e-5, bn_momentum=0.1, host_io=False, device="cuda"):
+                 bn_eps=1e-5, bn_momentum=0.1, host_io=False, device="cuda", loss="ce", aux_pool="avg"):
         import torch
         self._torch = torch
         self.Cin, self.Cout, self.H, self.W, self.F, self.classes, self.N = Cin, Cout, H, W, F, classes, N
@@ -187,7 +190,8 @@ class Layer:
         self.h = lib().nf_layer_create(Cin, Cout, H, W, F, classes)
         if not self.h:
             raise NfError("nf_layer_create failed")
-        o = nf_layer_opts(N, stride, int(maxpool), dtype, momentum, bn_eps, bn_momentum, int(host_io))
+        o = nf_layer_opts(N, stride, int(maxpool), dtype, momentum, bn_eps, bn_momentum, int(host_io),
+                          {"ce": NF_LOSS_CE, "mse": NF_LOSS_MSE}[loss], {"avg": NF_POOL_AVG, "max": NF_POOL_MAX}[aux_pool])
         _check(lib().nf_layer_configure(self.h, C.byref(o)), "nf_layer_configure")
         self.ws_bytes = int(lib().nf_layer_workspace_bytes(self.h))
         self.ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device=device)

@@ -36,14 +36,16 @@ def seeded_case(c, seed, bf16):
 
 def oracle_layer(c, P, momentum=0.9, store_bf16=False):
     L = nfo.Layer(c["Cin"], c["Cout"], c["H"], c["W"], c["F"], c["classes"], c["N"], stride=c.get("stride", 1),
-                  pool=c.get("pool", False), momentum=momentum, store_bf16=store_bf16)
+                  pool=c.get("pool", False), momentum=momentum, store_bf16=store_bf16, loss=c.get("loss", "ce"),
+                  aux_pool=c.get("aux_pool", "avg"))
     L.set(**{k: np.asarray(v, dtype=np.float64) for k, v in P.items()})
     return L
 
 
 def gpu_layer(nf, c, P, dtype, momentum=0.9, host_io=False):
     L = nf.Layer(c["Cin"], c["Cout"], c["H"], c["W"], c["F"], c["classes"], c["N"], stride=c.get("stride", 1),
-                 maxpool=c.get("pool", False), dtype=dtype, momentum=momentum, host_io=host_io)
+                 maxpool=c.get("pool", False), dtype=dtype, momentum=momentum, host_io=host_io, loss=c.get("loss", "ce"),
+                 aux_pool=c.get("aux_pool", "avg"))
     for k, v in P.items():
         L.set_param(k, v)
     return L
