@@ -307,7 +307,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c4", choices=["c2", "c3", "c4", "c4s", "c5"])
+    ap.add_argument("--workload", default="c4", choices=["c2", "c3", "c4", "c4s", "c5", "c6"])
     ap.add_argument("--block", type=int, default=0, help="which block of a multi-block workload (c3, c5) to step")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

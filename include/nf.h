@@ -245,6 +245,24 @@ int nf_conv3x3_wgrad_static(int dtype, const void* x, const void* g, int N, int 
  * batch size; returns the number of blocks, or NF_EINVAL. */
 int nf_partition(const int* max_batch, int n_layers, int B, double rho, int* block_first, int* block_batch);
 
+/* The Profiler (Section "Modules"; host only, no device work).
+ *
+ * nf_aan_filters: the AAN-LL rule for the auxiliary filter counts.  channels[i] = filters of CNN layer i;
+ * layers with index < first_downsample (those before the first down-sampling operation) get half the SMALLEST
+ * entry of channels, all later layers half the LARGEST (VGG: 32 and 256).  Writes n_layers counts.
+ *
+ * nf_profile_layer: the device memory this library needs to train one layer (its workspace plus one input
+ * batch) at each of the k given batch sizes, and the least-squares line bytes = intercept + slope * batch
+ * through them (k >= 2 distinct sizes; bytes_out may be NULL).  opts->N is ignored.
+ *
+ * nf_max_batch: the largest batch t with intercept + slope * t <= budget (first loop of Algorithm 1);
+ * 0 if even one sample does not fit.  Feed the results to nf_partition.
+ * All return NF_EINVAL on bad arguments. */
+int nf_aan_filters(const int* channels, int n_layers, int first_downsample, int* filters_out);
+int nf_profile_layer(int Cin, int Cout, int H, int W, int F, int classes, const nf_layer_opts* opts, const int* batches, int k,
+                     double* bytes_out, double* slope, double* intercept);
+long long nf_max_batch(double slope, double intercept, double budget_bytes);
+
 /* Stream for all later calls (a cudaStream_t); NULL selects the default stream. */
 int nf_set_stream(void* cuda_stream);
 

@@ -333,6 +333,22 @@ def partition(max_batch, B, rho):
     return blocks
 
 
+def aan_filters(channels, first_downsample):
+    """AAN-LL rule (Section "Opportunity 1"): layers before the first down-sampling operation get half the smallest
+    filter count of the CNN, the later ones half the largest."""
+    lo, hi = min(channels), max(channels)
+    return [max(1, (lo if i < first_downsample else hi) // 2) for i in range(len(channels))]
+
+
+def fit_line(batches, bytes_):
+    """Least-squares line through (batch, bytes): the Profiler's layer-wise linear model.  Returns (slope, intercept)."""
+    x = np.asarray(batches, dtype=np.float64)
+    y = np.asarray(bytes_, dtype=np.float64)
+    xm, ym = x.mean(), y.mean()
+    slope = float(((x - xm) * (y - ym)).sum() / ((x - xm) ** 2).sum())
+    return slope, float(ym - slope * xm)
+
+
 def max_batch_from_line(slope, intercept, M):
     """Algorithm 1, first loop: largest integer batch t with intercept + slope*t <= M."""
     return int(np.floor((M - intercept) / slope + 1e-12))

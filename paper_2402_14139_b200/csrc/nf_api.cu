@@ -86,6 +86,7 @@ size_t plan(nf_layer* L, char* base, bool assign) {
   D->mom = (float*)c.take(L->arena * 4);
   D->grad = (float*)c.take(L->arena * 4);
   D->shadow = (bf16*)c.take(L->arena * 2);
+  D->wa_t = (bf16*)c.take(F > 64 ? (size_t)9 * Co * F * 2 : 0);
   D->rmean = (float*)c.take(Co * 4);
   D->rvar = (float*)c.take(Co * 4);
   D->scale = (float*)c.take(Co * 4);
@@ -118,6 +119,11 @@ size_t plan(nf_layer* L, char* base, bool assign) {
   D->wpart_floats = w1 > w2 ? w1 : w2;
   const size_t tc = nf_tc_scratch_floats(L);
   if (tc > D->wpart_floats) D->wpart_floats = tc;
+  if (nf_head_is_large((int)N, (int)(4 * F), (int)K)) {  // tiled head: logits before the bias, up to 16 batch ranges of gWf
+    size_t hs = nf_head_scratch_floats((int)N, (int)(4 * F), (int)K);
+    if (hs < (size_t)16 * K * 4 * F) hs = (size_t)16 * K * 4 * F;
+    if (hs > D->wpart_floats) D->wpart_floats = hs;
+  }
   D->wpart = (float*)c.take(D->wpart_floats * 4);
   if (L->o.host_io) {
     D->stage_x = c.take(N * L->H * L->W * L->Cin * es);
@@ -360,10 +366,16 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
     if (rc == NF_EUNSUPPORTED) rc = nf_ref_avgpool(dt, L->h, N, Ha, Wa, F, L->p);
     if (rc != NF_OK) return rc;
   }
-  NF_TRY(nf_ref_fc_ce(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits,
-                      L->dp, L->lossn, L->status, L->o.loss));
-  // gradients of gamma_n, beta_n
-  NF_TRY(nf_ref_fc_wgrad(L->p, L->dlogits, L->lossn, N, D, K, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->status));
+  if (nf_head_is_large(N, D, K)) {  // late blocks: tens of thousands of samples, up to 1024 head inputs
+    NF_TRY(nf_head_step(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits, L->dp,
+                        L->lossn, L->status, L->o.loss, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->wpart,
+                        L->wpart_floats));
+  } else {
+    NF_TRY(nf_ref_fc_ce(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits,
+                        L->dp, L->lossn, L->status, L->o.loss));
+    // gradients of gamma_n
+    NF_TRY(nf_ref_fc_wgrad(L->p, L->dlogits, L->lossn, N, D, K, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->status));
+  }
   trace_end();
   trace_begin(4);
   int dh_nb = 0;
@@ -523,6 +535,11 @@ int nf_layer_predict(nf_layer* L, const void* x, int count, void* act_out, float
     if (rc != NF_OK) return rc;
   }
   // the caller's logits have `classes` columns over the logical 4*Flog inputs; the padded inputs are zero
+  if (nf_head_is_large(count, 4 * F, L->classes)) {
+    float* lg = logits_out ? logits_out : L->logits;
+    NF_TRY(nf_head_logits(L->p, count, 4 * F, L->classes, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], lg, L->wpart));
+    return nf_head_predict(lg, count, L->classes, pred_out);
+  }
   return nf_ref_fc_predict(L->p, count, 4 * F, L->classes, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], logits_out, pred_out);
 }
 
@@ -667,6 +684,54 @@ int nf_partition(const int* max_batch, int n_layers, int Bcap, double rho, int* 
     ++i;
   }
   return nblocks;
+}
+
+int nf_aan_filters(const int* channels, int n_layers, int first_downsample, int* filters_out) {
+  if (!channels || !filters_out || n_layers < 1 || first_downsample < 0) return NF_EINVAL;
+  int lo = channels[0], hi = channels[0];
+  for (int i = 0; i < n_layers; ++i) {
+    if (channels[i] < 1) return NF_EINVAL;
+    if (channels[i] < lo) lo = channels[i];
+    if (channels[i] > hi) hi = channels[i];
+  }
+  for (int i = 0; i < n_layers; ++i) {
+    const int f = (i < first_downsample ? lo : hi) / 2;
+    filters_out[i] = f < 1 ? 1 : f;
+  }
+  return NF_OK;
+}
+
+int nf_profile_layer(int Cin, int Cout, int H, int W, int F, int classes, const nf_layer_opts* opts, const int* batches, int k,
+                     double* bytes_out, double* slope, double* intercept) {
+  if (!opts || !batches || !slope || !intercept || k < 2) return NF_EINVAL;
+  nf_layer* L = nf_layer_create(Cin, Cout, H, W, F, classes);
+  if (!L) return NF_EINVAL;
+  double sx = 0, sy = 0, sxx = 0, sxy = 0;
+  for (int i = 0; i < k; ++i) {
+    nf_layer_opts o = *opts;
+    o.N = batches[i];
+    const int rc = nf_layer_configure(L, &o);
+    if (rc != NF_OK) {
+      nf_layer_destroy(L);
+      return rc;
+    }
+    const double bytes = (double)nf_layer_workspace_bytes(L) + (double)o.N * H * W * Cin * (double)nf_esize(o.dtype);
+    if (bytes_out) bytes_out[i] = bytes;
+    const double x = (double)o.N;
+    sx += x; sy += bytes; sxx += x * x; sxy += x * bytes;
+  }
+  nf_layer_destroy(L);
+  const double den = k * sxx - sx * sx;
+  if (!(den > 0.0)) return NF_EINVAL;  // all batch sizes equal
+  *slope = (k * sxy - sx * sy) / den;
+  *intercept = (sy - *slope * sx) / k;
+  return NF_OK;
+}
+
+long long nf_max_batch(double slope, double intercept, double budget_bytes) {
+  if (!(slope > 0.0)) return NF_EINVAL;
+  const double t = floor((budget_bytes - intercept) / slope + 1e-12);
+  return t < 0.0 ? 0 : (long long)t;
 }
 
 int nf_set_stream(void* s) {

@@ -32,6 +32,7 @@ struct nf_layer {
   int32_t* status;                     // device status word
   float *val, *mom, *grad;             // arenas
   bf16* shadow;                        // bf16 arena
+  bf16* wa_t;                          // [9][Cout][F] mirrored, transposed copy of Wa (only when F > 64)
   float *rmean, *rvar;                 // [Cout]
   float *scale, *shift, *mu, *invstd;  // [Cout] per-step BatchNorm coefficients
   float *sdz, *sdzx;                   // [Cout] reduced sums for BatchNorm backward
@@ -104,6 +105,15 @@ int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, con
 int nf_ref_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count);
 int nf_ref_auxmax(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p, int32_t* parg);
 int nf_ref_dh_max(int dtype, const void* h, const float* dp, const int32_t* parg, int N, int Ha, int Wa, int F, void* dh);
+int nf_ref_flip_weights(const bf16* w, int F, int C, bf16* out);
+// large-batch head (nf_head.cu)
+bool nf_head_is_large(int N, int D, int K);
+size_t nf_head_scratch_floats(int N, int D, int K);
+int nf_head_logits(const float* p, int N, int D, int K, const float* Wf, const float* bf, float* logits, float* scratch);
+int nf_head_predict(const float* logits, int N, int K, int32_t* pred);
+int nf_head_step(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf, float* logits,
+                 float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind, float* gWf, float* gbf, float* loss_out,
+                 float* scratch, size_t scratch_floats);
 int nf_ref_fc_predict(const float* p, int N, int D, int K, const float* Wf, const float* bf, float* logits, int32_t* pred);
 int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
                     float* gbf, float* loss_out, int32_t* status);

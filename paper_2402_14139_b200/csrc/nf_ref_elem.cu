@@ -1212,6 +1212,20 @@ int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, in
   return NF_OK;
 }
 
+// out[8 - tap][c][f] = w[tap][f][c]: the weights of the input-gradient convolution written as a forward convolution
+__global__ void flip_weights_kernel(const bf16* __restrict__ w, int F, int C, bf16* __restrict__ out) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (size_t)9 * F * C) return;
+  const int f = (int)(e % F), c = (int)((e / F) % C), tap = (int)(e / ((size_t)F * C));
+  out[e] = w[((size_t)(8 - tap) * F + f) * C + c];
+}
+
+int nf_ref_flip_weights(const bf16* w, int F, int C, bf16* out) {
+  flip_weights_kernel<<<nblk((size_t)9 * F * C, 256), 256, 0, g_nf_stream>>>(w, F, C, out);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
 int nf_ref_auxmax(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p, int32_t* parg) {
   DISPATCH(dtype, (auxmax_kernel<float><<<N * 4, 256, 0, g_nf_stream>>>((const float*)h, Ha, Wa, F, p, parg)),
            (auxmax_kernel<bf16><<<N * 4, 256, 0, g_nf_stream>>>((const bf16*)h, Ha, Wa, F, p, parg)));

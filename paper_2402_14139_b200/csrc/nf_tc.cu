@@ -228,7 +228,13 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[q * 8 + 2 * e]), __uint_as_float(v[q * 8 + 2 * e + 1]));
+            float o0 = __uint_as_float(v[q * 8 + 2 * e]), o1 = __uint_as_float(v[q * 8 + 2 * e + 1]);
+            if (p.bias) {  // wide aux forward: bias and ReLU before the value is rounded for storage
+              const float* bch = p.bias + nt * BN + j * 32 + q * 8 + 2 * e;
+              o0 = fmaxf(o0 + __ldg(bch), 0.f);
+              o1 = fmaxf(o1 + __ldg(bch + 1), 0.f);
+            }
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(o0, o1);
             w[e] = *reinterpret_cast<const uint32_t*>(&b2);
           }
           *reinterpret_cast<uint4*>(sub + (((u0 + q) ^ (r & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -550,6 +556,8 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             if constexpr (EPI == 1) {
               const int ch = q * 16 + c;
               o[h2] = ch < p.Cout ? fmaxf(o[h2] + p.bias[ch], 0.f) : 0.f;
+            } else {
+              if (p.bias) o[h2] = fmaxf(o[h2] + __ldg(p.bias + nt * 64 + q * 16 + c), 0.f);
             }
           }
           const __nv_bfloat162 b2 = __floats2bfloat162_rn(o[0], o[1]);
@@ -1048,7 +1056,7 @@ bool pick_tile(int H, int W, bool allow_multi, int* BW, int* BH, int* BI) {
       *BW = c[0]; *BH = c[1]; *BI = 1;
       return true;
     }
-  if (allow_multi && W * H <= 64 && W >= 2 && 128 % (W * H) == 0 && (W & (W - 1)) == 0) {  // 8x8, 4x4, 2x2, 8x4 ...
+  if (allow_multi && W * H <= 64 && 128 % (W * H) == 0 && (W & (W - 1)) == 0) {  // 8x8, 4x4, 2x2, 8x4, 1x1 ...
     *BW = W; *BH = H; *BI = 128 / (W * H);
     return true;
   }
@@ -1346,18 +1354,28 @@ int run_wgrad(int N, int Hin, int Win, int Cin, int Cout, const void* x, const v
 
 }  // namespace
 
+// The classic local-learning setting (256 auxiliary filters) and the paper's own rule for late layers give F > 64.
+// Then the aux conv is as wide as a main conv and uses the same three kernels: forward (bias and ReLU in its epilogue),
+// weight gradient, and the input gradient written as a forward conv over a mirrored, transposed weight copy.
+static bool wide_aux(const nf_layer* L) { return L->F > 64 && L->F % 64 == 0; }
+
 void nf_tc_select(nf_layer* L) {
   L->fam[0] = L->fam[1] = L->fam[2] = L->fam[3] = 0;
   if (L->o.dtype != NF_BF16) return;
   if (plan_fwd(L->Ho, L->Wo, L->Cin, L->Cout, L->o.N, 0, L->o.stride).ok) L->fam[0] = 1;
   if (plan_wgrad(L->Ho, L->Wo, L->Cin, L->Cout, L->o.N, 0, L->o.stride).ok) L->fam[1] = 1;
+  if (wide_aux(L)) {  // more than 64 filters: the aux conv runs on the kernels of the main conv
+    if (plan_fwd(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 0).ok) L->fam[2] = 1;
+    if (plan_wgrad(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 0).ok && plan_fwd(L->Ha, L->Wa, L->F, L->Cout, L->o.N, 0).ok) L->fam[3] = 1;
+    return;
+  }
   if (plan_fwd(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).ok) L->fam[2] = 1;
   if (plan_wgrad(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).ok && plan_fwd(L->Ha, L->Wa, L->F, L->Cout, L->o.N, 2).ok) L->fam[3] = 1;
 }
 
 size_t nf_tc_scratch_floats(const nf_layer* L) {
   const size_t a = L->fam[1] ? plan_wgrad(L->Ho, L->Wo, L->Cin, L->Cout, L->o.N, 0, L->o.stride).part_floats : 0;
-  const size_t b = L->fam[3] ? plan_wgrad(L->Ha, L->Wa, L->Cout, L->F, L->o.N, 1).part_floats : 0;
+  const size_t b = L->fam[3] ? plan_wgrad(L->Ha, L->Wa, L->Cout, L->F, L->o.N, wide_aux(L) ? 0 : 1).part_floats : 0;
   return a > b ? a : b;
 }
 
@@ -1385,6 +1403,10 @@ int nf_tc_conv_fwd_eval(nf_layer* L, const void* x, int count) {
 
 int nf_tc_aux_fwd(nf_layer* L, const void* a, int count) {
   int nb = 0;
+  if (wide_aux(L)) {
+    return run_fwd(count, L->Ha, L->Wa, L->Cout, L->F, a, L->shadow + L->off[NF_P_WA], L->h, 0, nullptr, 0, L->status, &nb, 0,
+                   L->val + L->off[NF_P_BA]);
+  }
   return run_fwd(count, L->Ha, L->Wa, L->Cout, L->F, a, L->shadow + L->off[NF_P_WA], L->h, 0, nullptr, 0, L->status, &nb, 1,
                  L->val + L->off[NF_P_BA]);
 }
@@ -1397,6 +1419,11 @@ int nf_tc_wgrad(nf_layer* L, const void* x) {
 int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb) {
   int nb = 0;
   *bn_nb = 0;
+  if (wide_aux(L)) {
+    const int rc = nf_ref_flip_weights(L->shadow + L->off[NF_P_WA], L->F, L->Cout, L->wa_t);
+    if (rc != NF_OK) return rc;
+    return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->wa_t, L->da, 0, nullptr, 0, L->status, &nb, 0);
+  }
   // without a pool da has the shape of y: the folded kernel also reduces (dz, dz*xhat) per channel while it holds the tile
   if (!L->o.maxpool && fold_ok(L->Ha, L->Wa, L->F, L->Cout, 2, 1) &&
       (size_t)(sm_count() / (L->Cout / 64)) * 8 * 2 * L->Cout <= L->red_floats) {
@@ -1410,7 +1437,7 @@ int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb) {
 
 int nf_tc_aux_wgrad(nf_layer* L, const void* a) {
   return run_wgrad(L->o.N, L->Ha, L->Wa, L->Cout, L->F, a, L->dh, L->wpart, L->wpart_floats, L->grad + L->off[NF_P_WA],
-                   L->status, 1);
+                   L->status, wide_aux(L) ? 0 : 1);
 }
 
 size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout, int stride) {

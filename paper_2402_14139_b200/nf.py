@@ -27,7 +27,7 @@ PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P
 EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_layer_workspace_bytes",
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
-           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
+           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_max_batch", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
            "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_op_status", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
@@ -76,6 +76,11 @@ def lib():
         L.nf_layer_param_count.restype = C.c_longlong
         L.nf_layer_param_count.argtypes = [vp, C.c_int]
         L.nf_count_equal.argtypes = [ip, ip, C.c_longlong, vp]
+        L.nf_aan_filters.argtypes = [C.POINTER(C.c_int), C.c_int, C.c_int, C.POINTER(C.c_int)]
+        L.nf_profile_layer.argtypes = [C.c_int] * 6 + [C.POINTER(nf_layer_opts), C.POINTER(C.c_int), C.c_int, C.POINTER(C.c_double),
+                                       C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.nf_max_batch.restype = C.c_longlong
+        L.nf_max_batch.argtypes = [C.c_double, C.c_double, C.c_double]
         L.nf_select_exit.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.c_int]
         L.nf_block_step.argtypes = [vp, vp, ip, C.c_float, fp, vp]
         L.nf_block_step_host.argtypes = [vp, vp, ip, C.c_float, fp, vp]
@@ -154,6 +159,30 @@ def nf_trace_read(slots: int = 1):
             if n.value:
                 out[(name, s)] = (ms.value, n.value)
     return out
+
+
+def nf_aan_filters(channels, first_downsample: int):
+    """AAN-LL rule: aux filter count per layer (half the smallest channel count before the first down-sampling, half the largest after)."""
+    n = len(channels)
+    ch = (C.c_int * n)(*[int(v) for v in channels])
+    out = (C.c_int * n)()
+    _check(lib().nf_aan_filters(ch, n, int(first_downsample), out), "nf_aan_filters")
+    return list(out)
+
+
+def nf_profile_layer(Cin, Cout, H, W, F, classes, batches, stride=1, maxpool=False, dtype=NF_BF16, loss="ce", aux_pool="avg"):
+    """Memory model of one layer: (bytes at each batch size, slope, intercept) of bytes = intercept + slope * batch."""
+    k = len(batches)
+    o = nf_layer_opts(1, stride, int(maxpool), dtype, 0.9, 1e-5, 0.1, 0, {"ce": 0, "mse": 1}[loss], {"avg": 0, "max": 1}[aux_pool])
+    b = (C.c_int * k)(*[int(v) for v in batches])
+    by = (C.c_double * k)()
+    sl, ic = C.c_double(), C.c_double()
+    _check(lib().nf_profile_layer(Cin, Cout, H, W, F, classes, C.byref(o), b, k, by, C.byref(sl), C.byref(ic)), "nf_profile_layer")
+    return list(by), sl.value, ic.value
+
+
+def nf_max_batch(slope, intercept, budget_bytes) -> int:
+    return int(lib().nf_max_batch(float(slope), float(intercept), float(budget_bytes)))
 
 
 def nf_count_equal(a, b, count_out):

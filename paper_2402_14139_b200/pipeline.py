@@ -40,6 +40,21 @@ def build_layers(nf, wl, block_index, seed):
     return layers, nf.Block(layers)
 
 
+def plan_blocks(nf, layers, classes, budget_bytes, batch_cap, rho=0.4, batches=(32, 64, 128, 256), dtype="bf16"):
+    """Profiler + Partitioner: the linear memory model of every layer (nf_profile_layer), its largest batch under the
+    budget (nf_max_batch) and Algorithm 1 (nf_partition).  Returns [(first_layer, last_layer, batch_size)]."""
+    dt = nf.NF_F32 if dtype == "f32" else nf.NF_BF16
+    max_batch = []
+    for l in layers:
+        _, slope, icpt = nf.nf_profile_layer(l["Cin"], l["Cout"], l["H"], l["W"], l["F"], classes, list(batches), stride=l["stride"],
+                                             maxpool=l["pool"], dtype=dt)
+        t = nf.nf_max_batch(slope, icpt, budget_bytes)
+        if t < 1:
+            raise ValueError(f"layer {len(max_batch)} does not fit the budget even at batch size 1")
+        max_batch.append(min(t, 2**31 - 1))
+    return nf.nf_partition(max_batch, batch_cap, rho)
+
+
 def evaluate_exits(nf, torch, layers, N, val_cur, val_labels):
     """Run the validation activations through the layers of one trained block, each layer as an exit.
     Returns ([correct count per layer], the block's output for the validation set)."""
@@ -129,10 +144,16 @@ def main():
     ap.add_argument("--epochs", type=int, default=3)
     ap.add_argument("--lr", type=float, default=0.01)
     ap.add_argument("--val-images", type=int, default=0, help="evaluate every layer as an exit on this many held-out images")
+    ap.add_argument("--budget-gb", type=float, default=0.0, help="re-plan the blocks with the Profiler and Algorithm 1 under this memory budget")
+    ap.add_argument("--rho", type=float, default=0.4)
     args = ap.parse_args()
     nf.lib()
     nf.nf_set_stream(torch.cuda.current_stream())
     wl = workloads.ALL[args.workload]()
+    if args.budget_gb > 0 and "layers" in wl:
+        plan = plan_blocks(nf, wl["layers"], wl["classes"], args.budget_gb * 1e9, args.images, args.rho, dtype=wl["dtype"])
+        print(json.dumps(dict(planned_blocks=plan)), flush=True)
+        wl = dict(wl, blocks=[(bs, wl["layers"][f:l + 1]) for f, l, bs in plan])
     C, H, W = wl["in_shape"]
     g = torch.Generator(device="cuda")
     g.manual_seed(0x4E460005)

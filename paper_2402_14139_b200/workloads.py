@@ -91,6 +91,28 @@ def c5(block_batches=None):
     return dict(name="c5", dtype="bf16", classes=200, in_shape=(3, 64, 64), blocks=blocks, layers=ls)
 
 
+def c6(block_batches=None):
+    """VGG-16-shaped net on 32x32x3, 100 classes, with the auxiliary filter counts of the AAN-LL rule (32 for the two
+    layers before the first down-sampling, 256 after).  The default blocks are what the Profiler calls of the library
+    (nf_profile_layer at batch sizes 32..256, nf_max_batch under a 2 GB budget) and Algorithm 1 (rho = 0.4, batch size
+    capped at the 50 000-image dataset) return: five blocks."""
+    chans = [v for v in VGG16 if v != "P"]
+    lo, hi = min(chans) // 2, max(chans) // 2
+    ls, S, Cin, k = [], 32, 3, 0
+    for i, v in enumerate(VGG16):
+        if v == "P":
+            continue
+        pool = i + 1 < len(VGG16) and VGG16[i + 1] == "P"
+        ls.append(_layer(Cin, v, S, S, lo if k < 2 else hi, pool=pool))
+        Cin, k = v, k + 1
+        if pool:
+            S //= 2
+    if block_batches is None:
+        block_batches = [(0, 2, 2978), (3, 5, 6309), (6, 8, 13576), (9, 9, 25799), (10, 12, 50000)]
+    blocks = [(bs, ls[f:l + 1]) for f, l, bs in block_batches]
+    return dict(name="c6", dtype="bf16", classes=100, in_shape=(3, 32, 32), blocks=blocks, layers=ls)
+
+
 def layer_bytes_per_image(l, classes, esize=2):
     """Device bytes one more image costs a layer of this library (stored activations and gradients):
     y, dy (conv output size), a, da (after pool), h, dh (aux conv output) plus the small head tensors."""
@@ -110,4 +132,4 @@ def step_flops(l, N):
     return dict(conv_fwd=main, wgrad=main, aux_fwd=aux, aux_bwd=2 * aux)
 
 
-ALL = dict(c1=c1, c2=c2, c3=c3, c4=c4, c5=c5, c4s=c4s)
+ALL = dict(c1=c1, c2=c2, c3=c3, c4=c4, c5=c5, c4s=c4s, c6=c6)

@@ -86,3 +86,45 @@ def test_select_exit_rule_matches_checker_on_the_host():
         acc = [round(float(v) * 4) / 4 for v in synth.uniform01(0x4E46E200, t, n)]     # many ties
         par = [int(v * 5) for v in synth.uniform01(0x4E46E201, t, n)]
         assert nf.nf_select_exit(acc, par) == nfo.select_exit(acc, par)
+
+
+def test_profiler_rule_line_fit_and_max_batch_on_the_host():
+    """The Profiler's three host steps against the checker and against what the paper states: the AAN-LL rule
+    (VGG: 32 filters before the first down-sampling, 256 after), the layer-wise linear memory model (the library's
+    own memory need is linear in the batch size up to alignment; its slope is the stored bytes per image) and the
+    largest batch under a budget."""
+    import numpy as np
+    from oracle import nfo
+    from paper_2402_14139_b200 import nf, workloads
+    vgg19 = [64, 64, 128, 128, 256, 256, 256, 256, 512, 512, 512, 512, 512, 512, 512, 512]
+    want = [32, 32] + [256] * 14                      # the paper's worked example for VGG
+    assert nf.nf_aan_filters(vgg19, 2) == want == nfo.aan_filters(vgg19, 2)
+    resnet = [64] * 5 + [128] * 4 + [256] * 4 + [512] * 4
+    assert nf.nf_aan_filters(resnet, 1) == nfo.aan_filters(resnet, 1) == [32] + [256] * 16
+    # checker's line fit against the library routine numpy offers, then the library against the checker
+    xs, ys = [8, 16, 32, 64, 96], [1.0e6, 1.9e6, 4.2e6, 8.1e6, 12.3e6]
+    sl, ic = nfo.fit_line(xs, ys)
+    ref = np.polyfit(xs, ys, 1)
+    assert abs(sl - ref[0]) <= 1e-9 * abs(ref[0]) and abs(ic - ref[1]) <= 1e-6 * abs(ref[1])
+    l = dict(Cin=64, Cout=64, H=32, W=32, F=32, stride=1, pool=True)
+    batches = [16, 32, 64, 128, 256]
+    by, slope, icpt = nf.nf_profile_layer(l["Cin"], l["Cout"], l["H"], l["W"], l["F"], 10, batches, maxpool=True)
+    s2, i2 = nfo.fit_line(batches, by)
+    assert abs(slope - s2) <= 1e-9 * s2 and abs(icpt - i2) <= 1e-6 * max(abs(i2), 1.0)
+    assert all(abs(b - (icpt + slope * n)) <= 0.01 * b for n, b in zip(batches, by))          # "linearly correlates with the batch size"
+    per_image = workloads.layer_bytes_per_image(l, 10)
+    assert abs(slope - per_image) <= 0.02 * per_image                                          # slope = stored bytes per image
+    for budget in (64e6, 630e6, 4e9):
+        t = nf.nf_max_batch(slope, icpt, budget)
+        assert t == nfo.max_batch_from_line(slope, icpt, budget)
+        assert icpt + slope * t <= budget < icpt + slope * (t + 1)
+    assert nf.nf_max_batch(slope, icpt, 0.0) == 0
+
+
+def test_planned_blocks_of_the_aan_workload_match_its_stored_default():
+    """The block list stored in the c6 workload is what the Profiler and Algorithm 1 of the library return."""
+    from paper_2402_14139_b200 import nf, pipeline, workloads
+    wl = workloads.c6()
+    assert [l["F"] for l in wl["layers"]] == nf.nf_aan_filters([l["Cout"] for l in wl["layers"]], 2)
+    plan = pipeline.plan_blocks(nf, wl["layers"], wl["classes"], 2e9, 50000, 0.4)
+    assert [(bs, len(ls)) for bs, ls in wl["blocks"]] == [(bs, l - f + 1) for f, l, bs in plan]

@@ -135,6 +135,11 @@ TC = [
     dict(N=9, Cin=128, Cout=128, H=8, W=8, F=16, classes=10, stride=1, pool=True),    # 8x8 maps: 2 images per tile (ragged), aux at 4x4
     dict(N=16, Cin=64, Cout=64, H=4, W=4, F=8, classes=10, stride=1, pool=False),     # 4x4 maps: 8 images per tile
     dict(N=12, Cin=64, Cout=128, H=16, W=16, F=32, classes=10, stride=2, pool=False), # stride 2 down to 8x8, multi-image tiles
+    dict(N=8, Cin=64, Cout=64, H=16, W=16, F=128, classes=10, stride=1, pool=False),    # more than 64 aux filters: main-conv kernels
+    dict(N=16, Cin=128, Cout=128, H=16, W=16, F=256, classes=100, stride=1, pool=True), # the classic setting of 256 aux filters
+    dict(N=200, Cin=64, Cout=64, H=2, W=2, F=32, classes=10, stride=1, pool=True),       # aux conv on 1x1 maps: 128 images per tile
+    dict(N=520, Cin=64, Cout=128, H=2, W=2, F=128, classes=10, stride=1, pool=True),     # the same with more than 64 aux filters
+    dict(N=300, Cin=64, Cout=64, H=1, W=1, F=16, classes=10, stride=1, pool=False),      # everything on 1x1 maps
 ]
 
 
@@ -145,6 +150,45 @@ def test_tensor_core_shapes_bf16(env, ci):
     P, x, y = pu.seeded_case(c, 1, bf16=True)
     G = pu.gpu_layer(nf, c, P, nf.NF_BF16)
     assert G.kernel_family(0) == "tcgen05" and G.kernel_family(1) == "tcgen05"
+    if c["F"] > 64 or c["H"] <= 2:
+        assert G.kernel_family(2) == "tcgen05" and G.kernel_family(3) == "tcgen05"
     G.close()
     w = pu.check_step(nf, torch, c, seed=400 + ci, dtype=nf.NF_BF16, lr=0.02, steps=2)
     print(w)
+
+
+LARGE_HEAD = [
+    (0, dict(N=600, Cin=8, Cout=16, H=4, W=4, F=32, classes=256, stride=1, pool=False)),      # fp32, 600*128*256 products
+    (1, dict(N=512, Cin=64, Cout=64, H=4, W=4, F=64, classes=128, stride=1, pool=False)),     # bf16 tensor-core layer
+    (1, dict(N=700, Cin=64, Cout=64, H=2, W=2, F=128, classes=100, stride=1, pool=True)),     # ragged tiles, 512 head inputs
+]
+
+
+@pytest.mark.parametrize("ci", range(len(LARGE_HEAD)))
+@pytest.mark.parametrize("loss", ["ce", "mse"])
+def test_large_batch_head(env, ci, loss):
+    """Batches large enough for the tiled head kernels (logits, dp and gWf as matrix products, the batch
+    reduction of gWf in ranges): whole steps against the checker, then the early-exit forward."""
+    nf, torch = env
+    dtype, c = LARGE_HEAD[ci]
+    c = dict(c, loss=loss)
+    pu.check_step(nf, torch, c, seed=900 + ci, dtype=dtype, lr=0.02, steps=2)
+    bf16 = dtype == 1
+    P, x, _ = pu.seeded_case(c, 950 + ci, bf16=bf16)
+    if c["Cin"] == 64:
+        x = np.maximum(x, 0.0)
+    O = pu.oracle_layer(c, P, store_bf16=bf16)
+    G = pu.gpu_layer(nf, c, P, nf.NF_BF16 if bf16 else nf.NF_F32)
+    _, logits_o, pred_o = O.predict(x)
+    logits_d = torch.zeros((c["N"], c["classes"]), device="cuda")
+    pred_d = torch.zeros(c["N"], dtype=torch.int32, device="cuda")
+    G.predict(pu.to_device_nhwc(torch, x, dtype), pred_d, logits_out=logits_d)
+    torch.cuda.synchronize()
+    tol = pu.TOL[dtype]["t"] * np.abs(logits_o).max()
+    lg = logits_d.cpu().numpy()
+    assert np.abs(lg - logits_o).max() <= tol
+    assert np.array_equal(pred_d.cpu().numpy(), np.argmax(lg, axis=1))
+    top2 = np.sort(logits_o, axis=1)[:, -2:]
+    decided = (top2[:, 1] - top2[:, 0]) > 2 * tol
+    assert decided.sum() > c["N"] // 8 and np.array_equal(pred_d.cpu().numpy()[decided], pred_o[decided])
+    G.close()
