@@ -8,6 +8,12 @@ previous block otherwise) and stepped through all layers of the block with nf_bl
 block has finished, its output for every sample is written to the cache by nf_block_cache (forward
 only, running statistics) and becomes the next block's input set.  Earlier blocks are never run again.
 
+Storage tier (the paper keeps the activation cache outside the GPU when it does not fit): with cache="host" the
+cache of every block lives in pinned host memory.  The cache fill copies each finished chunk to it asynchronously;
+training assembles batch k+1 with nf_cache_gather straight from the pinned rows on a second stream while
+batch k trains (two batch buffers, events between the streams), so the PCIe transfer hides behind the step.
+The gather is a bit-exact row copy, so both tiers give identical results.
+
 With a validation set, every trained layer is also evaluated as an exit point (nf_layer_predict on the
 validation activations that the earlier layers produced, nf_count_equal against the labels); the
 resulting (layer, accuracy, parameters) table goes through nf_select_exit.
@@ -75,8 +81,9 @@ def evaluate_exits(nf, torch, layers, N, val_cur, val_labels):
     return counts.cpu().tolist(), out
 
 
-def train_blockwise(nf, torch, wl, data, labels, epochs=1, lr=0.01, seed=1, log=None, val=None):
-    """data: device tensor [K, H, W, C] of the first layer's dtype; labels: device int32 [K];
+def train_blockwise(nf, torch, wl, data, labels, epochs=1, lr=0.01, seed=1, log=None, val=None, cache="hbm"):
+    """data: device (or pinned host) tensor [K, H, W, C] of the first layer's dtype; labels: device int32 [K];
+    cache: "hbm" keeps each block's output for all samples on the device, "host" in pinned host memory;
     val: optional (device tensor [V, H, W, C], device int32 [V]) validation set.
     Returns (per-block records, the last block's cached output) and, with val, also the exit report
     dict(table=[(layer, accuracy, parameters)], selected=layer index)."""
@@ -88,18 +95,41 @@ def train_blockwise(nf, torch, wl, data, labels, epochs=1, lr=0.01, seed=1, log=
         N = min(N, K)
         capped = dict(wl, blocks=[(N, l2) if i == bi else (n2, l2) for i, (n2, l2) in enumerate(wl["blocks"])])
         layers, block = build_layers(nf, capped, bi, seed)
-        xb = torch.empty((N,) + tuple(cur.shape[1:]), dtype=cur.dtype, device=cur.device)
-        yb = torch.empty(N, dtype=torch.int32, device=cur.device)
-        loss = torch.zeros(len(ls), dtype=torch.float32, device=cur.device)
+        dev = labels.device
+        bufs = [(torch.empty((N,) + tuple(cur.shape[1:]), dtype=cur.dtype, device=dev), torch.empty(N, dtype=torch.int32, device=dev))
+                for _ in range(2)]
+        loss = torch.zeros(len(ls), dtype=torch.float32, device=dev)
+        main, side = torch.cuda.current_stream(), torch.cuda.Stream()
+        ready = [torch.cuda.Event(), torch.cuda.Event()]      # batch buffer filled (side stream)
+        free = [torch.cuda.Event(), torch.cuda.Event()]       # batch buffer consumed (main stream)
+        perms = [torch.from_numpy(synth.permutation(seed + 7919 * bi, ep, K)).to(dev) for ep in range(epochs)]
+        per_ep = K // N
+        total = epochs * per_ep
+
+        def assemble(k):      # batch k into buffer k % 2, on the side stream
+            idx = perms[k // per_ep][(k % per_ep) * N:(k % per_ep + 1) * N].contiguous()
+            if k >= 2:
+                side.wait_event(free[k % 2])
+            nf.nf_set_stream(side)
+            nf.nf_cache_gather(cur, labels, idx, bufs[k % 2][0], bufs[k % 2][1])
+            ready[k % 2].record(side)
+            nf.nf_set_stream(main)
+            return idx        # kept alive by the caller until the gather has run
+
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        steps = 0
-        for ep in range(epochs):
-            perm = torch.from_numpy(synth.permutation(seed + 7919 * bi, ep, K)).to(cur.device)
-            for s in range(K // N):
-                nf.nf_cache_gather(cur, labels, perm[s * N:(s + 1) * N].contiguous(), xb, yb)
-                block.step(xb, yb, lr, loss)
-                steps += 1
+        steps, keep = 0, []
+        side.wait_stream(main)
+        if total:
+            keep.append(assemble(0))
+        for k in range(total):
+            if k + 1 < total:
+                keep.append(assemble(k + 1))
+            main.wait_event(ready[k % 2])
+            block.step(bufs[k % 2][0], bufs[k % 2][1], lr, loss)
+            free[k % 2].record(main)
+            steps += 1
+            keep = keep[-3:]
         torch.cuda.synchronize()
         t_train = time.perf_counter() - t0
         status = [L.status() for L in layers]
@@ -107,11 +137,24 @@ def train_blockwise(nf, torch, wl, data, labels, epochs=1, lr=0.01, seed=1, log=
             raise RuntimeError(f"block {bi}: device status {status}")
         # fill the cache: the block's output for every sample, in chunks of the block's batch size
         last = layers[-1]
-        out = torch.empty((K, last.Ha, last.Wa, last.Cout), dtype=cur.dtype, device=cur.device)
+        oshape = (K, last.Ha, last.Wa, last.Cout)
+        host = cache == "host"
+        out = torch.empty(oshape, dtype=cur.dtype, pin_memory=True) if host else torch.empty(oshape, dtype=cur.dtype, device=dev)
+        stage_in = torch.empty((N,) + tuple(cur.shape[1:]), dtype=cur.dtype, device=dev) if not cur.is_cuda else None
+        stage_out = [torch.empty((N,) + oshape[1:], dtype=cur.dtype, device=dev) for _ in range(2)] if host else None
         t1 = time.perf_counter()
-        for s in range(0, K, N):
+        for ci, s in enumerate(range(0, K, N)):
             cnt = min(N, K - s)
-            block.cache(cur[s:s + cnt], out[s:s + cnt], count=cnt)
+            src = cur[s:s + cnt]
+            if stage_in is not None:      # the block's input set lives in host memory: bring the chunk in
+                stage_in[:cnt].copy_(src, non_blocking=True)
+                src = stage_in[:cnt]
+            if host:                      # forward into a device chunk, then an asynchronous copy to the pinned cache
+                so = stage_out[ci % 2]
+                block.cache(src, so[:cnt], count=cnt)
+                out[s:s + cnt].copy_(so[:cnt], non_blocking=True)
+            else:
+                block.cache(src, out[s:s + cnt], count=cnt)
         torch.cuda.synchronize()
         t_cache = time.perf_counter() - t1
         rec = dict(block=bi, layers=len(ls), batch=N, steps=steps, train_s=round(t_train, 4), cache_s=round(t_cache, 4),
@@ -146,6 +189,7 @@ def main():
     ap.add_argument("--val-images", type=int, default=0, help="evaluate every layer as an exit on this many held-out images")
     ap.add_argument("--budget-gb", type=float, default=0.0, help="re-plan the blocks with the Profiler and Algorithm 1 under this memory budget")
     ap.add_argument("--rho", type=float, default=0.4)
+    ap.add_argument("--cache", default="hbm", choices=["hbm", "host"], help="where the activation cache of a finished block lives")
     args = ap.parse_args()
     nf.lib()
     nf.nf_set_stream(torch.cuda.current_stream())
@@ -166,7 +210,7 @@ def main():
                torch.randint(0, wl["classes"], (args.val_images,), generator=g, device="cuda", dtype=torch.int32))
     t0 = time.perf_counter()
     res = train_blockwise(nf, torch, wl, data, labels, epochs=args.epochs, lr=args.lr, log=lambda r: print(json.dumps(r), flush=True),
-                          val=val)
+                          val=val, cache=args.cache)
     wall = time.perf_counter() - t0
     if val:
         print(json.dumps(dict(exit_table=[(l, round(a, 4), p) for l, a, p in res[2]["table"]], selected_exit=res[2]["selected"])))

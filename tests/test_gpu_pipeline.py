@@ -64,3 +64,25 @@ def test_exit_evaluation_over_the_blockwise_pass():
     assert [t[2] for t in table] == [main[0] + aux[0], main[0] + main[1] + aux[1], sum(main) + aux[2]]
     assert ex["selected"] == nfo.select_exit([t[1] for t in table], [t[2] for t in table])
     assert max(t[1] for t in table) >= 0.9
+
+
+def test_host_cache_tier_gives_identical_results():
+    """The activation cache in pinned host memory (asynchronous fill, batches gathered from it on a second stream
+    while the previous batch trains) is a storage choice only: final cache and losses are bit-identical to the
+    run that keeps the cache on the device, also when the dataset itself sits in host memory."""
+    import torch
+    from paper_2402_14139_b200 import nf
+    nf.lib()
+    nf.nf_set_stream(None)
+    K = 24
+    x = synth.round_bf16(synth.normal(6, 1, (K, 16, 16, 3)))
+    data = torch.from_numpy(x).cuda().to(torch.bfloat16)
+    labels = torch.from_numpy(synth.labels(6, 2, K, 4)).cuda()
+    r0, out0 = pipeline.train_blockwise(nf, torch, _wl(), data, labels, epochs=3, lr=0.05, seed=3)
+    r1, out1 = pipeline.train_blockwise(nf, torch, _wl(), data, labels, epochs=3, lr=0.05, seed=3, cache="host")
+    r2, out2 = pipeline.train_blockwise(nf, torch, _wl(), data.cpu().pin_memory(), labels, epochs=3, lr=0.05, seed=3, cache="host")
+    assert out0.is_cuda and not out1.is_cuda and out1.is_pinned()
+    for r, out in ((r1, out1), (r2, out2)):
+        assert [b["losses"] for b in r] == [b["losses"] for b in r0]
+        assert torch.equal(out.cuda().view(torch.int16), out0.view(torch.int16))
+    nf.nf_set_stream(None)
