@@ -160,6 +160,23 @@ void nf_block_destroy(nf_block* block);
 int nf_block_cache(nf_block* block, const void* x, void* out);
 int nf_block_cache_n(nf_block* block, const void* x, void* out, int count);
 
+/* Data-parallel local step (the paper names distributed training as the direction beyond a single device): the batch
+ * of N * world samples is sharded over `world` ranks, every rank holds N of them and a full copy of the layer, and
+ * BatchNorm uses the statistics of the WHOLE batch, so the result equals nf_layer_step on the whole batch (up to
+ * summation order).  The step is cut where ranks must exchange sums; between phases the caller adds the buffer
+ * nf_layer_dp_buffer names over all ranks (an all-reduce sum, in place):
+ *   phase 0: conv forward, this rank's per-channel sums of y and y^2      -> all-reduce buffer 0 (2*Cout doubles)
+ *   phase 1: normalise, auxiliary forward, loss, auxiliary backward, this rank's BatchNorm-backward sums
+ *                                                                          -> all-reduce buffer 1 (2*Cout doubles)
+ *   phase 2: BatchNorm backward, weight gradient                           -> all-reduce buffer 2 (every parameter
+ *            gradient, fp32) and *loss_out (this rank's share of the mean loss)
+ *   phase 3: momentum update (identical on every rank).
+ * Same arguments in every phase; x, labels, act_out are this rank's shard.  NF_EINVAL for an unknown phase or world < 1. */
+int nf_layer_step_dp(nf_layer* layer, int phase, const void* x, const int32_t* labels, float lr, float* loss_out, void* act_out,
+                     int world);
+/* Device address and size of exchange buffer `which` (0, 1, 2 as above) inside the bound workspace. */
+int nf_layer_dp_buffer(nf_layer* layer, int which, void** dev_ptr, size_t* bytes);
+
 /* Early-exit evaluation (Section "Trained output CNN": every layer with its auxiliary network is a
  * prospective exit point).  Forward only, BatchNorm with running statistics, no parameter changes:
  *   act_out = x_{n+1} for `count` samples (device, [count][Ha][Wa][Cout]; NULL keeps it in the workspace),

@@ -105,6 +105,7 @@ size_t plan(nf_layer* L, char* base, bool assign) {
   D->p = (float*)c.take(N * 4 * F * 4);
   D->dp = (float*)c.take(N * 4 * F * 4);
   D->parg = (int32_t*)c.take(N * 4 * F * 4);
+  D->dptot = (double*)c.take(4 * Co * 8);
   D->logits = (float*)c.take(N * K * 4);
   D->dlogits = (float*)c.take(N * K * 4);
   D->lossn = (float*)c.take(N * 4);
@@ -324,19 +325,26 @@ int nf_layer_get_param(nf_layer* L, int which, float* host, size_t n) {
     if (rc_ != NF_OK) return rc_; \
   } while (0)
 
-int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, float* loss_out, void* act_out) {
+// The whole step (phase < 0, world = 1), or one of the four phases of the data-parallel step: 0 = conv forward and
+// the rank's per-channel sums; 1 = normalise with the statistics of the whole batch ... aux input gradient and the
+// rank's BatchNorm-backward sums; 2 = BatchNorm backward with the sums of the whole batch, weight gradient; 3 = update.
+static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float lr, float* loss_out, void* act_out, int phase,
+                       int world) {
   if (!L || !x || !labels || !loss_out || !act_out) return NF_EINVAL;
   if (!L->ws) return NF_ENOWS;
   if (misaligned(x) || misaligned(act_out) || ((uintptr_t)labels & 3) || ((uintptr_t)loss_out & 3)) return NF_EALIGN;
   const int dt = L->o.dtype, N = L->o.N, Ci = L->Cin, Co = L->Cout, F = L->F, K = L->classes, s = L->o.stride;
   const int pool = L->o.maxpool, Ho = L->Ho, Wo = L->Wo, Ha = L->Ha, Wa = L->Wa, D = 4 * F;
-  const double M = (double)N * Ho * Wo;
+  const double M = (double)N * Ho * Wo * world;   // BatchNorm sample count of the whole batch
+  const int n_scale = N * world;                  // batch size in the loss mean
+  const bool all = phase < 0;
   const void* Wm = dt == NF_F32 ? (const void*)(L->val + L->off[NF_P_W]) : (const void*)(L->shadow + L->off[NF_P_W]);
   const void* Wx = dt == NF_F32 ? (const void*)(L->val + L->off[NF_P_WA]) : (const void*)(L->shadow + L->off[NF_P_WA]);
   float* g = L->grad;
   int nb = 0;
 
   // Eq. 1: conv, BatchNorm (batch statistics), ReLU, optional max-pool -> act_out
+  if (all || phase == 0) {
   trace_begin(0);
   if (L->fam[0]) {
     NF_TRY(nf_tc_conv_fwd(L, x, nb));
@@ -345,9 +353,17 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
     NF_TRY(nf_ref_channel_sums(dt, L->y, (size_t)N * Ho * Wo, Co, L->red, L->red_floats, &nb));
   }
   trace_end();
+  if (!all) return nf_ref_partial_totals(L->red, nb, Co, L->dptot);
+  }
+  if (all || phase == 1) {
   trace_begin(1);
-  NF_TRY(nf_ref_bn_finalize(L->red, nb, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
-                            L->o.bn_momentum, L->scale, L->shift, L->mu, L->invstd, L->rmean, L->rvar));
+  if (all) {
+    NF_TRY(nf_ref_bn_finalize(L->red, nb, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
+                              L->o.bn_momentum, L->scale, L->shift, L->mu, L->invstd, L->rmean, L->rvar));
+  } else {
+    NF_TRY(nf_ref_bn_finalize_tot(L->dptot, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
+                                  L->o.bn_momentum, L->scale, L->shift, L->mu, L->invstd, L->rmean, L->rvar));
+  }
   NF_TRY(nf_ref_bn_apply(dt, L->y, N, Ho, Wo, Co, pool, L->scale, L->shift, act_out));
   trace_end();
   // Eq. 2: aux conv + ReLU, average pool to 2x2, linear; Eq. 3: softmax cross-entropy
@@ -369,12 +385,12 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
   if (nf_head_is_large(N, D, K)) {  // late blocks: tens of thousands of samples, up to 1024 head inputs
     NF_TRY(nf_head_step(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits, L->dp,
                         L->lossn, L->status, L->o.loss, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->wpart,
-                        L->wpart_floats));
+                        L->wpart_floats, n_scale));
   } else {
     NF_TRY(nf_ref_fc_ce(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits,
-                        L->dp, L->lossn, L->status, L->o.loss));
+                        L->dp, L->lossn, L->status, L->o.loss, n_scale));
     // gradients of gamma_n
-    NF_TRY(nf_ref_fc_wgrad(L->p, L->dlogits, L->lossn, N, D, K, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->status));
+    NF_TRY(nf_ref_fc_wgrad(L->p, L->dlogits, L->lossn, N, D, K, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->status, n_scale));
   }
   trace_end();
   trace_begin(4);
@@ -415,7 +431,14 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
     NF_TRY(nf_ref_bn_bwd_reduce(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->red,
                                 L->red_floats, &nb));
   }
-  NF_TRY(nf_ref_bn_bwd_finalize(L->red, nb, Co, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
+  if (!all) return nf_ref_partial_totals(L->red, nb, Co, L->dptot + 2 * Co);
+  }
+  if (all || phase == 2) {
+  if (all) {
+    NF_TRY(nf_ref_bn_bwd_finalize(L->red, nb, Co, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
+  } else {
+    NF_TRY(nf_ref_bn_bwd_finalize_tot(L->dptot + 2 * Co, Co, world, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
+  }
   NF_TRY(nf_ref_bn_bwd_apply(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->sdz, L->sdzx,
                              M, L->dy));
   trace_end();
@@ -427,9 +450,34 @@ int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, f
     NF_TRY(nf_ref_wgrad(dt, x, N, L->H, L->W, Ci, L->dy, Co, s, L->wpart, L->wpart_floats, g + L->off[NF_P_W]));
   }
   trace_end();
+  if (!all) return NF_OK;
+  }
   trace_begin(7);
   NF_TRY(nf_ref_sgd(L->val, L->mom, L->grad, L->shadow, L->arena, lr, L->o.momentum));
   trace_end();
+  return NF_OK;
+}
+
+int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, float* loss_out, void* act_out) {
+  return step_phases(L, x, labels, lr, loss_out, act_out, -1, 1);
+}
+
+int nf_layer_step_dp(nf_layer* L, int phase, const void* x, const int32_t* labels, float lr, float* loss_out, void* act_out,
+                     int world) {
+  if (phase < 0 || phase > 3 || world < 1) return NF_EINVAL;
+  return step_phases(L, x, labels, lr, loss_out, act_out, phase, world);
+}
+
+int nf_layer_dp_buffer(nf_layer* L, int which, void** dev_ptr, size_t* bytes) {
+  if (!L || !dev_ptr || !bytes || which < 0 || which > 2) return NF_EINVAL;
+  if (!L->ws) return NF_ENOWS;
+  if (which == 2) {
+    *dev_ptr = L->grad;
+    *bytes = L->arena * sizeof(float);
+  } else {
+    *dev_ptr = L->dptot + (size_t)which * 2 * L->Cout;
+    *bytes = (size_t)2 * L->Cout * sizeof(double);
+  }
   return NF_OK;
 }
 

@@ -75,7 +75,7 @@ __global__ void head_finish_kernel(const float* __restrict__ part, int Z, size_t
 // One warp per sample: the loss of Eq. 3 on a row of logits, its derivative dlogits, the per-sample loss.
 __global__ void __launch_bounds__(256) head_loss_rows_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int N,
                                                              int K, int loss_kind, float* __restrict__ dlogits,
-                                                             float* __restrict__ lossn, int32_t* status) {
+                                                             float* __restrict__ lossn, int32_t* status, int n_scale) {
   const int n = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (n >= N) return;
   const float* l = logits + (size_t)n * K;
@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(256) head_loss_rows_kernel(const float* __rest
   }
   if (loss_kind == 1) {
     float se = 0.f;
-    const float sc = 2.f / ((float)N * (float)K);
+    const float sc = 2.f / ((float)n_scale * (float)K);
     for (int k = lane; k < K; k += 32) {
       const float e = l[k] - (k == lab ? 1.f : 0.f);
       se = fmaf(e, e, se);
@@ -108,14 +108,15 @@ __global__ void __launch_bounds__(256) head_loss_rows_kernel(const float* __rest
   for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
   const float lse = mx + logf(se);
   if (lane == 0) lossn[n] = lse - l[lab];
-  const float invN = 1.f / (float)N;
+  const float invN = 1.f / (float)n_scale;
   for (int k = lane; k < K; k += 32) g[k] = (expf(l[k] - lse) - (k == lab ? 1.f : 0.f)) * invN;
 }
 
 // gbf[k] = sum_n dlogits[n][k] (32 columns x 8 row lanes per block, lanes added in order);
 // block 0 also reduces the per-sample losses in fp64 (256 lanes, then a fixed tree).
 __global__ void __launch_bounds__(256) head_colsum_loss_kernel(const float* __restrict__ dl, const float* __restrict__ lossn, int N, int K,
-                                                               float* __restrict__ gbf, float* __restrict__ loss_out, int32_t* status) {
+                                                               float* __restrict__ gbf, float* __restrict__ loss_out, int32_t* status,
+                                                               int n_scale) {
   __shared__ float sm[8][33];
   __shared__ double sd[256];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
@@ -141,7 +142,7 @@ __global__ void __launch_bounds__(256) head_colsum_loss_kernel(const float* __re
       __syncthreads();
     }
     if (threadIdx.x == 0) {
-      const float L = (float)(sd[0] / (double)N);
+      const float L = (float)(sd[0] / (double)n_scale);
       *loss_out = L;
       if (!isfinite(L)) atomicOr(status, NF_ENONFINITE);
     }
@@ -200,11 +201,11 @@ size_t nf_head_scratch_floats(int N, int D, int K) {
 
 int nf_head_step(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf, float* logits,
                  float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind, float* gWf, float* gbf, float* loss_out,
-                 float* scratch, size_t scratch_floats) {
+                 float* scratch, size_t scratch_floats, int n_scale) {
   if (scratch_floats < nf_head_scratch_floats(N, D, K)) return NF_ENOWS;
   int rc = nf_head_logits(p, N, D, K, Wf, bf, logits, scratch);
   if (rc != NF_OK) return rc;
-  head_loss_rows_kernel<<<(N + 7) / 8, 256, 0, g_nf_stream>>>(logits, labels, N, K, loss_kind, dlogits, lossn, status);
+  head_loss_rows_kernel<<<(N + 7) / 8, 256, 0, g_nf_stream>>>(logits, labels, N, K, loss_kind, dlogits, lossn, status, n_scale);
   NF_LAUNCHED();
   // dp[n][d] = sum_k dlogits[n][k] Wf[k][d]
   if ((rc = gemm(dlogits, K, 1, Wf, D, 1, N, D, K, 1, dp)) != NF_OK) return rc;
@@ -218,7 +219,7 @@ int nf_head_step(const float* p, const int32_t* labels, int N, int D, int K, con
   if ((rc = gemm(dlogits, 1, K, p, D, 1, K, D, N, Z, scratch)) != NF_OK) return rc;
   head_finish_kernel<<<(unsigned)((kd + 255) / 256), 256, 0, g_nf_stream>>>(scratch, Z, kd, D, nullptr, gWf);
   NF_LAUNCHED();
-  head_colsum_loss_kernel<<<(K + 31) / 32, 256, 0, g_nf_stream>>>(dlogits, lossn, N, K, gbf, loss_out, status);
+  head_colsum_loss_kernel<<<(K + 31) / 32, 256, 0, g_nf_stream>>>(dlogits, lossn, N, K, gbf, loss_out, status, n_scale);
   NF_LAUNCHED();
   return NF_OK;
 }

@@ -43,6 +43,7 @@ struct nf_layer {
   void* da;                            // [N][Ha][Wa][Cout]
   void* act;                           // [N][Ha][Wa][Cout] activation kept here when the caller gives no buffer
   float *p, *dp;                       // [N][4F]
+  double* dptot;                       // [2][2][Cout] per-channel totals exchanged between ranks (data-parallel step)
   int32_t* parg;                       // [N][4F] position i*Wa+j of each bin's maximum (max-pool down-sampling only)
   float *logits, *dlogits;             // [N][classes]
   float* lossn;                        // [N]
@@ -101,7 +102,7 @@ int nf_ref_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part
 int nf_ref_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh, float* red, size_t red_floats,
                    int* nblocks);
 int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
-                 float* logits, float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind);
+                 float* logits, float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind, int n_scale);
 int nf_ref_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count);
 int nf_ref_auxmax(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p, int32_t* parg);
 int nf_ref_dh_max(int dtype, const void* h, const float* dp, const int32_t* parg, int N, int Ha, int Wa, int F, void* dh);
@@ -113,10 +114,14 @@ int nf_head_logits(const float* p, int N, int D, int K, const float* Wf, const f
 int nf_head_predict(const float* logits, int N, int K, int32_t* pred);
 int nf_head_step(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf, float* logits,
                  float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind, float* gWf, float* gbf, float* loss_out,
-                 float* scratch, size_t scratch_floats);
+                 float* scratch, size_t scratch_floats, int n_scale);
+int nf_ref_partial_totals(const float* red, int nblocks, int C, double* tot);
+int nf_ref_bn_finalize_tot(const double* tot, int C, double M, const float* gamma, const float* beta, float eps, float bn_momentum,
+                           float* scale, float* shift, float* mu, float* invstd, float* rmean, float* rvar);
+int nf_ref_bn_bwd_finalize_tot(const double* tot, int C, int world, float* sdz, float* sdzx, float* ggamma, float* gbeta);
 int nf_ref_fc_predict(const float* p, int N, int D, int K, const float* Wf, const float* bf, float* logits, int32_t* pred);
 int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
-                    float* gbf, float* loss_out, int32_t* status);
+                    float* gbf, float* loss_out, int32_t* status, int n_scale);
 int nf_ref_dh(int dtype, const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh);
 int nf_ref_sum_partials(const float* red, int nblocks, int C, int which, float* out);
 int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,

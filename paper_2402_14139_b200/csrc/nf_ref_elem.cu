@@ -152,6 +152,46 @@ __global__ void bn_finalize_kernel(const float* __restrict__ red, int nb, int C,
   }
 }
 
+// Data-parallel BatchNorm: a rank turns its per-block partials into per-channel totals (fp64, [2][C]) that the
+// ranks add up; the statistics and the backward sums are then finished from the totals of the whole batch.
+__global__ void partial_totals_kernel(const float* __restrict__ red, int nb, int C, double* __restrict__ tot) {
+  double S, Q;
+  reduce_partials32(red, nb, C, S, Q);
+  const int c = blockIdx.x * 32 + threadIdx.x;
+  if (c >= C || threadIdx.y != 0) return;
+  tot[c] = S;
+  tot[C + c] = Q;
+}
+
+__global__ void bn_finalize_tot_kernel(const double* __restrict__ tot, int C, double M, const float* __restrict__ gamma,
+                                       const float* __restrict__ beta, float eps, float bnm, float* scale, float* shift, float* mu,
+                                       float* invstd, float* rmean, float* rvar) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  const double m = tot[c] / M;
+  double v = tot[C + c] / M - m * m;
+  if (v < 0.0) v = 0.0;
+  const double is = 1.0 / sqrt(v + (double)eps);
+  scale[c] = (float)((double)gamma[c] * is);
+  shift[c] = (float)((double)beta[c] - m * (double)gamma[c] * is);
+  mu[c] = (float)m;
+  invstd[c] = (float)is;
+  rmean[c] = (float)((1.0 - bnm) * (double)rmean[c] + (double)bnm * m);
+  const double unb = M > 1.0 ? v * M / (M - 1.0) : v;
+  rvar[c] = (float)((1.0 - bnm) * (double)rvar[c] + (double)bnm * unb);
+}
+
+// the gradients of gamma and beta are divided by the number of ranks: the sum over ranks that follows restores them
+__global__ void bn_bwd_finalize_tot_kernel(const double* __restrict__ tot, int C, double inv_world, float* sdz, float* sdzx, float* gg,
+                                           float* gb) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  sdz[c] = (float)tot[c];
+  sdzx[c] = (float)tot[C + c];
+  gb[c] = (float)(tot[c] * inv_world);
+  gg[c] = (float)(tot[C + c] * inv_world);
+}
+
 __global__ void bn_eval_coeffs_kernel(int C, const float* gamma, const float* beta, float eps, const float* rmean,
                                       const float* rvar, float* scale, float* shift) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -302,7 +342,7 @@ __global__ void __launch_bounds__(256) fc_ce_kernel(const float* __restrict__ p,
                                                     int D, int K, const float* __restrict__ Wf, const float* __restrict__ bf,
                                                     float* __restrict__ logits, float* __restrict__ dlogits,
                                                     float* __restrict__ dp, float* __restrict__ lossn, int32_t* status,
-                                                    int loss_kind) {
+                                                    int loss_kind, int n_scale) {
   extern __shared__ float dyn[];
   float* ps = dyn;          // [D]
   float* ls = dyn + D;      // [K]
@@ -328,7 +368,7 @@ __global__ void __launch_bounds__(256) fc_ce_kernel(const float* __restrict__ p,
   if (loss_kind == 1) {
     // mean squared error against the one-hot target: lossn = sum_k e^2 / K, dlogits = 2 e / (N K)
     float se = 0.f;
-    const float sc = 2.f / ((float)N * (float)K);
+    const float sc = 2.f / ((float)n_scale * (float)K);
     for (int k = t; k < K; k += 256) {
       const float e = ls[k] - (k == lab ? 1.f : 0.f);
       se = fmaf(e, e, se);
@@ -343,7 +383,7 @@ __global__ void __launch_bounds__(256) fc_ce_kernel(const float* __restrict__ p,
     se = block_reduce(se, red, false);
     const float lse = mx + logf(se);
     if (t == 0) lossn[n] = lse - ls[lab];
-    const float invN = 1.f / (float)N;
+    const float invN = 1.f / (float)n_scale;
     for (int k = t; k < K; k += 256) {
       const float g = (expf(ls[k] - lse) - (k == lab ? 1.f : 0.f)) * invN;
       ls[k] = g;
@@ -424,7 +464,7 @@ __global__ void __launch_bounds__(256) fc_predict_kernel(const float* __restrict
 __global__ void __launch_bounds__(256) fc_wgrad_kernel(const float* __restrict__ p, const float* __restrict__ dl,
                                                        const float* __restrict__ lossn, int N, int D, int K,
                                                        float* __restrict__ gWf, float* __restrict__ gbf,
-                                                       float* __restrict__ loss_out, int32_t* status) {
+                                                       float* __restrict__ loss_out, int32_t* status, int n_scale) {
   const int k = blockIdx.x, t = threadIdx.x;
   for (int d = t; d < D; d += 256) {
     float s = 0.f;
@@ -439,7 +479,7 @@ __global__ void __launch_bounds__(256) fc_wgrad_kernel(const float* __restrict__
   if (k == 0 && t == 32) {
     double s = 0.0;
     for (int n = 0; n < N; ++n) s += (double)lossn[n];
-    const float L = (float)(s / (double)N);
+    const float L = (float)(s / (double)n_scale);
     *loss_out = L;
     if (!isfinite(L)) atomicOr(status, NF_ENONFINITE);
   }
@@ -1100,6 +1140,26 @@ int nf_ref_bn_finalize(const float* red, int nblocks, int C, double M, const flo
   return NF_OK;
 }
 
+int nf_ref_partial_totals(const float* red, int nblocks, int C, double* tot) {
+  partial_totals_kernel<<<nblk(C, 32), dim3(32, 32), 0, g_nf_stream>>>(red, nblocks, C, tot);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_bn_finalize_tot(const double* tot, int C, double M, const float* gamma, const float* beta, float eps, float bn_momentum,
+                           float* scale, float* shift, float* mu, float* invstd, float* rmean, float* rvar) {
+  bn_finalize_tot_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(tot, C, M, gamma, beta, eps, bn_momentum, scale, shift, mu, invstd,
+                                                                rmean, rvar);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_ref_bn_bwd_finalize_tot(const double* tot, int C, int world, float* sdz, float* sdzx, float* ggamma, float* gbeta) {
+  bn_bwd_finalize_tot_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(tot, C, 1.0 / (double)world, sdz, sdzx, ggamma, gbeta);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
 int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float eps, const float* rmean,
                           const float* rvar, float* scale, float* shift) {
   bn_eval_coeffs_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(C, gamma, beta, eps, rmean, rvar, scale, shift);
@@ -1174,10 +1234,10 @@ int nf_ref_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float
 }
 
 int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
-                 float* logits, float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind) {
+                 float* logits, float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind, int n_scale) {
   const size_t smem = (size_t)(D + K) * sizeof(float);
   if (smem > 40000) return NF_EUNSUPPORTED;
-  fc_ce_kernel<<<N, 256, smem, g_nf_stream>>>(p, labels, N, D, K, Wf, bf, logits, dlogits, dp, lossn, status, loss_kind);
+  fc_ce_kernel<<<N, 256, smem, g_nf_stream>>>(p, labels, N, D, K, Wf, bf, logits, dlogits, dp, lossn, status, loss_kind, n_scale);
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -1206,8 +1266,8 @@ int nf_ref_fc_predict(const float* p, int N, int D, int K, const float* Wf, cons
 }
 
 int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
-                    float* gbf, float* loss_out, int32_t* status) {
-  fc_wgrad_kernel<<<K, 256, 0, g_nf_stream>>>(p, dlogits, lossn, N, D, K, gWf, gbf, loss_out, status);
+                    float* gbf, float* loss_out, int32_t* status, int n_scale) {
+  fc_wgrad_kernel<<<K, 256, 0, g_nf_stream>>>(p, dlogits, lossn, N, D, K, gWf, gbf, loss_out, status, n_scale);
   NF_LAUNCHED();
   return NF_OK;
 }

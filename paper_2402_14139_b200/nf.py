@@ -27,7 +27,7 @@ PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P
 EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_layer_workspace_bytes",
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
-           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_max_batch", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
+           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_max_batch", "nf_layer_step_dp", "nf_layer_dp_buffer", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
            "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_op_status", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
@@ -76,6 +76,8 @@ def lib():
         L.nf_layer_param_count.restype = C.c_longlong
         L.nf_layer_param_count.argtypes = [vp, C.c_int]
         L.nf_count_equal.argtypes = [ip, ip, C.c_longlong, vp]
+        L.nf_layer_step_dp.argtypes = [vp, C.c_int, vp, ip, C.c_float, fp, vp, C.c_int]
+        L.nf_layer_dp_buffer.argtypes = [vp, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
         L.nf_aan_filters.argtypes = [C.POINTER(C.c_int), C.c_int, C.c_int, C.POINTER(C.c_int)]
         L.nf_profile_layer.argtypes = [C.c_int] * 6 + [C.POINTER(nf_layer_opts), C.POINTER(C.c_int), C.c_int, C.POINTER(C.c_double),
                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]
@@ -271,6 +273,23 @@ class Layer:
         """nf_layer_predict: early-exit forward for `count` (default N) samples; device tensors."""
         _check(lib().nf_layer_predict(self.h, _ptr(x), int(self.N if count is None else count), _ptr(act_out), _ptr(logits_out),
                                       _ptr(pred_out)), "nf_layer_predict")
+
+    def dp_buffer(self, which):
+        """The exchange buffer `which` of the data-parallel step as a tensor view of the workspace (float64 for 0 and 1, float32 for 2)."""
+        ptr, nbytes = C.c_void_p(), C.c_size_t()
+        _check(lib().nf_layer_dp_buffer(self.h, which, C.byref(ptr), C.byref(nbytes)), "nf_layer_dp_buffer")
+        off = ptr.value - self.ws.data_ptr()
+        return self.ws[off:off + nbytes.value].view(self._torch.float64 if which < 2 else self._torch.float32)
+
+    def step_dp(self, x, labels, lr, loss_out, act_out, world, all_reduce):
+        """nf_layer_step_dp through its four phases; all_reduce(tensor) must add the tensor over all ranks in place."""
+        for phase in range(4):
+            _check(lib().nf_layer_step_dp(self.h, phase, _ptr(x), _ptr(labels), float(lr), _ptr(loss_out), _ptr(act_out), int(world)),
+                   "nf_layer_step_dp")
+            if phase < 3:
+                all_reduce(self.dp_buffer(phase))
+            if phase == 2:
+                all_reduce(loss_out)
 
     def param_count(self, part=2) -> int:
         return int(lib().nf_layer_param_count(self.h, part))
