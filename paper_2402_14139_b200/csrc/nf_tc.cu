@@ -972,6 +972,135 @@ conv_wgrad_kw_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   }
 }
 
+// ---------------------------------------------------------------- weight gradient, stride 1, few filters: gradient on the M side
+// An instruction holds the tensor pipe for about the same time whatever its shape, so for the auxiliary conv
+// (F <= 32 filters) the fewest instructions win.  Here the roles of conv_wgrad_kw_kernel are swapped:
+//   A (M = 4 * NB rows) = the three column-shifted gradient tiles as consecutive MN-major atoms (kw, f) plus one unused atom,
+//   B (N = 192)         = the three row taps of the activation box as consecutive 64-channel atoms (kh, ci),
+// so ONE instruction per 16 pixels produces all nine taps: D[(kw, f), (kh, ci)].  NB = 16 uses the 64-row shape
+// (row r in TMEM lane 32 * (r / 16) + r % 16), NB = 32 the 128-row shape (row r in lane r); in both, the warp of
+// lane quadrant q holds column tap kw = q and lane l holds filter f = l.
+template <int NB>
+__global__ void __launch_bounds__(kThreads, 1)
+conv_wgrad_gx_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_dy, const WgParams p) {
+  constexpr int kBRow = NB * 2;
+  constexpr uint32_t kGLayout = NB == 32 ? 4 : 6;
+  constexpr int kGTile = 128 * kBRow;                 // one shifted gradient tile
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int box_bytes = (p.BH + 2) * p.BW * 128;
+  const int stage_bytes = box_bytes + 4 * kGTile;     // the fourth atom is never loaded: its accumulator rows are not read
+  const int stages = p.stages;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + kMaxStages;
+  uint64_t* done = bars + 2 * kMaxStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  constexpr uint32_t kCols = 256;                     // 192 accumulator columns
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cic = blockIdx.x % p.ci_chunks, sp = blockIdx.x / p.ci_chunks;
+  const int t0 = (int)((long)p.pix_tiles * sp / p.splits), t1 = (int)((long)p.pix_tiles * (sp + 1) / p.splits);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    ptx::mbar_init(done, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tmap(&tm_x);
+    ptx::prefetch_tmap(&tm_dy);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    uint32_t it = 0;
+    for (int t = t0; t < t1; ++t, ++it) {
+      const int s = it % stages;
+      const uint32_t ph = (it / stages) & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) break;
+      if (lane == 0) {
+        const int w0 = (t % p.tiles_w) * p.BW, h0 = ((t / p.tiles_w) % p.tiles_h) * p.BH, n = t / (p.tiles_w * p.tiles_h);
+        uint8_t* st = smem + (size_t)s * stage_bytes;
+        ptx::mbar_expect_tx(&full[s], (uint32_t)(box_bytes + 3 * kGTile));
+        ptx::tma_load_4d(st, &tm_x, &full[s], cic * 64, w0, h0 - 1, n);
+#pragma unroll
+        for (int kw = 0; kw < 3; ++kw)  // gradient column j = j' - kw + 1
+          ptx::tma_load_4d(st + box_bytes + kw * kGTile, &tm_dy, &full[s], 0, w0 - kw + 1, h0, n);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    constexpr uint32_t idesc = ptx::idesc_bf16(4 * NB, 192, 1, 1);
+    const uint64_t a_hi = ptx::sdesc(0, kGTile, 8 * kBRow, kGLayout);  // next M atom: next shifted tile
+    const uint64_t b_hi = ptx::sdesc(0, p.BW * 128, 1024, 2);          // next N atom: one image row further (next kh)
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = t0; t < t1; ++t, ++it) {
+      const int s = it % stages;
+      const uint32_t ph = (it / stages) & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[s], ph, abort_flag))) { ok = false; break; }
+      ptx::tc_fence_after();
+      if (lane == 0) {
+        const uint32_t xb = ptx::smem_u32(smem + (size_t)s * stage_bytes);
+        const uint32_t x16 = xb >> 4, g16 = (xb + box_bytes) >> 4;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          ptx::mma_f16(tmem_base, a_hi | (uint64_t)(g16 + k * kBRow), b_hi | (uint64_t)(x16 + k * 128), idesc, (it | k) != 0);
+        ptx::mma_commit(&empty[s]);
+      }
+      __syncwarp();
+    }
+    if (ok && lane == 0) ptx::mma_commit(done);
+    __syncwarp();
+  } else {
+    const int lg = warp & 3;  // = column tap kw of this warp's rows
+    if (ptx::mbar_wait(done, 0, abort_flag) && t1 > t0) {
+      ptx::tc_fence_after();
+      const size_t plane = (size_t)p.Cout * p.Cin;
+      const bool mine = lg < 3 && lane < NB && lane < p.Cout;
+      float* base = p.part + (size_t)sp * 9 * plane + (size_t)lg * plane + (size_t)lane * p.Cin + cic * 64;
+#pragma unroll 1
+      for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t v[16];
+          ptx::tmem_ld16(tmem_base + ((uint32_t)(lg * 32) << 16) + kh * 64 + q * 16, v);
+          ptx::tmem_ld_wait();
+          if (mine) {
+            float4* dst = reinterpret_cast<float4*>(base + (size_t)(kh * 3) * plane + q * 16);
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]), __uint_as_float(v[4 * e + 2]),
+                                   __uint_as_float(v[4 * e + 3]));
+          }
+        }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(p.status, NF_ETIMEOUT);
+    const unsigned long long tt = ptx::globaltimer();
+    while (ptx::globaltimer() - tt < 2000000ull) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kCols);
+  }
+}
+
 __global__ void __launch_bounds__(256) sum_parts_kernel(const float* __restrict__ part, int splits, size_t n, float* __restrict__ out) {
   // 32 consecutive elements x 8 lanes over the splits; each lane adds its splits in index order, lane sums are added in lane order
   __shared__ float sm[8][33];
@@ -1261,7 +1390,7 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
 }
 
 struct WgPlan {
-  int ok, BW, BH, BI, PT, NB, splits, grid, stages;
+  int ok, BW, BH, BI, PT, NB, GX, splits, grid, stages;
   size_t smem, part_floats;
 };
 
@@ -1274,7 +1403,8 @@ WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0, int strid
   if (!pick_tile(H, W, true, &pl.BW, &pl.BH, &pl.BI)) return pl;
   pl.PT = (stride == 2 || pl.BI > 1) ? 1 : 0;
   pl.NB = aux ? (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64) : 64;
-  size_t g_region = (size_t)3 * 128 * pl.NB * 2;
+  pl.GX = (aux && !pl.PT && pl.NB <= 32) ? 1 : 0;  // few filters: one instruction per 16 pixels with the gradient on the M side
+  size_t g_region = (size_t)(pl.GX ? 4 : 3) * 128 * pl.NB * 2;
   if (g_region < 4096) g_region = 4096;
   const size_t stage = pl.PT ? 65536 : (size_t)(pl.BH + 2) * pl.BW * 128 + g_region;
   pl.stages = pl.PT ? 3 : (int)((232448 - 2048) / stage);
@@ -1303,6 +1433,18 @@ int launch_wgrad_kw(const WgPlan& pl, const CUtensorMap& mx, const CUtensorMap& 
     attr_done = true;
   }
   conv_wgrad_kw_kernel<NB><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mg, p);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+template <int NB>
+int launch_wgrad_gx(const WgPlan& pl, const CUtensorMap& mx, const CUtensorMap& mg, const WgParams& p) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    NF_CUDA(cudaFuncSetAttribute(conv_wgrad_gx_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    attr_done = true;
+  }
+  conv_wgrad_gx_kernel<NB><<<pl.grid, kThreads, pl.smem, g_nf_stream>>>(mx, mg, p);
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -1340,7 +1482,9 @@ int run_wgrad(int N, int Hin, int Win, int Cin, int Cout, const void* x, const v
   p.stride = stride; p.BI = pl.BI;
   p.ci_chunks = Cin / 64; p.co_chunks = aux ? 1 : Cout / 64; p.splits = pl.splits; p.part = part; p.status = status;
   p.stages = pl.stages;
-  if (pl.PT)
+  if (pl.GX)
+    rc = pl.NB == 32 ? launch_wgrad_gx<32>(pl, mx, mg, p) : launch_wgrad_gx<16>(pl, mx, mg, p);
+  else if (pl.PT)
     rc = pl.NB == 64 ? launch_wgrad<64, 1>(pl, mx, mg, p) : pl.NB == 32 ? launch_wgrad<32, 1>(pl, mx, mg, p) : launch_wgrad<16, 1>(pl, mx, mg, p);
   else
     rc = pl.NB == 64 ? launch_wgrad_kw<64>(pl, mx, mg, p)
