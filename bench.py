@@ -30,9 +30,12 @@ FALLBACK_PEAKS = dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=
 # DRAM bytes per image (read + write) of the kernels behind each traced op on the c4 layers 64->64 at 224x224,
 # from one ncu capture of the batch-24 case (profiles/ncu_full_c4s_conv_bn_kernels.md); every tensor is streamed
 # once, so traffic grows in proportion to the batch.  Valid for the kernels as captured; None elsewhere.
-NCU_TRAFFIC_C4_BYTES_PER_IMAGE = dict(conv_fwd=(154.27 + 106.65) * 1e6 / 24, wgrad=(324.46 + 3.77) * 1e6 / 24,
-                                      bn_fwd=(154.15 + 109.90) * 1e6 / 24,
-                                      bn_bwd=(308.30 + 122.84) * 1e6 / 24)   # the apply kernel; the finalize kernel moves < 1 MB
+NCU_TRAFFIC_C4_BYTES_PER_IMAGE = dict(conv_fwd=(154.28 + 106.19) * 1e6 / 24, wgrad=(324.20 + 3.72) * 1e6 / 24,
+                                      bn_fwd=(154.15 + 111.28) * 1e6 / 24, aux_fwd=(154.23 + 21.14) * 1e6 / 24,
+                                      bn_bwd=(308.29 + 124.88) * 1e6 / 24,   # the apply kernel; the finalize kernel moves < 1 MB
+                                      # dh_vec + aux weight gradient + aux input gradient (with the fused y read); the
+                                      # two small partial-sum kernels move < 1 MB
+                                      aux_bwd=(38.57 + 1.50 + 201.43 + 3.81 + 192.84 + 114.94) * 1e6 / 24)
 
 
 def load_peaks():
