@@ -84,7 +84,7 @@ typedef struct nf_layer_opts {
   float momentum;    /* SGD momentum; 0 gives the plain update of the paper's Appendix B */
   float bn_eps;      /* BatchNorm epsilon */
   float bn_momentum; /* running-statistics momentum */
-  int host_io;       /* 1: reserve staging so nf_layer_step_host can be used */
+  int host_io;       /* 1: reserve staging so the *_step_host calls can be used; 2: a second input buffer too (nf_block_step_host_next) */
   int loss;          /* nf_loss: the loss of Eq. 3 ("e.g., Mean Squared Error or Cross Entropy Error"); 0 = cross entropy */
   int aux_pool;      /* nf_aux_pool: the down-sampling F_n of Eq. 2 ("such as max pooling or average pooling"); 0 = average */
 } nf_layer_opts;
@@ -210,6 +210,14 @@ int nf_block_step(nf_block* block, const void* x, const int32_t* labels, float l
  * The first layer must have been configured with host_io = 1. */
 int nf_block_step_host(nf_block* block, const void* x_host, const int32_t* labels_host, float lr,
                        float* loss_host, void* act_out_host);
+
+/* nf_block_step_host for a stream of batches: while this batch trains, the NEXT batch's host buffers (pinned; may be
+ * NULL for the last one) are copied into the second staging buffer on a copy stream; the following call, given those
+ * same pointers as its batch, finds the copy done or in flight and only waits for it.  Every batch is still copied
+ * host -> device exactly once and the call still returns after the step has finished and the losses are in loss_host.
+ * Needs opts.host_io = 2 on the first layer.  The contents of a prefetched batch must not change until its step. */
+int nf_block_step_host_next(nf_block* block, const void* x_host, const int32_t* labels_host, float lr, float* loss_host,
+                            void* act_host, const void* next_x_host, const int32_t* next_labels_host);
 
 /* Re-batching from the cache: out[i] = cache[idx[i]] for i < count, rows of row_bytes bytes
  * (a multiple of 16); labels likewise if both label pointers are non-NULL.  All device pointers.

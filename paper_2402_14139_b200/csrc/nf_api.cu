@@ -131,6 +131,13 @@ size_t plan(nf_layer* L, char* base, bool assign) {
     D->stage_labels = (int32_t*)c.take(N * 4);
     D->stage_act = c.take(na * es);
     D->stage_loss = (float*)c.take(256);
+    D->stage_xb[0] = D->stage_x;
+    D->stage_lb[0] = D->stage_labels;
+    D->stage_xb[1] = L->o.host_io == 2 ? c.take(N * L->H * L->W * L->Cin * es) : nullptr;
+    D->stage_lb[1] = L->o.host_io == 2 ? (int32_t*)c.take(N * 4) : nullptr;
+    D->stage_cur = 0;
+    D->pre_x = nullptr;
+    D->pre_l = nullptr;
   } else {
     D->stage_x = D->stage_act = nullptr;
     D->stage_labels = nullptr;
@@ -237,7 +244,7 @@ int nf_layer_configure(nf_layer* L, const nf_layer_opts* o) {
   if ((o->loss != NF_LOSS_CE && o->loss != NF_LOSS_MSE) || (o->aux_pool != NF_POOL_AVG && o->aux_pool != NF_POOL_MAX)) return NF_EINVAL;
   L->o = *o;
   L->o.maxpool = o->maxpool ? 1 : 0;
-  L->o.host_io = o->host_io ? 1 : 0;
+  L->o.host_io = o->host_io == 2 ? 2 : o->host_io ? 1 : 0;
   L->ws = nullptr;
   derive(L);
   return NF_OK;
@@ -660,6 +667,46 @@ int nf_trace_read(int op, int slot, double* ms_total, long long* groups) {
   if (trace_flush() != NF_OK) return NF_ECUDA;
   *ms_total = g_trace_ms[op][slot];
   *groups = g_trace_cnt[op][slot];
+  return NF_OK;
+}
+
+// copy stream and event of the input prefetch (created on first use; they hold no device memory)
+static cudaStream_t g_copy_stream = nullptr;
+static cudaEvent_t g_copy_done = nullptr;
+
+int nf_block_step_host_next(nf_block* B, const void* xh, const int32_t* lh, float lr, float* loss_h, void* act_h,
+                            const void* next_xh, const int32_t* next_lh) {
+  if (!B || !xh || !lh || !loss_h) return NF_EINVAL;
+  nf_layer* L0 = B->layers[0];
+  nf_layer* Ll = B->layers[B->n - 1];
+  if (L0->o.host_io != 2 || B->n > 64 || ((next_xh == nullptr) != (next_lh == nullptr))) return NF_EINVAL;
+  if (!g_copy_stream) {
+    NF_CUDA(cudaStreamCreateWithFlags(&g_copy_stream, cudaStreamNonBlocking));
+    NF_CUDA(cudaEventCreateWithFlags(&g_copy_done, cudaEventDisableTiming));
+  }
+  const size_t es = nf_esize(L0->o.dtype), N = L0->o.N, xbytes = N * L0->H * L0->W * L0->Cin * es;
+  if (L0->pre_x == xh && L0->pre_l == lh) {  // this batch was started on its way during the previous call
+    L0->stage_cur ^= 1;
+    NF_CUDA(cudaStreamWaitEvent(g_nf_stream, g_copy_done, 0));
+  } else {
+    NF_CUDA(cudaMemcpyAsync(L0->stage_xb[L0->stage_cur], xh, xbytes, cudaMemcpyHostToDevice, g_nf_stream));
+    NF_CUDA(cudaMemcpyAsync(L0->stage_lb[L0->stage_cur], lh, N * 4, cudaMemcpyHostToDevice, g_nf_stream));
+  }
+  L0->pre_x = nullptr;
+  L0->pre_l = nullptr;
+  if (next_xh) {  // the other buffer is free: the step that read it has been waited for before its call returned
+    const int nb = L0->stage_cur ^ 1;
+    NF_CUDA(cudaMemcpyAsync(L0->stage_xb[nb], next_xh, xbytes, cudaMemcpyHostToDevice, g_copy_stream));
+    NF_CUDA(cudaMemcpyAsync(L0->stage_lb[nb], next_lh, N * 4, cudaMemcpyHostToDevice, g_copy_stream));
+    NF_CUDA(cudaEventRecord(g_copy_done, g_copy_stream));
+    L0->pre_x = next_xh;
+    L0->pre_l = next_lh;
+  }
+  NF_TRY(nf_block_step(B, L0->stage_xb[L0->stage_cur], L0->stage_lb[L0->stage_cur], lr, L0->stage_loss, nullptr));
+  NF_CUDA(cudaMemcpyAsync(loss_h, L0->stage_loss, 4 * (size_t)B->n, cudaMemcpyDeviceToHost, g_nf_stream));
+  if (act_h)
+    NF_CUDA(cudaMemcpyAsync(act_h, Ll->act, N * Ll->Ha * Ll->Wa * Ll->Cout * es, cudaMemcpyDeviceToHost, g_nf_stream));
+  NF_CUDA(cudaStreamSynchronize(g_nf_stream));
   return NF_OK;
 }
 

@@ -52,6 +52,11 @@ struct nf_layer {
   float* wpart;                        // split-K partials of the weight gradients
   size_t wpart_floats;
   void* stage_x;                       // host_io staging
+  void* stage_xb[2];                   // host_io = 2: two input staging buffers (stage_xb[0] == stage_x)
+  int32_t* stage_lb[2];
+  int stage_cur;                       // buffer the next step reads
+  const void* pre_x;                   // host batch already on its way into buffer 1 - stage_cur (or NULL)
+  const int32_t* pre_l;
   int32_t* stage_labels;
   void* stage_act;
   float* stage_loss;

@@ -27,7 +27,7 @@ PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P
 EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_layer_workspace_bytes",
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
-           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_max_batch", "nf_layer_step_dp", "nf_layer_dp_buffer", "nf_block_step", "nf_block_step_host", "nf_trace_enable", "nf_trace_read",
+           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_max_batch", "nf_layer_step_dp", "nf_layer_dp_buffer", "nf_block_step", "nf_block_step_host", "nf_block_step_host_next", "nf_trace_enable", "nf_trace_read",
            "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_op_status", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
@@ -86,6 +86,7 @@ def lib():
         L.nf_select_exit.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.c_int]
         L.nf_block_step.argtypes = [vp, vp, ip, C.c_float, fp, vp]
         L.nf_block_step_host.argtypes = [vp, vp, ip, C.c_float, fp, vp]
+        L.nf_block_step_host_next.argtypes = [vp, vp, ip, C.c_float, fp, vp, vp, ip]
         L.nf_trace_enable.argtypes = [C.c_int]
         L.nf_trace_read.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
         L.nf_cache_gather.argtypes = [vp, ip, ip, C.c_int, C.c_size_t, vp, ip]
@@ -324,6 +325,11 @@ class Block:
         """nf_block_step: loss_out is a float32 device tensor with one entry per layer."""
         _check(lib().nf_block_step(self.h, _ptr(x), _ptr(labels), float(lr), _ptr(loss_out), _ptr(act_out)),
                "nf_block_step")
+
+    def step_host_next(self, x_host, labels_host, lr, loss_host, next_x_host=None, next_labels_host=None, act_host=None):
+        """nf_block_step_host_next: trains on (x_host, labels_host) while the next batch is copied to the device."""
+        _check(lib().nf_block_step_host_next(self.h, _ptr(x_host), _ptr(labels_host), float(lr), _ptr(loss_host), _ptr(act_host),
+                                             _ptr(next_x_host), _ptr(next_labels_host)), "nf_block_step_host_next")
 
     def step_host(self, x_host, labels_host, lr, loss_host, act_host=None):
         _check(lib().nf_block_step_host(self.h, _ptr(x_host), _ptr(labels_host), float(lr), _ptr(loss_host),

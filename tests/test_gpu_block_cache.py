@@ -110,3 +110,39 @@ def test_cache_gather_is_bit_exact(env):
         assert torch.equal(out_l, labels[idx.long()])
     with pytest.raises(nf.NfError):
         nf.nf_cache_gather(cache, labels, idx, out, None)      # labels in without labels out
+
+
+def test_prefetching_host_step_equals_plain_host_step():
+    """A stream of different batches through nf_block_step_host_next (the next batch copied while this one trains)
+    gives bit-identical losses and parameters to the plain host step; a call whose batch was not announced falls
+    back to copying it itself."""
+    import torch
+    from paper_2402_14139_b200 import nf, synth
+    from tests import parity_util as pu
+    nf.lib()
+    nf.nf_set_stream(None)
+    c1 = dict(N=6, Cin=64, Cout=64, H=16, W=16, F=16, classes=10, stride=1, pool=False)
+    c2 = dict(N=6, Cin=64, Cout=64, H=16, W=16, F=8, classes=10, stride=1, pool=True)
+    P1, _, _ = pu.seeded_case(c1, 71, bf16=True)
+    P2, _, _ = pu.seeded_case(c2, 72, bf16=True)
+
+    def make(host_io):
+        layers = [pu.gpu_layer(nf, c1, P1, nf.NF_BF16, host_io=host_io), pu.gpu_layer(nf, c2, P2, nf.NF_BF16)]
+        return layers, nf.Block(layers)
+
+    la, A = make(1)
+    lb, B = make(2)
+    xs = [torch.from_numpy(synth.round_bf16(synth.normal(73, k, (6, 16, 16, 64)))).to(torch.bfloat16).pin_memory() for k in range(4)]
+    ys = [torch.from_numpy(synth.labels(74, k, 6, 10)).pin_memory() for k in range(4)]
+    la_h, lb_h = torch.zeros(2).pin_memory(), torch.zeros(2).pin_memory()
+    order = [0, 1, 2, 3, 1]
+    for i, k in enumerate(order):
+        A.step_host(xs[k], ys[k], 0.05, la_h)
+        nxt = order[i + 1] if i + 1 < len(order) and i != 2 else None      # step 3's batch is NOT announced
+        B.step_host_next(xs[k], ys[k], 0.05, lb_h, None if nxt is None else xs[nxt], None if nxt is None else ys[nxt])
+        assert torch.equal(la_h, lb_h), (i, la_h, lb_h)
+    for ga, gb in zip(la, lb):
+        for name in pu.PNAMES:
+            assert np.array_equal(ga.get_param(name), gb.get_param(name)), name
+    # the plain layer (host_io = 1) has no second buffer: the call is refused
+    assert nf.lib().nf_block_step_host_next(A.h, nf._ptr(xs[0]), nf._ptr(ys[0]), 0.05, nf._ptr(la_h), None, None, None) == nf.NF_EINVAL
