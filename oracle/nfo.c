@@ -347,6 +347,9 @@ typedef struct {
   int aux_pool;   /* F_n of Eq. 2: 0 = adaptive average pool to 2x2, 1 = adaptive max pool to 2x2.  In the bf16
                      configuration the auxiliary activation h is then rounded to bfloat16 where it is stored, so that
                      the arg-max of a bin is decided among the stored values. */
+  const double* skip; /* NULL, or an identity shortcut of a residual network: a tensor of the shape of the BatchNorm
+                     output that is added before the ReLU, x_{n+1} = P(ReLU(BN(theta_n x_n) + skip)).  It comes from an
+                     earlier layer and carries no gradient (training is local to the layer). */
 } nfo_dims;
 
 /* Round to the nearest bfloat16, ties to even (via float, as a bf16 store of an fp32 value does). */
@@ -415,6 +418,8 @@ double nfo_layer_step(const nfo_dims* d, const double* x, const int32_t* labels,
   nfo_conv3x3(x, N, Ci, H, W, Wq, Co, NULL, s, y);
   store_round(y, ny, d->store_bf16);
   nfo_bn_train(y, N, Co, Ho * Wo, P->gamma, P->beta, d->eps, mu, var, xhat, z);
+  if (d->skip)
+    for (size_t k = 0; k < ny; ++k) z[k] += d->skip[k];
   nfo_relu(z, ny, r);
   store_round(r, ny, d->store_bf16); /* rounding is monotone: pooling rounded values = rounding the pooled value */
   if (d->pool) nfo_maxpool2(r, N, Co, Ho, Wo, a, arg);
@@ -528,6 +533,8 @@ void nfo_layer_eval(const nfo_dims* d, const double* x, const nfo_params* P, dou
   free(Wq);
   store_round(y, ny, d->store_bf16);
   nfo_bn_eval(y, N, Co, Ho * Wo, P->gamma, P->beta, d->eps, P->rmean, P->rvar, z);
+  if (d->skip)
+    for (size_t k = 0; k < ny; ++k) z[k] += d->skip[k];
   nfo_relu(z, ny, r);
   store_round(r, ny, d->store_bf16);
   if (d->pool) {

@@ -32,7 +32,7 @@ _ip = C.POINTER(C.c_int32)
 class Dims(C.Structure):
     _fields_ = [(k, C.c_int) for k in ("N", "Cin", "Cout", "H", "W", "stride", "pool", "F", "classes")] + \
                [(k, C.c_double) for k in ("eps", "momentum", "bn_momentum")] + \
-               [(k, C.c_int) for k in ("store_bf16", "loss", "aux_pool")]
+               [(k, C.c_int) for k in ("store_bf16", "loss", "aux_pool")] + [("skip", C.c_void_p)]
 
 
 _PNAMES = ("W", "gamma", "beta", "Wa", "ba", "Wf", "bf")
@@ -208,7 +208,7 @@ class Layer:
     def __init__(self, Cin, Cout, H, W, F, classes, N, stride=1, pool=False, eps=1e-5, momentum=0.9,
                  bn_momentum=0.1, store_bf16=False, loss="ce", aux_pool="avg"):
         self.d = Dims(N, Cin, Cout, H, W, stride, int(pool), F, classes, eps, momentum, bn_momentum, int(store_bf16),
-                      {"ce": 0, "mse": 1}[loss], {"avg": 0, "max": 1}[aux_pool])
+                      {"ce": 0, "mse": 1}[loss], {"avg": 0, "max": 1}[aux_pool], None)
         self.Ho, self.Wo = out_size(H, stride), out_size(W, stride)
         self.Ha, self.Wa = (self.Ho // 2, self.Wo // 2) if pool else (self.Ho, self.Wo)
         sh = dict(W=(Cout, Cin, 3, 3), gamma=(Cout,), beta=(Cout,), Wa=(F, Cout, 3, 3), ba=(F,),
@@ -252,14 +252,24 @@ class Layer:
         arrs["argmax"] = np.zeros(ash, dtype=np.int32)
         return arrs
 
-    def step(self, x, labels, lr, update=True, trace=False, grads=False):
+    def _with_skip(self, d, skip, n):
+        """A copy of the dims with the shortcut tensor attached (kept alive by the returned array)."""
+        if skip is None:
+            return d, None
+        s = _c64(skip)
+        assert s.shape == (n, d.Cout, self.Ho, self.Wo), s.shape
+        d = Dims.from_buffer_copy(d)
+        d.skip = s.ctypes.data
+        return d, s
+
+    def step(self, x, labels, lr, update=True, trace=False, grads=False, skip=None):
         """One local training step.  Returns (loss, act_out, trace dict or None).
 
         ``trace=True`` keeps every intermediate; ``grads=True`` keeps only the parameter gradients
         and the batch statistics (cheap enough for large shapes)."""
         x = _c64(x)
         labels = np.ascontiguousarray(labels, dtype=np.int32)
-        d = self.d
+        d, _keep = self._with_skip(self.d, skip, self.d.N)
         assert x.shape == (d.N, d.Cin, d.H, d.W), x.shape
         act = np.empty((d.N, d.Cout, self.Ha, self.Wa))
         P = self._params()
@@ -279,11 +289,12 @@ class Layer:
                                     C.byref(P), _d(act), C.byref(T) if T is not None else None, int(update))
         return float(loss), act, arrs
 
-    def predict(self, x):
+    def predict(self, x, skip=None):
         """Early-exit prediction for any batch size: (act_out, logits, classes); class = first arg-max."""
         x = _c64(x)
         d = Dims.from_buffer_copy(self.d)
         d.N = x.shape[0]
+        d, _keep = self._with_skip(d, skip, d.N)
         act = np.empty((d.N, d.Cout, self.Ha, self.Wa))
         logits = np.empty((d.N, d.classes))
         P = self._params()
@@ -296,11 +307,12 @@ class Layer:
         aux = sum(self.p[k].size for k in ("Wa", "ba", "Wf", "bf"))
         return main, aux
 
-    def eval_forward(self, x):
+    def eval_forward(self, x, skip=None):
         """Eval-mode forward (running statistics) for any batch size."""
         x = _c64(x)
         d = Dims.from_buffer_copy(self.d)
         d.N = x.shape[0]
+        d, _keep = self._with_skip(d, skip, d.N)
         out = np.empty((d.N, d.Cout, self.Ha, self.Wa))
         P = self._params()
         lib().nfo_layer_eval(C.byref(d), _d(x), C.byref(P), _d(out))

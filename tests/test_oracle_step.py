@@ -297,3 +297,40 @@ def test_loss_and_downsampling_variants_against_library_autograd(ci, vi):
         pe = (F.adaptive_max_pool2d(he, 2) if pool_kind == "max" else F.adaptive_avg_pool2d(he, 2)).flatten(1)
         le = F.linear(pe, tp["Wf"], tp["bf"])
     np.testing.assert_allclose(L2.predict(x)[1], le.numpy(), atol=1e-11)
+
+
+@pytest.mark.parametrize("ci", [0, 2])
+def test_identity_shortcut_against_library_autograd(ci):
+    """A residual network's identity shortcut: a tensor added to the BatchNorm output before the ReLU.  It carries
+    no gradient (local training); one step and the eval forward re-derived with the library's ops and autograd."""
+    c = CASES[ci]
+    L, x, y = make_layer(c, 51 + ci)
+    Ho, Wo = L.Ho, L.Wo
+    skip = np.maximum(synth.normal(52 + ci, 1, (c["N"], c["Cout"], Ho, Wo)), 0.0)      # an earlier post-ReLU activation
+    tp = {k: torch.tensor(v.copy(), dtype=torch.float64, requires_grad=True) for k, v in L.p.items()}
+    rm, rv = torch.zeros(c["Cout"], dtype=torch.float64), torch.ones(c["Cout"], dtype=torch.float64)
+    xt, yt, st = torch.tensor(x), torch.tensor(y.astype(np.int64)), torch.tensor(skip)
+    F = torch.nn.functional
+    a = F.relu(F.batch_norm(F.conv2d(xt, tp["W"], None, stride=c["stride"], padding=1), rm, rv, tp["gamma"], tp["beta"],
+                            training=True, momentum=0.1, eps=1e-5) + st)
+    if c["pool"]:
+        a = F.max_pool2d(a, 2)
+    a_in = a.detach().numpy().copy()
+    h = F.relu(F.conv2d(a, tp["Wa"], tp["ba"], padding=1))
+    loss_t = F.cross_entropy(F.linear(F.adaptive_avg_pool2d(h, 2).flatten(1), tp["Wf"], tp["bf"]), yt)
+    loss_t.backward()
+    loss0 = L.step(x, y, 0.05, update=False)[0]
+    loss, act, tr = L.step(x, y, 0.05, update=True, trace=True, skip=skip)
+    assert abs(loss - float(loss_t.detach())) <= 1e-12 and abs(loss - loss0) > 1e-6
+    np.testing.assert_allclose(act, a_in, atol=1e-12)
+    for k, g in [("W", "gW"), ("gamma", "ggamma"), ("beta", "gbeta"), ("Wa", "gWa"), ("ba", "gba"), ("Wf", "gWf"), ("bf", "gbf")]:
+        np.testing.assert_allclose(tr[g], tp[k].grad.numpy(), atol=1e-11 * max(1.0, np.abs(tp[k].grad.numpy()).max()), err_msg=k)
+    with torch.no_grad():        # eval forward with the updated parameters and running statistics
+        t2 = {k: torch.tensor(v) for k, v in L.p.items()}
+        ae = F.relu(F.batch_norm(F.conv2d(xt, t2["W"], None, stride=c["stride"], padding=1), torch.tensor(L.rmean), torch.tensor(L.rvar),
+                                 t2["gamma"], t2["beta"], training=False, eps=1e-5) + st)
+        if c["pool"]:
+            ae = F.max_pool2d(ae, 2)
+    np.testing.assert_allclose(L.eval_forward(x, skip=skip), ae.numpy(), atol=1e-12)
+    np.testing.assert_allclose(L.predict(x, skip=skip)[0], ae.numpy(), atol=1e-12)
+    assert np.abs(L.eval_forward(x) - ae.numpy()).max() > 1e-3       # and the shortcut is not silently ignored
