@@ -160,6 +160,15 @@ void nf_block_destroy(nf_block* block);
 int nf_block_cache(nf_block* block, const void* x, void* out);
 int nf_block_cache_n(nf_block* block, const void* x, void* out, int count);
 
+/* Identity shortcut of a residual network (the paper trains ResNet-18 but does not say how a shortcut enters a
+ * layer-local step; the reading here: the shortcut tensor is added to the BatchNorm output before the ReLU,
+ * x_{n+1} = P(ReLU(BN(theta_n x_n) + skip)), and carries no gradient, like the layer input).  `skip` is a device tensor
+ * [N][Ho][Wo][Cout] of the layer's dtype — typically the input of the previous layer — used by every later
+ * nf_layer_step / nf_block_step / nf_layer_predict / nf_block_cache call on this layer (for a call with count < N, its
+ * first count samples) until it is changed; NULL removes it.  The caller keeps the tensor alive.  Layers with a
+ * shortcut run their BatchNorm passes on the generic kernels.  NF_EALIGN if not 16-byte aligned. */
+int nf_layer_set_skip(nf_layer* layer, const void* skip);
+
 /* Data-parallel local step (the paper names distributed training as the direction beyond a single device): the batch
  * of N * world samples is sharded over `world` ranks, every rank holds N of them and a full copy of the layer, and
  * BatchNorm uses the statistics of the WHOLE batch, so the result equals nf_layer_step on the whole batch (up to

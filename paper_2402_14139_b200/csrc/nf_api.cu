@@ -371,7 +371,7 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
     NF_TRY(nf_ref_bn_finalize_tot(L->dptot, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
                                   L->o.bn_momentum, L->scale, L->shift, L->mu, L->invstd, L->rmean, L->rvar));
   }
-  NF_TRY(nf_ref_bn_apply(dt, L->y, N, Ho, Wo, Co, pool, L->scale, L->shift, act_out));
+  NF_TRY(nf_ref_bn_apply(dt, L->y, N, Ho, Wo, Co, pool, L->scale, L->shift, act_out, L->skip));
   trace_end();
   // Eq. 2: aux conv + ReLU, average pool to 2x2, linear; Eq. 3: softmax cross-entropy
   trace_begin(2);
@@ -436,7 +436,7 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
     nb = bn_nb;
   } else {
     NF_TRY(nf_ref_bn_bwd_reduce(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->red,
-                                L->red_floats, &nb));
+                                L->red_floats, &nb, L->skip));
   }
   if (!all) return nf_ref_partial_totals(L->red, nb, Co, L->dptot + 2 * Co);
   }
@@ -447,7 +447,7 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
     NF_TRY(nf_ref_bn_bwd_finalize_tot(L->dptot + 2 * Co, Co, world, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
   }
   NF_TRY(nf_ref_bn_bwd_apply(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->sdz, L->sdzx,
-                             M, L->dy));
+                             M, L->dy, L->skip));
   trace_end();
   // gradient of theta_n (the layer input receives none), then the update
   trace_begin(6);
@@ -467,6 +467,13 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
 
 int nf_layer_step(nf_layer* L, const void* x, const int32_t* labels, float lr, float* loss_out, void* act_out) {
   return step_phases(L, x, labels, lr, loss_out, act_out, -1, 1);
+}
+
+int nf_layer_set_skip(nf_layer* L, const void* skip) {
+  if (!L) return NF_EINVAL;
+  if (skip && misaligned(skip)) return NF_EALIGN;
+  L->skip = skip;
+  return NF_OK;
 }
 
 int nf_layer_step_dp(nf_layer* L, int phase, const void* x, const int32_t* labels, float lr, float* loss_out, void* act_out,
@@ -565,7 +572,7 @@ static int layer_eval_forward(nf_layer* L, const void* in, int count, void* dst)
   }
   NF_TRY(nf_ref_bn_eval_coeffs(L->Cout, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps, L->rmean, L->rvar,
                                L->scale, L->shift));
-  return nf_ref_bn_apply(dt, L->y, count, L->Ho, L->Wo, L->Cout, L->o.maxpool, L->scale, L->shift, dst);
+  return nf_ref_bn_apply(dt, L->y, count, L->Ho, L->Wo, L->Cout, L->o.maxpool, L->scale, L->shift, dst, L->skip);
 }
 
 int nf_layer_predict(nf_layer* L, const void* x, int count, void* act_out, float* logits_out, int32_t* pred_out) {

@@ -32,6 +32,7 @@ struct nf_layer {
   int32_t* status;                     // device status word
   float *val, *mom, *grad;             // arenas
   bf16* shadow;                        // bf16 arena
+  const void* skip;                    // identity shortcut for the next calls (nf_layer_set_skip), or NULL
   bf16* wa_t;                          // [9][Cout][F] mirrored, transposed copy of Wa (only when F > 64)
   float *rmean, *rvar;                 // [Cout]
   float *scale, *shift, *mu, *invstd;  // [Cout] per-step BatchNorm coefficients
@@ -100,7 +101,7 @@ int nf_ref_bn_finalize(const float* red, int nblocks, int C, double M, const flo
 int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float eps, const float* rmean,
                           const float* rvar, float* scale, float* shift);
 int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
-                    const float* shift, void* out);
+                    const float* shift, void* out, const void* skip = nullptr);
 int nf_ref_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p);
 // bf16 fast paths (F % 8 == 0, even Ha and Wa); NF_EUNSUPPORTED means "use the generic kernel"
 int nf_ref_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part, size_t part_floats, float* p);
@@ -131,12 +132,12 @@ int nf_ref_dh(int dtype, const void* h, const float* dp, int N, int Ha, int Wa, 
 int nf_ref_sum_partials(const float* red, int nblocks, int C, int which, float* out);
 int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
                          const float* scale, const float* shift, const float* mu, const float* invstd, float* red,
-                         size_t red_floats, int* nblocks);
+                         size_t red_floats, int* nblocks, const void* skip = nullptr);
 int nf_ref_bn_bwd_finalize(const float* red, int nblocks, int C, float* sdz, float* sdzx, float* ggamma,
                            float* gbeta);
 int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
                         const float* scale, const float* shift, const float* mu, const float* invstd,
-                        const float* sdz, const float* sdzx, double M, void* dy);
+                        const float* sdz, const float* sdzx, double M, void* dy, const void* skip = nullptr);
 int nf_ref_sgd(float* val, float* mom, const float* grad, bf16* shadow, size_t n, float lr, float momentum);
 int nf_ref_shadow(const float* val, bf16* shadow, size_t n);
 int nf_ref_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count, size_t row_bytes,

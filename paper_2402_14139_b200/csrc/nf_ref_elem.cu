@@ -17,8 +17,8 @@ __host__ __device__ inline int pow2ceil_cap256(int c) {
 // output through ReLU and the optional 2x2 max-pool (first maximum in scan order wins).
 template <typename T>
 __device__ __forceinline__ float dz_at(const T* __restrict__ y, const T* __restrict__ da, size_t p, int c, int C,
-                                       int Ho, int Wo, int pool, float sc, float sh) {
-  const float z = fmaf(ldf(y, p * C + c), sc, sh);
+                                       int Ho, int Wo, int pool, float sc, float sh, const T* __restrict__ skip = nullptr) {
+  const float z = fmaf(ldf(y, p * C + c), sc, sh) + (skip ? ldf(skip, p * C + c) : 0.f);
   if (!(z > 0.f)) return 0.f;
   if (!pool) return ldf(da, p * C + c);
   const int j = (int)(p % Wo), i = (int)((p / Wo) % Ho);
@@ -29,7 +29,7 @@ __device__ __forceinline__ float dz_at(const T* __restrict__ y, const T* __restr
 #pragma unroll
   for (int d = 0; d < 4; ++d) {
     const size_t q = ((n * Ho + i0 + (d >> 1)) * Wo + j0 + (d & 1)) * C + c;
-    const float r = rnd<T>(fmaxf(fmaf(ldf(y, q), sc, sh), 0.f));
+    const float r = rnd<T>(fmaxf(fmaf(ldf(y, q), sc, sh) + (skip ? ldf(skip, q) : 0.f), 0.f));
     if (r > best) { best = r; arg = d; }
   }
   if (arg != (i - i0) * 2 + (j - j0)) return 0.f;
@@ -48,9 +48,10 @@ struct StatsFn {  // (v, v^2) of a stored tensor
 struct BnBwdFn {  // (dz, dz*xhat)
   int Ho, Wo, pool;
   const float *scale, *shift, *mu, *invstd;
+  const void* skip;  // identity shortcut added before the ReLU, or NULL
   template <typename T>
   __device__ __forceinline__ void operator()(const T* y, const T* da, size_t p, int c, int C, float& a, float& b) const {
-    const float dz = dz_at(y, da, p, c, C, Ho, Wo, pool, scale[c], shift[c]);
+    const float dz = dz_at(y, da, p, c, C, Ho, Wo, pool, scale[c], shift[c], (const T*)skip);
     a = dz;
     b = dz * (ldf(y, p * C + c) - mu[c]) * invstd[c];
   }
@@ -204,14 +205,14 @@ __global__ void bn_eval_coeffs_kernel(int C, const float* gamma, const float* be
 // out[n,ia,ja,c] = max over the pool window (or the single pixel) of ReLU(y*scale+shift)
 template <typename T>
 __global__ void bn_apply_kernel(const T* __restrict__ y, int Ho, int Wo, int C, int pool, const float* __restrict__ scale,
-                                const float* __restrict__ shift, size_t total, T* __restrict__ out) {
+                                const float* __restrict__ shift, size_t total, T* __restrict__ out, const T* __restrict__ skip) {
   const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= total) return;
   const int c = (int)(e % C);
   const size_t q = e / C;
   const float sc = scale[c], sh = shift[c];
   if (!pool) {
-    stf(out, e, fmaxf(fmaf(ldf(y, e), sc, sh), 0.f));
+    stf(out, e, fmaxf(fmaf(ldf(y, e), sc, sh) + (skip ? ldf(skip, e) : 0.f), 0.f));
     return;
   }
   const int Wa = Wo / 2, Ha = Ho / 2;
@@ -221,7 +222,7 @@ __global__ void bn_apply_kernel(const T* __restrict__ y, int Ho, int Wo, int C, 
 #pragma unroll
   for (int d = 0; d < 4; ++d) {
     const size_t src = ((n * Ho + 2 * ia + (d >> 1)) * Wo + 2 * ja + (d & 1)) * C + c;
-    best = fmaxf(best, fmaf(ldf(y, src), sc, sh));
+    best = fmaxf(best, fmaf(ldf(y, src), sc, sh) + (skip ? ldf(skip, src) : 0.f));
   }
   stf(out, e, best);
 }
@@ -540,12 +541,12 @@ __global__ void bn_bwd_apply_kernel(const T* __restrict__ y, const T* __restrict
                                     const float* __restrict__ scale, const float* __restrict__ shift,
                                     const float* __restrict__ mu, const float* __restrict__ invstd,
                                     const float* __restrict__ sdz, const float* __restrict__ sdzx, float invM,
-                                    size_t total, T* __restrict__ dy) {
+                                    size_t total, T* __restrict__ dy, const T* __restrict__ skip) {
   const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= total) return;
   const int c = (int)(e % C);
   const size_t p = e / C;
-  const float dz = dz_at(y, da, p, c, C, Ho, Wo, pool, scale[c], shift[c]);
+  const float dz = dz_at(y, da, p, c, C, Ho, Wo, pool, scale[c], shift[c], skip);
   const float xh = (ldf(y, e) - mu[c]) * invstd[c];
   stf(dy, e, scale[c] * (dz - sdz[c] * invM - xh * sdzx[c] * invM));
 }
@@ -1168,8 +1169,15 @@ int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float ep
 }
 
 int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
-                    const float* shift, void* out) {
+                    const float* shift, void* out, const void* skip) {
   const size_t total = (size_t)N * (pool ? Ho / 2 : Ho) * (pool ? Wo / 2 : Wo) * C;
+  if (skip) {  // residual layers take the generic kernels
+    DISPATCH(dtype,
+             (bn_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, Ho, Wo, C, pool, scale, shift, total, (float*)out, (const float*)skip)),
+             (bn_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, Ho, Wo, C, pool, scale, shift, total, (bf16*)out, (const bf16*)skip)));
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   if (pool && vec_ok(dtype, C, 0) && 256 % (C / 8) == 0) {
     bn_apply_pool_vec_kernel<<<vec_blocks(total / 8), 256, 0, g_nf_stream>>>((const uint4*)y, Ho, Wo, C / 8, scale, shift, total / 8,
                                                                             (uint4*)out);
@@ -1188,8 +1196,8 @@ int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int 
     return NF_OK;
   }
   DISPATCH(dtype,
-           (bn_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, Ho, Wo, C, pool, scale, shift, total, (float*)out)),
-           (bn_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, Ho, Wo, C, pool, scale, shift, total, (bf16*)out)));
+           (bn_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, Ho, Wo, C, pool, scale, shift, total, (float*)out, nullptr)),
+           (bn_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, Ho, Wo, C, pool, scale, shift, total, (bf16*)out, nullptr)));
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -1317,24 +1325,24 @@ int nf_ref_sum_partials(const float* red, int nblocks, int C, int which, float* 
 
 int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
                          const float* scale, const float* shift, const float* mu, const float* invstd, float* red,
-                         size_t red_floats, int* nblocks) {
+                         size_t red_floats, int* nblocks, const void* skip) {
   const size_t P = (size_t)N * Ho * Wo;
   const int nb = nf_ref_channel_blocks(P, C);
   if ((size_t)nb * 2 * C > red_floats) return NF_ENOWS;
-  if (pool && vec_ok(dtype, C, 0) && 256 % (C / 8) == 0) {
+  if (!skip && pool && vec_ok(dtype, C, 0) && 256 % (C / 8) == 0) {
     bn_bwd_reduce_pool_vec_kernel<<<nb, 256, 0, g_nf_stream>>>((const uint4*)y, (const uint4*)da, P / 4, Ho, Wo, C / 8, scale, shift, mu,
                                                               invstd, red);
     NF_LAUNCHED();
     *nblocks = nb;
     return NF_OK;
   }
-  if (vec_ok(dtype, C, pool) && 256 % (C / 8) == 0) {
+  if (!skip && vec_ok(dtype, C, pool) && 256 % (C / 8) == 0) {
     bn_bwd_reduce_vec_kernel<<<nb, 256, 0, g_nf_stream>>>((const uint4*)y, (const uint4*)da, P, C / 8, scale, shift, mu, invstd, red);
     NF_LAUNCHED();
     *nblocks = nb;
     return NF_OK;
   }
-  BnBwdFn fn{Ho, Wo, pool, scale, shift, mu, invstd};
+  BnBwdFn fn{Ho, Wo, pool, scale, shift, mu, invstd, skip};
   DISPATCH(dtype,
            (channel_reduce_kernel<float, BnBwdFn><<<nb, 256, 0, g_nf_stream>>>((const float*)y, (const float*)da, P, C, fn, red)),
            (channel_reduce_kernel<bf16, BnBwdFn><<<nb, 256, 0, g_nf_stream>>>((const bf16*)y, (const bf16*)da, P, C, fn, red)));
@@ -1352,9 +1360,16 @@ int nf_ref_bn_bwd_finalize(const float* red, int nblocks, int C, float* sdz, flo
 
 int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
                         const float* scale, const float* shift, const float* mu, const float* invstd,
-                        const float* sdz, const float* sdzx, double M, void* dy) {
+                        const float* sdz, const float* sdzx, double M, void* dy, const void* skip) {
   const size_t total = (size_t)N * Ho * Wo * C;
   const float invM = (float)(1.0 / M);
+  if (skip) {
+    DISPATCH(dtype,
+             (bn_bwd_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, (const float*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (float*)dy, (const float*)skip)),
+             (bn_bwd_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, (const bf16*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (bf16*)dy, (const bf16*)skip)));
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   if (pool && vec_ok(dtype, C, 0) && 256 % (C / 8) == 0) {
     bn_bwd_apply_pool_vec_kernel<<<vec_blocks(total / 32), 256, 0, g_nf_stream>>>((const uint4*)y, (const uint4*)da, Ho, Wo, C / 8, scale,
                                                                                  shift, mu, invstd, sdz, sdzx, invM, total / 32, (uint4*)dy);
@@ -1374,8 +1389,8 @@ int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho,
     return NF_OK;
   }
   DISPATCH(dtype,
-           (bn_bwd_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, (const float*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (float*)dy)),
-           (bn_bwd_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, (const bf16*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (bf16*)dy)));
+           (bn_bwd_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, (const float*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (float*)dy, nullptr)),
+           (bn_bwd_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, (const bf16*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (bf16*)dy, nullptr)));
   NF_LAUNCHED();
   return NF_OK;
 }

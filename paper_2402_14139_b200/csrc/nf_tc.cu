@@ -1569,7 +1569,7 @@ int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb) {
     return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->wa_t, L->da, 0, nullptr, 0, L->status, &nb, 0);
   }
   // without a pool da has the shape of y: the folded kernel also reduces (dz, dz*xhat) per channel while it holds the tile
-  if (!L->o.maxpool && fold_ok(L->Ha, L->Wa, L->F, L->Cout, 2, 1) &&
+  if (!L->o.maxpool && !L->skip && fold_ok(L->Ha, L->Wa, L->F, L->Cout, 2, 1) &&
       (size_t)(sm_count() / (L->Cout / 64)) * 8 * 2 * L->Cout <= L->red_floats) {
     const BnBwdIn bn{L->y, L->scale, L->shift, L->mu, L->invstd};
     return run_fold(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->shadow + L->off[NF_P_WA], L->da, 2, L->red, L->red_floats,

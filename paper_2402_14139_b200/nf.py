@@ -27,7 +27,7 @@ PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P
 EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_layer_workspace_bytes",
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
-           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_max_batch", "nf_layer_step_dp", "nf_layer_dp_buffer", "nf_block_step", "nf_block_step_host", "nf_block_step_host_next", "nf_trace_enable", "nf_trace_read",
+           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_max_batch", "nf_layer_step_dp", "nf_layer_dp_buffer", "nf_layer_set_skip", "nf_block_step", "nf_block_step_host", "nf_block_step_host_next", "nf_trace_enable", "nf_trace_read",
            "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_op_status", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
@@ -76,6 +76,7 @@ def lib():
         L.nf_layer_param_count.restype = C.c_longlong
         L.nf_layer_param_count.argtypes = [vp, C.c_int]
         L.nf_count_equal.argtypes = [ip, ip, C.c_longlong, vp]
+        L.nf_layer_set_skip.argtypes = [vp, vp]
         L.nf_layer_step_dp.argtypes = [vp, C.c_int, vp, ip, C.c_float, fp, vp, C.c_int]
         L.nf_layer_dp_buffer.argtypes = [vp, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
         L.nf_aan_filters.argtypes = [C.POINTER(C.c_int), C.c_int, C.c_int, C.POINTER(C.c_int)]
@@ -274,6 +275,11 @@ class Layer:
         """nf_layer_predict: early-exit forward for `count` (default N) samples; device tensors."""
         _check(lib().nf_layer_predict(self.h, _ptr(x), int(self.N if count is None else count), _ptr(act_out), _ptr(logits_out),
                                       _ptr(pred_out)), "nf_layer_predict")
+
+    def set_skip(self, skip):
+        """nf_layer_set_skip: identity shortcut [N, Ho, Wo, Cout] added before the ReLU in later calls (None removes it)."""
+        self._skip = skip       # keeps the tensor alive
+        _check(lib().nf_layer_set_skip(self.h, _ptr(skip)), "nf_layer_set_skip")
 
     def dp_buffer(self, which):
         """The exchange buffer `which` of the data-parallel step as a tensor view of the workspace (float64 for 0 and 1, float32 for 2)."""
