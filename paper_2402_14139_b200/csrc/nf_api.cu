@@ -266,9 +266,7 @@ int nf_layer_bind_workspace(nf_layer* L, void* dev, size_t bytes) {
   NF_CUDA(cudaMemcpyAsync(L->val + L->off[NF_P_GAMMA], ones.data(), L->Cout * 4, cudaMemcpyHostToDevice, g_nf_stream));
   NF_CUDA(cudaMemcpyAsync(L->rvar, ones.data(), L->Cout * 4, cudaMemcpyHostToDevice, g_nf_stream));
   NF_CUDA(cudaStreamSynchronize(g_nf_stream));
-  int rc = nf_ref_shadow(L->val, L->shadow, L->arena);
-  if (rc != NF_OK) return rc;
-  return nf_tc_prepare(L);
+  return nf_ref_shadow(L->val, L->shadow, L->arena);
 }
 
 static int param_ptr(nf_layer* L, int which, float** dev, size_t* n, int* conv_a, int* conv_b) {

@@ -1532,8 +1532,6 @@ size_t nf_tc_red_floats(const nf_layer* L) {
   return fwd > need ? fwd : need;
 }
 
-int nf_tc_prepare(nf_layer*) { return NF_OK; }
-
 int nf_tc_conv_fwd(nf_layer* L, const void* x, int& nb) {
   return run_fwd(L->o.N, L->H, L->W, L->Cin, L->Cout, x, L->shadow + L->off[NF_P_W], L->y, 1, L->red, L->red_floats,
                  L->status, &nb, 0, nullptr, L->o.stride);

@@ -6,8 +6,6 @@
 void nf_tc_select(nf_layer* L);
 // Floats of split-K scratch the tensor-core weight gradient needs (0 if unused).
 size_t nf_tc_scratch_floats(const nf_layer* L);
-// Called once the workspace is bound: encodes the TMA descriptors that point into it.
-int nf_tc_prepare(nf_layer* L);
 // y = conv(x) in bf16 plus per-CTA channel partials (sum, sum of squares) in L->red; nb = partial count.
 int nf_tc_conv_fwd(nf_layer* L, const void* x, int& nb);
 // Same convolution for `count` samples without statistics (cache-filling forward).
