@@ -165,6 +165,17 @@ def nf_trace_read(slots: int = 1):
     return out
 
 
+def run_dp_phases(run_phase, buffer_of, loss_out, all_reduce):
+    """The exchange schedule of the data-parallel step: phase k, then the sum over ranks of exchange buffer k
+    (k = 0, 1, 2); the loss share is summed with the gradients; phase 3 (the update) needs no exchange."""
+    for k in range(4):
+        run_phase(k)
+        if k < 3:
+            all_reduce(buffer_of(k))
+        if k == 2:
+            all_reduce(loss_out)
+
+
 def nf_aan_filters(channels, first_downsample: int):
     """AAN-LL rule: aux filter count per layer (half the smallest channel count before the first down-sampling, half the largest after)."""
     n = len(channels)
@@ -290,13 +301,10 @@ class Layer:
 
     def step_dp(self, x, labels, lr, loss_out, act_out, world, all_reduce):
         """nf_layer_step_dp through its four phases; all_reduce(tensor) must add the tensor over all ranks in place."""
-        for phase in range(4):
-            _check(lib().nf_layer_step_dp(self.h, phase, _ptr(x), _ptr(labels), float(lr), _ptr(loss_out), _ptr(act_out), int(world)),
+        def phase(k):
+            _check(lib().nf_layer_step_dp(self.h, k, _ptr(x), _ptr(labels), float(lr), _ptr(loss_out), _ptr(act_out), int(world)),
                    "nf_layer_step_dp")
-            if phase < 3:
-                all_reduce(self.dp_buffer(phase))
-            if phase == 2:
-                all_reduce(loss_out)
+        run_dp_phases(phase, self.dp_buffer, loss_out, all_reduce)
 
     def param_count(self, part=2) -> int:
         return int(lib().nf_layer_param_count(self.h, part))

@@ -55,3 +55,46 @@ def test_reference_arm_prints_one_json_line_with_the_required_keys():
     assert d["impl"] == "reference" and d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] == d["value"]
     assert d["e2e"] == dict(value=d["value"], unit=d["unit"], h2d_bytes_per_step=0, d2h_bytes_per_step=0)
     assert d["unit"] == "images/s" and d["higher_is_better"] is True and d["value"] > 0
+
+
+def _dp_worker(rank, world, port, q):
+    """A stand-in layer whose phases only write rank-dependent numbers into the exchange buffers: what is checked is
+    the schedule (which buffer is summed after which phase, the loss with the gradients, nothing after the update)."""
+    sys.path.insert(0, ROOT)
+    from paper_2402_14139_b200 import nf
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    bufs = [torch.zeros(4, dtype=torch.float64), torch.zeros(4, dtype=torch.float64), torch.zeros(6)]
+    loss = torch.zeros(1)
+    log = []
+
+    def run_phase(k):
+        log.append(("phase", k, [b.clone() for b in bufs]))
+        if k < 3:
+            bufs[k].fill_(float(10 * k + rank + 1))
+        if k == 2:
+            loss.fill_(0.25 * (rank + 1))
+
+    nf.run_dp_phases(run_phase, lambda k: bufs[k], loss, lambda t: dist.all_reduce(t))
+    q.put((rank, [b.tolist() for b in bufs], float(loss.item()), [(k, [b.tolist() for b in snap]) for _, k, snap in log]))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_data_parallel_exchange_schedule_over_two_gloo_ranks():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29500 + (os.getpid() * 3 + 1) % 2000
+    procs = [ctx.Process(target=_dp_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, bufs, loss, log in res:
+        assert bufs[0] == [3.0] * 4 and bufs[1] == [23.0] * 4 and bufs[2] == [43.0] * 6      # (10k+1) + (10k+2)
+        assert loss == 0.75
+        assert [k for k, _ in log] == [0, 1, 2, 3]
+        assert log[1][1][0] == [3.0] * 4          # buffer 0 was already summed when phase 1 started
+        assert log[2][1][1] == [23.0] * 4 and log[3][1][2] == [43.0] * 6
