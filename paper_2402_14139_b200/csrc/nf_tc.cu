@@ -1415,8 +1415,21 @@ WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0, int strid
   const int blocks = (Cin / 64) * (aux ? 1 : Cout / 64);
   const long pix_tiles = (long)((N + pl.BI - 1) / pl.BI) * (H / pl.BH) * (W / pl.BW);
   const int groups = pl.PT ? 3 : 1;  // kernel rows handled by separate CTAs
-  long sp = sm_count() / (blocks * groups);
-  if (sp < 1) sp = 1;
+  // pixel splits per (chunk pair, kernel-row group): the count whose CTAs fill whole waves of SMs best (smallest on ties),
+  // e.g. 512 -> 512 channels with three row groups: 192 units -> 3 splits = 576 CTAs = 3.9 waves instead of 1.3
+  const int units = blocks * groups, sms = sm_count();
+  long base = sms / units;
+  if (base < 1) base = 1;
+  long sp = base;
+  double best = 0.0;
+  for (long c = 1; c <= (base * 2 > 16 ? base * 2 : 16) && c <= pix_tiles; ++c) {
+    const long total = c * units, waves = (total + sms - 1) / sms;
+    const double eff = (double)total / (double)(waves * sms);
+    if (eff > best + 1e-9) {
+      best = eff;
+      sp = c;
+    }
+  }
   if (sp > pix_tiles) sp = pix_tiles;
   pl.splits = (int)sp;
   pl.grid = (int)(sp * blocks * groups);
