@@ -691,17 +691,18 @@ struct WgParams {
 template <int NB, int S2>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_dy, const WgParams p) {
-  constexpr int kBRow = NB * 2;                                // bytes of one pixel row of the dy tile
-  constexpr uint32_t kBLayout = NB == 64 ? 2 : NB == 32 ? 4 : 6;  // swizzle of that tile
-  constexpr int kBTile = 128 * kBRow;
+  constexpr int kAtoms = NB > 64 ? NB / 64 : 1;                // 64-channel atoms of the dy tile (NB = 128, 256: main conv only)
+  constexpr int kBRow = (NB > 64 ? 64 : NB) * 2;               // bytes of one pixel row of one atom
+  constexpr uint32_t kBLayout = NB >= 64 ? 2 : NB == 32 ? 4 : 6;  // swizzle of that tile
+  constexpr int kBTile = 128 * kBRow;                          // one atom
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   static_assert(S2 == 1, "stride 1 on tileable maps uses conv_wgrad_kw_kernel");
-  constexpr int kStages = 3;
+  constexpr int kStages = NB > 64 ? 2 : 3;
   constexpr int kJobs = 2;  // instructions (accumulators) per 16 pixels
   constexpr int copy_bytes = 16384;  // one 128-pixel tap tile
-  const int stage_bytes = 3 * copy_bytes + 16384;  // the dy tile always gets 16 KB so the unused rows read by the
-                                                   // half-empty last instruction stay inside the stage
+  const int stage_bytes = 3 * copy_bytes + kAtoms * 16384;  // a dy atom always gets 16 KB so the unused rows read by the
+                                                            // half-empty last instruction stay inside the stage
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * stage_bytes);
   uint64_t* full = bars;
   uint64_t* empty = bars + kStages;
@@ -749,11 +750,13 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       if (lane == 0) {
         const int w0 = (t % p.tiles_w) * p.BW, h0 = ((t / p.tiles_w) % p.tiles_h) * p.BH, n = (t / (p.tiles_w * p.tiles_h)) * p.BI;
         uint8_t* st = smem + (size_t)s * stage_bytes;
-        ptx::mbar_expect_tx(&full[s], (uint32_t)(3 * copy_bytes + kBTile));
+        ptx::mbar_expect_tx(&full[s], (uint32_t)(3 * copy_bytes + kAtoms * kBTile));
 #pragma unroll
         for (int kw = 0; kw < 3; ++kw)
           ptx::tma_load_4d(st + kw * copy_bytes, &tm_x, &full[s], cic * 64, p.stride * w0 + kw - 1, p.stride * h0 + khg - 1, n);
-        ptx::tma_load_4d(st + 3 * copy_bytes, &tm_dy, &full[s], coc * NB, w0, h0, n);
+#pragma unroll
+        for (int a = 0; a < kAtoms; ++a)
+          ptx::tma_load_4d(st + 3 * copy_bytes + a * 16384, &tm_dy, &full[s], coc * NB + a * 64, w0, h0, n);
       }
       __syncwarp();
     }
@@ -772,7 +775,7 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         const uint32_t copy16 = (uint32_t)copy_bytes >> 4;
         // descriptors differ only in the address field; the second stacked chunk sits one tap tile further
         const uint64_t a_copy_hi = ptx::sdesc(0, copy_bytes, 1024, 2);
-        const uint64_t b_hi = ptx::sdesc(0, 16, 8 * kBRow, kBLayout);
+        const uint64_t b_hi = ptx::sdesc(0, 16384, 8 * kBRow, kBLayout);  // next 64-channel atom: 16 KB further
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint32_t k16 = k * 128;  // 16 pixels x 128 bytes, in 16-byte units
@@ -1403,16 +1406,17 @@ WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0, int strid
   if (!pick_tile(H, W, true, &pl.BW, &pl.BH, &pl.BI)) return pl;
   pl.PT = (stride == 2 || pl.BI > 1) ? 1 : 0;
   pl.NB = aux ? (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64) : 64;
+  if (!aux && pl.PT) pl.NB = Cout % 256 == 0 ? 256 : Cout % 128 == 0 ? 128 : 64;  // per-tap form: as wide an instruction as Cout allows
   pl.GX = (aux && !pl.PT && pl.NB <= 32) ? 1 : 0;  // few filters: one instruction per 16 pixels with the gradient on the M side
   size_t g_region = (size_t)(pl.GX ? 4 : 3) * 128 * pl.NB * 2;
   if (g_region < 4096) g_region = 4096;
-  const size_t stage = pl.PT ? 65536 : (size_t)(pl.BH + 2) * pl.BW * 128 + g_region;
-  pl.stages = pl.PT ? 3 : (int)((232448 - 2048) / stage);
+  const size_t stage = pl.PT ? (size_t)49152 + (pl.NB > 64 ? pl.NB / 64 : 1) * 16384 : (size_t)(pl.BH + 2) * pl.BW * 128 + g_region;
+  pl.stages = pl.PT ? (pl.NB > 64 ? 2 : 3) : (int)((232448 - 2048) / stage);
   if (pl.stages > kMaxStages) pl.stages = kMaxStages;
   if (pl.stages < 2) return pl;
   pl.smem = (size_t)pl.stages * stage + 1024 + 1024;
   if (pl.smem > 232448) return pl;
-  const int blocks = (Cin / 64) * (aux ? 1 : Cout / 64);
+  const int blocks = (Cin / 64) * (aux ? 1 : Cout / pl.NB);
   const long pix_tiles = (long)((N + pl.BI - 1) / pl.BI) * (H / pl.BH) * (W / pl.BW);
   const int groups = pl.PT ? 3 : 1;  // kernel rows handled by separate CTAs
   // pixel splits per (chunk pair, kernel-row group): the count whose CTAs fill whole waves of SMs best (smallest on ties),
@@ -1485,7 +1489,7 @@ int run_wgrad(int N, int Hin, int Win, int Cin, int Cout, const void* x, const v
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)Win, (uint64_t)Hin, (uint64_t)N};
   const uint32_t bx[4] = {64, (uint32_t)pl.BW, (uint32_t)(pl.PT ? pl.BH : pl.BH + 2), (uint32_t)pl.BI};
   const uint64_t dg[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t bg[4] = {(uint32_t)pl.NB, (uint32_t)pl.BW, (uint32_t)pl.BH, (uint32_t)pl.BI};
+  const uint32_t bg[4] = {(uint32_t)(pl.NB > 64 ? 64 : pl.NB), (uint32_t)pl.BW, (uint32_t)pl.BH, (uint32_t)pl.BI};
   int rc;
   if ((rc = make_map4(&mx, x, dx, bx, stride)) != NF_OK) return rc;
   if ((rc = make_map4(&mg, dy, dg, bg)) != NF_OK) return rc;
@@ -1493,12 +1497,13 @@ int run_wgrad(int N, int Hin, int Win, int Cin, int Cout, const void* x, const v
   p.N = N; p.H = H; p.W = W; p.Cin = Cin; p.Cout = Cout; p.BW = pl.BW; p.BH = pl.BH;
   p.tiles_w = W / pl.BW; p.tiles_h = H / pl.BH; p.pix_tiles = ((N + pl.BI - 1) / pl.BI) * p.tiles_h * p.tiles_w;
   p.stride = stride; p.BI = pl.BI;
-  p.ci_chunks = Cin / 64; p.co_chunks = aux ? 1 : Cout / 64; p.splits = pl.splits; p.part = part; p.status = status;
+  p.ci_chunks = Cin / 64; p.co_chunks = aux ? 1 : Cout / pl.NB; p.splits = pl.splits; p.part = part; p.status = status;
   p.stages = pl.stages;
   if (pl.GX)
     rc = pl.NB == 32 ? launch_wgrad_gx<32>(pl, mx, mg, p) : launch_wgrad_gx<16>(pl, mx, mg, p);
   else if (pl.PT)
-    rc = pl.NB == 64 ? launch_wgrad<64, 1>(pl, mx, mg, p) : pl.NB == 32 ? launch_wgrad<32, 1>(pl, mx, mg, p) : launch_wgrad<16, 1>(pl, mx, mg, p);
+    rc = pl.NB == 256 ? launch_wgrad<256, 1>(pl, mx, mg, p) : pl.NB == 128 ? launch_wgrad<128, 1>(pl, mx, mg, p)
+       : pl.NB == 64 ? launch_wgrad<64, 1>(pl, mx, mg, p) : pl.NB == 32 ? launch_wgrad<32, 1>(pl, mx, mg, p) : launch_wgrad<16, 1>(pl, mx, mg, p);
   else
     rc = pl.NB == 64 ? launch_wgrad_kw<64>(pl, mx, mg, p)
                      : pl.NB == 32 ? launch_wgrad_kw<32>(pl, mx, mg, p) : launch_wgrad_kw<16>(pl, mx, mg, p);

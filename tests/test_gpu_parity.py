@@ -140,6 +140,8 @@ TC = [
     dict(N=200, Cin=64, Cout=64, H=2, W=2, F=32, classes=10, stride=1, pool=True),       # aux conv on 1x1 maps: 128 images per tile
     dict(N=520, Cin=64, Cout=128, H=2, W=2, F=128, classes=10, stride=1, pool=True),     # the same with more than 64 aux filters
     dict(N=300, Cin=64, Cout=64, H=1, W=1, F=16, classes=10, stride=1, pool=False),      # everything on 1x1 maps
+    dict(N=32, Cin=128, Cout=256, H=8, W=8, F=16, classes=10, stride=1, pool=False),     # per-tap weight gradient, 256-wide instructions
+    dict(N=16, Cin=64, Cout=256, H=16, W=16, F=32, classes=10, stride=2, pool=False),    # the same with stride 2
 ]
 
 
