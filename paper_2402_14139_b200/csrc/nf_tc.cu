@@ -202,6 +202,7 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     constexpr int kRowsPer = BN >= 128 ? 128 : 64;  // rows each thread sums for its channel
     const int sc = et % BN, shalf = et / BN;        // stats: channel and row half of this thread
     float ssum = 0.f, ssq = 0.f;
+    float ssum2 = 0.f, ssq2 = 0.f;                  // BN = 256: the thread's second channel, sc + 128
     uint32_t tl = 0;
     int my_nt = blockIdx.x % p.n_tiles;
     for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++tl) {
@@ -259,6 +260,11 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           const float v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(col + row * 128 + ((u ^ (row & 7)) * 16)));
           ssum += v;
           ssq = fmaf(v, v, ssq);
+          if constexpr (BN == 256) {
+            const float v2 = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(col + 2 * 16384 + row * 128 + ((u ^ (row & 7)) * 16)));
+            ssum2 += v2;
+            ssq2 = fmaf(v2, v2, ssq2);
+          }
         }
       }
     }
@@ -268,6 +274,10 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       const size_t b = (size_t)blockIdx.x * parts + shalf;
       p.red[(b * 2 + 0) * p.Cout + my_nt * BN + sc] = ssum;
       p.red[(b * 2 + 1) * p.Cout + my_nt * BN + sc] = ssq;
+      if constexpr (BN == 256) {
+        p.red[(b * 2 + 0) * p.Cout + my_nt * BN + 128 + sc] = ssum2;
+        p.red[(b * 2 + 1) * p.Cout + my_nt * BN + 128 + sc] = ssq2;
+      }
     }
     } else {
       const int et = threadIdx.x - 64;
@@ -1203,6 +1213,7 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride 
   if (!pick_tile(H, W, true, &pl.BW, &pl.BH, &pl.BI)) return pl;
   pl.PT = (stride == 2 || pl.BI > 1) ? 1 : 0;
   pl.BN = epi != 1 ? (Cout % 128 == 0 ? 128 : 64) : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64);
+  if (epi == 0 && pl.PT && Cout % 256 == 0) pl.BN = 256;  // per-tap form: weights of one tap and 256 channels are 32 KB a stage
   pl.KC = epi == 2 ? (Cin <= 16 ? 16 : Cin <= 32 ? 32 : 64) : 64;
   const size_t a_stride = pl.PT ? (size_t)128 * pl.KC * 2 : ((size_t)(pl.BH + 2) * pl.BW * pl.KC * 2 + 1023) & ~(size_t)1023;
   pl.RW = (!pl.PT && epi != 2 && Cin == 64 && pl.BN <= 64) ? 1 : 0;  // weights resident in shared memory
@@ -1366,7 +1377,9 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
     *nb = pl.grid * pl.parts;
   }
   if (pl.PT) {  // per-tap boxes: stride 2, or several small images per tile
-    if (epi == 0) return pl.BN == 128 ? launch_fwd<128, 0, 64, 0, 1>(pl, mx, mw, my, p) : launch_fwd<64, 0, 64, 0, 1>(pl, mx, mw, my, p);
+    if (epi == 0)
+      return pl.BN == 256 ? launch_fwd<256, 0, 64, 0, 1>(pl, mx, mw, my, p)
+                          : pl.BN == 128 ? launch_fwd<128, 0, 64, 0, 1>(pl, mx, mw, my, p) : launch_fwd<64, 0, 64, 0, 1>(pl, mx, mw, my, p);
     if (epi == 1)
       return pl.BN == 16 ? launch_fwd<16, 1, 64, 0, 1>(pl, mx, mw, my, p)
                          : pl.BN == 32 ? launch_fwd<32, 1, 64, 0, 1>(pl, mx, mw, my, p) : launch_fwd<64, 1, 64, 0, 1>(pl, mx, mw, my, p);
