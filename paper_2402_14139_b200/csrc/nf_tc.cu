@@ -1212,6 +1212,7 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride 
   if (epi == 0 ? (Cout % 64 != 0) : epi == 1 ? (Cout > 64) : false) return pl;
   if (!pick_tile(H, W, true, &pl.BW, &pl.BH, &pl.BI)) return pl;
   pl.PT = (stride == 2 || pl.BI > 1) ? 1 : 0;
+  if (epi == 0 && Cout % 256 == 0) pl.PT = 1;  // 256-wide instructions need the per-tap form (one tap of weights per stage)
   pl.BN = epi != 1 ? (Cout % 128 == 0 ? 128 : 64) : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64);
   if (epi == 0 && pl.PT && Cout % 256 == 0) pl.BN = 256;  // per-tap form: weights of one tap and 256 channels are 32 KB a stage
   pl.KC = epi == 2 ? (Cin <= 16 ? 16 : Cin <= 32 ? 32 : 64) : 64;

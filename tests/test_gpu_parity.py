@@ -142,6 +142,7 @@ TC = [
     dict(N=300, Cin=64, Cout=64, H=1, W=1, F=16, classes=10, stride=1, pool=False),      # everything on 1x1 maps
     dict(N=32, Cin=128, Cout=256, H=8, W=8, F=16, classes=10, stride=1, pool=False),     # per-tap weight gradient, 256-wide instructions
     dict(N=16, Cin=64, Cout=256, H=16, W=16, F=32, classes=10, stride=2, pool=False),    # the same with stride 2
+    dict(N=6, Cin=128, Cout=256, H=16, W=32, F=16, classes=10, stride=1, pool=True),     # 256-wide forward on a map that tiles
 ]
 
 
