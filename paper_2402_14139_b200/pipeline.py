@@ -46,9 +46,11 @@ def build_layers(nf, wl, block_index, seed):
     return layers, nf.Block(layers)
 
 
-def plan_blocks(nf, layers, classes, budget_bytes, batch_cap, rho=0.4, batches=(32, 64, 128, 256), dtype="bf16"):
+def plan_blocks(nf, layers, classes, budget_bytes, batch_cap, rho=0.4, batches=(512, 1024, 2048, 4096), dtype="bf16"):
     """Profiler + Partitioner: the linear memory model of every layer (nf_profile_layer), its largest batch under the
-    budget (nf_max_batch) and Algorithm 1 (nf_partition).  Returns [(first_layer, last_layer, batch_size)]."""
+    budget (nf_max_batch) and Algorithm 1 (nf_partition).  Returns [(first_layer, last_layer, batch_size)].
+    The profiled batch sizes are large enough that the split-reduction scratch of small late layers has reached its
+    final size (below that the memory need is not yet a straight line)."""
     dt = nf.NF_F32 if dtype == "f32" else nf.NF_BF16
     max_batch = []
     for l in layers:
