@@ -340,6 +340,18 @@ class Block:
         _check(lib().nf_block_step(self.h, _ptr(x), _ptr(labels), float(lr), _ptr(loss_out), _ptr(act_out)),
                "nf_block_step")
 
+    def capture(self, x, labels, lr, loss_out, act_out=None):
+        """Records one nf_block_step on these (fixed) device buffers into a CUDA graph and returns it; graph.replay()
+        then runs the whole step as one launch, which pays off when the kernels are short (small batches or maps).
+        Run one eager step first: the first use of a kernel sets its attributes, which is not part of a step."""
+        torch = self.layers[0]._torch
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            nf_set_stream(torch.cuda.current_stream())
+            self.step(x, labels, lr, loss_out, act_out)
+        nf_set_stream(torch.cuda.current_stream())
+        return g
+
     def step_host_next(self, x_host, labels_host, lr, loss_host, next_x_host=None, next_labels_host=None, act_host=None):
         """nf_block_step_host_next: trains on (x_host, labels_host) while the next batch is copied to the device."""
         _check(lib().nf_block_step_host_next(self.h, _ptr(x_host), _ptr(labels_host), float(lr), _ptr(loss_host), _ptr(act_host),

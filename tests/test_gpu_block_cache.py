@@ -146,3 +146,39 @@ def test_prefetching_host_step_equals_plain_host_step():
             assert np.array_equal(ga.get_param(name), gb.get_param(name)), name
     # the plain layer (host_io = 1) has no second buffer: the call is refused
     assert nf.lib().nf_block_step_host_next(A.h, nf._ptr(xs[0]), nf._ptr(ys[0]), 0.05, nf._ptr(la_h), None, None, None) == nf.NF_EINVAL
+
+
+def test_captured_block_step_replays_identically():
+    """nf.Block.capture: the whole block step recorded into a CUDA graph; replays give bit-identical losses and
+    parameters to the same number of eager steps."""
+    import torch
+    from paper_2402_14139_b200 import nf
+    nf.lib()
+    nf.nf_set_stream(None)
+    c1 = dict(N=8, Cin=3, Cout=64, H=16, W=16, F=16, classes=10, stride=1, pool=False)
+    c2 = dict(N=8, Cin=64, Cout=64, H=16, W=16, F=8, classes=10, stride=1, pool=True)
+    P1, x, y = pu.seeded_case(c1, 81, bf16=True)
+    P2, _, _ = pu.seeded_case(c2, 82, bf16=True)
+    xd, yd = pu.to_device_nhwc(torch, x, 1), torch.from_numpy(y).cuda()
+
+    def run(graph):
+        layers = [pu.gpu_layer(nf, c1, P1, nf.NF_BF16), pu.gpu_layer(nf, c2, P2, nf.NF_BF16)]
+        blk = nf.Block(layers)
+        loss = torch.zeros(2, device="cuda")
+        blk.step(xd, yd, 0.05, loss)                     # the eager step that must precede a capture
+        if graph:
+            g = blk.capture(xd, yd, 0.05, loss)
+            for _ in range(3):
+                g.replay()
+        else:
+            for _ in range(3):
+                blk.step(xd, yd, 0.05, loss)
+        torch.cuda.synchronize()
+        out = loss.cpu().numpy().copy(), [L.get_param("W") for L in layers], [L.status() for L in layers]
+        nf.nf_set_stream(None)
+        return out
+
+    (la, wa, sa), (lb, wb, sb) = run(False), run(True)
+    assert sa == sb == [0, 0] and np.array_equal(la, lb)
+    for a, b in zip(wa, wb):
+        assert np.array_equal(a, b)
