@@ -30,6 +30,10 @@ struct FwdParams {
   int32_t* status;    // device status word
   const float* bias;  // EPI 1: per-channel bias added before the ReLU
   bf16* out;          // EPI 1: destination [N][H][W][Cout], written straight from registers
+  // stats == 2 (EPI 0): the output is the gradient da at a BatchNorm+ReLU output of the same shape; the partial sums are
+  // (dz, dz * xhat) with dz = da * 1[y2*scale+shift > 0], and the tiles of y2 come through tm_y2
+  const float *bn_scale, *bn_shift, *bn_mu, *bn_invstd;
+  CUtensorMap tm_y2;
 };
 
 struct TcPlan {
@@ -52,7 +56,7 @@ struct TcPlan {
 template <int BN, int EPI, int KC = 64, int BMN = 0, int PT = 0, int RW = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-                   const __grid_constant__ CUtensorMap tm_y, const FwdParams p) {
+                   const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ FwdParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int kARow = KC * 2;  // bytes of one pixel row of the activation box
@@ -65,13 +69,16 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   constexpr int kSub = EPI == 0 ? BN / 64 : 0;  // 64-channel sub-tiles of the output staging
   uint8_t* wres = smem + (size_t)p.stages * stage_bytes;
   uint8_t* stg = wres + w_bytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + kSub * 16384);
+  uint8_t* ybuf = stg + kSub * 16384;  // stats 2: the y2 tile of the tile in the epilogue (kSub sub-tiles)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (p.stats == 2 ? 2 : 1) * kSub * 16384);
   uint64_t* full = bars;
   uint64_t* empty = bars + kMaxStages;
   uint64_t* tfull = bars + 2 * kMaxStages;
   uint64_t* tempty = tfull + 2;
   uint64_t* wfull = tempty + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wfull + 1);
+  uint64_t* yfull = wfull + 1;
+  uint64_t* yempty = yfull + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(yempty + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
@@ -88,6 +95,8 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       ptx::mbar_init(&tempty[a], 128);
     }
     ptx::mbar_init(wfull, 1);
+    ptx::mbar_init(yfull, 1);
+    ptx::mbar_init(yempty, 128);
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tmap(&tm_x);
@@ -116,7 +125,8 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       }
       __syncwarp();
     }
-    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x) {
+    uint32_t ptl = 0;
+    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++ptl) {
       const int nt = t % p.n_tiles, m = t / p.n_tiles;
       const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = (m / (p.tiles_w * p.tiles_h)) * p.BI;
       for (int ks = 0; ks < ksteps; ++ks, ++it) {
@@ -149,6 +159,19 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           }
         }
         __syncwarp();
+      }
+      if constexpr (EPI == 0) {
+        // the y2 tile of this output tile goes out after its operand loads: the single buffer is free once the epilogue
+        // has finished the statistics of the previous tile, which it does while this tile is being multiplied
+        if (ok && p.stats == 2) {
+          if (!__all_sync(0xffffffffu, ptx::mbar_wait(yempty, (ptl & 1) ^ 1, abort_flag))) break;
+          if (lane == 0) {
+            ptx::mbar_expect_tx(yfull, (uint32_t)(kSub * 16384));
+#pragma unroll
+            for (int sb = 0; sb < kSub; ++sb) ptx::tma_load_4d(ybuf + sb * 16384, &p.tm_y2, yfull, nt * BN + sb * 64, w0, h0, n);
+          }
+          __syncwarp();
+        }
       }
     }
   } else if (warp == 1) {
@@ -205,6 +228,16 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     float ssum2 = 0.f, ssq2 = 0.f;                  // BN = 256: the thread's second channel, sc + 128
     uint32_t tl = 0;
     int my_nt = blockIdx.x % p.n_tiles;
+    float bsc = 0.f, bsh = 0.f, bsc2 = 0.f, bsh2 = 0.f;  // stats 2: BatchNorm scale / shift of the thread's channel(s)
+    if (p.stats == 2) {
+      const int ch = my_nt * BN + sc;
+      bsc = p.bn_scale[ch];
+      bsh = p.bn_shift[ch];
+      if constexpr (BN == 256) {
+        bsc2 = p.bn_scale[ch + 128];
+        bsh2 = p.bn_shift[ch + 128];
+      }
+    }
     for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++tl) {
       const int nt = t % p.n_tiles, m = t / p.n_tiles;
       const int w0 = (m % p.tiles_w) * p.BW, h0 = ((m / p.tiles_w) % p.tiles_h) * p.BH, n = (m / (p.tiles_w * p.tiles_h)) * p.BI;
@@ -250,7 +283,31 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         for (int sb = 0; sb < kSub; ++sb) ptx::tma_store_4d(&tm_y, stg + sb * 16384, nt * BN + sb * 64, w0, h0, n);
         ptx::tma_store_commit();
       }
-      if (p.stats) {
+      if (p.stats == 2) {
+        // sums of dz and dz*y2 (the last step turns them into sum dz*xhat = invstd * (sum dz*y2 - mu * sum dz))
+        ptx::mbar_wait(yfull, tl & 1, abort_flag);
+        const int coff = (sc / 64) * 16384 + (sc % 8) * 2;
+        const int u = (sc % 64) / 8;
+        const int rb = shalf * kRowsPer;
+#pragma unroll 8
+        for (int rr = 0; rr < kRowsPer; ++rr) {
+          const int row = rb + rr;
+          const int off = coff + row * 128 + ((u ^ (row & 7)) * 16);
+          const float d = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(stg + off));
+          const float yv = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(ybuf + off));
+          const float dz = fmaf(yv, bsc, bsh) > 0.f ? d : 0.f;
+          ssum += dz;
+          ssq = fmaf(dz, yv, ssq);
+          if constexpr (BN == 256) {
+            const float d2 = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(stg + 2 * 16384 + off));
+            const float y2 = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(ybuf + 2 * 16384 + off));
+            const float dz2 = fmaf(y2, bsc2, bsh2) > 0.f ? d2 : 0.f;
+            ssum2 += dz2;
+            ssq2 = fmaf(dz2, y2, ssq2);
+          }
+        }
+        ptx::mbar_arrive(yempty);
+      } else if (p.stats) {
         const uint8_t* col = stg + (sc / 64) * 16384 + (sc % 8) * 2;
         const int u = (sc % 64) / 8;
         const int rb = shalf * kRowsPer;
@@ -272,6 +329,11 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     if (p.stats) {
       constexpr int parts = 128 / BN > 0 ? 128 / BN : 1;
       const size_t b = (size_t)blockIdx.x * parts + shalf;
+      if (p.stats == 2) {
+        const int ch = my_nt * BN + sc;
+        ssq = (float)((double)p.bn_invstd[ch] * ((double)ssq - (double)p.bn_mu[ch] * (double)ssum));
+        if constexpr (BN == 256) ssq2 = (float)((double)p.bn_invstd[ch + 128] * ((double)ssq2 - (double)p.bn_mu[ch + 128] * (double)ssum2));
+      }
       p.red[(b * 2 + 0) * p.Cout + my_nt * BN + sc] = ssum;
       p.red[(b * 2 + 1) * p.Cout + my_nt * BN + sc] = ssq;
       if constexpr (BN == 256) {
@@ -1205,7 +1267,8 @@ bool pick_tile(int H, int W, bool allow_multi, int* BW, int* BH, int* BI) {
   return false;
 }
 
-TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride = 1) {
+// ybuf = 1 reserves the y2 tile of the fused BatchNorm-backward sums (as large as the output staging)
+TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride = 1, int ybuf = 0) {
   TcPlan pl{};
   if (stride == 2 && (epi != 0 || Cin % 64)) return pl;
   if (epi == 2 ? (Cin > 64 || Cin % 8 || Cout % 64) : (Cin % 64 != 0)) return pl;
@@ -1221,7 +1284,7 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride 
   const size_t b_stage = pl.RW ? 0 : pl.PT ? (epi == 2 ? (size_t)(pl.BN / 64) * pl.KC * 128 : (size_t)pl.BN * 128)
                                            : epi == 2 ? (size_t)(pl.BN / 64) * 3 * pl.KC * 128 : (size_t)3 * pl.BN * 128;
   const size_t stage = ((a_stride + 1023) & ~(size_t)1023) + b_stage;
-  const size_t fixed = (size_t)(epi != 1 ? pl.BN / 64 : 0) * 16384 + (pl.RW ? (size_t)9 * pl.BN * 128 : 0) + 1024 + 1024;
+  const size_t fixed = (size_t)(epi != 1 ? pl.BN / 64 : 0) * 16384 * (ybuf ? 2 : 1) + (pl.RW ? (size_t)9 * pl.BN * 128 : 0) + 1024 + 1024;
   int st = (int)((232448 - fixed) / stage);
   if (st > kMaxStages) st = kMaxStages;
   if (st < 2) return pl;
@@ -1341,11 +1404,13 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
 // epi 0: y through TMA + optional statistics.  epi 1: out = ReLU(conv + bias) written directly (y unused).
 // H, W are the INPUT size; stride 2 halves them (rounding up) for the output.
 int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
-            size_t red_floats, int32_t* status, int* nb, int epi = 0, const float* bias = nullptr, int stride = 1) {
+            size_t red_floats, int32_t* status, int* nb, int epi = 0, const float* bias = nullptr, int stride = 1,
+            const BnBwdIn* bn = nullptr) {
   const int H = (Hin - 1) / stride + 1, W = (Win - 1) / stride + 1;
   if (fold_ok(H, W, Cin, Cout, epi, stride))
-    return run_fold(N, H, W, Cin, Cout, x, w, y, stats, red, red_floats, status, nb, epi, bias);
-  const TcPlan pl = plan_fwd(H, W, Cin, Cout, N, epi, stride);
+    return run_fold(N, H, W, Cin, Cout, x, w, y, stats, red, red_floats, status, nb, epi, bias, bn);
+  if (stats == 2 && (!bn || epi == 1)) return NF_EINVAL;
+  const TcPlan pl = plan_fwd(H, W, Cin, Cout, N, epi, stride, stats == 2);
   if (!pl.ok) return NF_EUNSUPPORTED;
   CUtensorMap mx, mw, my;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)Win, (uint64_t)Hin, (uint64_t)N};
@@ -1371,6 +1436,11 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
   p.total_tiles = ((N + pl.BI - 1) / pl.BI) * p.tiles_h * p.tiles_w * p.n_tiles;
   p.stride = stride; p.BI = pl.BI;
   p.kchunks = epi == 2 ? 1 : Cin / 64; p.stages = pl.stages; p.stats = stats; p.red = red; p.status = status;
+  p.tm_y2 = my;
+  if (stats == 2) {
+    if ((rc = make_map4(&p.tm_y2, bn->y2, dy, by)) != NF_OK) return rc;
+    p.bn_scale = bn->scale; p.bn_shift = bn->shift; p.bn_mu = bn->mu; p.bn_invstd = bn->invstd;
+  }
   if (stats) {
     const size_t need = (size_t)pl.grid * pl.parts * 2 * Cout;
     if (need > red_floats) return NF_ENOWS;
@@ -1593,20 +1663,30 @@ int nf_tc_wgrad(nf_layer* L, const void* x) {
 int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb) {
   int nb = 0;
   *bn_nb = 0;
-  if (wide_aux(L)) {
+  const bool wide = wide_aux(L);
+  const void* w = L->shadow + L->off[NF_P_WA];
+  if (wide) {
     const int rc = nf_ref_flip_weights(L->shadow + L->off[NF_P_WA], L->F, L->Cout, L->wa_t);
     if (rc != NF_OK) return rc;
-    return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->wa_t, L->da, 0, nullptr, 0, L->status, &nb, 0);
+    w = L->wa_t;
   }
-  // without a pool da has the shape of y: the folded kernel also reduces (dz, dz*xhat) per channel while it holds the tile
-  if (!L->o.maxpool && !L->skip && fold_ok(L->Ha, L->Wa, L->F, L->Cout, 2, 1) &&
-      (size_t)(sm_count() / (L->Cout / 64)) * 8 * 2 * L->Cout <= L->red_floats) {
+  const int epi = wide ? 0 : 2;
+  // Without a pool (and without a shortcut) da has the shape of y, and the kernel that produces it also reduces
+  // (dz, dz*xhat) per channel while it holds the tile: the BatchNorm backward then needs no reduction pass.
+  if (!L->o.maxpool && !L->skip) {
     const BnBwdIn bn{L->y, L->scale, L->shift, L->mu, L->invstd};
-    return run_fold(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->shadow + L->off[NF_P_WA], L->da, 2, L->red, L->red_floats,
-                    L->status, bn_nb, 2, nullptr, &bn);
+    bool fits;
+    if (fold_ok(L->Ha, L->Wa, L->F, L->Cout, epi, 1)) {
+      fits = (size_t)(sm_count() / (L->Cout / 64)) * 8 * 2 * L->Cout <= L->red_floats;
+    } else {
+      const TcPlan pl = plan_fwd(L->Ha, L->Wa, L->F, L->Cout, L->o.N, epi, 1, 1);
+      fits = pl.ok && (size_t)pl.grid * pl.parts * 2 * L->Cout <= L->red_floats;
+    }
+    if (fits)
+      return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, w, L->da, 2, L->red, L->red_floats, L->status, bn_nb, epi, nullptr,
+                     1, &bn);
   }
-  return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->shadow + L->off[NF_P_WA], L->da, 0, nullptr, 0, L->status,
-                 &nb, 2);
+  return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, w, L->da, 0, nullptr, 0, L->status, &nb, epi);
 }
 
 int nf_tc_aux_wgrad(nf_layer* L, const void* a) {
