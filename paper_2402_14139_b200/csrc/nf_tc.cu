@@ -877,8 +877,8 @@ conv_wgrad_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         const int tapA = khg * 3 + (j == 0 ? 0 : 2);
         const int tapB = j == 0 ? khg * 3 + 1 : -1;
         const int tap = m < 64 ? tapA : tapB;
-#pragma unroll
-        for (int q = 0; q < NB / 16; ++q) {
+#pragma unroll 2
+        for (int q = 0; q < NB / 16; ++q) {  // not fully unrolled: 16 column blocks of address arithmetic spill at NB = 256
           uint32_t v[16];
           ptx::tmem_ld16(tmem_base + ((uint32_t)(lg * 32) << 16) + j * NB + q * 16, v);
           ptx::tmem_ld_wait();
