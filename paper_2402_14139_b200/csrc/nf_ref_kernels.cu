@@ -120,12 +120,32 @@ __global__ void __launch_bounds__(256) wgrad_direct_kernel(const T* __restrict__
     for (int t = 0; t < 9; ++t) part[(((size_t)sp * 9 + t) * Co + co0 + co_l) * Ci + ci0 + ci_l] = acc[t];
 }
 
-__global__ void sum_splits_kernel(const float* __restrict__ part, int splits, size_t n, float* __restrict__ out) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
+// out[i] = sum over the splits of part[k][i]: 32 consecutive elements x 8 lanes over the splits per block; a lane adds its
+// splits in index order with four loads in flight, the lane sums are added in lane order (fixed order, no atomics)
+__global__ void __launch_bounds__(256) sum_splits_kernel(const float* __restrict__ part, int splits, size_t n, float* __restrict__ out) {
+  __shared__ float sm[8][33];
+  const size_t i = (size_t)blockIdx.x * 32 + threadIdx.x;
   float s = 0.f;
-  for (int k = 0; k < splits; ++k) s += part[(size_t)k * n + i];
-  out[i] = s;
+  if (i < n) {
+    int k = threadIdx.y;
+    for (; k + 3 * 8 < splits; k += 4 * 8) {
+      const float a = part[(size_t)k * n + i], b = part[(size_t)(k + 8) * n + i], c = part[(size_t)(k + 16) * n + i],
+                  d = part[(size_t)(k + 24) * n + i];
+      s += a;
+      s += b;
+      s += c;
+      s += d;
+    }
+    for (; k < splits; k += 8) s += part[(size_t)k * n + i];
+  }
+  sm[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0 && i < n) {
+    float t = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) t += sm[j][threadIdx.x];
+    out[i] = t;
+  }
 }
 
 
@@ -321,7 +341,7 @@ int nf_ref_wgrad(int dtype, const void* x, int N, int H, int W, int Ci, const vo
       wgrad_smallc_kernel<bf16><<<splits, blk, sm, g_nf_stream>>>((const bf16*)x, N, H, W, Ci, (const bf16*)g, Co, stride, Ho, Wo,
                                                                 splits, part);
     NF_LAUNCHED();
-    sum_splits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, g_nf_stream>>>(part, splits, n, dw);
+    sum_splits_kernel<<<(unsigned)((n + 31) / 32), dim3(32, 8), 0, g_nf_stream>>>(part, splits, n, dw);
     NF_LAUNCHED();
     return NF_OK;
   }
@@ -333,7 +353,7 @@ int nf_ref_wgrad(int dtype, const void* x, int N, int H, int W, int Ci, const vo
     wgrad_direct_kernel<bf16><<<blocks, 256, 0, g_nf_stream>>>((const bf16*)x, N, H, W, Ci, (const bf16*)g, Co,
                                                                stride, Ho, Wo, splits, part);
   NF_LAUNCHED();
-  sum_splits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, g_nf_stream>>>(part, splits, n, dw);
+  sum_splits_kernel<<<(unsigned)((n + 31) / 32), dim3(32, 8), 0, g_nf_stream>>>(part, splits, n, dw);
   NF_LAUNCHED();
   return NF_OK;
 }
