@@ -466,23 +466,39 @@ __global__ void __launch_bounds__(256) fc_wgrad_kernel(const float* __restrict__
                                                        const float* __restrict__ lossn, int N, int D, int K,
                                                        float* __restrict__ gWf, float* __restrict__ gbf,
                                                        float* __restrict__ loss_out, int32_t* status, int n_scale) {
+  // Sums over the batch run as four interleaved chains (samples n % 4) that are combined in a fixed order, and the
+  // two scalar sums are spread over a warp: the serial chains of one load per sample were pure latency.
   const int k = blockIdx.x, t = threadIdx.x;
   for (int d = t; d < D; d += 256) {
-    float s = 0.f;
-    for (int n = 0; n < N; ++n) s = fmaf(dl[(size_t)n * K + k], p[(size_t)n * D + d], s);
-    gWf[(size_t)k * D + d] = s;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    int n = 0;
+    for (; n + 3 < N; n += 4) {
+      s0 = fmaf(dl[(size_t)n * K + k], p[(size_t)n * D + d], s0);
+      s1 = fmaf(dl[(size_t)(n + 1) * K + k], p[(size_t)(n + 1) * D + d], s1);
+      s2 = fmaf(dl[(size_t)(n + 2) * K + k], p[(size_t)(n + 2) * D + d], s2);
+      s3 = fmaf(dl[(size_t)(n + 3) * K + k], p[(size_t)(n + 3) * D + d], s3);
+    }
+    for (; n < N; ++n) s0 = fmaf(dl[(size_t)n * K + k], p[(size_t)n * D + d], s0);
+    gWf[(size_t)k * D + d] = (s0 + s1) + (s2 + s3);
   }
-  if (t == 0) {
+  const int warp = t >> 5, lane = t & 31;
+  if (warp == 7) {  // gbf[k]: lane sums over n = lane, lane + 32, ..., then a fixed butterfly
     float s = 0.f;
-    for (int n = 0; n < N; ++n) s += dl[(size_t)n * K + k];
-    gbf[k] = s;
+    for (int n = lane; n < N; n += 32) s += dl[(size_t)n * K + k];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) gbf[k] = s;
   }
-  if (k == 0 && t == 32) {
+  if (k == 0 && warp == 6) {
     double s = 0.0;
-    for (int n = 0; n < N; ++n) s += (double)lossn[n];
-    const float L = (float)(s / (double)n_scale);
-    *loss_out = L;
-    if (!isfinite(L)) atomicOr(status, NF_ENONFINITE);
+    for (int n = lane; n < N; n += 32) s += (double)lossn[n];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) {
+      const float L = (float)(s / (double)n_scale);
+      *loss_out = L;
+      if (!isfinite(L)) atomicOr(status, NF_ENONFINITE);
+    }
   }
 }
 
