@@ -439,7 +439,11 @@ struct FoldParams {
 // KC / MIR: KC = channels of the activation box (64; 16 or 32 for the aux input gradient whose input dh has F
 // channels), MIR = 1 reads the weights [tap][f][c] MN-major with both taps mirrored (input-gradient convolution;
 // the CTA's 64-channel output tile is blockIdx.x % n_tiles).
-template <int G, int EPI, int KC = 64, int MIR = 0>
+// UF = 1 (input gradient with KC <= 32 only): the column taps are NOT folded.  With so few input channels a tile needs
+// only nine instructions (one per tap, N = 64) even unfolded, and the epilogue is what bounds the kernel: three
+// column-shifted activation boxes per stage replace the shift-add, the accumulator is 64 columns wide and all 16 x 8
+// pixels of a tile are outputs (W % 16 == 0).
+template <int G, int EPI, int KC = 64, int MIR = 0, int UF = 0>
 __global__ void __launch_bounds__(kFoldThreads, 1)
 conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                      const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_y2, const FoldParams p) {
@@ -447,11 +451,14 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int kARow = KC * 2;               // bytes of one pixel of the activation box
   constexpr uint32_t kALayout = KC == 64 ? 2 : KC == 32 ? 4 : 6;
-  constexpr int kABytes = 10 * 16 * kARow;    // (8+2) rows x 16 pixels x KC channels
+  static_assert(!UF || (MIR && EPI == 0 && G == 64 && KC <= 32), "unfolded form: input gradient with few input channels");
+  constexpr int kBox = 10 * 16 * kARow;       // (8+2) rows x 16 pixels x KC channels
+  constexpr int kABytes = (UF ? 3 : 1) * kBox;  // UF: one box per column tap
+  constexpr int kTW = UF ? 16 : 14;           // output columns of a tile
   constexpr int kWTile = MIR ? 3 * KC * 128 : 3 * G * 128;  // one kernel row: [kw*G + co][64 ci], or mirrored [kw][f][64 c]
   const int w_bytes = 3 * p.kchunks * kWTile; // [chunk][kh][kw*G + co][64 ci]
   uint8_t* wres = smem + (size_t)p.stages * kABytes;
-  uint8_t* stg = wres + w_bytes;              // EPI 0: 112 output pixels x 128 bytes
+  uint8_t* stg = wres + w_bytes;              // EPI 0: 112 (UF: 128) output pixels x 128 bytes
   uint8_t* ybuf = stg + 2 * 16384;            // EPI 0, stats 2: two tiles of y2 per epilogue group
   uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (EPI == 0 ? (p.stats == 2 ? 6 : 2) * 16384 : 0));  // one staging tile per epilogue group
   uint64_t* full = bars;
@@ -511,14 +518,20 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     bool ok = true;
     for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++tl) {
       const int m = t / p.n_tiles;
-      const int w0 = (m % p.tiles_w) * 14, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
+      const int w0 = (m % p.tiles_w) * kTW, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
       for (int ck = 0; ck < p.kchunks; ++ck, ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) { ok = false; break; }
         if (lane == 0) {
           ptx::mbar_expect_tx(&full[s], (uint32_t)kABytes);
-          ptx::tma_load_4d(smem + (size_t)s * kABytes, &tm_x, &full[s], ck * KC, w0 - 1, h0 - 1, n);
+          if constexpr (UF) {
+#pragma unroll
+            for (int kw = 0; kw < 3; ++kw)
+              ptx::tma_load_4d(smem + (size_t)s * kABytes + kw * kBox, &tm_x, &full[s], ck * KC, w0 - 1 + kw, h0 - 1, n);
+          } else {
+            ptx::tma_load_4d(smem + (size_t)s * kABytes, &tm_x, &full[s], ck * KC, w0 - 1, h0 - 1, n);
+          }
         }
         __syncwarp();
       }
@@ -527,7 +540,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           const uint32_t k2 = tl >> 1, slot = (tl & 1) * 2 + (k2 & 1);
           if (!__all_sync(0xffffffffu, ptx::mbar_wait(&yempty[slot], ((k2 >> 1) & 1) ^ 1, abort_flag))) break;
           if (lane == 0) {
-            ptx::mbar_expect_tx(&yfull[slot], 14 * 8 * 128);
+            ptx::mbar_expect_tx(&yfull[slot], kTW * 8 * 128);
             ptx::tma_load_4d(ybuf + slot * 16384, &tm_y2, &yfull[slot], (t % p.n_tiles) * 64, w0, h0, n);
           }
           __syncwarp();
@@ -535,7 +548,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       }
     }
   } else if (warp == 1) {
-    constexpr uint32_t idesc = ptx::idesc_bf16(128, 3 * G, 0, MIR);
+    constexpr uint32_t idesc = ptx::idesc_bf16(128, UF ? G : 3 * G, 0, MIR);
     const uint64_t a_hi = ptx::sdesc(0, 16, 8 * kARow, kALayout);
     const uint64_t b_hi = MIR ? ptx::sdesc(0, KC * 128, 1024, 2) : ptx::sdesc(0, 16, 1024, 2);
     const uint32_t w16 = ptx::smem_u32(wres) >> 4;
@@ -553,6 +566,18 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         ptx::tc_fence_after();
         if (lane == 0) {
           const uint32_t a16 = ptx::smem_u32(smem + (size_t)s * kABytes) >> 4;
+          if constexpr (UF) {  // one instruction per tap and 16 input channels; tap (kh, kw) reads the mirrored weight tile
+#pragma unroll
+            for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+              for (int kw = 0; kw < 3; ++kw)
+#pragma unroll
+                for (int k = 0; k < KC / 16; ++k) {
+                  const uint64_t ad = a_hi | (uint64_t)(a16 + kw * (kBox >> 4) + kh * (16 * kARow >> 4) + k * 2);
+                  const uint64_t bd = b_hi | (uint64_t)(w16 + (2 - kh) * (kWTile >> 4) + (2 - kw) * (KC * 128 >> 4) + k * 128);
+                  ptx::mma_f16(d, ad, bd, idesc, (kh | kw | k) != 0);
+                }
+          } else
 #pragma unroll
           for (int kh = 0; kh < 3; ++kh)
 #pragma unroll
@@ -577,8 +602,8 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     const int lg = warp & 3;
     const int r = lg * 32 + lane;            // TMEM lane = extended-tile pixel (we = r % 16, h = r / 16)
     const int we = r & 15, hh = r >> 4;
-    const bool valid = we >= 1 && we <= 14;
-    const int orow = (we - 1) + 14 * hh;     // row of the output staging tile
+    const bool valid = UF || (we >= 1 && we <= 14);
+    const int orow = UF ? r : (we - 1) + 14 * hh;  // row of the output staging tile
     // statistics: a thread owns 8 channels (one 16-byte chunk of a pixel row) and the 7 rows rg, rg+16, ...
     const int schunk = et & 7, srg = et >> 3;
     float s1[8], s2[8], bsc[8], bsh[8];
@@ -596,7 +621,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     for (int t = blockIdx.x + grp * gridDim.x; t < p.total_tiles; t += 2 * gridDim.x, tl += 2) {
       const int nt = t % p.n_tiles;
       const int m = t / p.n_tiles;
-      const int w0 = (m % p.tiles_w) * 14, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
+      const int w0 = (m % p.tiles_w) * kTW, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
       const uint32_t acc = grp, aph = (tl >> 1) & 1;
       ptx::mbar_wait(&tfull[acc], aph, abort_flag);
       ptx::tc_fence_after();
@@ -611,11 +636,20 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
       for (int q = 0; q < G / 16; ++q) {     // 16 output channels at a time
         uint32_t v0[16], v1[16], v2[16];
+        uint32_t w[8];
+        if constexpr (UF) {
+          ptx::tmem_ld16(tbase + q * 16, v1);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v1[2 * e]), __uint_as_float(v1[2 * e + 1]));
+            w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+          }
+        } else {
         ptx::tmem_ld16(tbase + (MIR ? 2 * G : 0) + q * 16, v0);  // group feeding the pixel on the left
         ptx::tmem_ld16(tbase + G + q * 16, v1);
         ptx::tmem_ld16(tbase + (MIR ? 0 : 2 * G) + q * 16, v2);  // group feeding the pixel on the right
         ptx::tmem_ld_wait();
-        uint32_t w[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           float o[2];
@@ -634,6 +668,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           }
           const __nv_bfloat162 b2 = __floats2bfloat162_rn(o[0], o[1]);
           w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+        }
         }
         if constexpr (EPI == 0) {
           if (valid) {
@@ -664,7 +699,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           ptx::mbar_wait(&yfull[slot], (k2 >> 1) & 1, abort_flag);
           const uint8_t* yb = ybuf + slot * 16384;
 #pragma unroll
-          for (int rr = 0; rr < 7; ++rr) {
+          for (int rr = 0; rr < kTW / 2; ++rr) {
             const int row = srg + 16 * rr;
             const int off = row * 128 + ((schunk ^ (row & 7)) * 16);
             const uint4 dq = *reinterpret_cast<const uint4*>(stg_g + off);
@@ -685,7 +720,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           ptx::mbar_arrive(&yempty[slot]);
         } else if (p.stats) {
 #pragma unroll
-          for (int rr = 0; rr < 7; ++rr) {
+          for (int rr = 0; rr < kTW / 2; ++rr) {
             const int row = srg + 16 * rr;
             const uint4 vq = *reinterpret_cast<const uint4*>(stg_g + row * 128 + ((schunk ^ (row & 7)) * 16));
             const uint32_t vw[4] = {vq.x, vq.y, vq.z, vq.w};
@@ -1316,10 +1351,15 @@ int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, c
 
 // The folded-tap kernel covers, when W % 14 == 0 and H % 8 == 0: the main forward 64 -> 64 (epi 0), the aux
 // forward with F <= 64, F % 8 == 0 (epi 1) if all weight tiles fit in shared memory beside >= 3 activation
-// stages, and the aux input gradient F -> Cout (epi 2; F <= 32, F % 8 == 0, Cout % 64 == 0).
+// stages, and the aux input gradient F -> Cout (epi 2; F <= 32, F % 8 == 0, Cout % 64 == 0).  The input gradient
+// also takes widths that tile by 16 instead of 14 (its unfolded form): always with the fused BatchNorm-backward
+// sums (stats 2) or 64 output channels; without the sums a wider layer is faster on the generic kernel's
+// 128-channel tiles (measured).
 int fold_group(int Cout, int epi) { return epi != 1 ? 64 : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64); }
-bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride) {
-  if (stride != 1 || W % 14 || H % 8) return false;
+bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride, int stats = 0) {
+  if (stride != 1 || H % 8) return false;
+  if (epi == 2 && W % 14 && W % 16 == 0 && (stats == 2 || Cout == 64)) return Cin <= 32 && Cin % 8 == 0 && Cout % 64 == 0;
+  if (W % 14) return false;
   if (epi == 2) return Cin <= 32 && Cin % 8 == 0 && Cout % 64 == 0;
   if (Cin % 64) return false;
   if (epi == 0 ? (Cin != 64 || Cout != 64) : (Cout > 64 || Cout % 8)) return false;
@@ -1327,15 +1367,15 @@ bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride) {
   return wbytes + (epi == 0 ? 2 * 16384 : 0) + 2048 + 3 * 20480 <= 232448;
 }
 
-template <int G, int EPI, int KC = 64, int MIR = 0>
+template <int G, int EPI, int KC = 64, int MIR = 0, int UF = 0>
 int launch_fold(int grid, size_t smem, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const CUtensorMap& my2,
                 const FoldParams& p) {
   static bool attr_done = false;
   if (!attr_done) {
-    NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel<G, EPI, KC, MIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel<G, EPI, KC, MIR, UF>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
   }
-  conv_fwd_fold_kernel<G, EPI, KC, MIR><<<grid, kFoldThreads, smem, g_nf_stream>>>(mx, mw, my, my2, p);
+  conv_fwd_fold_kernel<G, EPI, KC, MIR, UF><<<grid, kFoldThreads, smem, g_nf_stream>>>(mx, mw, my, my2, p);
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -1350,6 +1390,9 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
              size_t red_floats, int32_t* status, int* nb, int epi, const float* bias, const BnBwdIn* bn = nullptr) {
   const int G = fold_group(Cout, epi);
   const int KC = epi == 2 ? (Cin <= 16 ? 16 : 32) : 64;
+  // input gradient on widths that also tile by 16: the unfolded form (three shifted boxes, no shift-add in the epilogue)
+  const bool uf = epi == 2 && W % 16 == 0;
+  const int TW = uf ? 16 : 14;
   CUtensorMap mx, mw, my, my2;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
   const uint32_t bx[4] = {(uint32_t)KC, 16, 10, 1};
@@ -1358,7 +1401,7 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   const uint64_t dw[4] = {(uint64_t)(epi == 2 ? Cout : Cin), (uint64_t)(epi == 2 ? Cin : Cout), 3, 3};
   const uint32_t bw[4] = {64, (uint32_t)(epi == 2 ? KC : G), 3, 1};
   const uint64_t dy[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t by[4] = {64, 14, 8, 1};
+  const uint32_t by[4] = {64, (uint32_t)TW, 8, 1};
   int rc;
   if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
   if ((rc = make_map4(&mw, w, dw, bw)) != NF_OK) return rc;
@@ -1375,10 +1418,10 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   FoldParams p{};
   if (bn) { p.bn_scale = bn->scale; p.bn_shift = bn->shift; p.bn_mu = bn->mu; p.bn_invstd = bn->invstd; }
   p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = epi == 2 ? 1 : Cin / 64; p.n_tiles = epi == 2 ? Cout / 64 : 1;
-  p.tiles_w = W / 14; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
+  p.tiles_w = W / TW; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
   if ((long long)N * p.tiles_w * p.tiles_h * p.n_tiles > (1ll << 30)) return NF_EUNSUPPORTED;
   p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
-  const size_t a_bytes = (size_t)10 * 16 * KC * 2;
+  const size_t a_bytes = (size_t)(uf ? 3 : 1) * 10 * 16 * KC * 2;
   const size_t wbytes = epi == 2 ? (size_t)9 * KC * 128 : (size_t)9 * p.kchunks * G * 128;
   const size_t fixed = wbytes + (epi != 1 ? (stats == 2 ? 6 : 2) * 16384 : 0) + 1024 + 1024;
   int st = (int)((232448 - fixed) / a_bytes);
@@ -1395,6 +1438,8 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
     *nb = grid / p.n_tiles * 8;
   }
   if (epi == 0) return launch_fold<64, 0>(grid, smem, mx, mw, my, my2, p);
+  if (epi == 2 && uf)
+    return KC == 16 ? launch_fold<64, 0, 16, 1, 1>(grid, smem, mx, mw, my, my2, p) : launch_fold<64, 0, 32, 1, 1>(grid, smem, mx, mw, my, my2, p);
   if (epi == 2)
     return KC == 16 ? launch_fold<64, 0, 16, 1>(grid, smem, mx, mw, my, my2, p) : launch_fold<64, 0, 32, 1>(grid, smem, mx, mw, my, my2, p);
   return G == 16 ? launch_fold<16, 1>(grid, smem, mx, mw, my, my2, p)
@@ -1407,7 +1452,7 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
             size_t red_floats, int32_t* status, int* nb, int epi = 0, const float* bias = nullptr, int stride = 1,
             const BnBwdIn* bn = nullptr) {
   const int H = (Hin - 1) / stride + 1, W = (Win - 1) / stride + 1;
-  if (fold_ok(H, W, Cin, Cout, epi, stride))
+  if (fold_ok(H, W, Cin, Cout, epi, stride, stats))
     return run_fold(N, H, W, Cin, Cout, x, w, y, stats, red, red_floats, status, nb, epi, bias, bn);
   if (stats == 2 && (!bn || epi == 1)) return NF_EINVAL;
   const TcPlan pl = plan_fwd(H, W, Cin, Cout, N, epi, stride, stats == 2);
@@ -1676,7 +1721,7 @@ int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb) {
   if (!L->o.maxpool && !L->skip) {
     const BnBwdIn bn{L->y, L->scale, L->shift, L->mu, L->invstd};
     bool fits;
-    if (fold_ok(L->Ha, L->Wa, L->F, L->Cout, epi, 1)) {
+    if (fold_ok(L->Ha, L->Wa, L->F, L->Cout, epi, 1, 2)) {
       fits = (size_t)(sm_count() / (L->Cout / 64)) * 8 * 2 * L->Cout <= L->red_floats;
     } else {
       const TcPlan pl = plan_fwd(L->Ha, L->Wa, L->F, L->Cout, L->o.N, epi, 1, 1);

@@ -143,6 +143,8 @@ TC = [
     dict(N=32, Cin=128, Cout=256, H=8, W=8, F=16, classes=10, stride=1, pool=False),     # per-tap weight gradient, 256-wide instructions
     dict(N=16, Cin=64, Cout=256, H=16, W=16, F=32, classes=10, stride=2, pool=False),    # the same with stride 2
     dict(N=6, Cin=128, Cout=256, H=16, W=32, F=16, classes=10, stride=1, pool=True),     # 256-wide forward on a map that tiles
+    dict(N=3, Cin=64, Cout=64, H=16, W=56, F=16, classes=10, stride=1, pool=False),   # width not a multiple of 16: input gradient with folded taps
+    dict(N=2, Cin=64, Cout=128, H=8, W=112, F=24, classes=10, stride=1, pool=False),  # unfolded input gradient: two channel tiles, 32-channel K, F < 32
 ]
 
 
