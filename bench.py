@@ -32,12 +32,14 @@ FALLBACK_PEAKS = dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=
 # DRAM bytes per image (read + write) of the kernels behind each traced op on the c4 layers 64->64 at 224x224,
 # from one ncu capture of the batch-24 case (profiles/ncu_full_c4s_conv_bn_kernels.md); every tensor is streamed
 # once, so traffic grows in proportion to the batch.  Valid for the kernels as captured; None elsewhere.
-NCU_TRAFFIC_C4_BYTES_PER_IMAGE = dict(conv_fwd=(154.28 + 106.19) * 1e6 / 24, wgrad=(324.20 + 3.72) * 1e6 / 24,
-                                      bn_fwd=(154.15 + 111.28) * 1e6 / 24, aux_fwd=(154.23 + 21.14) * 1e6 / 24,
-                                      bn_bwd=(308.29 + 124.88) * 1e6 / 24,   # the apply kernel; the finalize kernel moves < 1 MB
+NCU_TRAFFIC_C4_BYTES_PER_IMAGE = dict(conv_fwd=(154.28 + 105.87) * 1e6 / 24, wgrad=(324.34 + 3.83) * 1e6 / 24,
+                                      # aux forward with the fused BatchNorm + ReLU: reads y, writes a and h (the separate
+                                      # normalisation pass no longer runs on these layers; bn_fwd is the finalize kernel, < 1 MB)
+                                      aux_fwd=(154.22 + 139.06) * 1e6 / 24,
+                                      bn_bwd=(308.29 + 125.15) * 1e6 / 24,   # the apply kernel; the finalize kernel moves < 1 MB
                                       # dh_vec + aux weight gradient + aux input gradient (with the fused y read); the
                                       # two small partial-sum kernels move < 1 MB
-                                      aux_bwd=(38.57 + 1.50 + 201.43 + 3.81 + 192.84 + 114.94) * 1e6 / 24)
+                                      aux_bwd=(38.57 + 1.41 + 201.46 + 3.50 + 192.79 + 115.71) * 1e6 / 24)
 
 
 def load_peaks():
@@ -132,11 +134,14 @@ def op_model(l, N, classes, es, fam):
     ny, na, nh = N * Ho * Wo * l["Cout"], N * Ha * Wa * l["Cout"], N * Ha * Wa * l["F"]
     nparam = 9 * l["Cin"] * l["Cout"] + 2 * l["Cout"] + 9 * l["Cout"] * l["F"] + l["F"] + classes * (4 * l["F"] + 1)
     tc = lambda k: "tensor" if fam[k] == "tcgen05" else "alu"
+    fused = len(fam) > 4 and fam[4] == "fused"   # BatchNorm + ReLU applied inside the aux forward kernel
     return dict(conv_fwd=(tc(0), fl["conv_fwd"], es * (nx + ny)),          # read x, write y
                 wgrad=(tc(1), fl["wgrad"], es * (nx + ny)),                # read x and dy
-                aux_fwd=(tc(2), fl["aux_fwd"], es * (na + nh)),            # read a, write h
+                # read a, write h; fused: read y, write a and h
+                aux_fwd=(tc(2), fl["aux_fwd"], es * ((ny if fused else 0) + na + nh)),
                 aux_bwd=(tc(3), fl["aux_bwd"], es * (4 * nh + 2 * na)),    # h -> dh; a, dh -> gWa; dh -> da
-                bn_fwd=("hbm", None, es * (ny + na)),                      # read y, write a
+                # read y, write a; fused: only the statistics are finished here (partial sums in, coefficients out)
+                bn_fwd=("hbm", None, 4 * 2 * l["Cout"] * 1184 if fused else es * (ny + na)),
                 bn_bwd=("hbm", None, es * (2 * ny + na)),                  # read y and da, write dy
                 head=("hbm", None, es * nh + 4 * N * (8 * l["F"] + 2 * classes)),
                 sgd=("hbm", None, 18 * nparam))                            # theta, v read+write (fp32), g read, bf16 copy write
@@ -240,7 +245,7 @@ def run_ours(args, rank, world):
     ms, e2e_s = max_over_ranks([ms, e2e_s], world, "cuda")
 
     peaks, peak_src = load_peaks()
-    fam = [[L.kernel_family(k) for k in range(4)] for L in layers]
+    fam = [[L.kernel_family(k) for k in range(5)] for L in layers]
     kernels, best = [], None
     tot_ms = sum(v[0] for v in trace.values())
     for (op, slot), (tms, cnt) in sorted(trace.items(), key=lambda kv: -kv[1][0]):

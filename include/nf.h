@@ -316,7 +316,9 @@ int nf_trace_read(int op, int slot, double* ms_total, long long* groups);
 long long nf_launch_count(void);
 
 /* Name of the kernel family a configured layer uses for op 0 = main forward,
- * 1 = main weight gradient, 2 = aux forward, 3 = aux backward: "tcgen05" or "cuda-core". */
+ * 1 = main weight gradient, 2 = aux forward, 3 = aux backward: "tcgen05" or "cuda-core".
+ * op 4: "fused" when the BatchNorm + ReLU pass of the step runs inside the aux forward kernel
+ * (which then also writes act_out), "separate" otherwise. */
 const char* nf_layer_kernel_family(const nf_layer* layer, int op);
 
 const char* nf_strerror(int status);

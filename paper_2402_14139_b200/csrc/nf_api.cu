@@ -369,11 +369,15 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
     NF_TRY(nf_ref_bn_finalize_tot(L->dptot, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
                                   L->o.bn_momentum, L->scale, L->shift, L->mu, L->invstd, L->rmean, L->rvar));
   }
-  NF_TRY(nf_ref_bn_apply(dt, L->y, N, Ho, Wo, Co, pool, L->scale, L->shift, act_out, L->skip));
+  // where the shape allows, the aux forward kernel normalises y on the way in and writes act_out itself
+  const bool fused_bn_aux = nf_tc_bn_aux_fused(L) && !L->skip;
+  if (!fused_bn_aux) NF_TRY(nf_ref_bn_apply(dt, L->y, N, Ho, Wo, Co, pool, L->scale, L->shift, act_out, L->skip));
   trace_end();
   // Eq. 2: aux conv + ReLU, average pool to 2x2, linear; Eq. 3: softmax cross-entropy
   trace_begin(2);
-  if (L->fam[2]) {
+  if (fused_bn_aux) {
+    NF_TRY(nf_tc_bn_aux_fwd(L, act_out));
+  } else if (L->fam[2]) {
     NF_TRY(nf_tc_aux_fwd(L, act_out, N));
   } else {
     NF_TRY(nf_ref_conv(dt, act_out, N, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
@@ -842,7 +846,8 @@ int nf_set_stream(void* s) {
 long long nf_launch_count(void) { return g_nf_launches; }
 
 const char* nf_layer_kernel_family(const nf_layer* L, int op) {
-  if (!L || op < 0 || op > 3) return "";
+  if (!L || op < 0 || op > 4) return "";
+  if (op == 4) return nf_tc_bn_aux_fused(L) && !L->skip ? "fused" : "separate";
   return L->fam[op] ? "tcgen05" : "cuda-core";
 }
 

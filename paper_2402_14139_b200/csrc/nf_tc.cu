@@ -19,6 +19,10 @@ namespace {
 
 constexpr int kThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
 constexpr int kMaxStages = 8;
+// normalisation threads of the fused BatchNorm + aux forward: groups of 128 that share the ten rows of a box.  One group:
+// with two (five rows each) the kernel measured slower, 0.25 -> 0.27 ms, as every added warp that reads shared memory
+// stretches the tensor-core instructions.
+constexpr int kXfThreads = 128;
 constexpr int kFoldThreads = 320;  // folded-tap forward: producer, MMA issuer and two epilogue groups of four warps
 
 struct FwdParams {
@@ -425,6 +429,9 @@ struct FoldParams {
   const float *bn_scale, *bn_shift, *bn_mu, *bn_invstd;  // stats == 2
   const float* bias;  // EPI 1
   bf16* out;          // EPI 1: [N][H][W][Cout]
+  // XF: the input map is the conv output y; a = ReLU(y*scale + shift) is formed in shared memory and written to xf_a
+  const float *xf_scale, *xf_shift;
+  bf16* xf_a;         // [N][H][W][64 * kchunks]
 };
 
 // G   : width of one column-tap group of the accumulator (N = 3*G): 64 for the main conv, 16/32/64 for the
@@ -443,8 +450,13 @@ struct FoldParams {
 // only nine instructions (one per tap, N = 64) even unfolded, and the epilogue is what bounds the kernel: three
 // column-shifted activation boxes per stage replace the shift-add, the accumulator is 64 columns wide and all 16 x 8
 // pixels of a tile are outputs (W % 16 == 0).
-template <int G, int EPI, int KC = 64, int MIR = 0, int UF = 0>
-__global__ void __launch_bounds__(kFoldThreads, 1)
+// XF = 1 (aux forward only): BatchNorm + ReLU of the layer are applied on the way in.  The boxes are loaded from the
+// conv output y; four more warps turn each box into a = ReLU(y*scale + shift) in place (zero outside the image, as the
+// padding of a must be), write the tile's own 14 x 8 pixels of a to global memory (the layer's output activation) and
+// only then hand the stage to the issuer.  The separate normalisation pass (read y, write a) and this kernel's read of
+// a disappear; the halo pixels are normalised by both neighbours.
+template <int G, int EPI, int KC = 64, int MIR = 0, int UF = 0, int XF = 0>
+__global__ void __launch_bounds__(kFoldThreads + kXfThreads * XF, 1)
 conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                      const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_y2, const FoldParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -452,6 +464,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   constexpr int kARow = KC * 2;               // bytes of one pixel of the activation box
   constexpr uint32_t kALayout = KC == 64 ? 2 : KC == 32 ? 4 : 6;
   static_assert(!UF || (MIR && EPI == 0 && G == 64 && KC <= 32), "unfolded form: input gradient with few input channels");
+  static_assert(!XF || (EPI == 1 && KC == 64 && !MIR && !UF), "fused normalisation: aux forward only");
   constexpr int kBox = 10 * 16 * kARow;       // (8+2) rows x 16 pixels x KC channels
   constexpr int kABytes = (UF ? 3 : 1) * kBox;  // UF: one box per column tap
   constexpr int kTW = UF ? 16 : 14;           // output columns of a tile
@@ -468,7 +481,8 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   uint64_t* wfull = tempty + 2;
   uint64_t* yfull = wfull + 1;
   uint64_t* yempty = yfull + 4;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(yempty + 4);
+  uint64_t* xfull = yempty + 4;  // XF: stage normalised, ready for the issuer
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(xfull + kMaxStages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);  // [2], one per epilogue group
   constexpr uint32_t kAccStride = G == 64 ? 256 : 128;  // columns between the two accumulators
@@ -479,6 +493,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     for (int s = 0; s < p.stages; ++s) {
       ptx::mbar_init(&full[s], 1);
       ptx::mbar_init(&empty[s], 1);
+      ptx::mbar_init(&xfull[s], kXfThreads);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(&tfull[a], 1);
@@ -562,7 +577,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       for (int ck = 0; ck < p.kchunks; ++ck, ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
-        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[s], ph, abort_flag))) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(XF ? &xfull[s] : &full[s], ph, abort_flag))) { ok = false; break; }
         ptx::tc_fence_after();
         if (lane == 0) {
           const uint32_t a16 = ptx::smem_u32(smem + (size_t)s * kABytes) >> 4;
@@ -593,6 +608,68 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       }
       if (ok && lane == 0) ptx::mma_commit(&tfull[acc]);
       __syncwarp();
+    }
+  } else if (XF && warp >= kFoldThreads / 32) {
+    // normalisation warps: a thread owns one 16-byte channel chunk (8 channels) of one box column and walks the 10 rows
+    const int xt = (threadIdx.x - kFoldThreads) & 127, xg = (threadIdx.x - kFoldThreads) >> 7;  // group xg takes rows xg, xg+2, ...
+    constexpr int kXg = kXfThreads / 128, kRows = 10 / kXg;
+    const int j = xt & 7, col = xt >> 3;                   // logical chunk, box column (0..15)
+    const uint32_t off0 = (uint32_t)col * 128 + (uint32_t)((j ^ (col & 7)) * 16);  // 128-byte swizzle: the row's low bits are col's
+    const int C = p.kchunks * 64;
+    uint32_t it = 0;
+    float sc[8], sh[8];
+    int coef_ck = -1;  // channel chunk whose coefficients the registers hold
+    for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x) {
+      const int m = t / p.n_tiles;
+      const int w0 = (m % p.tiles_w) * 14, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
+      const int w = w0 - 1 + col;
+      const bool w_in = w >= 0 && w < p.W, w_own = col >= 1 && col <= 14;
+      bool ok = true;
+      for (int ck = 0; ck < p.kchunks; ++ck, ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (ck != coef_ck) {
+          coef_ck = ck;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            sc[i] = __ldg(p.xf_scale + ck * 64 + j * 8 + i);
+            sh[i] = __ldg(p.xf_shift + ck * 64 + j * 8 + i);
+          }
+        }
+        if (!ptx::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+        const uint32_t box = ptx::smem_u32(smem + (size_t)s * kABytes) + off0 + xg * 2048;
+        // all rows are loaded first, then normalised, then stored: the loads overlap instead of queueing behind stores
+        uint4 q[kRows];
+#pragma unroll
+        for (int i = 0; i < kRows; ++i) q[i] = ptx::lds128(box + i * kXg * 2048);
+#pragma unroll
+        for (int i = 0; i < kRows; ++i) {
+          const int h = h0 - 1 + i * kXg + xg;
+          const uint32_t qw[4] = {q[i].x, q[i].y, q[i].z, q[i].w};
+          uint32_t ow[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float a0 = fmaxf(fmaf(__uint_as_float(qw[e] << 16), sc[2 * e], sh[2 * e]), 0.f);
+            const float a1 = fmaxf(fmaf(__uint_as_float(qw[e] & 0xffff0000u), sc[2 * e + 1], sh[2 * e + 1]), 0.f);
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(a0, a1);
+            ow[e] = *reinterpret_cast<const uint32_t*>(&b2);
+          }
+          const bool in = w_in && h >= 0 && h < p.H;
+          q[i] = in ? make_uint4(ow[0], ow[1], ow[2], ow[3]) : make_uint4(0u, 0u, 0u, 0u);
+          ptx::sts128(box + i * kXg * 2048, q[i]);
+        }
+        ptx::fence_async_smem();  // the tensor core reads the stage through the async proxy
+        ptx::mbar_arrive(&xfull[s]);
+        if (w_own) {  // the tile's own pixels go to global memory after the stage has been handed on
+          bf16* dst = p.xf_a + (((size_t)n * p.H + h0 - 1 + xg) * p.W + w) * C + ck * 64 + j * 8;
+#pragma unroll
+          for (int i = 0; i < kRows; ++i) {
+            const int r = i * kXg + xg;  // box row; rows 1..8 are the tile's own
+            if (r >= 1 && r <= 8) *reinterpret_cast<uint4*>(dst + (size_t)(i * kXg) * p.W * C) = q[i];
+          }
+        }
+      }
+      if (!ok) break;
     }
   } else {
     // two epilogue groups of 128 threads; group g owns accumulator g and takes every second tile of the CTA
@@ -1367,15 +1444,15 @@ bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride, int stats = 0
   return wbytes + (epi == 0 ? 2 * 16384 : 0) + 2048 + 3 * 20480 <= 232448;
 }
 
-template <int G, int EPI, int KC = 64, int MIR = 0, int UF = 0>
+template <int G, int EPI, int KC = 64, int MIR = 0, int UF = 0, int XF = 0>
 int launch_fold(int grid, size_t smem, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const CUtensorMap& my2,
                 const FoldParams& p) {
   static bool attr_done = false;
   if (!attr_done) {
-    NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel<G, EPI, KC, MIR, UF>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel<G, EPI, KC, MIR, UF, XF>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
   }
-  conv_fwd_fold_kernel<G, EPI, KC, MIR, UF><<<grid, kFoldThreads, smem, g_nf_stream>>>(mx, mw, my, my2, p);
+  conv_fwd_fold_kernel<G, EPI, KC, MIR, UF, XF><<<grid, kFoldThreads + kXfThreads * XF, smem, g_nf_stream>>>(mx, mw, my, my2, p);
   NF_LAUNCHED();
   return NF_OK;
 }
@@ -1386,8 +1463,15 @@ struct BnBwdIn {
   const float *scale, *shift, *mu, *invstd;
 };
 
+// Normalisation fused into the aux forward (epi 1): x is then the conv output and a = ReLU(x*scale + shift) is written to a
+struct XfIn {
+  const float *scale, *shift;
+  void* a;
+};
+
 int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
-             size_t red_floats, int32_t* status, int* nb, int epi, const float* bias, const BnBwdIn* bn = nullptr) {
+             size_t red_floats, int32_t* status, int* nb, int epi, const float* bias, const BnBwdIn* bn = nullptr,
+             const XfIn* xf = nullptr) {
   const int G = fold_group(Cout, epi);
   const int KC = epi == 2 ? (Cin <= 16 ? 16 : 32) : 64;
   // input gradient on widths that also tile by 16: the unfolded form (three shifted boxes, no shift-add in the epilogue)
@@ -1436,6 +1520,13 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
     const size_t need = (size_t)(grid / p.n_tiles) * 8 * 2 * Cout;  // every CTA writes all of its 8 partials
     if (need > red_floats) return NF_ENOWS;
     *nb = grid / p.n_tiles * 8;
+  }
+  if (xf) {
+    if (epi != 1) return NF_EINVAL;
+    p.xf_scale = xf->scale; p.xf_shift = xf->shift; p.xf_a = (bf16*)xf->a;
+    return G == 16 ? launch_fold<16, 1, 64, 0, 0, 1>(grid, smem, mx, mw, my, my2, p)
+                   : G == 32 ? launch_fold<32, 1, 64, 0, 0, 1>(grid, smem, mx, mw, my, my2, p)
+                             : launch_fold<64, 1, 64, 0, 0, 1>(grid, smem, mx, mw, my, my2, p);
   }
   if (epi == 0) return launch_fold<64, 0>(grid, smem, mx, mw, my, my2, p);
   if (epi == 2 && uf)
@@ -1698,6 +1789,18 @@ int nf_tc_aux_fwd(nf_layer* L, const void* a, int count) {
   }
   return run_fwd(count, L->Ha, L->Wa, L->Cout, L->F, a, L->shadow + L->off[NF_P_WA], L->h, 0, nullptr, 0, L->status, &nb, 1,
                  L->val + L->off[NF_P_BA]);
+}
+
+bool nf_tc_bn_aux_fused(const nf_layer* L) {
+  return L->fam[2] && !wide_aux(L) && !L->o.maxpool && fold_ok(L->Ha, L->Wa, L->Cout, L->F, 1, 1);
+}
+
+int nf_tc_bn_aux_fwd(nf_layer* L, void* act_out) {
+  if (!nf_tc_bn_aux_fused(L) || L->skip) return NF_EUNSUPPORTED;
+  int nb = 0;
+  const XfIn xf{L->scale, L->shift, act_out};
+  return run_fold(L->o.N, L->Ha, L->Wa, L->Cout, L->F, L->y, L->shadow + L->off[NF_P_WA], L->h, 0, nullptr, 0, L->status, &nb, 1,
+                  L->val + L->off[NF_P_BA], nullptr, &xf);
 }
 
 int nf_tc_wgrad(nf_layer* L, const void* x) {

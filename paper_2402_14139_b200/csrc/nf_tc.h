@@ -24,6 +24,11 @@ int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int C
                         size_t part_floats, float* dw);
 // Aux conv forward on tensor cores for `count` samples: L->h = ReLU(conv(a, Wa) + ba) in bf16.
 int nf_tc_aux_fwd(nf_layer* L, const void* a, int count);
+// BatchNorm + ReLU and the aux conv forward in one kernel: act_out = ReLU(L->y * scale + shift) and
+// L->h = ReLU(conv(act_out, Wa) + ba), both in bf16.  NF_EUNSUPPORTED (nothing launched) when the layer's shape is not
+// covered or it has a shortcut; nf_tc_bn_aux_fused tells whether the shape is covered.
+bool nf_tc_bn_aux_fused(const nf_layer* L);
+int nf_tc_bn_aux_fwd(nf_layer* L, void* act_out);
 // Aux conv weight gradient on tensor cores: grad(Wa) = wgrad(a, L->dh).
 int nf_tc_aux_wgrad(nf_layer* L, const void* a);
 // Aux conv input gradient on tensor cores: L->da = dgrad(L->dh, Wa) in bf16.  Where the kernel can also reduce

@@ -162,6 +162,17 @@ def test_tensor_core_shapes_bf16(env, ci):
     print(w)
 
 
+def test_fused_normalisation_is_selected(env):
+    """Where the folded aux forward applies (width a multiple of 14, no pool) it also applies BatchNorm + ReLU and writes
+    act_out, so the parity cases of those shapes above check the fused kernel; other shapes keep the separate pass."""
+    nf, torch = env
+    for c, want in ((TC[8], "fused"), (TC[9], "fused"), (TC[0], "separate"), (TC[1], "separate")):
+        P, x, y = pu.seeded_case(c, 1, bf16=True)
+        G = pu.gpu_layer(nf, c, P, nf.NF_BF16)
+        assert G.kernel_family(4) == want, (c, G.kernel_family(4))
+        G.close()
+
+
 LARGE_HEAD = [
     (0, dict(N=600, Cin=8, Cout=16, H=4, W=4, F=32, classes=256, stride=1, pool=False)),      # fp32, 600*128*256 products
     (1, dict(N=512, Cin=64, Cout=64, H=4, W=4, F=64, classes=128, stride=1, pool=False)),     # bf16 tensor-core layer
