@@ -145,6 +145,7 @@ TC = [
     dict(N=6, Cin=128, Cout=256, H=16, W=32, F=16, classes=10, stride=1, pool=True),     # 256-wide forward on a map that tiles
     dict(N=3, Cin=64, Cout=64, H=16, W=56, F=16, classes=10, stride=1, pool=False),   # width not a multiple of 16: input gradient with folded taps
     dict(N=2, Cin=64, Cout=128, H=8, W=112, F=24, classes=10, stride=1, pool=False),  # unfolded input gradient: two channel tiles, 32-channel K, F < 32
+    dict(N=5, Cin=64, Cout=64, H=16, W=16, F=16, classes=700, stride=1, pool=False),  # few samples, many classes in the per-sample head kernel
 ]
 
 
