@@ -316,6 +316,8 @@ class Layer:
         return rc
 
     def kernel_family(self, op: int) -> str:
+        """op 0-3: "tcgen05" or "cuda-core" for main forward, main weight gradient, aux forward, aux backward;
+        op 4: "fused" when BatchNorm + ReLU run inside the aux forward kernel, else "separate"."""
         return lib().nf_layer_kernel_family(self.h, op).decode()
 
 
