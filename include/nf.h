@@ -51,7 +51,8 @@ enum nf_status {
 enum nf_device_flag {
   NF_ELABEL = 1,     /* a label was outside [0, classes); it was clamped */
   NF_ENONFINITE = 2, /* the loss was NaN or infinite */
-  NF_ETIMEOUT = 4    /* a bounded wait inside a kernel ran out; results of that step are invalid */
+  NF_ETIMEOUT = 4,   /* a bounded wait inside a kernel ran out; results of that step are invalid */
+  NF_EINDEX = 8      /* nf_cache_gather: an index was outside [0, cache_rows); that output row was zero-filled */
 };
 
 enum nf_dtype { NF_F32 = 0, NF_BF16 = 1 };
@@ -85,8 +86,8 @@ typedef struct nf_layer_opts {
   float bn_eps;      /* BatchNorm epsilon */
   float bn_momentum; /* running-statistics momentum */
   int host_io;       /* 1: reserve staging so the *_step_host calls can be used; 2: a second input buffer too (nf_block_step_host_next) */
-  int loss;          /* nf_loss: the loss of Eq. 3 ("e.g., Mean Squared Error or Cross Entropy Error"); 0 = cross entropy */
-  int aux_pool;      /* nf_aux_pool: the down-sampling F_n of Eq. 2 ("such as max pooling or average pooling"); 0 = average */
+  int loss;          /* nf_loss: the loss L of Eq. 3 (the text beside it names squared error and cross entropy); 0 = cross entropy */
+  int aux_pool;      /* nf_aux_pool: the down-sampling F_n of Eq. 2 (the text beside it names max and average pooling); 0 = average */
 } nf_layer_opts;
 
 enum nf_loss { NF_LOSS_CE = 0, NF_LOSS_MSE = 1 };        /* MSE: mean over batch and classes of (z - onehot)^2 */
@@ -186,6 +187,19 @@ int nf_layer_step_dp(nf_layer* layer, int phase, const void* x, const int32_t* l
 /* Device address and size of exchange buffer `which` (0, 1, 2 as above) inside the bound workspace. */
 int nf_layer_dp_buffer(nf_layer* layer, int which, void** dev_ptr, size_t* bytes);
 
+/* The tensors a step leaves in the workspace, for inspection and element-wise checks: device address and size in bytes of
+ *   NF_T_Y conv output y [N][Ho][Wo][Cout], NF_T_DY gradient at y, NF_T_H aux conv output after ReLU [N][Ha][Wa][Fp],
+ *   NF_T_DH gradient at h, NF_T_DA gradient at the activation [N][Ha][Wa][Cout]  (all of the layer's dtype; Fp = F rounded
+ *   up to a multiple of 8, the extra channels are zero),
+ *   NF_T_P pooled aux output [N][4*Fp], NF_T_DP its gradient, NF_T_LOGITS [N][classes]  (float),
+ *   NF_T_HMASK the signs of h, one bit per element: bytes [N][Ha][Wa][Fp/8], bit f%8 of byte f/8 set where h > 0.  A layer
+ *   whose nf_layer_kernel_family(layer, 5) is "mask" keeps this instead of h (its aux forward pools h in its epilogue and
+ *   never stores it; the mask shares h's memory); otherwise h is stored and the mask is not.
+ * Valid after a step on that layer and until the next call on it; a kernel that does not need one of them on some
+ * shape may leave it unwritten.  NF_EINVAL for an unknown id, NF_ENOWS without workspace. */
+enum nf_stored { NF_T_Y = 0, NF_T_DY = 1, NF_T_H = 2, NF_T_DH = 3, NF_T_DA = 4, NF_T_P = 5, NF_T_DP = 6, NF_T_LOGITS = 7, NF_T_HMASK = 8 };
+int nf_layer_stored_tensor(nf_layer* layer, int which, void** dev_ptr, size_t* bytes);
+
 /* Early-exit evaluation (Section "Trained output CNN": every layer with its auxiliary network is a
  * prospective exit point).  Forward only, BatchNorm with running statistics, no parameter changes:
  *   act_out = x_{n+1} for `count` samples (device, [count][Ha][Wa][Cout]; NULL keeps it in the workspace),
@@ -230,8 +244,10 @@ int nf_block_step_host_next(nf_block* block, const void* x_host, const int32_t* 
 
 /* Re-batching from the cache: out[i] = cache[idx[i]] for i < count, rows of row_bytes bytes
  * (a multiple of 16); labels likewise if both label pointers are non-NULL.  All device pointers.
- * Bit-exact copy. */
-int nf_cache_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count,
+ * Bit-exact copy.  cache_rows is the number of rows the cache holds: an index outside [0, cache_rows)
+ * (a stale or corrupt permutation) reads nothing -- its output row is zero-filled, its label set to -1
+ * and NF_EINDEX is raised in the status word nf_op_status() returns. */
+int nf_cache_gather(const void* cache, const int32_t* cache_labels, int cache_rows, const int32_t* idx, int count,
                     size_t row_bytes, void* out, int32_t* out_labels);
 
 /* Stand-alone forms of the two dense contractions of the step (Eq. 1's theta_n x_n and the
@@ -289,12 +305,16 @@ int nf_partition(const int* max_batch, int n_layers, int B, double rho, int* blo
  * batch) at each of the k given batch sizes, and the least-squares line bytes = intercept + slope * batch
  * through them (k >= 2 distinct sizes; bytes_out may be NULL).  opts->N is ignored.
  *
+ * nf_fit_line: the same least-squares line through k >= 2 MEASURED (batch size, bytes) pairs, for a caller that profiles by
+ * running steps and reading the device's memory counters, as the paper's Profiler does.
+ *
  * nf_max_batch: the largest batch t with intercept + slope * t <= budget (first loop of Algorithm 1);
  * 0 if even one sample does not fit.  Feed the results to nf_partition.
  * All return NF_EINVAL on bad arguments. */
 int nf_aan_filters(const int* channels, int n_layers, int first_downsample, int* filters_out);
 int nf_profile_layer(int Cin, int Cout, int H, int W, int F, int classes, const nf_layer_opts* opts, const int* batches, int k,
                      double* bytes_out, double* slope, double* intercept);
+int nf_fit_line(const double* batches, const double* bytes, int k, double* slope, double* intercept);
 long long nf_max_batch(double slope, double intercept, double budget_bytes);
 
 /* Stream for all later calls (a cudaStream_t); NULL selects the default stream. */
@@ -312,13 +332,23 @@ enum { NF_TRACE_OPS = 8, NF_TRACE_SLOTS = 32 };
 int nf_trace_enable(int on);
 int nf_trace_read(int op, int slot, double* ms_total, long long* groups);
 
+/* Self-check of the hang safety of the tensor-core kernels.  Every wait inside them (on an mbarrier that a TMA copy or
+ * a tcgen05.commit completes) is bounded in time; when one runs out the waiter sets an abort flag, every role of the CTA
+ * leaves its loop, and NF_ETIMEOUT is raised instead of the kernel spinning forever.  This call exercises exactly that
+ * wait routine in isolation: one CTA of one warp, no TMA, no tensor memory, waits limit_ns (1 .. 1e9) on a barrier that
+ * nobody arrives at, gives up, raises NF_ETIMEOUT in the status word nf_op_status() returns and writes the nanoseconds
+ * it waited to *waited_ns_dev (device, 8-byte aligned).  Asynchronous on the library's stream. */
+int nf_selftest_bounded_wait(unsigned long long limit_ns, unsigned long long* waited_ns_dev);
+
 /* Kernel launches enqueued by this library since the process started. */
 long long nf_launch_count(void);
 
 /* Name of the kernel family a configured layer uses for op 0 = main forward,
  * 1 = main weight gradient, 2 = aux forward, 3 = aux backward: "tcgen05" or "cuda-core".
  * op 4: "fused" when the BatchNorm + ReLU pass of the step runs inside the aux forward kernel
- * (which then also writes act_out), "separate" otherwise. */
+ * (which then also writes act_out), "separate" otherwise.
+ * op 5: "mask" when that kernel also pools the aux output h in its epilogue and keeps only one sign bit per element of it
+ * (Eq. 2's F_n applied before h ever reaches memory), "stored" when h is written and pooled by separate kernels. */
 const char* nf_layer_kernel_family(const nf_layer* layer, int op);
 
 const char* nf_strerror(int status);

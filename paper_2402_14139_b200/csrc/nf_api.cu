@@ -5,6 +5,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <vector>
 
 #include "nf_internal.h"
@@ -30,6 +31,7 @@ bool g_trace_on = false;
 double g_trace_ms[NF_TRACE_OPS][NF_TRACE_SLOTS];
 long long g_trace_cnt[NF_TRACE_OPS][NF_TRACE_SLOTS];
 int g_trace_slot = 0;
+bool g_defer_update = false;  // nf_block_step: the layers' updates are launched together after the last layer
 
 void trace_begin(int op) {
   if (!g_trace_on) return;
@@ -109,20 +111,24 @@ size_t plan(nf_layer* L, char* base, bool assign) {
   D->logits = (float*)c.take(N * K * 4);
   D->dlogits = (float*)c.take(N * K * 4);
   D->lossn = (float*)c.take(N * 4);
-  size_t r1 = (size_t)nf_ref_channel_blocks(N * L->Ho * L->Wo, (int)Co) * 2 * Co;
-  size_t r2 = (size_t)nf_ref_channel_blocks(N * L->Ha * L->Wa, (int)F) * 2 * F;
+  size_t r1 = (size_t)nf_k_channel_blocks(N * L->Ho * L->Wo, (int)Co) * 2 * Co;
+  size_t r2 = (size_t)nf_k_channel_blocks(N * L->Ha * L->Wa, (int)F) * 2 * F;
   D->red_floats = r1 > r2 ? r1 : r2;
   const size_t r3 = nf_tc_red_floats(L);
   if (r3 > D->red_floats) D->red_floats = r3;
   D->red = (float*)c.take(D->red_floats * 4);
-  size_t w1 = (size_t)nf_ref_wgrad_splits((int)N, L->Ho, L->Cin, (int)Co) * 9 * Co * L->Cin;
-  size_t w2 = (size_t)nf_ref_wgrad_splits((int)N, L->Ha, (int)Co, (int)F) * 9 * F * Co;
+  size_t w1 = (size_t)nf_k_wgrad_splits((int)N, L->Ho, L->Cin, (int)Co) * 9 * Co * L->Cin;
+  size_t w2 = (size_t)nf_k_wgrad_splits((int)N, L->Ha, (int)Co, (int)F) * 9 * F * Co;
   D->wpart_floats = w1 > w2 ? w1 : w2;
   const size_t tc = nf_tc_scratch_floats(L);
   if (tc > D->wpart_floats) D->wpart_floats = tc;
+  if (nf_tc_aux_pool_fused(L) && nf_tc_pool_part_floats(L) > D->wpart_floats) D->wpart_floats = nf_tc_pool_part_floats(L);
   if (nf_head_is_large((int)N, (int)(4 * F), (int)K)) {  // tiled head: logits before the bias, up to 16 batch ranges of gWf
     size_t hs = nf_head_scratch_floats((int)N, (int)(4 * F), (int)K);
     if (hs < (size_t)16 * K * 4 * F) hs = (size_t)16 * K * 4 * F;
+    if (hs > D->wpart_floats) D->wpart_floats = hs;
+  } else {
+    const size_t hs = nf_head_small_scratch_floats((int)N, (int)(4 * F), (int)K);  // class-sliced head: shares of the softmax and of dp
     if (hs > D->wpart_floats) D->wpart_floats = hs;
   }
   D->wpart = (float*)c.take(D->wpart_floats * 4);
@@ -266,7 +272,7 @@ int nf_layer_bind_workspace(nf_layer* L, void* dev, size_t bytes) {
   NF_CUDA(cudaMemcpyAsync(L->val + L->off[NF_P_GAMMA], ones.data(), L->Cout * 4, cudaMemcpyHostToDevice, g_nf_stream));
   NF_CUDA(cudaMemcpyAsync(L->rvar, ones.data(), L->Cout * 4, cudaMemcpyHostToDevice, g_nf_stream));
   NF_CUDA(cudaStreamSynchronize(g_nf_stream));
-  return nf_ref_shadow(L->val, L->shadow, L->arena);
+  return nf_k_shadow(L->val, L->shadow, L->arena);
 }
 
 static int param_ptr(nf_layer* L, int which, float** dev, size_t* n, int* conv_a, int* conv_b) {
@@ -302,7 +308,7 @@ int nf_layer_set_param(nf_layer* L, int which, const float* host, size_t n) {
   NF_CUDA(cudaMemcpyAsync(dev, tmp.data(), cnt * 4, cudaMemcpyHostToDevice, g_nf_stream));
   NF_CUDA(cudaStreamSynchronize(g_nf_stream));
   if ((which & 0xf00) == NF_K_VALUE && id < NF_NPARAM) {
-    rc = nf_ref_shadow(L->val, L->shadow, L->arena);
+    rc = nf_k_shadow(L->val, L->shadow, L->arena);
     if (rc != NF_OK) return rc;
     NF_CUDA(cudaStreamSynchronize(g_nf_stream));
   }
@@ -354,24 +360,24 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
   if (L->fam[0]) {
     NF_TRY(nf_tc_conv_fwd(L, x, nb));
   } else {
-    NF_TRY(nf_ref_conv(dt, x, N, L->H, L->W, Ci, Wm, (long)Co * Ci, Ci, 1, 0, nullptr, 0, s, Co, L->y));
-    NF_TRY(nf_ref_channel_sums(dt, L->y, (size_t)N * Ho * Wo, Co, L->red, L->red_floats, &nb));
+    NF_TRY(nf_k_conv(dt, x, N, L->H, L->W, Ci, Wm, (long)Co * Ci, Ci, 1, 0, nullptr, 0, s, Co, L->y));
+    NF_TRY(nf_k_channel_sums(dt, L->y, (size_t)N * Ho * Wo, Co, L->red, L->red_floats, &nb));
   }
   trace_end();
-  if (!all) return nf_ref_partial_totals(L->red, nb, Co, L->dptot);
+  if (!all) return nf_k_partial_totals(L->red, nb, Co, L->dptot);
   }
   if (all || phase == 1) {
   trace_begin(1);
   if (all) {
-    NF_TRY(nf_ref_bn_finalize(L->red, nb, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
+    NF_TRY(nf_k_bn_finalize(L->red, nb, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
                               L->o.bn_momentum, L->scale, L->shift, L->mu, L->invstd, L->rmean, L->rvar));
   } else {
-    NF_TRY(nf_ref_bn_finalize_tot(L->dptot, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
+    NF_TRY(nf_k_bn_finalize_tot(L->dptot, Co, M, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps,
                                   L->o.bn_momentum, L->scale, L->shift, L->mu, L->invstd, L->rmean, L->rvar));
   }
   // where the shape allows, the aux forward kernel normalises y on the way in and writes act_out itself
   const bool fused_bn_aux = nf_tc_bn_aux_fused(L) && !L->skip;
-  if (!fused_bn_aux) NF_TRY(nf_ref_bn_apply(dt, L->y, N, Ho, Wo, Co, pool, L->scale, L->shift, act_out, L->skip));
+  if (!fused_bn_aux) NF_TRY(nf_k_bn_apply(dt, L->y, N, Ho, Wo, Co, pool, L->scale, L->shift, act_out, L->skip));
   trace_end();
   // Eq. 2: aux conv + ReLU, average pool to 2x2, linear; Eq. 3: softmax cross-entropy
   trace_begin(2);
@@ -380,15 +386,19 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
   } else if (L->fam[2]) {
     NF_TRY(nf_tc_aux_fwd(L, act_out, N));
   } else {
-    NF_TRY(nf_ref_conv(dt, act_out, N, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
+    NF_TRY(nf_k_conv(dt, act_out, N, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
   }
   trace_end();
   trace_begin(3);
-  if (L->o.aux_pool == NF_POOL_MAX) {
-    NF_TRY(nf_ref_auxmax(dt, L->h, N, Ha, Wa, F, L->p, L->parg));
+  // h_masked: the aux forward left pooling partials (L->wpart) and a sign mask (in L->h) instead of h
+  const bool h_masked = fused_bn_aux && nf_tc_aux_pool_fused(L);
+  if (h_masked) {
+    NF_TRY(nf_k_pool_finish(L->wpart, N, Ha / 8, Wa / 14, F, 1.f / (float)((Ha / 2) * (Wa / 2)), L->p));
+  } else if (L->o.aux_pool == NF_POOL_MAX) {
+    NF_TRY(nf_k_auxmax(dt, L->h, N, Ha, Wa, F, L->p, L->parg));
   } else {
-    int rc = dt == NF_BF16 ? nf_ref_avgpool_fast(L->h, N, Ha, Wa, F, L->wpart, L->wpart_floats, L->p) : NF_EUNSUPPORTED;
-    if (rc == NF_EUNSUPPORTED) rc = nf_ref_avgpool(dt, L->h, N, Ha, Wa, F, L->p);
+    int rc = dt == NF_BF16 ? nf_k_avgpool_fast(L->h, N, Ha, Wa, F, L->wpart, L->wpart_floats, L->p) : NF_EUNSUPPORTED;
+    if (rc == NF_EUNSUPPORTED) rc = nf_k_avgpool(dt, L->h, N, Ha, Wa, F, L->p);
     if (rc != NF_OK) return rc;
   }
   if (nf_head_is_large(N, D, K)) {  // late blocks: tens of thousands of samples, up to 1024 head inputs
@@ -396,40 +406,48 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
                         L->lossn, L->status, L->o.loss, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->wpart,
                         L->wpart_floats, n_scale));
   } else {
-    NF_TRY(nf_ref_fc_ce(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits,
+    // forward, loss and the gradients of gamma_n cut by class slices; heads wider than that covers: one block per sample
+    int rc = nf_head_small_step(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dp, L->lossn,
+                                L->status, L->o.loss, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->wpart, L->wpart_floats,
+                                n_scale);
+    if (rc == NF_EUNSUPPORTED) {
+      NF_TRY(nf_k_fc_ce(L->p, labels, N, D, K, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], L->logits, L->dlogits,
                         L->dp, L->lossn, L->status, L->o.loss, n_scale));
-    // gradients of gamma_n
-    NF_TRY(nf_ref_fc_wgrad(L->p, L->dlogits, L->lossn, N, D, K, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->status, n_scale));
+      rc = nf_k_fc_wgrad(L->p, L->dlogits, L->lossn, N, D, K, g + L->off[NF_P_WF], g + L->off[NF_P_BF], loss_out, L->status, n_scale);
+    }
+    if (rc != NF_OK) return rc;
   }
   trace_end();
   trace_begin(4);
   int dh_nb = 0;
-  if (L->o.aux_pool == NF_POOL_MAX) {
-    NF_TRY(nf_ref_dh_max(dt, L->h, L->dp, L->parg, N, Ha, Wa, F, L->dh));
+  if (h_masked) {
+    NF_TRY(nf_k_dh_mask((const uint8_t*)L->h, L->dp, N, Ha, Wa, F, L->dh, L->red, L->red_floats, &dh_nb));
+  } else if (L->o.aux_pool == NF_POOL_MAX) {
+    NF_TRY(nf_k_dh_max(dt, L->h, L->dp, L->parg, N, Ha, Wa, F, L->dh));
   } else {
-    int rc = dt == NF_BF16 ? nf_ref_dh_fast(L->h, L->dp, N, Ha, Wa, F, L->dh, L->red, L->red_floats, &dh_nb) : NF_EUNSUPPORTED;
+    int rc = dt == NF_BF16 ? nf_k_dh_fast(L->h, L->dp, N, Ha, Wa, F, L->dh, L->red, L->red_floats, &dh_nb) : NF_EUNSUPPORTED;
     if (rc == NF_EUNSUPPORTED) {
       dh_nb = 0;
-      rc = nf_ref_dh(dt, L->h, L->dp, N, Ha, Wa, F, L->dh);
+      rc = nf_k_dh(dt, L->h, L->dp, N, Ha, Wa, F, L->dh);
     }
     if (rc != NF_OK) return rc;
   }
-  if (dh_nb) NF_TRY(nf_ref_sum_partials(L->red, dh_nb, F, 0, g + L->off[NF_P_BA]));
+  if (dh_nb) NF_TRY(nf_k_sum_partials(L->red, dh_nb, F, 0, g + L->off[NF_P_BA]));
   if (L->fam[3]) {
     NF_TRY(nf_tc_aux_wgrad(L, act_out));
   } else {
-    NF_TRY(nf_ref_wgrad(dt, act_out, N, Ha, Wa, Co, L->dh, F, 1, L->wpart, L->wpart_floats, g + L->off[NF_P_WA]));
+    NF_TRY(nf_k_wgrad(dt, act_out, N, Ha, Wa, Co, L->dh, F, 1, L->wpart, L->wpart_floats, g + L->off[NF_P_WA]));
   }
   if (!dh_nb) {
-    NF_TRY(nf_ref_channel_sums(dt, L->dh, (size_t)N * Ha * Wa, F, L->red, L->red_floats, &nb));
-    NF_TRY(nf_ref_sum_partials(L->red, nb, F, 0, g + L->off[NF_P_BA]));
+    NF_TRY(nf_k_channel_sums(dt, L->dh, (size_t)N * Ha * Wa, F, L->red, L->red_floats, &nb));
+    NF_TRY(nf_k_sum_partials(L->red, nb, F, 0, g + L->off[NF_P_BA]));
   }
   // gradient at the aux input
   int bn_nb = 0;  // > 0: the input-gradient kernel has already left the BatchNorm-backward partial sums in L->red
   if (L->fam[3]) {
     NF_TRY(nf_tc_aux_dgrad(L, &bn_nb));
   } else {
-    NF_TRY(nf_ref_conv(dt, L->dh, N, Ha, Wa, F, Wx, (long)F * Co, 1, Co, 1, nullptr, 0, 1, Co, L->da));
+    NF_TRY(nf_k_conv(dt, L->dh, N, Ha, Wa, F, Wx, (long)F * Co, 1, Co, 1, nullptr, 0, 1, Co, L->da));
   }
   trace_end();
   // back through pool / ReLU / BatchNorm
@@ -437,18 +455,18 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
   if (bn_nb) {
     nb = bn_nb;
   } else {
-    NF_TRY(nf_ref_bn_bwd_reduce(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->red,
+    NF_TRY(nf_k_bn_bwd_reduce(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->red,
                                 L->red_floats, &nb, L->skip));
   }
-  if (!all) return nf_ref_partial_totals(L->red, nb, Co, L->dptot + 2 * Co);
+  if (!all) return nf_k_partial_totals(L->red, nb, Co, L->dptot + 2 * Co);
   }
   if (all || phase == 2) {
   if (all) {
-    NF_TRY(nf_ref_bn_bwd_finalize(L->red, nb, Co, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
+    NF_TRY(nf_k_bn_bwd_finalize(L->red, nb, Co, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
   } else {
-    NF_TRY(nf_ref_bn_bwd_finalize_tot(L->dptot + 2 * Co, Co, world, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
+    NF_TRY(nf_k_bn_bwd_finalize_tot(L->dptot + 2 * Co, Co, world, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
   }
-  NF_TRY(nf_ref_bn_bwd_apply(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->sdz, L->sdzx,
+  NF_TRY(nf_k_bn_bwd_apply(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->sdz, L->sdzx,
                              M, L->dy, L->skip));
   trace_end();
   // gradient of theta_n (the layer input receives none), then the update
@@ -456,13 +474,14 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
   if (L->fam[1]) {
     NF_TRY(nf_tc_wgrad(L, x));
   } else {
-    NF_TRY(nf_ref_wgrad(dt, x, N, L->H, L->W, Ci, L->dy, Co, s, L->wpart, L->wpart_floats, g + L->off[NF_P_W]));
+    NF_TRY(nf_k_wgrad(dt, x, N, L->H, L->W, Ci, L->dy, Co, s, L->wpart, L->wpart_floats, g + L->off[NF_P_W]));
   }
   trace_end();
   if (!all) return NF_OK;
   }
+  if (g_defer_update) return NF_OK;
   trace_begin(7);
-  NF_TRY(nf_ref_sgd(L->val, L->mom, L->grad, L->shadow, L->arena, lr, L->o.momentum));
+  NF_TRY(nf_k_sgd(L->val, L->mom, L->grad, L->shadow, L->arena, lr, L->o.momentum));
   trace_end();
   return NF_OK;
 }
@@ -493,6 +512,26 @@ int nf_layer_dp_buffer(nf_layer* L, int which, void** dev_ptr, size_t* bytes) {
   } else {
     *dev_ptr = L->dptot + (size_t)which * 2 * L->Cout;
     *bytes = (size_t)2 * L->Cout * sizeof(double);
+  }
+  return NF_OK;
+}
+
+int nf_layer_stored_tensor(nf_layer* L, int which, void** dev_ptr, size_t* bytes) {
+  if (!L || !dev_ptr || !bytes) return NF_EINVAL;
+  if (!L->ws) return NF_ENOWS;
+  const size_t es = nf_esize(L->o.dtype), N = L->o.N;
+  const size_t ny = N * L->Ho * L->Wo * L->Cout, na = N * L->Ha * L->Wa * L->Cout, nh = N * L->Ha * L->Wa * L->F;
+  switch (which) {
+    case NF_T_Y: *dev_ptr = L->y; *bytes = ny * es; break;
+    case NF_T_DY: *dev_ptr = L->dy; *bytes = ny * es; break;
+    case NF_T_H: *dev_ptr = L->h; *bytes = nh * es; break;
+    case NF_T_DH: *dev_ptr = L->dh; *bytes = nh * es; break;
+    case NF_T_DA: *dev_ptr = L->da; *bytes = na * es; break;
+    case NF_T_P: *dev_ptr = L->p; *bytes = N * 4 * L->F * sizeof(float); break;
+    case NF_T_DP: *dev_ptr = L->dp; *bytes = N * 4 * L->F * sizeof(float); break;
+    case NF_T_LOGITS: *dev_ptr = L->logits; *bytes = N * L->classes * sizeof(float); break;
+    case NF_T_HMASK: *dev_ptr = L->h; *bytes = nh / 8; break;
+    default: return NF_EINVAL;
   }
   return NF_OK;
 }
@@ -569,12 +608,12 @@ static int layer_eval_forward(nf_layer* L, const void* in, int count, void* dst)
   if (L->fam[0]) {
     NF_TRY(nf_tc_conv_fwd_eval(L, in, count));
   } else {
-    NF_TRY(nf_ref_conv(dt, in, count, L->H, L->W, L->Cin, Wm, (long)L->Cout * L->Cin, L->Cin, 1, 0, nullptr, 0, L->o.stride,
+    NF_TRY(nf_k_conv(dt, in, count, L->H, L->W, L->Cin, Wm, (long)L->Cout * L->Cin, L->Cin, 1, 0, nullptr, 0, L->o.stride,
                        L->Cout, L->y));
   }
-  NF_TRY(nf_ref_bn_eval_coeffs(L->Cout, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps, L->rmean, L->rvar,
+  NF_TRY(nf_k_bn_eval_coeffs(L->Cout, L->val + L->off[NF_P_GAMMA], L->val + L->off[NF_P_BETA], L->o.bn_eps, L->rmean, L->rvar,
                                L->scale, L->shift));
-  return nf_ref_bn_apply(dt, L->y, count, L->Ho, L->Wo, L->Cout, L->o.maxpool, L->scale, L->shift, dst, L->skip);
+  return nf_k_bn_apply(dt, L->y, count, L->Ho, L->Wo, L->Cout, L->o.maxpool, L->scale, L->shift, dst, L->skip);
 }
 
 int nf_layer_predict(nf_layer* L, const void* x, int count, void* act_out, float* logits_out, int32_t* pred_out) {
@@ -589,13 +628,13 @@ int nf_layer_predict(nf_layer* L, const void* x, int count, void* act_out, float
   if (L->fam[2]) {
     NF_TRY(nf_tc_aux_fwd(L, a, count));
   } else {
-    NF_TRY(nf_ref_conv(dt, a, count, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
+    NF_TRY(nf_k_conv(dt, a, count, Ha, Wa, Co, Wx, (long)F * Co, Co, 1, 0, L->val + L->off[NF_P_BA], 1, 1, F, L->h));
   }
   if (L->o.aux_pool == NF_POOL_MAX) {
-    NF_TRY(nf_ref_auxmax(dt, L->h, count, Ha, Wa, F, L->p, L->parg));
+    NF_TRY(nf_k_auxmax(dt, L->h, count, Ha, Wa, F, L->p, L->parg));
   } else {
-    int rc = dt == NF_BF16 ? nf_ref_avgpool_fast(L->h, count, Ha, Wa, F, L->wpart, L->wpart_floats, L->p) : NF_EUNSUPPORTED;
-    if (rc == NF_EUNSUPPORTED) rc = nf_ref_avgpool(dt, L->h, count, Ha, Wa, F, L->p);
+    int rc = dt == NF_BF16 ? nf_k_avgpool_fast(L->h, count, Ha, Wa, F, L->wpart, L->wpart_floats, L->p) : NF_EUNSUPPORTED;
+    if (rc == NF_EUNSUPPORTED) rc = nf_k_avgpool(dt, L->h, count, Ha, Wa, F, L->p);
     if (rc != NF_OK) return rc;
   }
   // the caller's logits have `classes` columns over the logical 4*Flog inputs; the padded inputs are zero
@@ -604,12 +643,12 @@ int nf_layer_predict(nf_layer* L, const void* x, int count, void* act_out, float
     NF_TRY(nf_head_logits(L->p, count, 4 * F, L->classes, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], lg, L->wpart));
     return nf_head_predict(lg, count, L->classes, pred_out);
   }
-  return nf_ref_fc_predict(L->p, count, 4 * F, L->classes, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], logits_out, pred_out);
+  return nf_k_fc_predict(L->p, count, 4 * F, L->classes, L->val + L->off[NF_P_WF], L->val + L->off[NF_P_BF], logits_out, pred_out);
 }
 
 int nf_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count) {
   if (!a || !b || !count || n < 1) return NF_EINVAL;
-  return nf_ref_count_equal(a, b, n, count);
+  return nf_k_count_equal(a, b, n, count);
 }
 
 long long nf_layer_param_count(const nf_layer* L, int part) {
@@ -639,11 +678,28 @@ int nf_block_step(nf_block* B, const void* x, const int32_t* labels, float lr, f
     nf_layer* L = B->layers[l];
     void* dst = (l == B->n - 1 && act_out) ? act_out : L->act;
     g_trace_slot = l < NF_TRACE_SLOTS ? l : NF_TRACE_SLOTS - 1;
+    g_defer_update = true;  // no layer reads another layer's parameters, so the updates can wait for the end of the pass
     const int rc = nf_layer_step(L, in, labels, lr, loss_out + l, dst);
+    g_defer_update = false;
     g_trace_slot = 0;
     if (rc != NF_OK) return rc;
     in = dst;
   }
+  // Algorithm 2's update of every layer of the block, one launch per group of layers with equal momentum
+  trace_begin(7);
+  for (int l0 = 0; l0 < B->n;) {
+    SgdTable tb{};
+    const float mu = B->layers[l0]->o.momentum;
+    int l = l0;
+    for (; l < B->n && tb.count < kSgdMaxArenas && B->layers[l]->o.momentum == mu; ++l) {
+      nf_layer* L = B->layers[l];
+      tb.val[tb.count] = L->val; tb.mom[tb.count] = L->mom; tb.grad[tb.count] = L->grad; tb.shadow[tb.count] = L->shadow;
+      tb.n[tb.count++] = L->arena;
+    }
+    NF_TRY(nf_k_sgd_multi(tb, lr, mu));
+    l0 = l;
+  }
+  trace_end();
   return NF_OK;
 }
 
@@ -719,12 +775,14 @@ int nf_block_step_host_next(nf_block* B, const void* xh, const int32_t* lh, floa
   return NF_OK;
 }
 
-int nf_cache_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count, size_t row_bytes,
-                    void* out, int32_t* out_labels) {
-  if (!cache || !idx || !out || count < 1 || row_bytes == 0 || (row_bytes & 15)) return NF_EINVAL;
+int nf_cache_gather(const void* cache, const int32_t* cache_labels, int cache_rows, const int32_t* idx, int count,
+                    size_t row_bytes, void* out, int32_t* out_labels) {
+  if (!cache || !idx || !out || cache_rows < 1 || count < 1 || row_bytes == 0 || (row_bytes & 15)) return NF_EINVAL;
   if ((cache_labels == nullptr) != (out_labels == nullptr)) return NF_EINVAL;
   if (misaligned(cache) || misaligned(out)) return NF_EALIGN;
-  return nf_ref_gather(cache, cache_labels, idx, count, row_bytes, out, out_labels);
+  int32_t* st = nullptr;
+  NF_TRY(nf_tc_op_status_ptr(&st));
+  return nf_k_gather(cache, cache_labels, cache_rows, idx, count, row_bytes, out, out_labels, st);
 }
 
 static bool conv_args_ok(int dtype, int N, int H, int W, int Cin, int Cout, int stride) {
@@ -740,13 +798,13 @@ int nf_conv3x3_forward(int dtype, const void* x, const void* w, int N, int H, in
     const int rc = nf_tc_conv3x3_forward(x, w, N, H, W, Cin, Cout, stride, y);
     if (rc != NF_EUNSUPPORTED) return rc;
   }
-  return nf_ref_conv(dtype, x, N, H, W, Cin, w, (long)Cout * Cin, Cin, 1, 0, nullptr, 0, stride, Cout, y);
+  return nf_k_conv(dtype, x, N, H, W, Cin, w, (long)Cout * Cin, Cin, 1, 0, nullptr, 0, stride, Cout, y);
 }
 
 size_t nf_conv3x3_wgrad_scratch_bytes(int N, int H, int W, int Cin, int Cout, int stride) {
   if (!conv_args_ok(NF_F32, N, H, W, Cin, Cout, stride)) return 0;
   const int Ho = (H - 1) / stride + 1;
-  size_t fl = (size_t)nf_ref_wgrad_splits(N, Ho, Cin, Cout) * 9 * Cout * Cin;
+  size_t fl = (size_t)nf_k_wgrad_splits(N, Ho, Cin, Cout) * 9 * Cout * Cin;
   const size_t tc = nf_tc_conv3x3_wgrad_scratch_floats(N, H, W, Cin, Cout, stride);
   if (tc > fl) fl = tc;
   return fl * sizeof(float);
@@ -760,7 +818,7 @@ int nf_conv3x3_wgrad(int dtype, const void* x, const void* g, int N, int H, int 
     const int rc = nf_tc_conv3x3_wgrad(x, g, N, H, W, Cin, Cout, stride, (float*)scratch, scratch_bytes / sizeof(float), dw);
     if (rc != NF_EUNSUPPORTED) return rc;
   }
-  return nf_ref_wgrad(dtype, x, N, H, W, Cin, g, Cout, stride, (float*)scratch, scratch_bytes / sizeof(float), dw);
+  return nf_k_wgrad(dtype, x, N, H, W, Cin, g, Cout, stride, (float*)scratch, scratch_bytes / sizeof(float), dw);
 }
 
 int nf_op_status(void) {
@@ -769,23 +827,30 @@ int nf_op_status(void) {
   return rc == NF_OK ? (int)v : rc;
 }
 
+int nf_selftest_bounded_wait(unsigned long long limit_ns, unsigned long long* waited_ns_dev) {
+  if (!waited_ns_dev || limit_ns == 0 || limit_ns > 1000000000ull) return NF_EINVAL;  // at most one second
+  if ((uintptr_t)waited_ns_dev & 7) return NF_EALIGN;
+  return nf_tc_bounded_wait_probe(limit_ns, waited_ns_dev);
+}
+
+// Algorithm 1, second part.  One pass over the layers: a block stays open while the capped batch size of the next layer
+// is within rho (relative to the current layer's) of the current one; the block's batch size is the running minimum of
+// its members.
 int nf_partition(const int* max_batch, int n_layers, int Bcap, double rho, int* block_first, int* block_batch) {
   if (!max_batch || !block_first || !block_batch || n_layers < 1 || Bcap < 1 || !(rho >= 0.0)) return NF_EINVAL;
-  std::vector<int> b(n_layers);
-  for (int i = 0; i < n_layers; ++i) {
+  for (int i = 0; i < n_layers; ++i)
     if (max_batch[i] < 1) return NF_EINVAL;
-    b[i] = max_batch[i] < Bcap ? max_batch[i] : Bcap;
-  }
-  int nblocks = 0, i = 0;
-  while (i < n_layers) {
-    int bs = b[i];
-    block_first[nblocks] = i;
-    while (i + 1 < n_layers && fabs((double)b[i + 1] - (double)b[i]) <= rho * (double)b[i]) {
-      if (b[i + 1] < bs) bs = b[i + 1];
-      ++i;
+  auto capped = [&](int i) { return std::min(max_batch[i], Bcap); };
+  int nblocks = 0;
+  for (int i = 0; i < n_layers; ++i) {
+    const int b = capped(i);
+    const bool joins = i > 0 && fabs((double)b - (double)capped(i - 1)) <= rho * (double)capped(i - 1);
+    if (joins) {
+      block_batch[nblocks - 1] = std::min(block_batch[nblocks - 1], b);
+    } else {
+      block_first[nblocks] = i;
+      block_batch[nblocks++] = b;
     }
-    block_batch[nblocks++] = bs;
-    ++i;
   }
   return nblocks;
 }
@@ -805,12 +870,25 @@ int nf_aan_filters(const int* channels, int n_layers, int first_downsample, int*
   return NF_OK;
 }
 
+int nf_fit_line(const double* batches, const double* bytes, int k, double* slope, double* intercept) {
+  if (!batches || !bytes || !slope || !intercept || k < 2) return NF_EINVAL;
+  double sx = 0, sy = 0, sxx = 0, sxy = 0;
+  for (int i = 0; i < k; ++i) {
+    sx += batches[i]; sy += bytes[i]; sxx += batches[i] * batches[i]; sxy += batches[i] * bytes[i];
+  }
+  const double den = k * sxx - sx * sx;
+  if (!(den > 0.0)) return NF_EINVAL;  // all batch sizes equal
+  *slope = (k * sxy - sx * sy) / den;
+  *intercept = (sy - *slope * sx) / k;
+  return NF_OK;
+}
+
 int nf_profile_layer(int Cin, int Cout, int H, int W, int F, int classes, const nf_layer_opts* opts, const int* batches, int k,
                      double* bytes_out, double* slope, double* intercept) {
   if (!opts || !batches || !slope || !intercept || k < 2) return NF_EINVAL;
   nf_layer* L = nf_layer_create(Cin, Cout, H, W, F, classes);
   if (!L) return NF_EINVAL;
-  double sx = 0, sy = 0, sxx = 0, sxy = 0;
+  std::vector<double> xs(k), ys(k);
   for (int i = 0; i < k; ++i) {
     nf_layer_opts o = *opts;
     o.N = batches[i];
@@ -819,17 +897,12 @@ int nf_profile_layer(int Cin, int Cout, int H, int W, int F, int classes, const 
       nf_layer_destroy(L);
       return rc;
     }
-    const double bytes = (double)nf_layer_workspace_bytes(L) + (double)o.N * H * W * Cin * (double)nf_esize(o.dtype);
-    if (bytes_out) bytes_out[i] = bytes;
-    const double x = (double)o.N;
-    sx += x; sy += bytes; sxx += x * x; sxy += x * bytes;
+    xs[i] = (double)o.N;
+    ys[i] = (double)nf_layer_workspace_bytes(L) + (double)o.N * H * W * Cin * (double)nf_esize(o.dtype);
+    if (bytes_out) bytes_out[i] = ys[i];
   }
   nf_layer_destroy(L);
-  const double den = k * sxx - sx * sx;
-  if (!(den > 0.0)) return NF_EINVAL;  // all batch sizes equal
-  *slope = (k * sxy - sx * sy) / den;
-  *intercept = (sy - *slope * sx) / k;
-  return NF_OK;
+  return nf_fit_line(xs.data(), ys.data(), k, slope, intercept);
 }
 
 long long nf_max_batch(double slope, double intercept, double budget_bytes) {
@@ -846,8 +919,9 @@ int nf_set_stream(void* s) {
 long long nf_launch_count(void) { return g_nf_launches; }
 
 const char* nf_layer_kernel_family(const nf_layer* L, int op) {
-  if (!L || op < 0 || op > 4) return "";
+  if (!L || op < 0 || op > 5) return "";
   if (op == 4) return nf_tc_bn_aux_fused(L) && !L->skip ? "fused" : "separate";
+  if (op == 5) return nf_tc_bn_aux_fused(L) && !L->skip && nf_tc_aux_pool_fused(L) ? "mask" : "stored";
   return L->fam[op] ? "tcgen05" : "cuda-core";
 }
 

@@ -276,7 +276,7 @@ inline bool smallc_ok(int Ci, int Co, int W) { return Ci <= 4 && Co % 16 == 0 &&
 
 }  // namespace
 
-int nf_ref_conv(int dtype, const void* x, int N, int H, int W, int Ci, const void* w, long ws_tap, long ws_co,
+int nf_k_conv(int dtype, const void* x, int N, int H, int W, int Ci, const void* w, long ws_tap, long ws_co,
                 long ws_ci, int flip, const float* bias, int relu, int stride, int Co, void* y) {
   const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
   if (smallc_ok(Ci, Co, W) && !flip && !bias && !relu && ws_ci == 1 && ws_co == Ci && ws_tap == (long)Co * Ci) {
@@ -307,7 +307,7 @@ int nf_ref_conv(int dtype, const void* x, int N, int H, int W, int Ci, const voi
   return NF_OK;
 }
 
-int nf_ref_wgrad_splits(int N, int Ho, int Ci, int Co) {
+int nf_k_wgrad_splits(int N, int Ho, int Ci, int Co) {
   if (Ci <= 4 && Co % 16 == 0 && Co <= 128) {  // first-layer kernel: one block per slice of rows
     long sp = (long)N * Ho;
     return (int)(sp > 1184 ? 1184 : sp);
@@ -319,10 +319,10 @@ int nf_ref_wgrad_splits(int N, int Ho, int Ci, int Co) {
   return (int)s;
 }
 
-int nf_ref_wgrad(int dtype, const void* x, int N, int H, int W, int Ci, const void* g, int Co, int stride,
+int nf_k_wgrad(int dtype, const void* x, int N, int H, int W, int Ci, const void* g, int Co, int stride,
                  float* part, size_t part_floats, float* dw) {
   const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
-  const int splits = nf_ref_wgrad_splits(N, Ho, Ci, Co);
+  const int splits = nf_k_wgrad_splits(N, Ho, Ci, Co);
   const size_t n = (size_t)9 * Co * Ci;
   if ((size_t)splits * n > part_floats) return NF_ENOWS;
   if (smallc_ok(Ci, Co, W)) {

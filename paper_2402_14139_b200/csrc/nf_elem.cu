@@ -567,15 +567,25 @@ __global__ void bn_bwd_apply_kernel(const T* __restrict__ y, const T* __restrict
   stf(dy, e, scale[c] * (dz - sdz[c] * invM - xh * sdzx[c] * invM));
 }
 
-__global__ void sgd_kernel(float* __restrict__ val, float* __restrict__ mom, const float* __restrict__ grad,
-                           bf16* __restrict__ shadow, size_t n, float lr, float mu) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const float v = fmaf(mu, mom[i], grad[i]);
-  const float t = fmaf(-lr, v, val[i]);
-  mom[i] = v;
-  val[i] = t;
-  shadow[i] = __float2bfloat16_rn(t);
+// Momentum SGD over up to kSgdMaxArenas parameter arenas in one launch (all layers of a block).  An arena is a multiple
+// of 64 floats and 256-byte aligned, so every thread owns four consecutive elements: 16-byte loads of value, momentum and
+// gradient, 16-byte stores of value and momentum, one 8-byte store of the four bf16 copies.  Blocks are dealt to arenas
+// through the table of first-block indices.
+__global__ void __launch_bounds__(256) sgd_multi_kernel(const SgdTable tb, float lr, float mu) {
+  int a = 0;
+  while (a + 1 < tb.count && (int)blockIdx.x >= tb.first_block[a + 1]) ++a;
+  const size_t i4 = (size_t)(blockIdx.x - tb.first_block[a]) * blockDim.x + threadIdx.x;
+  if (i4 * 4 >= tb.n[a]) return;
+  const float4 g = reinterpret_cast<const float4*>(tb.grad[a])[i4];
+  float4 m = reinterpret_cast<const float4*>(tb.mom[a])[i4];
+  float4 t = reinterpret_cast<const float4*>(tb.val[a])[i4];
+  m.x = fmaf(mu, m.x, g.x); m.y = fmaf(mu, m.y, g.y); m.z = fmaf(mu, m.z, g.z); m.w = fmaf(mu, m.w, g.w);
+  t.x = fmaf(-lr, m.x, t.x); t.y = fmaf(-lr, m.y, t.y); t.z = fmaf(-lr, m.z, t.z); t.w = fmaf(-lr, m.w, t.w);
+  reinterpret_cast<float4*>(tb.mom[a])[i4] = m;
+  reinterpret_cast<float4*>(tb.val[a])[i4] = t;
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(t.x, t.y), hi = __floats2bfloat162_rn(t.z, t.w);
+  reinterpret_cast<uint2*>(tb.shadow[a])[i4] =
+      make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
 }
 
 __global__ void shadow_kernel(const float* __restrict__ val, bf16* __restrict__ shadow, size_t n) {
@@ -584,15 +594,20 @@ __global__ void shadow_kernel(const float* __restrict__ val, bf16* __restrict__ 
 }
 
 // out row r = cache row idx[r], 16 bytes per thread
-__global__ void gather_kernel(const uint4* __restrict__ cache, const int32_t* __restrict__ cache_labels,
+// An index outside [0, cache_rows) reads nothing: its output row is zero-filled, its label set to -1 and NF_EINDEX raised.
+__global__ void gather_kernel(const uint4* __restrict__ cache, const int32_t* __restrict__ cache_labels, int cache_rows,
                               const int32_t* __restrict__ idx, int count, size_t row16, uint4* __restrict__ out,
-                              int32_t* __restrict__ out_labels) {
+                              int32_t* __restrict__ out_labels, int32_t* __restrict__ status) {
   const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= (size_t)count * row16) return;
   const size_t r = e / row16, k = e % row16;
-  const size_t src = (size_t)idx[r];
-  out[e] = cache[src * row16 + k];
-  if (k == 0 && out_labels) out_labels[r] = cache_labels[src];
+  const int32_t src = idx[r];
+  const bool ok = src >= 0 && src < cache_rows;
+  out[e] = ok ? cache[(size_t)src * row16 + k] : make_uint4(0u, 0u, 0u, 0u);
+  if (k == 0) {
+    if (out_labels) out_labels[r] = ok ? cache_labels[src] : -1;
+    if (!ok) atomicOr(status, NF_EINDEX);
+  }
 }
 
 
@@ -964,6 +979,72 @@ __global__ void __launch_bounds__(256) avgpool_part_vec_kernel(const uint4* __re
   }
 }
 // stage 2: p[n][f*4+bin] = sum over slices / |bin|
+// Average pool to 2 x 2 from the partials the fused aux forward leaves: part[tile][4][F] holds, per 14 x 8-pixel tile (tiles in
+// row-major order per image, th x tw of them) and epilogue warp, the channel sums over the warp's pixels.  One block per
+// (image, quadrant); thread (f, lane) adds every `lanes`-th of the quadrant's th/2 * tw/2 * 4 partials in index order, the lane
+// sums are added in lane order.
+__global__ void __launch_bounds__(256) pool_finish_kernel(const float* __restrict__ part, int th, int tw, int F, float inv_cnt,
+                                                          float* __restrict__ p) {
+  __shared__ float sm[256];
+  const int n = blockIdx.x >> 2, bin = blockIdx.x & 3, u = bin >> 1, v = bin & 1;
+  const int lanes = 256 / F, f = threadIdx.x % F, ln = threadIdx.x / F;
+  const int qh = th / 2, qw = tw / 2, cnt = qh * qw * 4;
+  float s = 0.f;
+  if (ln < lanes) {
+    for (int k = ln; k < cnt; k += lanes) {
+      const int w4 = k & 3, tq = k >> 2, ty = u * qh + tq / qw, tx = v * qw + tq % qw;
+      s += part[(((size_t)n * th + ty) * tw + tx) * 4 * F + (size_t)w4 * F + f];
+    }
+  }
+  sm[threadIdx.x] = s;
+  __syncthreads();
+  if (ln == 0) {
+    float t = 0.f;
+    for (int l = 0; l < lanes; ++l) t += sm[l * F + f];
+    p[(size_t)n * 4 * F + f * 4 + bin] = t * inv_cnt;
+  }
+}
+
+// dh from the sign mask of h (one bit per element, byte g of a pixel = channels 8g .. 8g+7): dh = bit ? dp[n][f*4+bin] / |bin| : 0,
+// stored in bf16; per-block partial sums of the stored values for the bias gradient, laid out as dh_vec_kernel does.
+__global__ void __launch_bounds__(256) dh_mask_vec_kernel(const uint8_t* __restrict__ mask, const float* __restrict__ dp, int Ha, int Wa,
+                                                          int F8, size_t P, uint4* __restrict__ dh, float* __restrict__ red) {
+  __shared__ float sm[8][256];
+  const int F = F8 * 8;
+  const int planes = 256 / F8, g = threadIdx.x % F8, pl = threadIdx.x / F8;
+  const float inv_bin = 1.f / (float)((Ha / 2) * (Wa / 2));
+  float a[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a[i] = 0.f;
+  const size_t p0 = P * blockIdx.x / gridDim.x, p1 = P * (blockIdx.x + 1) / gridDim.x;
+  for (size_t p = p0 + pl; pl < planes && p < p1; p += planes) {  // threads beyond planes * F8 (F8 not a divisor of 256) idle
+    const uint32_t m = mask[p * F8 + g];
+    const int j = (int)(p % Wa), i = (int)((p / Wa) % Ha);
+    const size_t n = p / ((size_t)Wa * Ha);
+    const int bin = (i >= Ha / 2 ? 2 : 0) + (j >= Wa / 2 ? 1 : 0);
+    const float* d = dp + n * 4 * F + (size_t)(g * 8) * 4 + bin;
+    float o[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) o[e] = (m >> e) & 1u ? d[e * 4] * inv_bin : 0.f;
+    const uint4 packed = pack8(o);
+    dh[p * F8 + g] = packed;
+    float r[8];
+    unpack8(packed, r);  // the bias gradient sums the values as stored
+#pragma unroll
+    for (int e = 0; e < 8; ++e) a[e] += r[e];
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) sm[e][threadIdx.x] = a[e];
+  __syncthreads();
+  for (int t = threadIdx.x; t < F; t += 256) {
+    const int gg = t / 8, e = t % 8;
+    float s = 0.f;
+    for (int q = 0; q < planes; ++q) s += sm[e][q * F8 + gg];
+    red[((size_t)blockIdx.x * 2 + 0) * F + t] = s;
+    red[((size_t)blockIdx.x * 2 + 1) * F + t] = 0.f;
+  }
+}
+
 __global__ void avgpool_finish_kernel(const float* __restrict__ part, int N, int F, int S, float inv_cnt, float* __restrict__ p) {
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= N * 4 * F) return;
@@ -1123,7 +1204,7 @@ inline unsigned nblk(size_t n, int per) { return (unsigned)((n + per - 1) / per)
     if ((dtype) == NF_F32) { CALL_F32; } else { CALL_BF16; } \
   } while (0)
 
-int nf_ref_channel_blocks(size_t P, int C) {
+int nf_k_channel_blocks(size_t P, int C) {
   const int planes = 256 / pow2ceil_cap256(C);
   size_t nb = (P + (size_t)planes * 16 - 1) / ((size_t)planes * 16);
   if (nb < 1) nb = 1;
@@ -1131,8 +1212,8 @@ int nf_ref_channel_blocks(size_t P, int C) {
   return (int)nb;
 }
 
-int nf_ref_channel_sums(int dtype, const void* src, size_t P, int C, float* red, size_t red_floats, int* nblocks) {
-  const int nb = nf_ref_channel_blocks(P, C);
+int nf_k_channel_sums(int dtype, const void* src, size_t P, int C, float* red, size_t red_floats, int* nblocks) {
+  const int nb = nf_k_channel_blocks(P, C);
   if ((size_t)nb * 2 * C > red_floats) return NF_ENOWS;
   if (vec_ok(dtype, C, 0) && 256 % (C / 8) == 0) {
     channel_sums_vec_kernel<<<nb, 256, 0, g_nf_stream>>>((const uint4*)src, P, C / 8, red);
@@ -1148,7 +1229,7 @@ int nf_ref_channel_sums(int dtype, const void* src, size_t P, int C, float* red,
   return NF_OK;
 }
 
-int nf_ref_bn_finalize(const float* red, int nblocks, int C, double M, const float* gamma, const float* beta,
+int nf_k_bn_finalize(const float* red, int nblocks, int C, double M, const float* gamma, const float* beta,
                        float eps, float bn_momentum, float* scale, float* shift, float* mu, float* invstd,
                        float* rmean, float* rvar) {
   bn_finalize_kernel<<<nblk(C, 32), dim3(32, 32), 0, g_nf_stream>>>(red, nblocks, C, M, gamma, beta, eps, bn_momentum, scale,
@@ -1157,13 +1238,13 @@ int nf_ref_bn_finalize(const float* red, int nblocks, int C, double M, const flo
   return NF_OK;
 }
 
-int nf_ref_partial_totals(const float* red, int nblocks, int C, double* tot) {
+int nf_k_partial_totals(const float* red, int nblocks, int C, double* tot) {
   partial_totals_kernel<<<nblk(C, 32), dim3(32, 32), 0, g_nf_stream>>>(red, nblocks, C, tot);
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_bn_finalize_tot(const double* tot, int C, double M, const float* gamma, const float* beta, float eps, float bn_momentum,
+int nf_k_bn_finalize_tot(const double* tot, int C, double M, const float* gamma, const float* beta, float eps, float bn_momentum,
                            float* scale, float* shift, float* mu, float* invstd, float* rmean, float* rvar) {
   bn_finalize_tot_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(tot, C, M, gamma, beta, eps, bn_momentum, scale, shift, mu, invstd,
                                                                 rmean, rvar);
@@ -1171,20 +1252,20 @@ int nf_ref_bn_finalize_tot(const double* tot, int C, double M, const float* gamm
   return NF_OK;
 }
 
-int nf_ref_bn_bwd_finalize_tot(const double* tot, int C, int world, float* sdz, float* sdzx, float* ggamma, float* gbeta) {
+int nf_k_bn_bwd_finalize_tot(const double* tot, int C, int world, float* sdz, float* sdzx, float* ggamma, float* gbeta) {
   bn_bwd_finalize_tot_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(tot, C, 1.0 / (double)world, sdz, sdzx, ggamma, gbeta);
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float eps, const float* rmean,
+int nf_k_bn_eval_coeffs(int C, const float* gamma, const float* beta, float eps, const float* rmean,
                           const float* rvar, float* scale, float* shift) {
   bn_eval_coeffs_kernel<<<nblk(C, 128), 128, 0, g_nf_stream>>>(C, gamma, beta, eps, rmean, rvar, scale, shift);
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
+int nf_k_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
                     const float* shift, void* out, const void* skip) {
   const size_t total = (size_t)N * (pool ? Ho / 2 : Ho) * (pool ? Wo / 2 : Wo) * C;
   if (skip) {  // residual layers take the generic kernels
@@ -1218,7 +1299,7 @@ int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int 
   return NF_OK;
 }
 
-int nf_ref_avgpool_slices(int N, int Ha, int Wa) {
+int nf_k_avgpool_slices(int N, int Ha, int Wa) {
   const long cnt = (long)(Ha / 2) * (Wa / 2);
   long S = 1184 / ((long)N * 4);
   if (S > cnt / 64) S = cnt / 64;
@@ -1226,9 +1307,9 @@ int nf_ref_avgpool_slices(int N, int Ha, int Wa) {
   return (int)S;
 }
 
-int nf_ref_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part, size_t part_floats, float* p) {
+int nf_k_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part, size_t part_floats, float* p) {
   if (F % 8 || 256 % (F / 8) || (Ha & 1) || (Wa & 1)) return NF_EUNSUPPORTED;
-  const int S = nf_ref_avgpool_slices(N, Ha, Wa);
+  const int S = nf_k_avgpool_slices(N, Ha, Wa);
   if ((size_t)N * 4 * S * F > part_floats) return NF_EUNSUPPORTED;
   avgpool_part_vec_kernel<<<N * 4 * S, 256, 0, g_nf_stream>>>((const uint4*)h, Ha, Wa, F / 8, S, part);
   NF_LAUNCHED();
@@ -1238,11 +1319,30 @@ int nf_ref_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part
 }
 
 // dh with the fused aux-bias gradient partials (bf16, F % 8 == 0, even sizes); nblocks partials in red
-int nf_ref_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh, float* red, size_t red_floats,
+int nf_k_pool_finish(const float* part, int N, int th, int tw, int F, float inv_cnt, float* p) {
+  if (F < 1 || F > 256) return NF_EUNSUPPORTED;
+  pool_finish_kernel<<<N * 4, 256, 0, g_nf_stream>>>(part, th, tw, F, inv_cnt, p);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_k_dh_mask(const uint8_t* mask, const float* dp, int N, int Ha, int Wa, int F, void* dh, float* red, size_t red_floats,
+                 int* nblocks) {
+  if (F % 8 || F > 2048 || (Ha & 1) || (Wa & 1)) return NF_EUNSUPPORTED;
+  const size_t P = (size_t)N * Ha * Wa;
+  const int nb = nf_k_channel_blocks(P, F);
+  if ((size_t)nb * 2 * F > red_floats) return NF_ENOWS;
+  dh_mask_vec_kernel<<<nb, 256, 0, g_nf_stream>>>(mask, dp, Ha, Wa, F / 8, P, (uint4*)dh, red);
+  NF_LAUNCHED();
+  *nblocks = nb;
+  return NF_OK;
+}
+
+int nf_k_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh, float* red, size_t red_floats,
                    int* nblocks) {
   if (F % 8 || 256 % (F / 8) || (Ha & 1) || (Wa & 1)) return NF_EUNSUPPORTED;
   const size_t P = (size_t)N * Ha * Wa;
-  const int nb = nf_ref_channel_blocks(P, F);
+  const int nb = nf_k_channel_blocks(P, F);
   if ((size_t)nb * 2 * F > red_floats) return NF_EUNSUPPORTED;
   dh_vec_kernel<<<nb, 256, 0, g_nf_stream>>>((const uint4*)h, dp, Ha, Wa, F / 8, P, (uint4*)dh, red);
   NF_LAUNCHED();
@@ -1250,14 +1350,14 @@ int nf_ref_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F,
   return NF_OK;
 }
 
-int nf_ref_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p) {
+int nf_k_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p) {
   DISPATCH(dtype, (avgpool_kernel<float><<<N * 4, 256, 0, g_nf_stream>>>((const float*)h, Ha, Wa, F, p)),
            (avgpool_kernel<bf16><<<N * 4, 256, 0, g_nf_stream>>>((const bf16*)h, Ha, Wa, F, p)));
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
+int nf_k_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
                  float* logits, float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind, int n_scale) {
   const size_t smem = (size_t)(D + K) * sizeof(float);
   if (smem > 40000) return NF_EUNSUPPORTED;
@@ -1274,14 +1374,14 @@ __global__ void __launch_bounds__(256) count_equal_kernel(const int32_t* __restr
   if ((threadIdx.x & 31) == 0 && c) atomicAdd(count, (unsigned long long)c);   // integer sum: order-independent
 }
 
-int nf_ref_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count) {
+int nf_k_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count) {
   const int blocks = (int)std::min<long long>((n + 255) / 256, 1184);
   count_equal_kernel<<<blocks, 256, 0, g_nf_stream>>>(a, b, n, count);
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_fc_predict(const float* p, int N, int D, int K, const float* Wf, const float* bf, float* logits, int32_t* pred) {
+int nf_k_fc_predict(const float* p, int N, int D, int K, const float* Wf, const float* bf, float* logits, int32_t* pred) {
   const size_t smem = (size_t)D * sizeof(float);
   if (smem > 40000) return NF_EUNSUPPORTED;
   fc_predict_kernel<<<N, 256, smem, g_nf_stream>>>(p, D, K, Wf, bf, logits, pred);
@@ -1289,7 +1389,7 @@ int nf_ref_fc_predict(const float* p, int N, int D, int K, const float* Wf, cons
   return NF_OK;
 }
 
-int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
+int nf_k_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
                     float* gbf, float* loss_out, int32_t* status, int n_scale) {
   fc_wgrad_kernel<<<K, 256, 0, g_nf_stream>>>(p, dlogits, lossn, N, D, K, gWf, gbf, loss_out, status, n_scale);
   NF_LAUNCHED();
@@ -1304,20 +1404,20 @@ __global__ void flip_weights_kernel(const bf16* __restrict__ w, int F, int C, bf
   out[e] = w[((size_t)(8 - tap) * F + f) * C + c];
 }
 
-int nf_ref_flip_weights(const bf16* w, int F, int C, bf16* out) {
+int nf_k_flip_weights(const bf16* w, int F, int C, bf16* out) {
   flip_weights_kernel<<<nblk((size_t)9 * F * C, 256), 256, 0, g_nf_stream>>>(w, F, C, out);
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_auxmax(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p, int32_t* parg) {
+int nf_k_auxmax(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p, int32_t* parg) {
   DISPATCH(dtype, (auxmax_kernel<float><<<N * 4, 256, 0, g_nf_stream>>>((const float*)h, Ha, Wa, F, p, parg)),
            (auxmax_kernel<bf16><<<N * 4, 256, 0, g_nf_stream>>>((const bf16*)h, Ha, Wa, F, p, parg)));
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_dh_max(int dtype, const void* h, const float* dp, const int32_t* parg, int N, int Ha, int Wa, int F, void* dh) {
+int nf_k_dh_max(int dtype, const void* h, const float* dp, const int32_t* parg, int N, int Ha, int Wa, int F, void* dh) {
   const size_t total = (size_t)N * Ha * Wa * F;
   DISPATCH(dtype, (dh_max_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)h, dp, parg, Ha, Wa, F, total, (float*)dh)),
            (dh_max_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)h, dp, parg, Ha, Wa, F, total, (bf16*)dh)));
@@ -1325,7 +1425,7 @@ int nf_ref_dh_max(int dtype, const void* h, const float* dp, const int32_t* parg
   return NF_OK;
 }
 
-int nf_ref_dh(int dtype, const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh) {
+int nf_k_dh(int dtype, const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh) {
   const size_t total = (size_t)N * Ha * Wa * F;
   DISPATCH(dtype, (dh_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)h, dp, Ha, Wa, F, total, (float*)dh)),
            (dh_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)h, dp, Ha, Wa, F, total, (bf16*)dh)));
@@ -1333,17 +1433,17 @@ int nf_ref_dh(int dtype, const void* h, const float* dp, int N, int Ha, int Wa, 
   return NF_OK;
 }
 
-int nf_ref_sum_partials(const float* red, int nblocks, int C, int which, float* out) {
+int nf_k_sum_partials(const float* red, int nblocks, int C, int which, float* out) {
   sum_partials_kernel<<<nblk(C, 32), dim3(32, 32), 0, g_nf_stream>>>(red, nblocks, C, which, out);
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
+int nf_k_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
                          const float* scale, const float* shift, const float* mu, const float* invstd, float* red,
                          size_t red_floats, int* nblocks, const void* skip) {
   const size_t P = (size_t)N * Ho * Wo;
-  const int nb = nf_ref_channel_blocks(P, C);
+  const int nb = nf_k_channel_blocks(P, C);
   if ((size_t)nb * 2 * C > red_floats) return NF_ENOWS;
   if (!skip && pool && vec_ok(dtype, C, 0) && 256 % (C / 8) == 0) {
     bn_bwd_reduce_pool_vec_kernel<<<nb, 256, 0, g_nf_stream>>>((const uint4*)y, (const uint4*)da, P / 4, Ho, Wo, C / 8, scale, shift, mu,
@@ -1367,14 +1467,14 @@ int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho
   return NF_OK;
 }
 
-int nf_ref_bn_bwd_finalize(const float* red, int nblocks, int C, float* sdz, float* sdzx, float* ggamma,
+int nf_k_bn_bwd_finalize(const float* red, int nblocks, int C, float* sdz, float* sdzx, float* ggamma,
                            float* gbeta) {
   bn_bwd_finalize_kernel<<<nblk(C, 32), dim3(32, 32), 0, g_nf_stream>>>(red, nblocks, C, sdz, sdzx, ggamma, gbeta);
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
+int nf_k_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
                         const float* scale, const float* shift, const float* mu, const float* invstd,
                         const float* sdz, const float* sdzx, double M, void* dy, const void* skip) {
   const size_t total = (size_t)N * Ho * Wo * C;
@@ -1411,23 +1511,38 @@ int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho,
   return NF_OK;
 }
 
-int nf_ref_sgd(float* val, float* mom, const float* grad, bf16* shadow, size_t n, float lr, float momentum) {
-  sgd_kernel<<<nblk(n, 256), 256, 0, g_nf_stream>>>(val, mom, grad, shadow, n, lr, momentum);
+int nf_k_sgd_multi(const SgdTable& tb_in, float lr, float momentum) {
+  if (tb_in.count < 1 || tb_in.count > kSgdMaxArenas) return NF_EINVAL;
+  SgdTable tb = tb_in;
+  int blocks = 0;
+  for (int a = 0; a < tb.count; ++a) {
+    if (tb.n[a] % 4) return NF_EINVAL;
+    tb.first_block[a] = blocks;
+    blocks += (int)nblk(tb.n[a] / 4, 256);
+  }
+  sgd_multi_kernel<<<blocks, 256, 0, g_nf_stream>>>(tb, lr, momentum);
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_shadow(const float* val, bf16* shadow, size_t n) {
+int nf_k_sgd(float* val, float* mom, const float* grad, bf16* shadow, size_t n, float lr, float momentum) {
+  SgdTable tb{};
+  tb.count = 1;
+  tb.val[0] = val; tb.mom[0] = mom; tb.grad[0] = grad; tb.shadow[0] = shadow; tb.n[0] = n;
+  return nf_k_sgd_multi(tb, lr, momentum);
+}
+
+int nf_k_shadow(const float* val, bf16* shadow, size_t n) {
   shadow_kernel<<<nblk(n, 256), 256, 0, g_nf_stream>>>(val, shadow, n);
   NF_LAUNCHED();
   return NF_OK;
 }
 
-int nf_ref_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count, size_t row_bytes,
-                  void* out, int32_t* out_labels) {
+int nf_k_gather(const void* cache, const int32_t* cache_labels, int cache_rows, const int32_t* idx, int count, size_t row_bytes,
+                  void* out, int32_t* out_labels, int32_t* status) {
   const size_t row16 = row_bytes / 16;
-  gather_kernel<<<nblk((size_t)count * row16, 256), 256, 0, g_nf_stream>>>((const uint4*)cache, cache_labels, idx, count,
-                                                                         row16, (uint4*)out, out_labels);
+  gather_kernel<<<nblk((size_t)count * row16, 256), 256, 0, g_nf_stream>>>((const uint4*)cache, cache_labels, cache_rows, idx,
+                                                                         count, row16, (uint4*)out, out_labels, status);
   NF_LAUNCHED();
   return NF_OK;
 }

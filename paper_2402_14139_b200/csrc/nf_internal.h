@@ -87,32 +87,36 @@ int nf_cuda_check(cudaError_t e, const char* what);
 static inline size_t nf_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline size_t nf_esize(int dtype) { return dtype == NF_F32 ? 4 : 2; }
 
-// ---- generic CUDA-core kernels (nf_ref_kernels.cu): any shape, fp32 or bf16 storage, fp32 accumulate
-int nf_ref_conv(int dtype, const void* x, int N, int H, int W, int Ci, const void* w, long ws_tap, long ws_co,
+// ---- generic CUDA-core kernels (nf_k_kernels.cu): any shape, fp32 or bf16 storage, fp32 accumulate
+int nf_k_conv(int dtype, const void* x, int N, int H, int W, int Ci, const void* w, long ws_tap, long ws_co,
                 long ws_ci, int flip, const float* bias, int relu, int stride, int Co, void* y);
-int nf_ref_wgrad_splits(int N, int Ho, int Ci, int Co);
-int nf_ref_wgrad(int dtype, const void* x, int N, int H, int W, int Ci, const void* g, int Co, int stride,
+int nf_k_wgrad_splits(int N, int Ho, int Ci, int Co);
+int nf_k_wgrad(int dtype, const void* x, int N, int H, int W, int Ci, const void* g, int Co, int stride,
                  float* part, size_t part_floats, float* dw);
-int nf_ref_channel_blocks(size_t P, int C);
-int nf_ref_channel_sums(int dtype, const void* src, size_t P, int C, float* red, size_t red_floats, int* nblocks);
-int nf_ref_bn_finalize(const float* red, int nblocks, int C, double M, const float* gamma, const float* beta,
+int nf_k_channel_blocks(size_t P, int C);
+int nf_k_channel_sums(int dtype, const void* src, size_t P, int C, float* red, size_t red_floats, int* nblocks);
+int nf_k_bn_finalize(const float* red, int nblocks, int C, double M, const float* gamma, const float* beta,
                        float eps, float bn_momentum, float* scale, float* shift, float* mu, float* invstd,
                        float* rmean, float* rvar);
-int nf_ref_bn_eval_coeffs(int C, const float* gamma, const float* beta, float eps, const float* rmean,
+int nf_k_bn_eval_coeffs(int C, const float* gamma, const float* beta, float eps, const float* rmean,
                           const float* rvar, float* scale, float* shift);
-int nf_ref_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
+int nf_k_bn_apply(int dtype, const void* y, int N, int Ho, int Wo, int C, int pool, const float* scale,
                     const float* shift, void* out, const void* skip = nullptr);
-int nf_ref_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p);
+int nf_k_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p);
 // bf16 fast paths (F % 8 == 0, even Ha and Wa); NF_EUNSUPPORTED means "use the generic kernel"
-int nf_ref_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part, size_t part_floats, float* p);
-int nf_ref_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh, float* red, size_t red_floats,
+int nf_k_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part, size_t part_floats, float* p);
+int nf_k_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh, float* red, size_t red_floats,
                    int* nblocks);
-int nf_ref_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
+// average pool from the per-tile partials of the fused aux forward, and dh from its sign mask (see nf_tc_aux_pool_fused)
+int nf_k_pool_finish(const float* part, int N, int th, int tw, int F, float inv_cnt, float* p);
+int nf_k_dh_mask(const uint8_t* mask, const float* dp, int N, int Ha, int Wa, int F, void* dh, float* red, size_t red_floats,
+                 int* nblocks);
+int nf_k_fc_ce(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf,
                  float* logits, float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind, int n_scale);
-int nf_ref_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count);
-int nf_ref_auxmax(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p, int32_t* parg);
-int nf_ref_dh_max(int dtype, const void* h, const float* dp, const int32_t* parg, int N, int Ha, int Wa, int F, void* dh);
-int nf_ref_flip_weights(const bf16* w, int F, int C, bf16* out);
+int nf_k_count_equal(const int32_t* a, const int32_t* b, long long n, unsigned long long* count);
+int nf_k_auxmax(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p, int32_t* parg);
+int nf_k_dh_max(int dtype, const void* h, const float* dp, const int32_t* parg, int N, int Ha, int Wa, int F, void* dh);
+int nf_k_flip_weights(const bf16* w, int F, int C, bf16* out);
 // large-batch head (nf_head.cu)
 bool nf_head_is_large(int N, int D, int K);
 size_t nf_head_scratch_floats(int N, int D, int K);
@@ -121,24 +125,41 @@ int nf_head_predict(const float* logits, int N, int K, int32_t* pred);
 int nf_head_step(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf, float* logits,
                  float* dlogits, float* dp, float* lossn, int32_t* status, int loss_kind, float* gWf, float* gbf, float* loss_out,
                  float* scratch, size_t scratch_floats, int n_scale);
-int nf_ref_partial_totals(const float* red, int nblocks, int C, double* tot);
-int nf_ref_bn_finalize_tot(const double* tot, int C, double M, const float* gamma, const float* beta, float eps, float bn_momentum,
+// small-batch head (nf_head_small.cu): class-sliced forward + backward of the linear layer and the loss; 0 floats = not covered
+size_t nf_head_small_scratch_floats(int N, int D, int K);
+int nf_head_small_step(const float* p, const int32_t* labels, int N, int D, int K, const float* Wf, const float* bf, float* logits,
+                       float* dp, float* lossn, int32_t* status, int loss_kind, float* gWf, float* gbf, float* loss_out,
+                       float* scratch, size_t scratch_floats, int n_scale);
+int nf_k_partial_totals(const float* red, int nblocks, int C, double* tot);
+int nf_k_bn_finalize_tot(const double* tot, int C, double M, const float* gamma, const float* beta, float eps, float bn_momentum,
                            float* scale, float* shift, float* mu, float* invstd, float* rmean, float* rvar);
-int nf_ref_bn_bwd_finalize_tot(const double* tot, int C, int world, float* sdz, float* sdzx, float* ggamma, float* gbeta);
-int nf_ref_fc_predict(const float* p, int N, int D, int K, const float* Wf, const float* bf, float* logits, int32_t* pred);
-int nf_ref_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
+int nf_k_bn_bwd_finalize_tot(const double* tot, int C, int world, float* sdz, float* sdzx, float* ggamma, float* gbeta);
+int nf_k_fc_predict(const float* p, int N, int D, int K, const float* Wf, const float* bf, float* logits, int32_t* pred);
+int nf_k_fc_wgrad(const float* p, const float* dlogits, const float* lossn, int N, int D, int K, float* gWf,
                     float* gbf, float* loss_out, int32_t* status, int n_scale);
-int nf_ref_dh(int dtype, const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh);
-int nf_ref_sum_partials(const float* red, int nblocks, int C, int which, float* out);
-int nf_ref_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
+int nf_k_dh(int dtype, const void* h, const float* dp, int N, int Ha, int Wa, int F, void* dh);
+int nf_k_sum_partials(const float* red, int nblocks, int C, int which, float* out);
+int nf_k_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
                          const float* scale, const float* shift, const float* mu, const float* invstd, float* red,
                          size_t red_floats, int* nblocks, const void* skip = nullptr);
-int nf_ref_bn_bwd_finalize(const float* red, int nblocks, int C, float* sdz, float* sdzx, float* ggamma,
+int nf_k_bn_bwd_finalize(const float* red, int nblocks, int C, float* sdz, float* sdzx, float* ggamma,
                            float* gbeta);
-int nf_ref_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
+int nf_k_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
                         const float* scale, const float* shift, const float* mu, const float* invstd,
                         const float* sdz, const float* sdzx, double M, void* dy, const void* skip = nullptr);
-int nf_ref_sgd(float* val, float* mom, const float* grad, bf16* shadow, size_t n, float lr, float momentum);
-int nf_ref_shadow(const float* val, bf16* shadow, size_t n);
-int nf_ref_gather(const void* cache, const int32_t* cache_labels, const int32_t* idx, int count, size_t row_bytes,
-                  void* out, int32_t* out_labels);
+int nf_k_sgd(float* val, float* mom, const float* grad, bf16* shadow, size_t n, float lr, float momentum);
+// the same update over several arenas (the layers of a block) in one launch; first_block is filled by the callee
+enum { kSgdMaxArenas = 48 };
+struct SgdTable {
+  int count;
+  float* val[kSgdMaxArenas];
+  float* mom[kSgdMaxArenas];
+  const float* grad[kSgdMaxArenas];
+  bf16* shadow[kSgdMaxArenas];
+  size_t n[kSgdMaxArenas];
+  int first_block[kSgdMaxArenas];
+};
+int nf_k_sgd_multi(const SgdTable& tb, float lr, float momentum);
+int nf_k_shadow(const float* val, bf16* shadow, size_t n);
+int nf_k_gather(const void* cache, const int32_t* cache_labels, int cache_rows, const int32_t* idx, int count, size_t row_bytes,
+                void* out, int32_t* out_labels, int32_t* status);

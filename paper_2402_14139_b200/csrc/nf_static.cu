@@ -1,6 +1,7 @@
 // Allocation-free weight gradient: the split partial sums live in a fixed device array that is
 // part of the library image, for callers that cannot provide (or allocate) scratch memory.
 #include "nf_internal.h"
+#include "nf_tc.h"
 
 // 16 MiB on every GPU that loads the library, until the process exits.
 static __device__ __align__(256) float g_static_scratch[NF_STATIC_SCRATCH_BYTES / sizeof(float)];
@@ -36,6 +37,12 @@ extern "C" int nf_conv3x3_wgrad_static(int dtype, const void* x, const void* g, 
   float* scratch = nullptr;
   const int rc = static_scratch(&scratch);
   if (rc != NF_OK) return rc;
-  // The kernels write every partial they later read, so stale contents of the shared array are harmless.
-  return nf_ref_wgrad(dtype, x, N, H, W, Cin, g, Cout, stride, scratch, NF_STATIC_SCRATCH_BYTES / sizeof(float), dw);
+  // Same dispatch as nf_conv3x3_wgrad: the tcgen05 kernels where they cover the shape, else the CUDA-core kernel.
+  // Both write every partial they later read, so stale contents of the shared array are harmless.
+  const size_t floats = NF_STATIC_SCRATCH_BYTES / sizeof(float);
+  if (dtype == NF_BF16) {
+    const int tc = nf_tc_conv3x3_wgrad(x, g, N, H, W, Cin, Cout, stride, scratch, floats, dw);
+    if (tc != NF_EUNSUPPORTED) return tc;
+  }
+  return nf_k_wgrad(dtype, x, N, H, W, Cin, g, Cout, stride, scratch, floats, dw);
 }

@@ -432,6 +432,11 @@ struct FoldParams {
   // XF: the input map is the conv output y; a = ReLU(y*scale + shift) is formed in shared memory and written to xf_a
   const float *xf_scale, *xf_shift;
   bf16* xf_a;         // [N][H][W][64 * kchunks]
+  // EPI 1 with pool_part != nullptr: h itself is not written.  What the rest of the step needs of it leaves the epilogue
+  // directly: per tile and epilogue warp the per-channel sums of h over the warp's pixels (the average pool to 2 x 2 adds
+  // them up; a tile never straddles a quadrant: H/2 % 8 == 0, W/2 % 14 == 0), and one bit per element, h > 0.
+  float* pool_part;   // [total_tiles][4][Cout]
+  uint8_t* mask;      // [N][H][W][Cout / 8], bit f % 8 of byte f / 8
 };
 
 // G   : width of one column-tap group of the accumulator (N = 3*G): 64 for the main conv, 16/32/64 for the
@@ -753,6 +758,48 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             *reinterpret_cast<uint4*>(dst + (((2 * q) ^ (orow & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
             *reinterpret_cast<uint4*>(dst + (((2 * q + 1) ^ (orow & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
           }
+        } else if (p.pool_part) {
+          // h stays in registers: its sign bits go to the mask, its sum over the warp's 32 pixels (halo pixels count as
+          // zero) to the pooling partials.  The 16 channel sums are formed by a reduce-scatter over the lanes: each step
+          // halves the channels a lane carries and doubles the pixels its sums cover (16 shuffles for 16 channels); the
+          // lane pair (2j, 2j+1) ends with the sum of channel j's bit pattern below.
+          const int c0 = q * 16;
+          float ov[16];
+          uint32_t bits = 0;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+            ov[2 * e] = valid ? lo : 0.f;
+            ov[2 * e + 1] = valid ? hi : 0.f;
+            bits |= (lo > 0.f ? 1u : 0u) << (2 * e);
+            bits |= (hi > 0.f ? 1u : 0u) << (2 * e + 1);
+          }
+          if (valid && c0 < p.Cout) {
+            uint8_t* mdst = p.mask + ((((size_t)n * p.H + h0 + hh) * p.W + w0 + we - 1) * (size_t)(p.Cout >> 3)) + (c0 >> 3);
+            mdst[0] = (uint8_t)(bits & 0xffu);
+            if (c0 + 8 < p.Cout) mdst[1] = (uint8_t)(bits >> 8);
+          }
+          float r8[8], r4[4], r2[2];
+          const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4, b1 = lane & 2;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float send = b4 ? ov[i] : ov[8 + i], keep = b4 ? ov[8 + i] : ov[i];
+            r8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float send = b3 ? r8[i] : r8[4 + i], keep = b3 ? r8[4 + i] : r8[i];
+            r4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+          }
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const float send = b2 ? r4[i] : r4[2 + i], keep = b2 ? r4[2 + i] : r4[i];
+            r2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+          }
+          float r1 = (b1 ? r2[1] : r2[0]) + __shfl_xor_sync(0xffffffffu, b1 ? r2[0] : r2[1], 2);
+          r1 += __shfl_xor_sync(0xffffffffu, r1, 1);
+          const int ch = c0 + (b4 ? 8 : 0) + (b3 ? 4 : 0) + (b2 ? 2 : 0) + (b1 ? 1 : 0);
+          if ((lane & 1) == 0 && ch < p.Cout) p.pool_part[((size_t)t * 4 + lg) * p.Cout + ch] = r1;
         } else {
           const int c0 = q * 16;             // Cout is a multiple of 8 here
           if (valid && c0 < p.Cout) {
@@ -1350,12 +1397,20 @@ int make_map4(CUtensorMap* m, const void* base, const uint64_t dims[4], const ui
   return r == CUDA_SUCCESS ? NF_OK : nf_cuda_check(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
 }
 
+// Per-process caches (kernel attributes, SM count, symbol addresses) are kept per device: a process may use several.
+constexpr int kMaxDevices = 64;
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+  return dev;
+}
+
 int sm_count() {
-  static int n = 0;
+  static int n_dev[kMaxDevices];
+  const int dev = current_device();
+  int& n = n_dev[dev];
   if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
-      n = 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
   }
   return n;
 }
@@ -1416,7 +1471,8 @@ TcPlan plan_fwd(int H, int W, int Cin, int Cout, int N, int epi = 0, int stride 
 
 template <int BN, int EPI, int KC = 64, int BMN = 0, int PT = 0, int RW = 0>
 int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const FwdParams& p) {
-  static bool attr_done = false;
+  static bool attr_done_dev[kMaxDevices];  // function attributes belong to a device's context: set once per device
+  bool& attr_done = attr_done_dev[current_device()];
   if (!attr_done) {
     NF_CUDA(cudaFuncSetAttribute(conv_fwd_tc_kernel<BN, EPI, KC, BMN, PT, RW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
@@ -1447,7 +1503,8 @@ bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride, int stats = 0
 template <int G, int EPI, int KC = 64, int MIR = 0, int UF = 0, int XF = 0>
 int launch_fold(int grid, size_t smem, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& my, const CUtensorMap& my2,
                 const FoldParams& p) {
-  static bool attr_done = false;
+  static bool attr_done_dev[kMaxDevices];  // function attributes belong to a device's context: set once per device
+  bool& attr_done = attr_done_dev[current_device()];
   if (!attr_done) {
     NF_CUDA(cudaFuncSetAttribute(conv_fwd_fold_kernel<G, EPI, KC, MIR, UF, XF>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
@@ -1467,6 +1524,8 @@ struct BnBwdIn {
 struct XfIn {
   const float *scale, *shift;
   void* a;
+  float* pool_part;  // non-null: pooling partials and sign mask instead of h (see FoldParams)
+  uint8_t* mask;
 };
 
 int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* w, void* y, int stats, float* red,
@@ -1524,6 +1583,7 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   if (xf) {
     if (epi != 1) return NF_EINVAL;
     p.xf_scale = xf->scale; p.xf_shift = xf->shift; p.xf_a = (bf16*)xf->a;
+    p.pool_part = xf->pool_part; p.mask = xf->mask;
     return G == 16 ? launch_fold<16, 1, 64, 0, 0, 1>(grid, smem, mx, mw, my, my2, p)
                    : G == 32 ? launch_fold<32, 1, 64, 0, 0, 1>(grid, smem, mx, mw, my, my2, p)
                              : launch_fold<64, 1, 64, 0, 0, 1>(grid, smem, mx, mw, my, my2, p);
@@ -1664,7 +1724,8 @@ WgPlan plan_wgrad(int H, int W, int Cin, int Cout, int N, int aux = 0, int strid
 
 template <int NB>
 int launch_wgrad_kw(const WgPlan& pl, const CUtensorMap& mx, const CUtensorMap& mg, const WgParams& p) {
-  static bool attr_done = false;
+  static bool attr_done_dev[kMaxDevices];  // function attributes belong to a device's context: set once per device
+  bool& attr_done = attr_done_dev[current_device()];
   if (!attr_done) {
     NF_CUDA(cudaFuncSetAttribute(conv_wgrad_kw_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
@@ -1676,7 +1737,8 @@ int launch_wgrad_kw(const WgPlan& pl, const CUtensorMap& mx, const CUtensorMap& 
 
 template <int NB>
 int launch_wgrad_gx(const WgPlan& pl, const CUtensorMap& mx, const CUtensorMap& mg, const WgParams& p) {
-  static bool attr_done = false;
+  static bool attr_done_dev[kMaxDevices];  // function attributes belong to a device's context: set once per device
+  bool& attr_done = attr_done_dev[current_device()];
   if (!attr_done) {
     NF_CUDA(cudaFuncSetAttribute(conv_wgrad_gx_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
@@ -1688,7 +1750,8 @@ int launch_wgrad_gx(const WgPlan& pl, const CUtensorMap& mx, const CUtensorMap& 
 
 template <int NB, int S2 = 0>
 int launch_wgrad(const WgPlan& pl, const CUtensorMap& mx, const CUtensorMap& mg, const WgParams& p) {
-  static bool attr_done = false;
+  static bool attr_done_dev[kMaxDevices];  // function attributes belong to a device's context: set once per device
+  bool& attr_done = attr_done_dev[current_device()];
   if (!attr_done) {
     NF_CUDA(cudaFuncSetAttribute(conv_wgrad_tc_kernel<NB, S2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     attr_done = true;
@@ -1795,10 +1858,23 @@ bool nf_tc_bn_aux_fused(const nf_layer* L) {
   return L->fam[2] && !wide_aux(L) && !L->o.maxpool && fold_ok(L->Ha, L->Wa, L->Cout, L->F, 1, 1);
 }
 
+// The fused aux forward can also keep h out of memory when the head pools by averaging and no tile straddles a pooling
+// quadrant (14 x 8-pixel tiles: Ha/2 a multiple of 8, Wa/2 of 14): the epilogue then emits pooling partials and a sign mask.
+bool nf_tc_aux_pool_fused(const nf_layer* L) {
+  return nf_tc_bn_aux_fused(L) && L->o.aux_pool == NF_POOL_AVG && (L->Ha / 2) % 8 == 0 && (L->Wa / 2) % 14 == 0 && L->Ha % 2 == 0 &&
+         L->Wa % 2 == 0;
+}
+
+size_t nf_tc_pool_part_floats(const nf_layer* L) {
+  return (size_t)L->o.N * (L->Wa / 14) * (L->Ha / 8) * 4 * L->F;
+}
+
 int nf_tc_bn_aux_fwd(nf_layer* L, void* act_out) {
   if (!nf_tc_bn_aux_fused(L) || L->skip) return NF_EUNSUPPORTED;
   int nb = 0;
-  const XfIn xf{L->scale, L->shift, act_out};
+  const bool pooled = nf_tc_aux_pool_fused(L);
+  // the partials live in the split-K scratch (free until the weight gradients), the mask in the unused h buffer
+  const XfIn xf{L->scale, L->shift, act_out, pooled ? L->wpart : nullptr, pooled ? (uint8_t*)L->h : nullptr};
   return run_fold(L->o.N, L->Ha, L->Wa, L->Cout, L->F, L->y, L->shadow + L->off[NF_P_WA], L->h, 0, nullptr, 0, L->status, &nb, 1,
                   L->val + L->off[NF_P_BA], nullptr, &xf);
 }
@@ -1814,7 +1890,7 @@ int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb) {
   const bool wide = wide_aux(L);
   const void* w = L->shadow + L->off[NF_P_WA];
   if (wide) {
-    const int rc = nf_ref_flip_weights(L->shadow + L->off[NF_P_WA], L->F, L->Cout, L->wa_t);
+    const int rc = nf_k_flip_weights(L->shadow + L->off[NF_P_WA], L->F, L->Cout, L->wa_t);
     if (rc != NF_OK) return rc;
     w = L->wa_t;
   }
@@ -1847,20 +1923,58 @@ size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout
   return pl.ok ? pl.part_floats : 0;
 }
 
-static __device__ int32_t g_op_status;  // status word of the stand-alone operations
+static __device__ int32_t g_op_status;  // status word of the stand-alone operations (one per device that loads the library)
+
+int nf_tc_op_status_ptr(int32_t** out) {
+  static int32_t* st_dev[kMaxDevices];
+  int32_t*& st = st_dev[current_device()];
+  if (!st) NF_CUDA(cudaGetSymbolAddress((void**)&st, g_op_status));
+  *out = st;
+  return NF_OK;
+}
 
 int nf_tc_conv3x3_forward(const void* x, const void* w, int N, int H, int W, int Cin, int Cout, int stride, void* y) {
-  static int32_t* st = nullptr;
-  if (!st) NF_CUDA(cudaGetSymbolAddress((void**)&st, g_op_status));
+  int32_t* st = nullptr;
+  if (nf_tc_op_status_ptr(&st) != NF_OK) return NF_ECUDA;
   int nb = 0;
   return run_fwd(N, H, W, Cin, Cout, x, w, y, 0, nullptr, 0, st, &nb, 0, nullptr, stride);
 }
 
 int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int Cin, int Cout, int stride, float* part,
                         size_t part_floats, float* dw) {
-  static int32_t* st = nullptr;
-  if (!st) NF_CUDA(cudaGetSymbolAddress((void**)&st, g_op_status));
+  int32_t* st = nullptr;
+  if (nf_tc_op_status_ptr(&st) != NF_OK) return NF_ECUDA;
   return run_wgrad(N, H, W, Cin, Cout, x, g, part, part_floats, dw, st, 0, stride);
+}
+
+// One CTA of one warp waits, with the bounded wait every tensor-core kernel uses, on a barrier that nobody ever
+// arrives at, and then leaves the way those kernels do: abort flag set by the waiter, NF_ETIMEOUT raised in the status
+// word, waited time reported.  No TMA, no tensor memory, nothing else in flight.
+__global__ void bounded_wait_probe_kernel(unsigned long long limit_ns, int32_t* status, unsigned long long* waited_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  const unsigned long long t0 = ptx::globaltimer();
+  const bool done = __all_sync(0xffffffffu, ptx::mbar_wait(&bar, 0, &abort_flag, limit_ns));
+  const unsigned long long t1 = ptx::globaltimer();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (!done && abort_flag) atomicOr(status, NF_ETIMEOUT);
+    *waited_ns = t1 - t0;
+  }
+}
+
+int nf_tc_bounded_wait_probe(unsigned long long limit_ns, unsigned long long* waited_ns_dev) {
+  int32_t* st = nullptr;
+  if (nf_tc_op_status_ptr(&st) != NF_OK) return NF_ECUDA;
+  bounded_wait_probe_kernel<<<1, 32, 0, g_nf_stream>>>(limit_ns, st, waited_ns_dev);
+  NF_LAUNCHED();
+  return NF_OK;
 }
 
 int nf_tc_op_status(int32_t* out) {

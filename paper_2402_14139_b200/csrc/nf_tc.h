@@ -18,6 +18,8 @@ size_t nf_tc_red_floats(const nf_layer* L);
 // status word (nf_device_flag bits) of the stand-alone operations.
 int nf_tc_conv3x3_forward(const void* x, const void* w, int N, int H, int W, int Cin, int Cout, int stride, void* y);
 int nf_tc_op_status(int32_t* out);
+// Device address of that status word on the current device (looked up once per device).
+int nf_tc_op_status_ptr(int32_t** out);
 // Stand-alone weight gradient on the tensor-core path and the split-K scratch (floats) it needs (0: shape not covered).
 size_t nf_tc_conv3x3_wgrad_scratch_floats(int N, int H, int W, int Cin, int Cout, int stride);
 int nf_tc_conv3x3_wgrad(const void* x, const void* g, int N, int H, int W, int Cin, int Cout, int stride, float* part,
@@ -28,6 +30,11 @@ int nf_tc_aux_fwd(nf_layer* L, const void* a, int count);
 // L->h = ReLU(conv(act_out, Wa) + ba), both in bf16.  NF_EUNSUPPORTED (nothing launched) when the layer's shape is not
 // covered or it has a shortcut; nf_tc_bn_aux_fused tells whether the shape is covered.
 bool nf_tc_bn_aux_fused(const nf_layer* L);
+// Whether that kernel also replaces h by pooling partials (L->wpart: [tile][4][F], tiles of 14 x 8 pixels in row-major order
+// per image) and a sign mask (in L->h: one bit per element, [N][Ha][Wa][F/8] bytes); nf_tc_pool_part_floats is the size of
+// the partials (the workspace plan reserves it in the split-K scratch).
+bool nf_tc_aux_pool_fused(const nf_layer* L);
+size_t nf_tc_pool_part_floats(const nf_layer* L);
 int nf_tc_bn_aux_fwd(nf_layer* L, void* act_out);
 // Aux conv weight gradient on tensor cores: grad(Wa) = wgrad(a, L->dh).
 int nf_tc_aux_wgrad(nf_layer* L, const void* a);
@@ -35,3 +42,6 @@ int nf_tc_aux_wgrad(nf_layer* L, const void* a);
 // the BatchNorm-backward sums (no pool, folded-tap shape) it leaves *bn_nb > 0 partial blocks in L->red
 // ([block][2][Cout]: sum dz, sum dz*xhat); otherwise *bn_nb = 0.
 int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb);
+// Self-check of the bounded wait: one small CTA waits limit_ns on a barrier nobody arrives at; *waited_ns_dev (device)
+// receives the time it waited and NF_ETIMEOUT is raised in the stand-alone status word.
+int nf_tc_bounded_wait_probe(unsigned long long limit_ns, unsigned long long* waited_ns_dev);

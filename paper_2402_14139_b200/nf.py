@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SO = os.path.join(_HERE, "libnf.so")
 
 NF_OK, NF_EINVAL, NF_EALIGN, NF_ENOWS, NF_EUNSUPPORTED, NF_ECUDA = 0, -1, -2, -3, -4, -5
-NF_ELABEL, NF_ENONFINITE, NF_ETIMEOUT = 1, 2, 4
+NF_ELABEL, NF_ENONFINITE, NF_ETIMEOUT, NF_EINDEX = 1, 2, 4, 8
 NF_F32, NF_BF16 = 0, 1
 NF_LOSS_CE, NF_LOSS_MSE = 0, 1
 NF_POOL_AVG, NF_POOL_MAX = 0, 1
@@ -27,8 +27,8 @@ PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P
 EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_layer_workspace_bytes",
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
-           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_max_batch", "nf_layer_step_dp", "nf_layer_dp_buffer", "nf_layer_set_skip", "nf_block_step", "nf_block_step_host", "nf_block_step_host_next", "nf_trace_enable", "nf_trace_read",
-           "nf_cache_gather", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_op_status", "nf_partition", "nf_set_stream", "nf_launch_count",
+           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_fit_line", "nf_max_batch", "nf_layer_step_dp", "nf_layer_dp_buffer", "nf_layer_set_skip", "nf_layer_stored_tensor", "nf_block_step", "nf_block_step_host", "nf_block_step_host_next", "nf_trace_enable", "nf_trace_read",
+           "nf_cache_gather", "nf_selftest_bounded_wait", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_op_status", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
 
@@ -77,11 +77,13 @@ def lib():
         L.nf_layer_param_count.argtypes = [vp, C.c_int]
         L.nf_count_equal.argtypes = [ip, ip, C.c_longlong, vp]
         L.nf_layer_set_skip.argtypes = [vp, vp]
+        L.nf_layer_stored_tensor.argtypes = [vp, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
         L.nf_layer_step_dp.argtypes = [vp, C.c_int, vp, ip, C.c_float, fp, vp, C.c_int]
         L.nf_layer_dp_buffer.argtypes = [vp, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
         L.nf_aan_filters.argtypes = [C.POINTER(C.c_int), C.c_int, C.c_int, C.POINTER(C.c_int)]
         L.nf_profile_layer.argtypes = [C.c_int] * 6 + [C.POINTER(nf_layer_opts), C.POINTER(C.c_int), C.c_int, C.POINTER(C.c_double),
                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.nf_fit_line.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.nf_max_batch.restype = C.c_longlong
         L.nf_max_batch.argtypes = [C.c_double, C.c_double, C.c_double]
         L.nf_select_exit.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.c_int]
@@ -90,12 +92,13 @@ def lib():
         L.nf_block_step_host_next.argtypes = [vp, vp, ip, C.c_float, fp, vp, vp, ip]
         L.nf_trace_enable.argtypes = [C.c_int]
         L.nf_trace_read.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
-        L.nf_cache_gather.argtypes = [vp, ip, ip, C.c_int, C.c_size_t, vp, ip]
+        L.nf_cache_gather.argtypes = [vp, ip, C.c_int, ip, C.c_int, C.c_size_t, vp, ip]
         L.nf_conv3x3_forward.argtypes = [C.c_int, vp, vp] + [C.c_int] * 6 + [vp]
         L.nf_conv3x3_wgrad_scratch_bytes.restype = C.c_size_t
         L.nf_conv3x3_wgrad_scratch_bytes.argtypes = [C.c_int] * 6
         L.nf_conv3x3_wgrad.argtypes = [C.c_int, vp, vp] + [C.c_int] * 6 + [vp, C.c_size_t, vp]
         L.nf_conv3x3_wgrad_static.argtypes = [C.c_int, vp, vp] + [C.c_int] * 6 + [vp]
+        L.nf_selftest_bounded_wait.argtypes = [C.c_ulonglong, vp]
         L.nf_partition.argtypes = [C.POINTER(C.c_int), C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int),
                                    C.POINTER(C.c_int)]
         L.nf_set_stream.argtypes = [vp]
@@ -196,6 +199,16 @@ def nf_profile_layer(Cin, Cout, H, W, F, classes, batches, stride=1, maxpool=Fal
     return list(by), sl.value, ic.value
 
 
+def nf_fit_line(batches, bytes_):
+    """Least-squares line bytes = intercept + slope * batch through measured pairs: (slope, intercept)."""
+    k = len(batches)
+    x = (C.c_double * k)(*[float(v) for v in batches])
+    y = (C.c_double * k)(*[float(v) for v in bytes_])
+    sl, ic = C.c_double(), C.c_double()
+    _check(lib().nf_fit_line(x, y, k, C.byref(sl), C.byref(ic)), "nf_fit_line")
+    return sl.value, ic.value
+
+
 def nf_max_batch(slope, intercept, budget_bytes) -> int:
     return int(lib().nf_max_batch(float(slope), float(intercept), float(budget_bytes)))
 
@@ -268,6 +281,24 @@ class Layer:
                f"nf_layer_get_param({name})")
         return a
 
+    STATE = ("W", "gamma", "beta", "Wa", "ba", "Wf", "bf")
+
+    def export_state(self):
+        """Everything that defines the trained layer, as host arrays: the seven parameter tensors, their momentum buffers
+        (keys "v" + name) and the running statistics.  With it a finished layer can leave the device (the paper keeps only
+        the active block in GPU memory) and be rebuilt later by import_state."""
+        st = {k: self.get_param(k) for k in self.STATE}
+        st.update({"v" + k: self.get_param(k, NF_K_MOMENTUM) for k in self.STATE})
+        st.update(rmean=self.get_param("rmean"), rvar=self.get_param("rvar"))
+        return st
+
+    def import_state(self, st):
+        for k in self.STATE:
+            self.set_param(k, st[k])
+            self.set_param(k, st["v" + k], kind=NF_K_MOMENTUM)
+        self.set_param("rmean", st["rmean"])
+        self.set_param("rvar", st["rvar"])
+
     def new_act(self):
         return self._torch.empty((self.N, self.Ha, self.Wa, self.Cout), dtype=self.tdtype, device=self.device)
 
@@ -291,6 +322,24 @@ class Layer:
         """nf_layer_set_skip: identity shortcut [N, Ho, Wo, Cout] added before the ReLU in later calls (None removes it)."""
         self._skip = skip       # keeps the tensor alive
         _check(lib().nf_layer_set_skip(self.h, _ptr(skip)), "nf_layer_set_skip")
+
+    STORED = dict(y=0, dy=1, h=2, dh=3, da=4, p=5, dp=6, logits=7, hmask=8)
+
+    def stored(self, name):
+        """nf_layer_stored_tensor as a tensor view of the workspace: y, dy [N,Ho,Wo,Cout]; h, dh [N,Ha,Wa,Fp]; da [N,Ha,Wa,Cout]
+        (layer dtype; Fp = F rounded up to a multiple of 8); p, dp [N,4*Fp]; logits [N,classes] (float32)."""
+        ptr, nbytes = C.c_void_p(), C.c_size_t()
+        _check(lib().nf_layer_stored_tensor(self.h, self.STORED[name], C.byref(ptr), C.byref(nbytes)), "nf_layer_stored_tensor")
+        off = ptr.value - self.ws.data_ptr()
+        raw = self.ws[off:off + nbytes.value]
+        Fp = (self.F + 7) // 8 * 8
+        if name in ("p", "dp", "logits"):
+            return raw.view(self._torch.float32).view(self.N, -1)
+        if name == "hmask":     # uint8 [N, Ha, Wa, Fp/8]: bit f%8 of byte f/8 is set where h > 0
+            return raw.view(self.N, self.Ha, self.Wa, Fp // 8)
+        shape = dict(y=(self.N, self.Ho, self.Wo, self.Cout), dy=(self.N, self.Ho, self.Wo, self.Cout), h=(self.N, self.Ha, self.Wa, Fp),
+                     dh=(self.N, self.Ha, self.Wa, Fp), da=(self.N, self.Ha, self.Wa, self.Cout))[name]
+        return raw.view(self.tdtype).view(shape)
 
     def dp_buffer(self, which):
         """The exchange buffer `which` of the data-parallel step as a tensor view of the workspace (float64 for 0 and 1, float32 for 2)."""
@@ -317,7 +366,8 @@ class Layer:
 
     def kernel_family(self, op: int) -> str:
         """op 0-3: "tcgen05" or "cuda-core" for main forward, main weight gradient, aux forward, aux backward;
-        op 4: "fused" when BatchNorm + ReLU run inside the aux forward kernel, else "separate"."""
+        op 4: "fused" when BatchNorm + ReLU run inside the aux forward kernel, else "separate";
+        op 5: "mask" when that kernel pools h in its epilogue and keeps only its sign bits, else "stored"."""
         return lib().nf_layer_kernel_family(self.h, op).decode()
 
 
@@ -376,10 +426,11 @@ class Block:
 
 
 def nf_cache_gather(cache, cache_labels, idx, out, out_labels):
-    """out[i] = cache[idx[i]] (rows) and labels likewise; device tensors, idx int32."""
+    """out[i] = cache[idx[i]] (rows) and labels likewise; device tensors, idx int32.  An index outside the cache's rows
+    yields a zero row, label -1 and NF_EINDEX in nf_op_status()."""
     row_bytes = cache[0].numel() * cache.element_size()
-    _check(lib().nf_cache_gather(_ptr(cache), _ptr(cache_labels), _ptr(idx), int(idx.numel()), row_bytes, _ptr(out),
-                                 _ptr(out_labels)), "nf_cache_gather")
+    _check(lib().nf_cache_gather(_ptr(cache), _ptr(cache_labels), int(cache.shape[0]), _ptr(idx), int(idx.numel()), row_bytes,
+                                 _ptr(out), _ptr(out_labels)), "nf_cache_gather")
 
 
 def nf_conv3x3_forward(dtype, x, w, stride, y):
@@ -411,6 +462,11 @@ def nf_conv3x3_wgrad_static(dtype, x, g, stride, dw):
     N, H, W, Cin = x.shape
     _check(lib().nf_conv3x3_wgrad_static(dtype, _ptr(x), _ptr(g), N, H, W, Cin, g.shape[3], stride, _ptr(dw)),
            "nf_conv3x3_wgrad_static")
+
+
+def nf_selftest_bounded_wait(limit_ns: int, waited_ns_out):
+    """One small CTA waits limit_ns on a barrier nobody arrives at and gives up; waited_ns_out: device int64[1]."""
+    _check(lib().nf_selftest_bounded_wait(int(limit_ns), _ptr(waited_ns_out)), "nf_selftest_bounded_wait")
 
 
 def nf_op_status() -> int:

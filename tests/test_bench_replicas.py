@@ -57,6 +57,39 @@ def test_reference_arm_prints_one_json_line_with_the_required_keys():
     assert d["unit"] == "images/s" and d["higher_is_better"] is True and d["value"] > 0
 
 
+def test_gpus_flag_starts_one_process_per_rank_when_no_launcher_did():
+    """`python bench.py --gpus 2 ...` without torchrun: the script starts two ranks itself; with the reference arm rank 0
+    alone prints the line (n_gpus 2) and the other rank exits 0 without work."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--workload", "c2",
+                          "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=600, cwd=ROOT, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    assert json.loads(lines[0])["n_gpus"] == 2
+
+
+def test_spawned_ranks_get_the_launcher_environment(tmp_path):
+    """spawn_ranks hands every child RANK, LOCAL_RANK, WORLD_SIZE and a loop-back rendezvous address."""
+    sys.path.insert(0, ROOT)
+    import bench
+    import subprocess
+    script = tmp_path / "echo_env.py"
+    script.write_text("import os, sys\n"
+                      "open(sys.argv[1] + os.environ['RANK'], 'w').write(' '.join(os.environ[k] for k in "
+                      "('RANK', 'LOCAL_RANK', 'WORLD_SIZE', 'MASTER_ADDR')) + ' ' + str(int(os.environ['MASTER_PORT']) > 0))\n")
+    real = bench.__file__
+    try:
+        bench.__file__ = str(script)
+        assert bench.spawn_ranks(3, [str(tmp_path / "r")]) == 0
+    finally:
+        bench.__file__ = real
+    for r in range(3):
+        assert (tmp_path / f"r{r}").read_text() == f"{r} {r} 3 127.0.0.1 True"
+
+
 def _dp_worker(rank, world, port, q):
     """A stand-in layer whose phases only write rank-dependent numbers into the exchange buffers: what is checked is
     the schedule (which buffer is summed after which phase, the loss with the gradients, nothing after the update)."""

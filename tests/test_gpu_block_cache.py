@@ -112,6 +112,31 @@ def test_cache_gather_is_bit_exact(env):
         nf.nf_cache_gather(cache, labels, idx, out, None)      # labels in without labels out
 
 
+def test_cache_gather_skips_indices_outside_the_cache(env):
+    """A stale or corrupt permutation entry (negative, or beyond the cache's rows) must not become an out-of-bounds read:
+    the kernel checks every index, zero-fills that output row, sets its label to -1 and raises NF_EINDEX; the rows with
+    valid indices are still copied bit for bit."""
+    nf, torch = env
+    K, row = 40, (2, 2, 16)
+    cache = torch.from_numpy(synth.to_bf16_bits(synth.normal(4, 1, (K,) + row)).view(np.int16)).cuda().view(torch.bfloat16)
+    labels = torch.from_numpy(synth.labels(4, 2, K, 10)).cuda()
+    idx_h = np.array([3, -1, 39, 40, 7, 2 ** 31 - 1, -2 ** 31, 0], dtype=np.int32)
+    idx = torch.from_numpy(idx_h).cuda()
+    out = torch.full((len(idx_h),) + row, 7.0, dtype=torch.bfloat16, device="cuda")
+    out_l = torch.full((len(idx_h),), 123, dtype=torch.int32, device="cuda")
+    assert nf.nf_op_status() == 0
+    nf.nf_cache_gather(cache, labels, idx, out, out_l)
+    torch.cuda.synchronize()
+    good = (idx_h >= 0) & (idx_h < K)
+    gi = torch.from_numpy(np.nonzero(good)[0]).cuda()
+    bi = torch.from_numpy(np.nonzero(~good)[0]).cuda()
+    assert torch.equal(out[gi].view(torch.int16), cache[idx[gi].long()].view(torch.int16))
+    assert torch.equal(out_l[gi], labels[idx[gi].long()])
+    assert int(out[bi].view(torch.int16).abs().max()) == 0 and bool((out_l[bi] == -1).all())
+    assert nf.nf_op_status() == nf.NF_EINDEX
+    assert nf.nf_op_status() == 0                                 # reading clears the word
+
+
 def test_prefetching_host_step_equals_plain_host_step():
     """A stream of different batches through nf_block_step_host_next (the next batch copied while this one trains)
     gives bit-identical losses and parameters to the plain host step; a call whose batch was not announced falls

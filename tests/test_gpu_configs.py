@@ -21,30 +21,11 @@ def env():
     return nf, torch
 
 
-def _cfg(l, N, classes):
-    return dict(N=N, Cin=l["Cin"], Cout=l["Cout"], H=l["H"], W=l["W"], F=l["F"], classes=classes, stride=l["stride"],
-                pool=l["pool"])
+_cfg = pu.layer_cfg
 
 
 def _step_both(nf, torch, c, P, x, y, lr=0.01):
-    """One step on both sides from the same state; returns (worst errors, checker's act_out, layers)."""
-    O = pu.oracle_layer(c, P, store_bf16=True)
-    G = pu.gpu_layer(nf, c, P, nf.NF_BF16)
-    xd = pu.to_device_nhwc(torch, x, 1)
-    loss_d = torch.zeros(1, device="cuda")
-    act_d = G.new_act()
-    loss_o, act_o, tr = O.step(x, y, lr, update=True, grads=True)
-    G.step(xd, torch.from_numpy(y).cuda(), lr, loss_d, act_d)
-    torch.cuda.synchronize()
-    assert G.status() == 0
-    tol = pu.TOL[1]
-    errs = dict(loss=abs(float(loss_d.item()) - loss_o) / abs(loss_o), act=pu.max_err(pu.from_device_nhwc(act_d), act_o))
-    for k in pu.PNAMES:
-        errs["g" + k] = pu.max_err(G.get_param(k, nf.NF_K_GRAD), tr["g" + k])
-        errs["p" + k] = pu.max_err(G.get_param(k), O.p[k])
-    assert errs["loss"] <= tol["loss"], errs
-    assert max(v for k, v in errs.items() if k != "loss") <= tol["t"], errs
-    return errs, act_o, O, G
+    return pu.step_both(nf, torch, c, P, x, y, lr)
 
 
 def test_c2_vgg_block_full_batch_chain(env):
@@ -62,26 +43,62 @@ def test_c2_vgg_block_full_batch_chain(env):
         G.close()
 
 
-C3_PICKS = [(0, 0), (0, 1), (1, 0), (2, 0), (3, 3)]   # (block, layer in block): stem, 64->64, two stride-2 layers, 512->512
-
-
-@pytest.mark.parametrize("pick", range(len(C3_PICKS)))
-def test_c3_resnet_shaped_layers_at_block_batch_size(env, pick):
+def test_c2_block_against_unrounded_fp64_checker(env):
+    """What the bf16 storage costs on the VGG block at its full batch of 128: the same chain against the checker in
+    pure fp64 (store_bf16 off), with the bounds parity_util.UNROUNDED_TOL derives from the arithmetic."""
     nf, torch = env
+    wl = workloads.c2()
+    N, ls = wl["blocks"][0]
+    x = synth.round_bf16(synth.normal(0x4E460002, 8, (N, 3, 32, 32))).astype(np.float64)
+    y = synth.labels(0x4E460002, 9, N, wl["classes"])
+    for li, l in enumerate(ls):
+        c = _cfg(l, N, wl["classes"])
+        P, _, _ = pu.seeded_case(dict(c, N=1), 0x4E460200 + li, bf16=True)
+        errs, act_o, O, G = pu.step_both(nf, torch, c, P, x, y, store_bf16=False, tol=pu.UNROUNDED_TOL)
+        assert errs["act"] <= pu.UNROUNDED_TOL["act"], errs
+        print(f"c2 layer {li} vs unrounded fp64:", {k: f"{v:.2e}" for k, v in errs.items()})
+        G.close()
+        x = synth.round_bf16(act_o).astype(np.float64)
+
+
+def _c3_layers():
     wl = workloads.c3()
-    b, li = C3_PICKS[pick]
-    N, ls = wl["blocks"][b]
-    l = ls[li]
-    c = _cfg(l, N, wl["classes"])
-    seed = 0x4E460300 + 16 * b + li
+    return [(b, li, N, l) for b, (N, ls) in enumerate(wl["blocks"]) for li, l in enumerate(ls)]
+
+
+def _one_layer(nf, torch, l, N, classes, seed):
+    c = _cfg(l, N, classes)
     P, _, _ = pu.seeded_case(dict(c, N=1), seed, bf16=True)
     x = synth.normal(seed, 8, (N, l["Cin"], l["H"], l["W"]))
     if l["Cin"] != 3:
         x = np.maximum(x, 0.0)                              # deeper layers see post-ReLU activations
     x = synth.round_bf16(x).astype(np.float64)
-    y = synth.labels(seed, 9, N, wl["classes"])
-    _, _, _, G = _step_both(nf, torch, c, P, x, y)
+    y = synth.labels(seed, 9, N, classes)
+    errs, _, _, G = _step_both(nf, torch, c, P, x, y)
     G.close()
+    return errs
+
+
+@pytest.mark.parametrize("k", range(17))
+def test_c3_every_layer_at_its_block_batch_size(env, k):
+    """All 17 layers of the ResNet-18-shaped stack, each at the batch size of its block (64 / 128 / 256 / 512)."""
+    nf, torch = env
+    b, li, N, l = _c3_layers()[k]
+    errs = _one_layer(nf, torch, l, N, workloads.c3()["classes"], 0x4E460300 + 16 * b + li)
+    print(f"c3 block {b} layer {li} N={N}:", {k2: f"{v:.2e}" for k2, v in errs.items()})
+
+
+# batch sizes for the 13 layer shapes of the VGG-16 workload: the block batch sizes (1260 ... 8602) are cut to what the
+# checker steps in a few seconds, more samples where the maps are small so that several tensor-core tiles are covered
+C5_BATCH = [8, 8, 12, 12, 24, 24, 24, 48, 48, 48, 160, 160, 160]
+
+
+@pytest.mark.parametrize("k", range(13))
+def test_c5_every_layer_shape(env, k):
+    nf, torch = env
+    wl = workloads.c5()
+    errs = _one_layer(nf, torch, wl["layers"][k], C5_BATCH[k], wl["classes"], 0x4E460540 + k)
+    print(f"c5 layer {k} N={C5_BATCH[k]}:", {k2: f"{v:.2e}" for k2, v in errs.items()})
 
 
 def test_c5_partition_train_cache_rebatch_next_block(env):

@@ -74,3 +74,23 @@ def test_conv_forward_and_wgrad(env, si, dtype):
     assert pu.max_err(dw.cpu().numpy(), ref) <= tol
     with pytest.raises(nf.NfError):
         nf.nf_conv3x3_wgrad(dtype, xd, gd, s, scratch[:16], dw)     # scratch too small
+
+
+def test_bounded_wait_runs_out_and_reports_a_timeout(env):
+    """The wait routine of the tensor-core kernels, in isolation: one small CTA waits on a barrier that nobody arrives at,
+    with a 1 ms limit.  It must give up by itself (the call returns, the context stays usable), report about the limit as
+    the time waited, and raise NF_ETIMEOUT in the status word; a kernel launched afterwards runs normally."""
+    nf, torch = env
+    assert nf.nf_op_status() == 0
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    nf.nf_selftest_bounded_wait(1_000_000, waited)
+    torch.cuda.synchronize()
+    assert nf.nf_op_status() == nf.NF_ETIMEOUT
+    assert nf.nf_op_status() == 0
+    assert 1_000_000 <= int(waited.item()) < 100_000_000
+    x = torch.ones(1024, device="cuda")
+    assert float((x * 2).sum().item()) == 2048.0              # the device still answers
+    with pytest.raises(nf.NfError):
+        nf.nf_selftest_bounded_wait(0, waited)
+    with pytest.raises(nf.NfError):
+        nf.nf_selftest_bounded_wait(2_000_000_000, waited)    # limits above one second are refused

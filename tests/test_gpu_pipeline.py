@@ -86,3 +86,69 @@ def test_host_cache_tier_gives_identical_results():
         assert [b["losses"] for b in r] == [b["losses"] for b in r0]
         assert torch.equal(out.cuda().view(torch.int16), out0.view(torch.int16))
     nf.nf_set_stream(None)
+
+
+def test_disk_cache_tier_and_offloaded_blocks_give_identical_results(tmp_path):
+    """The storage tier beyond host memory: the activation cache as a memory-mapped file (rows read back by a reader
+    thread while the previous batch trains) and finished blocks written out as .npz files.  Storage only: losses and the
+    final cache are bit-identical to the run that keeps everything on the device, and a block reloaded from its file
+    reproduces its cached output bit for bit."""
+    import torch
+    from paper_2402_14139_b200 import nf
+    nf.lib()
+    nf.nf_set_stream(None)
+    K = 24
+    x = synth.round_bf16(synth.normal(6, 1, (K, 16, 16, 3)))
+    data = torch.from_numpy(x).cuda().to(torch.bfloat16)
+    labels = torch.from_numpy(synth.labels(6, 2, K, 4)).cuda()
+    r0, out0 = pipeline.train_blockwise(nf, torch, _wl(), data, labels, epochs=3, lr=0.05, seed=3, offload="host")
+    r1, out1 = pipeline.train_blockwise(nf, torch, _wl(), data, labels, epochs=3, lr=0.05, seed=3, cache="disk", spill_dir=str(tmp_path),
+                                        offload=str(tmp_path))
+    assert isinstance(out1, np.memmap) and (tmp_path / "cache_block0.npy").exists() and (tmp_path / "cache_block1.npy").exists()
+    assert [b["losses"] for b in r1] == [b["losses"] for b in r0]
+    assert np.array_equal(np.asarray(out1), out0.view(torch.int16).cpu().numpy())
+    # a finished block comes back from its file (and from the host copy) and reproduces the cache it left behind
+    for state in (r1[0]["state"], r0[0]["state"]):
+        layers, block = pipeline.load_block(nf, _wl(), 0, state)
+        again = torch.empty((6, 8, 8, 64), dtype=torch.bfloat16, device="cuda")
+        block.cache(data[:6].contiguous(), again)
+        torch.cuda.synchronize()
+        cache0 = np.load(tmp_path / "cache_block0.npy", mmap_mode="r")
+        assert np.array_equal(again.view(torch.int16).cpu().numpy(), np.asarray(cache0[:6]))
+        block.close()
+        for L in layers:
+            L.close()
+    nf.nf_set_stream(None)
+
+
+def test_measured_profiler_agrees_with_the_sized_one():
+    """The Profiler that trains one step per batch size and reads the device's peak-memory counter against the one that adds
+    up the library's own buffers: the measured bytes can only exceed the sized ones by the allocator's rounding, both give a
+    straight line in the batch size whose largest batch under a budget agrees within a tenth (the measured one also counts
+    the step's output activation, labels and loss, and its line is fitted at small batch sizes); Algorithm 1 runs on either."""
+    import torch
+    from paper_2402_14139_b200 import nf
+    nf.lib()
+    nf.nf_set_stream(None)
+    wl = _wl()
+    ls = [l for _, b in wl["blocks"] for l in b]
+    batches = (8, 16, 32)
+    for l in ls:
+        measured = pipeline.measure_layer_memory(nf, torch, l, wl["classes"], batches)
+        sized, slope_s, icpt_s = nf.nf_profile_layer(l["Cin"], l["Cout"], l["H"], l["W"], l["F"], wl["classes"], list(batches),
+                                                     stride=l["stride"], maxpool=l["pool"])
+        slope_m, icpt_m = nf.nf_fit_line(list(batches), measured)
+        for m, s in zip(measured, sized):
+            assert s <= m <= s + 8 * 2 ** 20, (m, s)           # never less than the buffers; at most a few allocator blocks more
+        assert abs(slope_m - slope_s) <= 0.05 * slope_s + 2 ** 20 / 8
+    budget = 64e6
+    plan_m, model = pipeline.plan_blocks_measured(nf, torch, ls, wl["classes"], budget, 512, batches=batches)
+    max_m = [nf.nf_max_batch(sl, ic, budget) for sl, ic in model]
+    for l, bm in zip(ls, max_m):
+        _, sl, ic = nf.nf_profile_layer(l["Cin"], l["Cout"], l["H"], l["W"], l["F"], wl["classes"], list(batches), stride=l["stride"],
+                                        maxpool=l["pool"])
+        bs = nf.nf_max_batch(sl, ic, budget)
+        assert abs(bm - bs) <= 0.1 * bs + 1, (bm, bs)
+    assert plan_m == nf.nf_partition([min(b, 2 ** 31 - 1) for b in max_m], 512, 0.4)
+    assert plan_m[0][0] == 0 and plan_m[-1][1] == len(ls) - 1
+    nf.nf_set_stream(None)
