@@ -136,14 +136,19 @@ def op_model(l, N, classes, es, fam):
     nparam = 9 * l["Cin"] * l["Cout"] + 2 * l["Cout"] + 9 * l["Cout"] * l["F"] + l["F"] + classes * (4 * l["F"] + 1)
     tc = lambda k: "tensor" if fam[k] == "tcgen05" else "alu"
     fused = len(fam) > 4 and fam[4] == "fused"   # BatchNorm + ReLU applied inside the aux forward kernel
+    masked = len(fam) > 5 and fam[5] == "mask"   # h never stored: pooled in the aux forward's epilogue, sign bits kept
+    two_pass = len(fam) > 6 and fam[6] == "two-pass"   # da never stored: the input gradient runs once for the sums, once for dy
     return dict(conv_fwd=(tc(0), fl["conv_fwd"], es * (nx + ny)),          # read x, write y
                 wgrad=(tc(1), fl["wgrad"], es * (nx + ny)),                # read x and dy
                 # read a, write h; fused: read y, write a and h
-                aux_fwd=(tc(2), fl["aux_fwd"], es * ((ny if fused else 0) + na + nh)),
-                aux_bwd=(tc(3), fl["aux_bwd"], es * (4 * nh + 2 * na)),    # h -> dh; a, dh -> gWa; dh -> da
+                aux_fwd=(tc(2), fl["aux_fwd"], es * ((ny if fused else 0) + na + (0 if masked else nh))),
+                # h -> dh (from the sign mask: dh written only); a, dh -> gWa; dh -> da (two-pass: dh and y read, sums only)
+                aux_bwd=(tc(3), fl["aux_bwd"],
+                         es * ((3 if masked else 4) * nh + na + (ny if two_pass else na))),
                 # read y, write a; fused: only the statistics are finished here (partial sums in, coefficients out)
                 bn_fwd=("hbm", None, 4 * 2 * l["Cout"] * 1184 if fused else es * (ny + na)),
-                bn_bwd=("hbm", None, es * (2 * ny + na)),                  # read y and da, write dy
+                # read y and da, write dy; two-pass: the second run of the input gradient reads dh and y and writes dy
+                bn_bwd=("hbm", None, es * (nh + 2 * ny) if two_pass else es * (2 * ny + na)),
                 head=("hbm", None, es * nh + 4 * N * (8 * l["F"] + 2 * classes)),
                 sgd=("hbm", None, 18 * nparam))                            # theta, v read+write (fp32), g read, bf16 copy write
 
@@ -268,7 +273,7 @@ def run_ours(args, rank, world):
     ms, e2e_s = max_over_ranks([ms, e2e_s], world, "cuda")
 
     peaks, peak_src = load_peaks()
-    fam = [[L.kernel_family(k) for k in range(5)] for L in layers]
+    fam = [[L.kernel_family(k) for k in range(7)] for L in layers]
     clocks = sampler.summary()
     # Which measured bf16 peak the tensor kernels are held against: the timed region and the per-op pass last a fraction
     # of a second each, so unless the sampled SM clock has already dropped well below its maximum these are burst

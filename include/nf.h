@@ -348,7 +348,10 @@ long long nf_launch_count(void);
  * op 4: "fused" when the BatchNorm + ReLU pass of the step runs inside the aux forward kernel
  * (which then also writes act_out), "separate" otherwise.
  * op 5: "mask" when that kernel also pools the aux output h in its epilogue and keeps only one sign bit per element of it
- * (Eq. 2's F_n applied before h ever reaches memory), "stored" when h is written and pooled by separate kernels. */
+ * (Eq. 2's F_n applied before h ever reaches memory), "stored" when h is written and pooled by separate kernels.
+ * op 6: "two-pass" when the aux input gradient runs twice -- once to reduce the BatchNorm-backward sums, once more to write
+ * the gradient at the conv output directly -- so that the gradient at the activation (NF_T_DA) is never stored and no
+ * separate BatchNorm-backward pass runs; "stored" otherwise. */
 const char* nf_layer_kernel_family(const nf_layer* layer, int op);
 
 const char* nf_strerror(int status);

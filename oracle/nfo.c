@@ -66,6 +66,36 @@ void nfo_conv3x3(const double* x, int N, int Cin, int H, int W, const double* w,
         }
 }
 
+/* The projection shortcut of a down-sampling residual block (the paper trains ResNet-18, Section "Experimental
+ * Setup"): a 1x1 convolution with stride s, y[n,co,i,j] = sum_ci w[co,ci] * x[n,ci,i*s,j*s], and the derivative of that
+ * with respect to its weights, dw[co,ci] = sum_{n,i,j} g[n,co,i,j] * x[n,ci,i*s,j*s]. */
+void nfo_conv1x1(const double* x, int N, int Cin, int H, int W, const double* w, int Cout, int stride, double* y) {
+  const int Ho = nfo_out_size(H, stride), Wo = nfo_out_size(W, stride);
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int co = 0; co < Cout; ++co)
+      for (int i = 0; i < Ho; ++i)
+        for (int j = 0; j < Wo; ++j) {
+          double acc = 0.0;
+          for (int ci = 0; ci < Cin; ++ci) acc += w[(size_t)co * Cin + ci] * x[IDX4(n, ci, i * stride, j * stride, Cin, H, W)];
+          y[IDX4(n, co, i, j, Cout, Ho, Wo)] = acc;
+        }
+}
+
+void nfo_conv1x1_wgrad(const double* x, int N, int Cin, int H, int W, const double* g, int Cout, int stride, double* dw) {
+  const int Ho = nfo_out_size(H, stride), Wo = nfo_out_size(W, stride);
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int co = 0; co < Cout; ++co)
+    for (int ci = 0; ci < Cin; ++ci) {
+      double acc = 0.0;
+      for (int n = 0; n < N; ++n)
+        for (int i = 0; i < Ho; ++i)
+          for (int j = 0; j < Wo; ++j)
+            acc += g[IDX4(n, co, i, j, Cout, Ho, Wo)] * x[IDX4(n, ci, i * stride, j * stride, Cin, H, W)];
+      dw[(size_t)co * Cin + ci] = acc;
+    }
+}
+
 /* Algorithm 2, gradient step: derivative of the convolution with respect to its weights.
  * dw[co,ci,kh,kw] = sum_{n,i,j} g[n,co,i,j] * x[n,ci,i*s+kh-1,j*s+kw-1]. */
 void nfo_conv3x3_wgrad(const double* x, int N, int Cin, int H, int W, const double* g, int Cout,

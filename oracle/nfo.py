@@ -106,6 +106,24 @@ def conv3x3_dgrad(w, g, H, W, stride=1):
     return dx
 
 
+def conv1x1(x, w, stride=2):
+    x, w = _c64(x), _c64(w)
+    N, Ci, H, W = x.shape
+    Co = w.shape[0]
+    y = np.empty((N, Co, out_size(H, stride), out_size(W, stride)))
+    lib().nfo_conv1x1(_d(x), N, Ci, H, W, _d(w), Co, stride, _d(y))
+    return y
+
+
+def conv1x1_wgrad(x, g, stride=2):
+    x, g = _c64(x), _c64(g)
+    N, Ci, H, W = x.shape
+    Co = g.shape[1]
+    dw = np.empty((Co, Ci))
+    lib().nfo_conv1x1_wgrad(_d(x), N, Ci, H, W, _d(g), Co, stride, _d(dw))
+    return dw
+
+
 def bn_train(y, gamma, beta, eps=1e-5):
     y = _c64(y)
     N, Cc, H, W = y.shape
@@ -317,6 +335,64 @@ class Layer:
         P = self._params()
         lib().nfo_layer_eval(C.byref(d), _d(x), C.byref(P), _d(out))
         return out
+
+
+class Projection:
+    """Projection shortcut of a down-sampling residual block: s = BN(Wp (*) x_b), a 1x1 convolution with stride 2 on the
+    block input x_b followed by BatchNorm with batch statistics.  The paper trains ResNet-18 without saying how such a
+    shortcut enters a layer-local step; the reading here: it is part of the layer whose BatchNorm output it is added to
+    (x_{n+1} = P(ReLU(BN(theta_n x_n) + s))), so its parameters (Wp, gamma_p, beta_p) are trained by that layer's local
+    loss: the gradient at the sum, dz, is also the gradient at s; no gradient reaches x_b.  Same optimiser and running-
+    statistics conventions as the layer.  In the bf16 configuration the stored conv output and s are rounded to bfloat16
+    and the convolution reads a bfloat16 copy of Wp, as the layer does for y, a and W."""
+
+    def __init__(self, Cin, Cout, stride=2, eps=1e-5, momentum=0.9, bn_momentum=0.1, store_bf16=False):
+        self.Cin, self.Cout, self.stride, self.eps, self.momentum, self.bn_momentum = Cin, Cout, stride, eps, momentum, bn_momentum
+        self.store_bf16 = store_bf16
+        self.p = dict(W=np.zeros((Cout, Cin)), gamma=np.ones(Cout), beta=np.zeros(Cout))
+        self.v = {k: np.zeros_like(a) for k, a in self.p.items()}
+        self.rmean, self.rvar = np.zeros(Cout), np.ones(Cout)
+
+    def _round(self, a):
+        if not self.store_bf16:
+            return a
+        return np.asarray(np.float64(_bf16_array(a)))
+
+    def forward(self, xb):
+        """s for a batch, with batch statistics; keeps what backward needs."""
+        wq = self._round(self.p["W"])
+        ys = self._round(conv1x1(xb, wq, self.stride))
+        mu, var, shat, s = bn_train(ys, self.p["gamma"], self.p["beta"], self.eps)
+        self._saved = (_c64(xb), ys.shape, mu, var, shat)
+        return self._round(s)
+
+    def backward(self, dz, lr, update=True):
+        """Gradients from the gradient dz at the sum, then the momentum update.  Returns dict(gW, ggamma, gbeta)."""
+        xb, shape, mu, var, shat = self._saved
+        gg, gb, dys = bn_bwd(_c64(dz).reshape(shape), shat, self.p["gamma"], var, self.eps)
+        g = dict(W=conv1x1_wgrad(xb, dys, self.stride), gamma=gg, beta=gb)
+        if update:
+            M = shat.size // self.Cout
+            for k in ("W", "gamma", "beta"):
+                sgd(self.p[k], self.v[k], g[k], lr, self.momentum)
+            self.rmean[...] = (1 - self.bn_momentum) * self.rmean + self.bn_momentum * mu
+            self.rvar[...] = (1 - self.bn_momentum) * self.rvar + self.bn_momentum * var * M / (M - 1)
+        return dict(gW=g["W"], ggamma=gg, gbeta=gb)
+
+    def eval_forward(self, xb):
+        """s with the running statistics (cache fill, early-exit evaluation)."""
+        ys = self._round(conv1x1(xb, self._round(self.p["W"]), self.stride))
+        ch = (1, -1, 1, 1)
+        s = self.p["gamma"].reshape(ch) * (ys - self.rmean.reshape(ch)) / np.sqrt(self.rvar.reshape(ch) + self.eps) + self.p["beta"].reshape(ch)
+        return self._round(s)
+
+
+def _bf16_array(a):
+    """float64 array rounded to bfloat16 through the C routine's rule (round to nearest even via float32)."""
+    f = np.ascontiguousarray(a, dtype=np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    r = ((u + np.uint64(0x7FFF) + ((u >> np.uint64(16)) & np.uint64(1))) >> np.uint64(16)) << np.uint64(16)
+    return (r & np.uint64(0xFFFFFFFF)).astype(np.uint32).view(np.float32).reshape(f.shape)
 
 
 def select_exit(val_accuracy, params):

@@ -466,8 +466,12 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
   } else {
     NF_TRY(nf_k_bn_bwd_finalize_tot(L->dptot + 2 * Co, Co, world, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
   }
-  NF_TRY(nf_k_bn_bwd_apply(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->sdz, L->sdzx,
+  if (nf_tc_dgrad_two_pass(L) && !L->skip) {  // second pass of the input gradient writes dy itself; da was never stored
+    NF_TRY(nf_tc_aux_dgrad_dy(L, M));
+  } else {
+    NF_TRY(nf_k_bn_bwd_apply(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->sdz, L->sdzx,
                              M, L->dy, L->skip));
+  }
   trace_end();
   // gradient of theta_n (the layer input receives none), then the update
   trace_begin(6);
@@ -919,9 +923,10 @@ int nf_set_stream(void* s) {
 long long nf_launch_count(void) { return g_nf_launches; }
 
 const char* nf_layer_kernel_family(const nf_layer* L, int op) {
-  if (!L || op < 0 || op > 5) return "";
+  if (!L || op < 0 || op > 6) return "";
   if (op == 4) return nf_tc_bn_aux_fused(L) && !L->skip ? "fused" : "separate";
   if (op == 5) return nf_tc_bn_aux_fused(L) && !L->skip && nf_tc_aux_pool_fused(L) ? "mask" : "stored";
+  if (op == 6) return nf_tc_dgrad_two_pass(L) && !L->skip ? "two-pass" : "stored";
   return L->fam[op] ? "tcgen05" : "cuda-core";
 }
 

@@ -991,10 +991,19 @@ __global__ void __launch_bounds__(256) pool_finish_kernel(const float* __restric
   const int qh = th / 2, qw = tw / 2, cnt = qh * qw * 4;
   float s = 0.f;
   if (ln < lanes) {
-    for (int k = ln; k < cnt; k += lanes) {
+    auto at = [&](int k) {
       const int w4 = k & 3, tq = k >> 2, ty = u * qh + tq / qw, tx = v * qw + tq % qw;
-      s += part[(((size_t)n * th + ty) * tw + tx) * 4 * F + (size_t)w4 * F + f];
+      return part[(((size_t)n * th + ty) * tw + tx) * 4 * F + (size_t)w4 * F + f];
+    };
+    int k = ln;
+    for (; k + 3 * lanes < cnt; k += 4 * lanes) {  // four loads in flight, added in index order
+      const float a0 = at(k), a1 = at(k + lanes), a2 = at(k + 2 * lanes), a3 = at(k + 3 * lanes);
+      s += a0;
+      s += a1;
+      s += a2;
+      s += a3;
     }
+    for (; k < cnt; k += lanes) s += at(k);
   }
   sm[threadIdx.x] = s;
   __syncthreads();
@@ -1010,6 +1019,7 @@ __global__ void __launch_bounds__(256) pool_finish_kernel(const float* __restric
 __global__ void __launch_bounds__(256) dh_mask_vec_kernel(const uint8_t* __restrict__ mask, const float* __restrict__ dp, int Ha, int Wa,
                                                           int F8, size_t P, uint4* __restrict__ dh, float* __restrict__ red) {
   __shared__ float sm[8][256];
+  __shared__ __align__(16) float tab[4][4][64];  // dp / |bin| of up to four images, [image][bin][channel]: 16-byte reads per thread
   const int F = F8 * 8;
   const int planes = 256 / F8, g = threadIdx.x % F8, pl = threadIdx.x / F8;
   const float inv_bin = 1.f / (float)((Ha / 2) * (Wa / 2));
@@ -1017,15 +1027,32 @@ __global__ void __launch_bounds__(256) dh_mask_vec_kernel(const uint8_t* __restr
 #pragma unroll
   for (int i = 0; i < 8; ++i) a[i] = 0.f;
   const size_t p0 = P * blockIdx.x / gridDim.x, p1 = P * (blockIdx.x + 1) / gridDim.x;
+  const size_t img = (size_t)Wa * Ha;
+  const size_t n_lo = p0 / img, n_hi = p1 > p0 ? (p1 - 1) / img : n_lo;
+  const bool tabled = F <= 64 && n_hi - n_lo < 4;  // the block's pixel range touches few images: their dp rows fit the table
+  if (tabled)
+    for (int i = threadIdx.x; i < (int)(n_hi - n_lo + 1) * 4 * F; i += 256) {
+      const int f = i % F, bin = (i / F) % 4, ni = i / (4 * F);
+      tab[ni][bin][f] = dp[(n_lo + ni) * 4 * F + (size_t)f * 4 + bin] * inv_bin;
+    }
+  __syncthreads();
   for (size_t p = p0 + pl; pl < planes && p < p1; p += planes) {  // threads beyond planes * F8 (F8 not a divisor of 256) idle
     const uint32_t m = mask[p * F8 + g];
     const int j = (int)(p % Wa), i = (int)((p / Wa) % Ha);
-    const size_t n = p / ((size_t)Wa * Ha);
+    const size_t n = p / img;
     const int bin = (i >= Ha / 2 ? 2 : 0) + (j >= Wa / 2 ? 1 : 0);
-    const float* d = dp + n * 4 * F + (size_t)(g * 8) * 4 + bin;
     float o[8];
+    if (tabled) {
+      const float4 t0 = *reinterpret_cast<const float4*>(&tab[n - n_lo][bin][g * 8]);
+      const float4 t1 = *reinterpret_cast<const float4*>(&tab[n - n_lo][bin][g * 8 + 4]);
+      const float tv[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
 #pragma unroll
-    for (int e = 0; e < 8; ++e) o[e] = (m >> e) & 1u ? d[e * 4] * inv_bin : 0.f;
+      for (int e = 0; e < 8; ++e) o[e] = (m >> e) & 1u ? tv[e] : 0.f;
+    } else {
+      const float* d = dp + n * 4 * F + (size_t)(g * 8) * 4 + bin;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) o[e] = (m >> e) & 1u ? d[e * 4] * inv_bin : 0.f;
+    }
     const uint4 packed = pack8(o);
     dh[p * F8 + g] = packed;
     float r[8];

@@ -24,6 +24,10 @@ constexpr int kMaxStages = 8;
 // stretches the tensor-core instructions.
 constexpr int kXfThreads = 128;
 constexpr int kFoldThreads = 320;  // folded-tap forward: producer, MMA issuer and two epilogue groups of four warps
+// Tiles of y2 (the conv output read beside the input gradient, stats >= 2) in flight per CTA.  A slot turns over once per
+// load latency plus epilogue time, so with the earlier two slots per epilogue group the kernel ran at the pace of these loads
+// (about four tiles per HBM round trip) whatever else it did; with five the loads run as far ahead as the operand stages.
+constexpr int kYSlots = 5;
 
 struct FwdParams {
   int N, H, W, Cin, Cout;
@@ -426,7 +430,9 @@ struct FoldParams {
   int N, H, W, Cout, kchunks, n_tiles, tiles_w, tiles_h, total_tiles, stages, stats;
   float* red;         // EPI 0, stats != 0: [grid / n_tiles * 8][2][Cout]
   int32_t* status;
-  const float *bn_scale, *bn_shift, *bn_mu, *bn_invstd;  // stats == 2
+  const float *bn_scale, *bn_shift, *bn_mu, *bn_invstd;  // stats >= 2
+  const float *bn_sdz, *bn_sdzx;                         // stats == 4: the reduced sums of the whole batch
+  float inv_m;                                           // stats == 4: 1 / (elements per channel)
   const float* bias;  // EPI 1
   bf16* out;          // EPI 1: [N][H][W][Cout]
   // XF: the input map is the conv output y; a = ReLU(y*scale + shift) is formed in shared memory and written to xf_a
@@ -447,7 +453,11 @@ struct FoldParams {
 // stats (EPI 0): 1 = per-channel sums of (y, y^2) of the stored values (BatchNorm forward statistics);
 //       2 = the output is the gradient da at a BatchNorm+ReLU output of the same shape: per-channel sums of
 //       (dz, dz * xhat) with dz = da * 1[y2*scale+shift > 0], xhat = (y2 - mu) * invstd, where the tile of the
-//       pre-normalisation values y2 is fetched through tm_y2 (BatchNorm backward reduction fused into the producer of da).
+//       pre-normalisation values y2 is fetched through tm_y2 (BatchNorm backward reduction fused into the producer of da);
+//       3 = the same sums, but da is not written at all; 4 = the second pass of that pair: da is formed again, turned
+//       into dy = scale * (dz - sum(dz)/M - xhat * sum(dz*xhat)/M) in the staging tile with the sums of pass 3, and dy is
+//       what the TMA store writes.  Passes 3 + 4 replace "write da; read y and da; write dy" by one more read of the
+//       narrow dh tensor: da never reaches memory.
 // KC / MIR: KC = channels of the activation box (64; 16 or 32 for the aux input gradient whose input dh has F
 // channels), MIR = 1 reads the weights [tap][f][c] MN-major with both taps mirrored (input-gradient convolution;
 // the CTA's 64-channel output tile is blockIdx.x % n_tiles).
@@ -477,21 +487,28 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   const int w_bytes = 3 * p.kchunks * kWTile; // [chunk][kh][kw*G + co][64 ci]
   uint8_t* wres = smem + (size_t)p.stages * kABytes;
   uint8_t* stg = wres + w_bytes;              // EPI 0: 112 (UF: 128) output pixels x 128 bytes
-  uint8_t* ybuf = stg + 2 * 16384;            // EPI 0, stats 2: two tiles of y2 per epilogue group
-  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (EPI == 0 ? (p.stats == 2 ? 6 : 2) * 16384 : 0));  // one staging tile per epilogue group
+  uint8_t* ybuf = stg + 2 * 16384;            // EPI 0, stats >= 2: kYSlots tiles of y2, taken in turn by the CTA's tiles
+  constexpr int kAStg = 112 * 128;            // XF: one 14 x 8-pixel tile of a on its way to global memory (three in rotation)
+  // one staging tile per epilogue group (EPI 0), or the three tiles of a (XF)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (EPI == 0 ? (p.stats >= 2 ? 2 + kYSlots : 2) * 16384 : XF ? 3 * kAStg : 0));
   uint64_t* full = bars;
   uint64_t* empty = bars + kMaxStages;
   uint64_t* tfull = bars + 2 * kMaxStages;
-  uint64_t* tempty = tfull + 2;
-  uint64_t* wfull = tempty + 2;
+  uint64_t* tempty = tfull + 4;
+  uint64_t* wfull = tempty + 4;
   uint64_t* yfull = wfull + 1;
-  uint64_t* yempty = yfull + 4;
-  uint64_t* xfull = yempty + 4;  // XF: stage normalised, ready for the issuer
+  uint64_t* yempty = yfull + kYSlots;
+  uint64_t* xfull = yempty + kYSlots;  // XF: stage normalised, ready for the issuer
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(xfull + kMaxStages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);  // [2], one per epilogue group
-  constexpr uint32_t kAccStride = G == 64 ? 256 : 128;  // columns between the two accumulators
-  constexpr uint32_t kTmemCols = 2 * kAccStride;
+  volatile int* xf_go = reinterpret_cast<volatile int*>(tmem_slot + 4);   // [2], alternating between the iterations of the XF warps
+  // Accumulators in tensor memory.  The unfolded form needs 64 columns each and keeps four, so that the issuer can run two
+  // tiles ahead of each epilogue group (group g takes the tiles tl = g, g + 2, ... and so alternates between two of them);
+  // the folded forms need up to 192 columns each and keep two, one per group.
+  constexpr uint32_t kAccs = UF ? 4 : 2;
+  constexpr uint32_t kAccStride = UF ? 128 : G == 64 ? 256 : 128;  // columns between two accumulators
+  constexpr uint32_t kTmemCols = kAccs * kAccStride;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -500,11 +517,11 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       ptx::mbar_init(&empty[s], 1);
       ptx::mbar_init(&xfull[s], kXfThreads);
     }
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < (int)kAccs; ++a) {
       ptx::mbar_init(&tfull[a], 1);
       ptx::mbar_init(&tempty[a], 128);
     }
-    for (int a = 0; a < 4; ++a) {
+    for (int a = 0; a < kYSlots; ++a) {
       ptx::mbar_init(&yfull[a], 1);
       ptx::mbar_init(&yempty[a], 128);
     }
@@ -556,9 +573,9 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         __syncwarp();
       }
       if constexpr (EPI == 0) {
-        if (ok && p.stats == 2) {  // the y2 tile of this output tile, for the epilogue group that owns it
-          const uint32_t k2 = tl >> 1, slot = (tl & 1) * 2 + (k2 & 1);
-          if (!__all_sync(0xffffffffu, ptx::mbar_wait(&yempty[slot], ((k2 >> 1) & 1) ^ 1, abort_flag))) break;
+        if (ok && p.stats >= 2) {  // the y2 tile of this output tile, for the epilogue group that owns it
+          const uint32_t slot = tl % kYSlots;
+          if (!__all_sync(0xffffffffu, ptx::mbar_wait(&yempty[slot], ((tl / kYSlots) & 1) ^ 1, abort_flag))) break;
           if (lane == 0) {
             ptx::mbar_expect_tx(&yfull[slot], kTW * 8 * 128);
             ptx::tma_load_4d(ybuf + slot * 16384, &tm_y2, &yfull[slot], (t % p.n_tiles) * 64, w0, h0, n);
@@ -575,7 +592,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     uint32_t it = 0, tl = 0;
     bool ok = blockIdx.x >= p.total_tiles || __all_sync(0xffffffffu, ptx::mbar_wait(wfull, 0, abort_flag));
     for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++tl) {
-      const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+      const uint32_t acc = tl % kAccs, aph = (tl / kAccs) & 1;
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(&tempty[acc], aph ^ 1, abort_flag))) break;
       ptx::tc_fence_after();
       const uint32_t d = tmem_base + acc * kAccStride;
@@ -615,21 +632,23 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       __syncwarp();
     }
   } else if (XF && warp >= kFoldThreads / 32) {
-    // normalisation warps: a thread owns one 16-byte channel chunk (8 channels) of one box column and walks the 10 rows
+    // normalisation warps: a thread owns one 16-byte channel chunk (8 channels) of one box column and walks the 10 rows.
+    // The tile's own 14 x 8 pixels of a leave through a TMA store: the threads copy them from registers into a dense staging
+    // tile (three in rotation) and one thread issues the store, so no global store instruction runs in these warps.
     const int xt = (threadIdx.x - kFoldThreads) & 127, xg = (threadIdx.x - kFoldThreads) >> 7;  // group xg takes rows xg, xg+2, ...
     constexpr int kXg = kXfThreads / 128, kRows = 10 / kXg;
+    static_assert(kXg == 1, "the staging of a assumes one normalisation group");
     const int j = xt & 7, col = xt >> 3;                   // logical chunk, box column (0..15)
     const uint32_t off0 = (uint32_t)col * 128 + (uint32_t)((j ^ (col & 7)) * 16);  // 128-byte swizzle: the row's low bits are col's
-    const int C = p.kchunks * 64;
     uint32_t it = 0;
     float sc[8], sh[8];
     int coef_ck = -1;  // channel chunk whose coefficients the registers hold
-    for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x) {
+    bool go = true;
+    for (int t = blockIdx.x; go && t < p.total_tiles; t += gridDim.x) {
       const int m = t / p.n_tiles;
       const int w0 = (m % p.tiles_w) * 14, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
       const int w = w0 - 1 + col;
       const bool w_in = w >= 0 && w < p.W, w_own = col >= 1 && col <= 14;
-      bool ok = true;
       for (int ck = 0; ck < p.kchunks; ++ck, ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
@@ -641,41 +660,52 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             sh[i] = __ldg(p.xf_shift + ck * 64 + j * 8 + i);
           }
         }
-        if (!ptx::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
-        const uint32_t box = ptx::smem_u32(smem + (size_t)s * kABytes) + off0 + xg * 2048;
-        // all rows are loaded first, then normalised, then stored: the loads overlap instead of queueing behind stores
-        uint4 q[kRows];
+        const bool ok = ptx::mbar_wait(&full[s], ph, abort_flag);
+        const uint32_t astg = ptx::smem_u32(stg) + (it % 3) * kAStg;
+        if (ok) {
+          const uint32_t box = ptx::smem_u32(smem + (size_t)s * kABytes) + off0 + xg * 2048;
+          // all rows are loaded first, then normalised, then stored: the loads overlap instead of queueing behind stores
+          uint4 q[kRows];
 #pragma unroll
-        for (int i = 0; i < kRows; ++i) q[i] = ptx::lds128(box + i * kXg * 2048);
-#pragma unroll
-        for (int i = 0; i < kRows; ++i) {
-          const int h = h0 - 1 + i * kXg + xg;
-          const uint32_t qw[4] = {q[i].x, q[i].y, q[i].z, q[i].w};
-          uint32_t ow[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float a0 = fmaxf(fmaf(__uint_as_float(qw[e] << 16), sc[2 * e], sh[2 * e]), 0.f);
-            const float a1 = fmaxf(fmaf(__uint_as_float(qw[e] & 0xffff0000u), sc[2 * e + 1], sh[2 * e + 1]), 0.f);
-            const __nv_bfloat162 b2 = __floats2bfloat162_rn(a0, a1);
-            ow[e] = *reinterpret_cast<const uint32_t*>(&b2);
-          }
-          const bool in = w_in && h >= 0 && h < p.H;
-          q[i] = in ? make_uint4(ow[0], ow[1], ow[2], ow[3]) : make_uint4(0u, 0u, 0u, 0u);
-          ptx::sts128(box + i * kXg * 2048, q[i]);
-        }
-        ptx::fence_async_smem();  // the tensor core reads the stage through the async proxy
-        ptx::mbar_arrive(&xfull[s]);
-        if (w_own) {  // the tile's own pixels go to global memory after the stage has been handed on
-          bf16* dst = p.xf_a + (((size_t)n * p.H + h0 - 1 + xg) * p.W + w) * C + ck * 64 + j * 8;
+          for (int i = 0; i < kRows; ++i) q[i] = ptx::lds128(box + i * kXg * 2048);
 #pragma unroll
           for (int i = 0; i < kRows; ++i) {
-            const int r = i * kXg + xg;  // box row; rows 1..8 are the tile's own
-            if (r >= 1 && r <= 8) *reinterpret_cast<uint4*>(dst + (size_t)(i * kXg) * p.W * C) = q[i];
+            const int h = h0 - 1 + i * kXg + xg;
+            const uint32_t qw[4] = {q[i].x, q[i].y, q[i].z, q[i].w};
+            uint32_t ow[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float a0 = fmaxf(fmaf(__uint_as_float(qw[e] << 16), sc[2 * e], sh[2 * e]), 0.f);
+              const float a1 = fmaxf(fmaf(__uint_as_float(qw[e] & 0xffff0000u), sc[2 * e + 1], sh[2 * e + 1]), 0.f);
+              const __nv_bfloat162 b2 = __floats2bfloat162_rn(a0, a1);
+              ow[e] = *reinterpret_cast<const uint32_t*>(&b2);
+            }
+            const bool in = w_in && h >= 0 && h < p.H;
+            q[i] = in ? make_uint4(ow[0], ow[1], ow[2], ow[3]) : make_uint4(0u, 0u, 0u, 0u);
+            ptx::sts128(box + i * kXg * 2048, q[i]);
           }
+          if (w_own) {  // box rows 1..8 x columns 1..14 are the tile's own pixels: dense rows of the staging tile, same swizzle
+#pragma unroll
+            for (int i = 1; i <= 8; ++i) {
+              const uint32_t orow = (uint32_t)((i - 1) * 14 + col - 1);
+              ptx::sts128(astg + orow * 128 + ((j ^ (orow & 7)) * 16), q[i]);
+            }
+          }
+          ptx::fence_async_smem();  // the tensor core and the TMA store read shared memory through the async proxy
+          ptx::mbar_arrive(&xfull[s]);
+        }
+        // one thread decides for all 128 whether to go on, so nobody is left alone at the barrier
+        if (xt == 0) xf_go[it & 1] = ok && !*abort_flag ? 1 : 0;
+        ptx::named_barrier(3, kXfThreads);
+        if (!xf_go[it & 1]) { go = false; break; }
+        if (xt == 0) {
+          ptx::tma_store_4d(&tm_y, reinterpret_cast<const void*>(stg + (it % 3) * kAStg), ck * 64, w0, h0, n);
+          ptx::tma_store_commit();
+          ptx::tma_store_wait_read_but_one();  // the store before this one has read its tile: the tile after next may be written
         }
       }
-      if (!ok) break;
     }
+    if (xt == 0) ptx::tma_store_wait_all();
   } else {
     // two epilogue groups of 128 threads; group g owns accumulator g and takes every second tile of the CTA
     const int grp = (threadIdx.x - 64) >> 7;
@@ -692,10 +722,18 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
     for (int i = 0; i < 8; ++i) s1[i] = s2[i] = bsc[i] = bsh[i] = 0.f;
     if constexpr (EPI == 0) {
-      if (p.stats == 2) {
+      if (p.stats >= 2) {
         const int ch = (int)(blockIdx.x % p.n_tiles) * 64 + schunk * 8;
 #pragma unroll
         for (int i = 0; i < 8; ++i) { bsc[i] = p.bn_scale[ch + i]; bsh[i] = p.bn_shift[ch + i]; }
+        if (p.stats == 4) {  // s1, s2 hold the per-channel constants of dy = scale*dz + s1*y + s2 instead of running sums
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float sc = bsc[i], m1 = p.bn_sdz[ch + i] * p.inv_m, m2 = p.bn_sdzx[ch + i] * p.inv_m, is = p.bn_invstd[ch + i];
+            s1[i] = -sc * m2 * is;
+            s2[i] = sc * (m2 * is * p.bn_mu[ch + i] - m1);
+          }
+        }
       }
     }
     uint32_t tl = grp;
@@ -704,7 +742,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       const int nt = t % p.n_tiles;
       const int m = t / p.n_tiles;
       const int w0 = (m % p.tiles_w) * kTW, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
-      const uint32_t acc = grp, aph = (tl >> 1) & 1;
+      const uint32_t acc = tl % kAccs, aph = (tl / kAccs) & 1;
       ptx::mbar_wait(&tfull[acc], aph, abort_flag);
       ptx::tc_fence_after();
       if (et == 0) {
@@ -813,14 +851,44 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       if constexpr (EPI == 0) {
         ptx::fence_async_smem();
         ptx::named_barrier(1 + grp, 128);
-        if (et == 0) {
+        if (p.stats == 4) {
+          // second pass: the staged da tile becomes dy in place (thread <-> 8 channels x 7 or 8 rows, as for the sums)
+          const uint32_t slot = tl % kYSlots;
+          ptx::mbar_wait(&yfull[slot], (tl / kYSlots) & 1, abort_flag);
+          const uint8_t* yb = ybuf + slot * 16384;
+#pragma unroll
+          for (int rr = 0; rr < kTW / 2; ++rr) {
+            const int row = srg + 16 * rr;
+            const int off = row * 128 + ((schunk ^ (row & 7)) * 16);
+            const uint4 dq = *reinterpret_cast<const uint4*>(stg_g + off);
+            const uint4 yq = *reinterpret_cast<const uint4*>(yb + off);
+            const uint32_t dw[4] = {dq.x, dq.y, dq.z, dq.w}, yw[4] = {yq.x, yq.y, yq.z, yq.w};
+            uint32_t ow[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float d0 = __uint_as_float(dw[e] << 16), d1 = __uint_as_float(dw[e] & 0xffff0000u);
+              const float y0 = __uint_as_float(yw[e] << 16), y1 = __uint_as_float(yw[e] & 0xffff0000u);
+              const float z0 = fmaf(y0, bsc[2 * e], bsh[2 * e]) > 0.f ? d0 : 0.f;
+              const float z1 = fmaf(y1, bsc[2 * e + 1], bsh[2 * e + 1]) > 0.f ? d1 : 0.f;
+              const float o0 = fmaf(bsc[2 * e], z0, fmaf(s1[2 * e], y0, s2[2 * e]));
+              const float o1 = fmaf(bsc[2 * e + 1], z1, fmaf(s1[2 * e + 1], y1, s2[2 * e + 1]));
+              const __nv_bfloat162 b2 = __floats2bfloat162_rn(o0, o1);
+              ow[e] = *reinterpret_cast<const uint32_t*>(&b2);
+            }
+            *reinterpret_cast<uint4*>(stg_g + off) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+          }
+          ptx::mbar_arrive(&yempty[slot]);
+          ptx::fence_async_smem();
+          ptx::named_barrier(1 + grp, 128);
+        }
+        if (et == 0 && p.stats != 3) {
           ptx::tma_store_4d(&tm_y, stg_g, nt * 64, w0, h0, n);
           ptx::tma_store_commit();
         }
-        if (p.stats == 2) {
+        if (p.stats == 2 || p.stats == 3) {
           // sums of dz and dz*y2 (the caller of the kernel gets sum dz*xhat = invstd * (sum dz*y2 - mu * sum dz))
-          const uint32_t k2 = tl >> 1, slot = grp * 2 + (k2 & 1);
-          ptx::mbar_wait(&yfull[slot], (k2 >> 1) & 1, abort_flag);
+          const uint32_t slot = tl % kYSlots;
+          ptx::mbar_wait(&yfull[slot], (tl / kYSlots) & 1, abort_flag);
           const uint8_t* yb = ybuf + slot * 16384;
 #pragma unroll
           for (int rr = 0; rr < kTW / 2; ++rr) {
@@ -842,7 +910,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             }
           }
           ptx::mbar_arrive(&yempty[slot]);
-        } else if (p.stats) {
+        } else if (p.stats == 1) {
 #pragma unroll
           for (int rr = 0; rr < kTW / 2; ++rr) {
             const int row = srg + 16 * rr;
@@ -862,7 +930,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     }
     if constexpr (EPI == 0) {
       if (et == 0) ptx::tma_store_wait_all();
-      if (p.stats) {  // one partial per warp: lanes with the same chunk (lane & 7) are added in a fixed order
+      if (p.stats && p.stats != 4) {  // one partial per warp: lanes with the same chunk (lane & 7) are added in a fixed order
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 8);
@@ -876,7 +944,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             float second = s2[i];
-            if (p.stats == 2)
+            if (p.stats >= 2)
               second = (float)((double)p.bn_invstd[ch + i] * ((double)s2[i] - (double)p.bn_mu[ch + i] * (double)s1[i]));
             p.red[(b * 2 + 0) * p.Cout + ch + i] = s1[i];
             p.red[(b * 2 + 1) * p.Cout + ch + i] = second;
@@ -1489,15 +1557,15 @@ int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, c
 // sums (stats 2) or 64 output channels; without the sums a wider layer is faster on the generic kernel's
 // 128-channel tiles (measured).
 int fold_group(int Cout, int epi) { return epi != 1 ? 64 : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64); }
-bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride, int stats = 0) {
+bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride, int stats = 0, size_t extra_smem = 0) {
   if (stride != 1 || H % 8) return false;
-  if (epi == 2 && W % 14 && W % 16 == 0 && (stats == 2 || Cout == 64)) return Cin <= 32 && Cin % 8 == 0 && Cout % 64 == 0;
+  if (epi == 2 && W % 14 && W % 16 == 0 && (stats >= 2 || Cout == 64)) return Cin <= 32 && Cin % 8 == 0 && Cout % 64 == 0;
   if (W % 14) return false;
   if (epi == 2) return Cin <= 32 && Cin % 8 == 0 && Cout % 64 == 0;
   if (Cin % 64) return false;
   if (epi == 0 ? (Cin != 64 || Cout != 64) : (Cout > 64 || Cout % 8)) return false;
   const size_t wbytes = (size_t)9 * (Cin / 64) * fold_group(Cout, epi) * 128;
-  return wbytes + (epi == 0 ? 2 * 16384 : 0) + 2048 + 3 * 20480 <= 232448;
+  return wbytes + (epi == 0 ? 2 * 16384 : 0) + extra_smem + 2048 + 3 * 20480 <= 232448;
 }
 
 template <int G, int EPI, int KC = 64, int MIR = 0, int UF = 0, int XF = 0>
@@ -1518,6 +1586,8 @@ int launch_fold(int grid, size_t smem, const CUtensorMap& mx, const CUtensorMap&
 struct BnBwdIn {
   const void* y2;
   const float *scale, *shift, *mu, *invstd;
+  const float *sdz = nullptr, *sdzx = nullptr;  // second pass (stats 4): the reduced sums and 1 / (elements per channel)
+  float inv_m = 0.f;
 };
 
 // Normalisation fused into the aux forward (epi 1): x is then the conv output and a = ReLU(x*scale + shift) is written to a
@@ -1553,20 +1623,27 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   } else {
     my = mx;
   }
+  if (xf) {  // the normalised activation leaves the aux forward through TMA stores of 14 x 8-pixel tiles, 64 channels each
+    const uint32_t ba[4] = {64, 14, 8, 1};
+    if ((rc = make_map4(&my, xf->a, dx, ba)) != NF_OK) return rc;
+  }
   my2 = my;
-  if (stats == 2) {
-    if (epi != 2 || !bn) return NF_EINVAL;
+  if (stats >= 2) {
+    if (epi != 2 || !bn || (stats == 4 && (!bn->sdz || !bn->sdzx))) return NF_EINVAL;
     if ((rc = make_map4(&my2, bn->y2, dy, by)) != NF_OK) return rc;
   }
   FoldParams p{};
-  if (bn) { p.bn_scale = bn->scale; p.bn_shift = bn->shift; p.bn_mu = bn->mu; p.bn_invstd = bn->invstd; }
+  if (bn) {
+    p.bn_scale = bn->scale; p.bn_shift = bn->shift; p.bn_mu = bn->mu; p.bn_invstd = bn->invstd;
+    p.bn_sdz = bn->sdz; p.bn_sdzx = bn->sdzx; p.inv_m = bn->inv_m;
+  }
   p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = epi == 2 ? 1 : Cin / 64; p.n_tiles = epi == 2 ? Cout / 64 : 1;
   p.tiles_w = W / TW; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
   if ((long long)N * p.tiles_w * p.tiles_h * p.n_tiles > (1ll << 30)) return NF_EUNSUPPORTED;
   p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
   const size_t a_bytes = (size_t)(uf ? 3 : 1) * 10 * 16 * KC * 2;
   const size_t wbytes = epi == 2 ? (size_t)9 * KC * 128 : (size_t)9 * p.kchunks * G * 128;
-  const size_t fixed = wbytes + (epi != 1 ? (stats == 2 ? 6 : 2) * 16384 : 0) + 1024 + 1024;
+  const size_t fixed = wbytes + (epi != 1 ? (stats >= 2 ? 2 + kYSlots : 2) * 16384 : xf ? 3 * 112 * 128 : 0) + 1024 + 1024;
   int st = (int)((232448 - fixed) / a_bytes);
   if (st > kMaxStages) st = kMaxStages;
   p.stages = st;
@@ -1575,7 +1652,7 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   grid -= grid % p.n_tiles;  // a CTA keeps one output-channel tile (and its resident weights) for its whole life
   if (grid < p.n_tiles) grid = p.n_tiles;
   if (grid > p.total_tiles) grid = p.total_tiles;
-  if (stats) {
+  if (stats && stats != 4) {
     const size_t need = (size_t)(grid / p.n_tiles) * 8 * 2 * Cout;  // every CTA writes all of its 8 partials
     if (need > red_floats) return NF_ENOWS;
     *nb = grid / p.n_tiles * 8;
@@ -1605,6 +1682,7 @@ int run_fwd(int N, int Hin, int Win, int Cin, int Cout, const void* x, const voi
   const int H = (Hin - 1) / stride + 1, W = (Win - 1) / stride + 1;
   if (fold_ok(H, W, Cin, Cout, epi, stride, stats))
     return run_fold(N, H, W, Cin, Cout, x, w, y, stats, red, red_floats, status, nb, epi, bias, bn);
+  if (stats > 2) return NF_EUNSUPPORTED;  // the two-pass input gradient exists in the folded kernel only
   if (stats == 2 && (!bn || epi == 1)) return NF_EINVAL;
   const TcPlan pl = plan_fwd(H, W, Cin, Cout, N, epi, stride, stats == 2);
   if (!pl.ok) return NF_EUNSUPPORTED;
@@ -1855,7 +1933,8 @@ int nf_tc_aux_fwd(nf_layer* L, const void* a, int count) {
 }
 
 bool nf_tc_bn_aux_fused(const nf_layer* L) {
-  return L->fam[2] && !wide_aux(L) && !L->o.maxpool && fold_ok(L->Ha, L->Wa, L->Cout, L->F, 1, 1);
+  // beside the weights and three activation stages the kernel then also holds three staging tiles of a
+  return L->fam[2] && !wide_aux(L) && !L->o.maxpool && fold_ok(L->Ha, L->Wa, L->Cout, L->F, 1, 1, 0, 3 * 112 * 128);
 }
 
 // The fused aux forward can also keep h out of memory when the head pools by averaging and no tile straddles a pooling
@@ -1884,9 +1963,32 @@ int nf_tc_wgrad(nf_layer* L, const void* x) {
                    L->status, 0, L->o.stride);
 }
 
+// Two-pass form of the input gradient (folded kernel, no pool, no shortcut, fewer than 64 aux filters): the first pass only
+// reduces the BatchNorm-backward sums, the second (nf_tc_aux_dgrad_dy, after the sums have been finished) forms da again and
+// writes dy = BatchNorm-backward(da) directly, so da is never stored and the separate apply pass (read y and da, write dy)
+// disappears: 1.75 activation-sized tensors less memory traffic per layer step for one more read of the narrow dh.
+bool nf_tc_dgrad_two_pass(const nf_layer* L) {
+  return L->fam[3] && !wide_aux(L) && !L->o.maxpool && fold_ok(L->Ha, L->Wa, L->F, L->Cout, 2, 1, 3) &&
+         (size_t)(sm_count() / (L->Cout / 64)) * 8 * 2 * L->Cout <= L->red_floats;
+}
+
+int nf_tc_aux_dgrad_dy(nf_layer* L, double M) {
+  if (!nf_tc_dgrad_two_pass(L) || L->skip) return NF_EUNSUPPORTED;
+  int nb = 0;
+  BnBwdIn bn{L->y, L->scale, L->shift, L->mu, L->invstd};
+  bn.sdz = L->sdz; bn.sdzx = L->sdzx; bn.inv_m = (float)(1.0 / M);
+  return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->shadow + L->off[NF_P_WA], L->dy, 4, nullptr, 0, L->status, &nb, 2,
+                 nullptr, 1, &bn);
+}
+
 int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb) {
   int nb = 0;
   *bn_nb = 0;
+  if (nf_tc_dgrad_two_pass(L) && !L->skip) {  // first pass: sums only, nothing stored
+    const BnBwdIn bn{L->y, L->scale, L->shift, L->mu, L->invstd};
+    return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->shadow + L->off[NF_P_WA], L->da, 3, L->red, L->red_floats, L->status,
+                   bn_nb, 2, nullptr, 1, &bn);
+  }
   const bool wide = wide_aux(L);
   const void* w = L->shadow + L->off[NF_P_WA];
   if (wide) {

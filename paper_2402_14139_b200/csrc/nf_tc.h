@@ -45,3 +45,8 @@ int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb);
 // Self-check of the bounded wait: one small CTA waits limit_ns on a barrier nobody arrives at; *waited_ns_dev (device)
 // receives the time it waited and NF_ETIMEOUT is raised in the stand-alone status word.
 int nf_tc_bounded_wait_probe(unsigned long long limit_ns, unsigned long long* waited_ns_dev);
+// Two-pass input gradient: when nf_tc_dgrad_two_pass(L) holds (and the layer has no shortcut), nf_tc_aux_dgrad only reduces
+// the BatchNorm-backward sums (L->da stays unwritten) and, once L->sdz / L->sdzx hold the finished sums, nf_tc_aux_dgrad_dy
+// writes L->dy = BatchNorm-backward(da) with da formed again inside the kernel; M = elements per channel of the whole batch.
+bool nf_tc_dgrad_two_pass(const nf_layer* L);
+int nf_tc_aux_dgrad_dy(nf_layer* L, double M);

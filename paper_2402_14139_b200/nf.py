@@ -367,7 +367,9 @@ class Layer:
     def kernel_family(self, op: int) -> str:
         """op 0-3: "tcgen05" or "cuda-core" for main forward, main weight gradient, aux forward, aux backward;
         op 4: "fused" when BatchNorm + ReLU run inside the aux forward kernel, else "separate";
-        op 5: "mask" when that kernel pools h in its epilogue and keeps only its sign bits, else "stored"."""
+        op 5: "mask" when that kernel pools h in its epilogue and keeps only its sign bits, else "stored";
+        op 6: "two-pass" when the aux input gradient runs once for the BatchNorm-backward sums and once more to write dy, so
+        that da is never stored, else "stored"."""
         return lib().nf_layer_kernel_family(self.h, op).decode()
 
 

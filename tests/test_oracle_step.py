@@ -334,3 +334,66 @@ def test_identity_shortcut_against_library_autograd(ci):
     np.testing.assert_allclose(L.eval_forward(x, skip=skip), ae.numpy(), atol=1e-12)
     np.testing.assert_allclose(L.predict(x, skip=skip)[0], ae.numpy(), atol=1e-12)
     assert np.abs(L.eval_forward(x) - ae.numpy()).max() > 1e-3       # and the shortcut is not silently ignored
+
+
+def test_projection_shortcut_against_library_autograd_and_optimizer():
+    """The projection shortcut of a down-sampling residual block (1x1 convolution with stride 2 on the block input, then
+    BatchNorm with batch statistics) added to the layer's BatchNorm output before the ReLU; its three parameter tensors are
+    trained by the layer's local loss, the block input receives no gradient.  Two consecutive steps (gradients, updated
+    parameters, momentum, running statistics of both parts) and the eval forward re-derived with the library's ops,
+    autograd and SGD."""
+    c = dict(N=5, Cin=4, Cout=6, H=6, W=6, F=3, classes=4, stride=1, pool=False)
+    L, x, y = make_layer(c, 71)
+    Cs = 3
+    xb = synth.normal(72, 1, (c["N"], Cs, 12, 12))                 # the block input, twice the layer's map size
+    Pj = nfo.Projection(Cs, c["Cout"])
+    Pj.p["W"][...] = synth.normal(72, 2, (c["Cout"], Cs), np.sqrt(2.0 / Cs))
+    Pj.p["gamma"][...] = 1.0 + 0.2 * synth.normal(72, 3, (c["Cout"],))
+    Pj.p["beta"][...] = 0.1 * synth.normal(72, 4, (c["Cout"],))
+    F = torch.nn.functional
+    tp = {k: torch.tensor(v.copy(), dtype=torch.float64, requires_grad=True) for k, v in L.p.items()}
+    tq = {k: torch.tensor(v.copy(), dtype=torch.float64, requires_grad=True) for k, v in Pj.p.items()}
+    names = list(tp) + ["p" + k for k in tq]
+    opt = torch.optim.SGD(list(tp.values()) + list(tq.values()), lr=0.05, momentum=0.9)
+    rm, rv = torch.zeros(c["Cout"], dtype=torch.float64), torch.ones(c["Cout"], dtype=torch.float64)
+    rms, rvs = torch.zeros(c["Cout"], dtype=torch.float64), torch.ones(c["Cout"], dtype=torch.float64)
+    xt, xbt, yt = torch.tensor(x), torch.tensor(xb, requires_grad=True), torch.tensor(y.astype(np.int64))
+    for step in range(2):
+        opt.zero_grad()
+        s_t = F.batch_norm(F.conv2d(xbt, tq["W"][:, :, None, None], None, stride=2), rms, rvs, tq["gamma"], tq["beta"], training=True,
+                           momentum=0.1, eps=1e-5)
+        a = F.relu(F.batch_norm(F.conv2d(xt, tp["W"], None, padding=1), rm, rv, tp["gamma"], tp["beta"], training=True, momentum=0.1,
+                                eps=1e-5) + s_t)
+        h = F.relu(F.conv2d(a.detach() * 0 + a, tp["Wa"], tp["ba"], padding=1))
+        loss_t = F.cross_entropy(F.linear(F.adaptive_avg_pool2d(h, 2).flatten(1), tp["Wf"], tp["bf"]), yt)
+        loss_t.backward()
+        grads = {k: v.grad.numpy().copy() for k, v in tp.items()}
+        pgrads = {k: v.grad.numpy().copy() for k, v in tq.items()}
+        s = Pj.forward(xb)
+        np.testing.assert_allclose(s, s_t.detach().numpy(), atol=1e-12)
+        loss, act, tr = L.step(x, y, 0.05, update=True, trace=True, skip=s)
+        pg = Pj.backward(tr["dz"], 0.05)
+        assert abs(loss - float(loss_t.detach())) <= 1e-12
+        np.testing.assert_allclose(act, a.detach().numpy(), atol=1e-12)
+        for k, g in [("W", "gW"), ("gamma", "ggamma"), ("beta", "gbeta"), ("Wa", "gWa"), ("ba", "gba"), ("Wf", "gWf"), ("bf", "gbf")]:
+            np.testing.assert_allclose(tr[g], grads[k], atol=1e-11 * max(1.0, np.abs(grads[k]).max()), err_msg=k)
+        np.testing.assert_allclose(pg["gW"], pgrads["W"], atol=1e-11 * max(1.0, np.abs(pgrads["W"]).max()))
+        np.testing.assert_allclose(pg["ggamma"], pgrads["gamma"], atol=1e-11)
+        np.testing.assert_allclose(pg["gbeta"], pgrads["beta"], atol=1e-11)
+        assert np.abs(pgrads["W"]).max() > 1e-4                      # the shortcut really is trained by this loss
+        opt.step()
+        for k in tp:
+            np.testing.assert_allclose(L.p[k], tp[k].detach().numpy(), atol=1e-12, err_msg=k)
+        for k in tq:
+            np.testing.assert_allclose(Pj.p[k], tq[k].detach().numpy(), atol=1e-12, err_msg="p" + k)
+        np.testing.assert_allclose(Pj.rmean, rms.numpy(), atol=1e-12)
+        np.testing.assert_allclose(Pj.rvar, rvs.numpy(), atol=1e-12)
+    with torch.no_grad():
+        se = F.batch_norm(F.conv2d(torch.tensor(xb), tq["W"][:, :, None, None], None, stride=2), rms, rvs, tq["gamma"], tq["beta"],
+                          training=False, eps=1e-5)
+    np.testing.assert_allclose(Pj.eval_forward(xb), se.numpy(), atol=1e-12)
+    # bf16 storage mode: s and the stored conv output are bfloat16 values, the convolution reads a bfloat16 copy of Wp
+    Pb = nfo.Projection(Cs, c["Cout"], store_bf16=True)
+    Pb.p["W"][...] = Pj.p["W"]
+    sb = Pb.forward(xb)
+    assert np.array_equal(sb, synth.round_bf16(sb).astype(np.float64)) and np.abs(sb - Pj.forward(xb)).max() > 0
