@@ -170,6 +170,37 @@ int nf_block_cache_n(nf_block* block, const void* x, void* out, int count);
  * shortcut run their BatchNorm passes on the generic kernels.  NF_EALIGN if not 16-byte aligned. */
 int nf_layer_set_skip(nf_layer* layer, const void* skip);
 
+/* A TRAINABLE shortcut.  nf_layer_set_skip_grad makes every later step on this layer also write dz, the gradient at the sum
+ * BN(theta_n x_n) + skip (after the ReLU mask and the pool routing), to dz_out: device, [N][Ho][Wo][Cout] of the layer's
+ * dtype; NULL switches it off.  That is the gradient at the shortcut, from which whatever produced the shortcut can train.
+ *
+ * nf_proj: the projection shortcut of a down-sampling residual block (the paper trains ResNet-18, Section "Experimental
+ * Setup", without saying how such a block enters a layer-local step).  Reading taken here: s = BN_p(Wp (*) x_b), a 1x1
+ * convolution with stride 2 on the block input x_b [N][H][W][Cin] followed by BatchNorm with batch statistics, joins the
+ * layer whose BatchNorm output has its shape, x_{n+1} = P(ReLU(BN(theta_n x_n) + s)); its parameters (Wp [Cout][Cin],
+ * gamma_p, beta_p) are trained by THAT layer's local loss and the block input receives no gradient, like every layer input.
+ * One local step of such a layer:
+ *   nf_proj_forward(proj, x_b, s);  nf_layer_set_skip(layer, s);  nf_layer_set_skip_grad(layer, dz);
+ *   nf_layer_step(layer, x, ...);   nf_proj_backward(proj, x_b, dz, lr);
+ * nf_proj_forward normalises with the statistics of this batch and updates the running ones; nf_proj_forward_eval uses the
+ * running statistics for `count` <= N samples (cache fill, early-exit evaluation); nf_proj_backward computes the gradients of
+ * (Wp, gamma_p, beta_p) from dz and applies the momentum update with learning rate lr.  The projection owns no device
+ * memory: like a layer it works in a caller-provided workspace (256-byte aligned).  Parameters are addressed by
+ * NF_P_W / NF_P_GAMMA / NF_P_BETA / NF_P_RMEAN / NF_P_RVAR plus an nf_param_kind.  Same conventions and error codes as the
+ * layer calls; NF_EUNSUPPORTED when Cin exceeds 1536 channels. */
+typedef struct nf_proj nf_proj;
+int nf_layer_set_skip_grad(nf_layer* layer, void* dz_out);
+nf_proj* nf_proj_create(int Cin, int Cout, int H, int W);
+void nf_proj_destroy(nf_proj* proj);
+int nf_proj_configure(nf_proj* proj, int N, int dtype, float momentum, float bn_eps, float bn_momentum);
+size_t nf_proj_workspace_bytes(const nf_proj* proj);
+int nf_proj_bind_workspace(nf_proj* proj, void* dev, size_t bytes);
+int nf_proj_set_param(nf_proj* proj, int which, const float* host, size_t n);
+int nf_proj_get_param(nf_proj* proj, int which, float* host, size_t n);
+int nf_proj_forward(nf_proj* proj, const void* xb, void* s_out);
+int nf_proj_forward_eval(nf_proj* proj, const void* xb, int count, void* s_out);
+int nf_proj_backward(nf_proj* proj, const void* xb, const void* dz, float lr);
+
 /* Data-parallel local step (the paper names distributed training as the direction beyond a single device): the batch
  * of N * world samples is sharded over `world` ranks, every rank holds N of them and a full copy of the layer, and
  * BatchNorm uses the statistics of the WHOLE batch, so the result equals nf_layer_step on the whole batch (up to

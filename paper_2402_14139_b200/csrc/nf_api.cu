@@ -449,6 +449,8 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
   } else {
     NF_TRY(nf_k_conv(dt, L->dh, N, Ha, Wa, F, Wx, (long)F * Co, 1, Co, 1, nullptr, 0, 1, Co, L->da));
   }
+  // a trainable shortcut joined at the BatchNorm output gets the gradient at that sum
+  if (L->skip_grad) NF_TRY(nf_k_write_dz(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->skip, L->skip_grad));
   trace_end();
   // back through pool / ReLU / BatchNorm
   trace_begin(5);
@@ -466,7 +468,7 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
   } else {
     NF_TRY(nf_k_bn_bwd_finalize_tot(L->dptot + 2 * Co, Co, world, L->sdz, L->sdzx, g + L->off[NF_P_GAMMA], g + L->off[NF_P_BETA]));
   }
-  if (nf_tc_dgrad_two_pass(L) && !L->skip) {  // second pass of the input gradient writes dy itself; da was never stored
+  if (nf_tc_dgrad_two_pass(L) && !L->skip && !L->skip_grad) {  // second pass of the input gradient writes dy itself; da was never stored
     NF_TRY(nf_tc_aux_dgrad_dy(L, M));
   } else {
     NF_TRY(nf_k_bn_bwd_apply(dt, L->y, L->da, N, Ho, Wo, Co, pool, L->scale, L->shift, L->mu, L->invstd, L->sdz, L->sdzx,
@@ -498,6 +500,13 @@ int nf_layer_set_skip(nf_layer* L, const void* skip) {
   if (!L) return NF_EINVAL;
   if (skip && misaligned(skip)) return NF_EALIGN;
   L->skip = skip;
+  return NF_OK;
+}
+
+int nf_layer_set_skip_grad(nf_layer* L, void* dz_out) {
+  if (!L) return NF_EINVAL;
+  if (dz_out && misaligned(dz_out)) return NF_EALIGN;
+  L->skip_grad = dz_out;
   return NF_OK;
 }
 
@@ -926,7 +935,7 @@ const char* nf_layer_kernel_family(const nf_layer* L, int op) {
   if (!L || op < 0 || op > 6) return "";
   if (op == 4) return nf_tc_bn_aux_fused(L) && !L->skip ? "fused" : "separate";
   if (op == 5) return nf_tc_bn_aux_fused(L) && !L->skip && nf_tc_aux_pool_fused(L) ? "mask" : "stored";
-  if (op == 6) return nf_tc_dgrad_two_pass(L) && !L->skip ? "two-pass" : "stored";
+  if (op == 6) return nf_tc_dgrad_two_pass(L) && !L->skip && !L->skip_grad ? "two-pass" : "stored";
   return L->fam[op] ? "tcgen05" : "cuda-core";
 }
 

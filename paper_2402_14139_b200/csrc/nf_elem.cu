@@ -567,6 +567,18 @@ __global__ void bn_bwd_apply_kernel(const T* __restrict__ y, const T* __restrict
   stf(dy, e, scale[c] * (dz - sdz[c] * invM - xh * sdzx[c] * invM));
 }
 
+// dz = da * 1[BN(y) + skip > 0], routed through the optional max-pool: the gradient at the layer's BatchNorm output, which is
+// also the gradient at a trainable shortcut added there
+template <typename T>
+__global__ void write_dz_kernel(const T* __restrict__ y, const T* __restrict__ da, int Ho, int Wo, int C, int pool,
+                                const float* __restrict__ scale, const float* __restrict__ shift, const T* __restrict__ skip,
+                                size_t total, T* __restrict__ dz) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const int c = (int)(e % C);
+  stf(dz, e, dz_at(y, da, e / C, c, C, Ho, Wo, pool, scale[c], shift[c], skip));
+}
+
 // Momentum SGD over up to kSgdMaxArenas parameter arenas in one launch (all layers of a block).  An arena is a multiple
 // of 64 floats and 256-byte aligned, so every thread owns four consecutive elements: 16-byte loads of value, momentum and
 // gradient, 16-byte stores of value and momentum, one 8-byte store of the four bf16 copies.  Blocks are dealt to arenas
@@ -1491,6 +1503,16 @@ int nf_k_bn_bwd_reduce(int dtype, const void* y, const void* da, int N, int Ho, 
            (channel_reduce_kernel<bf16, BnBwdFn><<<nb, 256, 0, g_nf_stream>>>((const bf16*)y, (const bf16*)da, P, C, fn, red)));
   NF_LAUNCHED();
   *nblocks = nb;
+  return NF_OK;
+}
+
+int nf_k_write_dz(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool, const float* scale,
+                  const float* shift, const void* skip, void* dz) {
+  const size_t total = (size_t)N * Ho * Wo * C;
+  DISPATCH(dtype,
+           (write_dz_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, (const float*)da, Ho, Wo, C, pool, scale, shift, (const float*)skip, total, (float*)dz)),
+           (write_dz_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, (const bf16*)da, Ho, Wo, C, pool, scale, shift, (const bf16*)skip, total, (bf16*)dz)));
+  NF_LAUNCHED();
   return NF_OK;
 }
 

@@ -33,6 +33,7 @@ struct nf_layer {
   float *val, *mom, *grad;             // arenas
   bf16* shadow;                        // bf16 arena
   const void* skip;                    // identity shortcut for the next calls (nf_layer_set_skip), or NULL
+  void* skip_grad;                     // where each step also writes dz, the gradient at the shortcut (nf_layer_set_skip_grad), or NULL
   bf16* wa_t;                          // [9][Cout][F] mirrored, transposed copy of Wa (only when F > 64)
   float *rmean, *rvar;                 // [Cout]
   float *scale, *shift, *mu, *invstd;  // [Cout] per-step BatchNorm coefficients
@@ -147,6 +148,8 @@ int nf_k_bn_bwd_finalize(const float* red, int nblocks, int C, float* sdz, float
 int nf_k_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool,
                         const float* scale, const float* shift, const float* mu, const float* invstd,
                         const float* sdz, const float* sdzx, double M, void* dy, const void* skip = nullptr);
+int nf_k_write_dz(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool, const float* scale,
+                  const float* shift, const void* skip, void* dz);
 int nf_k_sgd(float* val, float* mom, const float* grad, bf16* shadow, size_t n, float lr, float momentum);
 // the same update over several arenas (the layers of a block) in one launch; first_block is filled by the callee
 enum { kSgdMaxArenas = 48 };

@@ -1973,7 +1973,7 @@ bool nf_tc_dgrad_two_pass(const nf_layer* L) {
 }
 
 int nf_tc_aux_dgrad_dy(nf_layer* L, double M) {
-  if (!nf_tc_dgrad_two_pass(L) || L->skip) return NF_EUNSUPPORTED;
+  if (!nf_tc_dgrad_two_pass(L) || L->skip || L->skip_grad) return NF_EUNSUPPORTED;
   int nb = 0;
   BnBwdIn bn{L->y, L->scale, L->shift, L->mu, L->invstd};
   bn.sdz = L->sdz; bn.sdzx = L->sdzx; bn.inv_m = (float)(1.0 / M);
@@ -1984,7 +1984,7 @@ int nf_tc_aux_dgrad_dy(nf_layer* L, double M) {
 int nf_tc_aux_dgrad(nf_layer* L, int* bn_nb) {
   int nb = 0;
   *bn_nb = 0;
-  if (nf_tc_dgrad_two_pass(L) && !L->skip) {  // first pass: sums only, nothing stored
+  if (nf_tc_dgrad_two_pass(L) && !L->skip && !L->skip_grad) {  // first pass: sums only, nothing stored
     const BnBwdIn bn{L->y, L->scale, L->shift, L->mu, L->invstd};
     return run_fwd(L->o.N, L->Ha, L->Wa, L->F, L->Cout, L->dh, L->shadow + L->off[NF_P_WA], L->da, 3, L->red, L->red_floats, L->status,
                    bn_nb, 2, nullptr, 1, &bn);

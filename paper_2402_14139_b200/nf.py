@@ -27,7 +27,9 @@ PARAM_IDS = dict(W=NF_P_W, gamma=NF_P_GAMMA, beta=NF_P_BETA, Wa=NF_P_WA, ba=NF_P
 EXPORTS = ["nf_layer_create", "nf_layer_destroy", "nf_layer_configure", "nf_layer_workspace_bytes",
            "nf_layer_bind_workspace", "nf_layer_set_param", "nf_layer_get_param", "nf_layer_step",
            "nf_layer_step_host", "nf_layer_status", "nf_block_create", "nf_block_destroy", "nf_block_cache",
-           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_fit_line", "nf_max_batch", "nf_layer_step_dp", "nf_layer_dp_buffer", "nf_layer_set_skip", "nf_layer_stored_tensor", "nf_block_step", "nf_block_step_host", "nf_block_step_host_next", "nf_trace_enable", "nf_trace_read",
+           "nf_block_cache_n", "nf_layer_predict", "nf_layer_param_count", "nf_select_exit", "nf_count_equal", "nf_aan_filters", "nf_profile_layer", "nf_fit_line", "nf_max_batch", "nf_layer_step_dp", "nf_layer_dp_buffer", "nf_layer_set_skip", "nf_layer_set_skip_grad", "nf_proj_create", "nf_proj_destroy", "nf_proj_configure",
+           "nf_proj_workspace_bytes", "nf_proj_bind_workspace", "nf_proj_set_param", "nf_proj_get_param", "nf_proj_forward",
+           "nf_proj_forward_eval", "nf_proj_backward", "nf_layer_stored_tensor", "nf_block_step", "nf_block_step_host", "nf_block_step_host_next", "nf_trace_enable", "nf_trace_read",
            "nf_cache_gather", "nf_selftest_bounded_wait", "nf_conv3x3_forward", "nf_conv3x3_wgrad_scratch_bytes", "nf_conv3x3_wgrad", "nf_conv3x3_wgrad_static", "nf_op_status", "nf_partition", "nf_set_stream", "nf_launch_count",
            "nf_layer_kernel_family", "nf_strerror", "nf_last_cuda_error"]
 
@@ -77,6 +79,20 @@ def lib():
         L.nf_layer_param_count.argtypes = [vp, C.c_int]
         L.nf_count_equal.argtypes = [ip, ip, C.c_longlong, vp]
         L.nf_layer_set_skip.argtypes = [vp, vp]
+        L.nf_layer_set_skip_grad.argtypes = [vp, vp]
+        L.nf_proj_create.restype = vp
+        L.nf_proj_create.argtypes = [C.c_int] * 4
+        L.nf_proj_destroy.restype = None
+        L.nf_proj_destroy.argtypes = [vp]
+        L.nf_proj_configure.argtypes = [vp, C.c_int, C.c_int, C.c_float, C.c_float, C.c_float]
+        L.nf_proj_workspace_bytes.restype = C.c_size_t
+        L.nf_proj_workspace_bytes.argtypes = [vp]
+        L.nf_proj_bind_workspace.argtypes = [vp, vp, C.c_size_t]
+        L.nf_proj_set_param.argtypes = [vp, C.c_int, fp, C.c_size_t]
+        L.nf_proj_get_param.argtypes = [vp, C.c_int, fp, C.c_size_t]
+        L.nf_proj_forward.argtypes = [vp, vp, vp]
+        L.nf_proj_forward_eval.argtypes = [vp, vp, C.c_int, vp]
+        L.nf_proj_backward.argtypes = [vp, vp, vp, C.c_float]
         L.nf_layer_stored_tensor.argtypes = [vp, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
         L.nf_layer_step_dp.argtypes = [vp, C.c_int, vp, ip, C.c_float, fp, vp, C.c_int]
         L.nf_layer_dp_buffer.argtypes = [vp, C.c_int, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
@@ -341,6 +357,11 @@ class Layer:
                      dh=(self.N, self.Ha, self.Wa, Fp), da=(self.N, self.Ha, self.Wa, self.Cout))[name]
         return raw.view(self.tdtype).view(shape)
 
+    def set_skip_grad(self, dz_out):
+        """nf_layer_set_skip_grad: every later step also writes the gradient at the shortcut sum to dz_out [N, Ho, Wo, Cout]."""
+        self._skip_grad = dz_out
+        _check(lib().nf_layer_set_skip_grad(self.h, _ptr(dz_out)), "nf_layer_set_skip_grad")
+
     def dp_buffer(self, which):
         """The exchange buffer `which` of the data-parallel step as a tensor view of the workspace (float64 for 0 and 1, float32 for 2)."""
         ptr, nbytes = C.c_void_p(), C.c_size_t()
@@ -371,6 +392,60 @@ class Layer:
         op 6: "two-pass" when the aux input gradient runs once for the BatchNorm-backward sums and once more to write dy, so
         that da is never stored, else "stored"."""
         return lib().nf_layer_kernel_family(self.h, op).decode()
+
+
+class Projection:
+    """Projection shortcut of a down-sampling residual block (wraps nf_proj_*): s = BN(Wp (*) x_b), 1x1 convolution with
+    stride 2 on the block input x_b [N, H, W, Cin], trained by the local loss of the layer it joins."""
+
+    def __init__(self, Cin, Cout, H, W, N, dtype=NF_BF16, momentum=0.9, bn_eps=1e-5, bn_momentum=0.1, device="cuda"):
+        import torch
+        self._torch = torch
+        self.Cin, self.Cout, self.H, self.W, self.N, self.dtype = Cin, Cout, H, W, N, dtype
+        self.Ho, self.Wo = (H - 1) // 2 + 1, (W - 1) // 2 + 1
+        self.h = lib().nf_proj_create(Cin, Cout, H, W)
+        if not self.h:
+            raise NfError("nf_proj_create failed")
+        _check(lib().nf_proj_configure(self.h, N, dtype, momentum, bn_eps, bn_momentum), "nf_proj_configure")
+        nbytes = int(lib().nf_proj_workspace_bytes(self.h))
+        self.ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+        base = (self.ws.data_ptr() + 255) // 256 * 256
+        _check(lib().nf_proj_bind_workspace(self.h, C.c_void_p(base), nbytes), "nf_proj_bind_workspace")
+        self.shapes = dict(W=(Cout, Cin), gamma=(Cout,), beta=(Cout,), rmean=(Cout,), rvar=(Cout,))
+        self.tdtype = torch.float32 if dtype == NF_F32 else torch.bfloat16
+        self.device = device
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().nf_proj_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_param(self, name, array, kind=NF_K_VALUE):
+        a = np.ascontiguousarray(array, dtype=np.float32).reshape(self.shapes[name])
+        _check(lib().nf_proj_set_param(self.h, PARAM_IDS[name] | kind, a.ctypes.data_as(C.c_void_p), a.size), f"nf_proj_set_param({name})")
+
+    def get_param(self, name, kind=NF_K_VALUE):
+        a = np.empty(self.shapes[name], dtype=np.float32)
+        _check(lib().nf_proj_get_param(self.h, PARAM_IDS[name] | kind, a.ctypes.data_as(C.c_void_p), a.size), f"nf_proj_get_param({name})")
+        return a
+
+    def new_out(self):
+        return self._torch.empty((self.N, self.Ho, self.Wo, self.Cout), dtype=self.tdtype, device=self.device)
+
+    def forward(self, xb, s_out):
+        _check(lib().nf_proj_forward(self.h, _ptr(xb), _ptr(s_out)), "nf_proj_forward")
+
+    def forward_eval(self, xb, s_out, count=None):
+        _check(lib().nf_proj_forward_eval(self.h, _ptr(xb), int(self.N if count is None else count), _ptr(s_out)), "nf_proj_forward_eval")
+
+    def backward(self, xb, dz, lr):
+        _check(lib().nf_proj_backward(self.h, _ptr(xb), _ptr(dz), float(lr)), "nf_proj_backward")
 
 
 class Block:

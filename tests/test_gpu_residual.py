@@ -110,3 +110,85 @@ def test_two_layer_residual_block_through_block_step(env):
     blk.close()
     G1.close()
     G2.close()
+
+
+PROJ_CASES = [  # (dtype, layer config, channels of the block input) -- the block input has twice the layer's map size
+    (0, dict(N=4, Cin=6, Cout=10, H=6, W=6, F=3, classes=5, stride=1, pool=False), 5),
+    (1, dict(N=8, Cin=128, Cout=128, H=16, W=16, F=32, classes=100, stride=1, pool=False), 64),   # ResNet-18 stage 2, second conv
+    (1, dict(N=6, Cin=64, Cout=64, H=8, W=8, F=16, classes=10, stride=1, pool=True), 32),          # with a pool after the sum
+]
+
+
+@pytest.mark.parametrize("ci", range(len(PROJ_CASES)))
+def test_projection_shortcut_step_matches_checker(env, ci):
+    """A layer joined by a projection shortcut (1x1 convolution with stride 2 on the block input + BatchNorm), two steps:
+    the shortcut s, the layer's loss, activation and gradients, the gradient dz at the sum, the projection's own gradients,
+    updated parameters, momentum and running statistics, and the eval-mode shortcut, all against the checker."""
+    nf, torch = env
+    from oracle import nfo
+    dtype, c, Cs = PROJ_CASES[ci]
+    bf = dtype == 1
+    tol = pu.TOL[dtype]
+    rnd = synth.round_bf16 if bf else (lambda a: np.asarray(a, dtype=np.float32))
+    P, x, y = pu.seeded_case(c, 600 + ci, bf16=bf)
+    xb = rnd(np.maximum(synth.normal(600 + ci, 20, (c["N"], Cs, 2 * c["H"], 2 * c["W"])), 0.0))
+    Wp = rnd(synth.normal(600 + ci, 21, (c["Cout"], Cs), np.sqrt(2.0 / Cs)))
+    gp = (1.0 + 0.2 * synth.normal(600 + ci, 22, (c["Cout"],))).astype(np.float32)
+    bp = (0.1 * synth.normal(600 + ci, 23, (c["Cout"],))).astype(np.float32)
+    O = pu.oracle_layer(c, P, store_bf16=bf)
+    OP = nfo.Projection(Cs, c["Cout"], store_bf16=bf)
+    OP.p["W"][...], OP.p["gamma"][...], OP.p["beta"][...] = Wp, gp, bp
+    G = pu.gpu_layer(nf, c, P, dtype)
+    GP = nf.Projection(Cs, c["Cout"], 2 * c["H"], 2 * c["W"], c["N"], dtype=dtype)
+    for k, v in (("W", Wp), ("gamma", gp), ("beta", bp)):
+        GP.set_param(k, v)
+    xd, xbd = pu.to_device_nhwc(torch, x, dtype), pu.to_device_nhwc(torch, xb, dtype)
+    yd = torch.from_numpy(y).cuda()
+    s_d, dz_d, act_d = GP.new_out(), GP.new_out(), G.new_act()
+    loss_d = torch.zeros(1, device="cuda")
+    G.set_skip(s_d)
+    G.set_skip_grad(dz_d)
+    assert G.kernel_family(6) == "stored"
+    for it in range(2):
+        s_o = OP.forward(xb)
+        loss_o, act_o, tr = O.step(x, y, 0.02, update=True, trace=True, skip=s_o)
+        pg = OP.backward(tr["dz"], 0.02)
+        GP.forward(xbd, s_d)
+        G.step(xd, yd, 0.02, loss_d, act_d)
+        GP.backward(xbd, dz_d, 0.02)
+        torch.cuda.synchronize()
+        assert G.status() == 0
+        assert abs(float(loss_d.item()) - loss_o) <= tol["loss"] * abs(loss_o)
+        assert pu.max_err(pu.from_device_nhwc(s_d), s_o) <= tol["t"]
+        assert pu.max_err(pu.from_device_nhwc(act_d), act_o) <= tol["t"]
+        assert pu.max_err(pu.from_device_nhwc(dz_d), tr["dz"]) <= tol["t"]
+        for k in pu.PNAMES:
+            assert pu.max_err(G.get_param(k, nf.NF_K_GRAD), tr["g" + k]) <= tol["t"], (it, k)
+        for k, g in (("W", "gW"), ("gamma", "ggamma"), ("beta", "gbeta")):
+            assert pu.max_err(GP.get_param(k, nf.NF_K_GRAD), pg[g]) <= tol["t"], (it, "proj grad", k)
+            assert pu.max_err(GP.get_param(k), OP.p[k]) <= tol["t"], (it, "proj param", k)
+            assert pu.max_err(GP.get_param(k, nf.NF_K_MOMENTUM), OP.v[k]) <= tol["t"], (it, "proj momentum", k)
+        assert pu.max_err(GP.get_param("rmean"), OP.rmean) <= tol["t"] and pu.max_err(GP.get_param("rvar"), OP.rvar) <= tol["t"]
+        if bf:      # both sides continue from the checker's state (bf16 trajectories drift otherwise)
+            for k in pu.PNAMES:
+                v32, m32 = O.p[k].astype(np.float32), O.v[k].astype(np.float32)
+                O.set(**{k: v32, "v" + k: m32})
+                G.set_param(k, v32)
+                G.set_param(k, m32, kind=nf.NF_K_MOMENTUM)
+            for k in ("rmean", "rvar"):
+                v32 = getattr(O, k).astype(np.float32)
+                O.set(**{k: v32})
+                G.set_param(k, v32)
+            for k in ("W", "gamma", "beta"):
+                v32, m32 = OP.p[k].astype(np.float32), OP.v[k].astype(np.float32)
+                OP.p[k][...], OP.v[k][...] = v32, m32
+                GP.set_param(k, v32)
+                GP.set_param(k, m32, kind=nf.NF_K_MOMENTUM)
+            OP.rmean[...], OP.rvar[...] = OP.rmean.astype(np.float32), OP.rvar.astype(np.float32)
+            GP.set_param("rmean", OP.rmean)
+            GP.set_param("rvar", OP.rvar)
+    GP.forward_eval(xbd[:3].contiguous(), s_d, count=3)
+    torch.cuda.synchronize()
+    assert pu.max_err(pu.from_device_nhwc(s_d[:3]), OP.eval_forward(xb[:3])) <= tol["t"]
+    G.close()
+    GP.close()
