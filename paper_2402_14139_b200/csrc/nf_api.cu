@@ -89,6 +89,8 @@ size_t plan(nf_layer* L, char* base, bool assign) {
   D->grad = (float*)c.take(L->arena * 4);
   D->shadow = (bf16*)c.take(L->arena * 2);
   D->wa_t = (bf16*)c.take(F > 64 ? (size_t)9 * Co * F * 2 : 0);
+  D->wpad = (bf16*)c.take(L->cin_pad ? (size_t)9 * Co * L->cin_pad * 2 : 0);
+  D->gwpad = (float*)c.take(L->cin_pad ? (size_t)9 * Co * L->cin_pad * 4 : 0);
   D->rmean = (float*)c.take(Co * 4);
   D->rvar = (float*)c.take(Co * 4);
   D->scale = (float*)c.take(Co * 4);
@@ -104,6 +106,7 @@ size_t plan(nf_layer* L, char* base, bool assign) {
   D->dh = c.take(nh * es);
   D->da = c.take(na * es);
   D->act = c.take(na * es);
+  D->xpad = c.take(L->cin_pad ? N * L->H * L->W * L->cin_pad * es : 0);
   D->p = (float*)c.take(N * 4 * F * 4);
   D->dp = (float*)c.take(N * 4 * F * 4);
   D->parg = (int32_t*)c.take(N * 4 * F * 4);

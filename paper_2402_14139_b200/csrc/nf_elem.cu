@@ -579,6 +579,31 @@ __global__ void write_dz_kernel(const T* __restrict__ y, const T* __restrict__ d
   stf(dz, e, dz_at(y, da, e / C, c, C, Ho, Wo, pool, scale[c], shift[c], skip));
 }
 
+// xpad[p][0..Cp) = (x[p][0..C), 0, ...): one thread per 8-channel chunk (16 bytes) of the padded pixel, C <= 8
+__global__ void pad_channels_kernel(const bf16* __restrict__ x, size_t P, int C, int Cp8, uint4* __restrict__ xpad) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= P * Cp8) return;
+  const size_t p = e / Cp8;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  if (e % Cp8 == 0) {
+    unsigned short h[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int c = 0; c < C; ++c) h[c] = __bfloat16_as_ushort(x[p * C + c]);
+    v = make_uint4(h[0] | ((uint32_t)h[1] << 16), h[2] | ((uint32_t)h[3] << 16), h[4] | ((uint32_t)h[5] << 16), h[6] | ((uint32_t)h[7] << 16));
+  }
+  xpad[e] = v;
+}
+__global__ void pad_weights_kernel(const bf16* __restrict__ w, size_t rows, int C, int Cp, bf16* __restrict__ wpad) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= rows * Cp) return;
+  const int c = (int)(e % Cp);
+  wpad[e] = c < C ? w[(e / Cp) * C + c] : __float2bfloat16(0.f);
+}
+__global__ void unpad_grad_kernel(const float* __restrict__ gwpad, size_t rows, int C, int Cp, float* __restrict__ gw) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= rows * C) return;
+  gw[e] = gwpad[(e / C) * Cp + e % C];
+}
+
 // Momentum SGD over up to kSgdMaxArenas parameter arenas in one launch (all layers of a block).  An arena is a multiple
 // of 64 floats and 256-byte aligned, so every thread owns four consecutive elements: 16-byte loads of value, momentum and
 // gradient, 16-byte stores of value and momentum, one 8-byte store of the four bf16 copies.  Blocks are dealt to arenas
@@ -1556,6 +1581,23 @@ int nf_k_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, i
   DISPATCH(dtype,
            (bn_bwd_apply_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)y, (const float*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (float*)dy, nullptr)),
            (bn_bwd_apply_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)y, (const bf16*)da, Ho, Wo, C, pool, scale, shift, mu, invstd, sdz, sdzx, invM, total, (bf16*)dy, nullptr)));
+  NF_LAUNCHED();
+  return NF_OK;
+}
+
+int nf_k_pad_channels(const void* x, size_t P, int C, int Cp, void* xpad) {
+  if (C < 1 || C > 8 || Cp % 8) return NF_EUNSUPPORTED;
+  pad_channels_kernel<<<nblk(P * (Cp / 8), 256), 256, 0, g_nf_stream>>>((const bf16*)x, P, C, Cp / 8, (uint4*)xpad);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+int nf_k_pad_weights(const bf16* w, size_t rows, int C, int Cp, bf16* wpad) {
+  pad_weights_kernel<<<nblk(rows * Cp, 256), 256, 0, g_nf_stream>>>(w, rows, C, Cp, wpad);
+  NF_LAUNCHED();
+  return NF_OK;
+}
+int nf_k_unpad_grad(const float* gwpad, size_t rows, int C, int Cp, float* gw) {
+  unpad_grad_kernel<<<nblk(rows * C, 256), 256, 0, g_nf_stream>>>(gwpad, rows, C, Cp, gw);
   NF_LAUNCHED();
   return NF_OK;
 }

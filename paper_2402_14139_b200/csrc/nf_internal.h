@@ -64,6 +64,12 @@ struct nf_layer {
   float* stage_loss;
   // kernel families chosen at configure time: 0 = cuda-core, 1 = tcgen05
   int fam[4];
+  // First layers (a few input channels, e.g. RGB): cin_pad = 64 makes the main conv run on the tensor-core kernels over a
+  // copy of the input batch whose pixels are zero-padded to 64 channels; 0 = the input is used as it is.
+  int cin_pad;
+  void* xpad;                          // [N][H][W][cin_pad] (bf16)
+  bf16* wpad;                          // [9][Cout][cin_pad] operand copy of W, zero beyond Cin
+  float* gwpad;                        // [9][Cout][cin_pad] weight gradient over the padded channels
 };
 
 struct nf_block {
@@ -150,6 +156,10 @@ int nf_k_bn_bwd_apply(int dtype, const void* y, const void* da, int N, int Ho, i
                         const float* sdz, const float* sdzx, double M, void* dy, const void* skip = nullptr);
 int nf_k_write_dz(int dtype, const void* y, const void* da, int N, int Ho, int Wo, int C, int pool, const float* scale,
                   const float* shift, const void* skip, void* dz);
+// channel padding of a first layer's input and weights, and the gradient of the real channels out of the padded result
+int nf_k_pad_channels(const void* x, size_t P, int C, int Cp, void* xpad);
+int nf_k_pad_weights(const bf16* w, size_t rows, int C, int Cp, bf16* wpad);
+int nf_k_unpad_grad(const float* gwpad, size_t rows, int C, int Cp, float* gw);
 int nf_k_sgd(float* val, float* mom, const float* grad, bf16* shadow, size_t n, float lr, float momentum);
 // the same update over several arenas (the layers of a block) in one launch; first_block is filled by the callee
 enum { kSgdMaxArenas = 48 };

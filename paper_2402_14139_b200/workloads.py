@@ -95,7 +95,8 @@ def c6(block_batches=None):
     """VGG-16-shaped net on 32x32x3, 100 classes, with the auxiliary filter counts of the AAN-LL rule (32 for the two
     layers before the first down-sampling, 256 after).  The default blocks are what the Profiler calls of the library
     (nf_profile_layer at batch sizes 512..4096, nf_max_batch under a 2 GB budget) and Algorithm 1 (rho = 0.4, batch size
-    capped at the 50 000-image dataset) return: five blocks."""
+    capped at the 50 000-image dataset) return: six blocks (the RGB first layer, whose input batch is also held as a
+    64-channel padded copy, stands alone)."""
     chans = [v for v in VGG16 if v != "P"]
     lo, hi = min(chans) // 2, max(chans) // 2
     ls, S, Cin, k = [], 32, 3, 0
@@ -108,7 +109,7 @@ def c6(block_batches=None):
         if pool:
             S //= 2
     if block_batches is None:
-        block_batches = [(0, 2, 2978), (3, 5, 6366), (6, 8, 13526), (9, 9, 25672), (10, 12, 50000)]
+        block_batches = [(0, 0, 2486), (1, 2, 3452), (3, 5, 6366), (6, 8, 13526), (9, 9, 25672), (10, 12, 50000)]
     blocks = [(bs, ls[f:l + 1]) for f, l, bs in block_batches]
     return dict(name="c6", dtype="bf16", classes=100, in_shape=(3, 32, 32), blocks=blocks, layers=ls)
 

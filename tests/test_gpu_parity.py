@@ -27,7 +27,7 @@ SMALL = [
     dict(N=2, Cin=35, Cout=18, H=19, W=21, F=5, classes=11, stride=2, pool=False), # several tiles + ragged tails
     dict(N=2, Cin=1, Cout=1, H=1, W=1, F=1, classes=2, stride=1, pool=False),      # degenerate 1x1 image
     dict(N=2, Cin=4, Cout=8, H=2, W=2, F=2, classes=3, stride=1, pool=True),       # pool down to 1x1
-    dict(N=70, Cin=3, Cout=4, H=4, W=4, F=6, classes=130, stride=1, pool=False),   # class-sliced head: 3 slices, 2 sample chunks
+    dict(N=70, Cin=3, Cout=4, H=4, W=4, F=6, classes=300, stride=1, pool=False),   # class-sliced head: 43 slices, 2 sample chunks
 ]
 WIDE_HEAD = dict(N=2, Cin=2, Cout=3, H=4, W=4, F=520, classes=3, stride=1, pool=False)  # 2080 head inputs: one block per sample
 
