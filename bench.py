@@ -38,9 +38,10 @@ NCU_TRAFFIC_C4_BYTES_PER_IMAGE = dict(conv_fwd=(154.29 + 107.60) * 1e6 / 24, wgr
                                       aux_fwd=(154.22 + 111.14) * 1e6 / 24,
                                       # second pass of the aux input gradient: reads dh and y, writes dy; the finalize kernel < 1 MB
                                       bn_bwd=(192.76 + 114.73) * 1e6 / 24,
-                                      # dh from the mask + aux weight gradient + first pass of the input gradient (dh and y read,
-                                      # sums only); the two small partial-sum kernels move < 1 MB
-                                      aux_bwd=(2.44 + 0.01 + 201.49 + 5.32 + 192.76 + 3.68) * 1e6 / 24)
+                                      # dh from the mask + aux weight gradient; the two small partial-sum kernels move < 1 MB
+                                      aux_wgrad=(2.44 + 0.01 + 201.49 + 5.32) * 1e6 / 24,
+                                      # first pass of the input gradient (dh and y read, sums only)
+                                      aux_dgrad=(192.76 + 3.68) * 1e6 / 24)
 
 
 def load_peaks():
@@ -143,9 +144,10 @@ def op_model(l, N, classes, es, fam):
                 wgrad=(tc(1), fl["wgrad"], es * (nx + ny)),                # read x and dy
                 # read a, write h; fused: read y, write a and h
                 aux_fwd=(tc(2), fl["aux_fwd"], es * ((ny if fused else 0) + na + (0 if masked else nh))),
-                # h -> dh (from the sign mask: dh written only); a, dh -> gWa; dh -> da (two-pass: dh and y read, sums only)
-                aux_bwd=(tc(3), fl["aux_bwd"],
-                         es * ((3 if masked else 4) * nh + na + (ny if two_pass else na))),
+                # h -> dh (from the sign mask: dh written only); a, dh -> gWa
+                aux_wgrad=(tc(3), fl["aux_bwd"] / 2, es * ((2 if masked else 3) * nh + na)),
+                # dh -> da (two-pass: dh and y read, sums only)
+                aux_dgrad=(tc(3), fl["aux_bwd"] / 2, es * (nh + (ny if two_pass else na))),
                 # read y, write a; fused: only the statistics are finished here (partial sums in, coefficients out)
                 bn_fwd=("hbm", None, 4 * 2 * l["Cout"] * 1184 if fused else es * (ny + na)),
                 # read y and da, write dy; two-pass: the second run of the input gradient reads dh and y and writes dy

@@ -357,9 +357,10 @@ int nf_set_stream(void* cuda_stream);
  * of the layer inside the block for nf_block_step, 0 for a bare nf_layer_step), the summed
  * milliseconds and the number of timed groups.
  * Ops: 0 main conv forward (+statistics partials), 1 BatchNorm finalize+apply, 2 aux conv forward,
- * 3 pooling + linear + cross-entropy forward/backward, 4 aux conv backward (dh, weight and input
- * gradients), 5 BatchNorm backward, 6 main conv weight gradient, 7 SGD update. */
-enum { NF_TRACE_OPS = 8, NF_TRACE_SLOTS = 32 };
+ * 3 pooling + linear + cross-entropy forward/backward, 4 aux conv backward, first part (dh and the aux weight and bias
+ * gradients), 5 BatchNorm backward, 6 main conv weight gradient, 7 SGD update, 8 aux conv backward, second part (the
+ * gradient at the aux input; on two-pass shapes its first run, the second being part of op 5). */
+enum { NF_TRACE_OPS = 9, NF_TRACE_SLOTS = 32 };
 int nf_trace_enable(int on);
 int nf_trace_read(int op, int slot, double* ms_total, long long* groups);
 

@@ -445,7 +445,9 @@ static int step_phases(nf_layer* L, const void* x, const int32_t* labels, float 
     NF_TRY(nf_k_channel_sums(dt, L->dh, (size_t)N * Ha * Wa, F, L->red, L->red_floats, &nb));
     NF_TRY(nf_k_sum_partials(L->red, nb, F, 0, g + L->off[NF_P_BA]));
   }
+  trace_end();
   // gradient at the aux input
+  trace_begin(8);
   int bn_nb = 0;  // > 0: the input-gradient kernel has already left the BatchNorm-backward partial sums in L->red
   if (L->fam[3]) {
     NF_TRY(nf_tc_aux_dgrad(L, &bn_nb));

@@ -480,9 +480,16 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   constexpr uint32_t kALayout = KC == 64 ? 2 : KC == 32 ? 4 : 6;
   static_assert(!UF || (MIR && EPI == 0 && G == 64 && KC <= 32), "unfolded form: input gradient with few input channels");
   static_assert(!XF || (EPI == 1 && KC == 64 && !MIR && !UF), "fused normalisation: aux forward only");
-  constexpr int kBox = 10 * 16 * kARow;       // (8+2) rows x 16 pixels x KC channels
-  constexpr int kABytes = (UF ? 3 : 1) * kBox;  // UF: one box per column tap
-  constexpr int kTW = UF ? 16 : 14;           // output columns of a tile
+  // UF = 2: tiles of 8 columns x 16 rows fed by ONE box of 10 x 18 pixels.  An image row of the tile is then exactly one
+  // 8-row group of the operand, so the nine taps are nine start addresses (kh * 10 + kw pixels into the box) with a constant
+  // pitch of 10 pixels between groups: a third of the TMA rows of the three-box form, whose narrow 32-byte rows made the
+  // producer the slowest role of the kernel.  The shared-memory swizzle is a function of the address, so TMA and the tensor
+  // core agree wherever a tap starts.
+  constexpr int kBox = UF == 2 ? 18 * 10 * kARow : 10 * 16 * kARow;  // (8+2) rows x 16 pixels x KC channels
+  constexpr int kABytes = UF == 2 ? (kBox + 1023) / 1024 * 1024 : (UF ? 3 : 1) * kBox;  // UF 1: one box per column tap
+  constexpr int kTW = UF == 2 ? 8 : UF ? 16 : 14;  // output columns of a tile
+  constexpr int kTH = UF == 2 ? 16 : 8;            // output rows of a tile
+  constexpr int kStatIters = UF ? 8 : 7;           // 16-row slices of the staged tile (128 or 112 pixels)
   constexpr int kWTile = MIR ? 3 * KC * 128 : 3 * G * 128;  // one kernel row: [kw*G + co][64 ci], or mirrored [kw][f][64 c]
   const int w_bytes = 3 * p.kchunks * kWTile; // [chunk][kh][kw*G + co][64 ci]
   uint8_t* wres = smem + (size_t)p.stages * kABytes;
@@ -555,14 +562,16 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     bool ok = true;
     for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++tl) {
       const int m = t / p.n_tiles;
-      const int w0 = (m % p.tiles_w) * kTW, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
+      const int w0 = (m % p.tiles_w) * kTW, h0 = ((m / p.tiles_w) % p.tiles_h) * kTH, n = m / (p.tiles_w * p.tiles_h);
       for (int ck = 0; ck < p.kchunks; ++ck, ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
         if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag))) { ok = false; break; }
         if (lane == 0) {
-          ptx::mbar_expect_tx(&full[s], (uint32_t)kABytes);
-          if constexpr (UF) {
+          ptx::mbar_expect_tx(&full[s], (uint32_t)(UF == 2 ? kBox : kABytes));
+          if constexpr (UF == 2) {
+            ptx::tma_load_4d(smem + (size_t)s * kABytes, &tm_x, &full[s], ck * KC, w0 - 1, h0 - 1, n);
+          } else if constexpr (UF) {
 #pragma unroll
             for (int kw = 0; kw < 3; ++kw)
               ptx::tma_load_4d(smem + (size_t)s * kABytes + kw * kBox, &tm_x, &full[s], ck * KC, w0 - 1 + kw, h0 - 1, n);
@@ -577,7 +586,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           const uint32_t slot = tl % kYSlots;
           if (!__all_sync(0xffffffffu, ptx::mbar_wait(&yempty[slot], ((tl / kYSlots) & 1) ^ 1, abort_flag))) break;
           if (lane == 0) {
-            ptx::mbar_expect_tx(&yfull[slot], kTW * 8 * 128);
+            ptx::mbar_expect_tx(&yfull[slot], kTW * kTH * 128);
             ptx::tma_load_4d(ybuf + slot * 16384, &tm_y2, &yfull[slot], (t % p.n_tiles) * 64, w0, h0, n);
           }
           __syncwarp();
@@ -586,7 +595,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     }
   } else if (warp == 1) {
     constexpr uint32_t idesc = ptx::idesc_bf16(128, UF ? G : 3 * G, 0, MIR);
-    const uint64_t a_hi = ptx::sdesc(0, 16, 8 * kARow, kALayout);
+    const uint64_t a_hi = ptx::sdesc(0, 16, (UF == 2 ? 10 : 8) * kARow, kALayout);  // UF 2: next 8-pixel group = next box row
     const uint64_t b_hi = MIR ? ptx::sdesc(0, KC * 128, 1024, 2) : ptx::sdesc(0, 16, 1024, 2);
     const uint32_t w16 = ptx::smem_u32(wres) >> 4;
     uint32_t it = 0, tl = 0;
@@ -610,7 +619,8 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
               for (int kw = 0; kw < 3; ++kw)
 #pragma unroll
                 for (int k = 0; k < KC / 16; ++k) {
-                  const uint64_t ad = a_hi | (uint64_t)(a16 + kw * (kBox >> 4) + kh * (16 * kARow >> 4) + k * 2);
+                  const uint64_t ad = UF == 2 ? a_hi | (uint64_t)(a16 + ((kh * 10 + kw) * kARow >> 4) + k * 2)
+                                              : a_hi | (uint64_t)(a16 + kw * (kBox >> 4) + kh * (16 * kARow >> 4) + k * 2);
                   const uint64_t bd = b_hi | (uint64_t)(w16 + (2 - kh) * (kWTile >> 4) + (2 - kw) * (KC * 128 >> 4) + k * 128);
                   ptx::mma_f16(d, ad, bd, idesc, (kh | kw | k) != 0);
                 }
@@ -741,7 +751,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     for (int t = blockIdx.x + grp * gridDim.x; t < p.total_tiles; t += 2 * gridDim.x, tl += 2) {
       const int nt = t % p.n_tiles;
       const int m = t / p.n_tiles;
-      const int w0 = (m % p.tiles_w) * kTW, h0 = ((m / p.tiles_w) % p.tiles_h) * 8, n = m / (p.tiles_w * p.tiles_h);
+      const int w0 = (m % p.tiles_w) * kTW, h0 = ((m / p.tiles_w) % p.tiles_h) * kTH, n = m / (p.tiles_w * p.tiles_h);
       const uint32_t acc = tl % kAccs, aph = (tl / kAccs) & 1;
       ptx::mbar_wait(&tfull[acc], aph, abort_flag);
       ptx::tc_fence_after();
@@ -857,7 +867,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           ptx::mbar_wait(&yfull[slot], (tl / kYSlots) & 1, abort_flag);
           const uint8_t* yb = ybuf + slot * 16384;
 #pragma unroll
-          for (int rr = 0; rr < kTW / 2; ++rr) {
+          for (int rr = 0; rr < kStatIters; ++rr) {
             const int row = srg + 16 * rr;
             const int off = row * 128 + ((schunk ^ (row & 7)) * 16);
             const uint4 dq = *reinterpret_cast<const uint4*>(stg_g + off);
@@ -891,7 +901,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           ptx::mbar_wait(&yfull[slot], (tl / kYSlots) & 1, abort_flag);
           const uint8_t* yb = ybuf + slot * 16384;
 #pragma unroll
-          for (int rr = 0; rr < kTW / 2; ++rr) {
+          for (int rr = 0; rr < kStatIters; ++rr) {
             const int row = srg + 16 * rr;
             const int off = row * 128 + ((schunk ^ (row & 7)) * 16);
             const uint4 dq = *reinterpret_cast<const uint4*>(stg_g + off);
@@ -912,7 +922,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           ptx::mbar_arrive(&yempty[slot]);
         } else if (p.stats == 1) {
 #pragma unroll
-          for (int rr = 0; rr < kTW / 2; ++rr) {
+          for (int rr = 0; rr < kStatIters; ++rr) {
             const int row = srg + 16 * rr;
             const uint4 vq = *reinterpret_cast<const uint4*>(stg_g + row * 128 + ((schunk ^ (row & 7)) * 16));
             const uint32_t vw[4] = {vq.x, vq.y, vq.z, vq.w};
@@ -1603,18 +1613,20 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
              const XfIn* xf = nullptr) {
   const int G = fold_group(Cout, epi);
   const int KC = epi == 2 ? (Cin <= 16 ? 16 : 32) : 64;
-  // input gradient on widths that also tile by 16: the unfolded form (three shifted boxes, no shift-add in the epilogue)
+  // input gradient on widths that also tile by 16: the unfolded form (three shifted boxes, no shift-add in the epilogue);
+  // where the map tiles by 8 x 16 as well: its single-box form
   const bool uf = epi == 2 && W % 16 == 0;
-  const int TW = uf ? 16 : 14;
+  const bool uf2 = uf && H % 16 == 0;
+  const int TW = uf2 ? 8 : uf ? 16 : 14, TH = uf2 ? 16 : 8;
   CUtensorMap mx, mw, my, my2;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t bx[4] = {(uint32_t)KC, 16, 10, 1};
+  const uint32_t bx[4] = {(uint32_t)KC, (uint32_t)(uf2 ? 10 : 16), (uint32_t)(uf2 ? 18 : 10), 1};
   // forward: weights [kh][kw][Cout][Cin], box = G rows of co x 64 ci for the three kw of one kh;
   // input gradient: weights [kh][kw][F][Cout], box = KC rows of f x 64 c for the three kw of one kh
   const uint64_t dw[4] = {(uint64_t)(epi == 2 ? Cout : Cin), (uint64_t)(epi == 2 ? Cin : Cout), 3, 3};
   const uint32_t bw[4] = {64, (uint32_t)(epi == 2 ? KC : G), 3, 1};
   const uint64_t dy[4] = {(uint64_t)Cout, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t by[4] = {64, (uint32_t)TW, 8, 1};
+  const uint32_t by[4] = {64, (uint32_t)TW, (uint32_t)TH, 1};
   int rc;
   if ((rc = make_map4(&mx, x, dx, bx)) != NF_OK) return rc;
   if ((rc = make_map4(&mw, w, dw, bw)) != NF_OK) return rc;
@@ -1638,10 +1650,10 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
     p.bn_sdz = bn->sdz; p.bn_sdzx = bn->sdzx; p.inv_m = bn->inv_m;
   }
   p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = epi == 2 ? 1 : Cin / 64; p.n_tiles = epi == 2 ? Cout / 64 : 1;
-  p.tiles_w = W / TW; p.tiles_h = H / 8; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
+  p.tiles_w = W / TW; p.tiles_h = H / TH; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
   if ((long long)N * p.tiles_w * p.tiles_h * p.n_tiles > (1ll << 30)) return NF_EUNSUPPORTED;
   p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
-  const size_t a_bytes = (size_t)(uf ? 3 : 1) * 10 * 16 * KC * 2;
+  const size_t a_bytes = uf2 ? ((size_t)18 * 10 * KC * 2 + 1023) / 1024 * 1024 : (size_t)(uf ? 3 : 1) * 10 * 16 * KC * 2;
   const size_t wbytes = epi == 2 ? (size_t)9 * KC * 128 : (size_t)9 * p.kchunks * G * 128;
   const size_t fixed = wbytes + (epi != 1 ? (stats >= 2 ? 2 + kYSlots : 2) * 16384 : xf ? 3 * 112 * 128 : 0) + 1024 + 1024;
   int st = (int)((232448 - fixed) / a_bytes);
@@ -1666,6 +1678,8 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
                              : launch_fold<64, 1, 64, 0, 0, 1>(grid, smem, mx, mw, my, my2, p);
   }
   if (epi == 0) return launch_fold<64, 0>(grid, smem, mx, mw, my, my2, p);
+  if (epi == 2 && uf2)
+    return KC == 16 ? launch_fold<64, 0, 16, 1, 2>(grid, smem, mx, mw, my, my2, p) : launch_fold<64, 0, 32, 1, 2>(grid, smem, mx, mw, my, my2, p);
   if (epi == 2 && uf)
     return KC == 16 ? launch_fold<64, 0, 16, 1, 1>(grid, smem, mx, mw, my, my2, p) : launch_fold<64, 0, 32, 1, 1>(grid, smem, mx, mw, my, my2, p);
   if (epi == 2)

@@ -165,7 +165,7 @@ def nf_partition(max_batch, B: int, rho: float):
     return out
 
 
-TRACE_OPS = ("conv_fwd", "bn_fwd", "aux_fwd", "head", "aux_bwd", "bn_bwd", "wgrad", "sgd")
+TRACE_OPS = ("conv_fwd", "bn_fwd", "aux_fwd", "head", "aux_wgrad", "bn_bwd", "wgrad", "sgd", "aux_dgrad")
 
 
 def nf_trace_enable(on: bool):
