@@ -19,10 +19,12 @@ namespace {
 
 constexpr int kThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
 constexpr int kMaxStages = 8;
-// normalisation threads of the fused BatchNorm + aux forward: groups of 128 that share the ten rows of a box.  One group:
-// with two (five rows each) the kernel measured slower, 0.25 -> 0.27 ms, as every added warp that reads shared memory
-// stretches the tensor-core instructions.
-constexpr int kXfThreads = 128;
+// normalisation threads of the fused BatchNorm + aux forward: two groups of 128 that take the stages in turn.  A single group
+// was the slowest role of the kernel (busy 2350 of every 2450 cycles per tile while the issuer waited 520 on it: one warp per
+// scheduler cannot hide the latency of its load - arithmetic - store - fence chain).  Splitting the ten rows of ONE box over
+// two groups had measured slower (0.25 -> 0.27 ms); alternating whole stages gives each group twice the time per box.
+constexpr int kXfGroups = 2;
+constexpr int kXfThreads = 128 * kXfGroups;
 constexpr int kFoldThreads = 320;  // folded-tap forward: producer, MMA issuer and two epilogue groups of four warps
 // Tiles of y2 (the conv output read beside the input gradient, stats >= 2) in flight per CTA.  A slot turns over once per
 // load latency plus epilogue time, so with the earlier two slots per epilogue group the kernel ran at the pace of these loads
@@ -495,9 +497,9 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   uint8_t* wres = smem + (size_t)p.stages * kABytes;
   uint8_t* stg = wres + w_bytes;              // EPI 0: 112 (UF: 128) output pixels x 128 bytes
   uint8_t* ybuf = stg + 2 * 16384;            // EPI 0, stats >= 2: kYSlots tiles of y2, taken in turn by the CTA's tiles
-  constexpr int kAStg = 112 * 128;            // XF: one 14 x 8-pixel tile of a on its way to global memory (three in rotation)
+  constexpr int kAStg = 112 * 128;            // XF: one 14 x 8-pixel tile of a on its way to global memory (three in rotation per group)
   // one staging tile per epilogue group (EPI 0), or the three tiles of a (XF)
-  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (EPI == 0 ? (p.stats >= 2 ? 2 + kYSlots : 2) * 16384 : XF ? 3 * kAStg : 0));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + (EPI == 0 ? (p.stats >= 2 ? 2 + kYSlots : 2) * 16384 : XF ? 3 * kXfGroups * kAStg : 0));
   uint64_t* full = bars;
   uint64_t* empty = bars + kMaxStages;
   uint64_t* tfull = bars + 2 * kMaxStages;
@@ -509,7 +511,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(xfull + kMaxStages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);  // [2], one per epilogue group
-  volatile int* xf_go = reinterpret_cast<volatile int*>(tmem_slot + 4);   // [2], alternating between the iterations of the XF warps
+  volatile int* xf_go = reinterpret_cast<volatile int*>(tmem_slot + 4);   // [2 per group], alternating between a group's iterations
   // Accumulators in tensor memory.  The unfolded form needs 64 columns each and keeps four, so that the issuer can run two
   // tiles ahead of each epilogue group (group g takes the tiles tl = g, g + 2, ... and so alternates between two of them);
   // the folded forms need up to 192 columns each and keep two, one per group.
@@ -522,7 +524,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     for (int s = 0; s < p.stages; ++s) {
       ptx::mbar_init(&full[s], 1);
       ptx::mbar_init(&empty[s], 1);
-      ptx::mbar_init(&xfull[s], kXfThreads);
+      ptx::mbar_init(&xfull[s], 128);
     }
     for (int a = 0; a < (int)kAccs; ++a) {
       ptx::mbar_init(&tfull[a], 1);
@@ -645,9 +647,9 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     // normalisation warps: a thread owns one 16-byte channel chunk (8 channels) of one box column and walks the 10 rows.
     // The tile's own 14 x 8 pixels of a leave through a TMA store: the threads copy them from registers into a dense staging
     // tile (three in rotation) and one thread issues the store, so no global store instruction runs in these warps.
-    const int xt = (threadIdx.x - kFoldThreads) & 127, xg = (threadIdx.x - kFoldThreads) >> 7;  // group xg takes rows xg, xg+2, ...
-    constexpr int kXg = kXfThreads / 128, kRows = 10 / kXg;
-    static_assert(kXg == 1, "the staging of a assumes one normalisation group");
+    const int xt = (threadIdx.x - kFoldThreads) & 127, xgrp = (threadIdx.x - kFoldThreads) >> 7;  // group xgrp takes the stages it % kXfGroups == xgrp
+    constexpr int kXg = 1, kRows = 10, xg = 0;
+    uint8_t* const stg_x = stg + xgrp * 3 * kAStg;
     const int j = xt & 7, col = xt >> 3;                   // logical chunk, box column (0..15)
     const uint32_t off0 = (uint32_t)col * 128 + (uint32_t)((j ^ (col & 7)) * 16);  // 128-byte swizzle: the row's low bits are col's
     uint32_t it = 0;
@@ -660,6 +662,8 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       const int w = w0 - 1 + col;
       const bool w_in = w >= 0 && w < p.W, w_own = col >= 1 && col <= 14;
       for (int ck = 0; ck < p.kchunks; ++ck, ++it) {
+        if ((int)(it % kXfGroups) != xgrp) continue;
+        const uint32_t jt = it / kXfGroups;  // this group's iteration count
         const int s = it % p.stages;
         const uint32_t ph = (it / p.stages) & 1;
         if (ck != coef_ck) {
@@ -671,7 +675,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           }
         }
         const bool ok = ptx::mbar_wait(&full[s], ph, abort_flag);
-        const uint32_t astg = ptx::smem_u32(stg) + (it % 3) * kAStg;
+        const uint32_t astg = ptx::smem_u32(stg_x) + (jt % 3) * kAStg;
         if (ok) {
           const uint32_t box = ptx::smem_u32(smem + (size_t)s * kABytes) + off0 + xg * 2048;
           // all rows are loaded first, then normalised, then stored: the loads overlap instead of queueing behind stores
@@ -705,11 +709,11 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           ptx::mbar_arrive(&xfull[s]);
         }
         // one thread decides for all 128 whether to go on, so nobody is left alone at the barrier
-        if (xt == 0) xf_go[it & 1] = ok && !*abort_flag ? 1 : 0;
-        ptx::named_barrier(3, kXfThreads);
-        if (!xf_go[it & 1]) { go = false; break; }
+        if (xt == 0) xf_go[xgrp * 2 + (jt & 1)] = ok && !*abort_flag ? 1 : 0;
+        ptx::named_barrier(3 + xgrp, 128);
+        if (!xf_go[xgrp * 2 + (jt & 1)]) { go = false; break; }
         if (xt == 0) {
-          ptx::tma_store_4d(&tm_y, reinterpret_cast<const void*>(stg + (it % 3) * kAStg), ck * 64, w0, h0, n);
+          ptx::tma_store_4d(&tm_y, reinterpret_cast<const void*>(stg_x + (jt % 3) * kAStg), ck * 64, w0, h0, n);
           ptx::tma_store_commit();
           ptx::tma_store_wait_read_but_one();  // the store before this one has read its tile: the tile after next may be written
         }
@@ -1655,7 +1659,7 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
   const size_t a_bytes = uf2 ? ((size_t)18 * 10 * KC * 2 + 1023) / 1024 * 1024 : (size_t)(uf ? 3 : 1) * 10 * 16 * KC * 2;
   const size_t wbytes = epi == 2 ? (size_t)9 * KC * 128 : (size_t)9 * p.kchunks * G * 128;
-  const size_t fixed = wbytes + (epi != 1 ? (stats >= 2 ? 2 + kYSlots : 2) * 16384 : xf ? 3 * 112 * 128 : 0) + 1024 + 1024;
+  const size_t fixed = wbytes + (epi != 1 ? (stats >= 2 ? 2 + kYSlots : 2) * 16384 : xf ? 3 * kXfGroups * 112 * 128 : 0) + 1024 + 1024;
   int st = (int)((232448 - fixed) / a_bytes);
   if (st > kMaxStages) st = kMaxStages;
   p.stages = st;
@@ -1987,7 +1991,7 @@ int nf_tc_aux_fwd(nf_layer* L, const void* a, int count) {
 
 bool nf_tc_bn_aux_fused(const nf_layer* L) {
   // beside the weights and three activation stages the kernel then also holds three staging tiles of a
-  return L->fam[2] && !wide_aux(L) && !L->o.maxpool && fold_ok(L->Ha, L->Wa, L->Cout, L->F, 1, 1, 0, 3 * 112 * 128);
+  return L->fam[2] && !wide_aux(L) && !L->o.maxpool && fold_ok(L->Ha, L->Wa, L->Cout, L->F, 1, 1, 0, 3 * kXfGroups * 112 * 128);
 }
 
 // The fused aux forward can also keep h out of memory when the head pools by averaging and no tile straddles a pooling
