@@ -121,6 +121,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
       : "r"(taddr)
       : "memory");
 }
+// 16 lanes x 16 consecutive columns in the layout of a matrix-multiply accumulator fragment: with i the thread's index in the
+// warp, v[4k + 0..1] = lane (base + i / 4), columns 8k + 2 (i % 4) + {0, 1}; v[4k + 2..3] = the same columns of lane (base + i / 4 + 8)
+__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t (&v)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr)
+               : "memory");
+}
+// Four 8 x 8 matrices of 16-bit elements, each stored TRANSPOSED: thread i holds, of matrix j, the two elements (column i / 4,
+// rows 2 (i % 4) + {0, 1}) in the halves of r[j]; row q of matrix j is written as 16 contiguous bytes at the shared address
+// that thread 8j + q passes.
+__device__ __forceinline__ void stmatrix_x4_trans(uint32_t saddr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+               : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // 16-byte shared-memory accesses by 32-bit shared address

@@ -981,6 +981,300 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   }
 }
 
+// ---------------------------------------------------------------- aux input gradient, 256 pixels per instruction
+// The narrow input gradient da = dh (*) Wa^T (K = F <= 32 per tap) is bound by the NUMBER of its K = 16 instructions, each of
+// which holds the tensor pipe for about the same time whatever its shape.  With the pixels on the M side an instruction covers
+// 128 of them; here the operands are swapped: A = the mirrored weight tile of a tap, [64 output channels] x [16 f] (M = 64,
+// MN-major as stored), B = 256 pixels x [16 f] of the dh box (N = 256, K-major), so the nine taps of a 256-pixel tile are nine
+// instructions instead of eighteen.  A tile is 8 columns x 32 rows; ONE 10 x 34-pixel box feeds all taps (a tap is a start
+// address kh * 10 + kw pixels into the box, an image row of the tile is one 8-row group, pitch 10 pixels: the swizzle is a
+// function of the address).  The accumulator holds D[channel][pixel]: with M = 64, channel c sits in lane 32 * (c / 16) + c % 16,
+// so warp q of an epilogue group reads channels 16q .. 16q+15 in lanes 0..15 of its quadrant as accumulator fragments and
+// transposes them into the pixel-major staging tile with transposing matrix stores (16 bytes = 8 channels per pixel and store row).
+// From there on everything is as in the folded kernel: BatchNorm-backward sums (stats 2, 3), the second pass that turns the
+// tile into dy (stats 4), TMA store (not for stats 3).  Needs W % 8 == 0 and H % 16 == 0 (a last tile row of 16 image rows: the
+// box rows below the image load as zeros, the store is clipped, the sums skip them); one 64-channel output tile per CTA.
+constexpr int kWideThreads = 320;
+constexpr int kWideYSlots = 3;
+
+template <int KC>
+__global__ void __launch_bounds__(kWideThreads, 1)
+aux_dgrad_wide_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+                      const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_y2, const FoldParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr int kARow = KC * 2;                                    // bytes of one pixel of the dh box
+  constexpr uint32_t kALayout = KC == 32 ? 4 : 6;
+  constexpr int kBox = 34 * 10 * kARow;                            // (32+2) rows x (8+2) pixels
+  constexpr int kStage = (kBox + 1023) / 1024 * 1024;
+  constexpr int kWTile = 3 * KC * 128;                             // one kernel row: [kw][f][64 c]
+  constexpr int kTile = 256 * 128;                                 // 256 pixels x 64 channels bf16
+  uint8_t* wres = smem + (size_t)p.stages * kStage;
+  uint8_t* stg = wres + 3 * kWTile;                                // one staging tile per epilogue group
+  uint8_t* ybuf = stg + 2 * kTile;                                 // stats >= 2: kWideYSlots tiles of y2
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ybuf + (p.stats >= 2 ? kWideYSlots : 0) * kTile);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + kMaxStages;
+  uint64_t* tfull = bars + 2 * kMaxStages;
+  uint64_t* tempty = tfull + 2;
+  uint64_t* wfull = tempty + 2;
+  uint64_t* yfull = wfull + 1;
+  uint64_t* yempty = yfull + kWideYSlots;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(yempty + kWideYSlots);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* epi_go = reinterpret_cast<volatile int*>(tmem_slot + 2);
+  constexpr uint32_t kTmemCols = 512;                              // two accumulators of 256 columns
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(&tfull[a], 1);
+      ptx::mbar_init(&tempty[a], 128);
+    }
+    for (int a = 0; a < kWideYSlots; ++a) {
+      ptx::mbar_init(&yfull[a], 1);
+      ptx::mbar_init(&yempty[a], 128);
+    }
+    ptx::mbar_init(wfull, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tmap(&tm_x);
+    ptx::prefetch_tmap(&tm_w);
+    ptx::prefetch_tmap(&tm_y);
+    ptx::prefetch_tmap(&tm_y2);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- producer: the CTA's weights once, then per tile one dh box and (stats >= 2) the y2 tile
+    if (lane == 0 && blockIdx.x < p.total_tiles) {
+      ptx::mbar_expect_tx(wfull, (uint32_t)(3 * kWTile));
+#pragma unroll
+      for (int kh = 0; kh < 3; ++kh) ptx::tma_load_4d(wres + kh * kWTile, &tm_w, wfull, (int)(blockIdx.x % p.n_tiles) * 64, 0, 0, kh);
+    }
+    __syncwarp();
+    uint32_t tl = 0;
+    for (int t = blockIdx.x; t < p.total_tiles; t += gridDim.x, ++tl) {
+      const int m = t / p.n_tiles;
+      const int w0 = (m % p.tiles_w) * 8, h0 = ((m / p.tiles_w) % p.tiles_h) * 32, n = m / (p.tiles_w * p.tiles_h);
+      const int s = tl % p.stages;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&empty[s], ((tl / p.stages) & 1) ^ 1, abort_flag))) break;
+      if (lane == 0) {
+        ptx::mbar_expect_tx(&full[s], (uint32_t)kBox);
+        ptx::tma_load_4d(smem + (size_t)s * kStage, &tm_x, &full[s], 0, w0 - 1, h0 - 1, n);
+      }
+      __syncwarp();
+      if (p.stats >= 2) {
+        const uint32_t slot = tl % kWideYSlots;
+        if (!__all_sync(0xffffffffu, ptx::mbar_wait(&yempty[slot], ((tl / kWideYSlots) & 1) ^ 1, abort_flag))) break;
+        if (lane == 0) {
+          ptx::mbar_expect_tx(&yfull[slot], (uint32_t)kTile);
+          ptx::tma_load_4d(ybuf + slot * kTile, &tm_y2, &yfull[slot], (t % p.n_tiles) * 64, w0, h0, n);
+        }
+        __syncwarp();
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- issuer: nine instructions per tile, D[channel][pixel] += Wa_mirrored(tap)[channel][f] * dh[pixel + tap][f]
+    constexpr uint32_t idesc = ptx::idesc_bf16(64, 256, 1, 0);
+    const uint64_t a_hi = ptx::sdesc(0, KC * 128, 1024, 2);          // weight tile of a tap: [f][64 c], MN-major
+    const uint64_t b_hi = ptx::sdesc(0, 16, 10 * kARow, kALayout);   // pixels: next 8-pixel group = next box row
+    const uint32_t w16 = ptx::smem_u32(wres) >> 4;
+    uint32_t tl = 0;
+    bool ok = blockIdx.x >= p.total_tiles || __all_sync(0xffffffffu, ptx::mbar_wait(wfull, 0, abort_flag));
+    for (int t = blockIdx.x; ok && t < p.total_tiles; t += gridDim.x, ++tl) {
+      const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&tempty[acc], aph ^ 1, abort_flag))) break;
+      ptx::tc_fence_after();
+      const int s = tl % p.stages;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&full[s], (tl / p.stages) & 1, abort_flag))) break;
+      ptx::tc_fence_after();
+      if (lane == 0) {
+        const uint32_t d = tmem_base + acc * 256;
+        const uint32_t x16 = ptx::smem_u32(smem + (size_t)s * kStage) >> 4;
+#pragma unroll
+        for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+          for (int kw = 0; kw < 3; ++kw)
+#pragma unroll
+            for (int k = 0; k < KC / 16; ++k) {
+              const uint64_t ad = a_hi | (uint64_t)(w16 + (2 - kh) * (kWTile >> 4) + (2 - kw) * (KC * 128 >> 4) + k * 128);
+              const uint64_t bd = b_hi | (uint64_t)(x16 + ((kh * 10 + kw) * kARow >> 4) + k * 2);
+              ptx::mma_f16(d, ad, bd, idesc, (kh | kw | k) != 0);
+            }
+        ptx::mma_commit(&empty[s]);
+        ptx::mma_commit(&tfull[acc]);
+      }
+      __syncwarp();
+    }
+  } else {
+    // ---------------- two epilogue groups of 128 threads; group g takes the tiles tl = g, g + 2, ... (accumulator g)
+    const int grp = (threadIdx.x - 64) >> 7;
+    const int et = (threadIdx.x - 64) & 127;
+    uint8_t* const stg_g = stg + grp * kTile;
+    const int lg = warp & 3;                     // lane quadrant of tensor memory: channels 16*lg .. 16*lg + 15 in lanes 0..15
+    // sums / second pass: a thread owns 8 channels (one 16-byte chunk) and the 16 rows srg, srg + 16, ... of the 256
+    const int schunk = et & 7, srg = et >> 3;
+    float s1[8], s2[8], bsc[8], bsh[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s1[i] = s2[i] = bsc[i] = bsh[i] = 0.f;
+    if (p.stats >= 2) {
+      const int c0 = (int)(blockIdx.x % p.n_tiles) * 64 + schunk * 8;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { bsc[i] = p.bn_scale[c0 + i]; bsh[i] = p.bn_shift[c0 + i]; }
+      if (p.stats == 4) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float sc = bsc[i], m1 = p.bn_sdz[c0 + i] * p.inv_m, m2 = p.bn_sdzx[c0 + i] * p.inv_m, is = p.bn_invstd[c0 + i];
+          s1[i] = -sc * m2 * is;
+          s2[i] = sc * (m2 * is * p.bn_mu[c0 + i] - m1);
+        }
+      }
+    }
+    uint32_t tl = grp;
+    for (int t = blockIdx.x + grp * gridDim.x; t < p.total_tiles; t += 2 * gridDim.x, tl += 2) {
+      const int nt = t % p.n_tiles;
+      const int m = t / p.n_tiles;
+      const int w0 = (m % p.tiles_w) * 8, h0 = ((m / p.tiles_w) % p.tiles_h) * 32, n = m / (p.tiles_w * p.tiles_h);
+      const uint32_t acc = grp, aph = (tl >> 1) & 1;
+      ptx::mbar_wait(&tfull[acc], aph, abort_flag);
+      ptx::tc_fence_after();
+      if (et == 0) {
+        ptx::tma_store_wait_read();              // the previous store of this group has read the staging tile
+        epi_go[grp] = *abort_flag ? 0 : 1;
+      }
+      ptx::named_barrier(1 + grp, 128);
+      if (!epi_go[grp]) break;
+      const uint32_t tbase = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * 256;
+      // Transpose through the matrix-store instruction: a fragment load hands thread i channel i / 4 (and i / 4 + 8) of the
+      // warp's 16 with two neighbouring pixels; as bfloat16 pairs these are the column fragments of 8 x 8 matrices whose
+      // transposed store writes, per pixel, the 8 channels of a chunk as 16 contiguous bytes of the pixel-major tile.
+      const uint32_t sbase = ptx::smem_u32(stg_g);
+      const int mrow = lane & 7, mat = lane >> 3;                       // this thread addresses row mrow of matrix mat
+      const uint32_t mchunk = (uint32_t)(2 * lg + (mat & 1));           // matrices 0, 2: channels 16 lg + 0..7; 1, 3: + 8..15
+#pragma unroll 4
+      for (int j = 0; j < 16; ++j) {             // 16 pixels at a time
+        uint32_t v[8];
+        ptx::tmem_ld_16x256b_x2(tbase + j * 16, v);
+        ptx::tmem_ld_wait();
+        uint32_t r[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {            // r[0]: ch 0-7, px 0-7; r[1]: ch 8-15, px 0-7; r[2], r[3]: px 8-15
+          const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[2 * q]), __uint_as_float(v[2 * q + 1]));
+          r[q] = *reinterpret_cast<const uint32_t*>(&b2);
+        }
+        const uint32_t px = (uint32_t)(j * 16 + (mat >> 1) * 8 + mrow);
+        ptx::stmatrix_x4_trans(sbase + px * 128 + ((mchunk ^ (px & 7)) * 16), r[0], r[1], r[2], r[3]);
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&tempty[acc]);
+      ptx::fence_async_smem();
+      ptx::named_barrier(1 + grp, 128);
+      const uint32_t slot = tl % kWideYSlots;
+      if (p.stats == 4) {
+        ptx::mbar_wait(&yfull[slot], (tl / kWideYSlots) & 1, abort_flag);
+        const uint8_t* yb = ybuf + slot * kTile;
+#pragma unroll 4
+        for (int rr = 0; rr < 16; ++rr) {
+          const int row = srg + 16 * rr;
+          const int off = row * 128 + ((schunk ^ (row & 7)) * 16);
+          const uint4 dq = *reinterpret_cast<const uint4*>(stg_g + off);
+          const uint4 yq = *reinterpret_cast<const uint4*>(yb + off);
+          const uint32_t dw[4] = {dq.x, dq.y, dq.z, dq.w}, yw[4] = {yq.x, yq.y, yq.z, yq.w};
+          uint32_t ow[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float d0 = __uint_as_float(dw[e] << 16), d1 = __uint_as_float(dw[e] & 0xffff0000u);
+            const float y0 = __uint_as_float(yw[e] << 16), y1 = __uint_as_float(yw[e] & 0xffff0000u);
+            const float z0 = fmaf(y0, bsc[2 * e], bsh[2 * e]) > 0.f ? d0 : 0.f;
+            const float z1 = fmaf(y1, bsc[2 * e + 1], bsh[2 * e + 1]) > 0.f ? d1 : 0.f;
+            const float o0 = fmaf(bsc[2 * e], z0, fmaf(s1[2 * e], y0, s2[2 * e]));
+            const float o1 = fmaf(bsc[2 * e + 1], z1, fmaf(s1[2 * e + 1], y1, s2[2 * e + 1]));
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(o0, o1);
+            ow[e] = *reinterpret_cast<const uint32_t*>(&b2);
+          }
+          *reinterpret_cast<uint4*>(stg_g + off) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+        }
+        ptx::mbar_arrive(&yempty[slot]);
+        ptx::fence_async_smem();
+        ptx::named_barrier(1 + grp, 128);
+      }
+      if (et == 0 && p.stats != 3) {
+        ptx::tma_store_4d(&tm_y, stg_g, nt * 64, w0, h0, n);
+        ptx::tma_store_commit();
+      }
+      if (p.stats == 2 || p.stats == 3) {
+        ptx::mbar_wait(&yfull[slot], (tl / kWideYSlots) & 1, abort_flag);
+        const uint8_t* yb = ybuf + slot * kTile;
+#pragma unroll 4
+        for (int rr = 0; rr < 16; ++rr) {
+          const int row = srg + 16 * rr;
+          const bool rv = h0 + (row >> 3) < p.H;  // a last tile row may reach below the image: those pixels count for nothing
+          const int off = row * 128 + ((schunk ^ (row & 7)) * 16);
+          const uint4 dq = *reinterpret_cast<const uint4*>(stg_g + off);
+          const uint4 yq = *reinterpret_cast<const uint4*>(yb + off);
+          const uint32_t dw[4] = {dq.x, dq.y, dq.z, dq.w}, yw[4] = {yq.x, yq.y, yq.z, yq.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float d0 = __uint_as_float(dw[e] << 16), d1 = __uint_as_float(dw[e] & 0xffff0000u);
+            const float y0 = __uint_as_float(yw[e] << 16), y1 = __uint_as_float(yw[e] & 0xffff0000u);
+            const float z0 = rv && fmaf(y0, bsc[2 * e], bsh[2 * e]) > 0.f ? d0 : 0.f;
+            const float z1 = rv && fmaf(y1, bsc[2 * e + 1], bsh[2 * e + 1]) > 0.f ? d1 : 0.f;
+            s1[2 * e] += z0;
+            s1[2 * e + 1] += z1;
+            s2[2 * e] = fmaf(z0, y0, s2[2 * e]);
+            s2[2 * e + 1] = fmaf(z1, y1, s2[2 * e + 1]);
+          }
+        }
+        ptx::mbar_arrive(&yempty[slot]);
+      }
+    }
+    if (et == 0) ptx::tma_store_wait_all();
+    if (p.stats == 2 || p.stats == 3) {  // one partial per warp: lanes with the same chunk (lane & 7) are added in a fixed order
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 8);
+        s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], 8);
+        s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 16);
+        s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], 16);
+      }
+      if (lane < 8) {
+        const size_t b = (size_t)(blockIdx.x / p.n_tiles) * 8 + grp * 4 + lg;
+        const int c0 = (int)(blockIdx.x % p.n_tiles) * 64 + lane * 8;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float second = (float)((double)p.bn_invstd[c0 + i] * ((double)s2[i] - (double)p.bn_mu[c0 + i] * (double)s1[i]));
+          p.red[(b * 2 + 0) * p.Cout + c0 + i] = s1[i];
+          p.red[(b * 2 + 1) * p.Cout + c0 + i] = second;
+        }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicOr(p.status, NF_ETIMEOUT);
+    const unsigned long long t0 = ptx::globaltimer();
+    while (ptx::globaltimer() - t0 < 2000000ull) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
 // ---------------------------------------------------------------- weight gradient
 // dW[tap][co][ci] = sum over pixels of dy[pixel, co] * x[pixel shifted by tap, ci].  The K dimension of the
 // GEMM is the pixel index, so both operands are MN-major in shared memory exactly as TMA delivers the
@@ -1621,10 +1915,12 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   // where the map tiles by 8 x 16 as well: its single-box form
   const bool uf = epi == 2 && W % 16 == 0;
   const bool uf2 = uf && H % 16 == 0;
-  const int TW = uf2 ? 8 : uf ? 16 : 14, TH = uf2 ? 16 : 8;
+  // ... and by 8 x 32 with 16 channels of dh: the form with 256 pixels per instruction
+  const bool wide = uf2 && KC == 16;  // H % 16 == 0: the last tile row may be half a tile
+  const int TW = uf2 ? 8 : uf ? 16 : 14, TH = wide ? 32 : uf2 ? 16 : 8;
   CUtensorMap mx, mw, my, my2;
   const uint64_t dx[4] = {(uint64_t)Cin, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  const uint32_t bx[4] = {(uint32_t)KC, (uint32_t)(uf2 ? 10 : 16), (uint32_t)(uf2 ? 18 : 10), 1};
+  const uint32_t bx[4] = {(uint32_t)KC, (uint32_t)(uf2 ? 10 : 16), (uint32_t)(wide ? 34 : uf2 ? 18 : 10), 1};
   // forward: weights [kh][kw][Cout][Cin], box = G rows of co x 64 ci for the three kw of one kh;
   // input gradient: weights [kh][kw][F][Cout], box = KC rows of f x 64 c for the three kw of one kh
   const uint64_t dw[4] = {(uint64_t)(epi == 2 ? Cout : Cin), (uint64_t)(epi == 2 ? Cin : Cout), 3, 3};
@@ -1654,12 +1950,14 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
     p.bn_sdz = bn->sdz; p.bn_sdzx = bn->sdzx; p.inv_m = bn->inv_m;
   }
   p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = epi == 2 ? 1 : Cin / 64; p.n_tiles = epi == 2 ? Cout / 64 : 1;
-  p.tiles_w = W / TW; p.tiles_h = H / TH; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
+  p.tiles_w = W / TW; p.tiles_h = (H + TH - 1) / TH; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
   if ((long long)N * p.tiles_w * p.tiles_h * p.n_tiles > (1ll << 30)) return NF_EUNSUPPORTED;
   p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
-  const size_t a_bytes = uf2 ? ((size_t)18 * 10 * KC * 2 + 1023) / 1024 * 1024 : (size_t)(uf ? 3 : 1) * 10 * 16 * KC * 2;
+  const size_t a_bytes = wide ? ((size_t)34 * 10 * KC * 2 + 1023) / 1024 * 1024
+                         : uf2 ? ((size_t)18 * 10 * KC * 2 + 1023) / 1024 * 1024 : (size_t)(uf ? 3 : 1) * 10 * 16 * KC * 2;
   const size_t wbytes = epi == 2 ? (size_t)9 * KC * 128 : (size_t)9 * p.kchunks * G * 128;
-  const size_t fixed = wbytes + (epi != 1 ? (stats >= 2 ? 2 + kYSlots : 2) * 16384 : xf ? 3 * kXfGroups * 112 * 128 : 0) + 1024 + 1024;
+  const size_t fixed = wide ? wbytes + (size_t)(stats >= 2 ? 2 + kWideYSlots : 2) * 32768 + 1024 + 1024
+                            : wbytes + (epi != 1 ? (stats >= 2 ? 2 + kYSlots : 2) * 16384 : xf ? 3 * kXfGroups * 112 * 128 : 0) + 1024 + 1024;
   int st = (int)((232448 - fixed) / a_bytes);
   if (st > kMaxStages) st = kMaxStages;
   p.stages = st;
@@ -1682,6 +1980,17 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
                              : launch_fold<64, 1, 64, 0, 0, 1>(grid, smem, mx, mw, my, my2, p);
   }
   if (epi == 0) return launch_fold<64, 0>(grid, smem, mx, mw, my, my2, p);
+  if (wide) {
+    static bool attr_done_dev[kMaxDevices];
+    bool& attr_done = attr_done_dev[current_device()];
+    if (!attr_done) {
+      NF_CUDA(cudaFuncSetAttribute(aux_dgrad_wide_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+      attr_done = true;
+    }
+    aux_dgrad_wide_kernel<16><<<grid, kWideThreads, smem, g_nf_stream>>>(mx, mw, my, my2, p);
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   if (epi == 2 && uf2)
     return KC == 16 ? launch_fold<64, 0, 16, 1, 2>(grid, smem, mx, mw, my, my2, p) : launch_fold<64, 0, 32, 1, 2>(grid, smem, mx, mw, my, my2, p);
   if (epi == 2 && uf)
