@@ -32,16 +32,16 @@ FALLBACK_PEAKS = dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=
 # DRAM bytes per image (read + write) of the kernels behind each traced op on the c4 layers 64->64 at 224x224,
 # from one ncu capture of the batch-24 case (profiles/ncu_full_c4s_conv_bn_kernels.md); every tensor is streamed
 # once, so traffic grows in proportion to the batch.  Valid for the kernels as captured; None elsewhere.
-NCU_TRAFFIC_C4_BYTES_PER_IMAGE = dict(conv_fwd=(154.29 + 106.68) * 1e6 / 24, wgrad=(324.73 + 4.03) * 1e6 / 24,
+NCU_TRAFFIC_C4_BYTES_PER_IMAGE = dict(conv_fwd=(154.31 + 107.70) * 1e6 / 24, wgrad=(324.60 + 3.75) * 1e6 / 24,
                                       # aux forward with the fused BatchNorm + ReLU: reads y, writes a, the sign mask and the
                                       # pooling partials (h is not stored)
-                                      aux_fwd=(154.21 + 116.76) * 1e6 / 24,
+                                      aux_fwd=(154.21 + 115.70) * 1e6 / 24,
                                       # second pass of the aux input gradient: reads dh and y, writes dy; the finalize kernel < 1 MB
-                                      bn_bwd=(192.76 + 114.10) * 1e6 / 24,
+                                      bn_bwd=(192.74 + 108.21) * 1e6 / 24,
                                       # dh from the mask + aux weight gradient; the two small partial-sum kernels move < 1 MB
-                                      aux_wgrad=(2.44 + 0.01 + 201.47 + 3.79) * 1e6 / 24,
+                                      aux_wgrad=(2.45 + 0.01 + 201.43 + 3.72) * 1e6 / 24,
                                       # first pass of the input gradient (dh and y read, sums only)
-                                      aux_dgrad=(192.76 + 3.50) * 1e6 / 24)
+                                      aux_dgrad=(192.74 + 5.13) * 1e6 / 24)
 
 
 def load_peaks():

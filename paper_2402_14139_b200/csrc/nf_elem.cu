@@ -1073,10 +1073,11 @@ __global__ void __launch_bounds__(256) dh_mask_vec_kernel(const uint8_t* __restr
       tab[ni][bin][f] = dp[(n_lo + ni) * 4 * F + (size_t)f * 4 + bin] * inv_bin;
     }
   __syncthreads();
-  for (size_t p = p0 + pl; pl < planes && p < p1; p += planes) {  // threads beyond planes * F8 (F8 not a divisor of 256) idle
-    const uint32_t m = mask[p * F8 + g];
-    const int j = (int)(p % Wa), i = (int)((p / Wa) % Ha);
-    const size_t n = p / img;
+  auto one = [&](size_t p, uint32_t m) {
+    // 32-bit index arithmetic (the host keeps P below 2^31): three 64-bit divisions per pixel had made this kernel compute-bound
+    const uint32_t p32 = (uint32_t)p, row = p32 / (uint32_t)Wa;
+    const int j = (int)(p32 - row * (uint32_t)Wa), i = (int)(row % (uint32_t)Ha);
+    const size_t n = row / (uint32_t)Ha;
     const int bin = (i >= Ha / 2 ? 2 : 0) + (j >= Wa / 2 ? 1 : 0);
     float o[8];
     if (tabled) {
@@ -1096,6 +1097,17 @@ __global__ void __launch_bounds__(256) dh_mask_vec_kernel(const uint8_t* __restr
     unpack8(packed, r);  // the bias gradient sums the values as stored
 #pragma unroll
     for (int e = 0; e < 8; ++e) a[e] += r[e];
+  };
+  if (pl < planes) {  // threads beyond planes * F8 (F8 not a divisor of 256) idle
+    size_t p = p0 + pl;
+    for (; p + 3 * (size_t)planes < p1; p += 4 * (size_t)planes) {  // four mask bytes in flight, handled in index order
+      uint32_t m[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) m[u] = mask[(p + (size_t)u * planes) * F8 + g];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) one(p + (size_t)u * planes, m[u]);
+    }
+    for (; p < p1; p += planes) one(p, mask[p * F8 + g]);
   }
 #pragma unroll
   for (int e = 0; e < 8; ++e) sm[e][threadIdx.x] = a[e];
@@ -1394,6 +1406,7 @@ int nf_k_dh_mask(const uint8_t* mask, const float* dp, int N, int Ha, int Wa, in
                  int* nblocks) {
   if (F % 8 || F > 2048 || (Ha & 1) || (Wa & 1)) return NF_EUNSUPPORTED;
   const size_t P = (size_t)N * Ha * Wa;
+  if (P >= ((size_t)1 << 31)) return NF_EUNSUPPORTED;
   const int nb = nf_k_channel_blocks(P, F);
   if ((size_t)nb * 2 * F > red_floats) return NF_ENOWS;
   dh_mask_vec_kernel<<<nb, 256, 0, g_nf_stream>>>(mask, dp, Ha, Wa, F / 8, P, (uint4*)dh, red);

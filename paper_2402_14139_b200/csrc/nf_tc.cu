@@ -2307,7 +2307,7 @@ bool nf_tc_bn_aux_fused(const nf_layer* L) {
 // quadrant (14 x 8-pixel tiles: Ha/2 a multiple of 8, Wa/2 of 14): the epilogue then emits pooling partials and a sign mask.
 bool nf_tc_aux_pool_fused(const nf_layer* L) {
   return nf_tc_bn_aux_fused(L) && L->o.aux_pool == NF_POOL_AVG && (L->Ha / 2) % 8 == 0 && (L->Wa / 2) % 14 == 0 && L->Ha % 2 == 0 &&
-         L->Wa % 2 == 0;
+         L->Wa % 2 == 0 && (size_t)L->o.N * L->Ha * L->Wa < ((size_t)1 << 31);
 }
 
 size_t nf_tc_pool_part_floats(const nf_layer* L) {
