@@ -22,7 +22,9 @@ constexpr int kMaxStages = 8;
 // normalisation threads of the fused BatchNorm + aux forward: two groups of 128 that take the stages in turn.  A single group
 // was the slowest role of the kernel (busy 2350 of every 2450 cycles per tile while the issuer waited 520 on it: one warp per
 // scheduler cannot hide the latency of its load - arithmetic - store - fence chain).  Splitting the ten rows of ONE box over
-// two groups had measured slower (0.25 -> 0.27 ms); alternating whole stages gives each group twice the time per box.
+// two groups had measured slower (0.25 -> 0.27 ms); alternating whole stages gives each group twice the time per box.  Three
+// groups measured slower again (aux forward 0.637 -> 0.681 ms over the c4 block): the tensor-core instructions stretch with
+// every warp that works on shared memory.
 constexpr int kXfGroups = 2;
 constexpr int kXfThreads = 128 * kXfGroups;
 constexpr int kFoldThreads = 320;  // folded-tap forward: producer, MMA issuer and two epilogue groups of four warps
