@@ -240,3 +240,40 @@ def test_large_batch_head(env, ci, loss):
     decided = (top2[:, 1] - top2[:, 0]) > 2 * tol
     assert decided.sum() > c["N"] // 8 and np.array_equal(pred_d.cpu().numpy()[decided], pred_o[decided])
     G.close()
+
+
+@pytest.mark.parametrize("ci", [0, 8, 5])
+def test_stored_intermediates_match_checker(env, ci):
+    """The tensors a step leaves in the workspace (nf_layer_stored_tensor), element by element against the checker's trace: the
+    conv output y, the pooled aux output p, the logits, dp, dh (rebuilt from the sign mask where h is never stored) and the
+    gradient dy at the conv output; da too where the layer stores it (two-pass layers never form it in memory).  On the layers
+    that keep a sign mask instead of h the mask itself is compared bit for bit with the checker's h > 0."""
+    nf, torch = env
+    c = TC[ci]
+    P, x, y = pu.seeded_case(c, 1300 + ci, bf16=True)
+    O = pu.oracle_layer(c, P, store_bf16=True)
+    G = pu.gpu_layer(nf, c, P, nf.NF_BF16)
+    loss = torch.zeros(1, device="cuda")
+    G.step(pu.to_device_nhwc(torch, x, 1), torch.from_numpy(y).cuda(), 0.02, loss, G.new_act())
+    torch.cuda.synchronize()
+    _, _, tr = O.step(x, y, 0.02, update=False, trace=True)
+    t = pu.TOL[1]["t"]
+    F = c["F"]
+    assert pu.max_err(pu.from_device_nhwc(G.stored("y")), tr["y"]) <= t
+    pg = G.stored("p").cpu().numpy().reshape(c["N"], -1, 4)[:, :F].reshape(c["N"], -1)
+    assert pu.max_err(pg, tr["p"]) <= t
+    assert pu.max_err(G.stored("logits").cpu().numpy(), tr["logits"]) <= t
+    dpg = G.stored("dp").cpu().numpy().reshape(c["N"], -1, 4)[:, :F].reshape(c["N"], -1)
+    assert pu.max_err(dpg, tr["dp"]) <= t
+    if G.kernel_family(5) == "mask":
+        m = np.unpackbits(G.stored("hmask").cpu().numpy(), axis=3, bitorder="little")[..., :F].transpose(0, 3, 1, 2).astype(bool)
+        flips = int((m != (tr["h"] > 0)).sum())
+        assert flips <= 2, flips                      # a sign may differ where h is within rounding of zero
+    else:
+        flips = int(((pu.from_device_nhwc(G.stored("h"))[:, :F] > 0) != (tr["h"] > 0)).sum())
+    if flips == 0:      # with identical ReLU decisions the backward tensors agree element by element
+        assert pu.max_err(pu.from_device_nhwc(G.stored("dh"))[:, :F], tr["dh"]) <= t
+        if G.kernel_family(6) == "stored":
+            assert pu.max_err(pu.from_device_nhwc(G.stored("da")), tr["da"]) <= t
+        assert pu.max_err(pu.from_device_nhwc(G.stored("dy")), tr["dy"]) <= t
+    G.close()
