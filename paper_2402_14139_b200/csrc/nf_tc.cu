@@ -430,6 +430,41 @@ conv_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 // done in the epilogue with warp shuffles: a tile is 16 columns x 8 rows of pixels of which the outer
 // two columns are halo, so the left/right neighbours of every output pixel are adjacent TMEM lanes of the
 // same warp.  14 x 8 output pixels per tile; needs W % 14 == 0 and H % 8 == 0.
+// Per-channel partial sums of one epilogue group (128 threads = 4 warps; a thread holds 8 channels, lane & 7 selects which):
+// shuffles add the lanes of a warp, the warps are added through `scratch` (2 KB of shared memory the group owns) in warp order,
+// and lanes 0..7 of the group's first warp write the 64 channel totals: red[0][c0 + ..] the first sums, red[1][..] the second
+// (bn_second: turned into sum(dz * xhat) = invstd * (sum(dz * y) - mu * sum(dz)) in fp64).
+__device__ __forceinline__ void fold_group_partial(float (&s1)[8], float (&s2)[8], float* scratch, int grp, int lg, int lane,
+                                                   bool bn_second, const float* mu, const float* invstd, int c0, float* red, int C) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 8);
+    s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], 8);
+    s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 16);
+    s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], 16);
+  }
+  ptx::named_barrier(1 + grp, 128);  // the group's last TMA store has read the staging tile (its issuer waited before this)
+  if (lane < 8) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      scratch[(lg * 2 + 0) * 64 + lane * 8 + i] = s1[i];
+      scratch[(lg * 2 + 1) * 64 + lane * 8 + i] = s2[i];
+    }
+  }
+  ptx::named_barrier(1 + grp, 128);
+  if (lg == 0 && lane < 8) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int c = lane * 8 + i;
+      const float a = ((scratch[0 * 64 + c] + scratch[2 * 64 + c]) + scratch[4 * 64 + c]) + scratch[6 * 64 + c];
+      float b = ((scratch[1 * 64 + c] + scratch[3 * 64 + c]) + scratch[5 * 64 + c]) + scratch[7 * 64 + c];
+      if (bn_second) b = (float)((double)invstd[c0 + c] * ((double)b - (double)mu[c0 + c] * (double)a));
+      red[c0 + c] = a;
+      red[C + c0 + c] = b;
+    }
+  }
+}
+
 struct FoldParams {
   int N, H, W, Cout, kchunks, n_tiles, tiles_w, tiles_h, total_tiles, stages, stats;
   float* red;         // EPI 0, stats != 0: [grid / n_tiles * 8][2][Cout]
@@ -767,6 +802,9 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       }
       ptx::named_barrier(1 + grp, 128);
       if (!epi_go[grp]) break;
+      // a last tile column may reach beyond the image (widths that are not multiples of 14): those pixels are stored as
+      // zeros in the staging tile (they add nothing to the statistics; the TMA store clips them) and never written directly
+      const bool vcol = valid && (UF || w0 + we - 1 < p.W);
       const uint32_t tbase = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * kAccStride;
       bf16* gdst = EPI == 1 ? p.out + (((size_t)n * p.H + h0 + hh) * p.W + w0 + we - 1) * p.Cout : nullptr;
 #pragma unroll
@@ -809,8 +847,8 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         if constexpr (EPI == 0) {
           if (valid) {
             uint8_t* dst = stg_g + orow * 128;
-            *reinterpret_cast<uint4*>(dst + (((2 * q) ^ (orow & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
-            *reinterpret_cast<uint4*>(dst + (((2 * q + 1) ^ (orow & 7)) * 16)) = make_uint4(w[4], w[5], w[6], w[7]);
+            *reinterpret_cast<uint4*>(dst + (((2 * q) ^ (orow & 7)) * 16)) = vcol ? make_uint4(w[0], w[1], w[2], w[3]) : make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(dst + (((2 * q + 1) ^ (orow & 7)) * 16)) = vcol ? make_uint4(w[4], w[5], w[6], w[7]) : make_uint4(0u, 0u, 0u, 0u);
           }
         } else if (p.pool_part) {
           // h stays in registers: its sign bits go to the mask, its sum over the warp's 32 pixels (halo pixels count as
@@ -823,12 +861,12 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-            ov[2 * e] = valid ? lo : 0.f;
-            ov[2 * e + 1] = valid ? hi : 0.f;
+            ov[2 * e] = vcol ? lo : 0.f;
+            ov[2 * e + 1] = vcol ? hi : 0.f;
             bits |= (lo > 0.f ? 1u : 0u) << (2 * e);
             bits |= (hi > 0.f ? 1u : 0u) << (2 * e + 1);
           }
-          if (valid && c0 < p.Cout) {
+          if (vcol && c0 < p.Cout) {
             uint8_t* mdst = p.mask + ((((size_t)n * p.H + h0 + hh) * p.W + w0 + we - 1) * (size_t)(p.Cout >> 3)) + (c0 >> 3);
             mdst[0] = (uint8_t)(bits & 0xffu);
             if (c0 + 8 < p.Cout) mdst[1] = (uint8_t)(bits >> 8);
@@ -856,7 +894,7 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
           if ((lane & 1) == 0 && ch < p.Cout) p.pool_part[((size_t)t * 4 + lg) * p.Cout + ch] = r1;
         } else {
           const int c0 = q * 16;             // Cout is a multiple of 8 here
-          if (valid && c0 < p.Cout) {
+          if (vcol && c0 < p.Cout) {
             *reinterpret_cast<uint4*>(gdst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
             if (c0 + 8 < p.Cout) *reinterpret_cast<uint4*>(gdst + c0 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
           }
@@ -946,26 +984,11 @@ conv_fwd_fold_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     }
     if constexpr (EPI == 0) {
       if (et == 0) ptx::tma_store_wait_all();
-      if (p.stats && p.stats != 4) {  // one partial per warp: lanes with the same chunk (lane & 7) are added in a fixed order
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 8);
-          s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], 8);
-          s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 16);
-          s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], 16);
-        }
-        if (lane < 8) {
-          const size_t b = (size_t)(blockIdx.x / p.n_tiles) * 8 + grp * 4 + lg;
-          const int ch = (int)(blockIdx.x % p.n_tiles) * 64 + lane * 8;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            float second = s2[i];
-            if (p.stats >= 2)
-              second = (float)((double)p.bn_invstd[ch + i] * ((double)s2[i] - (double)p.bn_mu[ch + i] * (double)s1[i]));
-            p.red[(b * 2 + 0) * p.Cout + ch + i] = s1[i];
-            p.red[(b * 2 + 1) * p.Cout + ch + i] = second;
-          }
-        }
+      if (p.stats && p.stats != 4) {
+        // one partial per epilogue group: lanes with the same chunk (lane & 7) are added by shuffles, the group's four warps
+        // through the (now idle) staging tile, all in a fixed order
+        fold_group_partial(s1, s2, reinterpret_cast<float*>(stg_g), grp, lg, lane, p.stats >= 2, p.bn_mu, p.bn_invstd,
+                           (int)(blockIdx.x % p.n_tiles) * 64, p.red + ((size_t)(blockIdx.x / p.n_tiles) * 2 + grp) * 2 * p.Cout, p.Cout);
       }
     }
   }
@@ -1243,25 +1266,9 @@ aux_dgrad_wide_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
       }
     }
     if (et == 0) ptx::tma_store_wait_all();
-    if (p.stats == 2 || p.stats == 3) {  // one partial per warp: lanes with the same chunk (lane & 7) are added in a fixed order
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 8);
-        s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], 8);
-        s1[i] += __shfl_xor_sync(0xffffffffu, s1[i], 16);
-        s2[i] += __shfl_xor_sync(0xffffffffu, s2[i], 16);
-      }
-      if (lane < 8) {
-        const size_t b = (size_t)(blockIdx.x / p.n_tiles) * 8 + grp * 4 + lg;
-        const int c0 = (int)(blockIdx.x % p.n_tiles) * 64 + lane * 8;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float second = (float)((double)p.bn_invstd[c0 + i] * ((double)s2[i] - (double)p.bn_mu[c0 + i] * (double)s1[i]));
-          p.red[(b * 2 + 0) * p.Cout + c0 + i] = s1[i];
-          p.red[(b * 2 + 1) * p.Cout + c0 + i] = second;
-        }
-      }
-    }
+    if (p.stats == 2 || p.stats == 3)  // one partial per epilogue group, as in the folded kernel
+      fold_group_partial(s1, s2, reinterpret_cast<float*>(stg_g), grp, lg, lane, true, p.bn_mu, p.bn_invstd,
+                         (int)(blockIdx.x % p.n_tiles) * 64, p.red + ((size_t)(blockIdx.x / p.n_tiles) * 2 + grp) * 2 * p.Cout, p.Cout);
   }
 
   ptx::tc_fence_before();
@@ -1867,10 +1874,17 @@ int launch_fwd(const TcPlan& pl, const CUtensorMap& mx, const CUtensorMap& mw, c
 // sums (stats 2) or 64 output channels; without the sums a wider layer is faster on the generic kernel's
 // 128-channel tiles (measured).
 int fold_group(int Cout, int epi) { return epi != 1 ? 64 : (Cout <= 16 ? 16 : Cout <= 32 ? 32 : 64); }
+// widths the 14-column tiles of the folded forward cover: multiples of 14, and wider maps whose ragged last tile column wastes
+// at most a third (32, 48, 64, ...: the zero-filled loads and clipped stores of TMA make the overhang harmless)
+bool fold_width_ok(int W) { return W % 14 == 0 || (W >= 28 && ((W + 13) / 14) * 14 * 3 <= W * 4); }
+
 bool fold_ok(int H, int W, int Cin, int Cout, int epi, int stride, int stats = 0, size_t extra_smem = 0) {
   if (stride != 1 || H % 8) return false;
   if (epi == 2 && W % 14 && W % 16 == 0 && (stats >= 2 || Cout == 64)) return Cin <= 32 && Cin % 8 == 0 && Cout % 64 == 0;
-  if (W % 14) return false;
+  if (epi == 2 ? W % 14 != 0 : !fold_width_ok(W)) return false;
+  // the plain aux forward (no fused normalisation: extra_smem == 0) stays on the generic kernel for ragged widths: with 64
+  // filters at 32 columns the folded form measured slower there (0.33 vs 0.25 ms), the fused form faster everywhere
+  if (epi == 1 && W % 14 != 0 && extra_smem == 0) return false;
   if (epi == 2) return Cin <= 32 && Cin % 8 == 0 && Cout % 64 == 0;
   if (Cin % 64) return false;
   if (epi == 0 ? (Cin != 64 || Cout != 64) : (Cout > 64 || Cout % 8)) return false;
@@ -1952,7 +1966,7 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
     p.bn_sdz = bn->sdz; p.bn_sdzx = bn->sdzx; p.inv_m = bn->inv_m;
   }
   p.N = N; p.H = H; p.W = W; p.Cout = Cout; p.kchunks = epi == 2 ? 1 : Cin / 64; p.n_tiles = epi == 2 ? Cout / 64 : 1;
-  p.tiles_w = W / TW; p.tiles_h = (H + TH - 1) / TH; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
+  p.tiles_w = (W + TW - 1) / TW; p.tiles_h = (H + TH - 1) / TH; p.total_tiles = N * p.tiles_w * p.tiles_h * p.n_tiles;
   if ((long long)N * p.tiles_w * p.tiles_h * p.n_tiles > (1ll << 30)) return NF_EUNSUPPORTED;
   p.stats = stats; p.red = red; p.status = status; p.bias = bias; p.out = (bf16*)y;
   const size_t a_bytes = wide ? ((size_t)34 * 10 * KC * 2 + 1023) / 1024 * 1024
@@ -1969,9 +1983,9 @@ int run_fold(int N, int H, int W, int Cin, int Cout, const void* x, const void* 
   if (grid < p.n_tiles) grid = p.n_tiles;
   if (grid > p.total_tiles) grid = p.total_tiles;
   if (stats && stats != 4) {
-    const size_t need = (size_t)(grid / p.n_tiles) * 8 * 2 * Cout;  // every CTA writes all of its 8 partials
+    const size_t need = (size_t)(grid / p.n_tiles) * 2 * 2 * Cout;  // every CTA writes its two partials (one per epilogue group)
     if (need > red_floats) return NF_ENOWS;
-    *nb = grid / p.n_tiles * 8;
+    *nb = grid / p.n_tiles * 2;
   }
   if (xf) {
     if (epi != 1) return NF_EINVAL;
@@ -2301,7 +2315,10 @@ int nf_tc_aux_fwd(nf_layer* L, const void* a, int count) {
 }
 
 bool nf_tc_bn_aux_fused(const nf_layer* L) {
-  // beside the weights and three activation stages the kernel then also holds three staging tiles of a
+  // beside the weights and three activation stages the kernel then also holds three staging tiles of a.  On widths that are
+  // no multiple of 14 (ragged last tile column) only for up to 32 filters: with 64 the wide shift-add epilogue ate the gain
+  // (32 x 32 maps, 64 filters: aux forward + normalisation 0.174 ms separate, 0.197 ms fused).
+  if (L->Wa % 14 != 0 && L->F > 32) return false;
   return L->fam[2] && !wide_aux(L) && !L->o.maxpool && fold_ok(L->Ha, L->Wa, L->Cout, L->F, 1, 1, 0, 3 * kXfGroups * 112 * 128);
 }
 

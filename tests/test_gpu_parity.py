@@ -155,6 +155,8 @@ TC = [
     dict(N=5, Cin=64, Cout=64, H=16, W=16, F=16, classes=700, stride=1, pool=False),  # few samples, many classes: 47 class slices in the head
     dict(N=3, Cin=64, Cout=64, H=24, W=112, F=16, classes=10, stride=1, pool=False),   # fused normalisation, but a tile row straddles the pooling quadrants: h stored
     dict(N=2, Cin=64, Cout=64, H=32, W=56, F=40, classes=10, stride=1, pool=False),   # pooled epilogue with three 16-channel groups (F = 40), 2 x 2 tiles per quadrant
+    dict(N=3, Cin=64, Cout=64, H=16, W=48, F=24, classes=10, stride=1, pool=False),   # folded kernels on a width that is no multiple of 14: ragged last tile column
+    dict(N=2, Cin=128, Cout=64, H=8, W=64, F=8, classes=10, stride=1, pool=False),    # the same with two input-channel chunks in the aux forward's sibling, 64 columns
 ]
 
 
@@ -190,7 +192,7 @@ def test_fused_normalisation_is_selected(env):
     """Where the folded aux forward applies (width a multiple of 14, no pool) it also applies BatchNorm + ReLU and writes
     act_out, so the parity cases of those shapes above check the fused kernel; other shapes keep the separate pass."""
     nf, torch = env
-    for c, want in ((TC[8], "fused"), (TC[9], "fused"), (TC[0], "separate"), (TC[1], "separate")):
+    for c, want in ((TC[8], "fused"), (TC[9], "fused"), (TC[3], "separate"), (TC[1], "separate")):
         P, x, y = pu.seeded_case(c, 1, bf16=True)
         G = pu.gpu_layer(nf, c, P, nf.NF_BF16)
         assert G.kernel_family(4) == want, (c, G.kernel_family(4))
@@ -198,6 +200,10 @@ def test_fused_normalisation_is_selected(env):
         # epilogue and keeps only its sign bits
         assert G.kernel_family(5) == ("mask" if want == "fused" else "stored")
         G.close()
+    P, x, y = pu.seeded_case(TC[0], 1, bf16=True)      # 32 columns: three 14-column tiles, the last one ragged; no whole-tile quadrants
+    G = pu.gpu_layer(nf, TC[0], P, nf.NF_BF16)
+    assert G.kernel_family(4) == "fused" and G.kernel_family(5) == "stored"
+    G.close()
     c = dict(TC[8], H=24)       # 24 rows: the quadrant boundary (row 12) cuts through a tile row, h is stored
     P, x, y = pu.seeded_case(c, 1, bf16=True)
     G = pu.gpu_layer(nf, c, P, nf.NF_BF16)
