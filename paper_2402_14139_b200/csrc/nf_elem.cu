@@ -233,6 +233,22 @@ __device__ __forceinline__ void bin_range(int u, int H, int& lo, int& hi) {
 }
 
 // p[n][f*4 + u*2 + v] = mean of h over bin (u,v);  one block per (n, bin)
+// the same for bins of at most 16 pixels: one thread per output p[n][f*4 + bin] (consecutive threads = consecutive channels)
+template <typename T>
+__global__ void avgpool_small_kernel(const T* __restrict__ h, int Ha, int Wa, int F, size_t total, float* __restrict__ p) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const int f = (int)(e % F), bin = (int)((e / F) % 4);
+  const size_t n = e / ((size_t)4 * F);
+  int i0, i1, j0, j1;
+  bin_range(bin / 2, Ha, i0, i1);
+  bin_range(bin % 2, Wa, j0, j1);
+  float a = 0.f;
+  for (int i = i0; i < i1; ++i)
+    for (int j = j0; j < j1; ++j) a += ldf(h, ((n * Ha + i) * Wa + j) * F + f);
+  p[n * 4 * F + (size_t)f * 4 + bin] = a / (float)((i1 - i0) * (j1 - j0));
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) avgpool_kernel(const T* __restrict__ h, int Ha, int Wa, int F, float* __restrict__ p) {
   __shared__ float sm[256];
@@ -1385,6 +1401,7 @@ int nf_k_avgpool_slices(int N, int Ha, int Wa) {
 
 int nf_k_avgpool_fast(const void* h, int N, int Ha, int Wa, int F, float* part, size_t part_floats, float* p) {
   if (F % 8 || 256 % (F / 8) || (Ha & 1) || (Wa & 1)) return NF_EUNSUPPORTED;
+  if ((long)(Ha / 2) * (Wa / 2) <= 16) return NF_EUNSUPPORTED;  // tiny maps: the caller's generic path has a kernel for them
   const int S = nf_k_avgpool_slices(N, Ha, Wa);
   if ((size_t)N * 4 * S * F > part_floats) return NF_EUNSUPPORTED;
   avgpool_part_vec_kernel<<<N * 4 * S, 256, 0, g_nf_stream>>>((const uint4*)h, Ha, Wa, F / 8, S, part);
@@ -1428,6 +1445,13 @@ int nf_k_dh_fast(const void* h, const float* dp, int N, int Ha, int Wa, int F, v
 }
 
 int nf_k_avgpool(int dtype, const void* h, int N, int Ha, int Wa, int F, float* p) {
+  if ((long)((Ha + 1) / 2) * ((Wa + 1) / 2) <= 16) {  // tiny maps (late blocks train at thousands of samples): a thread per output
+    const size_t total = (size_t)N * 4 * F;
+    DISPATCH(dtype, (avgpool_small_kernel<float><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const float*)h, Ha, Wa, F, total, p)),
+             (avgpool_small_kernel<bf16><<<nblk(total, 256), 256, 0, g_nf_stream>>>((const bf16*)h, Ha, Wa, F, total, p)));
+    NF_LAUNCHED();
+    return NF_OK;
+  }
   DISPATCH(dtype, (avgpool_kernel<float><<<N * 4, 256, 0, g_nf_stream>>>((const float*)h, Ha, Wa, F, p)),
            (avgpool_kernel<bf16><<<N * 4, 256, 0, g_nf_stream>>>((const bf16*)h, Ha, Wa, F, p)));
   NF_LAUNCHED();

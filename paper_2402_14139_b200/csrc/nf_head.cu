@@ -112,27 +112,30 @@ __global__ void __launch_bounds__(256) head_loss_rows_kernel(const float* __rest
   for (int k = lane; k < K; k += 32) g[k] = (expf(l[k] - lse) - (k == lab ? 1.f : 0.f)) * invN;
 }
 
-// gbf[k] = sum_n dlogits[n][k] (32 columns x 8 row lanes per block, lanes added in order);
-// block 0 also reduces the per-sample losses in fp64 (256 lanes, then a fixed tree).
+// part[rb][k] = sum over the rb-th of gridDim.y row ranges of dlogits[n][k] (32 columns x 8 row lanes per block, lanes added in
+// order; the ranges are added in range order by head_finish_kernel: with tens of thousands of rows and a few hundred columns
+// a single block per 32 columns was the slowest kernel of the head).  Block (0, 0) also reduces the per-sample losses in
+// fp64 (256 lanes, then a fixed tree).
 __global__ void __launch_bounds__(256) head_colsum_loss_kernel(const float* __restrict__ dl, const float* __restrict__ lossn, int N, int K,
-                                                               float* __restrict__ gbf, float* __restrict__ loss_out, int32_t* status,
+                                                               float* __restrict__ part, float* __restrict__ loss_out, int32_t* status,
                                                                int n_scale) {
   __shared__ float sm[8][33];
   __shared__ double sd[256];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int k = blockIdx.x * 32 + tx;
+  const int n0 = (int)((long)N * blockIdx.y / gridDim.y), n1 = (int)((long)N * (blockIdx.y + 1) / gridDim.y);
   float s = 0.f;
   if (k < K)
-    for (int n = ty; n < N; n += 8) s += dl[(size_t)n * K + k];
+    for (int n = n0 + ty; n < n1; n += 8) s += dl[(size_t)n * K + k];
   sm[ty][tx] = s;
   __syncthreads();
   if (ty == 0 && k < K) {
     float tsum = 0.f;
 #pragma unroll
     for (int j = 0; j < 8; ++j) tsum += sm[j][tx];
-    gbf[k] = tsum;
+    part[(size_t)blockIdx.y * K + k] = tsum;
   }
-  if (blockIdx.x == 0) {
+  if (blockIdx.x == 0 && blockIdx.y == 0) {
     double a = 0.0;
     for (int n = threadIdx.x; n < N; n += 256) a += (double)lossn[n];
     sd[threadIdx.x] = a;
@@ -219,7 +222,12 @@ int nf_head_step(const float* p, const int32_t* labels, int N, int D, int K, con
   if ((rc = gemm(dlogits, 1, K, p, D, 1, K, D, N, Z, scratch)) != NF_OK) return rc;
   head_finish_kernel<<<(unsigned)((kd + 255) / 256), 256, 0, g_nf_stream>>>(scratch, Z, kd, D, nullptr, gWf);
   NF_LAUNCHED();
-  head_colsum_loss_kernel<<<(K + 31) / 32, 256, 0, g_nf_stream>>>(dlogits, lossn, N, K, gbf, loss_out, status, n_scale);
+  // gbf[k] = sum_n dlogits[n][k]: row ranges in parallel (the scratch is free again), then the ranges in order
+  int RB = std::max(1, std::min(64, N / 128));
+  if ((size_t)RB * K > scratch_floats) RB = 1;
+  head_colsum_loss_kernel<<<dim3((K + 31) / 32, RB), 256, 0, g_nf_stream>>>(dlogits, lossn, N, K, scratch, loss_out, status, n_scale);
+  NF_LAUNCHED();
+  head_finish_kernel<<<(unsigned)((K + 255) / 256), 256, 0, g_nf_stream>>>(scratch, RB, (size_t)K, K, nullptr, gbf);
   NF_LAUNCHED();
   return NF_OK;
 }
