@@ -948,8 +948,18 @@ __global__ void __launch_bounds__(256) dh_vec_kernel(const uint4* __restrict__ h
   for (int i = 0; i < 8; ++i) a[i] = 0.f;
   const size_t p0 = P * blockIdx.x / gridDim.x, p1 = P * (blockIdx.x + 1) / gridDim.x;
   auto one = [&](size_t p, const uint4 hq) {
-    const int j = (int)(p % Wa), i = (int)((p / Wa) % Ha);
-    const size_t n = p / ((size_t)Wa * Ha);
+    int i, j;
+    size_t n;
+    if (p <= 0xffffffffull) {  // 32-bit index arithmetic where it fits
+      const uint32_t p32 = (uint32_t)p, row = p32 / (uint32_t)Wa;
+      j = (int)(p32 - row * (uint32_t)Wa);
+      n = row / (uint32_t)Ha;
+      i = (int)(row - (uint32_t)n * (uint32_t)Ha);
+    } else {
+      j = (int)(p % Wa);
+      i = (int)((p / Wa) % Ha);
+      n = p / ((size_t)Wa * Ha);
+    }
     const int bin = (i >= Ha / 2 ? 2 : 0) + (j >= Wa / 2 ? 1 : 0);
     float hv[8], o[8];
     unpack8(hq, hv);
@@ -1149,8 +1159,16 @@ __global__ void avgpool_finish_kernel(const float* __restrict__ part, int N, int
 
 // ------------------------------------------------------------------ vectorised bf16 paths for pooled layers
 // One thread owns 8 channels of one POOLED pixel: it reads the four conv outputs of the 2x2 window.
+__device__ __forceinline__ size_t div_small(size_t e, int d) {  // e / d in 32 bits where e fits
+  return e <= 0xffffffffull ? (size_t)((uint32_t)e / (uint32_t)d) : e / (size_t)d;
+}
 __device__ __forceinline__ size_t win_base(size_t q, int Ho, int Wo, int C8) {  // q = pooled pixel index
   const int Wa = Wo / 2, Ha = Ho / 2;
+  if (q <= 0xffffffffull) {  // 32-bit index arithmetic where it fits: three 64-bit divisions per window made these kernels compute-bound
+    const uint32_t q32 = (uint32_t)q, row = q32 / (uint32_t)Wa;
+    const uint32_t ja = q32 - row * (uint32_t)Wa, n = row / (uint32_t)Ha, ia = row - n * (uint32_t)Ha;
+    return (((size_t)n * Ho + 2 * ia) * Wo + 2 * ja) * C8;
+  }
   const int ja = (int)(q % Wa), ia = (int)((q / Wa) % Ha);
   const size_t n = q / ((size_t)Wa * Ha);
   return ((n * Ho + 2 * ia) * Wo + 2 * ja) * C8;
@@ -1164,7 +1182,7 @@ __global__ void __launch_bounds__(256) bn_apply_pool_vec_kernel(const uint4* __r
 #pragma unroll
   for (int i = 0; i < 8; ++i) { A[i] = scale[c0 + i]; B[i] = shift[c0 + i]; }
   for (size_t e = (size_t)blockIdx.x * 256 + threadIdx.x; e < total8; e += (size_t)gridDim.x * 256) {
-    const size_t b = win_base(e / C8, Ho, Wo, C8) + e % C8;
+    const size_t b = win_base(div_small(e, C8), Ho, Wo, C8) + threadIdx.x % C8;  // 256 % C8 == 0: the chunk of a thread is fixed
     const uint4 v4[4] = {__ldg(y + b), __ldg(y + b + C8), __ldg(y + b + (size_t)Wo * C8), __ldg(y + b + (size_t)Wo * C8 + C8)};
     float best[8];
 #pragma unroll
@@ -1261,7 +1279,7 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_pool_vec_kernel(const uint4*
     K0[i] = s * (m2 * is * mu[c0 + i] - m1);
   }
   for (size_t e = (size_t)blockIdx.x * 256 + threadIdx.x; e < total8; e += (size_t)gridDim.x * 256) {  // e over pooled vectors
-    const size_t bb = win_base(e / C8, Ho, Wo, C8) + e % C8;
+    const size_t bb = win_base(div_small(e, C8), Ho, Wo, C8) + threadIdx.x % C8;
     const size_t off[4] = {0, (size_t)C8, (size_t)Wo * C8, (size_t)Wo * C8 + C8};
     float yv[4][8], dv[8];
 #pragma unroll
