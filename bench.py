@@ -329,7 +329,7 @@ def run_ours(args, rank, world):
         out = dict(metric=METRIC, value=round(aggregate_images_per_s(N * args.steps, world, ms), 2), unit="images/s", n_gpus=world, steps=args.steps,
                    warmup=args.warmup, ms_per_step=round(ms / args.steps, 4), higher_is_better=True, scaling="weak",
                    vs_baseline=None, dtype="bf16" if es == 2 else "f32", data="synthetic",
-                   config=dict(workload=f"{wl['name']}: " + workloads.ALL[args.workload].__doc__.split(".")[0].strip(),
+                   config=dict(workload=f"{wl['name']}: " + " ".join(workloads.ALL[args.workload].__doc__.split(".")[0].split()),
                                block=bi, batch=N, layers=len(ls), l2="inputs larger than L2" if n_pool == 1 else
                                f"{n_pool} input batches rotated (pool larger than L2)", replicas=world, cuda_graph=bool(args.graph),
                                per_op_timing="the same K steps launched one by one after the timed graph replays" if args.graph else "inside the timed region",
@@ -380,7 +380,7 @@ def run_reference(args):
     return dict(impl="reference", metric=METRIC, value=v, unit="images/s", n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=round(1e3 * total / args.steps, 2), higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                config=dict(workload=f"{wl['name']}: " + workloads.ALL[args.workload].__doc__.split(".")[0].strip(),
+                config=dict(workload=f"{wl['name']}: " + " ".join(workloads.ALL[args.workload].__doc__.split(".")[0].split()),
                             sample=sample),
                 cpu_baseline=dict(value=v, unit="images/s", cores=cores, kind="oracle", sample=sample),
                 e2e=dict(value=v, unit="images/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
