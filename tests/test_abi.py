@@ -106,6 +106,10 @@ def test_profiler_rule_line_fit_and_max_batch_on_the_host():
     sl, ic = nfo.fit_line(xs, ys)
     ref = np.polyfit(xs, ys, 1)
     assert abs(sl - ref[0]) <= 1e-9 * abs(ref[0]) and abs(ic - ref[1]) <= 1e-6 * abs(ref[1])
+    sl2, ic2 = nf.nf_fit_line(xs, ys)                 # the stand-alone fit the measured Profiler uses
+    assert abs(sl2 - sl) <= 1e-9 * abs(sl) and abs(ic2 - ic) <= 1e-6 * abs(ic)
+    with pytest.raises(nf.NfError):
+        nf.nf_fit_line([8, 8], [1.0, 2.0])            # all batch sizes equal: no line
     l = dict(Cin=64, Cout=64, H=32, W=32, F=32, stride=1, pool=True)
     batches = [16, 32, 64, 128, 256]
     by, slope, icpt = nf.nf_profile_layer(l["Cin"], l["Cout"], l["H"], l["W"], l["F"], 10, batches, maxpool=True)
