@@ -132,3 +132,25 @@ def test_planned_blocks_of_the_aan_workload_match_its_stored_default():
     assert [l["F"] for l in wl["layers"]] == nf.nf_aan_filters([l["Cout"] for l in wl["layers"]], 2)
     plan = pipeline.plan_blocks(nf, wl["layers"], wl["classes"], 2e9, 50000, 0.4)
     assert [(bs, len(ls)) for bs, ls in wl["blocks"]] == [(bs, l - f + 1) for f, l, bs in plan]
+
+
+def test_projection_description_is_host_only(nf):
+    """nf_proj_create / configure / workspace_bytes do no device work: they size the workspace a caller must provide."""
+    L = nf.lib()
+    assert not L.nf_proj_create(0, 8, 8, 8)
+    h = L.nf_proj_create(64, 128, 32, 32)
+    assert h
+    assert L.nf_proj_configure(h, 8, nf.NF_BF16, 0.9, 1e-5, 0.1) == nf.NF_OK
+    small = L.nf_proj_workspace_bytes(h)
+    assert L.nf_proj_configure(h, 64, nf.NF_BF16, 0.9, 1e-5, 0.1) == nf.NF_OK
+    big = L.nf_proj_workspace_bytes(h)
+    # two stored tensors of N x 16 x 16 x 128 bf16 (conv output and its gradient) dominate the growth
+    assert big > small > 0 and abs((big - small) - 2 * 56 * 16 * 16 * 128 * 2) <= 0.1 * (big - small)
+    for bad in (dict(N=0), dict(dtype=5), dict(momentum=1.0), dict(eps=0.0)):
+        a = dict(N=8, dtype=nf.NF_BF16, momentum=0.9, eps=1e-5)
+        a.update(bad)
+        assert L.nf_proj_configure(h, a["N"], a["dtype"], a["momentum"], a["eps"], 0.1) == nf.NF_EINVAL
+    buf = np.zeros(128, dtype=np.float32)
+    assert L.nf_proj_get_param(h, nf.NF_P_GAMMA, buf.ctypes.data_as(C.c_void_p), 128) == nf.NF_ENOWS    # no workspace bound
+    assert L.nf_proj_forward(h, None, None) == nf.NF_EINVAL
+    L.nf_proj_destroy(h)
